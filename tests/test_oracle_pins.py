@@ -1,0 +1,263 @@
+"""Pins for the fp64 oracle: every check here compares the oracle with something
+other than itself -- hand-worked exact values, closed forms, finite differences,
+invariants of softmax attention, a brute-force evaluation and torch's CPU
+autograd -- so that a dropped term, a wrong sign or index, or a transposed
+operand anywhere in it fails at least one test.  CPU only."""
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+
+
+def _val(x):
+    table = {"ln3": math.log(3), "ln4": math.log(4), "ln(4/3)": math.log(4 / 3),
+             "-0.75*ln3": -0.75 * math.log(3), "-1.5*ln3": -1.5 * math.log(3)}
+    if isinstance(x, str):
+        return table[x]
+    if isinstance(x, list):
+        return [_val(v) for v in x]
+    return float(x)
+
+
+def _rand(n, d, seed, gain=1.0):
+    rng = np.random.default_rng(seed)
+    return tuple(gain * rng.standard_normal((n, d)) for _ in range(4))
+
+
+# ---------------------------------------------------------------- P1: hand 2x2
+@pytest.mark.parametrize("causal", [False, True])
+def test_hand_2x2(causal):
+    g = json.load(open(os.path.join(HERE, "golden", "hand_2x2.json")))
+    inp = g["inputs"]
+    Q, K, V, dO = (np.array(_val(inp[k])) for k in ("Q", "K", "V", "dO"))
+    r = oracle.attn_head_full(Q, K, V, dO, causal, inp["scale"])
+    want = g["causal" if causal else "noncausal"]
+    for key in ("P", "O", "L", "D", "dS", "dQ", "dK", "dV"):
+        np.testing.assert_allclose(r[key], np.array(_val(want[key])), rtol=0, atol=1e-14, err_msg=key)
+
+
+def test_hand_2x2_scale_enters_inside_softmax():
+    g = json.load(open(os.path.join(HERE, "golden", "hand_2x2.json")))
+    inp = g["inputs"]
+    Q, K, V, dO = (np.array(_val(inp[k])) for k in ("Q", "K", "V", "dO"))
+    a = oracle.attn_head_full(Q, K, V, dO, False, 1.0)
+    b = oracle.attn_head_full(Q, 2 * K, V, dO, False, 0.5)
+    for key in ("O", "L", "dQ", "dV", "P", "dS"):
+        np.testing.assert_allclose(b[key], a[key], atol=1e-14, err_msg=key)
+    np.testing.assert_allclose(b["dK"], np.array(g["scale_pin"]["dK_noncausal"]), atol=1e-14)
+
+
+# ------------------------------------------------- P2: uniform attention (Q = 0)
+@pytest.mark.parametrize("causal", [False, True])
+def test_uniform_attention_closed_form(causal):
+    n, d, scale = 9, 5, 0.37
+    _, K, V, dO = _rand(n, d, 11)
+    Q = np.zeros((n, d))
+    r = oracle.attn_head_full(Q, K, V, dO, causal, scale)
+    for i in range(n):
+        cnt = i + 1 if causal else n
+        np.testing.assert_allclose(r["P"][i, :cnt], 1.0 / cnt, atol=1e-15)
+        assert np.all(r["P"][i, cnt:] == 0.0)
+        np.testing.assert_allclose(r["O"][i], V[:cnt].mean(0), atol=1e-14)
+        np.testing.assert_allclose(r["L"][i], math.log(cnt), atol=1e-14)
+        vbar = V[:cnt].mean(0)
+        want_dq = scale / cnt * sum((dO[i] @ (V[j] - vbar)) * K[j] for j in range(cnt))
+        np.testing.assert_allclose(r["dQ"][i], want_dq, atol=1e-13)
+    np.testing.assert_allclose(r["dK"], 0.0, atol=1e-14)  # Q = 0
+    if not causal:
+        np.testing.assert_allclose(r["dV"], np.tile(dO.sum(0) / n, (n, 1)), atol=1e-14)
+    else:
+        want = np.array([sum(dO[i] / (i + 1) for i in range(j, n)) for j in range(n)])
+        np.testing.assert_allclose(r["dV"], want, atol=1e-14)
+        np.testing.assert_allclose(r["O"][0], V[0], atol=0)
+        np.testing.assert_allclose(r["dQ"][0], 0.0, atol=1e-15)
+
+
+# ---------------------------------------------- P3: central finite differences
+@pytest.mark.parametrize("causal", [False, True])
+def test_finite_differences(causal):
+    n, d, scale, h = 6, 3, 0.61, 1e-5
+    Q, K, V, dO = _rand(n, d, 5)
+    r = oracle.attn_head_full(Q, K, V, dO, causal, scale)
+
+    def loss(q, k, v):
+        return float(np.sum(oracle.attn_head_full(q, k, v, dO, causal, scale)["O"] * dO))
+
+    for name, idx in (("dQ", 0), ("dK", 1), ("dV", 2)):
+        num = np.zeros((n, d))
+        for i in range(n):
+            for k in range(d):
+                args_p = [Q.copy(), K.copy(), V.copy()]
+                args_m = [Q.copy(), K.copy(), V.copy()]
+                args_p[idx][i, k] += h
+                args_m[idx][i, k] -= h
+                num[i, k] = (loss(*args_p) - loss(*args_m)) / (2 * h)
+        np.testing.assert_allclose(r[name], num, rtol=2e-7, atol=2e-8, err_msg=name)
+
+
+# ------------------------------------------------------------- P4: invariants
+@pytest.mark.parametrize("causal", [False, True])
+def test_invariants(causal):
+    n, d, scale = 37, 8, 0.3
+    Q, K, V, dO = _rand(n, d, 21)
+    r = oracle.attn_head_full(Q, K, V, dO, causal, scale)
+    P, dS = r["P"], r["dS"]
+    np.testing.assert_allclose(P.sum(1), 1.0, atol=1e-14)
+    np.testing.assert_allclose(dS.sum(1), 0.0, atol=1e-13)
+    np.testing.assert_allclose(r["dK"].sum(0), 0.0, atol=1e-12)
+    np.testing.assert_allclose(r["dV"].sum(0), dO.sum(0), atol=1e-12)
+    assert np.all(r["O"] <= V.max(0) + 1e-14) and np.all(r["O"] >= V.min(0) - 1e-14)
+    S = scale * Q @ K.T
+    if causal:
+        S = np.where(np.tri(n, dtype=bool), S, -np.inf)
+        assert np.all(np.triu(P, 1) == 0) and np.all(np.triu(dS, 1) == 0)
+    np.testing.assert_allclose(np.exp(S - r["L"][:, None]), P, atol=1e-14)
+    # the identity the backward's "precompute pass" rests on: D_i = dO_i . O_i
+    np.testing.assert_allclose(r["D"], np.sum(dO * r["O"], 1), atol=1e-13)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_symmetries(causal):
+    n, d, scale = 19, 4, 0.45
+    Q, K, V, dO = _rand(n, d, 31)
+    base = oracle.attn_head_full(Q, K, V, dO, causal, scale)
+    # adding one vector to every key shifts each score row by a constant
+    c = np.arange(1, d + 1) * 0.25
+    sh = oracle.attn_head_full(Q, K + c, V, dO, causal, scale)
+    for key in ("O", "P", "dS", "dQ", "dK", "dV"):
+        np.testing.assert_allclose(sh[key], base[key], atol=1e-12, err_msg=key)
+    # (Q, K) -> (aQ, K/a)
+    a = 1.7
+    sc = oracle.attn_head_full(a * Q, K / a, V, dO, causal, scale)
+    np.testing.assert_allclose(sc["O"], base["O"], atol=1e-13)
+    np.testing.assert_allclose(sc["dV"], base["dV"], atol=1e-13)
+    np.testing.assert_allclose(sc["dQ"], base["dQ"] / a, atol=1e-13)
+    np.testing.assert_allclose(sc["dK"], base["dK"] * a, atol=1e-13)
+    if not causal:
+        perm = np.random.default_rng(0).permutation(n)
+        pr = oracle.attn_head_full(Q, K[perm], V[perm], dO, causal, scale)
+        np.testing.assert_allclose(pr["O"], base["O"], atol=1e-13)
+        np.testing.assert_allclose(pr["dQ"], base["dQ"], atol=1e-13)
+        np.testing.assert_allclose(pr["dK"], base["dK"][perm], atol=1e-13)
+        np.testing.assert_allclose(pr["dV"], base["dV"][perm], atol=1e-13)
+
+
+def test_causality():
+    n, d, scale = 12, 3, 0.8
+    Q, K, V, dO = _rand(n, d, 41)
+    base = oracle.attn_head_full(Q, K, V, dO, True, scale)
+    K2, V2 = K.copy(), V.copy()
+    K2[8:] += 3.0
+    V2[8:] -= 2.0
+    pert = oracle.attn_head_full(Q, K2, V2, dO, True, scale)
+    np.testing.assert_array_equal(pert["O"][:8], base["O"][:8])
+    # the last key is seen by the last query only
+    p_last = base["P"][n - 1, n - 1]
+    np.testing.assert_allclose(base["dV"][n - 1], p_last * dO[n - 1], atol=1e-15)
+    np.testing.assert_allclose(base["dK"][n - 1], scale * base["dS"][n - 1, n - 1] * Q[n - 1], atol=1e-15)
+
+
+# ---------------------------------------------- P5: torch CPU autograd (library)
+@pytest.mark.parametrize("causal", [False, True])
+def test_against_torch_autograd(causal):
+    torch = pytest.importorskip("torch")
+    B, H, n, d, scale = 2, 3, 33, 7, 0.29
+    rng = np.random.default_rng(3)
+    Q, K, V, dO = (rng.standard_normal((B, H, n, d)) for _ in range(4))
+    r = oracle.attn_fwd_bwd(Q, K, V, dO, causal, scale)
+    q, k, v = (torch.tensor(x, dtype=torch.float64, requires_grad=True) for x in (Q, K, V))
+    o = torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=causal, scale=scale)
+    o.backward(torch.tensor(dO))
+    for key, t in (("O", o.detach()), ("dQ", q.grad), ("dK", k.grad), ("dV", v.grad)):
+        np.testing.assert_allclose(r[key], t.numpy(), atol=1e-13, err_msg=key)
+    s = scale * torch.einsum("bhid,bhjd->bhij", q.detach(), k.detach())
+    if causal:
+        s = s.masked_fill(~torch.tril(torch.ones(n, n, dtype=torch.bool)), float("-inf"))
+    np.testing.assert_allclose(r["L"], torch.logsumexp(s, -1).numpy(), atol=1e-13)
+
+
+# --------------------------------------------------------- P6: brute force, tiny
+@pytest.mark.parametrize("causal", [False, True])
+def test_brute_force_no_max_subtraction(causal):
+    n, d, scale = 7, 2, 0.5
+    Q, K, V, dO = _rand(n, d, 51, gain=0.5)
+    r = oracle.attn_head_full(Q, K, V, dO, causal, scale)
+    P = [[0.0] * n for _ in range(n)]
+    for i in range(n):
+        e = [math.exp(scale * sum(Q[i][k] * K[j][k] for k in range(d))) if (j <= i or not causal) else 0.0
+             for j in range(n)]
+        z = sum(e)
+        P[i] = [x / z for x in e]
+    for i in range(n):
+        for k in range(d):
+            assert abs(r["O"][i, k] - sum(P[i][j] * V[j][k] for j in range(n))) < 1e-14
+    for j in range(n):
+        for k in range(d):
+            assert abs(r["dV"][j, k] - sum(P[i][j] * dO[i][k] for i in range(n))) < 1e-14
+    dS = [[0.0] * n for _ in range(n)]
+    for i in range(n):
+        dP = [sum(dO[i][k] * V[j][k] for k in range(d)) for j in range(n)]
+        Di = sum(P[i][j] * dP[j] for j in range(n))
+        dS[i] = [P[i][j] * (dP[j] - Di) for j in range(n)]
+    for i in range(n):
+        for k in range(d):
+            assert abs(r["dQ"][i, k] - scale * sum(dS[i][j] * K[j][k] for j in range(n))) < 1e-14
+            assert abs(r["dK"][i, k] - scale * sum(dS[j][i] * Q[j][k] for j in range(n))) < 1e-14
+
+
+def test_large_scores_need_max_subtraction():
+    """Scores ~N(0, 30^2 d): exp overflows without the row-max subtraction."""
+    n, d = 16, 4
+    Q, K, V, dO = _rand(n, d, 61)
+    r = oracle.attn_head_full(30 * Q, 30 * K, V, dO, False, 1.0)
+    for key in ("O", "L", "dQ", "dK", "dV"):
+        assert np.all(np.isfinite(r[key])), key
+    np.testing.assert_allclose(r["P"].sum(1), 1.0, atol=1e-14)
+
+
+# ------------------------------- sampled-row / sampled-column entry points agree
+@pytest.mark.parametrize("causal", [False, True])
+def test_sampled_rows_and_cols_match_full(causal):
+    n, d, scale = 45, 6, 0.4
+    Q, K, V, dO = _rand(n, d, 71)
+    full = oracle.attn_head_full(Q, K, V, dO, causal, scale)
+    rows = [0, 1, 17, 44]
+    cols = [0, 3, 30, 44]
+    rr = oracle.attn_rows(Q, K, V, dO, causal, scale, rows)
+    cc = oracle.attn_cols(Q, K, V, dO, causal, scale, cols)
+    np.testing.assert_allclose(rr["O"], full["O"][rows], atol=1e-14)
+    np.testing.assert_allclose(rr["L"], full["L"][rows], atol=1e-14)
+    np.testing.assert_allclose(rr["dQ"], full["dQ"][rows], atol=1e-14)
+    np.testing.assert_allclose(cc["dK"], full["dK"][cols], atol=1e-13)
+    np.testing.assert_allclose(cc["dV"], full["dV"][cols], atol=1e-13)
+
+
+def test_batched_matches_per_head():
+    B, H, n, d = 2, 2, 10, 3
+    rng = np.random.default_rng(8)
+    Q, K, V, dO = (rng.standard_normal((B, H, n, d)) for _ in range(4))
+    r = oracle.attn_fwd_bwd(Q, K, V, dO, True, 0.7)
+    one = oracle.attn_head_full(Q[1, 0], K[1, 0], V[1, 0], dO[1, 0], True, 0.7)
+    for key in ("O", "L", "dQ", "dK", "dV"):
+        np.testing.assert_array_equal(r[key][1, 0], one[key])
+
+
+def test_paper_counts_fix_array_shapes():
+    """The paper's printed byte and atomic counts fix the shapes of the arrays
+    the oracle holds: Q,K,V,Out are B*N*D doubles, A is B*N*N doubles, and one
+    atomic site touches B*N*N*D elements."""
+    g = json.load(open(os.path.join(HERE, "golden", "paper_counts.json")))
+    B, N, D = 2, 2048, 64
+    t = g["dram_table_n2048"]
+    assert round(3 * B * N * D * 8 / 1e6, 3) == t["qkv_read_MB"]
+    assert round((B * N * N * 8 + B * N * D * 8) / 1e6, 3) == t["a_and_out_write_MB"]
+    assert round((3 * B * N * D * 8 + B * N * N * 8 + B * N * D * 8) / 1e6, 3) == t["total_MB"]
+    a = g["atomic_counts_n2048"]
+    assert B * N * N * D == a["backward_gk_only"]
+    assert 2 * B * N * N * D == a["fused_gv_and_gk"]
