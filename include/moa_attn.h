@@ -1,0 +1,138 @@
+/*
+ * moa_attn.h -- C ABI of the B200 (sm_100a) fused attention forward+backward library.
+ *
+ * The operation.  For every (batch b, head h) pair independently, with
+ * Q, K, V, dO in R^{n x d} and a scalar `scale`:
+ *
+ *     S = scale * Q K^T            (causal: S_ij = -inf for j > i; the diagonal is visible)
+ *     P = rowsoftmax(S)            L_i = log sum_j exp(S_ij)      (natural log)
+ *     O = P V
+ *     dV = P^T dO      dP = dO V^T      D_i = sum_k dO_ik O_ik
+ *     dS = P o (dP - D 1^T)        dQ = scale * dS K       dK = scale * dS^T Q
+ *
+ * These are the arrays the paper calls Q, K, V, Out, A (= P), GS (= dS), GQ, GK,
+ * GV (Sec. 3 traffic table; Sec. 4 backward and fused kernels).  The paper's
+ * point, and this library's contract, is that the fused path never stores the
+ * n x n arrays A and GS in device memory (Sec. 1.1, the two-ONF figure): extra
+ * memory is O(n d).  The paper's four-pass restructuring (Sec. 4, "the fix"),
+ * one-writer-per-element passes instead of one monolithic kernel with atomics
+ * on GV and GK, is kept: dK and dV are written without atomics by the CTA that
+ * owns the key tile.  How dQ is accumulated is selectable (`dq_mode`), because
+ * that step is where the paper's own regression (atomic contention) sat.
+ *
+ * Conventions common to every call
+ *  - All tensor arguments are DEVICE pointers to contiguous [B,H,n,d] arrays,
+ *    d fastest, 16-byte aligned; element type bfloat16 (MOA_BF16) or float
+ *    (MOA_F32) per desc->dtype.  L is a DEVICE pointer to float [B,H,n].
+ *  - The caller owns every buffer, workspace included.  The library never
+ *    allocates or frees device memory and keeps no per-call state.
+ *  - Calls enqueue kernels on `stream` (a cudaStream_t passed as void*; NULL is
+ *    the legacy default stream) and return without synchronising the host.
+ *  - Outputs are overwritten, never accumulated into.
+ *  - Errors are reported only through the returned moa_status; the library does
+ *    not abort or throw.  On any error nothing has been enqueued.
+ *  - Supported: d in {64, 128}; any n >= 1 and B, H >= 1 with B*H <= 65535*... (see
+ *    MOA_ERR_UNSUPPORTED); n need not be a multiple of the tile size.
+ *    A device that is not compute capability 10.x gives MOA_ERR_ARCH.
+ */
+#ifndef MOA_ATTN_H
+#define MOA_ATTN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MOA_OK = 0,
+    MOA_ERR_INVALID_ARG = 1, /* NULL pointer, misaligned pointer, non-positive size, bad enum  */
+    MOA_ERR_UNSUPPORTED = 2, /* well-formed request this build cannot run (e.g. d = 96)       */
+    MOA_ERR_WORKSPACE = 3,   /* ws == NULL or ws_bytes < moa_attn_workspace_bytes(...)         */
+    MOA_ERR_ARCH = 4,        /* current device is not sm_100                                   */
+    MOA_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed (launch, descriptor encode)  */
+    MOA_ERR_TIMEOUT = 6      /* a bounded device-side wait expired (reported by moa_last_device_status) */
+} moa_status;
+
+typedef enum { MOA_BF16 = 0, MOA_F32 = 1 } moa_dtype;
+
+/* How dQ_i = scale * sum_j dS_ij K_j is accumulated across key tiles (Sec. 4: the
+ * paper's GK/GV atomic sites and their removal, transposed here onto dQ because
+ * the backward kernel is parallel over key tiles). */
+typedef enum {
+    MOA_DQ_AUTO = 0,          /* library's choice (currently MOA_DQ_RED)                      */
+    MOA_DQ_RED = 1,           /* fp32 red.global.add into a [B,H,n,d] fp32 accumulator        */
+    MOA_DQ_BULK_REDUCE = 2,   /* shared-memory tile + cp.reduce.async.bulk add.f32            */
+    MOA_DQ_SEPARATE_PASS = 3  /* no atomics: a second, query-parallel kernel recomputes dS     */
+} moa_dq_mode;
+
+/* Which kernels run the contractions. */
+typedef enum {
+    MOA_PATH_AUTO = 0,  /* tensor cores when dtype is bf16, SIMT fp32 otherwise                */
+    MOA_PATH_SIMT = 1,  /* fp32 FMA kernels (any dtype); the only path for MOA_F32             */
+    MOA_PATH_TC = 2     /* tcgen05/TMEM/TMA kernels (bf16 only)                                */
+} moa_path;
+
+typedef enum { MOA_OP_FWD = 0, MOA_OP_BWD = 1, MOA_OP_FUSED = 2 } moa_op;
+
+typedef struct {
+    int32_t B, H, n, d;
+    int32_t causal;      /* 0 or 1                                                            */
+    float   scale;       /* multiplies Q K^T inside the softmax (the configs use 1/sqrt(d))    */
+    int32_t dtype;       /* moa_dtype of Q,K,V,dO,O,dQ,dK,dV                                   */
+    int32_t dq_mode;     /* moa_dq_mode                                                        */
+    int32_t materialize; /* 0: fused (no n x n array in memory).  1: comparison variant that
+                            writes P and dS to the workspace and reads them back (the paper's
+                            "left" ONF, Sec. 1.1); needs an O(n^2) workspace.                  */
+    int32_t path;        /* moa_path                                                           */
+} moa_attn_desc;
+
+/* Bytes of caller-provided workspace `op` (a moa_op) needs for `desc`.  Returns 0
+ * when none is needed and also when desc is invalid (the call itself reports why).
+ * Fused path: D [B,H,n] fp32 plus, for bf16 with an atomic dq_mode, an fp32
+ * [B,H,n,d] dQ accumulator: O(n d), never O(n^2). */
+size_t moa_attn_workspace_bytes(const moa_attn_desc *desc, int op);
+
+/* Forward: O = softmax(scale Q K^T) V and the per-row logsumexp L (needed by the
+ * backward).  Reads Q,K,V; writes O [B,H,n,d] and L [B,H,n].  (Paper: forward
+ * kernel, Sec. 3; fused ONF, Sec. 1.1.) */
+moa_status moa_attn_fwd(const moa_attn_desc *desc,
+                        const void *Q, const void *K, const void *V,
+                        void *O, float *L,
+                        void *ws, size_t ws_bytes, void *stream);
+
+/* Backward: dQ, dK, dV from dO, recomputing P tile by tile from L (written by
+ * moa_attn_fwd for the same Q,K,V,desc) and D = rowsum(dO o O) (the paper's
+ * "precompute pass", Sec. 4).  Reads Q,K,V,O,L,dO; writes dQ,dK,dV. */
+moa_status moa_attn_bwd(const moa_attn_desc *desc,
+                        const void *Q, const void *K, const void *V,
+                        const void *O, const float *L, const void *dO,
+                        void *dQ, void *dK, void *dV,
+                        void *ws, size_t ws_bytes, void *stream);
+
+/* Fused forward+backward (the paper's Algorithm 2 as one library call): several
+ * launches on one stream, no n x n array in memory.  Reads Q,K,V,dO; writes O, L,
+ * dQ, dK, dV. */
+moa_status moa_attn_fused_fwd_bwd(const moa_attn_desc *desc,
+                                  const void *Q, const void *K, const void *V, const void *dO,
+                                  void *O, float *L, void *dQ, void *dK, void *dV,
+                                  void *ws, size_t ws_bytes, void *stream);
+
+/* Synchronises `stream` and returns MOA_ERR_TIMEOUT if any kernel launched by this
+ * library on the current device gave up a bounded wait since the last call of this
+ * function (the flag is then cleared), MOA_ERR_CUDA if the stream reports an error,
+ * else MOA_OK.  Outputs of a timed-out kernel are undefined. */
+moa_status moa_last_device_status(void *stream);
+
+/* Number of kernel launches the library has enqueued in this process since it was
+ * loaded (all devices, all streams).  Host-side counter; for benchmarks. */
+uint64_t moa_launch_count(void);
+
+const char *moa_status_string(moa_status s);
+int moa_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOA_ATTN_H */

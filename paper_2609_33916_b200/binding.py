@@ -1,0 +1,146 @@
+"""ctypes binding of libmoa_attn.so: the same entry points as include/moa_attn.h.
+
+Argument marshalling only -- every step of the attention path runs in the
+library's CUDA kernels.  Tensor arguments may be torch CUDA tensors (their
+data_ptr() is passed) or plain integer device addresses.  There is no CPU or
+PyTorch fallback: if the library cannot be loaded, `lib()` raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libmoa_attn.so")
+
+MOA_OK, MOA_ERR_INVALID_ARG, MOA_ERR_UNSUPPORTED, MOA_ERR_WORKSPACE, MOA_ERR_ARCH, MOA_ERR_CUDA, MOA_ERR_TIMEOUT = range(7)
+MOA_BF16, MOA_F32 = 0, 1
+MOA_DQ_AUTO, MOA_DQ_RED, MOA_DQ_BULK_REDUCE, MOA_DQ_SEPARATE_PASS = 0, 1, 2, 3
+MOA_PATH_AUTO, MOA_PATH_SIMT, MOA_PATH_TC = 0, 1, 2
+MOA_OP_FWD, MOA_OP_BWD, MOA_OP_FUSED = 0, 1, 2
+
+#: every symbol include/moa_attn.h declares
+EXPORTS = (
+    "moa_attn_workspace_bytes", "moa_attn_fwd", "moa_attn_bwd", "moa_attn_fused_fwd_bwd",
+    "moa_last_device_status", "moa_launch_count", "moa_status_string", "moa_version",
+)
+
+
+class moa_attn_desc(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("n", ctypes.c_int32), ("d", ctypes.c_int32),
+                ("causal", ctypes.c_int32), ("scale", ctypes.c_float), ("dtype", ctypes.c_int32),
+                ("dq_mode", ctypes.c_int32), ("materialize", ctypes.c_int32), ("path", ctypes.c_int32)]
+
+
+class MoaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (moa_status {status})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libmoa_attn.so (built in-tree by paper_2609_33916_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2609_33916_b200.build` "
+                               "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, sz, dp = ctypes.c_void_p, ctypes.c_size_t, ctypes.POINTER(moa_attn_desc)
+        L.moa_attn_workspace_bytes.restype = sz
+        L.moa_attn_workspace_bytes.argtypes = [dp, ctypes.c_int]
+        L.moa_attn_fwd.restype = ctypes.c_int
+        L.moa_attn_fwd.argtypes = [dp] + [vp] * 5 + [vp, sz, vp]
+        L.moa_attn_bwd.restype = ctypes.c_int
+        L.moa_attn_bwd.argtypes = [dp] + [vp] * 9 + [vp, sz, vp]
+        L.moa_attn_fused_fwd_bwd.restype = ctypes.c_int
+        L.moa_attn_fused_fwd_bwd.argtypes = [dp] + [vp] * 9 + [vp, sz, vp]
+        L.moa_last_device_status.restype = ctypes.c_int
+        L.moa_last_device_status.argtypes = [vp]
+        L.moa_launch_count.restype = ctypes.c_uint64
+        L.moa_status_string.restype = ctypes.c_char_p
+        L.moa_status_string.argtypes = [ctypes.c_int]
+        L.moa_version.restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def make_desc(B, H, n, d, causal, scale, dtype=MOA_BF16, dq_mode=MOA_DQ_AUTO, materialize=0,
+              path=MOA_PATH_AUTO) -> moa_attn_desc:
+    return moa_attn_desc(int(B), int(H), int(n), int(d), int(bool(causal)), float(scale), int(dtype),
+                         int(dq_mode), int(materialize), int(path))
+
+
+def _ptr(x):
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return ctypes.c_void_p(x)
+    return ctypes.c_void_p(x.data_ptr())   # torch tensor
+
+
+def _nbytes(ws) -> int:
+    if ws is None:
+        return 0
+    return ws.numel() * ws.element_size()
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        if not torch.cuda.is_available():
+            return ctypes.c_void_p(0)   # host-side checks only; any launch will report MOA_ERR_CUDA
+        return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, int):
+        return ctypes.c_void_p(stream)
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def status_string(status: int) -> str:
+    return lib().moa_status_string(int(status)).decode()
+
+
+def moa_version() -> int:
+    return int(lib().moa_version())
+
+
+def moa_launch_count() -> int:
+    return int(lib().moa_launch_count())
+
+
+def moa_attn_workspace_bytes(desc: moa_attn_desc, op: int) -> int:
+    return int(lib().moa_attn_workspace_bytes(ctypes.byref(desc), int(op)))
+
+
+def moa_attn_fwd(desc, Q, K, V, O, L, ws=None, stream=None, ws_bytes=None, check=True) -> int:
+    s = lib().moa_attn_fwd(ctypes.byref(desc), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(L), _ptr(ws),
+                           _nbytes(ws) if ws_bytes is None else ws_bytes, _stream(stream))
+    if check and s != MOA_OK:
+        raise MoaError(s, "moa_attn_fwd")
+    return s
+
+
+def moa_attn_bwd(desc, Q, K, V, O, L, dO, dQ, dK, dV, ws=None, stream=None, ws_bytes=None, check=True) -> int:
+    s = lib().moa_attn_bwd(ctypes.byref(desc), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(L), _ptr(dO),
+                           _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(ws),
+                           _nbytes(ws) if ws_bytes is None else ws_bytes, _stream(stream))
+    if check and s != MOA_OK:
+        raise MoaError(s, "moa_attn_bwd")
+    return s
+
+
+def moa_attn_fused_fwd_bwd(desc, Q, K, V, dO, O, L, dQ, dK, dV, ws=None, stream=None, ws_bytes=None,
+                           check=True) -> int:
+    s = lib().moa_attn_fused_fwd_bwd(ctypes.byref(desc), _ptr(Q), _ptr(K), _ptr(V), _ptr(dO), _ptr(O),
+                                     _ptr(L), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(ws),
+                                     _nbytes(ws) if ws_bytes is None else ws_bytes, _stream(stream))
+    if check and s != MOA_OK:
+        raise MoaError(s, "moa_attn_fused_fwd_bwd")
+    return s
+
+
+def moa_last_device_status(stream=None) -> int:
+    return int(lib().moa_last_device_status(_stream(stream)))

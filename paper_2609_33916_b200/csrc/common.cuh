@@ -1,0 +1,49 @@
+// Shared declarations of the CUDA library's translation units (internal; the
+// public interface is include/moa_attn.h).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "moa_attn.h"
+
+namespace moa {
+
+struct Problem {
+    int B, H, n, d;
+    int causal;
+    float scale;
+    int BH() const { return B * H; }
+};
+
+// Host-side launch counter (moa_launch_count).
+void count_launch(int k = 1);
+
+// Device address of the status word kernels write when a bounded wait expires.
+unsigned int *device_status_ptr();
+
+template <typename T> __device__ __forceinline__ float to_float(T v);
+template <> __device__ __forceinline__ float to_float<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T> __device__ __forceinline__ T from_float(float v);
+template <> __device__ __forceinline__ float from_float<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// ---- SIMT fp32 path (simt_kernels.cu) -------------------------------------------------
+// dtype: MOA_BF16 or MOA_F32 storage; arithmetic is fp32 FMA throughout.
+cudaError_t simt_fwd(const Problem &p, int dtype, const void *Q, const void *K, const void *V,
+                     void *O, float *L, cudaStream_t st);
+// D_i = sum_k dO_ik O_ik
+cudaError_t row_dot(const Problem &p, int dtype, const void *dO, const void *O, float *Dv, cudaStream_t st);
+// dK, dV always; dQ contributions are atomically added into dQacc (fp32 [B,H,n,d], pre-zeroed)
+// when dQacc != nullptr.
+cudaError_t simt_bwd_kv(const Problem &p, int dtype, const void *Q, const void *K, const void *V,
+                        const void *dO, const float *L, const float *Dv,
+                        void *dK, void *dV, float *dQacc, cudaStream_t st);
+// atomic-free query-parallel dQ pass
+cudaError_t simt_bwd_dq(const Problem &p, int dtype, const void *Q, const void *K, const void *V,
+                        const void *dO, const float *L, const float *Dv, void *dQ, cudaStream_t st);
+// dst[i] = (bf16) src[i]
+cudaError_t convert_f32_to_bf16(const float *src, void *dst, size_t count, cudaStream_t st);
+
+}  // namespace moa

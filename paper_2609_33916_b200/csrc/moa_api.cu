@@ -1,0 +1,219 @@
+// C-ABI entry points (include/moa_attn.h): argument checks, workspace carving and
+// the sequence of kernel launches of each operation.  No arithmetic here.
+#include "common.cuh"
+#include <atomic>
+#include <mutex>
+
+namespace moa {
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int k) { g_launches.fetch_add((uint64_t)k, std::memory_order_relaxed); }
+
+// One status word per device image of this library; kernels with bounded waits set
+// it to a non-zero code when a wait expires.
+__device__ unsigned int g_device_status[4];
+
+unsigned int *device_status_ptr()
+{
+    constexpr int kMaxDev = 64;
+    static unsigned int *cache[kMaxDev] = {};
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return nullptr;
+    std::lock_guard<std::mutex> lk(mu);
+    if (!cache[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_device_status) != cudaSuccess) return nullptr;
+        cache[dev] = (unsigned int *)p;
+    }
+    return cache[dev];
+}
+
+namespace {
+
+constexpr size_t kAlign = 256;
+size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+moa_status check_arch()
+{
+    constexpr int kMaxDev = 64;
+    static std::atomic<int> cache[kMaxDev];  // 0 unknown, 1 ok, 2 wrong arch
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MOA_ERR_CUDA;
+    if (dev >= 0 && dev < kMaxDev && cache[dev].load() != 0)
+        return cache[dev].load() == 1 ? MOA_OK : MOA_ERR_ARCH;
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return MOA_ERR_CUDA;
+    const bool ok = major == 10;
+    if (dev >= 0 && dev < kMaxDev) cache[dev].store(ok ? 1 : 2);
+    return ok ? MOA_OK : MOA_ERR_ARCH;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Shape/enum checks that need no device.
+moa_status check_desc(const moa_attn_desc *d)
+{
+    if (!d) return MOA_ERR_INVALID_ARG;
+    if (d->B <= 0 || d->H <= 0 || d->n <= 0 || d->d <= 0) return MOA_ERR_INVALID_ARG;
+    if (d->causal != 0 && d->causal != 1) return MOA_ERR_INVALID_ARG;
+    if (d->dtype != MOA_BF16 && d->dtype != MOA_F32) return MOA_ERR_INVALID_ARG;
+    if (d->dq_mode < MOA_DQ_AUTO || d->dq_mode > MOA_DQ_SEPARATE_PASS) return MOA_ERR_INVALID_ARG;
+    if (d->materialize != 0 && d->materialize != 1) return MOA_ERR_INVALID_ARG;
+    if (d->path < MOA_PATH_AUTO || d->path > MOA_PATH_TC) return MOA_ERR_INVALID_ARG;
+    if (!(d->scale == d->scale) || d->scale - d->scale != 0.f) return MOA_ERR_INVALID_ARG;  // NaN / inf
+    if (d->d != 64 && d->d != 128) return MOA_ERR_UNSUPPORTED;
+    if ((long long)d->B * d->H > (1 << 20)) return MOA_ERR_UNSUPPORTED;
+    // one CTA per (tile, head) in grid.x
+    const long long tiles = ((long long)d->n + 63) / 64;
+    if (tiles * d->B * d->H >= (1LL << 31)) return MOA_ERR_UNSUPPORTED;
+    if (d->path == MOA_PATH_TC && d->dtype != MOA_BF16) return MOA_ERR_UNSUPPORTED;
+    if (d->path == MOA_PATH_TC) return MOA_ERR_UNSUPPORTED;   // tensor-core kernels not built yet
+    if (d->materialize) return MOA_ERR_UNSUPPORTED;           // comparison variant not built yet
+    if (d->dq_mode == MOA_DQ_BULK_REDUCE) return MOA_ERR_UNSUPPORTED;
+    return MOA_OK;
+}
+
+int resolved_dq_mode(const moa_attn_desc *d) { return d->dq_mode == MOA_DQ_AUTO ? MOA_DQ_RED : d->dq_mode; }
+
+struct BwdWorkspace {
+    size_t d_bytes, dqacc_bytes, total;
+};
+BwdWorkspace bwd_workspace(const moa_attn_desc *d)
+{
+    BwdWorkspace w{};
+    const size_t rows = (size_t)d->B * d->H * d->n;
+    w.d_bytes = align_up(rows * sizeof(float));
+    const bool need_acc = d->dtype == MOA_BF16 && resolved_dq_mode(d) != MOA_DQ_SEPARATE_PASS;
+    w.dqacc_bytes = need_acc ? align_up(rows * d->d * sizeof(float)) : 0;
+    w.total = w.d_bytes + w.dqacc_bytes;
+    return w;
+}
+
+Problem to_problem(const moa_attn_desc *d) { return Problem{d->B, d->H, d->n, d->d, d->causal, d->scale}; }
+
+moa_status run_fwd(const moa_attn_desc *d, const void *Q, const void *K, const void *V, void *O, float *L,
+                   cudaStream_t st)
+{
+    return simt_fwd(to_problem(d), d->dtype, Q, K, V, O, L, st) == cudaSuccess ? MOA_OK : MOA_ERR_CUDA;
+}
+
+moa_status run_bwd(const moa_attn_desc *d, const void *Q, const void *K, const void *V, const void *O,
+                   const float *L, const void *dO, void *dQ, void *dK, void *dV, void *ws, cudaStream_t st)
+{
+    const Problem p = to_problem(d);
+    const BwdWorkspace w = bwd_workspace(d);
+    float *Dv = (float *)ws;
+    float *dQacc = w.dqacc_bytes ? (float *)((char *)ws + w.d_bytes) : nullptr;
+    const size_t elems = (size_t)p.BH() * p.n * p.d;
+    const int mode = resolved_dq_mode(d);
+#define MOA_TRY(x) do { if ((x) != cudaSuccess) return MOA_ERR_CUDA; } while (0)
+    MOA_TRY(row_dot(p, d->dtype, dO, O, Dv, st));
+    if (mode == MOA_DQ_SEPARATE_PASS) {
+        MOA_TRY(simt_bwd_kv(p, d->dtype, Q, K, V, dO, L, Dv, dK, dV, nullptr, st));
+        MOA_TRY(simt_bwd_dq(p, d->dtype, Q, K, V, dO, L, Dv, dQ, st));
+    } else {
+        float *acc = d->dtype == MOA_F32 ? (float *)dQ : dQacc;   // fp32 output accumulates in place
+        MOA_TRY(cudaMemsetAsync(acc, 0, elems * sizeof(float), st));
+        MOA_TRY(simt_bwd_kv(p, d->dtype, Q, K, V, dO, L, Dv, dK, dV, acc, st));
+        if (d->dtype == MOA_BF16) MOA_TRY(convert_f32_to_bf16(dQacc, dQ, elems, st));
+    }
+#undef MOA_TRY
+    return MOA_OK;
+}
+
+}  // namespace
+}  // namespace moa
+
+using namespace moa;
+
+extern "C" {
+
+size_t moa_attn_workspace_bytes(const moa_attn_desc *desc, int op)
+{
+    if (check_desc(desc) != MOA_OK) return 0;
+    if (op == MOA_OP_FWD) return 0;
+    if (op == MOA_OP_BWD || op == MOA_OP_FUSED) return bwd_workspace(desc).total;
+    return 0;
+}
+
+moa_status moa_attn_fwd(const moa_attn_desc *desc, const void *Q, const void *K, const void *V,
+                        void *O, float *L, void *ws, size_t ws_bytes, void *stream)
+{
+    moa_status s = check_desc(desc);
+    if (s != MOA_OK) return s;
+    if (!Q || !K || !V || !O || !L) return MOA_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(L)) return MOA_ERR_INVALID_ARG;
+    (void)ws; (void)ws_bytes;
+    if ((s = check_arch()) != MOA_OK) return s;
+    return run_fwd(desc, Q, K, V, O, L, (cudaStream_t)stream);
+}
+
+moa_status moa_attn_bwd(const moa_attn_desc *desc, const void *Q, const void *K, const void *V,
+                        const void *O, const float *L, const void *dO,
+                        void *dQ, void *dK, void *dV, void *ws, size_t ws_bytes, void *stream)
+{
+    moa_status s = check_desc(desc);
+    if (s != MOA_OK) return s;
+    if (!Q || !K || !V || !O || !L || !dO || !dQ || !dK || !dV) return MOA_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(L) || !aligned16(dO) ||
+        !aligned16(dQ) || !aligned16(dK) || !aligned16(dV))
+        return MOA_ERR_INVALID_ARG;
+    const size_t need = bwd_workspace(desc).total;
+    if (!ws || ws_bytes < need) return MOA_ERR_WORKSPACE;
+    if (!aligned16(ws)) return MOA_ERR_INVALID_ARG;
+    if ((s = check_arch()) != MOA_OK) return s;
+    return run_bwd(desc, Q, K, V, O, L, dO, dQ, dK, dV, ws, (cudaStream_t)stream);
+}
+
+moa_status moa_attn_fused_fwd_bwd(const moa_attn_desc *desc, const void *Q, const void *K, const void *V,
+                                  const void *dO, void *O, float *L, void *dQ, void *dK, void *dV,
+                                  void *ws, size_t ws_bytes, void *stream)
+{
+    moa_status s = check_desc(desc);
+    if (s != MOA_OK) return s;
+    if (!Q || !K || !V || !O || !L || !dO || !dQ || !dK || !dV) return MOA_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(L) || !aligned16(dO) ||
+        !aligned16(dQ) || !aligned16(dK) || !aligned16(dV))
+        return MOA_ERR_INVALID_ARG;
+    const size_t need = bwd_workspace(desc).total;
+    if (!ws || ws_bytes < need) return MOA_ERR_WORKSPACE;
+    if (!aligned16(ws)) return MOA_ERR_INVALID_ARG;
+    if ((s = check_arch()) != MOA_OK) return s;
+    if ((s = run_fwd(desc, Q, K, V, O, L, (cudaStream_t)stream)) != MOA_OK) return s;
+    return run_bwd(desc, Q, K, V, O, L, dO, dQ, dK, dV, ws, (cudaStream_t)stream);
+}
+
+moa_status moa_last_device_status(void *stream)
+{
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return MOA_ERR_CUDA;
+    unsigned int *p = device_status_ptr();
+    if (!p) return MOA_ERR_CUDA;
+    unsigned int h[4] = {0, 0, 0, 0};
+    if (cudaMemcpy(h, p, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) return MOA_ERR_CUDA;
+    if (h[0] != 0) {
+        cudaMemset(p, 0, sizeof(h));
+        return MOA_ERR_TIMEOUT;
+    }
+    return MOA_OK;
+}
+
+uint64_t moa_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char *moa_status_string(moa_status s)
+{
+    switch (s) {
+        case MOA_OK: return "ok";
+        case MOA_ERR_INVALID_ARG: return "invalid argument";
+        case MOA_ERR_UNSUPPORTED: return "unsupported configuration";
+        case MOA_ERR_WORKSPACE: return "workspace missing or too small";
+        case MOA_ERR_ARCH: return "device is not sm_100";
+        case MOA_ERR_CUDA: return "CUDA call failed";
+        case MOA_ERR_TIMEOUT: return "bounded device wait expired";
+    }
+    return "unknown status";
+}
+
+int moa_version(void) { return 100; }
+
+}  // extern "C"

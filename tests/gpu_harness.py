@@ -1,0 +1,66 @@
+"""Helpers for the GPU parity tests: move seeded inputs to the device, call the
+library through its C ABI (via the ctypes binding) and bring results back as
+float64 numpy arrays.  torch is used for device memory only."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from paper_2609_33916_b200 import binding as mb
+from paper_2609_33916_b200 import inputs as mi
+
+TOL_BF16 = 1e-2   # max|err|/max|ref| per output, bf16 storage with fp32 accumulation
+TOL_F32 = 1e-5    # the fp32 path
+
+
+def to_device(arr: np.ndarray, dtype: str) -> torch.Tensor:
+    if dtype == "bf16":
+        return torch.from_numpy(arr.view(np.int16)).cuda().view(torch.bfloat16)
+    return torch.from_numpy(arr).cuda()
+
+
+def to_host_f64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to(torch.float64).cpu().numpy()
+
+
+def run_library(inp: dict, dtype: str, causal: bool, scale: float, *, op: str = "fused",
+                dq_mode: int = mb.MOA_DQ_AUTO, path: int = mb.MOA_PATH_AUTO, materialize: int = 0,
+                poison: bool = True) -> dict:
+    """op: 'fused' (one call) or 'split' (moa_attn_fwd then moa_attn_bwd) or 'fwd'."""
+    B, H, n, d = inp["Q"].shape
+    Q, K, V, dO = (to_device(inp[k], dtype) for k in ("Q", "K", "V", "dO"))
+    desc = mb.make_desc(B, H, n, d, causal, scale, mb.MOA_BF16 if dtype == "bf16" else mb.MOA_F32,
+                        dq_mode, materialize, path)
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    fill = float("nan") if poison else 0.0   # unwritten elements must show up
+    O, dQ, dK, dV = (torch.full((B, H, n, d), fill, dtype=tdt, device="cuda") for _ in range(4))
+    L = torch.full((B, H, n), fill, dtype=torch.float32, device="cuda")
+    ws_bytes = mb.moa_attn_workspace_bytes(desc, mb.MOA_OP_FUSED if op != "fwd" else mb.MOA_OP_FWD)
+    ws = torch.full((max(ws_bytes, 16),), 0xFF, dtype=torch.uint8, device="cuda")
+    if op == "fused":
+        mb.moa_attn_fused_fwd_bwd(desc, Q, K, V, dO, O, L, dQ, dK, dV, ws)
+    elif op == "split":
+        mb.moa_attn_fwd(desc, Q, K, V, O, L, ws)
+        mb.moa_attn_bwd(desc, Q, K, V, O, L, dO, dQ, dK, dV, ws)
+    elif op == "fwd":
+        mb.moa_attn_fwd(desc, Q, K, V, O, L, ws)
+    else:
+        raise ValueError(op)
+    st = mb.moa_last_device_status()
+    assert st == mb.MOA_OK, mb.status_string(st)
+    out = dict(O=to_host_f64(O), L=to_host_f64(L))
+    if op != "fwd":
+        out.update(dQ=to_host_f64(dQ), dK=to_host_f64(dK), dV=to_host_f64(dV))
+    out["ws_bytes"] = ws_bytes
+    return out
+
+
+def f64_inputs(inp: dict, dtype: str) -> dict:
+    return {k: mi.to_f64(v, dtype) for k, v in inp.items()}
+
+
+def assert_close(got: dict, ref: dict, tol: float, keys=("O", "dQ", "dK", "dV"), tag=""):
+    errs = {k: mi.rel_err(got[k], ref[k]) for k in keys}
+    bad = {k: e for k, e in errs.items() if not (e <= tol)}
+    assert not bad, f"{tag} max|err|/max|ref| over tolerance {tol}: {errs}"
+    return errs

@@ -1,0 +1,72 @@
+"""The C-ABI library loads and exports every symbol the header declares; host-side
+argument checks return the documented codes.  No kernel is launched here."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2609_33916_b200 import binding as mb
+from paper_2609_33916_b200 import build as mbuild
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    mbuild.build()
+    return mb.lib()
+
+
+def test_header_symbols_are_exported(lib):
+    hdr = open(os.path.join(ROOT, "include", "moa_attn.h")).read()
+    declared = set(re.findall(r"\b(moa_[a-z_0-9]+)\s*\(", hdr))
+    assert declared == set(mb.EXPORTS), declared ^ set(mb.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_version_and_strings(lib):
+    assert mb.moa_version() >= 100
+    assert mb.status_string(mb.MOA_OK) == "ok"
+    for s in range(1, 7):
+        assert mb.status_string(s) not in ("ok", "unknown status")
+    assert mb.status_string(99) == "unknown status"
+
+
+def test_desc_struct_layout_matches_header():
+    assert ctypes.sizeof(mb.moa_attn_desc) == 40
+    assert mb.moa_attn_desc.scale.offset == 20
+
+
+def test_workspace_is_linear_in_n(lib):
+    def ws(n, mode=mb.MOA_DQ_RED, dtype=mb.MOA_BF16):
+        return mb.moa_attn_workspace_bytes(mb.make_desc(1, 32, n, 128, True, 0.1, dtype, mode), mb.MOA_OP_FUSED)
+    assert ws(512, mb.MOA_DQ_RED) == 32 * 512 * 4 + 32 * 512 * 128 * 4
+    assert ws(32768) == 64 * ws(512)                      # O(n d): no n^2 term
+    assert ws(512, mb.MOA_DQ_SEPARATE_PASS) == 32 * 512 * 4
+    assert ws(512, mb.MOA_DQ_RED, mb.MOA_F32) == 32 * 512 * 4
+    assert mb.moa_attn_workspace_bytes(mb.make_desc(1, 32, 512, 128, True, 0.1), mb.MOA_OP_FWD) == 0
+
+
+def test_argument_errors_need_no_device(lib):
+    good = mb.make_desc(1, 1, 128, 64, False, 0.125, mb.MOA_F32)
+    a = 4096  # fake, aligned, never dereferenced: checks fail first
+    assert mb.moa_attn_fwd(good, 0, a, a, a, a, check=False) == mb.MOA_ERR_INVALID_ARG
+    assert mb.moa_attn_fwd(good, a + 2, a, a, a, a, check=False) == mb.MOA_ERR_INVALID_ARG
+    for field, val, want in (("n", 0, mb.MOA_ERR_INVALID_ARG), ("d", 96, mb.MOA_ERR_UNSUPPORTED),
+                             ("causal", 2, mb.MOA_ERR_INVALID_ARG), ("dtype", 7, mb.MOA_ERR_INVALID_ARG),
+                             ("dq_mode", 9, mb.MOA_ERR_INVALID_ARG), ("scale", float("nan"), mb.MOA_ERR_INVALID_ARG)):
+        d = mb.make_desc(1, 1, 128, 64, False, 0.125, mb.MOA_F32)
+        setattr(d, field, val)
+        assert mb.moa_attn_fwd(d, a, a, a, a, a, check=False) == want, field
+        assert mb.moa_attn_workspace_bytes(d, mb.MOA_OP_FUSED) == 0
+    # backward without / with a short workspace
+    d = mb.make_desc(1, 1, 128, 64, False, 0.125, mb.MOA_BF16)
+    need = mb.moa_attn_workspace_bytes(d, mb.MOA_OP_BWD)
+    assert need > 0
+    assert mb.moa_attn_bwd(d, a, a, a, a, a, a, a, a, a, None, check=False) == mb.MOA_ERR_WORKSPACE
+    assert mb.moa_attn_bwd(d, a, a, a, a, a, a, a, a, a, a, ws_bytes=need - 1, check=False) == mb.MOA_ERR_WORKSPACE
+    assert mb.moa_attn_fused_fwd_bwd(d, a, a, a, a, a, a, a, a, a, a, ws_bytes=need - 1, check=False) == mb.MOA_ERR_WORKSPACE
+    with pytest.raises(mb.MoaError):
+        mb.moa_attn_fwd(good, 0, a, a, a, a)
