@@ -1,0 +1,366 @@
+#!/usr/bin/env python
+"""Benchmark of the fused attention forward+backward path.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--dq-mode M]
+  python bench.py --impl reference ...      # times the fp64 CPU oracle instead
+
+A step is one moa_attn_fused_fwd_bwd call (forward, preprocess, backward, dQ
+conversion) over one batch of synthetic bf16 inputs.  The metric is model
+TFLOP/s: 4 n^2 d forward + 10 n^2 d backward per head, halved when causal.
+With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank
+runs the whole workload on its own GPU -- (batch, head) pairs are independent,
+so there is no collective on the data path -- and the value is the sum over
+ranks divided by the slowest rank's time (weak scaling).
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "fused attn fwd+bwd TFLOP/s and % of B200 dense BF16 tensor peak"
+NOMINAL_BF16_TFLOPS = 2250.0   # datasheet dense bf16, for context
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            d = json.load(f)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------- clock sampling
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs
+    (read-only queries)."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.nv is not None:
+            self._stop.clear()
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+
+    def stop(self):
+        if self._thr is not None:
+            self._stop.set()
+            self._thr.join()
+            self._thr = None
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# --------------------------------------------------------------------- CPU oracle legs
+def time_oracle_sample(w, budget_s: float):
+    """Times the oracle, as it stands, on a bounded sample of workload `w`: whole heads
+    (forward + backward, all n^2 work of each) when one head fits the budget, otherwise
+    sampled query rows of head (0,0).  Returns (tflops, seconds, cores, description)."""
+    import numpy as np
+    import oracle
+    from paper_2609_33916_b200 import inputs as mi
+
+    cores = oracle.num_threads()
+    # calibrate on a small head
+    nc = min(w.n, 1024)
+    cal = mi.make_inputs(1, 1, nc, w.d, seed=99, dtype=w.dtype)
+    f = {k: mi.to_f64(v, w.dtype) for k, v in cal.items()}
+    t0 = time.perf_counter()
+    oracle.attn_fwd_bwd(f["Q"], f["K"], f["V"], f["dO"], w.causal, w.scale)
+    rate = 14.0 * nc * nc * w.d / max(time.perf_counter() - t0, 1e-6)     # flop/s, dense count
+    head_flops_dense = 14.0 * float(w.n) ** 2 * w.d
+    head_model = head_flops_dense * (0.5 if w.causal else 1.0)
+    est_head = head_flops_dense / rate * 1.6          # large n runs slower per flop than the calibration
+    mem_ok = 2.0 * w.n * w.n * 8 < 24e9
+    inp = mi.make_inputs(1, 1, w.n, w.d, seed=w.seed, dtype=w.dtype)
+    f = {k: mi.to_f64(v, w.dtype) for k, v in inp.items()}
+    if est_head <= budget_s and mem_ok:
+        heads = max(1, min(w.B * w.H, int(budget_s / est_head)))
+        t0 = time.perf_counter()
+        for _ in range(heads):
+            oracle.attn_fwd_bwd(f["Q"], f["K"], f["V"], f["dO"], w.causal, w.scale)
+        dt = time.perf_counter() - t0
+        return heads * head_model / dt / 1e12, dt, cores, f"{heads} of {w.B * w.H} heads, full fwd+bwd"
+    # row sample: S, P, O, dP, dS, dQ of r rows = 8 n d executed flops per row (4 n d
+    # forward + 4 n d of the backward); credited as that share of the model count
+    per_row = 8.0 * w.n * w.d
+    r = int(max(8, min(w.n, budget_s * rate / 1.6 / per_row)))
+    rows = np.linspace(0, w.n - 1, r).astype(np.int32)
+    t0 = time.perf_counter()
+    oracle.attn_rows(f["Q"][0, 0], f["K"][0, 0], f["V"][0, 0], f["dO"][0, 0], w.causal, w.scale, rows)
+    dt = time.perf_counter() - t0
+    credit = per_row * r * (0.5 if w.causal else 1.0)
+    return credit / dt / 1e12, dt, cores, (f"{r} query rows of head (0,0): S,P,O,dP,dS,dQ only, "
+                                             f"8nd flop per row credited")
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    total_budget = 150.0
+    per_step = total_budget / max(1, args.steps + args.warmup)
+    vals, secs, cores, desc = [], [], 0, ""
+    for i in range(args.warmup + args.steps):
+        v, dt, cores, desc = time_oracle_sample(w, per_step)
+        if i >= args.warmup:
+            vals.append(v)
+            secs.append(dt)
+    value = sum(vals) / len(vals)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(secs) / len(secs),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w, args),
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def workload_config(w, args):
+    return {"workload": w.name, "B": w.B, "H": w.H, "n": w.n, "d": w.d, "causal": w.causal,
+            "scale": "1/sqrt(d)", "dq_mode": args.dq_mode, "path": args.path,
+            "l2": "inputs+outputs per step exceed the 126 MB L2; no explicit flush",
+            "parallelism": f"independent (b,h) shards x{args.gpus}"}
+
+
+# ------------------------------------------------------------------------------ main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="moa", choices=["moa", "reference"])
+    ap.add_argument("--workload", default="c4_long")
+    ap.add_argument("--dq-mode", type=int, default=0)
+    ap.add_argument("--path", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "moa" else args.warmup
+
+    from paper_2609_33916_b200 import inputs as mi
+    w = mi.CONFIGS[args.workload]
+    if args.impl == "reference":
+        return run_reference(args, w)
+
+    import torch
+    from paper_2609_33916_b200 import binding as mb
+    from paper_2609_33916_b200 import build as mbuild
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        mbuild.build()
+    if dist is not None:
+        dist.barrier()
+    mb.lib()
+    peaks, peaks_kind = load_peaks()
+
+    B, H, n, d = w.B, w.H, w.n, w.d
+    desc = mb.make_desc(B, H, n, d, w.causal, w.scale, mb.MOA_BF16, args.dq_mode, 0, args.path)
+    shape = (B, H, n, d)
+    base_mem = torch.cuda.memory_allocated()
+    gen = torch.Generator(device="cuda").manual_seed(w.seed + 1000 * rank)
+    Q, K, V, dO = (torch.randn(shape, generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+                   for _ in range(4))
+    O, dQ, dK, dV = (torch.empty(shape, dtype=torch.bfloat16, device="cuda") for _ in range(4))
+    L = torch.empty((B, H, n), dtype=torch.float32, device="cuda")
+    ws_bytes = mb.moa_attn_workspace_bytes(desc, mb.MOA_OP_FUSED)
+    ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device="cuda")
+    torch.cuda.synchronize()
+    resident_bytes = torch.cuda.memory_allocated() - base_mem
+    stream = torch.cuda.current_stream()
+
+    def step():
+        mb.moa_attn_fused_fwd_bwd(desc, Q, K, V, dO, O, L, dQ, dK, dV, ws, stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    for _ in range(args.warmup):
+        step()
+    st = mb.moa_last_device_status(stream)
+    if st != mb.MOA_OK:
+        raise SystemExit(f"device status after warm-up: {mb.status_string(st)}")
+
+    # ---- timed region: K steps, device-resident inputs ----
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    mb.moa_profile_read()
+    mb.moa_profile_enable(True)
+    barrier()
+    sampler.start()
+    launches0 = mb.moa_launch_count()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    launches = mb.moa_launch_count() - launches0
+    sampler.stop()
+    mb.moa_profile_enable(False)
+    prof = mb.moa_profile_read()
+    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    ms_per_step = ms_total / args.steps
+    flops_step = w.model_flops
+    value = world * flops_step / (ms_per_step * 1e-3) / 1e12
+    peak_bytes = torch.cuda.max_memory_allocated() - base_mem
+
+    # ---- end to end: pinned host inputs -> device, call, results -> pinned host ----
+    hQ, hK, hV, hdO = (t.cpu().pin_memory() for t in (Q, K, V, dO))
+    hO, hdQ, hdK, hdV = (torch.empty(shape, dtype=torch.bfloat16).pin_memory() for _ in range(4))
+    hL = torch.empty((B, H, n), dtype=torch.float32).pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in (hQ, hK, hV, hdO))
+    d2h = sum(t.numel() * t.element_size() for t in (hO, hdQ, hdK, hdV, hL))
+
+    def e2e_step():
+        Q.copy_(hQ, non_blocking=True); K.copy_(hK, non_blocking=True)
+        V.copy_(hV, non_blocking=True); dO.copy_(hdO, non_blocking=True)
+        step()
+        hO.copy_(O, non_blocking=True); hdQ.copy_(dQ, non_blocking=True)
+        hdK.copy_(dK, non_blocking=True); hdV.copy_(dV, non_blocking=True); hL.copy_(L, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e2e_steps = max(3, min(args.steps, 10))
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
+    e2e_value = world * flops_step / (e2e_ms * 1e-3) / 1e12
+    st = mb.moa_last_device_status(stream)
+    if st != mb.MOA_OK:
+        raise SystemExit(f"device status: {mb.status_string(st)}")
+
+    # ---- roofline of the dominant kernel (the key-tile-parallel backward) ----
+    heads = B * H
+    causal_f = 0.5 if w.causal else 1.0
+    alg_flops = {"fwd": 4.0 * heads * n * n * d * causal_f, "bwd_kv": 10.0 * heads * n * n * d * causal_f,
+                 "bwd_dq": 0.0}
+    if prof["bwd_dq"][1] > 0:   # separate pass: dQ's 2 n^2 d moves to that kernel (its recompute is not credited)
+        alg_flops["bwd_kv"] = 8.0 * heads * n * n * d * causal_f
+        alg_flops["bwd_dq"] = 2.0 * heads * n * n * d * causal_f
+    dominant = max(("fwd", "bwd_kv", "bwd_dq"), key=lambda k: prof[k][0])
+    dom_ms = prof[dominant][0] / max(1, prof[dominant][1])
+    achieved = alg_flops[dominant] / (dom_ms * 1e-3) / 1e12 if dom_ms > 0 else None
+    tc_path = args.path in (0, 2)
+    peak = peaks["bf16_tflops_sustained"]
+    roofline = {"bound": "tensor", "kernel": dominant, "achieved": achieved, "peak": peak,
+                "unit": "TFLOP/s", "frac": (achieved / peak) if achieved else None, "traffic": None,
+                "peak_source": f"{peaks_kind} bf16_tflops_sustained (kernel timed inside a long step)",
+                "kernel_ms": dom_ms,
+                "per_kernel_ms": {k: (v[0] / max(1, v[1]), v[1]) for k, v in prof.items() if v[1]}}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(w, args),
+        "pct_of_peak": {"of_measured_burst": 100 * value / world / peaks["bf16_tflops"],
+                        "of_measured_sustained": 100 * value / world / peaks["bf16_tflops_sustained"],
+                        "of_nominal_2250": 100 * value / world / NOMINAL_BF16_TFLOPS, "peaks": peaks_kind},
+        "hbm_bytes": {"resident_inputs_outputs_workspace": resident_bytes, "peak_allocated": peak_bytes,
+                      "workspace": ws_bytes, "one_nxn_fp32_array_all_heads_not_allocated": 4 * heads * n * n},
+        "clocks": sampler.summary(),
+        "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_ms},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, dt, cores, desc_s = time_oracle_sample(w, 20.0)
+        line["cpu_baseline"] = {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+                                "sample": desc_s, "seconds": dt}
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

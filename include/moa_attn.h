@@ -31,8 +31,9 @@
  *  - Outputs are overwritten, never accumulated into.
  *  - Errors are reported only through the returned moa_status; the library does
  *    not abort or throw.  On any error nothing has been enqueued.
- *  - Supported: d in {64, 128}; any n >= 1 and B, H >= 1 with B*H <= 65535*... (see
- *    MOA_ERR_UNSUPPORTED); n need not be a multiple of the tile size.
+ *  - Supported: d in {64, 128}; any n >= 1 and B, H >= 1 (B*H <= 2^20 and
+ *    ceil(n/64)*B*H < 2^31, else MOA_ERR_UNSUPPORTED); n need not be a multiple
+ *    of the tile size.
  *    A device that is not compute capability 10.x gives MOA_ERR_ARCH.
  */
 #ifndef MOA_ATTN_H
@@ -124,6 +125,21 @@ moa_status moa_attn_fused_fwd_bwd(const moa_attn_desc *desc,
  * function (the flag is then cleared), MOA_ERR_CUDA if the stream reports an error,
  * else MOA_OK.  Outputs of a timed-out kernel are undefined. */
 moa_status moa_last_device_status(void *stream);
+
+/* Per-kernel device timing, for benchmarks.  The paper's lesson that device time and
+ * wall time differ (Sec. 3, device-timer vs wall clock) is why this exists: while
+ * enabled, the library records a CUDA event pair on the caller's stream around each
+ * kernel it launches (at most MOA_PROFILE_MAX_RECORDS launches between two reads; later
+ * ones go untimed).  moa_profile_read synchronises on the recorded events, adds up
+ * elapsed milliseconds and launch counts per kernel kind into out (arrays of
+ * MOA_KERNEL_KINDS entries), and clears the records.  Not thread-safe; one device at a
+ * time.  Returns MOA_ERR_CUDA if an event call fails. */
+enum { MOA_KERNEL_FWD = 0, MOA_KERNEL_PREPROCESS = 1, MOA_KERNEL_BWD_KV = 2, MOA_KERNEL_BWD_DQ = 3,
+       MOA_KERNEL_CONVERT = 4, MOA_KERNEL_OTHER = 5, MOA_KERNEL_KINDS = 6 };
+enum { MOA_PROFILE_MAX_RECORDS = 4096 };
+typedef struct { float ms[MOA_KERNEL_KINDS]; uint32_t launches[MOA_KERNEL_KINDS]; } moa_profile;
+moa_status moa_profile_enable(int on);
+moa_status moa_profile_read(moa_profile *out);
 
 /* Number of kernel launches the library has enqueued in this process since it was
  * loaded (all devices, all streams).  Host-side counter; for benchmarks. */

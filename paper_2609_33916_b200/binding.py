@@ -23,6 +23,7 @@ MOA_OP_FWD, MOA_OP_BWD, MOA_OP_FUSED = 0, 1, 2
 EXPORTS = (
     "moa_attn_workspace_bytes", "moa_attn_fwd", "moa_attn_bwd", "moa_attn_fused_fwd_bwd",
     "moa_last_device_status", "moa_launch_count", "moa_status_string", "moa_version",
+    "moa_profile_enable", "moa_profile_read",
 )
 
 
@@ -30,6 +31,14 @@ class moa_attn_desc(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("n", ctypes.c_int32), ("d", ctypes.c_int32),
                 ("causal", ctypes.c_int32), ("scale", ctypes.c_float), ("dtype", ctypes.c_int32),
                 ("dq_mode", ctypes.c_int32), ("materialize", ctypes.c_int32), ("path", ctypes.c_int32)]
+
+
+MOA_KERNEL_KINDS = 6
+KERNEL_KIND_NAMES = ("fwd", "preprocess", "bwd_kv", "bwd_dq", "convert", "other")
+
+
+class moa_profile(ctypes.Structure):
+    _fields_ = [("ms", ctypes.c_float * MOA_KERNEL_KINDS), ("launches", ctypes.c_uint32 * MOA_KERNEL_KINDS)]
 
 
 class MoaError(RuntimeError):
@@ -64,6 +73,10 @@ def lib() -> ctypes.CDLL:
         L.moa_status_string.restype = ctypes.c_char_p
         L.moa_status_string.argtypes = [ctypes.c_int]
         L.moa_version.restype = ctypes.c_int
+        L.moa_profile_enable.restype = ctypes.c_int
+        L.moa_profile_enable.argtypes = [ctypes.c_int]
+        L.moa_profile_read.restype = ctypes.c_int
+        L.moa_profile_read.argtypes = [ctypes.POINTER(moa_profile)]
         _lib = L
     return _lib
 
@@ -144,3 +157,16 @@ def moa_attn_fused_fwd_bwd(desc, Q, K, V, dO, O, L, dQ, dK, dV, ws=None, stream=
 
 def moa_last_device_status(stream=None) -> int:
     return int(lib().moa_last_device_status(_stream(stream)))
+
+
+def moa_profile_enable(on: bool) -> int:
+    return int(lib().moa_profile_enable(int(bool(on))))
+
+
+def moa_profile_read() -> dict:
+    """{kind name: (total ms, launches)} since the last read."""
+    p = moa_profile()
+    s = lib().moa_profile_read(ctypes.byref(p))
+    if s != MOA_OK:
+        raise MoaError(s, "moa_profile_read")
+    return {KERNEL_KIND_NAMES[k]: (float(p.ms[k]), int(p.launches[k])) for k in range(MOA_KERNEL_KINDS)}

@@ -18,6 +18,15 @@ struct Problem {
 // Host-side launch counter (moa_launch_count).
 void count_launch(int k = 1);
 
+// Brackets one kernel launch with an event pair when profiling is enabled
+// (moa_profile_enable); also counts the launch.
+struct LaunchScope {
+    LaunchScope(int kind, cudaStream_t st);
+    ~LaunchScope();
+    int slot;
+    cudaStream_t st;
+};
+
 // Device address of the status word kernels write when a bounded wait expires.
 unsigned int *device_status_ptr();
 

@@ -3,11 +3,42 @@
 #include "common.cuh"
 #include <atomic>
 #include <mutex>
+#include <vector>
 
 namespace moa {
 
 static std::atomic<uint64_t> g_launches{0};
 void count_launch(int k) { g_launches.fetch_add((uint64_t)k, std::memory_order_relaxed); }
+
+// ---- optional per-kernel event timing -------------------------------------------------
+namespace {
+struct ProfRecord { cudaEvent_t a, b; int kind; };
+bool g_prof_on = false;
+std::vector<ProfRecord> g_prof_records;   // in use
+std::vector<ProfRecord> g_prof_pool;      // created, idle
+}  // namespace
+
+LaunchScope::LaunchScope(int kind, cudaStream_t s) : slot(-1), st(s)
+{
+    count_launch();
+    if (!g_prof_on || g_prof_records.size() >= MOA_PROFILE_MAX_RECORDS) return;
+    ProfRecord r;
+    if (!g_prof_pool.empty()) {
+        r = g_prof_pool.back();
+        g_prof_pool.pop_back();
+    } else if (cudaEventCreate(&r.a) != cudaSuccess || cudaEventCreate(&r.b) != cudaSuccess) {
+        return;
+    }
+    r.kind = kind;
+    if (cudaEventRecord(r.a, st) != cudaSuccess) { g_prof_pool.push_back(r); return; }
+    g_prof_records.push_back(r);
+    slot = (int)g_prof_records.size() - 1;
+}
+
+LaunchScope::~LaunchScope()
+{
+    if (slot >= 0) cudaEventRecord(g_prof_records[slot].b, st);
+}
 
 // One status word per device image of this library; kernels with bounded waits set
 // it to a non-zero code when a wait expires.
@@ -196,6 +227,31 @@ moa_status moa_last_device_status(void *stream)
         return MOA_ERR_TIMEOUT;
     }
     return MOA_OK;
+}
+
+moa_status moa_profile_enable(int on)
+{
+    g_prof_on = on != 0;
+    return MOA_OK;
+}
+
+moa_status moa_profile_read(moa_profile *out)
+{
+    if (!out) return MOA_ERR_INVALID_ARG;
+    for (int k = 0; k < MOA_KERNEL_KINDS; ++k) { out->ms[k] = 0.f; out->launches[k] = 0; }
+    moa_status rc = MOA_OK;
+    for (auto &r : g_prof_records) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(r.b) != cudaSuccess || cudaEventElapsedTime(&ms, r.a, r.b) != cudaSuccess) {
+            rc = MOA_ERR_CUDA;
+        } else if (r.kind >= 0 && r.kind < MOA_KERNEL_KINDS) {
+            out->ms[r.kind] += ms;
+            out->launches[r.kind] += 1;
+        }
+        g_prof_pool.push_back(r);
+    }
+    g_prof_records.clear();
+    return rc;
 }
 
 uint64_t moa_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

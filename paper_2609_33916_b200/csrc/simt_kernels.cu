@@ -398,9 +398,9 @@ cudaError_t fwd_t(const Problem &p, const void *Q, const void *K, const void *V,
     const int nqt = (p.n + BM - 1) / BM;
     cudaError_t e = set_smem(simt_fwd_kernel<T, D>, fwd_smem(D));
     if (e != cudaSuccess) return e;
+    LaunchScope scope(MOA_KERNEL_FWD, st);
     simt_fwd_kernel<T, D><<<(unsigned)(nqt * p.BH()), NTHREADS, fwd_smem(D), st>>>(
         (const T *)Q, (const T *)K, (const T *)V, (T *)O, L, p.n, p.causal, p.scale, nqt);
-    count_launch();
     return cudaGetLastError();
 }
 
@@ -411,10 +411,10 @@ cudaError_t bwd_kv_t(const Problem &p, const void *Q, const void *K, const void 
     const int nkt = (p.n + BN - 1) / BN;
     cudaError_t e = set_smem(simt_bwd_kv_kernel<T, D>, bwd_smem(D));
     if (e != cudaSuccess) return e;
+    LaunchScope scope(MOA_KERNEL_BWD_KV, st);
     simt_bwd_kv_kernel<T, D><<<(unsigned)(nkt * p.BH()), NTHREADS, bwd_smem(D), st>>>(
         (const T *)Q, (const T *)K, (const T *)V, (const T *)dO, L, Dv, (T *)dK, (T *)dV, dQacc,
         p.n, p.causal, p.scale, nkt);
-    count_launch();
     return cudaGetLastError();
 }
 
@@ -425,9 +425,9 @@ cudaError_t bwd_dq_t(const Problem &p, const void *Q, const void *K, const void 
     const int nqt = (p.n + BM - 1) / BM;
     cudaError_t e = set_smem(simt_bwd_dq_kernel<T, D>, bwd_smem(D));
     if (e != cudaSuccess) return e;
+    LaunchScope scope(MOA_KERNEL_BWD_DQ, st);
     simt_bwd_dq_kernel<T, D><<<(unsigned)(nqt * p.BH()), NTHREADS, bwd_smem(D), st>>>(
         (const T *)Q, (const T *)K, (const T *)V, (const T *)dO, L, Dv, (T *)dQ, p.n, p.causal, p.scale, nqt);
-    count_launch();
     return cudaGetLastError();
 }
 
@@ -469,12 +469,12 @@ cudaError_t row_dot(const Problem &p, int dtype, const void *dO, const void *O, 
     const size_t rows = (size_t)p.BH() * p.n;
     const int wpb = 8;
     const unsigned grid = (unsigned)((rows + wpb - 1) / wpb);
+    LaunchScope scope(MOA_KERNEL_PREPROCESS, st);
     if (dtype == MOA_F32)
         row_dot_kernel<float><<<grid, wpb * 32, 0, st>>>((const float *)dO, (const float *)O, Dv, rows, p.d);
     else
         row_dot_kernel<__nv_bfloat16><<<grid, wpb * 32, 0, st>>>((const __nv_bfloat16 *)dO,
                                                                  (const __nv_bfloat16 *)O, Dv, rows, p.d);
-    count_launch();
     return cudaGetLastError();
 }
 
@@ -482,8 +482,8 @@ cudaError_t convert_f32_to_bf16(const float *src, void *dst, size_t count, cudaS
 {
     const size_t quads = (count + 3) / 4;
     const unsigned grid = (unsigned)((quads + 255) / 256);
+    LaunchScope scope(MOA_KERNEL_CONVERT, st);
     convert_kernel<<<grid, 256, 0, st>>>(src, (__nv_bfloat16 *)dst, count);
-    count_launch();
     return cudaGetLastError();
 }
 
