@@ -38,6 +38,9 @@ template <typename T> __device__ __forceinline__ T from_float(float v);
 template <> __device__ __forceinline__ float from_float<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
+// ---- tensor-core path (tc_fwd.cu), bf16 only ---------------------------------------------
+cudaError_t tc_fwd(const Problem &p, const void *Q, const void *K, const void *V, void *O, float *L, cudaStream_t st);
+
 // ---- SIMT fp32 path (simt_kernels.cu) -------------------------------------------------
 // dtype: MOA_BF16 or MOA_F32 storage; arithmetic is fp32 FMA throughout.
 cudaError_t simt_fwd(const Problem &p, int dtype, const void *Q, const void *K, const void *V,

@@ -99,7 +99,6 @@ moa_status check_desc(const moa_attn_desc *d)
     const long long tiles = ((long long)d->n + 63) / 64;
     if (tiles * d->B * d->H >= (1LL << 31)) return MOA_ERR_UNSUPPORTED;
     if (d->path == MOA_PATH_TC && d->dtype != MOA_BF16) return MOA_ERR_UNSUPPORTED;
-    if (d->path == MOA_PATH_TC) return MOA_ERR_UNSUPPORTED;   // tensor-core kernels not built yet
     if (d->materialize) return MOA_ERR_UNSUPPORTED;           // comparison variant not built yet
     if (d->dq_mode == MOA_DQ_BULK_REDUCE) return MOA_ERR_UNSUPPORTED;
     return MOA_OK;
@@ -126,7 +125,10 @@ Problem to_problem(const moa_attn_desc *d) { return Problem{d->B, d->H, d->n, d-
 moa_status run_fwd(const moa_attn_desc *d, const void *Q, const void *K, const void *V, void *O, float *L,
                    cudaStream_t st)
 {
-    return simt_fwd(to_problem(d), d->dtype, Q, K, V, O, L, st) == cudaSuccess ? MOA_OK : MOA_ERR_CUDA;
+    const bool tc = d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT;
+    const cudaError_t e = tc ? tc_fwd(to_problem(d), Q, K, V, O, L, st)
+                             : simt_fwd(to_problem(d), d->dtype, Q, K, V, O, L, st);
+    return e == cudaSuccess ? MOA_OK : MOA_ERR_CUDA;
 }
 
 moa_status run_bwd(const moa_attn_desc *d, const void *Q, const void *K, const void *V, const void *O,

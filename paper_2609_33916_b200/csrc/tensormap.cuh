@@ -1,0 +1,16 @@
+// Host-side construction of TMA descriptors for [BH, n, d] tensors.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda.h>
+#include <stdint.h>
+
+namespace moa {
+
+// Tiled map over a contiguous [heads, rows, cols] tensor (cols fastest) with boxes of
+// [1, box_rows, box_cols]; 128-byte swizzle when box_cols * elem_bytes == 128, none
+// otherwise.  Out-of-range rows read as zero and are clipped on store/reduce.
+// Returns false if the driver entry point is unavailable or the encode fails.
+bool make_tensor_map_3d(CUtensorMap *map, const void *base, CUtensorMapDataType dt, int elem_bytes,
+                        uint64_t heads, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_cols);
+
+}  // namespace moa

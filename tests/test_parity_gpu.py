@@ -70,13 +70,36 @@ BF16_CASES = [
 
 @pytest.mark.parametrize("B,Hh,n,d,causal", BF16_CASES)
 @pytest.mark.parametrize("dq_mode", [1, 3])
-@pytest.mark.parametrize("path", [1])
+@pytest.mark.parametrize("path", [1, 2])
 def test_bf16_shapes(H, B, Hh, n, d, causal, dq_mode, path):
     inp = mi.make_inputs(B, Hh, n, d, seed=200 + n, dtype="bf16")
     scale = 1.0 / math.sqrt(d)
     ref = _oracle(inp, "bf16", causal, scale)
     got = H.run_library(inp, "bf16", causal, scale, dq_mode=dq_mode, path=path)
     H.assert_close(got, ref, H.TOL_BF16, tag=f"n{n} d{d} path{path}")
+    assert mi.rel_err(got["L"], ref["L"]) <= 1e-3
+
+
+@pytest.mark.parametrize("n", [1, 64, 127, 129, 255, 640, 1111])
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("causal", [False, True])
+def test_tc_forward_ragged(H, n, d, causal):
+    inp = mi.make_inputs(1, 3, n, d, seed=300 + n, dtype="bf16")
+    scale = 1.0 / math.sqrt(d)
+    ref = _oracle(inp, "bf16", causal, scale)
+    got = H.run_library(inp, "bf16", causal, scale, op="fwd", path=2)
+    H.assert_close(got, ref, H.TOL_BF16, keys=("O",), tag=f"fwd n{n} d{d}")
+    assert mi.rel_err(got["L"], ref["L"]) <= 1e-3
+
+
+def test_tc_forward_large_scores(H):
+    """Q scaled by 30 makes the running max jump between tiles: exercises the lazy
+    rescale of the O accumulator."""
+    inp = mi.make_inputs(1, 2, 1024, 128, seed=9, dtype="bf16", gain=30.0)
+    ref = _oracle(inp, "bf16", True, 0.09)
+    got = H.run_library(inp, "bf16", True, 0.09, op="fwd", path=2)
+    assert np.all(np.isfinite(got["O"])) and np.all(np.isfinite(got["L"]))
+    H.assert_close(got, ref, H.TOL_BF16, keys=("O",), tag="gain30")
     assert mi.rel_err(got["L"], ref["L"]) <= 1e-3
 
 
