@@ -41,6 +41,13 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(f
 // ---- tensor-core path (tc_fwd.cu), bf16 only ---------------------------------------------
 cudaError_t tc_fwd(const Problem &p, const void *Q, const void *K, const void *V, void *O, float *L, cudaStream_t st);
 
+// Lp = L*log2(e) and Dp = rowsum(dO o O), each padded per head to a multiple of 128 rows
+cudaError_t tc_bwd_preprocess(const Problem &p, const void *dO, const void *O, const float *L, float *Lp, float *Dp,
+                              cudaStream_t st);
+// dK, dV; dQ contributions red-added into dQacc (fp32 [B,H,n,d], pre-zeroed)
+cudaError_t tc_bwd_kv(const Problem &p, const void *Q, const void *K, const void *V, const void *dO,
+                      const float *Lp, const float *Dp, void *dK, void *dV, float *dQacc, cudaStream_t st);
+
 // ---- SIMT fp32 path (simt_kernels.cu) -------------------------------------------------
 // dtype: MOA_BF16 or MOA_F32 storage; arithmetic is fp32 FMA throughout.
 cudaError_t simt_fwd(const Problem &p, int dtype, const void *Q, const void *K, const void *V,

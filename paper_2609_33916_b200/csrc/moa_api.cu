@@ -101,22 +101,36 @@ moa_status check_desc(const moa_attn_desc *d)
     if (d->path == MOA_PATH_TC && d->dtype != MOA_BF16) return MOA_ERR_UNSUPPORTED;
     if (d->materialize) return MOA_ERR_UNSUPPORTED;           // comparison variant not built yet
     if (d->dq_mode == MOA_DQ_BULK_REDUCE) return MOA_ERR_UNSUPPORTED;
+    if (d->path == MOA_PATH_TC && d->dq_mode == MOA_DQ_SEPARATE_PASS) return MOA_ERR_UNSUPPORTED;
     return MOA_OK;
 }
 
 int resolved_dq_mode(const moa_attn_desc *d) { return d->dq_mode == MOA_DQ_AUTO ? MOA_DQ_RED : d->dq_mode; }
 
+bool use_tc_fwd(const moa_attn_desc *d) { return d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT; }
+bool use_tc_bwd(const moa_attn_desc *d)
+{
+    return d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && resolved_dq_mode(d) == MOA_DQ_RED;
+}
+
+// Workspace of the backward: [ D | Lp (tensor-core path only) | dQacc (bf16 with an atomic mode) ]
 struct BwdWorkspace {
-    size_t d_bytes, dqacc_bytes, total;
+    size_t d_bytes, lp_bytes, dqacc_bytes, total;
 };
 BwdWorkspace bwd_workspace(const moa_attn_desc *d)
 {
     BwdWorkspace w{};
     const size_t rows = (size_t)d->B * d->H * d->n;
-    w.d_bytes = align_up(rows * sizeof(float));
+    if (use_tc_bwd(d)) {
+        const size_t prows = (size_t)d->B * d->H * (((size_t)d->n + 127) / 128 * 128);
+        w.d_bytes = align_up(prows * sizeof(float));
+        w.lp_bytes = align_up(prows * sizeof(float));
+    } else {
+        w.d_bytes = align_up(rows * sizeof(float));
+    }
     const bool need_acc = d->dtype == MOA_BF16 && resolved_dq_mode(d) != MOA_DQ_SEPARATE_PASS;
     w.dqacc_bytes = need_acc ? align_up(rows * d->d * sizeof(float)) : 0;
-    w.total = w.d_bytes + w.dqacc_bytes;
+    w.total = w.d_bytes + w.lp_bytes + w.dqacc_bytes;
     return w;
 }
 
@@ -125,8 +139,7 @@ Problem to_problem(const moa_attn_desc *d) { return Problem{d->B, d->H, d->n, d-
 moa_status run_fwd(const moa_attn_desc *d, const void *Q, const void *K, const void *V, void *O, float *L,
                    cudaStream_t st)
 {
-    const bool tc = d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT;
-    const cudaError_t e = tc ? tc_fwd(to_problem(d), Q, K, V, O, L, st)
+    const cudaError_t e = use_tc_fwd(d) ? tc_fwd(to_problem(d), Q, K, V, O, L, st)
                              : simt_fwd(to_problem(d), d->dtype, Q, K, V, O, L, st);
     return e == cudaSuccess ? MOA_OK : MOA_ERR_CUDA;
 }
@@ -137,10 +150,18 @@ moa_status run_bwd(const moa_attn_desc *d, const void *Q, const void *K, const v
     const Problem p = to_problem(d);
     const BwdWorkspace w = bwd_workspace(d);
     float *Dv = (float *)ws;
-    float *dQacc = w.dqacc_bytes ? (float *)((char *)ws + w.d_bytes) : nullptr;
+    float *Lp = (float *)((char *)ws + w.d_bytes);
+    float *dQacc = w.dqacc_bytes ? (float *)((char *)ws + w.d_bytes + w.lp_bytes) : nullptr;
     const size_t elems = (size_t)p.BH() * p.n * p.d;
     const int mode = resolved_dq_mode(d);
 #define MOA_TRY(x) do { if ((x) != cudaSuccess) return MOA_ERR_CUDA; } while (0)
+    if (use_tc_bwd(d)) {
+        MOA_TRY(tc_bwd_preprocess(p, dO, O, L, Lp, Dv, st));
+        MOA_TRY(cudaMemsetAsync(dQacc, 0, elems * sizeof(float), st));
+        MOA_TRY(tc_bwd_kv(p, Q, K, V, dO, Lp, Dv, dK, dV, dQacc, st));
+        MOA_TRY(convert_f32_to_bf16(dQacc, dQ, elems, st));
+        return MOA_OK;
+    }
     MOA_TRY(row_dot(p, d->dtype, dO, O, Dv, st));
     if (mode == MOA_DQ_SEPARATE_PASS) {
         MOA_TRY(simt_bwd_kv(p, d->dtype, Q, K, V, dO, L, Dv, dK, dV, nullptr, st));

@@ -69,8 +69,7 @@ BF16_CASES = [
 
 
 @pytest.mark.parametrize("B,Hh,n,d,causal", BF16_CASES)
-@pytest.mark.parametrize("dq_mode", [1, 3])
-@pytest.mark.parametrize("path", [1, 2])
+@pytest.mark.parametrize("path,dq_mode", [(1, 1), (1, 3), (2, 1), (0, 3)])
 def test_bf16_shapes(H, B, Hh, n, d, causal, dq_mode, path):
     inp = mi.make_inputs(B, Hh, n, d, seed=200 + n, dtype="bf16")
     scale = 1.0 / math.sqrt(d)
