@@ -53,7 +53,9 @@ typedef enum {
     MOA_ERR_WORKSPACE = 3,   /* ws == NULL or ws_bytes < moa_attn_workspace_bytes(...)         */
     MOA_ERR_ARCH = 4,        /* current device is not sm_100                                   */
     MOA_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed (launch, descriptor encode)  */
-    MOA_ERR_TIMEOUT = 6      /* a bounded device-side wait expired (reported by moa_last_device_status) */
+    MOA_ERR_TIMEOUT = 6,     /* a bounded device-side wait expired (reported by moa_last_device_status) */
+    MOA_ERR_SCRATCH_LIMIT = 7 /* moa_attn_bwd_static_scratch: the problem needs more scratch than
+                                 MOA_STATIC_SCRATCH_BYTES                                        */
 } moa_status;
 
 typedef enum { MOA_BF16 = 0, MOA_F32 = 1 } moa_dtype;
@@ -111,6 +113,34 @@ moa_status moa_attn_bwd(const moa_attn_desc *desc,
                         const void *O, const float *L, const void *dO,
                         void *dQ, void *dK, void *dV,
                         void *ws, size_t ws_bytes, void *stream);
+
+/* Backward for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: its benchmarks allocate everything up front on the host.)
+ *
+ * Some callers of this library have no way to hand it a workspace: code running
+ * inside a memory pool whose allocator they do not control, plugins invoked with a
+ * fixed argument list of inputs and outputs, or hosts where cudaMalloc is forbidden
+ * after start-up.  For them this entry point computes exactly what moa_attn_bwd
+ * computes, same arguments minus ws/ws_bytes, but takes its scratch (D, the padded
+ * logsumexp and the fp32 dQ accumulator) from an array of MOA_STATIC_SCRATCH_BYTES
+ * bytes that is part of the library image itself.  Every GPU that loads the library
+ * carries that array until the process exits, which is why it is kept modest.
+ *
+ *  - It calls no cudaMalloc, cudaFree or any other allocating routine.
+ *  - If moa_attn_workspace_bytes(desc, MOA_OP_BWD) exceeds MOA_STATIC_SCRATCH_BYTES the
+ *    call returns MOA_ERR_SCRATCH_LIMIT and enqueues nothing; use moa_attn_bwd then.
+ *  - The first call on each device looks up the array's device address (a one-time,
+ *    per-device set-up done with that device current).  Make that first call before
+ *    any stream capture begins.
+ *  - All calls on a device share the one array, and it keeps whatever the previous
+ *    call left in it; the parts that must start from zero are cleared on the stream at
+ *    the start of every call.  Two calls that can overlap on the GPU (different
+ *    streams, or different host threads) therefore race on it: serialise them. */
+#define MOA_STATIC_SCRATCH_BYTES (16u << 20)
+moa_status moa_attn_bwd_static_scratch(const moa_attn_desc *desc,
+                                       const void *Q, const void *K, const void *V,
+                                       const void *O, const float *L, const void *dO,
+                                       void *dQ, void *dK, void *dV, void *stream);
 
 /* Fused forward+backward (the paper's Algorithm 2 as one library call): several
  * launches on one stream, no n x n array in memory.  Reads Q,K,V,dO; writes O, L,

@@ -14,6 +14,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libmoa_attn.so")
 
 MOA_OK, MOA_ERR_INVALID_ARG, MOA_ERR_UNSUPPORTED, MOA_ERR_WORKSPACE, MOA_ERR_ARCH, MOA_ERR_CUDA, MOA_ERR_TIMEOUT = range(7)
+MOA_ERR_SCRATCH_LIMIT = 7
+MOA_STATIC_SCRATCH_BYTES = 16 << 20
 MOA_BF16, MOA_F32 = 0, 1
 MOA_DQ_AUTO, MOA_DQ_RED, MOA_DQ_BULK_REDUCE, MOA_DQ_SEPARATE_PASS = 0, 1, 2, 3
 MOA_PATH_AUTO, MOA_PATH_SIMT, MOA_PATH_TC = 0, 1, 2
@@ -23,7 +25,7 @@ MOA_OP_FWD, MOA_OP_BWD, MOA_OP_FUSED = 0, 1, 2
 EXPORTS = (
     "moa_attn_workspace_bytes", "moa_attn_fwd", "moa_attn_bwd", "moa_attn_fused_fwd_bwd",
     "moa_last_device_status", "moa_launch_count", "moa_status_string", "moa_version",
-    "moa_profile_enable", "moa_profile_read",
+    "moa_profile_enable", "moa_profile_read", "moa_attn_bwd_static_scratch",
 )
 
 
@@ -65,6 +67,8 @@ def lib() -> ctypes.CDLL:
         L.moa_attn_fwd.argtypes = [dp] + [vp] * 5 + [vp, sz, vp]
         L.moa_attn_bwd.restype = ctypes.c_int
         L.moa_attn_bwd.argtypes = [dp] + [vp] * 9 + [vp, sz, vp]
+        L.moa_attn_bwd_static_scratch.restype = ctypes.c_int
+        L.moa_attn_bwd_static_scratch.argtypes = [dp] + [vp] * 9 + [vp]
         L.moa_attn_fused_fwd_bwd.restype = ctypes.c_int
         L.moa_attn_fused_fwd_bwd.argtypes = [dp] + [vp] * 9 + [vp, sz, vp]
         L.moa_last_device_status.restype = ctypes.c_int
@@ -142,6 +146,17 @@ def moa_attn_bwd(desc, Q, K, V, O, L, dO, dQ, dK, dV, ws=None, stream=None, ws_b
                            _nbytes(ws) if ws_bytes is None else ws_bytes, _stream(stream))
     if check and s != MOA_OK:
         raise MoaError(s, "moa_attn_bwd")
+    return s
+
+
+def moa_attn_bwd_static_scratch(desc, Q, K, V, O, L, dO, dQ, dK, dV, stream=None, check=True) -> int:
+    """moa_attn_bwd for callers that cannot allocate: no workspace argument, the library's
+    built-in scratch array (MOA_STATIC_SCRATCH_BYTES) is used.  Calls sharing a device must
+    not overlap on the GPU; make the first call on a device outside any stream capture."""
+    s = lib().moa_attn_bwd_static_scratch(ctypes.byref(desc), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(L),
+                                          _ptr(dO), _ptr(dQ), _ptr(dK), _ptr(dV), _stream(stream))
+    if check and s != MOA_OK:
+        raise MoaError(s, "moa_attn_bwd_static_scratch")
     return s
 
 

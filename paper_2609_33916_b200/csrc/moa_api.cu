@@ -176,6 +176,28 @@ moa_status run_bwd(const moa_attn_desc *d, const void *Q, const void *K, const v
     return MOA_OK;
 }
 
+// Built-in scratch of moa_attn_bwd_static_scratch.  In host code this name is only a
+// handle for the symbol, not a device address: the address each device gives it is
+// looked up once per device below and that pointer is what the kernels receive.
+static __device__ __align__(256) unsigned char g_static_scratch[MOA_STATIC_SCRATCH_BYTES];
+
+// Device address of g_static_scratch on the current device (nullptr on failure).
+void *static_scratch_ptr()
+{
+    constexpr int kMaxDev = 64;
+    static void *cache[kMaxDev] = {};
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return nullptr;
+    std::lock_guard<std::mutex> lk(mu);
+    if (!cache[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess) return nullptr;
+        cache[dev] = p;
+    }
+    return cache[dev];
+}
+
 }  // namespace
 }  // namespace moa
 
@@ -218,6 +240,24 @@ moa_status moa_attn_bwd(const moa_attn_desc *desc, const void *Q, const void *K,
     if (!aligned16(ws)) return MOA_ERR_INVALID_ARG;
     if ((s = check_arch()) != MOA_OK) return s;
     return run_bwd(desc, Q, K, V, O, L, dO, dQ, dK, dV, ws, (cudaStream_t)stream);
+}
+
+moa_status moa_attn_bwd_static_scratch(const moa_attn_desc *desc, const void *Q, const void *K, const void *V,
+                                       const void *O, const float *L, const void *dO,
+                                       void *dQ, void *dK, void *dV, void *stream)
+{
+    moa_status s = check_desc(desc);
+    if (s != MOA_OK) return s;
+    if (!Q || !K || !V || !O || !L || !dO || !dQ || !dK || !dV) return MOA_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(L) || !aligned16(dO) ||
+        !aligned16(dQ) || !aligned16(dK) || !aligned16(dV))
+        return MOA_ERR_INVALID_ARG;
+    if (bwd_workspace(desc).total > (size_t)MOA_STATIC_SCRATCH_BYTES) return MOA_ERR_SCRATCH_LIMIT;
+    if ((s = check_arch()) != MOA_OK) return s;
+    void *scratch = static_scratch_ptr();   // first call on this device resolves the symbol's address
+    if (!scratch) return MOA_ERR_CUDA;
+    // run_bwd clears the dQ accumulator on the stream and overwrites D / Lp before use
+    return run_bwd(desc, Q, K, V, O, L, dO, dQ, dK, dV, scratch, (cudaStream_t)stream);
 }
 
 moa_status moa_attn_fused_fwd_bwd(const moa_attn_desc *desc, const void *Q, const void *K, const void *V,
@@ -289,6 +329,7 @@ const char *moa_status_string(moa_status s)
         case MOA_ERR_ARCH: return "device is not sm_100";
         case MOA_ERR_CUDA: return "CUDA call failed";
         case MOA_ERR_TIMEOUT: return "bounded device wait expired";
+        case MOA_ERR_SCRATCH_LIMIT: return "problem needs more scratch than the built-in static array holds";
     }
     return "unknown status";
 }
