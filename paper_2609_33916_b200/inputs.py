@@ -49,6 +49,8 @@ CONFIGS = {
     "c3_causal_mid": Workload("c3_causal_mid", 2, 16, 4096, 128, True, "bf16", 2),
     "c4_long": Workload("c4_long", 1, 16, 16384, 128, False, "bf16", 3),
 }
+# a small non-causal case for profiler captures: larger than L2 in total, short kernels
+CONFIGS["prof_h8_n8192"] = Workload("prof_h8_n8192", 1, 8, 8192, 128, False, "bf16", 5)
 C5_SIZES = (512, 1024, 2048, 4096, 8192, 16384, 32768)
 for _n in C5_SIZES:
     CONFIGS[f"c5_causal_n{_n}"] = Workload(f"c5_causal_n{_n}", 1, 32, _n, 128, True, "bf16", 4)
