@@ -44,7 +44,8 @@ cudaError_t tc_fwd(const Problem &p, const void *Q, const void *K, const void *V
 // Lp = L*log2(e) and Dp = rowsum(dO o O), each padded per head to a multiple of 128 rows
 cudaError_t tc_bwd_preprocess(const Problem &p, const void *dO, const void *O, const float *L, float *Lp, float *Dp,
                               cudaStream_t st);
-// dK, dV; dQ contributions red-added into dQacc (fp32 [B,H,n,d], pre-zeroed)
+// dK, dV; UNSCALED dQ contributions (dS K, without the factor scale) red-added into dQacc
+// (fp32 [B,H,n,d], pre-zeroed)
 cudaError_t tc_bwd_kv(const Problem &p, const void *Q, const void *K, const void *V, const void *dO,
                       const float *Lp, const float *Dp, void *dK, void *dV, float *dQacc, cudaStream_t st);
 
@@ -62,7 +63,7 @@ cudaError_t simt_bwd_kv(const Problem &p, int dtype, const void *Q, const void *
 // atomic-free query-parallel dQ pass
 cudaError_t simt_bwd_dq(const Problem &p, int dtype, const void *Q, const void *K, const void *V,
                         const void *dO, const float *L, const float *Dv, void *dQ, cudaStream_t st);
-// dst[i] = (bf16) src[i]
-cudaError_t convert_f32_to_bf16(const float *src, void *dst, size_t count, cudaStream_t st);
+// dst[i] = (bf16)(mul * src[i])
+cudaError_t convert_f32_to_bf16(const float *src, void *dst, size_t count, float mul, cudaStream_t st);
 
 }  // namespace moa

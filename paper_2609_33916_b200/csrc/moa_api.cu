@@ -159,7 +159,7 @@ moa_status run_bwd(const moa_attn_desc *d, const void *Q, const void *K, const v
         MOA_TRY(tc_bwd_preprocess(p, dO, O, L, Lp, Dv, st));
         MOA_TRY(cudaMemsetAsync(dQacc, 0, elems * sizeof(float), st));
         MOA_TRY(tc_bwd_kv(p, Q, K, V, dO, Lp, Dv, dK, dV, dQacc, st));
-        MOA_TRY(convert_f32_to_bf16(dQacc, dQ, elems, st));
+        MOA_TRY(convert_f32_to_bf16(dQacc, dQ, elems, p.scale, st));
         return MOA_OK;
     }
     MOA_TRY(row_dot(p, d->dtype, dO, O, Dv, st));
@@ -170,7 +170,7 @@ moa_status run_bwd(const moa_attn_desc *d, const void *Q, const void *K, const v
         float *acc = d->dtype == MOA_F32 ? (float *)dQ : dQacc;   // fp32 output accumulates in place
         MOA_TRY(cudaMemsetAsync(acc, 0, elems * sizeof(float), st));
         MOA_TRY(simt_bwd_kv(p, d->dtype, Q, K, V, dO, L, Dv, dK, dV, acc, st));
-        if (d->dtype == MOA_BF16) MOA_TRY(convert_f32_to_bf16(dQacc, dQ, elems, st));
+        if (d->dtype == MOA_BF16) MOA_TRY(convert_f32_to_bf16(dQacc, dQ, elems, 1.f, st));
     }
 #undef MOA_TRY
     return MOA_OK;

@@ -368,18 +368,19 @@ simt_bwd_dq_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__
     }
 }
 
-__global__ void convert_kernel(const float *__restrict__ src, __nv_bfloat16 *__restrict__ dst, size_t count)
+__global__ void convert_kernel(const float *__restrict__ src, __nv_bfloat16 *__restrict__ dst, size_t count,
+                               float mul)
 {
     size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
     if (i + 3 < count) {
         const float4 v = *reinterpret_cast<const float4 *>(src + i);
-        __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+        __nv_bfloat162 a = __floats2bfloat162_rn(v.x * mul, v.y * mul), b = __floats2bfloat162_rn(v.z * mul, v.w * mul);
         uint2 u;
         u.x = *reinterpret_cast<uint32_t *>(&a);
         u.y = *reinterpret_cast<uint32_t *>(&b);
         *reinterpret_cast<uint2 *>(dst + i) = u;
     } else {
-        for (; i < count; ++i) dst[i] = __float2bfloat16_rn(src[i]);
+        for (; i < count; ++i) dst[i] = __float2bfloat16_rn(src[i] * mul);
     }
 }
 
@@ -478,12 +479,12 @@ cudaError_t row_dot(const Problem &p, int dtype, const void *dO, const void *O, 
     return cudaGetLastError();
 }
 
-cudaError_t convert_f32_to_bf16(const float *src, void *dst, size_t count, cudaStream_t st)
+cudaError_t convert_f32_to_bf16(const float *src, void *dst, size_t count, float mul, cudaStream_t st)
 {
     const size_t quads = (count + 3) / 4;
     const unsigned grid = (unsigned)((quads + 255) / 256);
     LaunchScope scope(MOA_KERNEL_CONVERT, st);
-    convert_kernel<<<grid, 256, 0, st>>>(src, (__nv_bfloat16 *)dst, count);
+    convert_kernel<<<grid, 256, 0, st>>>(src, (__nv_bfloat16 *)dst, count, mul);
     return cudaGetLastError();
 }
 

@@ -7,16 +7,21 @@
 //     S^T  = K Q_i^T                 (SS-UMMA, both operands K-major)
 //     dP^T = V dO_i^T                (SS-UMMA)
 //     P^T  = exp2(S^T scale log2e - L_i log2e)         (registers; L from the forward)
-//     dS^T = scale * P^T o (dP^T - D_i)                (D = rowsum(dO o O))
+//     dS^T = P^T o (dP^T - D_i)                        (D = rowsum(dO o O); the factor
+//                                                       `scale` of dK and dQ is applied at the end)
 //     dV  += P^T dO_i                (TS-UMMA: P^T bf16 in TMEM, dO_i MN-major in smem)
 //     dK  += dS^T Q_i                (TS-UMMA: dS^T bf16 in TMEM, Q_i MN-major in smem)
 //     dQ_i = dS K                    (SS-UMMA: dS^T tile in smem as MN-major A, K MN-major)
 // dQ_i is one key tile's contribution; it is added into an fp32 [B,H,n,d] accumulator
 // with vector red.global.add (the contended step the dq_mode knob is about).
 //
-// Roles (320 threads): warps 0-7 elementwise work (thread = TMEM lane, the two
-// warpgroups split the columns), warp 8 TMA producer (K,V once; Q_i, dO_i, L_i, D_i in a
-// two-stage ring), warp 9 UMMA issuer and TMEM owner.
+// Roles (512 threads; registers are re-split per warpgroup with setmaxnreg: 152 / 152 / 56): warps 0-7 elementwise work (thread = TMEM lane = key, the two
+// warpgroups split the query columns), warps 8-11 read each finished dQ tile out of TMEM
+// and issue the reds, warp 12 TMA producer (K,V once; Q_i with L_i, D_i and dO_i in
+// two-slot rings with separate release points), warp 13 UMMA issuer and TMEM owner.
+// UMMA issue order per query tile: dP(i), dV(i), S(i+1), dK(i), dQ(i), so that the
+// exp2 work of tile i+1 overlaps the dK/dQ UMMAs of tile i and the dS work of tile i
+// overlaps dV(i) and S(i+1).
 //
 // TMEM columns (512): S^T [0,128), dP^T [128,256), dV [256,256+D), dK [256+D,256+2D);
 // P^T / dS^T (bf16) overwrite the front of their fp32 source columns; for D = 128 the dQ
@@ -27,13 +32,15 @@
 #include "common.cuh"
 #include "ptx.cuh"
 #include "tensormap.cuh"
+#include <cstdlib>
 
 namespace moa {
 namespace {
 
 using namespace ptx;
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 512;   // warps 0-7 elementwise, 8-11 dQ reduce, 12 TMA, 13 UMMA, 14-15 idle
+constexpr int kReduceWarp0 = 8, kLoadWarp = 12, kMmaWarp = 13;
 constexpr int kTmemCols = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -47,6 +54,11 @@ __device__ __forceinline__ void bulk_load_1d(void *dst, const void *src, uint32_
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(smem_u32(bar))
                  : "memory");
+}
+
+__device__ __forceinline__ void red_add_f32(float *addr, float a)
+{
+    asm volatile("red.global.add.f32 [%0], %1;" ::"l"(addr), "f"(a) : "memory");
 }
 
 __device__ __forceinline__ void red_add_v4(float *addr, float a, float b, float c, float d)
@@ -94,13 +106,19 @@ struct BwdSmem {
     static constexpr int kdS = 128 * 128 * 2;        // dS^T tile, [128 keys][128 queries] bf16
     static constexpr int offK = 0;
     static constexpr int offV = offK + kTile;
-    static constexpr int offQ = offV + kTile;        // 2 stages
-    static constexpr int offdO = offQ + 2 * kTile;   // 2 stages
+    static constexpr int offQ = offV + kTile;        // 2 slots
+    static constexpr int offdO = offQ + 2 * kTile;   // 2 slots
     static constexpr int offdS = offdO + 2 * kTile;
-    static constexpr int offL = offdS + kdS;         // 2 x 128 floats
-    static constexpr int offD = offL + 2 * 512;      // 2 x 128 floats
-    static constexpr int offBar = offD + 2 * 512;    // 8 mbarriers + tmem base + abort flag
-    static constexpr int kTotal = offBar + 128;
+    static constexpr int offL = offdS + kdS;         // 2 x 128 floats, travels with the Q slot
+    static constexpr int offD = offL + 2 * 512;      // 2 x 128 floats, travels with the Q slot
+    static constexpr int offBar = offD + 2 * 512;    // mbarriers + tmem base + abort flag
+    static constexpr int kTotal = offBar + 192;
+};
+
+// Barrier slots inside the shared-memory barrier block
+enum {
+    B_KV = 0, B_QFULL = 1 /*2*/, B_QEMPTY = 3 /*2*/, B_DOFULL = 5 /*2*/, B_DOEMPTY = 7 /*2*/,
+    B_S = 9, B_P = 10, B_DP = 11, B_DS = 12, B_DQ = 13, B_DQR = 14, B_COUNT = 15
 };
 
 template <int D>
@@ -109,21 +127,24 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
               const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapdO,
               const float *__restrict__ Lp, const float *__restrict__ Dp,
               __nv_bfloat16 *__restrict__ dK, __nv_bfloat16 *__restrict__ dV, float *__restrict__ dQacc,
-              int n, int n_pad, int causal, float scale, float scale_log2, int nkt, unsigned int *status)
+              int n, int n_pad, int causal, float scale, float scale_log2, int nkt, unsigned int *status, int dbg)
 {
     using SM = BwdSmem<D>;
     constexpr int kBoxes = D / 64;
     constexpr int kBoxBytes = 128 * 128;
-    constexpr uint32_t colS = 0, colDP = 128, colDV = 256, colDK = 256 + D, colDQ = (D == 128) ? 128 : 384;
+    constexpr bool kAliasDQ = (D == 128);   // dQ tile shares the dP^T columns
+    // For D = 128 the tile is produced transposed (lanes = d) so that one warp-wide red covers
+    // 32 consecutive floats of one dQ row: a full 128-byte line per request instead of 32
+    // half-used sectors.  (UMMA needs M = 128, so D = 64 keeps lanes = queries.)
+    constexpr bool kTransposeDQ = (D == 128);
+    constexpr uint32_t colS = 0, colDP = 128, colDV = 256, colDK = 256 + D, colDQ = kAliasDQ ? 128 : 384;
     extern __shared__ __align__(1024) uint8_t sm[];
     uint8_t *sK = sm + SM::offK, *sV = sm + SM::offV, *sdS = sm + SM::offdS;
     float *sL = reinterpret_cast<float *>(sm + SM::offL);
     float *sD = reinterpret_cast<float *>(sm + SM::offD);
     uint64_t *bars = reinterpret_cast<uint64_t *>(sm + SM::offBar);
-    uint64_t *bar_kv = bars + 0, *bar_full = bars + 1 /*[2]*/, *bar_empty = bars + 3 /*[2]*/;
-    uint64_t *bar_sdp = bars + 5, *bar_pds = bars + 6, *bar_dq = bars + 7, *bar_dqr = bars + 8;
-    uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(bars + 9);
-    volatile uint32_t *abortp = reinterpret_cast<uint32_t *>(bars + 10);
+    uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(bars + B_COUNT);
+    volatile uint32_t *abortp = reinterpret_cast<uint32_t *>(bars + B_COUNT + 1);
 
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
     const int bh = blockIdx.x / nkt;
@@ -131,83 +152,105 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     const int k0 = kt * 128;
     const int nqt = n_pad / 128;
     const int i_begin = causal ? kt : 0;
-    const int niter = nqt - i_begin;
+    const int niter_all = nqt - i_begin;
 
     if (tid == 0) {
-        mbar_init(bar_kv, 1);
-        mbar_init(bar_full + 0, 1); mbar_init(bar_full + 1, 1);
-        mbar_init(bar_empty + 0, 1); mbar_init(bar_empty + 1, 1);
-        mbar_init(bar_sdp, 1); mbar_init(bar_pds, 256); mbar_init(bar_dq, 1); mbar_init(bar_dqr, 256);
+        for (int b = 0; b < B_COUNT; ++b) {
+            const uint32_t cnt = (b == B_P || b == B_DS) ? 256u : (b == B_DQR ? 128u : 1u);
+            mbar_init(bars + b, cnt);
+        }
         *abortp = (smem_u32(sm) & 1023u) ? 1u : 0u;
         if (*abortp && status) atomicCAS(status, 0u, (unsigned)ERR_ALIGN);
         fence_mbar_init();
         prefetch_tensormap(&mapQ); prefetch_tensormap(&mapK); prefetch_tensormap(&mapV); prefetch_tensormap(&mapdO);
     }
-    if (warp == 9) { tmem_alloc(tmem_base_s, kTmemCols); tmem_relinquish(); }
+    if (warp == kMmaWarp) { tmem_alloc(tmem_base_s, kTmemCols); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tbase = *tmem_base_s;
-    const bool aligned_ok = (*abortp == 0);
+    // a misaligned shared-memory base (swizzled tiles would be misplaced) turns every role into a no-op
+    const int niter = (*abortp == 0) ? niter_all : 0;
 
-    if (!aligned_ok) {
-        // shared memory base is not 1024-byte aligned: swizzled tiles would be misplaced
-    } else if (warp == 8) {
+    // 512 threads start with 128 registers each (the whole register file); the last
+    // warpgroup (TMA, UMMA, two idle warps) gives most of its share to the others
+    // (setmaxnreg at the top of each role's branch).
+    if (warp >= kLoadWarp) {
+      // one instruction for the whole last warpgroup (TMA warp, UMMA warp, two idle warps)
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+      if (warp == kLoadWarp) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            mbar_arrive_expect_tx(bar_kv, 2 * SM::kTile);
+        if (lane == 0 && niter > 0) {
+            mbar_arrive_expect_tx(bars + B_KV, 2 * SM::kTile);
             for (int b = 0; b < kBoxes; ++b) {
-                tma_load_3d(sK + b * kBoxBytes, &mapK, bar_kv, 64 * b, k0, bh);
-                tma_load_3d(sV + b * kBoxBytes, &mapV, bar_kv, 64 * b, k0, bh);
+                tma_load_3d(sK + b * kBoxBytes, &mapK, bars + B_KV, 64 * b, k0, bh);
+                tma_load_3d(sV + b * kBoxBytes, &mapV, bars + B_KV, 64 * b, k0, bh);
             }
         }
         for (int it = 0; it < niter; ++it) {
             const int s = it & 1;
             const int q0 = (i_begin + it) * 128;
-            if (it >= 2 && !mbar_wait(bar_empty + s, ((it >> 1) - 1) & 1, abortp, status, ERR_EMPTY)) break;
+            // dO slot first: it is released (after dV) earlier than the Q slot (after dK, dQ)
+            if (it >= 2 && !mbar_wait(bars + B_DOEMPTY + s, ((it >> 1) - 1) & 1, abortp, status, ERR_EMPTY)) break;
             if (lane == 0) {
-                uint8_t *sQ = sm + SM::offQ + s * SM::kTile, *sdO = sm + SM::offdO + s * SM::kTile;
-                mbar_arrive_expect_tx(bar_full + s, 2 * SM::kTile + 1024);
-                for (int b = 0; b < kBoxes; ++b) {
-                    tma_load_3d(sQ + b * kBoxBytes, &mapQ, bar_full + s, 64 * b, q0, bh);
-                    tma_load_3d(sdO + b * kBoxBytes, &mapdO, bar_full + s, 64 * b, q0, bh);
-                }
-                bulk_load_1d(sL + s * 128, Lp + (size_t)bh * n_pad + q0, 512, bar_full + s);
-                bulk_load_1d(sD + s * 128, Dp + (size_t)bh * n_pad + q0, 512, bar_full + s);
+                uint8_t *sdO = sm + SM::offdO + s * SM::kTile;
+                mbar_arrive_expect_tx(bars + B_DOFULL + s, SM::kTile);
+                for (int b = 0; b < kBoxes; ++b)
+                    tma_load_3d(sdO + b * kBoxBytes, &mapdO, bars + B_DOFULL + s, 64 * b, q0, bh);
+            }
+            if (it >= 2 && !mbar_wait(bars + B_QEMPTY + s, ((it >> 1) - 1) & 1, abortp, status, ERR_EMPTY)) break;
+            if (lane == 0) {
+                uint8_t *sQ = sm + SM::offQ + s * SM::kTile;
+                mbar_arrive_expect_tx(bars + B_QFULL + s, SM::kTile + 1024);
+                for (int b = 0; b < kBoxes; ++b)
+                    tma_load_3d(sQ + b * kBoxBytes, &mapQ, bars + B_QFULL + s, 64 * b, q0, bh);
+                bulk_load_1d(sL + s * 128, Lp + (size_t)bh * n_pad + q0, 512, bars + B_QFULL + s);
+                bulk_load_1d(sD + s * 128, Dp + (size_t)bh * n_pad + q0, 512, bars + B_QFULL + s);
             }
             __syncwarp();
         }
-    } else if (warp == 9) {
+      } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------- UMMA issuer
+        // Issue order per query tile i:  dP(i), dV(i), S(i+1), dK(i), dQ(i).
         constexpr uint32_t idesc_st = idesc_bf16_f32(128, 128, 0, 0);   // S^T, dP^T
         constexpr uint32_t idesc_acc = idesc_bf16_f32(128, D, 0, 1);    // dV, dK: A in TMEM, B MN-major
         constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, 1, 1);     // dQ: A and B MN-major
+        constexpr uint32_t idesc_dqt = idesc_bf16_f32(128, 128, 1, 1);  // dQ^T (D = 128 only)
         const uint32_t k_addr = smem_u32(sK), v_addr = smem_u32(sV), ds_addr = smem_u32(sdS);
-        bool ok = mbar_wait(bar_kv, 0, abortp, status, ERR_KV);
+        auto issue_S = [&](uint32_t q_addr) {
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks) {
+                const uint32_t off = (ks / 4) * kBoxBytes + (ks % 4) * 32;
+                umma_ss(tbase + colS, smem_desc_sw128(k_addr + off, 16, 1024),
+                        smem_desc_sw128(q_addr + off, 16, 1024), idesc_st, ks > 0);
+            }
+            umma_commit(bars + B_S);
+        };
+        bool ok = niter > 0 && mbar_wait(bars + B_KV, 0, abortp, status, ERR_KV);
+        ok = ok && mbar_wait(bars + B_QFULL + 0, 0, abortp, status, ERR_FULL);
+        if (ok) {
+            tc_fence_after();
+            if (lane == 0) issue_S(smem_u32(sm + SM::offQ));
+            __syncwarp();
+        }
         for (int it = 0; ok && it < niter; ++it) {
             const int s = it & 1;
             const uint32_t q_addr = smem_u32(sm + SM::offQ + s * SM::kTile);
             const uint32_t do_addr = smem_u32(sm + SM::offdO + s * SM::kTile);
-            if (!mbar_wait(bar_full + s, (it >> 1) & 1, abortp, status, ERR_FULL)) break;
-            if (it > 0 && !mbar_wait(bar_dqr, (it - 1) & 1, abortp, status, ERR_DQR)) break;   // dQ tile read out
+            if (!mbar_wait(bars + B_DOFULL + s, (it >> 1) & 1, abortp, status, ERR_FULL)) break;
+            if (kAliasDQ && it > 0 && !mbar_wait(bars + B_DQR, (it - 1) & 1, abortp, status, ERR_DQR)) break;
             tc_fence_after();
             if (lane == 0) {
-#pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = (ks / 4) * kBoxBytes + (ks % 4) * 32;
-                    umma_ss(tbase + colS, smem_desc_sw128(k_addr + off, 16, 1024),
-                            smem_desc_sw128(q_addr + off, 16, 1024), idesc_st, ks > 0);
-                }
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t off = (ks / 4) * kBoxBytes + (ks % 4) * 32;
                     umma_ss(tbase + colDP, smem_desc_sw128(v_addr + off, 16, 1024),
                             smem_desc_sw128(do_addr + off, 16, 1024), idesc_st, ks > 0);
                 }
-                umma_commit(bar_sdp);
+                umma_commit(bars + B_DP);
             }
             __syncwarp();
-            if (!mbar_wait(bar_pds, it & 1, abortp, status, ERR_PDS)) break;
+            if (!mbar_wait(bars + B_P, it & 1, abortp, status, ERR_PDS)) break;
             tc_fence_after();
             if (lane == 0) {
 #pragma unroll
@@ -216,6 +259,20 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                     umma_ts(tbase + colDV, tbase + colS + a_col,
                             smem_desc_sw128(do_addr + ks * 2048, kBoxBytes, 1024), idesc_acc, (it > 0 || ks > 0));
                 }
+                umma_commit(bars + B_DOEMPTY + s);
+            }
+            __syncwarp();
+            if (it + 1 < niter) {
+                const int s1 = (it + 1) & 1;
+                if (!mbar_wait(bars + B_QFULL + s1, ((it + 1) >> 1) & 1, abortp, status, ERR_FULL)) break;
+                tc_fence_after();
+                if (lane == 0) issue_S(smem_u32(sm + SM::offQ + s1 * SM::kTile));
+                __syncwarp();
+            }
+            if (!mbar_wait(bars + B_DS, it & 1, abortp, status, ERR_PDS)) break;
+            if (!kAliasDQ && it > 0 && !mbar_wait(bars + B_DQR, (it - 1) & 1, abortp, status, ERR_DQR)) break;
+            tc_fence_after();
+            if (lane == 0) {
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     const uint32_t a_col = 64 * (ks / 4) + 8 * (ks % 4);
@@ -224,53 +281,132 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 }
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {   // 16 keys per step
-                    umma_ss(tbase + colDQ, smem_desc_sw128(ds_addr + ks * 2048, kBoxBytes, 1024),
-                            smem_desc_sw128(k_addr + ks * 2048, kBoxBytes, 1024), idesc_dq, ks > 0);
+                    const uint64_t ds_desc = smem_desc_sw128(ds_addr + ks * 2048, kBoxBytes, 1024);
+                    const uint64_t k_desc = smem_desc_sw128(k_addr + ks * 2048, kBoxBytes, 1024);
+                    if (kTransposeDQ)   // dQ^T = K^T dS^T: lanes are d, columns are queries
+                        umma_ss(tbase + colDQ, k_desc, ds_desc, idesc_dqt, ks > 0);
+                    else                // dQ = dS K: lanes are queries, columns are d
+                        umma_ss(tbase + colDQ, ds_desc, k_desc, idesc_dq, ks > 0);
                 }
-                umma_commit(bar_empty + s);
-                umma_commit(bar_dq);
+                umma_commit(bars + B_QEMPTY + s);
+                umma_commit(bars + B_DQ);
             }
             __syncwarp();
         }
+      }
+    } else if (warp >= kReduceWarp0) {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 152;");
+        // ------------------------------------------------- dQ reduce warps: lanes are query rows
+        const int lane_row = 32 * (warp % 4) + lane;
+        const uint32_t lane_addr = tbase + ((uint32_t)(32 * (warp % 4)) << 16);
+        for (int it = 0; it < niter; ++it) {
+            const int qrow = (i_begin + it) * 128 + lane_row;
+            if (!mbar_wait(bars + B_DQ, it & 1, abortp, status, ERR_DQ)) break;
+            tc_fence_after();
+            uint32_t r[D / 32][32];
+            if (kTransposeDQ) {
+                // lanes are d (this thread: column lane_row of every dQ row), TMEM columns are queries
+                const int q0 = (i_begin + it) * 128;
+                float *dst = dQacc + ((size_t)bh * n + q0) * D + lane_row;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) tmem_ld(lane_addr + colDQ + 32 * c, r[c]);
+                tc_wait_ld();
+                tc_fence_before();
+                mbar_arrive(bars + B_DQR);      // TMEM columns are free again; the reds go out from registers
+                if (!(dbg & 1)) {
+                    const int valid = min(128, n - q0);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (32 * c + e < valid) red_add_f32(dst + (size_t)(32 * c + e) * D, __uint_as_float(r[c][e]));
+                }
+            } else {
+                float *dst = dQacc + ((size_t)bh * n + qrow) * D;
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) tmem_ld(lane_addr + colDQ + 32 * c, r[c]);
+                tc_wait_ld();
+                tc_fence_before();
+                mbar_arrive(bars + B_DQR);
+                if (qrow < n && !(dbg & 1)) {
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c)
+#pragma unroll
+                        for (int e = 0; e < 32; e += 4)
+                            red_add_v4(dst + 32 * c + e, __uint_as_float(r[c][e]), __uint_as_float(r[c][e + 1]),
+                                       __uint_as_float(r[c][e + 2]), __uint_as_float(r[c][e + 3]));
+                }
+            }
+        }
     } else {
         // ----------------------------------------------------------- elementwise warps 0-7
-        const int wg = warp / 4;                          // which half of the columns
-        const int lane_row = 32 * (warp % 4) + lane;      // TMEM lane of this thread
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 152;");
+        const int wg = warp / 4;                          // which half of the query columns
+        const int lane_row = 32 * (warp % 4) + lane;      // TMEM lane of this thread = key index in the tile
         const uint32_t lane_addr = tbase + ((uint32_t)(32 * (warp % 4)) << 16);
+        float p[64];                                      // this thread's probabilities of the current tile
         bool ok = true;
-        for (int it = 0; it < niter; ++it) {
+
+        // P-phase of tile `it`: P^T = exp2(S^T scale log2e - L log2e), kept in registers and
+        // written as bf16 over the first half of this warpgroup's S^T columns.
+        auto p_phase = [&](int it) -> bool {
             const int s = it & 1;
-            const int i = i_begin + it;
-            const int q0 = i * 128;
-            const bool diag = causal && (i == kt);
-            if (!mbar_wait(bar_sdp, it & 1, abortp, status, ERR_SDP)) { ok = false; break; }
+            const bool diag = causal && (i_begin + it == kt);
+            if (!mbar_wait(bars + B_S, it & 1, abortp, status, ERR_SDP)) return false;
             tc_fence_after();
-            const float *Ls = sL + s * 128, *Ds = sD + s * 128;
+            const float *Ls = sL + s * 128;
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
-                const int qc0 = 64 * wg + 32 * c;         // first query column of this chunk
-                uint32_t rs[32], rd[32];
+                const int qc0 = 64 * wg + 32 * c;
+                uint32_t rs[32];
                 tmem_ld(lane_addr + colS + qc0, rs);
-                tmem_ld(lane_addr + colDP + qc0, rd);
                 tc_wait_ld();
-                uint32_t pk[16], gk[16];
+                uint32_t pk[16];
 #pragma unroll
                 for (int e = 0; e < 32; e += 4) {
                     const float4 l4 = *reinterpret_cast<const float4 *>(Ls + qc0 + e);
-                    const float4 d4 = *reinterpret_cast<const float4 *>(Ds + qc0 + e);
-                    const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dv[4] = {d4.x, d4.y, d4.z, d4.w};
-                    float p[4], g[4];
+                    const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
                         float pv = ex2(fmaf(__uint_as_float(rs[e + u]), scale_log2, -lv[u]));
                         if (diag && (qc0 + e + u) < lane_row) pv = 0.f;   // query index < key index: masked
-                        p[u] = pv;
-                        g[u] = pv * (__uint_as_float(rd[e + u]) - dv[u]) * scale;
+                        p[32 * c + e + u] = pv;
                     }
-                    pk[e / 2] = pack_bf16(p[0], p[1]); pk[e / 2 + 1] = pack_bf16(p[2], p[3]);
-                    gk[e / 2] = pack_bf16(g[0], g[1]); gk[e / 2 + 1] = pack_bf16(g[2], g[3]);
+                    pk[e / 2] = pack_bf16(p[32 * c + e], p[32 * c + e + 1]);
+                    pk[e / 2 + 1] = pack_bf16(p[32 * c + e + 2], p[32 * c + e + 3]);
                 }
                 tmem_st(lane_addr + colS + 64 * wg + 16 * c, pk);
+            }
+            tc_wait_st();
+            tc_fence_before();
+            mbar_arrive(bars + B_P);
+            return true;
+        };
+
+        ok = niter > 0 && p_phase(0);
+        for (int it = 0; ok && it < niter; ++it) {
+            const int s = it & 1;
+            // dS-phase: dS^T = P^T o (dP^T - D)   (the factor `scale` is applied to dK and dQ at the end)
+            if (!mbar_wait(bars + B_DP, it & 1, abortp, status, ERR_SDP)) { ok = false; break; }
+            tc_fence_after();
+            const float *Ds = sD + s * 128;
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                const int qc0 = 64 * wg + 32 * c;
+                uint32_t rd[32];
+                tmem_ld(lane_addr + colDP + qc0, rd);
+                tc_wait_ld();
+                uint32_t gk[16];
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                    const float4 d4 = *reinterpret_cast<const float4 *>(Ds + qc0 + e);
+                    const float g0 = p[32 * c + e] * (__uint_as_float(rd[e]) - d4.x);
+                    const float g1 = p[32 * c + e + 1] * (__uint_as_float(rd[e + 1]) - d4.y);
+                    const float g2 = p[32 * c + e + 2] * (__uint_as_float(rd[e + 2]) - d4.z);
+                    const float g3 = p[32 * c + e + 3] * (__uint_as_float(rd[e + 3]) - d4.w);
+                    gk[e / 2] = pack_bf16(g0, g1);
+                    gk[e / 2 + 1] = pack_bf16(g2, g3);
+                }
                 tmem_st(lane_addr + colDP + 64 * wg + 16 * c, gk);
                 // dS^T row (this key) into the MN-major smem tile: box wg, 128-byte row, swizzled 16-byte chunks
                 uint8_t *rowp = sdS + wg * kBoxBytes + lane_row * 128;
@@ -284,37 +420,18 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             tc_wait_st();
             tc_fence_before();
             fence_proxy_async_smem();
-            mbar_arrive(bar_pds);
-
-            if (!mbar_wait(bar_dq, it & 1, abortp, status, ERR_DQ)) { ok = false; break; }
-            tc_fence_after();
-            // dQ tile: lanes are query rows now; this warpgroup takes D/2 columns
-            const int qrow = q0 + lane_row;
-            float *dst = dQacc + ((size_t)bh * n + qrow) * D + (D / 2) * wg;
-#pragma unroll
-            for (int c = 0; c < D / 2; c += 32) {
-                uint32_t r[32];
-                tmem_ld(lane_addr + colDQ + (D / 2) * wg + c, r);
-                tc_wait_ld();
-                if (qrow < n) {
-#pragma unroll
-                    for (int e = 0; e < 32; e += 4)
-                        red_add_v4(dst + c + e, __uint_as_float(r[e]), __uint_as_float(r[e + 1]),
-                                   __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
-                }
-            }
-            tc_fence_before();
-            mbar_arrive(bar_dqr);
+            mbar_arrive(bars + B_DS);
+            if (it + 1 < niter) ok = p_phase(it + 1);
         }
-        if (ok) {
-            // all UMMAs have completed (the last bar_dq wait): write dV and dK rows of this key
+        if (ok && mbar_wait(bars + B_DQ, (niter - 1) & 1, abortp, status, ERR_DQ)) {
+            // all UMMAs have completed: write dV and scale*dK rows of this key
+            tc_fence_after();
             const int krow = k0 + lane_row;
-            __nv_bfloat16 *dvp = dV + ((size_t)bh * n + krow) * D + (D / 2) * wg;
-            __nv_bfloat16 *dkp = dK + ((size_t)bh * n + krow) * D + (D / 2) * wg;
 #pragma unroll
             for (int which = 0; which < 2; ++which) {
                 const uint32_t col = (which == 0 ? colDV : colDK) + (D / 2) * wg;
-                __nv_bfloat16 *outp = which == 0 ? dvp : dkp;
+                const float mul = which == 0 ? 1.f : scale;
+                __nv_bfloat16 *outp = (which == 0 ? dV : dK) + ((size_t)bh * n + krow) * D + (D / 2) * wg;
 #pragma unroll
                 for (int c = 0; c < D / 2; c += 32) {
                     uint32_t r[32];
@@ -324,10 +441,10 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
 #pragma unroll
                         for (int e = 0; e < 32; e += 8) {
                             uint4 v;
-                            v.x = pack_bf16(__uint_as_float(r[e + 0]), __uint_as_float(r[e + 1]));
-                            v.y = pack_bf16(__uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
-                            v.z = pack_bf16(__uint_as_float(r[e + 4]), __uint_as_float(r[e + 5]));
-                            v.w = pack_bf16(__uint_as_float(r[e + 6]), __uint_as_float(r[e + 7]));
+                            v.x = pack_bf16(__uint_as_float(r[e + 0]) * mul, __uint_as_float(r[e + 1]) * mul);
+                            v.y = pack_bf16(__uint_as_float(r[e + 2]) * mul, __uint_as_float(r[e + 3]) * mul);
+                            v.z = pack_bf16(__uint_as_float(r[e + 4]) * mul, __uint_as_float(r[e + 5]) * mul);
+                            v.w = pack_bf16(__uint_as_float(r[e + 6]) * mul, __uint_as_float(r[e + 7]) * mul);
                             *reinterpret_cast<uint4 *>(outp + c + e) = v;
                         }
                     }
@@ -337,7 +454,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 9) tmem_dealloc(tbase, kTmemCols);
+    if (warp == kMmaWarp) tmem_dealloc(tbase, kTmemCols);
 }
 
 template <int D>
@@ -358,7 +475,7 @@ cudaError_t launch_bwd(const Problem &p, const void *Q, const void *K, const voi
     LaunchScope scope(MOA_KERNEL_BWD_KV, st);
     tc_bwd_kernel<D><<<(unsigned)(nkt * p.BH()), kThreads, kSmem, st>>>(
         mq, mk, mv, mdo, Lp, Dp, (__nv_bfloat16 *)dK, (__nv_bfloat16 *)dV, dQacc, p.n, nkt * 128, p.causal,
-        p.scale, p.scale * kLog2e, nkt, device_status_ptr());
+        p.scale, p.scale * kLog2e, nkt, device_status_ptr(), getenv("MOA_BWD_DEBUG") ? atoi(getenv("MOA_BWD_DEBUG")) : 0);
     return cudaGetLastError();
 }
 
