@@ -102,15 +102,17 @@ moa_status check_desc(const moa_attn_desc *d)
     if (d->materialize) return MOA_ERR_UNSUPPORTED;           // comparison variant not built yet
     if (d->dq_mode == MOA_DQ_BULK_REDUCE) return MOA_ERR_UNSUPPORTED;
     if (d->path == MOA_PATH_TC && d->dq_mode == MOA_DQ_SEPARATE_PASS) return MOA_ERR_UNSUPPORTED;
+    if (d->path == MOA_PATH_TC && !(d->scale > 0.f)) return MOA_ERR_UNSUPPORTED;   // non-positive scale: SIMT path only
     return MOA_OK;
 }
 
 int resolved_dq_mode(const moa_attn_desc *d) { return d->dq_mode == MOA_DQ_AUTO ? MOA_DQ_RED : d->dq_mode; }
 
-bool use_tc_fwd(const moa_attn_desc *d) { return d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT; }
+// the tensor-core kernels take the row max before scaling, which needs scale > 0
+bool use_tc_fwd(const moa_attn_desc *d) { return d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->scale > 0.f; }
 bool use_tc_bwd(const moa_attn_desc *d)
 {
-    return d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && resolved_dq_mode(d) == MOA_DQ_RED;
+    return d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->scale > 0.f && resolved_dq_mode(d) == MOA_DQ_RED;
 }
 
 // Workspace of the backward: [ D | Lp (tensor-core path only) | dQacc (bf16 with an atomic mode) ]

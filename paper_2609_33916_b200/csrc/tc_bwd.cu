@@ -216,37 +216,41 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         constexpr uint32_t idesc_acc = idesc_bf16_f32(128, D, 0, 1);    // dV, dK: A in TMEM, B MN-major
         constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, 1, 1);     // dQ: A and B MN-major
         constexpr uint32_t idesc_dqt = idesc_bf16_f32(128, 128, 1, 1);  // dQ^T (D = 128 only)
-        const uint32_t k_addr = smem_u32(sK), v_addr = smem_u32(sV), ds_addr = smem_u32(sdS);
-        auto issue_S = [&](uint32_t q_addr) {
+        // Descriptors are built once; inside the loops only a constant is added to the address
+        // field, so that the issuing thread stays well ahead of the 64-cycle UMMAs.
+        const uint64_t k_km = smem_desc_sw128(smem_u32(sK), 16, 1024);          // K, K-major (S^T: A)
+        const uint64_t v_km = smem_desc_sw128(smem_u32(sV), 16, 1024);          // V, K-major (dP^T: A)
+        const uint64_t k_mn = smem_desc_sw128(smem_u32(sK), kBoxBytes, 1024);   // K, MN-major (dQ)
+        const uint64_t ds_mn = smem_desc_sw128(smem_u32(sdS), kBoxBytes, 1024); // dS^T tile, MN-major (dQ)
+        const uint64_t q_km0 = smem_desc_sw128(smem_u32(sm + SM::offQ), 16, 1024);
+        const uint64_t q_mn0 = smem_desc_sw128(smem_u32(sm + SM::offQ), kBoxBytes, 1024);
+        const uint64_t do_km0 = smem_desc_sw128(smem_u32(sm + SM::offdO), 16, 1024);
+        const uint64_t do_mn0 = smem_desc_sw128(smem_u32(sm + SM::offdO), kBoxBytes, 1024);
+        constexpr uint64_t kSlot = (uint64_t)(SM::kTile >> 4);   // address-field step between the two slots
+        auto koff = [](int ks) { return (uint64_t)(((ks / 4) * kBoxBytes + (ks % 4) * 32) >> 4); };
+        auto moff = [](int ks) { return (uint64_t)((ks * 2048) >> 4); };
+        auto issue_S = [&](uint64_t q_km) {
 #pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks) {
-                const uint32_t off = (ks / 4) * kBoxBytes + (ks % 4) * 32;
-                umma_ss(tbase + colS, smem_desc_sw128(k_addr + off, 16, 1024),
-                        smem_desc_sw128(q_addr + off, 16, 1024), idesc_st, ks > 0);
-            }
+            for (int ks = 0; ks < D / 16; ++ks) umma_ss(tbase + colS, k_km + koff(ks), q_km + koff(ks), idesc_st, ks > 0);
             umma_commit(bars + B_S);
         };
         bool ok = niter > 0 && mbar_wait(bars + B_KV, 0, abortp, status, ERR_KV);
         ok = ok && mbar_wait(bars + B_QFULL + 0, 0, abortp, status, ERR_FULL);
         if (ok) {
             tc_fence_after();
-            if (lane == 0) issue_S(smem_u32(sm + SM::offQ));
+            if (lane == 0) issue_S(q_km0);
             __syncwarp();
         }
         for (int it = 0; ok && it < niter; ++it) {
             const int s = it & 1;
-            const uint32_t q_addr = smem_u32(sm + SM::offQ + s * SM::kTile);
-            const uint32_t do_addr = smem_u32(sm + SM::offdO + s * SM::kTile);
+            const uint64_t q_mn = q_mn0 + s * kSlot, do_km = do_km0 + s * kSlot, do_mn = do_mn0 + s * kSlot;
             if (!mbar_wait(bars + B_DOFULL + s, (it >> 1) & 1, abortp, status, ERR_FULL)) break;
             if (kAliasDQ && it > 0 && !mbar_wait(bars + B_DQR, (it - 1) & 1, abortp, status, ERR_DQR)) break;
             tc_fence_after();
             if (lane == 0) {
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = (ks / 4) * kBoxBytes + (ks % 4) * 32;
-                    umma_ss(tbase + colDP, smem_desc_sw128(v_addr + off, 16, 1024),
-                            smem_desc_sw128(do_addr + off, 16, 1024), idesc_st, ks > 0);
-                }
+                for (int ks = 0; ks < D / 16; ++ks)
+                    umma_ss(tbase + colDP, v_km + koff(ks), do_km + koff(ks), idesc_st, ks > 0);
                 umma_commit(bars + B_DP);
             }
             __syncwarp();
@@ -256,8 +260,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {   // 16 queries per step
                     const uint32_t a_col = 64 * (ks / 4) + 8 * (ks % 4);
-                    umma_ts(tbase + colDV, tbase + colS + a_col,
-                            smem_desc_sw128(do_addr + ks * 2048, kBoxBytes, 1024), idesc_acc, (it > 0 || ks > 0));
+                    umma_ts(tbase + colDV, tbase + colS + a_col, do_mn + moff(ks), idesc_acc, (it > 0 || ks > 0));
                 }
                 umma_commit(bars + B_DOEMPTY + s);
             }
@@ -266,7 +269,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 const int s1 = (it + 1) & 1;
                 if (!mbar_wait(bars + B_QFULL + s1, ((it + 1) >> 1) & 1, abortp, status, ERR_FULL)) break;
                 tc_fence_after();
-                if (lane == 0) issue_S(smem_u32(sm + SM::offQ + s1 * SM::kTile));
+                if (lane == 0) issue_S(q_km0 + s1 * kSlot);
                 __syncwarp();
             }
             if (!mbar_wait(bars + B_DS, it & 1, abortp, status, ERR_PDS)) break;
@@ -276,17 +279,14 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     const uint32_t a_col = 64 * (ks / 4) + 8 * (ks % 4);
-                    umma_ts(tbase + colDK, tbase + colDP + a_col,
-                            smem_desc_sw128(q_addr + ks * 2048, kBoxBytes, 1024), idesc_acc, (it > 0 || ks > 0));
+                    umma_ts(tbase + colDK, tbase + colDP + a_col, q_mn + moff(ks), idesc_acc, (it > 0 || ks > 0));
                 }
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {   // 16 keys per step
-                    const uint64_t ds_desc = smem_desc_sw128(ds_addr + ks * 2048, kBoxBytes, 1024);
-                    const uint64_t k_desc = smem_desc_sw128(k_addr + ks * 2048, kBoxBytes, 1024);
                     if (kTransposeDQ)   // dQ^T = K^T dS^T: lanes are d, columns are queries
-                        umma_ss(tbase + colDQ, k_desc, ds_desc, idesc_dqt, ks > 0);
+                        umma_ss(tbase + colDQ, k_mn + moff(ks), ds_mn + moff(ks), idesc_dqt, ks > 0);
                     else                // dQ = dS K: lanes are queries, columns are d
-                        umma_ss(tbase + colDQ, ds_desc, k_desc, idesc_dq, ks > 0);
+                        umma_ss(tbase + colDQ, ds_mn + moff(ks), k_mn + moff(ks), idesc_dq, ks > 0);
                 }
                 umma_commit(bars + B_QEMPTY + s);
                 umma_commit(bars + B_DQ);
@@ -355,6 +355,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             if (!mbar_wait(bars + B_S, it & 1, abortp, status, ERR_SDP)) return false;
             tc_fence_after();
             const float *Ls = sL + s * 128;
+            if (!(dbg & 2))
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 const int qc0 = 64 * wg + 32 * c;
@@ -390,6 +391,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             if (!mbar_wait(bars + B_DP, it & 1, abortp, status, ERR_SDP)) { ok = false; break; }
             tc_fence_after();
             const float *Ds = sD + s * 128;
+            if (!(dbg & 2))
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 const int qc0 = 64 * wg + 32 * c;

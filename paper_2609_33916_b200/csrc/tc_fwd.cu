@@ -101,7 +101,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         // ------------------------------------------------------------------- UMMA issuer
         constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0);
         constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, 0, 1);
-        const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
+        // Descriptors are built once; inside the loops only a constant is added to the address
+        // field (the issuing thread's instruction stream must stay far shorter than the 64 cycles
+        // one 128x128x16 UMMA takes, or the tensor pipe starves).
+        const uint64_t q_desc = smem_desc_sw128(smem_u32(sQ), 16, 1024);
+        const uint64_t k_desc = smem_desc_sw128(smem_u32(sK), 16, 1024);
+        const uint64_t v_desc = smem_desc_sw128(smem_u32(sV), kBoxBytes, 1024);   // MN-major
         bool ok = mbar_wait(&bar_q, 0, abortp, status, ERR_Q);
         for (int j = 0; ok && j < nkt; ++j) {
             if (!mbar_wait(&bar_k, j & 1, abortp, status, ERR_K)) break;
@@ -109,9 +114,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             if (lane == 0) {
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = (ks / 4) * kBoxBytes + (ks % 4) * 32;
-                    umma_ss(tbase + kColS, smem_desc_sw128(q_addr + off, 16, 1024),
-                            smem_desc_sw128(k_addr + off, 16, 1024), idesc_s, ks > 0);
+                    const uint64_t off = (uint64_t)(((ks / 4) * kBoxBytes + (ks % 4) * 32) >> 4);
+                    umma_ss(tbase + kColS, q_desc + off, k_desc + off, idesc_s, ks > 0);
                 }
                 umma_commit(&bar_s);
             }
@@ -122,8 +126,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             if (lane == 0) {
 #pragma unroll
                 for (int ks = 0; ks < BN / 16; ++ks) {
-                    umma_ts(tbase + kColO, tbase + kColP + ks * 8,
-                            smem_desc_sw128(v_addr + ks * 2048, kBoxBytes, 1024), idesc_pv, (j > 0 || ks > 0));
+                    umma_ts(tbase + kColO, tbase + kColP + ks * 8, v_desc + (uint64_t)((ks * 2048) >> 4), idesc_pv,
+                            (j > 0 || ks > 0));
                 }
                 umma_commit(&bar_o);
             }
@@ -140,25 +144,31 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             tc_fence_after();
             const int k0 = j * BN;
             const bool need_mask = (k0 + BN > n) || (causal && k0 + BN - 1 > q0);
-            // pass 1: row max of the scaled, masked scores (log2 domain)
-            float mx = -INFINITY;
+            // The whole score row (128 fp32) comes into registers with one round trip to TMEM.
+            uint32_t r[4][32];
 #pragma unroll
-            for (int c = 0; c < BN; c += 32) {
-                uint32_t r[32];
-                tmem_ld(lane_addr + kColS + c, r);
-                tc_wait_ld();
-                if (need_mask) {
+            for (int c = 0; c < 4; ++c) tmem_ld(lane_addr + kColS + 32 * c, r[c]);
+            tc_wait_ld();
+            if (need_mask) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
-                        const int col = k0 + c + i;
-                        const bool live = col < n && !(causal && col > row);
-                        mx = fmaxf(mx, live ? __uint_as_float(r[i]) * scale_log2 : -INFINITY);
+                        const int col = k0 + 32 * c + i;
+                        if (col >= n || (causal && col > row)) r[c][i] = 0xff800000u;   // -inf
                     }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(r[i]) * scale_log2);
-                }
             }
+            // row max of the raw scores (scale_log2 > 0, so scaling commutes with max)
+            float mx4[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                float a = fmaxf(__uint_as_float(r[c][0]), __uint_as_float(r[c][1]));
+#pragma unroll
+                for (int i = 2; i < 32; i += 2)
+                    a = fmaxf(a, fmaxf(__uint_as_float(r[c][i]), __uint_as_float(r[c][i + 1])));
+                mx4[c] = a;
+            }
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
             if (j == 0) {
                 m_used = (mx == -INFINITY) ? 0.f : mx;
             } else {
@@ -168,43 +178,35 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                     const float alpha = grow ? ex2(m_used - mx) : 1.f;
                     if (grow) m_used = mx;
                     l *= alpha;
-#pragma unroll
-                    for (int c = 0; c < D; c += 32) {
-                        uint32_t r[32];
-                        tmem_ld(lane_addr + kColO + c, r);
+                    // rare path, kept small: the 128 score registers stay live across it
+#pragma unroll 1
+                    for (int c = 0; c < D; c += 8) {
+                        uint32_t o[8];
+                        tmem_ld(lane_addr + kColO + c, o);
                         tc_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                        tmem_st(lane_addr + kColO + c, r);
+                        for (int i = 0; i < 8; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st(lane_addr + kColO + c, o);
                     }
                 }
             }
-            // pass 2: P = 2^(s - m_used), row sum, bf16 P into TMEM over the S columns already read
+            // P = 2^(s scale_log2 - m_used), row sum (four independent partial sums), bf16 P into
+            // TMEM over the first 64 of the S columns
             const float neg_m = -m_used;
+            float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int c = 0; c < BN; c += 32) {
-                uint32_t r[32];
-                tmem_ld(lane_addr + kColS + c, r);
-                tc_wait_ld();
+            for (int c = 0; c < 4; ++c) {
                 uint32_t pk[16];
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
-                    float p0, p1;
-                    if (need_mask) {
-                        const int col = k0 + c + i;
-                        const bool live0 = col < n && !(causal && col > row);
-                        const bool live1 = col + 1 < n && !(causal && col + 1 > row);
-                        p0 = live0 ? ex2(fmaf(__uint_as_float(r[i]), scale_log2, neg_m)) : 0.f;
-                        p1 = live1 ? ex2(fmaf(__uint_as_float(r[i + 1]), scale_log2, neg_m)) : 0.f;
-                    } else {
-                        p0 = ex2(fmaf(__uint_as_float(r[i]), scale_log2, neg_m));
-                        p1 = ex2(fmaf(__uint_as_float(r[i + 1]), scale_log2, neg_m));
-                    }
-                    l += p0 + p1;
+                    const float p0 = ex2(fmaf(__uint_as_float(r[c][i]), scale_log2, neg_m));
+                    const float p1 = ex2(fmaf(__uint_as_float(r[c][i + 1]), scale_log2, neg_m));
+                    ls[(i / 2) & 3] += p0 + p1;
                     pk[i / 2] = pack_bf16(p0, p1);
                 }
-                tmem_st(lane_addr + kColP + c / 2, pk);
+                tmem_st(lane_addr + kColP + 16 * c, pk);
             }
+            l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
             tc_wait_st();
             tc_fence_before();
             mbar_arrive(&bar_p);
