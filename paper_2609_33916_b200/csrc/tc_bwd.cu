@@ -177,7 +177,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     // (setmaxnreg at the top of each role's branch).
     if (warp >= kLoadWarp) {
       // one instruction for the whole last warpgroup (TMA warp, UMMA warp, two idle warps)
-      asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
       if (warp == kLoadWarp) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0 && niter > 0) {
@@ -216,22 +216,27 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         constexpr uint32_t idesc_acc = idesc_bf16_f32(128, D, 0, 1);    // dV, dK: A in TMEM, B MN-major
         constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, 1, 1);     // dQ: A and B MN-major
         constexpr uint32_t idesc_dqt = idesc_bf16_f32(128, 128, 1, 1);  // dQ^T (D = 128 only)
-        // Descriptors are built once; inside the loops only a constant is added to the address
-        // field, so that the issuing thread stays well ahead of the 64-cycle UMMAs.
-        const uint64_t k_km = smem_desc_sw128(smem_u32(sK), 16, 1024);          // K, K-major (S^T: A)
-        const uint64_t v_km = smem_desc_sw128(smem_u32(sV), 16, 1024);          // V, K-major (dP^T: A)
-        const uint64_t k_mn = smem_desc_sw128(smem_u32(sK), kBoxBytes, 1024);   // K, MN-major (dQ)
-        const uint64_t ds_mn = smem_desc_sw128(smem_u32(sdS), kBoxBytes, 1024); // dS^T tile, MN-major (dQ)
-        const uint64_t q_km0 = smem_desc_sw128(smem_u32(sm + SM::offQ), 16, 1024);
-        const uint64_t q_mn0 = smem_desc_sw128(smem_u32(sm + SM::offQ), kBoxBytes, 1024);
-        const uint64_t do_km0 = smem_desc_sw128(smem_u32(sm + SM::offdO), 16, 1024);
-        const uint64_t do_mn0 = smem_desc_sw128(smem_u32(sm + SM::offdO), kBoxBytes, 1024);
-        constexpr uint64_t kSlot = (uint64_t)(SM::kTile >> 4);   // address-field step between the two slots
-        auto koff = [](int ks) { return (uint64_t)(((ks / 4) * kBoxBytes + (ks % 4) * 32) >> 4); };
-        auto moff = [](int ks) { return (uint64_t)((ks * 2048) >> 4); };
-        auto issue_S = [&](uint64_t q_km) {
+        // Descriptors are built once and kept as 32-bit halves.  Only the low half (address field)
+        // changes between k-steps and slots, so an UMMA costs the issuing thread one or two
+        // integer adds, a setp and the tcgen05.mma itself.  This matters: the issuing warp shares
+        // its scheduler with three busy warps, and at a dozen instructions per UMMA it could not
+        // keep the 64-cycle UMMAs fed.
+        const uint64_t km_proto = smem_desc_sw128(0, 16, 1024), mn_proto = smem_desc_sw128(0, kBoxBytes, 1024);
+        const uint32_t km_hi = (uint32_t)(km_proto >> 32), mn_hi = (uint32_t)(mn_proto >> 32);
+        const uint32_t km_lo = (uint32_t)km_proto, mn_lo = (uint32_t)mn_proto;
+        auto field = [](const void *ptr) { return (smem_u32(ptr) >> 4) & 0x3FFFu; };
+        const uint32_t k_km = km_lo + field(sK), v_km = km_lo + field(sV);            // A of S^T, dP^T
+        const uint32_t k_mn = mn_lo + field(sK), ds_mn = mn_lo + field(sdS);          // dQ operands
+        const uint32_t q_km0 = km_lo + field(sm + SM::offQ), q_mn0 = mn_lo + field(sm + SM::offQ);
+        const uint32_t do_km0 = km_lo + field(sm + SM::offdO), do_mn0 = mn_lo + field(sm + SM::offdO);
+        constexpr uint32_t kSlot = (uint32_t)(SM::kTile >> 4);   // address-field step between the two slots
+        auto koff = [](int ks) { return (uint32_t)(((ks / 4) * kBoxBytes + (ks % 4) * 32) >> 4); };
+        auto moff = [](int ks) { return (uint32_t)((ks * 2048) >> 4); };
+        auto issue_S = [&](uint32_t q_km) {
+            umma_ss2<false>(tbase + colS, k_km, km_hi, q_km, km_hi, idesc_st);
 #pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks) umma_ss(tbase + colS, k_km + koff(ks), q_km + koff(ks), idesc_st, ks > 0);
+            for (int ks = 1; ks < D / 16; ++ks)
+                umma_ss2<true>(tbase + colS, k_km + koff(ks), km_hi, q_km + koff(ks), km_hi, idesc_st);
             umma_commit(bars + B_S);
         };
         bool ok = niter > 0 && mbar_wait(bars + B_KV, 0, abortp, status, ERR_KV);
@@ -241,67 +246,89 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             if (lane == 0) issue_S(q_km0);
             __syncwarp();
         }
+        long long *tl = reinterpret_cast<long long *>(dQacc);
+        const bool rec = (dbg & 8) && blockIdx.x == 0 && lane == 0;
+#define TL(slot) do { if (rec && it < 32) tl[it * 16 + (slot)] = clock64(); } while (0)
         for (int it = 0; ok && it < niter; ++it) {
             const int s = it & 1;
-            const uint64_t q_mn = q_mn0 + s * kSlot, do_km = do_km0 + s * kSlot, do_mn = do_mn0 + s * kSlot;
+            TL(0);
+            const uint32_t q_mn = q_mn0 + s * kSlot, do_km = do_km0 + s * kSlot, do_mn = do_mn0 + s * kSlot;
             if (!mbar_wait(bars + B_DOFULL + s, (it >> 1) & 1, abortp, status, ERR_FULL)) break;
+            TL(1);
             if (kAliasDQ && it > 0 && !mbar_wait(bars + B_DQR, (it - 1) & 1, abortp, status, ERR_DQR)) break;
+            TL(2);
             tc_fence_after();
             if (lane == 0) {
+                umma_ss2<false>(tbase + colDP, v_km, km_hi, do_km, km_hi, idesc_st);
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks)
-                    umma_ss(tbase + colDP, v_km + koff(ks), do_km + koff(ks), idesc_st, ks > 0);
+                for (int ks = 1; ks < D / 16; ++ks)
+                    umma_ss2<true>(tbase + colDP, v_km + koff(ks), km_hi, do_km + koff(ks), km_hi, idesc_st);
                 umma_commit(bars + B_DP);
             }
             __syncwarp();
+            TL(3);
             if (!mbar_wait(bars + B_P, it & 1, abortp, status, ERR_PDS)) break;
+            TL(4);
             tc_fence_after();
             if (lane == 0) {
+                // 16 queries per step; the very first UMMA of the CTA overwrites the accumulator
+                if (it > 0) umma_ts2<true>(tbase + colDV, tbase + colS, do_mn, mn_hi, idesc_acc);
+                else        umma_ts2<false>(tbase + colDV, tbase + colS, do_mn, mn_hi, idesc_acc);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {   // 16 queries per step
+                for (int ks = 1; ks < 8; ++ks) {
                     const uint32_t a_col = 64 * (ks / 4) + 8 * (ks % 4);
-                    umma_ts(tbase + colDV, tbase + colS + a_col, do_mn + moff(ks), idesc_acc, (it > 0 || ks > 0));
+                    umma_ts2<true>(tbase + colDV, tbase + colS + a_col, do_mn + moff(ks), mn_hi, idesc_acc);
                 }
                 umma_commit(bars + B_DOEMPTY + s);
             }
             __syncwarp();
             if (it + 1 < niter) {
                 const int s1 = (it + 1) & 1;
+                TL(5);
                 if (!mbar_wait(bars + B_QFULL + s1, ((it + 1) >> 1) & 1, abortp, status, ERR_FULL)) break;
+                TL(6);
                 tc_fence_after();
                 if (lane == 0) issue_S(q_km0 + s1 * kSlot);
                 __syncwarp();
             }
+            TL(7);
             if (!mbar_wait(bars + B_DS, it & 1, abortp, status, ERR_PDS)) break;
+            TL(8);
             if (!kAliasDQ && it > 0 && !mbar_wait(bars + B_DQR, (it - 1) & 1, abortp, status, ERR_DQR)) break;
             tc_fence_after();
             if (lane == 0) {
+                if (it > 0) umma_ts2<true>(tbase + colDK, tbase + colDP, q_mn, mn_hi, idesc_acc);
+                else        umma_ts2<false>(tbase + colDK, tbase + colDP, q_mn, mn_hi, idesc_acc);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
+                for (int ks = 1; ks < 8; ++ks) {
                     const uint32_t a_col = 64 * (ks / 4) + 8 * (ks % 4);
-                    umma_ts(tbase + colDK, tbase + colDP + a_col, q_mn + moff(ks), idesc_acc, (it > 0 || ks > 0));
+                    umma_ts2<true>(tbase + colDK, tbase + colDP + a_col, q_mn + moff(ks), mn_hi, idesc_acc);
                 }
+                // 16 keys per step.  D = 128: dQ^T = K^T dS^T (lanes are d, columns are queries);
+                // D = 64: dQ = dS K (lanes are queries, columns are d)
+                if (kTransposeDQ) umma_ss2<false>(tbase + colDQ, k_mn, mn_hi, ds_mn, mn_hi, idesc_dqt);
+                else              umma_ss2<false>(tbase + colDQ, ds_mn, mn_hi, k_mn, mn_hi, idesc_dq);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {   // 16 keys per step
-                    if (kTransposeDQ)   // dQ^T = K^T dS^T: lanes are d, columns are queries
-                        umma_ss(tbase + colDQ, k_mn + moff(ks), ds_mn + moff(ks), idesc_dqt, ks > 0);
-                    else                // dQ = dS K: lanes are queries, columns are d
-                        umma_ss(tbase + colDQ, ds_mn + moff(ks), k_mn + moff(ks), idesc_dq, ks > 0);
+                for (int ks = 1; ks < 8; ++ks) {
+                    if (kTransposeDQ) umma_ss2<true>(tbase + colDQ, k_mn + moff(ks), mn_hi, ds_mn + moff(ks), mn_hi, idesc_dqt);
+                    else              umma_ss2<true>(tbase + colDQ, ds_mn + moff(ks), mn_hi, k_mn + moff(ks), mn_hi, idesc_dq);
                 }
                 umma_commit(bars + B_QEMPTY + s);
                 umma_commit(bars + B_DQ);
             }
+            TL(9);
             __syncwarp();
         }
       }
     } else if (warp >= kReduceWarp0) {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 152;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 144;");
         // ------------------------------------------------- dQ reduce warps: lanes are query rows
         const int lane_row = 32 * (warp % 4) + lane;
         const uint32_t lane_addr = tbase + ((uint32_t)(32 * (warp % 4)) << 16);
         for (int it = 0; it < niter; ++it) {
             const int qrow = (i_begin + it) * 128 + lane_row;
             if (!mbar_wait(bars + B_DQ, it & 1, abortp, status, ERR_DQ)) break;
+            if ((dbg & 8) && blockIdx.x == 0 && tid == kReduceWarp0 * 32 && it < 32) reinterpret_cast<long long *>(dQacc)[it * 16 + 10] = clock64();
             tc_fence_after();
             uint32_t r[D / 32][32];
             if (kTransposeDQ) {
@@ -313,6 +340,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 tc_wait_ld();
                 tc_fence_before();
                 mbar_arrive(bars + B_DQR);      // TMEM columns are free again; the reds go out from registers
+                if ((dbg & 8) && blockIdx.x == 0 && tid == kReduceWarp0 * 32 && it < 32) reinterpret_cast<long long *>(dQacc)[it * 16 + 11] = clock64();
                 if (!(dbg & 1)) {
                     const int valid = min(128, n - q0);
 #pragma unroll
@@ -340,7 +368,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         }
     } else {
         // ----------------------------------------------------------- elementwise warps 0-7
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 152;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 144;");
         const int wg = warp / 4;                          // which half of the query columns
         const int lane_row = 32 * (warp % 4) + lane;      // TMEM lane of this thread = key index in the tile
         const uint32_t lane_addr = tbase + ((uint32_t)(32 * (warp % 4)) << 16);
@@ -389,6 +417,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             const int s = it & 1;
             // dS-phase: dS^T = P^T o (dP^T - D)   (the factor `scale` is applied to dK and dQ at the end)
             if (!mbar_wait(bars + B_DP, it & 1, abortp, status, ERR_SDP)) { ok = false; break; }
+            if ((dbg & 8) && blockIdx.x == 0 && tid == 0 && it < 32) reinterpret_cast<long long *>(dQacc)[it * 16 + 12] = clock64();
             tc_fence_after();
             const float *Ds = sD + s * 128;
             if (!(dbg & 2))
@@ -423,7 +452,9 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             tc_fence_before();
             fence_proxy_async_smem();
             mbar_arrive(bars + B_DS);
+            if ((dbg & 8) && blockIdx.x == 0 && tid == 0 && it < 32) reinterpret_cast<long long *>(dQacc)[it * 16 + 13] = clock64();
             if (it + 1 < niter) ok = p_phase(it + 1);
+            if ((dbg & 8) && blockIdx.x == 0 && tid == 0 && it < 32) reinterpret_cast<long long *>(dQacc)[it * 16 + 14] = clock64();
         }
         if (ok && mbar_wait(bars + B_DQ, (niter - 1) & 1, abortp, status, ERR_DQ)) {
             // all UMMAs have completed: write dV and scale*dK rows of this key

@@ -107,15 +107,18 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         const uint64_t q_desc = smem_desc_sw128(smem_u32(sQ), 16, 1024);
         const uint64_t k_desc = smem_desc_sw128(smem_u32(sK), 16, 1024);
         const uint64_t v_desc = smem_desc_sw128(smem_u32(sV), kBoxBytes, 1024);   // MN-major
+        const uint32_t q_lo = (uint32_t)q_desc, k_lo = (uint32_t)k_desc, v_lo = (uint32_t)v_desc;
+        const uint32_t km_hi = (uint32_t)(q_desc >> 32), mn_hi = (uint32_t)(v_desc >> 32);
         bool ok = mbar_wait(&bar_q, 0, abortp, status, ERR_Q);
         for (int j = 0; ok && j < nkt; ++j) {
             if (!mbar_wait(&bar_k, j & 1, abortp, status, ERR_K)) break;
             tc_fence_after();
             if (lane == 0) {
+                umma_ss2<false>(tbase + kColS, q_lo, km_hi, k_lo, km_hi, idesc_s);
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint64_t off = (uint64_t)(((ks / 4) * kBoxBytes + (ks % 4) * 32) >> 4);
-                    umma_ss(tbase + kColS, q_desc + off, k_desc + off, idesc_s, ks > 0);
+                for (int ks = 1; ks < D / 16; ++ks) {
+                    const uint32_t off = (uint32_t)(((ks / 4) * kBoxBytes + (ks % 4) * 32) >> 4);
+                    umma_ss2<true>(tbase + kColS, q_lo + off, km_hi, k_lo + off, km_hi, idesc_s);
                 }
                 umma_commit(&bar_s);
             }
@@ -124,11 +127,11 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             if (!mbar_wait(&bar_p, j & 1, abortp, status, ERR_P)) break;
             tc_fence_after();
             if (lane == 0) {
+                if (j > 0) umma_ts2<true>(tbase + kColO, tbase + kColP, v_lo, mn_hi, idesc_pv);
+                else       umma_ts2<false>(tbase + kColO, tbase + kColP, v_lo, mn_hi, idesc_pv);
 #pragma unroll
-                for (int ks = 0; ks < BN / 16; ++ks) {
-                    umma_ts(tbase + kColO, tbase + kColP + ks * 8, v_desc + (uint64_t)((ks * 2048) >> 4), idesc_pv,
-                            (j > 0 || ks > 0));
-                }
+                for (int ks = 1; ks < BN / 16; ++ks)
+                    umma_ts2<true>(tbase + kColO, tbase + kColP + ks * 8, v_lo + (uint32_t)((ks * 2048) >> 4), mn_hi, idesc_pv);
                 umma_commit(&bar_o);
             }
             __syncwarp();
