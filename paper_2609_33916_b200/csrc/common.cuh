@@ -47,7 +47,8 @@ cudaError_t tc_bwd_preprocess(const Problem &p, const void *dO, const void *O, c
 // dK, dV; UNSCALED dQ contributions (dS K, without the factor scale) red-added into dQacc
 // (fp32 [B,H,n,d], pre-zeroed)
 cudaError_t tc_bwd_kv(const Problem &p, const void *Q, const void *K, const void *V, const void *dO,
-                      const float *Lp, const float *Dp, void *dK, void *dV, float *dQacc, cudaStream_t st);
+                      const float *Lp, const float *Dp, void *dK, void *dV, float *dQacc, int dq_bulk,
+                      cudaStream_t st);   // dq_bulk: TMA bulk add-reduce instead of red.global (d = 128 only)
 
 // ---- SIMT fp32 path (simt_kernels.cu) -------------------------------------------------
 // dtype: MOA_BF16 or MOA_F32 storage; arithmetic is fp32 FMA throughout.

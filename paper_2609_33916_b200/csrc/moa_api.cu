@@ -100,7 +100,10 @@ moa_status check_desc(const moa_attn_desc *d)
     if (tiles * d->B * d->H >= (1LL << 31)) return MOA_ERR_UNSUPPORTED;
     if (d->path == MOA_PATH_TC && d->dtype != MOA_BF16) return MOA_ERR_UNSUPPORTED;
     if (d->materialize) return MOA_ERR_UNSUPPORTED;           // comparison variant not built yet
-    if (d->dq_mode == MOA_DQ_BULK_REDUCE) return MOA_ERR_UNSUPPORTED;
+    // the bulk-reduce strategy exists in the tensor-core backward for d = 128 only
+    if (d->dq_mode == MOA_DQ_BULK_REDUCE &&
+        !(d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->d == 128 && d->scale > 0.f))
+        return MOA_ERR_UNSUPPORTED;
     if (d->path == MOA_PATH_TC && d->dq_mode == MOA_DQ_SEPARATE_PASS) return MOA_ERR_UNSUPPORTED;
     if (d->path == MOA_PATH_TC && !(d->scale > 0.f)) return MOA_ERR_UNSUPPORTED;   // non-positive scale: SIMT path only
     return MOA_OK;
@@ -112,7 +115,9 @@ int resolved_dq_mode(const moa_attn_desc *d) { return d->dq_mode == MOA_DQ_AUTO 
 bool use_tc_fwd(const moa_attn_desc *d) { return d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->scale > 0.f; }
 bool use_tc_bwd(const moa_attn_desc *d)
 {
-    return d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->scale > 0.f && resolved_dq_mode(d) == MOA_DQ_RED;
+    const int mode = resolved_dq_mode(d);
+    return d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->scale > 0.f &&
+           (mode == MOA_DQ_RED || mode == MOA_DQ_BULK_REDUCE);
 }
 
 // Workspace of the backward: [ D | Lp (tensor-core path only) | dQacc (bf16 with an atomic mode) ]
@@ -160,7 +165,7 @@ moa_status run_bwd(const moa_attn_desc *d, const void *Q, const void *K, const v
     if (use_tc_bwd(d)) {
         MOA_TRY(tc_bwd_preprocess(p, dO, O, L, Lp, Dv, st));
         MOA_TRY(cudaMemsetAsync(dQacc, 0, elems * sizeof(float), st));
-        MOA_TRY(tc_bwd_kv(p, Q, K, V, dO, Lp, Dv, dK, dV, dQacc, st));
+        MOA_TRY(tc_bwd_kv(p, Q, K, V, dO, Lp, Dv, dK, dV, dQacc, mode == MOA_DQ_BULK_REDUCE, st));
         MOA_TRY(convert_f32_to_bf16(dQacc, dQ, elems, p.scale, st));
         return MOA_OK;
     }

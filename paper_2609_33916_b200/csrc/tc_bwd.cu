@@ -32,7 +32,6 @@
 #include "common.cuh"
 #include "ptx.cuh"
 #include "tensormap.cuh"
-#include <cstdlib>
 
 namespace moa {
 namespace {
@@ -46,7 +45,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 
 enum : uint32_t {
     ERR_KV = 0x201, ERR_FULL = 0x202, ERR_EMPTY = 0x203, ERR_SDP = 0x204, ERR_PDS = 0x205, ERR_DQ = 0x206,
-    ERR_DQR = 0x207, ERR_ALIGN = 0x208
+    ERR_DQR = 0x207, ERR_ALIGN = 0x208, ERR_STAGE = 0x209
 };
 
 __device__ __forceinline__ void bulk_load_1d(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
@@ -100,15 +99,21 @@ __global__ void bwd_preprocess_kernel(const __nv_bfloat16 *__restrict__ dO, cons
     if (lane == 0) { Dp[prow] = acc; Lp[prow] = L[row] * kLog2e; }
 }
 
-template <int D>
+// kBulk: the dQ tile goes out through the TMA add-reduce; that needs 32 KB of staging, which is
+// taken from the second dO slot (dO_i is only read early in tile i, by dP and dV, so one slot
+// works, at the price of a later refill).  Without it dO has two slots like Q.
+template <int D, bool kBulk>
 struct BwdSmem {
     static constexpr int kTile = 128 * D * 2;        // K, V, Q_i, dO_i tiles
     static constexpr int kdS = 128 * 128 * 2;        // dS^T tile, [128 keys][128 queries] bf16
     static constexpr int offK = 0;
     static constexpr int offV = offK + kTile;
     static constexpr int offQ = offV + kTile;        // 2 slots
-    static constexpr int offdO = offQ + 2 * kTile;   // 2 slots
-    static constexpr int offdS = offdO + 2 * kTile;
+    static constexpr int kDoSlots = kBulk ? 1 : 2;
+    static constexpr int offdO = offQ + 2 * kTile;
+    static constexpr int offStage = offdO + kDoSlots * kTile;   // 2 x [32 rows][D] fp32 staging (kBulk only)
+    static constexpr int kStage = kBulk ? 32 * D * 4 : 0;
+    static constexpr int offdS = offStage + 2 * kStage;
     static constexpr int offL = offdS + kdS;         // 2 x 128 floats, travels with the Q slot
     static constexpr int offD = offL + 2 * 512;      // 2 x 128 floats, travels with the Q slot
     static constexpr int offBar = offD + 2 * 512;    // mbarriers + tmem base + abort flag
@@ -118,18 +123,21 @@ struct BwdSmem {
 // Barrier slots inside the shared-memory barrier block
 enum {
     B_KV = 0, B_QFULL = 1 /*2*/, B_QEMPTY = 3 /*2*/, B_DOFULL = 5 /*2*/, B_DOEMPTY = 7 /*2*/,
-    B_S = 9, B_P = 10, B_DP = 11, B_DS = 12, B_DQ = 13, B_DQR = 14, B_COUNT = 15
+    B_S = 9, B_P = 10, B_DP = 11, B_DS = 12, B_DQ = 13, B_DQR = 14, B_STGFREE = 15 /*2*/, B_STGFULL = 17 /*2*/,
+    B_COUNT = 19
 };
 
-template <int D>
+template <int D, bool kBulk>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
               const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapdO,
-              const float *__restrict__ Lp, const float *__restrict__ Dp,
+              const __grid_constant__ CUtensorMap mapdQ, const float *__restrict__ Lp, const float *__restrict__ Dp,
               __nv_bfloat16 *__restrict__ dK, __nv_bfloat16 *__restrict__ dV, float *__restrict__ dQacc,
-              int n, int n_pad, int causal, float scale, float scale_log2, int nkt, unsigned int *status, int dbg)
+              int n, int n_pad, int causal, float scale, float scale_log2, int nkt, unsigned int *status)
 {
-    using SM = BwdSmem<D>;
+    using SM = BwdSmem<D, kBulk>;
+    constexpr int kDoSlots = SM::kDoSlots;
+    constexpr bool dq_bulk = kBulk;
     constexpr int kBoxes = D / 64;
     constexpr int kBoxBytes = 128 * 128;
     constexpr bool kAliasDQ = (D == 128);   // dQ tile shares the dP^T columns
@@ -156,13 +164,15 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
 
     if (tid == 0) {
         for (int b = 0; b < B_COUNT; ++b) {
-            const uint32_t cnt = (b == B_P || b == B_DS) ? 256u : (b == B_DQR ? 128u : 1u);
+            const uint32_t cnt = (b == B_P || b == B_DS) ? 256u
+                               : (b == B_DQR || b == B_STGFULL || b == B_STGFULL + 1) ? 128u : 1u;
             mbar_init(bars + b, cnt);
         }
         *abortp = (smem_u32(sm) & 1023u) ? 1u : 0u;
         if (*abortp && status) atomicCAS(status, 0u, (unsigned)ERR_ALIGN);
         fence_mbar_init();
         prefetch_tensormap(&mapQ); prefetch_tensormap(&mapK); prefetch_tensormap(&mapV); prefetch_tensormap(&mapdO);
+        if (dq_bulk) prefetch_tensormap(&mapdQ);
     }
     if (warp == kMmaWarp) { tmem_alloc(tmem_base_s, kTmemCols); tmem_relinquish(); }
     tc_fence_before();
@@ -187,29 +197,42 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 tma_load_3d(sV + b * kBoxBytes, &mapV, bars + B_KV, 64 * b, k0, bh);
             }
         }
+        // Q tiles (with L, D) go through a two-slot ring and are fetched two tiles ahead: S(i+1) is
+        // issued in the middle of tile i.  dO has one slot: it is read only by dP(i) and dV(i),
+        // early in tile i, and is refilled as soon as dV(i) has completed.
+        auto load_q = [&](int it) {
+            const int s = it & 1, q0 = (i_begin + it) * 128;
+            uint8_t *sQ = sm + SM::offQ + s * SM::kTile;
+            mbar_arrive_expect_tx(bars + B_QFULL + s, SM::kTile + 1024);
+            for (int b = 0; b < kBoxes; ++b) tma_load_3d(sQ + b * kBoxBytes, &mapQ, bars + B_QFULL + s, 64 * b, q0, bh);
+            bulk_load_1d(sL + s * 128, Lp + (size_t)bh * n_pad + q0, 512, bars + B_QFULL + s);
+            bulk_load_1d(sD + s * 128, Dp + (size_t)bh * n_pad + q0, 512, bars + B_QFULL + s);
+        };
+        auto load_do = [&](int it) {
+            const int s = it % kDoSlots, q0 = (i_begin + it) * 128;
+            uint8_t *sdO = sm + SM::offdO + s * SM::kTile;
+            mbar_arrive_expect_tx(bars + B_DOFULL + s, SM::kTile);
+            for (int b = 0; b < kBoxes; ++b) tma_load_3d(sdO + b * kBoxBytes, &mapdO, bars + B_DOFULL + s, 64 * b, q0, bh);
+        };
+        if (lane == 0 && niter > 0) {
+            load_q(0);
+            load_do(0);
+            if (niter > 1) load_q(1);
+            if (kDoSlots == 2 && niter > 1) load_do(1);
+        }
         for (int it = 0; it < niter; ++it) {
-            const int s = it & 1;
-            const int q0 = (i_begin + it) * 128;
-            // dO slot first: it is released (after dV) earlier than the Q slot (after dK, dQ)
-            if (it >= 2 && !mbar_wait(bars + B_DOEMPTY + s, ((it >> 1) - 1) & 1, abortp, status, ERR_EMPTY)) break;
-            if (lane == 0) {
-                uint8_t *sdO = sm + SM::offdO + s * SM::kTile;
-                mbar_arrive_expect_tx(bars + B_DOFULL + s, SM::kTile);
-                for (int b = 0; b < kBoxes; ++b)
-                    tma_load_3d(sdO + b * kBoxBytes, &mapdO, bars + B_DOFULL + s, 64 * b, q0, bh);
+            if (it + kDoSlots < niter) {     // dV(it) done: its dO slot takes tile it + kDoSlots
+                if (!mbar_wait(bars + B_DOEMPTY + it % kDoSlots, (it / kDoSlots) & 1, abortp, status, ERR_EMPTY)) break;
+                if (lane == 0) load_do(it + kDoSlots);
             }
-            if (it >= 2 && !mbar_wait(bars + B_QEMPTY + s, ((it >> 1) - 1) & 1, abortp, status, ERR_EMPTY)) break;
-            if (lane == 0) {
-                uint8_t *sQ = sm + SM::offQ + s * SM::kTile;
-                mbar_arrive_expect_tx(bars + B_QFULL + s, SM::kTile + 1024);
-                for (int b = 0; b < kBoxes; ++b)
-                    tma_load_3d(sQ + b * kBoxBytes, &mapQ, bars + B_QFULL + s, 64 * b, q0, bh);
-                bulk_load_1d(sL + s * 128, Lp + (size_t)bh * n_pad + q0, 512, bars + B_QFULL + s);
-                bulk_load_1d(sD + s * 128, Dp + (size_t)bh * n_pad + q0, 512, bars + B_QFULL + s);
+            if (it + 2 < niter) {     // dK(it) done: its Q slot takes tile it+2
+                if (!mbar_wait(bars + B_QEMPTY + (it & 1), (it >> 1) & 1, abortp, status, ERR_EMPTY)) break;
+                if (lane == 0) load_q(it + 2);
             }
             __syncwarp();
         }
-      } else if (warp == kMmaWarp) {
+      } else if (warp == kMmaWarp && lane == 0) {
+        // the whole role runs in one thread: no warp re-convergence between waits and issues
         // ------------------------------------------------------------------- UMMA issuer
         // Issue order per query tile i:  dP(i), dV(i), S(i+1), dK(i), dQ(i).
         constexpr uint32_t idesc_st = idesc_bf16_f32(128, 128, 0, 0);   // S^T, dP^T
@@ -244,19 +267,13 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         if (ok) {
             tc_fence_after();
             if (lane == 0) issue_S(q_km0);
-            __syncwarp();
         }
-        long long *tl = reinterpret_cast<long long *>(dQacc);
-        const bool rec = (dbg & 8) && blockIdx.x == 0 && lane == 0;
-#define TL(slot) do { if (rec && it < 32) tl[it * 16 + (slot)] = clock64(); } while (0)
         for (int it = 0; ok && it < niter; ++it) {
             const int s = it & 1;
-            TL(0);
-            const uint32_t q_mn = q_mn0 + s * kSlot, do_km = do_km0 + s * kSlot, do_mn = do_mn0 + s * kSlot;
-            if (!mbar_wait(bars + B_DOFULL + s, (it >> 1) & 1, abortp, status, ERR_FULL)) break;
-            TL(1);
+            const int sdo = it % kDoSlots;
+            const uint32_t q_mn = q_mn0 + s * kSlot, do_km = do_km0 + sdo * kSlot, do_mn = do_mn0 + sdo * kSlot;
+            if (!mbar_wait(bars + B_DOFULL + sdo, (it / kDoSlots) & 1, abortp, status, ERR_FULL)) break;
             if (kAliasDQ && it > 0 && !mbar_wait(bars + B_DQR, (it - 1) & 1, abortp, status, ERR_DQR)) break;
-            TL(2);
             tc_fence_after();
             if (lane == 0) {
                 umma_ss2<false>(tbase + colDP, v_km, km_hi, do_km, km_hi, idesc_st);
@@ -265,10 +282,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                     umma_ss2<true>(tbase + colDP, v_km + koff(ks), km_hi, do_km + koff(ks), km_hi, idesc_st);
                 umma_commit(bars + B_DP);
             }
-            __syncwarp();
-            TL(3);
             if (!mbar_wait(bars + B_P, it & 1, abortp, status, ERR_PDS)) break;
-            TL(4);
             tc_fence_after();
             if (lane == 0) {
                 // 16 queries per step; the very first UMMA of the CTA overwrites the accumulator
@@ -279,21 +293,15 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                     const uint32_t a_col = 64 * (ks / 4) + 8 * (ks % 4);
                     umma_ts2<true>(tbase + colDV, tbase + colS + a_col, do_mn + moff(ks), mn_hi, idesc_acc);
                 }
-                umma_commit(bars + B_DOEMPTY + s);
+                umma_commit(bars + B_DOEMPTY + sdo);
             }
-            __syncwarp();
             if (it + 1 < niter) {
                 const int s1 = (it + 1) & 1;
-                TL(5);
                 if (!mbar_wait(bars + B_QFULL + s1, ((it + 1) >> 1) & 1, abortp, status, ERR_FULL)) break;
-                TL(6);
                 tc_fence_after();
                 if (lane == 0) issue_S(q_km0 + s1 * kSlot);
-                __syncwarp();
-            }
-            TL(7);
+                }
             if (!mbar_wait(bars + B_DS, it & 1, abortp, status, ERR_PDS)) break;
-            TL(8);
             if (!kAliasDQ && it > 0 && !mbar_wait(bars + B_DQR, (it - 1) & 1, abortp, status, ERR_DQR)) break;
             tc_fence_after();
             if (lane == 0) {
@@ -304,6 +312,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                     const uint32_t a_col = 64 * (ks / 4) + 8 * (ks % 4);
                     umma_ts2<true>(tbase + colDK, tbase + colDP + a_col, q_mn + moff(ks), mn_hi, idesc_acc);
                 }
+                umma_commit(bars + B_QEMPTY + s);   // Q slot is free once dK is done (dQ does not read it)
                 // 16 keys per step.  D = 128: dQ^T = K^T dS^T (lanes are d, columns are queries);
                 // D = 64: dQ = dS K (lanes are queries, columns are d)
                 if (kTransposeDQ) umma_ss2<false>(tbase + colDQ, k_mn, mn_hi, ds_mn, mn_hi, idesc_dqt);
@@ -313,11 +322,8 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                     if (kTransposeDQ) umma_ss2<true>(tbase + colDQ, k_mn + moff(ks), mn_hi, ds_mn + moff(ks), mn_hi, idesc_dqt);
                     else              umma_ss2<true>(tbase + colDQ, ds_mn + moff(ks), mn_hi, k_mn + moff(ks), mn_hi, idesc_dq);
                 }
-                umma_commit(bars + B_QEMPTY + s);
                 umma_commit(bars + B_DQ);
             }
-            TL(9);
-            __syncwarp();
         }
       }
     } else if (warp >= kReduceWarp0) {
@@ -328,7 +334,6 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         for (int it = 0; it < niter; ++it) {
             const int qrow = (i_begin + it) * 128 + lane_row;
             if (!mbar_wait(bars + B_DQ, it & 1, abortp, status, ERR_DQ)) break;
-            if ((dbg & 8) && blockIdx.x == 0 && tid == kReduceWarp0 * 32 && it < 32) reinterpret_cast<long long *>(dQacc)[it * 16 + 10] = clock64();
             tc_fence_after();
             uint32_t r[D / 32][32];
             if (kTransposeDQ) {
@@ -340,8 +345,36 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 tc_wait_ld();
                 tc_fence_before();
                 mbar_arrive(bars + B_DQR);      // TMEM columns are free again; the reds go out from registers
-                if ((dbg & 8) && blockIdx.x == 0 && tid == kReduceWarp0 * 32 && it < 32) reinterpret_cast<long long *>(dQacc)[it * 16 + 11] = clock64();
-                if (!(dbg & 1)) {
+                if (dq_bulk) {
+                    // Stage 32 query rows x 128 floats at a time in shared memory (this thread writes
+                    // column lane_row of each row: conflict-free) and hand each stage to the TMA engine
+                    // as one add-reduce into the fp32 accumulator; rows past n are clipped by the map.
+                    // All hand-offs inside the reduce group go through bounded mbarrier waits
+                    // (no named barriers), so a timed-out CTA can still drain.
+                    const bool leader = (tid == kReduceWarp0 * 32);
+                    bool stage_ok = true;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const int g = it * 4 + c, st = c & 1;       // g: running chunk count, two stages
+                        float *stage = reinterpret_cast<float *>(sm + SM::offStage + st * SM::kStage);
+                        if (g >= 2) {
+                            if (leader) { bulk_wait_read<1>(); mbar_arrive(bars + B_STGFREE + st); }   // TMA has read the stage
+                            if (stage_ok && !mbar_wait(bars + B_STGFREE + st, ((g >> 1) - 1) & 1, abortp, status, ERR_STAGE))
+                                stage_ok = false;
+                        }
+                        if (stage_ok) {
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) stage[e * D + lane_row] = __uint_as_float(r[c][e]);
+                            fence_proxy_async_smem();
+                        }
+                        mbar_arrive(bars + B_STGFULL + st);
+                        if (leader && stage_ok && mbar_wait(bars + B_STGFULL + st, (g >> 1) & 1, abortp, status, ERR_STAGE)) {
+                            tma_reduce_add_3d(&mapdQ, stage, 0, q0 + 32 * c, bh);
+                            bulk_commit();
+                        }
+                    }
+                    if (!stage_ok) break;
+                } else {
                     const int valid = min(128, n - q0);
 #pragma unroll
                     for (int c = 0; c < 4; ++c)
@@ -356,7 +389,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 tc_wait_ld();
                 tc_fence_before();
                 mbar_arrive(bars + B_DQR);
-                if (qrow < n && !(dbg & 1)) {
+                if (qrow < n) {
 #pragma unroll
                     for (int c = 0; c < D / 32; ++c)
 #pragma unroll
@@ -366,6 +399,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 }
             }
         }
+        if (kTransposeDQ && dq_bulk && tid == kReduceWarp0 * 32) bulk_wait<0>();   // all reduces done before exit
     } else {
         // ----------------------------------------------------------- elementwise warps 0-7
         asm volatile("setmaxnreg.inc.sync.aligned.u32 144;");
@@ -383,7 +417,6 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             if (!mbar_wait(bars + B_S, it & 1, abortp, status, ERR_SDP)) return false;
             tc_fence_after();
             const float *Ls = sL + s * 128;
-            if (!(dbg & 2))
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 const int qc0 = 64 * wg + 32 * c;
@@ -417,10 +450,8 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             const int s = it & 1;
             // dS-phase: dS^T = P^T o (dP^T - D)   (the factor `scale` is applied to dK and dQ at the end)
             if (!mbar_wait(bars + B_DP, it & 1, abortp, status, ERR_SDP)) { ok = false; break; }
-            if ((dbg & 8) && blockIdx.x == 0 && tid == 0 && it < 32) reinterpret_cast<long long *>(dQacc)[it * 16 + 12] = clock64();
             tc_fence_after();
             const float *Ds = sD + s * 128;
-            if (!(dbg & 2))
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 const int qc0 = 64 * wg + 32 * c;
@@ -452,9 +483,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             tc_fence_before();
             fence_proxy_async_smem();
             mbar_arrive(bars + B_DS);
-            if ((dbg & 8) && blockIdx.x == 0 && tid == 0 && it < 32) reinterpret_cast<long long *>(dQacc)[it * 16 + 13] = clock64();
             if (it + 1 < niter) ok = p_phase(it + 1);
-            if ((dbg & 8) && blockIdx.x == 0 && tid == 0 && it < 32) reinterpret_cast<long long *>(dQacc)[it * 16 + 14] = clock64();
         }
         if (ok && mbar_wait(bars + B_DQ, (niter - 1) & 1, abortp, status, ERR_DQ)) {
             // all UMMAs have completed: write dV and scale*dK rows of this key
@@ -490,25 +519,28 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     if (warp == kMmaWarp) tmem_dealloc(tbase, kTmemCols);
 }
 
-template <int D>
+template <int D, bool kBulk>
 cudaError_t launch_bwd(const Problem &p, const void *Q, const void *K, const void *V, const void *dO,
                        const float *Lp, const float *Dp, void *dK, void *dV, float *dQacc, cudaStream_t st)
 {
-    CUtensorMap mq, mk, mv, mdo;
+    CUtensorMap mq, mk, mv, mdo, mdq;
     const uint64_t heads = (uint64_t)p.BH();
     if (!make_tensor_map_3d(&mq, Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
         !make_tensor_map_3d(&mk, K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
         !make_tensor_map_3d(&mv, V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
         !make_tensor_map_3d(&mdo, dO, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64))
         return cudaErrorInvalidValue;
-    constexpr int kSmem = BwdSmem<D>::kTotal;
-    cudaError_t e = cudaFuncSetAttribute(tc_bwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    // fp32 accumulator as [heads, n, D] with boxes of 32 rows x D floats (no swizzle); also encoded when unused
+    if (!make_tensor_map_3d(&mdq, dQacc, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, heads, p.n, D, 32, D))
+        return cudaErrorInvalidValue;
+    constexpr int kSmem = BwdSmem<D, kBulk>::kTotal;
+    cudaError_t e = cudaFuncSetAttribute(tc_bwd_kernel<D, kBulk>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
     const int nkt = (p.n + 127) / 128;
     LaunchScope scope(MOA_KERNEL_BWD_KV, st);
-    tc_bwd_kernel<D><<<(unsigned)(nkt * p.BH()), kThreads, kSmem, st>>>(
-        mq, mk, mv, mdo, Lp, Dp, (__nv_bfloat16 *)dK, (__nv_bfloat16 *)dV, dQacc, p.n, nkt * 128, p.causal,
-        p.scale, p.scale * kLog2e, nkt, device_status_ptr(), getenv("MOA_BWD_DEBUG") ? atoi(getenv("MOA_BWD_DEBUG")) : 0);
+    tc_bwd_kernel<D, kBulk><<<(unsigned)(nkt * p.BH()), kThreads, kSmem, st>>>(
+        mq, mk, mv, mdo, mdq, Lp, Dp, (__nv_bfloat16 *)dK, (__nv_bfloat16 *)dV, dQacc, p.n, nkt * 128, p.causal,
+        p.scale, p.scale * kLog2e, nkt, device_status_ptr());
     return cudaGetLastError();
 }
 
@@ -532,10 +564,11 @@ cudaError_t tc_bwd_preprocess(const Problem &p, const void *dO, const void *O, c
 }
 
 cudaError_t tc_bwd_kv(const Problem &p, const void *Q, const void *K, const void *V, const void *dO,
-                      const float *Lp, const float *Dp, void *dK, void *dV, float *dQacc, cudaStream_t st)
+                      const float *Lp, const float *Dp, void *dK, void *dV, float *dQacc, int dq_bulk, cudaStream_t st)
 {
-    if (p.d == 64) return launch_bwd<64>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
-    if (p.d == 128) return launch_bwd<128>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
+    if (p.d == 64 && !dq_bulk) return launch_bwd<64, false>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
+    if (p.d == 128 && !dq_bulk) return launch_bwd<128, false>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
+    if (p.d == 128 && dq_bulk) return launch_bwd<128, true>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
     return cudaErrorInvalidValue;
 }
 
