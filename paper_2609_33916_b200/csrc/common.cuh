@@ -45,10 +45,14 @@ cudaError_t tc_fwd(const Problem &p, const void *Q, const void *K, const void *V
 cudaError_t tc_bwd_preprocess(const Problem &p, const void *dO, const void *O, const float *L, float *Lp, float *Dp,
                               cudaStream_t st);
 // dK, dV; UNSCALED dQ contributions (dS K, without the factor scale) red-added into dQacc
-// (fp32 [B,H,n,d], pre-zeroed)
+// (fp32 [B,H,n,d], pre-zeroed); dQacc == nullptr skips the dQ contraction altogether
 cudaError_t tc_bwd_kv(const Problem &p, const void *Q, const void *K, const void *V, const void *dO,
                       const float *Lp, const float *Dp, void *dK, void *dV, float *dQacc, int dq_bulk,
                       cudaStream_t st);   // dq_bulk: TMA bulk add-reduce instead of red.global (d = 128 only)
+
+// atomic-free query-parallel dQ pass on the tensor cores (tc_dq.cu); writes dQ (bf16) directly
+cudaError_t tc_bwd_dq(const Problem &p, const void *Q, const void *K, const void *V, const void *dO,
+                      const float *Lp, const float *Dp, void *dQ, cudaStream_t st);
 
 // ---- SIMT fp32 path (simt_kernels.cu) -------------------------------------------------
 // dtype: MOA_BF16 or MOA_F32 storage; arithmetic is fp32 FMA throughout.

@@ -104,7 +104,6 @@ moa_status check_desc(const moa_attn_desc *d)
     if (d->dq_mode == MOA_DQ_BULK_REDUCE &&
         !(d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->d == 128 && d->scale > 0.f))
         return MOA_ERR_UNSUPPORTED;
-    if (d->path == MOA_PATH_TC && d->dq_mode == MOA_DQ_SEPARATE_PASS) return MOA_ERR_UNSUPPORTED;
     if (d->path == MOA_PATH_TC && !(d->scale > 0.f)) return MOA_ERR_UNSUPPORTED;   // non-positive scale: SIMT path only
     return MOA_OK;
 }
@@ -117,7 +116,7 @@ bool use_tc_bwd(const moa_attn_desc *d)
 {
     const int mode = resolved_dq_mode(d);
     return d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->scale > 0.f &&
-           (mode == MOA_DQ_RED || mode == MOA_DQ_BULK_REDUCE);
+           (mode == MOA_DQ_RED || mode == MOA_DQ_BULK_REDUCE || mode == MOA_DQ_SEPARATE_PASS);
 }
 
 // Workspace of the backward: [ D | Lp (tensor-core path only) | dQacc (bf16 with an atomic mode) ]
@@ -164,6 +163,11 @@ moa_status run_bwd(const moa_attn_desc *d, const void *Q, const void *K, const v
 #define MOA_TRY(x) do { if ((x) != cudaSuccess) return MOA_ERR_CUDA; } while (0)
     if (use_tc_bwd(d)) {
         MOA_TRY(tc_bwd_preprocess(p, dO, O, L, Lp, Dv, st));
+        if (mode == MOA_DQ_SEPARATE_PASS) {
+            MOA_TRY(tc_bwd_kv(p, Q, K, V, dO, Lp, Dv, dK, dV, nullptr, 0, st));
+            MOA_TRY(tc_bwd_dq(p, Q, K, V, dO, Lp, Dv, dQ, st));
+            return MOA_OK;
+        }
         MOA_TRY(cudaMemsetAsync(dQacc, 0, elems * sizeof(float), st));
         MOA_TRY(tc_bwd_kv(p, Q, K, V, dO, Lp, Dv, dK, dV, dQacc, mode == MOA_DQ_BULK_REDUCE, st));
         MOA_TRY(convert_f32_to_bf16(dQacc, dQ, elems, p.scale, st));

@@ -133,7 +133,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
               const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapdO,
               const __grid_constant__ CUtensorMap mapdQ, const float *__restrict__ Lp, const float *__restrict__ Dp,
               __nv_bfloat16 *__restrict__ dK, __nv_bfloat16 *__restrict__ dV, float *__restrict__ dQacc,
-              int n, int n_pad, int causal, float scale, float scale_log2, int nkt, unsigned int *status)
+              int n, int n_pad, int causal, float scale, float scale_log2, int nkt, int skip_dq, unsigned int *status)
 {
     using SM = BwdSmem<D, kBulk>;
     constexpr int kDoSlots = SM::kDoSlots;
@@ -273,7 +273,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             const int sdo = it % kDoSlots;
             const uint32_t q_mn = q_mn0 + s * kSlot, do_km = do_km0 + sdo * kSlot, do_mn = do_mn0 + sdo * kSlot;
             if (!mbar_wait(bars + B_DOFULL + sdo, (it / kDoSlots) & 1, abortp, status, ERR_FULL)) break;
-            if (kAliasDQ && it > 0 && !mbar_wait(bars + B_DQR, (it - 1) & 1, abortp, status, ERR_DQR)) break;
+            if (kAliasDQ && !skip_dq && it > 0 && !mbar_wait(bars + B_DQR, (it - 1) & 1, abortp, status, ERR_DQR)) break;
             tc_fence_after();
             if (lane == 0) {
                 umma_ss2<false>(tbase + colDP, v_km, km_hi, do_km, km_hi, idesc_st);
@@ -302,7 +302,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 if (lane == 0) issue_S(q_km0 + s1 * kSlot);
                 }
             if (!mbar_wait(bars + B_DS, it & 1, abortp, status, ERR_PDS)) break;
-            if (!kAliasDQ && it > 0 && !mbar_wait(bars + B_DQR, (it - 1) & 1, abortp, status, ERR_DQR)) break;
+            if (!kAliasDQ && !skip_dq && it > 0 && !mbar_wait(bars + B_DQR, (it - 1) & 1, abortp, status, ERR_DQR)) break;
             tc_fence_after();
             if (lane == 0) {
                 if (it > 0) umma_ts2<true>(tbase + colDK, tbase + colDP, q_mn, mn_hi, idesc_acc);
@@ -315,12 +315,14 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 umma_commit(bars + B_QEMPTY + s);   // Q slot is free once dK is done (dQ does not read it)
                 // 16 keys per step.  D = 128: dQ^T = K^T dS^T (lanes are d, columns are queries);
                 // D = 64: dQ = dS K (lanes are queries, columns are d)
-                if (kTransposeDQ) umma_ss2<false>(tbase + colDQ, k_mn, mn_hi, ds_mn, mn_hi, idesc_dqt);
-                else              umma_ss2<false>(tbase + colDQ, ds_mn, mn_hi, k_mn, mn_hi, idesc_dq);
+                if (!skip_dq) {   // (the atomic-free mode computes dQ in its own query-parallel kernel)
+                    if (kTransposeDQ) umma_ss2<false>(tbase + colDQ, k_mn, mn_hi, ds_mn, mn_hi, idesc_dqt);
+                    else              umma_ss2<false>(tbase + colDQ, ds_mn, mn_hi, k_mn, mn_hi, idesc_dq);
 #pragma unroll
-                for (int ks = 1; ks < 8; ++ks) {
-                    if (kTransposeDQ) umma_ss2<true>(tbase + colDQ, k_mn + moff(ks), mn_hi, ds_mn + moff(ks), mn_hi, idesc_dqt);
-                    else              umma_ss2<true>(tbase + colDQ, ds_mn + moff(ks), mn_hi, k_mn + moff(ks), mn_hi, idesc_dq);
+                    for (int ks = 1; ks < 8; ++ks) {
+                        if (kTransposeDQ) umma_ss2<true>(tbase + colDQ, k_mn + moff(ks), mn_hi, ds_mn + moff(ks), mn_hi, idesc_dqt);
+                        else              umma_ss2<true>(tbase + colDQ, ds_mn + moff(ks), mn_hi, k_mn + moff(ks), mn_hi, idesc_dq);
+                    }
                 }
                 umma_commit(bars + B_DQ);
             }
@@ -331,7 +333,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         // ------------------------------------------------- dQ reduce warps: lanes are query rows
         const int lane_row = 32 * (warp % 4) + lane;
         const uint32_t lane_addr = tbase + ((uint32_t)(32 * (warp % 4)) << 16);
-        for (int it = 0; it < niter; ++it) {
+        for (int it = 0; it < (skip_dq ? 0 : niter); ++it) {
             const int qrow = (i_begin + it) * 128 + lane_row;
             if (!mbar_wait(bars + B_DQ, it & 1, abortp, status, ERR_DQ)) break;
             tc_fence_after();
@@ -531,7 +533,7 @@ cudaError_t launch_bwd(const Problem &p, const void *Q, const void *K, const voi
         !make_tensor_map_3d(&mdo, dO, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64))
         return cudaErrorInvalidValue;
     // fp32 accumulator as [heads, n, D] with boxes of 32 rows x D floats (no swizzle); also encoded when unused
-    if (!make_tensor_map_3d(&mdq, dQacc, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, heads, p.n, D, 32, D))
+    if (!make_tensor_map_3d(&mdq, dQacc ? (const void *)dQacc : Q, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, heads, p.n, D, 32, D))
         return cudaErrorInvalidValue;
     constexpr int kSmem = BwdSmem<D, kBulk>::kTotal;
     cudaError_t e = cudaFuncSetAttribute(tc_bwd_kernel<D, kBulk>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
@@ -540,7 +542,7 @@ cudaError_t launch_bwd(const Problem &p, const void *Q, const void *K, const voi
     LaunchScope scope(MOA_KERNEL_BWD_KV, st);
     tc_bwd_kernel<D, kBulk><<<(unsigned)(nkt * p.BH()), kThreads, kSmem, st>>>(
         mq, mk, mv, mdo, mdq, Lp, Dp, (__nv_bfloat16 *)dK, (__nv_bfloat16 *)dV, dQacc, p.n, nkt * 128, p.causal,
-        p.scale, p.scale * kLog2e, nkt, device_status_ptr());
+        p.scale, p.scale * kLog2e, nkt, dQacc == nullptr ? 1 : 0, device_status_ptr());
     return cudaGetLastError();
 }
 

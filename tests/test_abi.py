@@ -44,7 +44,7 @@ def test_workspace_is_linear_in_n(lib):
         return mb.moa_attn_workspace_bytes(mb.make_desc(1, 32, n, 128, True, 0.1, dtype, mode), mb.MOA_OP_FUSED)
     assert ws(512, mb.MOA_DQ_RED) == 2 * 32 * 512 * 4 + 32 * 512 * 128 * 4
     assert ws(32768) == 64 * ws(512)                      # O(n d): no n^2 term
-    assert ws(512, mb.MOA_DQ_SEPARATE_PASS) == 32 * 512 * 4
+    assert ws(512, mb.MOA_DQ_SEPARATE_PASS) == 2 * 32 * 512 * 4
     assert ws(512, mb.MOA_DQ_RED, mb.MOA_F32) == 32 * 512 * 4
     assert mb.moa_attn_workspace_bytes(mb.make_desc(1, 32, 512, 128, True, 0.1), mb.MOA_OP_FWD) == 0
 

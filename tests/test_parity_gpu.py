@@ -69,7 +69,7 @@ BF16_CASES = [
 
 
 @pytest.mark.parametrize("B,Hh,n,d,causal", BF16_CASES)
-@pytest.mark.parametrize("path,dq_mode", [(1, 1), (1, 3), (2, 1), (0, 3), (2, 2)])
+@pytest.mark.parametrize("path,dq_mode", [(1, 1), (1, 3), (2, 1), (2, 3), (2, 2)])
 def test_bf16_shapes(H, B, Hh, n, d, causal, dq_mode, path):
     if dq_mode == 2 and d != 128:
         pytest.skip("TMA bulk-reduce dQ exists for d = 128 only")
@@ -104,18 +104,20 @@ def test_tc_forward_large_scores(H):
     assert mi.rel_err(got["L"], ref["L"]) <= 1e-3
 
 
-def test_fused_call_equals_fwd_then_bwd(H):
+@pytest.mark.parametrize("path", [1, 2])
+def test_fused_call_equals_fwd_then_bwd(H, path):
     inp = mi.make_inputs(2, 2, 320, 128, seed=5, dtype="bf16")
-    a = H.run_library(inp, "bf16", True, 0.09, op="fused", dq_mode=3)
-    b = H.run_library(inp, "bf16", True, 0.09, op="split", dq_mode=3)
+    a = H.run_library(inp, "bf16", True, 0.09, op="fused", dq_mode=3, path=path)
+    b = H.run_library(inp, "bf16", True, 0.09, op="split", dq_mode=3, path=path)
     for k in ("O", "L", "dQ", "dK", "dV"):
         np.testing.assert_array_equal(a[k], b[k], err_msg=k)
 
 
-def test_separate_pass_is_bitwise_reproducible(H):
+@pytest.mark.parametrize("path", [1, 2])
+def test_separate_pass_is_bitwise_reproducible(H, path):
     inp = mi.make_inputs(1, 4, 512, 64, seed=6, dtype="bf16")
-    a = H.run_library(inp, "bf16", False, 0.125, dq_mode=3)
-    b = H.run_library(inp, "bf16", False, 0.125, dq_mode=3)
+    a = H.run_library(inp, "bf16", False, 0.125, dq_mode=3, path=path)
+    b = H.run_library(inp, "bf16", False, 0.125, dq_mode=3, path=path)
     for k in ("O", "L", "dQ", "dK", "dV"):
         np.testing.assert_array_equal(a[k], b[k], err_msg=k)
 
@@ -184,3 +186,23 @@ def test_c3_causal_mid_sampled(H):
 def test_c5_causal_sweep_small_sizes_sampled(H, n):
     w = mi.CONFIGS[f"c5_causal_n{n}"]
     _sampled_check(H, w, heads=[(0, 0), (0, 31)])
+
+
+def test_c4_long_full_size_sampled(H):
+    """Config 4 at full size, in the configuration the benchmark times (fused call, default
+    modes): sampled rows/columns of the first and last head against the oracle, invariants on
+    all heads."""
+    w = mi.CONFIGS["c4_long"]
+    _sampled_check(H, w, heads=[(0, 0), (0, 15)], nrows=16, ncols=16)
+
+
+@pytest.mark.parametrize("n", [8192, 32768])
+def test_c5_causal_sweep_large_sizes_sampled(H, n):
+    w = mi.CONFIGS[f"c5_causal_n{n}"]
+    _sampled_check(H, w, heads=[(0, 31)] if n > 8192 else [(0, 0), (0, 31)], nrows=12, ncols=12)
+
+
+@pytest.mark.parametrize("dq_mode", [2, 3])
+def test_c3_other_dq_modes_sampled(H, dq_mode):
+    w = mi.CONFIGS["c3_causal_mid"]
+    _sampled_check(H, w, heads=[(1, 7)], dq_mode=dq_mode)
