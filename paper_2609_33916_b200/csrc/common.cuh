@@ -54,6 +54,13 @@ cudaError_t tc_bwd_kv(const Problem &p, const void *Q, const void *K, const void
 cudaError_t tc_bwd_dq(const Problem &p, const void *Q, const void *K, const void *V, const void *dO,
                       const float *Lp, const float *Dp, void *dQ, cudaStream_t st);
 
+// ---- n x n-materialising comparison variant (tc_materialize.cu), bf16 --------------------
+// P^T and dS^T are [heads][n_pad][n_pad] bf16 arrays in the caller's workspace.
+cudaError_t mat_fwd(const Problem &p, const void *Q, const void *K, const void *V, void *O, float *L, void *PT,
+                    cudaStream_t st);
+cudaError_t mat_bwd(const Problem &p, const void *Q, const void *K, const void *V, const void *dO, const float *Dp,
+                    const void *PT, void *GST, void *dQ, void *dK, void *dV, cudaStream_t st);
+
 // ---- SIMT fp32 path (simt_kernels.cu) -------------------------------------------------
 // dtype: MOA_BF16 or MOA_F32 storage; arithmetic is fp32 FMA throughout.
 cudaError_t simt_fwd(const Problem &p, int dtype, const void *Q, const void *K, const void *V,

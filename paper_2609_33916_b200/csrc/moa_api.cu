@@ -99,7 +99,8 @@ moa_status check_desc(const moa_attn_desc *d)
     const long long tiles = ((long long)d->n + 63) / 64;
     if (tiles * d->B * d->H >= (1LL << 31)) return MOA_ERR_UNSUPPORTED;
     if (d->path == MOA_PATH_TC && d->dtype != MOA_BF16) return MOA_ERR_UNSUPPORTED;
-    if (d->materialize) return MOA_ERR_UNSUPPORTED;           // comparison variant not built yet
+    // the materialising comparison variant runs on the tensor-core path only
+    if (d->materialize && !(d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->scale > 0.f)) return MOA_ERR_UNSUPPORTED;
     // the bulk-reduce strategy exists in the tensor-core backward for d = 128 only
     if (d->dq_mode == MOA_DQ_BULK_REDUCE &&
         !(d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->d == 128 && d->scale > 0.f))
@@ -140,7 +141,60 @@ BwdWorkspace bwd_workspace(const moa_attn_desc *d)
     return w;
 }
 
+// Materialising variant: heads are processed in groups so that the two n x n arrays (P^T, dS^T,
+// bf16, row stride n_pad) of one group stay under kMatCapBytes.
+constexpr size_t kMatCapBytes = (size_t)16 << 30;
+struct MatWorkspace {
+    int group;            // heads per group
+    size_t npad, arr_bytes /* one array, one group */, lp_bytes, d_bytes, total;
+};
+MatWorkspace mat_workspace(const moa_attn_desc *d, int op)
+{
+    MatWorkspace w{};
+    const size_t heads = (size_t)d->B * d->H;
+    w.npad = ((size_t)d->n + 127) / 128 * 128;
+    const size_t per_head = w.npad * w.npad * 2;
+    size_t g = kMatCapBytes / (2 * per_head);
+    if (g < 1) g = 1;
+    if (g > heads) g = heads;
+    w.group = (int)g;
+    w.arr_bytes = align_up(g * per_head);
+    w.lp_bytes = align_up(g * w.npad * sizeof(float));
+    w.d_bytes = w.lp_bytes;
+    w.total = op == MOA_OP_FWD ? w.arr_bytes : 2 * w.arr_bytes + w.lp_bytes + w.d_bytes;
+    return w;
+}
+
 Problem to_problem(const moa_attn_desc *d) { return Problem{d->B, d->H, d->n, d->d, d->causal, d->scale}; }
+
+// Materialising variant.  with_bwd = false: forward only (P^T is written and dropped).
+moa_status run_materialized(const moa_attn_desc *d, const void *Q, const void *K, const void *V, const void *dO,
+                            void *O, float *L, void *dQ, void *dK, void *dV, void *ws, bool with_bwd, cudaStream_t st)
+{
+    const MatWorkspace w = mat_workspace(d, with_bwd ? MOA_OP_FUSED : MOA_OP_FWD);
+    char *base = (char *)ws;
+    void *PT = base;
+    void *GST = base + w.arr_bytes;
+    float *Lp = (float *)(base + 2 * w.arr_bytes);
+    float *Dp = (float *)(base + 2 * w.arr_bytes + w.lp_bytes);
+    const int heads = d->B * d->H;
+    const size_t esz = 2, hs = (size_t)d->n * d->d * esz;
+    for (int g0 = 0; g0 < heads; g0 += w.group) {
+        const int g = heads - g0 < w.group ? heads - g0 : w.group;
+        Problem p{1, g, d->n, d->d, d->causal, d->scale};
+        const char *q = (const char *)Q + g0 * hs, *k = (const char *)K + g0 * hs, *v = (const char *)V + g0 * hs;
+        char *o = (char *)O + g0 * hs;
+        float *l = L + (size_t)g0 * d->n;
+        if (mat_fwd(p, q, k, v, o, l, PT, st) != cudaSuccess) return MOA_ERR_CUDA;
+        if (!with_bwd) continue;
+        const char *g_do = (const char *)dO + g0 * hs;
+        if (tc_bwd_preprocess(p, g_do, o, l, Lp, Dp, st) != cudaSuccess) return MOA_ERR_CUDA;
+        if (mat_bwd(p, q, k, v, g_do, Dp, PT, GST, (char *)dQ + g0 * hs, (char *)dK + g0 * hs, (char *)dV + g0 * hs, st) !=
+            cudaSuccess)
+            return MOA_ERR_CUDA;
+    }
+    return MOA_OK;
+}
 
 moa_status run_fwd(const moa_attn_desc *d, const void *Q, const void *K, const void *V, void *O, float *L,
                    cudaStream_t st)
@@ -219,6 +273,7 @@ extern "C" {
 size_t moa_attn_workspace_bytes(const moa_attn_desc *desc, int op)
 {
     if (check_desc(desc) != MOA_OK) return 0;
+    if (desc->materialize) return (op == MOA_OP_FWD || op == MOA_OP_FUSED) ? mat_workspace(desc, op).total : 0;
     if (op == MOA_OP_FWD) return 0;
     if (op == MOA_OP_BWD || op == MOA_OP_FUSED) return bwd_workspace(desc).total;
     return 0;
@@ -231,8 +286,13 @@ moa_status moa_attn_fwd(const moa_attn_desc *desc, const void *Q, const void *K,
     if (s != MOA_OK) return s;
     if (!Q || !K || !V || !O || !L) return MOA_ERR_INVALID_ARG;
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(L)) return MOA_ERR_INVALID_ARG;
-    (void)ws; (void)ws_bytes;
+    if (desc->materialize) {
+        if (!ws || ws_bytes < mat_workspace(desc, MOA_OP_FWD).total) return MOA_ERR_WORKSPACE;
+        if (!aligned16(ws)) return MOA_ERR_INVALID_ARG;
+    }
     if ((s = check_arch()) != MOA_OK) return s;
+    if (desc->materialize)
+        return run_materialized(desc, Q, K, V, nullptr, O, L, nullptr, nullptr, nullptr, ws, false, (cudaStream_t)stream);
     return run_fwd(desc, Q, K, V, O, L, (cudaStream_t)stream);
 }
 
@@ -242,6 +302,8 @@ moa_status moa_attn_bwd(const moa_attn_desc *desc, const void *Q, const void *K,
 {
     moa_status s = check_desc(desc);
     if (s != MOA_OK) return s;
+    // the materialising variant's backward consumes the P array its own forward wrote: fused call only
+    if (desc->materialize) return MOA_ERR_UNSUPPORTED;
     if (!Q || !K || !V || !O || !L || !dO || !dQ || !dK || !dV) return MOA_ERR_INVALID_ARG;
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(L) || !aligned16(dO) ||
         !aligned16(dQ) || !aligned16(dK) || !aligned16(dV))
@@ -263,6 +325,7 @@ moa_status moa_attn_bwd_static_scratch(const moa_attn_desc *desc, const void *Q,
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(L) || !aligned16(dO) ||
         !aligned16(dQ) || !aligned16(dK) || !aligned16(dV))
         return MOA_ERR_INVALID_ARG;
+    if (desc->materialize) return MOA_ERR_UNSUPPORTED;
     if (bwd_workspace(desc).total > (size_t)MOA_STATIC_SCRATCH_BYTES) return MOA_ERR_SCRATCH_LIMIT;
     if ((s = check_arch()) != MOA_OK) return s;
     void *scratch = static_scratch_ptr();   // first call on this device resolves the symbol's address
@@ -281,10 +344,11 @@ moa_status moa_attn_fused_fwd_bwd(const moa_attn_desc *desc, const void *Q, cons
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(L) || !aligned16(dO) ||
         !aligned16(dQ) || !aligned16(dK) || !aligned16(dV))
         return MOA_ERR_INVALID_ARG;
-    const size_t need = bwd_workspace(desc).total;
+    const size_t need = desc->materialize ? mat_workspace(desc, MOA_OP_FUSED).total : bwd_workspace(desc).total;
     if (!ws || ws_bytes < need) return MOA_ERR_WORKSPACE;
     if (!aligned16(ws)) return MOA_ERR_INVALID_ARG;
     if ((s = check_arch()) != MOA_OK) return s;
+    if (desc->materialize) return run_materialized(desc, Q, K, V, dO, O, L, dQ, dK, dV, ws, true, (cudaStream_t)stream);
     if ((s = run_fwd(desc, Q, K, V, O, L, (cudaStream_t)stream)) != MOA_OK) return s;
     return run_bwd(desc, Q, K, V, O, L, dO, dQ, dK, dV, ws, (cudaStream_t)stream);
 }

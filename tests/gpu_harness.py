@@ -36,6 +36,8 @@ def run_library(inp: dict, dtype: str, causal: bool, scale: float, *, op: str = 
     O, dQ, dK, dV = (torch.full((B, H, n, d), fill, dtype=tdt, device="cuda") for _ in range(4))
     L = torch.full((B, H, n), fill, dtype=torch.float32, device="cuda")
     ws_bytes = mb.moa_attn_workspace_bytes(desc, mb.MOA_OP_FUSED if op != "fwd" else mb.MOA_OP_FWD)
+    if materialize and op == "split":
+        raise ValueError("the materialising variant has no separate backward call")
     ws = torch.full((max(ws_bytes, 16),), 0xFF, dtype=torch.uint8, device="cuda")
     if op == "fused":
         mb.moa_attn_fused_fwd_bwd(desc, Q, K, V, dO, O, L, dQ, dK, dV, ws)

@@ -49,6 +49,21 @@ def test_workspace_is_linear_in_n(lib):
     assert mb.moa_attn_workspace_bytes(mb.make_desc(1, 32, 512, 128, True, 0.1), mb.MOA_OP_FWD) == 0
 
 
+def test_materializing_workspace_is_quadratic_and_capped(lib):
+    def ws(n, heads=4):
+        return mb.moa_attn_workspace_bytes(mb.make_desc(1, heads, n, 128, True, 0.1, materialize=1), mb.MOA_OP_FUSED)
+    assert ws(1024) >= 2 * 4 * 1024 * 1024 * 2
+    assert ws(2048) > 3.9 * ws(1024)                      # ~n^2
+    # heads are processed in groups under a 16 GiB cap for the two arrays
+    assert ws(32768, heads=32) <= (16 << 30) + (64 << 20)
+    d = mb.make_desc(1, 4, 1024, 128, True, 0.1, materialize=1)
+    a = 4096
+    assert mb.moa_attn_bwd(d, a, a, a, a, a, a, a, a, a, a, ws_bytes=1 << 40, check=False) == mb.MOA_ERR_UNSUPPORTED
+    assert mb.moa_attn_fused_fwd_bwd(d, a, a, a, a, a, a, a, a, a, a, ws_bytes=16, check=False) == mb.MOA_ERR_WORKSPACE
+    d32 = mb.make_desc(1, 4, 1024, 128, True, 0.1, mb.MOA_F32, materialize=1)
+    assert mb.moa_attn_fwd(d32, a, a, a, a, a, a, ws_bytes=1 << 40, check=False) == mb.MOA_ERR_UNSUPPORTED
+
+
 def test_argument_errors_need_no_device(lib):
     good = mb.make_desc(1, 1, 128, 64, False, 0.125, mb.MOA_F32)
     a = 4096  # fake, aligned, never dereferenced: checks fail first

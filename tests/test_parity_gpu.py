@@ -135,6 +135,24 @@ def test_invariants_on_gpu_outputs(H):
     assert np.all(got["O"] >= f["V"].min(2, keepdims=True) - 1e-5)
 
 
+# ------------------------------------------- the n x n-materialising comparison variant
+@pytest.mark.parametrize("B,Hh,n,d,causal", [
+    (1, 2, 128, 128, False), (2, 2, 256, 64, True), (1, 3, 333, 128, True), (1, 2, 1000, 128, False),
+    (1, 1, 77, 64, False), (1, 2, 640, 64, True),
+])
+def test_materializing_variant(H, B, Hh, n, d, causal):
+    inp = mi.make_inputs(B, Hh, n, d, seed=400 + n, dtype="bf16")
+    scale = 1.0 / math.sqrt(d)
+    ref = _oracle(inp, "bf16", causal, scale)
+    got = H.run_library(inp, "bf16", causal, scale, materialize=1)
+    H.assert_close(got, ref, H.TOL_BF16, tag=f"materialize n{n} d{d}")
+    assert mi.rel_err(got["L"], ref["L"]) <= 1e-3
+    npad = (n + 127) // 128 * 128
+    assert got["ws_bytes"] >= 2 * B * Hh * npad * npad * 2      # two n x n arrays: the O(n^2) workspace
+    fwd = H.run_library(inp, "bf16", causal, scale, materialize=1, op="fwd")
+    np.testing.assert_array_equal(fwd["O"], got["O"])
+
+
 # ------------------------------------------------------------- configs 2 and 3, whole
 def test_c2_small_bf16_all_heads(H):
     w = mi.CONFIGS["c2_small_bf16"]
