@@ -183,9 +183,84 @@ def run_reference(args, w):
 
 def workload_config(w, args):
     return {"workload": w.name, "B": w.B, "H": w.H, "n": w.n, "d": w.d, "causal": w.causal,
-            "scale": "1/sqrt(d)", "dq_mode": args.dq_mode, "path": args.path,
+            "scale": "1/sqrt(d)", "dq_mode": args.dq_mode, "path": args.path, "materialize": getattr(args, "materialize", 0),
             "l2": "inputs+outputs per step exceed the 126 MB L2; no explicit flush",
             "parallelism": f"independent (b,h) shards x{args.gpus}"}
+
+
+# ----------------------------------------------------------------------------- sweep
+def run_sweep(args):
+    """Config-5 style sweep: for each n and each strategy (the three dQ modes of the fused path
+    and the n x n-materialising variant) one JSON line with time, TFLOP/s, per-kernel times and
+    peak device bytes; then the local scaling exponents log2(t(2n)/t(n)) per strategy.  Not the
+    contract line: a study table."""
+    import torch
+    from paper_2609_33916_b200 import binding as mb
+    from paper_2609_33916_b200 import build as mbuild
+    from paper_2609_33916_b200 import inputs as mi
+    mbuild.build()
+    torch.cuda.set_device(0)
+    peaks, peaks_kind = load_peaks()
+    strategies = [("fused_red", 1, 0), ("fused_bulk_reduce", 2, 0), ("fused_separate_pass", 3, 0), ("materialize", 0, 1)]
+    sizes = [int(x) for x in args.sweep_sizes.split(",")] if args.sweep_sizes else list(mi.C5_SIZES)
+    times = {}
+    for n in sizes:
+        w = mi.CONFIGS[f"c5_causal_n{n}"] if f"c5_causal_n{n}" in mi.CONFIGS else mi.Workload(f"sweep_n{n}", 1, 32, n, 128, True, "bf16", 4)
+        shape = (w.B, w.H, w.n, w.d)
+        gen = torch.Generator(device="cuda").manual_seed(w.seed)
+        Q, K, V, dO = (torch.randn(shape, generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16) for _ in range(4))
+        O, dQ, dK, dV = (torch.empty(shape, dtype=torch.bfloat16, device="cuda") for _ in range(4))
+        L = torch.empty((w.B, w.H, w.n), dtype=torch.float32, device="cuda")
+        io_bytes = sum(t.numel() * t.element_size() for t in (Q, K, V, dO, O, dQ, dK, dV, L))
+        for name, dq_mode, mat in strategies:
+            desc = mb.make_desc(w.B, w.H, w.n, w.d, w.causal, w.scale, mb.MOA_BF16, dq_mode, mat, 0)
+            ws_bytes = mb.moa_attn_workspace_bytes(desc, mb.MOA_OP_FUSED)
+            free, _ = torch.cuda.mem_get_info()
+            line = {"sweep": "c5", "n": n, "strategy": name, "workspace_bytes": ws_bytes, "io_bytes": io_bytes,
+                    "peak_device_bytes": io_bytes + ws_bytes}
+            if ws_bytes + (1 << 30) > free:
+                line["skipped"] = f"needs {ws_bytes / 2**30:.1f} GiB of workspace"
+                print(json.dumps(line), flush=True)
+                continue
+            ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device="cuda")
+            stream = torch.cuda.current_stream()
+            steps = 3 if n >= 16384 else (5 if n >= 4096 else 20)
+            for _ in range(3):
+                mb.moa_attn_fused_fwd_bwd(desc, Q, K, V, dO, O, L, dQ, dK, dV, ws, stream)
+            torch.cuda.synchronize()
+            mb.moa_profile_read(); mb.moa_profile_enable(True)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(steps):
+                mb.moa_attn_fused_fwd_bwd(desc, Q, K, V, dO, O, L, dQ, dK, dV, ws, stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            mb.moa_profile_enable(False)
+            prof = mb.moa_profile_read()
+            st = mb.moa_last_device_status(stream)
+            ms = e0.elapsed_time(e1) / steps
+            tf = w.model_flops / (ms * 1e-3) / 1e12
+            times[(name, n)] = ms
+            line.update({"ms": ms, "tflops": tf, "pct_of_measured_burst_peak": 100 * tf / peaks["bf16_tflops"],
+                         "status": mb.status_string(st),
+                         "per_kernel_ms": {k: v[0] / max(1, v[1]) * (v[1] / steps) for k, v in prof.items() if v[1]}})
+            if mat:   # HBM-bound variant: n^2 traffic per head = P^T and dS^T written once and read once
+                npad = (n + 127) // 128 * 128
+                tri = 0.5 if w.causal else 1.0
+                line["nxn_bytes_moved_model"] = 8.0 * w.B * w.H * npad * npad * tri
+                line["nxn_gbs"] = line["nxn_bytes_moved_model"] / (ms * 1e-3) / 1e9
+            print(json.dumps(line), flush=True)
+            del ws
+            torch.cuda.empty_cache()
+        del Q, K, V, dO, O, dQ, dK, dV, L
+        torch.cuda.empty_cache()
+    for name, _, _ in strategies:
+        exps = {}
+        for a, b in zip(sizes[:-1], sizes[1:]):
+            if (name, a) in times and (name, b) in times and b == 2 * a:
+                exps[f"{a}->{b}"] = math.log2(times[(name, b)] / times[(name, a)])
+        print(json.dumps({"sweep": "c5", "strategy": name, "local_time_exponent": exps}), flush=True)
+    return 0
 
 
 # ------------------------------------------------------------------------------ main
@@ -199,6 +274,9 @@ def main():
     ap.add_argument("--dq-mode", type=int, default=0)
     ap.add_argument("--path", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--materialize", type=int, default=0)
+    ap.add_argument("--sweep", action="store_true", help="config-5 strategy sweep (study table, not the contract line)")
+    ap.add_argument("--sweep-sizes", default="")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "moa" else args.warmup
 
@@ -206,6 +284,8 @@ def main():
     w = mi.CONFIGS[args.workload]
     if args.impl == "reference":
         return run_reference(args, w)
+    if args.sweep:
+        return run_sweep(args)
 
     import torch
     from paper_2609_33916_b200 import binding as mb
@@ -229,7 +309,7 @@ def main():
     peaks, peaks_kind = load_peaks()
 
     B, H, n, d = w.B, w.H, w.n, w.d
-    desc = mb.make_desc(B, H, n, d, w.causal, w.scale, mb.MOA_BF16, args.dq_mode, 0, args.path)
+    desc = mb.make_desc(B, H, n, d, w.causal, w.scale, mb.MOA_BF16, args.dq_mode, args.materialize, args.path)
     shape = (B, H, n, d)
     base_mem = torch.cuda.memory_allocated()
     gen = torch.Generator(device="cuda").manual_seed(w.seed + 1000 * rank)
