@@ -409,8 +409,12 @@ def main():
     achieved = alg_flops[dominant] / (dom_ms * 1e-3) / 1e12 if dom_ms > 0 else None
     tc_path = args.path in (0, 2)
     peak = peaks["bf16_tflops_sustained"]
+    # DRAM bytes per launch of the backward kernel: ncu capture of a small case (B1 H8 n8192 d128:
+    # 124.9 MB read+written over 65536 tokens), scaled by tokens -- traffic is linear in B*H*n
+    traffic = 124.9e6 / 65536.0 * heads * n if (dominant == "bwd_kv" and d == 128) else None
     roofline = {"bound": "tensor", "kernel": dominant, "achieved": achieved, "peak": peak,
-                "unit": "TFLOP/s", "frac": (achieved / peak) if achieved else None, "traffic": None,
+                "unit": "TFLOP/s", "frac": (achieved / peak) if achieved else None, "traffic": traffic,
+                "traffic_source": "ncu dram__bytes_read+write of a smaller case, scaled by tokens" if traffic else None,
                 "peak_source": f"{peaks_kind} bf16_tflops_sustained (kernel timed inside a long step)",
                 "kernel_ms": dom_ms,
                 "per_kernel_ms": {k: (v[0] / max(1, v[1]), v[1]) for k, v in prof.items() if v[1]}}

@@ -109,7 +109,14 @@ moa_status check_desc(const moa_attn_desc *d)
     return MOA_OK;
 }
 
-int resolved_dq_mode(const moa_attn_desc *d) { return d->dq_mode == MOA_DQ_AUTO ? MOA_DQ_RED : d->dq_mode; }
+// AUTO: the TMA bulk add-reduce where it exists (tensor-core path, d = 128: measured slightly
+// ahead of plain reds at every size), plain reds otherwise.
+int resolved_dq_mode(const moa_attn_desc *d)
+{
+    if (d->dq_mode != MOA_DQ_AUTO) return d->dq_mode;
+    const bool tc = d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->scale > 0.f;
+    return (tc && d->d == 128) ? MOA_DQ_BULK_REDUCE : MOA_DQ_RED;
+}
 
 // the tensor-core kernels take the row max before scaling, which needs scale > 0
 bool use_tc_fwd(const moa_attn_desc *d) { return d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->scale > 0.f; }
