@@ -41,7 +41,8 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(f
 // ---- tensor-core path (tc_fwd.cu), bf16 only ---------------------------------------------
 cudaError_t tc_fwd(const Problem &p, const void *Q, const void *K, const void *V, void *O, float *L, cudaStream_t st);
 
-// Lp = L*log2(e) and Dp = rowsum(dO o O), each padded per head to a multiple of 128 rows
+// Lp = -L*log2(e) and Dp = -rowsum(dO o O) (negated: fma/add operands), each padded per head to a
+// multiple of 128 rows (-inf / 0 past n)
 cudaError_t tc_bwd_preprocess(const Problem &p, const void *dO, const void *O, const float *L, float *Lp, float *Dp,
                               cudaStream_t st);
 // dK, dV; UNSCALED dQ contributions (dS K, without the factor scale) red-added into dQacc

@@ -66,8 +66,9 @@ __device__ __forceinline__ void red_add_v4(float *addr, float a, float b, float 
                  : "memory");
 }
 
-// Lp = L log2(e) and D = rowsum(dO o O), both padded per head to n_pad rows
-// (+inf and 0 past n).  One warp per padded row.
+// Lp = -L log2(e) and Dp = -rowsum(dO o O), both padded per head to n_pad rows (-inf and 0
+// past n).  Stored negated so that the kernels can use them as fma / add operands directly.
+// One warp per padded row.
 template <int D>
 __global__ void bwd_preprocess_kernel(const __nv_bfloat16 *__restrict__ dO, const __nv_bfloat16 *__restrict__ O,
                                       const float *__restrict__ L, float *__restrict__ Lp, float *__restrict__ Dp,
@@ -79,7 +80,7 @@ __global__ void bwd_preprocess_kernel(const __nv_bfloat16 *__restrict__ dO, cons
     const size_t bh = prow / n_pad;
     const int r = (int)(prow % n_pad);
     if (r >= n) {
-        if (lane == 0) { Lp[prow] = INFINITY; Dp[prow] = 0.f; }
+        if (lane == 0) { Lp[prow] = -INFINITY; Dp[prow] = 0.f; }
         return;
     }
     const size_t row = bh * n + r;
@@ -96,7 +97,7 @@ __global__ void bwd_preprocess_kernel(const __nv_bfloat16 *__restrict__ dO, cons
     }
 #pragma unroll
     for (int o = 16; o >= 1; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) { Dp[prow] = acc; Lp[prow] = L[row] * kLog2e; }
+    if (lane == 0) { Dp[prow] = -acc; Lp[prow] = -L[row] * kLog2e; }
 }
 
 // kBulk: the dQ tile goes out through the TMA add-reduce; that needs 32 KB of staging, which is
@@ -408,17 +409,20 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         const int wg = warp / 4;                          // which half of the query columns
         const int lane_row = 32 * (warp % 4) + lane;      // TMEM lane of this thread = key index in the tile
         const uint32_t lane_addr = tbase + ((uint32_t)(32 * (warp % 4)) << 16);
-        float p[64];                                      // this thread's probabilities of the current tile
+        uint64_t p2[32];                                  // this thread's 64 probabilities of the current tile, as fp32 pairs
+        const uint64_t sl2 = pack_f32x2(scale_log2, scale_log2);
         bool ok = true;
 
         // P-phase of tile `it`: P^T = exp2(S^T scale log2e - L log2e), kept in registers and
-        // written as bf16 over the first half of this warpgroup's S^T columns.
+        // written as bf16 over the first half of this warpgroup's S^T columns.  Arithmetic is
+        // on fp32 pairs (f32x2) to halve the instruction count: the UMMA-issuing warp shares
+        // its scheduler with these warps.
         auto p_phase = [&](int it) -> bool {
             const int s = it & 1;
             const bool diag = causal && (i_begin + it == kt);
             if (!mbar_wait(bars + B_S, it & 1, abortp, status, ERR_SDP)) return false;
             tc_fence_after();
-            const float *Ls = sL + s * 128;
+            const float *Ls = sL + s * 128;    // -L log2e
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 const int qc0 = 64 * wg + 32 * c;
@@ -428,16 +432,23 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 uint32_t pk[16];
 #pragma unroll
                 for (int e = 0; e < 32; e += 4) {
-                    const float4 l4 = *reinterpret_cast<const float4 *>(Ls + qc0 + e);
-                    const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        float pv = ex2(fmaf(__uint_as_float(rs[e + u]), scale_log2, -lv[u]));
-                        if (diag && (qc0 + e + u) < lane_row) pv = 0.f;   // query index < key index: masked
-                        p[32 * c + e + u] = pv;
+                    const ulonglong2 l4 = *reinterpret_cast<const ulonglong2 *>(Ls + qc0 + e);   // two pairs
+                    const uint64_t t0 = fma_f32x2(pack_f32x2(__uint_as_float(rs[e]), __uint_as_float(rs[e + 1])), sl2, l4.x);
+                    const uint64_t t1 = fma_f32x2(pack_f32x2(__uint_as_float(rs[e + 2]), __uint_as_float(rs[e + 3])), sl2, l4.y);
+                    float a0, a1, a2, a3;
+                    unpack_f32x2(t0, a0, a1);
+                    unpack_f32x2(t1, a2, a3);
+                    a0 = ex2(a0); a1 = ex2(a1); a2 = ex2(a2); a3 = ex2(a3);
+                    if (diag) {   // query index < key index: masked
+                        if (qc0 + e < lane_row) a0 = 0.f;
+                        if (qc0 + e + 1 < lane_row) a1 = 0.f;
+                        if (qc0 + e + 2 < lane_row) a2 = 0.f;
+                        if (qc0 + e + 3 < lane_row) a3 = 0.f;
                     }
-                    pk[e / 2] = pack_bf16(p[32 * c + e], p[32 * c + e + 1]);
-                    pk[e / 2 + 1] = pack_bf16(p[32 * c + e + 2], p[32 * c + e + 3]);
+                    p2[16 * c + e / 2] = pack_f32x2(a0, a1);
+                    p2[16 * c + e / 2 + 1] = pack_f32x2(a2, a3);
+                    pk[e / 2] = pack_bf16(a0, a1);
+                    pk[e / 2 + 1] = pack_bf16(a2, a3);
                 }
                 tmem_st(lane_addr + colS + 64 * wg + 16 * c, pk);
             }
@@ -453,7 +464,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             // dS-phase: dS^T = P^T o (dP^T - D)   (the factor `scale` is applied to dK and dQ at the end)
             if (!mbar_wait(bars + B_DP, it & 1, abortp, status, ERR_SDP)) { ok = false; break; }
             tc_fence_after();
-            const float *Ds = sD + s * 128;
+            const float *Ds = sD + s * 128;    // -D
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 const int qc0 = 64 * wg + 32 * c;
@@ -463,11 +474,12 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 uint32_t gk[16];
 #pragma unroll
                 for (int e = 0; e < 32; e += 4) {
-                    const float4 d4 = *reinterpret_cast<const float4 *>(Ds + qc0 + e);
-                    const float g0 = p[32 * c + e] * (__uint_as_float(rd[e]) - d4.x);
-                    const float g1 = p[32 * c + e + 1] * (__uint_as_float(rd[e + 1]) - d4.y);
-                    const float g2 = p[32 * c + e + 2] * (__uint_as_float(rd[e + 2]) - d4.z);
-                    const float g3 = p[32 * c + e + 3] * (__uint_as_float(rd[e + 3]) - d4.w);
+                    const ulonglong2 d4 = *reinterpret_cast<const ulonglong2 *>(Ds + qc0 + e);
+                    const uint64_t u0 = add_f32x2(pack_f32x2(__uint_as_float(rd[e]), __uint_as_float(rd[e + 1])), d4.x);
+                    const uint64_t u1 = add_f32x2(pack_f32x2(__uint_as_float(rd[e + 2]), __uint_as_float(rd[e + 3])), d4.y);
+                    float g0, g1, g2, g3;
+                    unpack_f32x2(mul_f32x2(p2[16 * c + e / 2], u0), g0, g1);
+                    unpack_f32x2(mul_f32x2(p2[16 * c + e / 2 + 1], u1), g2, g3);
                     gk[e / 2] = pack_bf16(g0, g1);
                     gk[e / 2 + 1] = pack_bf16(g2, g3);
                 }

@@ -142,8 +142,8 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
         const int wg = warp / 4;
         const int lane_row = 32 * (warp % 4) + lane;              // query row inside the tile
         const uint32_t lane_addr = tbase + ((uint32_t)(32 * (warp % 4)) << 16);
-        const float Lrow = Lp[(size_t)bh * n_pad + q0 + lane_row];   // +inf past n: P = 0
-        const float Drow = Dp[(size_t)bh * n_pad + q0 + lane_row];
+        const float Lrow = Lp[(size_t)bh * n_pad + q0 + lane_row];   // -L log2e; -inf past n: P = 0
+        const float Drow = Dp[(size_t)bh * n_pad + q0 + lane_row];   // -D
         bool ok = nkt > 0;
         for (int j = 0; ok && j < nkt; ++j) {
             if (!mbar_wait(bars + B_SDP, j & 1, abortp, status, ERR_SDP)) { ok = false; break; }
@@ -159,13 +159,13 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
                 uint32_t gk[16];
 #pragma unroll
                 for (int e = 0; e < 32; e += 2) {
-                    float p0 = ex2(fmaf(__uint_as_float(rs[e]), scale_log2, -Lrow));
-                    float p1 = ex2(fmaf(__uint_as_float(rs[e + 1]), scale_log2, -Lrow));
+                    float p0 = ex2(fmaf(__uint_as_float(rs[e]), scale_log2, Lrow));
+                    float p1 = ex2(fmaf(__uint_as_float(rs[e + 1]), scale_log2, Lrow));
                     if (diag) {                                   // key index > query index: masked
                         if (kc0 + e > lane_row) p0 = 0.f;
                         if (kc0 + e + 1 > lane_row) p1 = 0.f;
                     }
-                    gk[e / 2] = pack_bf16(p0 * (__uint_as_float(rd[e]) - Drow), p1 * (__uint_as_float(rd[e + 1]) - Drow));
+                    gk[e / 2] = pack_bf16(p0 * (__uint_as_float(rd[e]) + Drow), p1 * (__uint_as_float(rd[e + 1]) + Drow));
                 }
                 tmem_st(lane_addr + colDP + 64 * wg + 16 * c, gk);
             }

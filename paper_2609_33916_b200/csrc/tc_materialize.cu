@@ -383,7 +383,7 @@ mat_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
                     const uint32_t pp = pk[c][e / 2];
                     const float p0 = __uint_as_float(pp << 16), p1 = __uint_as_float(pp & 0xffff0000u);
                     const float2 d2 = *reinterpret_cast<const float2 *>(Ds + 64 * wg + 32 * c + e);
-                    gk[e / 2] = pack_bf16(p0 * (__uint_as_float(rd[e]) - d2.x), p1 * (__uint_as_float(rd[e + 1]) - d2.y));
+                    gk[e / 2] = pack_bf16(p0 * (__uint_as_float(rd[e]) + d2.x), p1 * (__uint_as_float(rd[e + 1]) + d2.y));   // Dp holds -D
                 }
                 tmem_st(lane_addr + colDP + 64 * wg + 16 * c, gk);
 #pragma unroll
