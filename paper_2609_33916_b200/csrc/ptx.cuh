@@ -281,6 +281,13 @@ __device__ __forceinline__ uint64_t mul_f32x2(uint64_t a, uint64_t b)
     return r;
 }
 
+__device__ __forceinline__ float fmax3(float a, float b, float c)
+{
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
 __device__ __forceinline__ float ex2(float x)
 {
     float y;

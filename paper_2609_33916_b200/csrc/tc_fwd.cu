@@ -161,14 +161,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                         if (col >= n || (causal && col > row)) r[c][i] = 0xff800000u;   // -inf
                     }
             }
-            // row max of the raw scores (scale_log2 > 0, so scaling commutes with max)
+            // row max of the raw scores (scale_log2 > 0, so scaling commutes with max); 3-input max
             float mx4[4];
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 float a = fmaxf(__uint_as_float(r[c][0]), __uint_as_float(r[c][1]));
 #pragma unroll
-                for (int i = 2; i < 32; i += 2)
-                    a = fmaxf(a, fmaxf(__uint_as_float(r[c][i]), __uint_as_float(r[c][i + 1])));
+                for (int i = 2; i < 32; i += 2) a = fmax3(a, __uint_as_float(r[c][i]), __uint_as_float(r[c][i + 1]));
                 mx4[c] = a;
             }
             const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
@@ -193,23 +192,32 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                     }
                 }
             }
-            // P = 2^(s scale_log2 - m_used), row sum (four independent partial sums), bf16 P into
-            // TMEM over the first 64 of the S columns
-            const float neg_m = -m_used;
-            float ls[4] = {0.f, 0.f, 0.f, 0.f};
+            // P = 2^(s scale_log2 - m_used), row sum, bf16 P into TMEM over the first 64 of the S
+            // columns.  Arithmetic runs on fp32 pairs (f32x2) to halve the instruction count.
+            const uint64_t sl2 = pack_f32x2(scale_log2, scale_log2);
+            const uint64_t negm2 = pack_f32x2(-m_used, -m_used);
+            uint64_t ls2[2] = {0ull, 0ull};
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t pk[16];
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
-                    const float p0 = ex2(fmaf(__uint_as_float(r[c][i]), scale_log2, neg_m));
-                    const float p1 = ex2(fmaf(__uint_as_float(r[c][i + 1]), scale_log2, neg_m));
-                    ls[(i / 2) & 3] += p0 + p1;
+                    const uint64_t t = fma_f32x2(pack_f32x2(__uint_as_float(r[c][i]), __uint_as_float(r[c][i + 1])), sl2, negm2);
+                    float p0, p1;
+                    unpack_f32x2(t, p0, p1);
+                    p0 = ex2(p0);
+                    p1 = ex2(p1);
+                    ls2[(i >> 1) & 1] = add_f32x2(ls2[(i >> 1) & 1], pack_f32x2(p0, p1));
                     pk[i / 2] = pack_bf16(p0, p1);
                 }
                 tmem_st(lane_addr + kColP + 16 * c, pk);
             }
-            l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+            {
+                float s0, s1, s2, s3;
+                unpack_f32x2(ls2[0], s0, s1);
+                unpack_f32x2(ls2[1], s2, s3);
+                l += (s0 + s1) + (s2 + s3);
+            }
             tc_wait_st();
             tc_fence_before();
             mbar_arrive(&bar_p);
