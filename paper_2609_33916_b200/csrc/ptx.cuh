@@ -7,6 +7,10 @@
 #include <stdint.h>
 #include <cuda/ptx>
 
+#ifndef MOA_SUSPEND_HINT_NS
+#define MOA_SUSPEND_HINT_NS 20000u
+#endif
+
 namespace moa {
 namespace ptx {
 
@@ -53,7 +57,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.b32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity), "r"(20000u)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(MOA_SUSPEND_HINT_NS)
         : "memory");
     return ok != 0;
 }
@@ -63,9 +67,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 // abort flag so that every other role gives up quickly as well, and returns false.
 constexpr long long kWaitCycles = 4000000000LL;
 
+// Non-blocking probe: much cheaper than try_wait when the phase has already completed (try_wait
+// is a potentially suspending instruction and costs the caller ~100 cycles even on success).
+__device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
                                           unsigned int *status, uint32_t code)
 {
+    if (mbar_test_wait(bar, parity)) return true;
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t spins = 0;

@@ -1,25 +1,29 @@
 // Forward attention on the sm_100a tensor cores (tcgen05 + TMEM + TMA), bf16 in,
 // fp32 accumulate.
 //
-// One CTA owns 128 query rows of one (batch, head) and walks the key/value tiles of
-// 128 keys.  Roles (192 threads):
-//   warps 0-3  softmax: thread t owns query row t = TMEM lane t.  Reads the fp32 score
-//              tile S from TMEM, keeps the running row max / row sum, writes the bf16
-//              probabilities P back into TMEM (over the first half of S), rescales the
-//              O accumulator in TMEM when the row max has grown, and writes O and the
-//              logsumexp L at the end.
-//   warp 4     TMA producer: Q once, then K and V tiles into single buffers that are
-//              refilled as soon as the UMMA that read them has completed.
-//   warp 5     UMMA issuer: S = Q K^T (both operands K-major in shared memory), then
-//              O += P V (P from TMEM, V MN-major in shared memory).  Owns the TMEM
-//              allocation.
-// S, P and the O accumulator never leave the SM: nothing of size n x n reaches HBM.
-// Two CTAs fit on one SM (256 TMEM columns and at most 97 KB shared memory each), so
-// one CTA's softmax overlaps the other's UMMAs.
+// One CTA (one per SM) owns 128 query rows of one (batch, head) and walks the key/value
+// tiles of 128 keys.  Roles (352 threads):
+//   warps 0-7  softmax: thread = query row = TMEM lane; warpgroup h = warp / 4 owns key
+//              columns [64h, 64h+64) of every tile with its own running max, row sum and O
+//              accumulator, so the two halves are independent online-softmax streams that are
+//              merged only in the epilogue.  Per tile: 64 fp32 scores from TMEM into registers,
+//              max (3-input, independent chains), exp2 + row sum on packed fp32 pairs, bf16 P back
+//              into TMEM over the front of the same score columns; O_h in TMEM is rescaled only
+//              when the max has grown by more than 8 (log2 domain).
+//   warp 8     TMA producer: Q once, K and V tiles in two-slot rings.
+//   warp 9     UMMA issuer (one thread) for S = Q K^T (SS, both operands K-major), into two
+//              alternating score buffers: S(j+1) is computed while the softmax works on S(j).
+//   warp 10    UMMA issuer (one thread) for O_h += P_h V (TS: P from TMEM, V MN-major in smem).
+// Two issuing threads because a barrier probe or a commit costs an issuer ~100 cycles in which
+// it feeds nothing and the tensor pipe queues only a few UMMAs; UMMAs of different threads are
+// unordered, so the one hazard between the streams (S(j) overwriting the buffer that held
+// P(j-2)) goes through an mbarrier.
+// TMEM (512 columns): score buffers [0,128) and [128,256), O_0 [256,256+D), O_1 [256+D,256+2D).
+// S, P and the O accumulators never leave the SM: nothing of size n x n reaches HBM.
 //
-// The running max is lazy: O and the row sum are rescaled only when the new tile's max
-// exceeds the max in use by more than 8 (a factor 256 in P), which leaves the result
-// unchanged mathematically and keeps P well inside bf16/fp32 range.
+// What bounds it (config 4, d = 128): one exp2 per score keeps the MUFU unit as busy as the
+// tensor pipe (both 0.92 ms of a 2.0 ms kernel); the rest is the softmax warps' non-MUFU work
+// and hand-off latency.
 #include "common.cuh"
 #include "ptx.cuh"
 #include "tensormap.cuh"
@@ -31,17 +35,21 @@ using namespace ptx;
 
 constexpr int BM = 128;            // query rows per CTA
 constexpr int BN = 128;            // keys per tile
-constexpr int kThreads = 192;
-constexpr int kTmemCols = 256;     // S: columns [0,128), O: [128,128+D)
-constexpr uint32_t kColS = 0, kColP = 0, kColO = 128;
+constexpr int kThreads = 352;      // warps 0-7 softmax, 8 TMA, 9 UMMA issuer for S, 10 UMMA issuer for PV
+constexpr int kTmemCols = 512;     // two score buffers: columns [0,128), [128,256); two O accumulators from 256
+constexpr uint32_t kColS = 0, kColO = 256;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.f;
 
 enum : uint32_t { ERR_Q = 0x101, ERR_K = 0x102, ERR_V = 0x103, ERR_S = 0x104, ERR_P = 0x105, ERR_O = 0x106 };
 
+enum { F_Q = 0, F_KFULL = 1 /*2*/, F_KEMPTY = 3 /*2*/, F_VFULL = 5 /*2*/, F_VEMPTY = 7 /*2*/, F_S = 9 /*2*/,
+       F_P = 11 /*[buffer][half]: 4*/, F_O = 15, F_X = 16 /*epilogue exchange*/, F_OB = 17 /*2: score buffer consumed*/,
+       F_COUNT = 19 };
+
 template <int D>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
               const __grid_constant__ CUtensorMap mapV, __nv_bfloat16 *__restrict__ O, float *__restrict__ L,
               int n, int causal, float scale_log2, int nqt, unsigned int *status)
@@ -49,12 +57,11 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     constexpr int kTileBytes = 128 * D * 2;
     constexpr int kBoxes = D / 64;         // 64-column (128-byte) swizzled boxes per tile
     constexpr int kBoxBytes = 128 * 128;   // 128 rows x 128 bytes
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t *sm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t *sQ = sm, *sK = sm + kTileBytes, *sV = sm + 2 * kTileBytes;
-    __shared__ uint64_t bar_q, bar_k, bar_v, bar_s, bar_p, bar_o;
-    __shared__ uint32_t tmem_base_s;
-    __shared__ uint32_t abort_flag;
+    extern __shared__ __align__(1024) uint8_t sm[];
+    uint8_t *sQ = sm, *sK = sm + kTileBytes /*2 slots*/, *sV = sm + 3 * kTileBytes /*2 slots*/;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(sm + 5 * kTileBytes);
+    uint32_t *tmem_base_p = reinterpret_cast<uint32_t *>(bars + F_COUNT);
+    volatile uint32_t *abortp = reinterpret_cast<uint32_t *>(bars + F_COUNT + 1);
 
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
     const int bh = blockIdx.x / nqt;
@@ -62,143 +69,181 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     const int qt = causal ? nqt - 1 - t : t;   // causal: longest rows first
     const int q0 = qt * BM;
     const int nkt_all = (n + BN - 1) / BN;
-    const int nkt = causal ? min(qt + 1, nkt_all) : nkt_all;
+    const int nkt_want = causal ? min(qt + 1, nkt_all) : nkt_all;
 
     if (tid == 0) {
-        mbar_init(&bar_q, 1); mbar_init(&bar_k, 1); mbar_init(&bar_v, 1);
-        mbar_init(&bar_s, 1); mbar_init(&bar_p, 128); mbar_init(&bar_o, 1);
-        abort_flag = 0;
+        for (int b = 0; b < F_COUNT; ++b) mbar_init(bars + b, (b >= F_P && b < F_P + 4) ? 128u : (b == F_X ? 256u : 1u));
+        *abortp = (smem_u32(sm) & 1023u) ? 1u : 0u;
+        if (*abortp && status) atomicCAS(status, 0u, 0x108u);
         fence_mbar_init();
         prefetch_tensormap(&mapQ); prefetch_tensormap(&mapK); prefetch_tensormap(&mapV);
     }
-    if (warp == 5) { tmem_alloc(&tmem_base_s, kTmemCols); tmem_relinquish(); }
+    if (warp == 9) { tmem_alloc(tmem_base_p, kTmemCols); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tbase = tmem_base_s;
-    volatile uint32_t *abortp = &abort_flag;
+    const uint32_t tbase = *tmem_base_p;
+    const int nkt = (*abortp == 0) ? nkt_want : 0;   // misaligned shared memory: every role is a no-op
 
-    if (warp == 4) {
+    if (warp == 8) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            mbar_arrive_expect_tx(&bar_q, kTileBytes);
-            for (int b = 0; b < kBoxes; ++b) tma_load_3d(sQ + b * kBoxBytes, &mapQ, &bar_q, 64 * b, q0, bh);
+        if (lane == 0 && nkt > 0) {
+            mbar_arrive_expect_tx(bars + F_Q, kTileBytes);
+            for (int b = 0; b < kBoxes; ++b) tma_load_3d(sQ + b * kBoxBytes, &mapQ, bars + F_Q, 64 * b, q0, bh);
         }
         for (int j = 0; j < nkt; ++j) {
-            if (j > 0 && !mbar_wait(&bar_s, (j - 1) & 1, abortp, status, ERR_S)) break;   // K buffer free
+            const int s = j & 1;
+            if (j >= 2 && !mbar_wait(bars + F_KEMPTY + s, ((j >> 1) - 1) & 1, abortp, status, ERR_K)) break;
             if (lane == 0) {
-                mbar_arrive_expect_tx(&bar_k, kTileBytes);
-                for (int b = 0; b < kBoxes; ++b) tma_load_3d(sK + b * kBoxBytes, &mapK, &bar_k, 64 * b, j * BN, bh);
+                mbar_arrive_expect_tx(bars + F_KFULL + s, kTileBytes);
+                for (int b = 0; b < kBoxes; ++b)
+                    tma_load_3d(sK + s * kTileBytes + b * kBoxBytes, &mapK, bars + F_KFULL + s, 64 * b, j * BN, bh);
             }
-            if (j > 0 && !mbar_wait(&bar_o, (j - 1) & 1, abortp, status, ERR_O)) break;   // V buffer free
+            if (j >= 2 && !mbar_wait(bars + F_VEMPTY + s, ((j >> 1) - 1) & 1, abortp, status, ERR_V)) break;
             if (lane == 0) {
-                mbar_arrive_expect_tx(&bar_v, kTileBytes);
-                for (int b = 0; b < kBoxes; ++b) tma_load_3d(sV + b * kBoxBytes, &mapV, &bar_v, 64 * b, j * BN, bh);
+                mbar_arrive_expect_tx(bars + F_VFULL + s, kTileBytes);
+                for (int b = 0; b < kBoxes; ++b)
+                    tma_load_3d(sV + s * kTileBytes + b * kBoxBytes, &mapV, bars + F_VFULL + s, 64 * b, j * BN, bh);
             }
             __syncwarp();
         }
-    } else if (warp == 5) {
-        // ------------------------------------------------------------------- UMMA issuer
+    } else if (warp == 9 && lane == 0) {
+        // ------------------------------------------- UMMA issuer for the score GEMMs (one thread)
+        // Two issuing threads (this one for S = Q K^T, warp 10 for O += P V): a successful barrier
+        // probe or a commit costs an issuing thread ~100 cycles during which it feeds nothing, and
+        // the tensor pipe only queues a few UMMAs, so with a single issuer the pipe idled for a
+        // third of every tile.  UMMAs of different threads are not ordered, so every hazard between
+        // the two streams goes through an mbarrier: S(j) may overwrite score buffer j&1 only after
+        // PV(j-2), which read P(j-2) there, has completed (F_OB).
         constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0);
-        constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, 0, 1);
-        // Descriptors are built once; inside the loops only a constant is added to the address
-        // field (the issuing thread's instruction stream must stay far shorter than the 64 cycles
-        // one 128x128x16 UMMA takes, or the tensor pipe starves).
-        const uint64_t q_desc = smem_desc_sw128(smem_u32(sQ), 16, 1024);
-        const uint64_t k_desc = smem_desc_sw128(smem_u32(sK), 16, 1024);
-        const uint64_t v_desc = smem_desc_sw128(smem_u32(sV), kBoxBytes, 1024);   // MN-major
-        const uint32_t q_lo = (uint32_t)q_desc, k_lo = (uint32_t)k_desc, v_lo = (uint32_t)v_desc;
-        const uint32_t km_hi = (uint32_t)(q_desc >> 32), mn_hi = (uint32_t)(v_desc >> 32);
-        bool ok = mbar_wait(&bar_q, 0, abortp, status, ERR_Q);
+        const uint64_t km_proto = smem_desc_sw128(0, 16, 1024);
+        const uint32_t km_hi = (uint32_t)(km_proto >> 32);
+        auto field = [](const void *ptr) { return (smem_u32(ptr) >> 4) & 0x3FFFu; };
+        const uint32_t q_lo = (uint32_t)km_proto + field(sQ), k_lo0 = (uint32_t)km_proto + field(sK);
+        constexpr uint32_t kSlot = (uint32_t)(kTileBytes >> 4);
+        bool ok = nkt > 0 && mbar_wait(bars + F_Q, 0, abortp, status, ERR_Q);
         for (int j = 0; ok && j < nkt; ++j) {
-            if (!mbar_wait(&bar_k, j & 1, abortp, status, ERR_K)) break;
+            const int b = j & 1;
+            const uint32_t k_lo = k_lo0 + b * kSlot, dcol = tbase + kColS + 128 * b;
+            if (!mbar_wait(bars + F_KFULL + b, (j >> 1) & 1, abortp, status, ERR_K)) break;
+            if (j >= 2 && !mbar_wait(bars + F_OB + b, ((j >> 1) - 1) & 1, abortp, status, ERR_O)) break;
             tc_fence_after();
-            if (lane == 0) {
-                umma_ss2<false>(tbase + kColS, q_lo, km_hi, k_lo, km_hi, idesc_s);
+            umma_ss2<false>(dcol, q_lo, km_hi, k_lo, km_hi, idesc_s);
 #pragma unroll
-                for (int ks = 1; ks < D / 16; ++ks) {
-                    const uint32_t off = (uint32_t)(((ks / 4) * kBoxBytes + (ks % 4) * 32) >> 4);
-                    umma_ss2<true>(tbase + kColS, q_lo + off, km_hi, k_lo + off, km_hi, idesc_s);
-                }
-                umma_commit(&bar_s);
+            for (int ks = 1; ks < D / 16; ++ks) {
+                const uint32_t off = (uint32_t)(((ks / 4) * kBoxBytes + (ks % 4) * 32) >> 4);
+                umma_ss2<true>(dcol, q_lo + off, km_hi, k_lo + off, km_hi, idesc_s);
             }
-            __syncwarp();
-            if (!mbar_wait(&bar_v, j & 1, abortp, status, ERR_V)) break;
-            if (!mbar_wait(&bar_p, j & 1, abortp, status, ERR_P)) break;
-            tc_fence_after();
-            if (lane == 0) {
-                if (j > 0) umma_ts2<true>(tbase + kColO, tbase + kColP, v_lo, mn_hi, idesc_pv);
-                else       umma_ts2<false>(tbase + kColO, tbase + kColP, v_lo, mn_hi, idesc_pv);
-#pragma unroll
-                for (int ks = 1; ks < BN / 16; ++ks)
-                    umma_ts2<true>(tbase + kColO, tbase + kColP + ks * 8, v_lo + (uint32_t)((ks * 2048) >> 4), mn_hi, idesc_pv);
-                umma_commit(&bar_o);
-            }
-            __syncwarp();
+            umma_commit(bars + F_S + b);
+            umma_commit(bars + F_KEMPTY + b);
         }
-    } else {
-        // ---------------------------------------------------------------- softmax warps
-        const int row = q0 + tid;
-        const uint32_t lane_addr = tbase + ((uint32_t)(warp * 32) << 16);
-        float m_used = 0.f, l = 0.f;
-        bool ok = true;
+    } else if (warp == 10 && lane == 0) {
+        // ------------------------------------------------ UMMA issuer for O += P V (one thread)
+        constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, 0, 1);
+        const uint64_t mn_proto = smem_desc_sw128(0, kBoxBytes, 1024);
+        const uint32_t mn_hi = (uint32_t)(mn_proto >> 32);
+        const uint32_t v_lo0 = (uint32_t)mn_proto + ((smem_u32(sV) >> 4) & 0x3FFFu);
+        constexpr uint32_t kSlot = (uint32_t)(kTileBytes >> 4);
         for (int j = 0; j < nkt; ++j) {
-            if (!mbar_wait(&bar_s, j & 1, abortp, status, ERR_S)) { ok = false; break; }
-            tc_fence_after();
-            const int k0 = j * BN;
-            const bool need_mask = (k0 + BN > n) || (causal && k0 + BN - 1 > q0);
-            // The whole score row (128 fp32) comes into registers with one round trip to TMEM.
-            uint32_t r[4][32];
+            const int b = j & 1;
+            const uint32_t v_lo = v_lo0 + b * kSlot, pcol = tbase + kColS + 128 * b;
+            if (!mbar_wait(bars + F_VFULL + b, (j >> 1) & 1, abortp, status, ERR_V)) break;
+            bool ok = true;
+            // key half h of the tile: P_h (64 keys = 32 TMEM columns at the front of that half of the
+            // score buffer) times V rows 64h.., into its own accumulator O_h
 #pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld(lane_addr + kColS + 32 * c, r[c]);
+            for (int h = 0; h < 2; ++h) {
+                if (!mbar_wait(bars + F_P + 2 * b + h, (j >> 1) & 1, abortp, status, ERR_P)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t ocol = tbase + kColO + h * D, acol = pcol + 64 * h, vh = v_lo + (uint32_t)((h * 4 * 2048) >> 4);
+                if (j > 0) umma_ts2<true>(ocol, acol, vh, mn_hi, idesc_pv);
+                else       umma_ts2<false>(ocol, acol, vh, mn_hi, idesc_pv);
+#pragma unroll
+                for (int ks = 1; ks < 4; ++ks)
+                    umma_ts2<true>(ocol, acol + ks * 8, vh + (uint32_t)((ks * 2048) >> 4), mn_hi, idesc_pv);
+            }
+            if (!ok) break;
+            umma_commit(bars + F_OB + b);
+            umma_commit(bars + F_VEMPTY + b);
+            umma_commit(bars + F_O);
+        }
+    } else if (warp < 8) {
+        // ---------------------------------------------------------------- softmax warps
+        // Thread = query row (TMEM lane); warpgroup h = warp / 4 owns key columns [64h, 64h+64) of
+        // every tile, with its own running max, row sum and O accumulator: the two halves never
+        // talk to each other until the epilogue, which merges them like two online-softmax streams.
+        const int h = warp / 4;
+        const int lane_row = 32 * (warp % 4) + lane;
+        const int row = q0 + lane_row;
+        const uint32_t lane_addr = tbase + ((uint32_t)(32 * (warp % 4)) << 16);
+        const uint32_t ocol = kColO + h * D;
+        float m_used = 0.f, l = 0.f;
+        bool ok = nkt > 0;
+        // The exp2 phase of a tile is MUFU-bound and the rest of a tile's work (TMEM load, max,
+        // hand-offs) is not: start the second warpgroup a few hundred cycles late, once, so that on
+        // each scheduler one warp's exp2 phase overlaps the other's remaining work.  Nothing in the
+        // loop re-synchronises the two halves.
+        if (h == 1) __nanosleep(300);
+        for (int j = 0; ok && j < nkt; ++j) {
+            const uint32_t scol = kColS + 128 * (j & 1) + 64 * h;      // this thread's 64 score columns
+            if (!mbar_wait(bars + F_S + (j & 1), (j >> 1) & 1, abortp, status, ERR_S)) { ok = false; break; }
+            tc_fence_after();
+            const int k0 = j * BN + 64 * h;
+            const bool need_mask = (k0 + 64 > n) || (causal && k0 + 63 > q0);
+            uint32_t r[2][32];
+#pragma unroll
+            for (int c = 0; c < 2; ++c) tmem_ld(lane_addr + scol + 32 * c, r[c]);
             tc_wait_ld();
             if (need_mask) {
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
+                for (int c = 0; c < 2; ++c)
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
                         const int col = k0 + 32 * c + i;
                         if (col >= n || (causal && col > row)) r[c][i] = 0xff800000u;   // -inf
                     }
             }
-            // row max of the raw scores (scale_log2 > 0, so scaling commutes with max); 3-input max
-            float mx4[4];
+            // max of the raw scores (scale_log2 > 0, so scaling commutes with max): 3-input max, eight
+            // independent chains so that the dependent-issue latency does not add up
+            float mx8[8];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                float a = fmaxf(__uint_as_float(r[c][0]), __uint_as_float(r[c][1]));
-#pragma unroll
-                for (int i = 2; i < 32; i += 2) a = fmax3(a, __uint_as_float(r[c][i]), __uint_as_float(r[c][i + 1]));
-                mx4[c] = a;
+            for (int q = 0; q < 8; ++q) {
+                const int c = q >> 2, i0 = 8 * (q & 3);
+                float a = fmax3(__uint_as_float(r[c][i0]), __uint_as_float(r[c][i0 + 1]), __uint_as_float(r[c][i0 + 2]));
+                a = fmax3(a, __uint_as_float(r[c][i0 + 3]), __uint_as_float(r[c][i0 + 4]));
+                a = fmax3(a, __uint_as_float(r[c][i0 + 5]), __uint_as_float(r[c][i0 + 6]));
+                mx8[q] = fmaxf(a, __uint_as_float(r[c][i0 + 7]));
             }
-            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
+            const float mx = fmax3(fmax3(mx8[0], mx8[1], mx8[2]), fmax3(mx8[3], mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])) * scale_log2;
             if (j == 0) {
-                m_used = (mx == -INFINITY) ? 0.f : mx;
+                m_used = (mx == -INFINITY) ? -1e30f : mx;     // a half with no visible key yet: any finite reference
             } else {
                 const bool grow = mx > m_used + kRescaleThreshold;
                 if (__any_sync(0xffffffffu, grow)) {
-                    // all UMMAs issued before S(j), PV(j-1) included, have completed: O is stable
+                    // O_h must be stable: PV(j-1) complete (PV(j) is not issued before this thread arrives)
+                    if (!mbar_wait(bars + F_O, (j - 1) & 1, abortp, status, ERR_O)) { ok = false; break; }
+                    tc_fence_after();
                     const float alpha = grow ? ex2(m_used - mx) : 1.f;
                     if (grow) m_used = mx;
                     l *= alpha;
-                    // rare path, kept small: the 128 score registers stay live across it
 #pragma unroll 1
-                    for (int c = 0; c < D; c += 8) {
-                        uint32_t o[8];
-                        tmem_ld(lane_addr + kColO + c, o);
+                    for (int c = 0; c < D; c += 16) {   // rare path
+                        uint32_t o[16];
+                        tmem_ld(lane_addr + ocol + c, o);
                         tc_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                        tmem_st(lane_addr + kColO + c, o);
+                        for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st(lane_addr + ocol + c, o);
                     }
                 }
             }
-            // P = 2^(s scale_log2 - m_used), row sum, bf16 P into TMEM over the first 64 of the S
-            // columns.  Arithmetic runs on fp32 pairs (f32x2) to halve the instruction count.
+            // P = 2^(s scale_log2 - m_used), row sum, bf16 P into TMEM over the first 32 of this half's
+            // score columns.  Arithmetic runs on fp32 pairs (f32x2) to halve the instruction count.
             const uint64_t sl2 = pack_f32x2(scale_log2, scale_log2);
             const uint64_t negm2 = pack_f32x2(-m_used, -m_used);
             uint64_t ls2[2] = {0ull, 0ull};
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < 2; ++c) {
                 uint32_t pk[16];
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
@@ -210,7 +255,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                     ls2[(i >> 1) & 1] = add_f32x2(ls2[(i >> 1) & 1], pack_f32x2(p0, p1));
                     pk[i / 2] = pack_bf16(p0, p1);
                 }
-                tmem_st(lane_addr + kColP + 16 * c, pk);
+                tmem_st(lane_addr + scol + 16 * c, pk);
             }
             {
                 float s0, s1, s2, s3;
@@ -220,42 +265,55 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             }
             tc_wait_st();
             tc_fence_before();
-            mbar_arrive(&bar_p);
+            mbar_arrive(bars + F_P + 2 * (j & 1) + h);
         }
-        if (ok && mbar_wait(&bar_o, (nkt - 1) & 1, abortp, status, ERR_O)) {
+        // ---- epilogue: merge the two key halves.  Each thread publishes (m, l) of its half, then
+        // writes D/2 output columns of its row from both accumulators.
+        float2 *xch = reinterpret_cast<float2 *>(bars + F_COUNT + 2);   // [2][128] (m, l)
+        xch[h * 128 + lane_row] = make_float2(m_used, l);
+        mbar_arrive(bars + F_X);
+        if (ok && mbar_wait(bars + F_X, 0, abortp, status, ERR_P) &&
+            mbar_wait(bars + F_O, (nkt - 1) & 1, abortp, status, ERR_O)) {
             tc_fence_after();
-            const float inv = 1.f / l;
-            __nv_bfloat16 *orow = O + ((size_t)bh * n + row) * D;
+            const float2 other = xch[(h ^ 1) * 128 + lane_row];
+            const float m_all = fmaxf(m_used, other.x);
+            const float a_me = ex2(m_used - m_all), a_ot = ex2(other.x - m_all);
+            const float l_all = l * a_me + other.y * a_ot;
+            const float inv = 1.f / l_all;
+            const float w0 = (h == 0 ? a_me : a_ot) * inv, w1 = (h == 0 ? a_ot : a_me) * inv;   // weights of O_0, O_1
+            __nv_bfloat16 *orow = O + ((size_t)bh * n + row) * D + (D / 2) * h;
 #pragma unroll
-            for (int c = 0; c < D; c += 32) {
-                uint32_t r[32];
-                tmem_ld(lane_addr + kColO + c, r);
+            for (int c = 0; c < D / 2; c += 32) {
+                uint32_t o0[32], o1[32];
+                tmem_ld(lane_addr + kColO + (D / 2) * h + c, o0);
+                tmem_ld(lane_addr + kColO + D + (D / 2) * h + c, o1);
                 tc_wait_ld();
                 if (row < n) {
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {
-                        uint4 v;
-                        v.x = pack_bf16(__uint_as_float(r[i + 0]) * inv, __uint_as_float(r[i + 1]) * inv);
-                        v.y = pack_bf16(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
-                        v.z = pack_bf16(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv);
-                        v.w = pack_bf16(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv);
-                        *reinterpret_cast<uint4 *>(orow + c + i) = v;
+                        float v[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) v[u] = __uint_as_float(o0[i + u]) * w0 + __uint_as_float(o1[i + u]) * w1;
+                        uint4 q;
+                        q.x = pack_bf16(v[0], v[1]); q.y = pack_bf16(v[2], v[3]);
+                        q.z = pack_bf16(v[4], v[5]); q.w = pack_bf16(v[6], v[7]);
+                        *reinterpret_cast<uint4 *>(orow + c + i) = q;
                     }
                 }
             }
-            if (row < n) L[(size_t)bh * n + row] = m_used * kLn2 + logf(l);
+            if (row < n && h == 0) L[(size_t)bh * n + row] = m_all * kLn2 + logf(l_all);
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) tmem_dealloc(tbase, kTmemCols);
+    if (warp == 9) tmem_dealloc(tbase, kTmemCols);
 }
 
 template <int D>
 cudaError_t launch_fwd(const Problem &p, const void *Q, const void *K, const void *V, void *O, float *L,
                        cudaStream_t st)
 {
-    constexpr int kSmem = 3 * 128 * D * 2 + 1024;
+    constexpr int kSmem = 5 * 128 * D * 2 + 8 * (F_COUNT + 2) + 2 * 128 * 8;
     CUtensorMap mq, mk, mv;
     const uint64_t heads = (uint64_t)p.BH();
     if (!make_tensor_map_3d(&mq, Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
