@@ -368,20 +368,30 @@ simt_bwd_dq_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__
     }
 }
 
-__global__ void convert_kernel(const float *__restrict__ src, __nv_bfloat16 *__restrict__ dst, size_t count,
-                               float mul)
+// HBM-bound (4 bytes read, 2 written per element): grid-stride over float4 groups, four
+// independent loads in flight per thread, streaming loads (the accumulator is not read again).
+__global__ void __launch_bounds__(256)
+convert_kernel(const float *__restrict__ src, __nv_bfloat16 *__restrict__ dst, size_t count, float mul)
 {
-    size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
-    if (i + 3 < count) {
-        const float4 v = *reinterpret_cast<const float4 *>(src + i);
+    const size_t quads = count / 4;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    size_t q = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    auto put = [&](size_t at, const float4 v) {
         __nv_bfloat162 a = __floats2bfloat162_rn(v.x * mul, v.y * mul), b = __floats2bfloat162_rn(v.z * mul, v.w * mul);
         uint2 u;
         u.x = *reinterpret_cast<uint32_t *>(&a);
         u.y = *reinterpret_cast<uint32_t *>(&b);
-        *reinterpret_cast<uint2 *>(dst + i) = u;
-    } else {
-        for (; i < count; ++i) dst[i] = __float2bfloat16_rn(src[i] * mul);
+        *reinterpret_cast<uint2 *>(dst + 4 * at) = u;
+    };
+    const float4 *s4 = reinterpret_cast<const float4 *>(src);
+    for (; q + 3 * stride < quads; q += 4 * stride) {
+        const float4 v0 = __ldcs(s4 + q), v1 = __ldcs(s4 + q + stride), v2 = __ldcs(s4 + q + 2 * stride),
+                     v3 = __ldcs(s4 + q + 3 * stride);
+        put(q, v0); put(q + stride, v1); put(q + 2 * stride, v2); put(q + 3 * stride, v3);
     }
+    for (; q < quads; q += stride) put(q, __ldcs(s4 + q));
+    if (blockIdx.x == 0 && threadIdx.x == 0)
+        for (size_t i = quads * 4; i < count; ++i) dst[i] = __float2bfloat16_rn(src[i] * mul);
 }
 
 constexpr size_t fwd_smem(int D) { return (size_t)(3 * BM * (D + 1) + BM * SLD) * sizeof(float); }
@@ -482,7 +492,10 @@ cudaError_t row_dot(const Problem &p, int dtype, const void *dO, const void *O, 
 cudaError_t convert_f32_to_bf16(const float *src, void *dst, size_t count, float mul, cudaStream_t st)
 {
     const size_t quads = (count + 3) / 4;
-    const unsigned grid = (unsigned)((quads + 255) / 256);
+    size_t blocks = (quads + 4 * 256 - 1) / (4 * 256);
+    if (blocks < 1) blocks = 1;
+    if (blocks > 148 * 16) blocks = 148 * 16;     // grid-stride beyond 16 blocks per SM
+    const unsigned grid = (unsigned)blocks;
     LaunchScope scope(MOA_KERNEL_CONVERT, st);
     convert_kernel<<<grid, 256, 0, st>>>(src, (__nv_bfloat16 *)dst, count, mul);
     return cudaGetLastError();

@@ -68,36 +68,58 @@ __device__ __forceinline__ void red_add_v4(float *addr, float a, float b, float 
 
 // Lp = -L log2(e) and Dp = -rowsum(dO o O), both padded per head to n_pad rows (-inf and 0
 // past n).  Stored negated so that the kernels can use them as fma / add operands directly.
-// One warp per padded row.
+// HBM-bound (reads 2 * D * 2 bytes per row): every lane fetches 16 bytes of dO and of O, a row
+// takes D/8 lanes, and a warp has kPasses independent row groups in flight before it reduces.
 template <int D>
-__global__ void bwd_preprocess_kernel(const __nv_bfloat16 *__restrict__ dO, const __nv_bfloat16 *__restrict__ O,
-                                      const float *__restrict__ L, float *__restrict__ Lp, float *__restrict__ Dp,
-                                      int n, int n_pad, size_t padded_rows)
+__global__ void __launch_bounds__(256)
+bwd_preprocess_kernel(const __nv_bfloat16 *__restrict__ dO, const __nv_bfloat16 *__restrict__ O,
+                      const float *__restrict__ L, float *__restrict__ Lp, float *__restrict__ Dp,
+                      int n, int n_pad, size_t padded_rows)
 {
-    const size_t prow = (size_t)blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
-    if (prow >= padded_rows) return;
+    constexpr int kLanesPerRow = D / 8;
+    constexpr int kRowsPerPass = 32 / kLanesPerRow;
+    constexpr int kPasses = 4;
     const int lane = threadIdx.x % 32;
-    const size_t bh = prow / n_pad;
-    const int r = (int)(prow % n_pad);
-    if (r >= n) {
-        if (lane == 0) { Lp[prow] = -INFINITY; Dp[prow] = 0.f; }
-        return;
-    }
-    const size_t row = bh * n + r;
-    float acc = 0.f;
-    constexpr int kPerLane = D / 32;   // 2 or 4 consecutive elements
-    const __nv_bfloat16 *a = dO + row * D + lane * kPerLane;
-    const __nv_bfloat16 *b = O + row * D + lane * kPerLane;
+    const int sub = lane / kLanesPerRow, l = lane % kLanesPerRow;
+    const size_t warp_global = (size_t)blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
+    const size_t prow0 = warp_global * (kRowsPerPass * kPasses) + sub;
+    uint4 a[kPasses], b[kPasses];
+    float lv[kPasses];
+    bool real[kPasses];
 #pragma unroll
-    for (int i = 0; i < kPerLane; i += 2) {
-        const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(a + i));
-        const float2 y = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(b + i));
-        acc = fmaf(x.x, y.x, acc);
-        acc = fmaf(x.y, y.y, acc);
+    for (int p = 0; p < kPasses; ++p) {
+        const size_t prow = prow0 + (size_t)p * kRowsPerPass;
+        const size_t bh = prow / (size_t)n_pad;
+        const int r = (int)(prow - bh * (size_t)n_pad);
+        real[p] = prow < padded_rows && r < n;
+        a[p] = b[p] = make_uint4(0u, 0u, 0u, 0u);
+        lv[p] = 0.f;
+        if (real[p]) {
+            const size_t row = bh * (size_t)n + r;
+            a[p] = __ldcs(reinterpret_cast<const uint4 *>(dO + row * D) + l);
+            b[p] = __ldcs(reinterpret_cast<const uint4 *>(O + row * D) + l);
+            if (l == 0) lv[p] = L[row];
+        }
     }
 #pragma unroll
-    for (int o = 16; o >= 1; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) { Dp[prow] = -acc; Lp[prow] = -L[row] * kLog2e; }
+    for (int p = 0; p < kPasses; ++p) {
+        const uint32_t x[4] = {a[p].x, a[p].y, a[p].z, a[p].w}, y[4] = {b[p].x, b[p].y, b[p].z, b[p].w};
+        float acc = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 u = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&x[i]));
+            const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&y[i]));
+            acc = fmaf(u.x, v.x, acc);
+            acc = fmaf(u.y, v.y, acc);
+        }
+#pragma unroll
+        for (int o = kLanesPerRow / 2; o >= 1; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        const size_t prow = prow0 + (size_t)p * kRowsPerPass;
+        if (l == 0 && prow < padded_rows) {
+            Dp[prow] = real[p] ? -acc : 0.f;
+            Lp[prow] = real[p] ? -lv[p] * kLog2e : -INFINITY;
+        }
+    }
 }
 
 // kBulk: the dQ tile goes out through the TMA add-reduce; that needs 32 KB of staging, which is
@@ -566,7 +588,8 @@ cudaError_t tc_bwd_preprocess(const Problem &p, const void *dO, const void *O, c
     const int n_pad = (p.n + 127) / 128 * 128;
     const size_t rows = (size_t)p.BH() * n_pad;
     const int wpb = 8;
-    const unsigned grid = (unsigned)((rows + wpb - 1) / wpb);
+    const size_t rows_per_block = (size_t)wpb * (32 / (p.d / 8)) * 4;   // warps x rows per pass x passes
+    const unsigned grid = (unsigned)((rows + rows_per_block - 1) / rows_per_block);
     LaunchScope scope(MOA_KERNEL_PREPROCESS, st);
     if (p.d == 64)
         bwd_preprocess_kernel<64><<<grid, wpb * 32, 0, st>>>((const __nv_bfloat16 *)dO, (const __nv_bfloat16 *)O, L,
