@@ -156,7 +156,8 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
               const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapdO,
               const __grid_constant__ CUtensorMap mapdQ, const float *__restrict__ Lp, const float *__restrict__ Dp,
               __nv_bfloat16 *__restrict__ dK, __nv_bfloat16 *__restrict__ dV, float *__restrict__ dQacc,
-              int n, int n_pad, int causal, float scale, float scale_log2, int nkt, int skip_dq, unsigned int *status)
+              int n, int n_pad, int causal, float scale, float scale_log2, int nkt, int hpg, int skip_dq,
+              unsigned int *status)
 {
     using SM = BwdSmem<D, kBulk>;
     constexpr int kDoSlots = SM::kDoSlots;
@@ -178,8 +179,8 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     volatile uint32_t *abortp = reinterpret_cast<uint32_t *>(bars + B_COUNT + 1);
 
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
-    const int bh = blockIdx.x / nkt;
-    const int kt = blockIdx.x % nkt;          // causal: key tile 0 has the most query tiles and goes first
+    int bh, kt;                               // causal: key tile 0 has the most query tiles and goes first
+    job_from_block((int)blockIdx.x, nkt, (int)gridDim.x / nkt, hpg, bh, kt);
     const int k0 = kt * 128;
     const int nqt = n_pad / 128;
     const int i_begin = causal ? kt : 0;
@@ -576,7 +577,7 @@ cudaError_t launch_bwd(const Problem &p, const void *Q, const void *K, const voi
     LaunchScope scope(MOA_KERNEL_BWD_KV, st);
     tc_bwd_kernel<D, kBulk><<<(unsigned)(nkt * p.BH()), kThreads, kSmem, st>>>(
         mq, mk, mv, mdo, mdq, Lp, Dp, (__nv_bfloat16 *)dK, (__nv_bfloat16 *)dV, dQacc, p.n, nkt * 128, p.causal,
-        p.scale, p.scale * kLog2e, nkt, dQacc == nullptr ? 1 : 0, device_status_ptr());
+        p.scale, p.scale * kLog2e, nkt, heads_per_group(p, nkt), dQacc == nullptr ? 1 : 0, device_status_ptr());
     return cudaGetLastError();
 }
 

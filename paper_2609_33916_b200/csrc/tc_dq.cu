@@ -43,7 +43,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 tc_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
              const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapdO,
              const float *__restrict__ Lp, const float *__restrict__ Dp, __nv_bfloat16 *__restrict__ dQ,
-             int n, int n_pad, int causal, float scale, float scale_log2, int nqt, unsigned int *status)
+             int n, int n_pad, int causal, float scale, float scale_log2, int nqt, int hpg,
+             unsigned int *status)
 {
     using SM = DqSmem<D>;
     constexpr int kBoxes = D / 64;
@@ -55,8 +56,8 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
     volatile uint32_t *abortp = reinterpret_cast<uint32_t *>(bars + B_COUNT + 1);
 
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
-    const int bh = blockIdx.x / nqt;
-    const int t = blockIdx.x % nqt;
+    int bh, t;
+    job_from_block((int)blockIdx.x, nqt, (int)gridDim.x / nqt, hpg, bh, t);
     const int qt = causal ? nqt - 1 - t : t;   // causal: longest rows first
     const int q0 = qt * 128;
     const int nkt_all = n_pad / 128;
@@ -219,7 +220,7 @@ cudaError_t launch_dq(const Problem &p, const void *Q, const void *K, const void
     LaunchScope scope(MOA_KERNEL_BWD_DQ, st);
     tc_dq_kernel<D><<<(unsigned)(nqt * p.BH()), kThreads, kSmem, st>>>(
         mq, mk, mv, mdo, Lp, Dp, (__nv_bfloat16 *)dQ, p.n, nqt * 128, p.causal, p.scale, p.scale * kLog2e, nqt,
-        device_status_ptr());
+        heads_per_group(p, nqt), device_status_ptr());
     return cudaGetLastError();
 }
 

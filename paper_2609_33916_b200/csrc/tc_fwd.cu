@@ -52,7 +52,7 @@ template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
               const __grid_constant__ CUtensorMap mapV, __nv_bfloat16 *__restrict__ O, float *__restrict__ L,
-              int n, int causal, float scale_log2, int nqt, unsigned int *status)
+              int n, int causal, float scale_log2, int nqt, int hpg, unsigned int *status)
 {
     constexpr int kTileBytes = 128 * D * 2;
     constexpr int kBoxes = D / 64;         // 64-column (128-byte) swizzled boxes per tile
@@ -64,8 +64,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     volatile uint32_t *abortp = reinterpret_cast<uint32_t *>(bars + F_COUNT + 1);
 
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
-    const int bh = blockIdx.x / nqt;
-    const int t = blockIdx.x % nqt;
+    int bh, t;
+    job_from_block((int)blockIdx.x, nqt, (int)gridDim.x / nqt, hpg, bh, t);
     const int qt = causal ? nqt - 1 - t : t;   // causal: longest rows first
     const int q0 = qt * BM;
     const int nkt_all = (n + BN - 1) / BN;
@@ -325,7 +325,7 @@ cudaError_t launch_fwd(const Problem &p, const void *Q, const void *K, const voi
     const int nqt = (p.n + BM - 1) / BM;
     LaunchScope scope(MOA_KERNEL_FWD, st);
     tc_fwd_kernel<D><<<(unsigned)(nqt * p.BH()), kThreads, kSmem, st>>>(
-        mq, mk, mv, (__nv_bfloat16 *)O, L, p.n, p.causal, p.scale * kLog2e, nqt, device_status_ptr());
+        mq, mk, mv, (__nv_bfloat16 *)O, L, p.n, p.causal, p.scale * kLog2e, nqt, heads_per_group(p, nqt), device_status_ptr());
     return cudaGetLastError();
 }
 
