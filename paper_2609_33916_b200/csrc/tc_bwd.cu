@@ -147,15 +147,16 @@ struct BwdSmem {
 enum {
     B_KV = 0, B_QFULL = 1 /*2*/, B_QEMPTY = 3 /*2*/, B_DOFULL = 5 /*2*/, B_DOEMPTY = 7 /*2*/,
     B_S = 9, B_P = 10, B_DP = 11, B_DS = 12, B_DQ = 13, B_DQR = 14, B_STGFREE = 15 /*2*/, B_STGFULL = 17 /*2*/,
-    B_COUNT = 19
+    B_EPI = 19 /*dK, dV tiles staged in shared memory*/, B_COUNT = 20
 };
 
 template <int D, bool kBulk>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
               const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapdO,
-              const __grid_constant__ CUtensorMap mapdQ, const float *__restrict__ Lp, const float *__restrict__ Dp,
-              __nv_bfloat16 *__restrict__ dK, __nv_bfloat16 *__restrict__ dV, float *__restrict__ dQacc,
+              const __grid_constant__ CUtensorMap mapdQ, const __grid_constant__ CUtensorMap mapdK,
+              const __grid_constant__ CUtensorMap mapdV, const float *__restrict__ Lp, const float *__restrict__ Dp,
+              float *__restrict__ dQacc,
               int n, int n_pad, int causal, float scale, float scale_log2, int nkt, int hpg, int skip_dq,
               unsigned int *status)
 {
@@ -188,7 +189,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
 
     if (tid == 0) {
         for (int b = 0; b < B_COUNT; ++b) {
-            const uint32_t cnt = (b == B_P || b == B_DS) ? 256u
+            const uint32_t cnt = (b == B_P || b == B_DS || b == B_EPI) ? 256u
                                : (b == B_DQR || b == B_STGFULL || b == B_STGFULL + 1) ? 128u : 1u;
             mbar_init(bars + b, cnt);
         }
@@ -197,6 +198,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         fence_mbar_init();
         prefetch_tensormap(&mapQ); prefetch_tensormap(&mapK); prefetch_tensormap(&mapV); prefetch_tensormap(&mapdO);
         if (dq_bulk) prefetch_tensormap(&mapdQ);
+        prefetch_tensormap(&mapdK); prefetch_tensormap(&mapdV);
     }
     if (warp == kMmaWarp) { tmem_alloc(tmem_base_s, kTmemCols); tmem_relinquish(); }
     tc_fence_before();
@@ -523,31 +525,44 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             if (it + 1 < niter) ok = p_phase(it + 1);
         }
         if (ok && mbar_wait(bars + B_DQ, (niter - 1) & 1, abortp, status, ERR_DQ)) {
-            // all UMMAs have completed: write dV and scale*dK rows of this key
+            // All UMMAs have completed.  dV and scale*dK go out as bf16 through shared memory (the K and V
+            // tiles are no longer read) and TMA stores: a thread owns a row, so direct stores would be 16
+            // bytes at a 2D-byte stride, one 128-byte line per lane and instruction -- 4096 line requests
+            // per CTA, which kept the load/store unit busy for ~3 us; staged, the tile leaves as
+            // full lines, and rows past n are clipped by the tensor map.
             tc_fence_after();
-            const int krow = k0 + lane_row;
 #pragma unroll
             for (int which = 0; which < 2; ++which) {
                 const uint32_t col = (which == 0 ? colDV : colDK) + (D / 2) * wg;
                 const float mul = which == 0 ? 1.f : scale;
-                __nv_bfloat16 *outp = (which == 0 ? dV : dK) + ((size_t)bh * n + krow) * D + (D / 2) * wg;
+                uint8_t *stage = which == 0 ? sV : sK;
 #pragma unroll
                 for (int c = 0; c < D / 2; c += 32) {
                     uint32_t r[32];
                     tmem_ld(lane_addr + col + c, r);
                     tc_wait_ld();
-                    if (krow < n) {
 #pragma unroll
-                        for (int e = 0; e < 32; e += 8) {
-                            uint4 v;
-                            v.x = pack_bf16(__uint_as_float(r[e + 0]) * mul, __uint_as_float(r[e + 1]) * mul);
-                            v.y = pack_bf16(__uint_as_float(r[e + 2]) * mul, __uint_as_float(r[e + 3]) * mul);
-                            v.z = pack_bf16(__uint_as_float(r[e + 4]) * mul, __uint_as_float(r[e + 5]) * mul);
-                            v.w = pack_bf16(__uint_as_float(r[e + 6]) * mul, __uint_as_float(r[e + 7]) * mul);
-                            *reinterpret_cast<uint4 *>(outp + c + e) = v;
-                        }
+                    for (int e = 0; e < 32; e += 8) {
+                        uint4 v;
+                        v.x = pack_bf16(__uint_as_float(r[e + 0]) * mul, __uint_as_float(r[e + 1]) * mul);
+                        v.y = pack_bf16(__uint_as_float(r[e + 2]) * mul, __uint_as_float(r[e + 3]) * mul);
+                        v.z = pack_bf16(__uint_as_float(r[e + 4]) * mul, __uint_as_float(r[e + 5]) * mul);
+                        v.w = pack_bf16(__uint_as_float(r[e + 6]) * mul, __uint_as_float(r[e + 7]) * mul);
+                        const int cabs = (D / 2) * wg + c + e;          // first of 8 columns
+                        const int chunk = ((cabs & 63) >> 3) ^ (lane_row & 7);   // 128-byte swizzle, as the maps expect
+                        *reinterpret_cast<uint4 *>(stage + (cabs >> 6) * kBoxBytes + lane_row * 128 + chunk * 16) = v;
                     }
                 }
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(bars + B_EPI);
+            if (tid == 0 && mbar_wait(bars + B_EPI, 0, abortp, status, ERR_DQ)) {
+                for (int b = 0; b < kBoxes; ++b) {
+                    tma_store_3d(&mapdV, sV + b * kBoxBytes, 64 * b, k0, bh);
+                    tma_store_3d(&mapdK, sK + b * kBoxBytes, 64 * b, k0, bh);
+                }
+                bulk_commit();
+                bulk_wait_read<0>();      // shared memory is read before the CTA may exit
             }
         }
     }
@@ -560,12 +575,14 @@ template <int D, bool kBulk>
 cudaError_t launch_bwd(const Problem &p, const void *Q, const void *K, const void *V, const void *dO,
                        const float *Lp, const float *Dp, void *dK, void *dV, float *dQacc, cudaStream_t st)
 {
-    CUtensorMap mq, mk, mv, mdo, mdq;
+    CUtensorMap mq, mk, mv, mdo, mdq, mdk, mdv;
     const uint64_t heads = (uint64_t)p.BH();
     if (!make_tensor_map_3d(&mq, Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
         !make_tensor_map_3d(&mk, K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
         !make_tensor_map_3d(&mv, V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mdo, dO, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64))
+        !make_tensor_map_3d(&mdo, dO, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
+        !make_tensor_map_3d(&mdk, dK, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
+        !make_tensor_map_3d(&mdv, dV, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64))
         return cudaErrorInvalidValue;
     // fp32 accumulator as [heads, n, D] with boxes of 32 rows x D floats (no swizzle); also encoded when unused
     if (!make_tensor_map_3d(&mdq, dQacc ? (const void *)dQacc : Q, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, heads, p.n, D, 32, D))
@@ -576,7 +593,7 @@ cudaError_t launch_bwd(const Problem &p, const void *Q, const void *K, const voi
     const int nkt = (p.n + 127) / 128;
     LaunchScope scope(MOA_KERNEL_BWD_KV, st);
     tc_bwd_kernel<D, kBulk><<<(unsigned)(nkt * p.BH()), kThreads, kSmem, st>>>(
-        mq, mk, mv, mdo, mdq, Lp, Dp, (__nv_bfloat16 *)dK, (__nv_bfloat16 *)dV, dQacc, p.n, nkt * 128, p.causal,
+        mq, mk, mv, mdo, mdq, mdk, mdv, Lp, Dp, dQacc, p.n, nkt * 128, p.causal,
         p.scale, p.scale * kLog2e, nkt, heads_per_group(p, nkt), dQacc == nullptr ? 1 : 0, device_status_ptr());
     return cudaGetLastError();
 }
