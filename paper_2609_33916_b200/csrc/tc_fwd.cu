@@ -46,12 +46,13 @@ enum : uint32_t { ERR_Q = 0x101, ERR_K = 0x102, ERR_V = 0x103, ERR_S = 0x104, ER
 
 enum { F_Q = 0, F_KFULL = 1 /*2*/, F_KEMPTY = 3 /*2*/, F_VFULL = 5 /*2*/, F_VEMPTY = 7 /*2*/, F_S = 9 /*2*/,
        F_P = 11 /*[buffer][half]: 4*/, F_O = 15, F_X = 16 /*epilogue exchange*/, F_OB = 17 /*2: score buffer consumed*/,
-       F_COUNT = 19 };
+       F_E = 19 /*O tile staged in shared memory*/, F_COUNT = 20 };
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
-              const __grid_constant__ CUtensorMap mapV, __nv_bfloat16 *__restrict__ O, float *__restrict__ L,
+              const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapO,
+              float *__restrict__ L,
               int n, int causal, float scale_log2, int nqt, int hpg, unsigned int *status)
 {
     constexpr int kTileBytes = 128 * D * 2;
@@ -72,11 +73,11 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     const int nkt_want = causal ? min(qt + 1, nkt_all) : nkt_all;
 
     if (tid == 0) {
-        for (int b = 0; b < F_COUNT; ++b) mbar_init(bars + b, (b >= F_P && b < F_P + 4) ? 128u : (b == F_X ? 256u : 1u));
+        for (int b = 0; b < F_COUNT; ++b) mbar_init(bars + b, (b >= F_P && b < F_P + 4) ? 128u : ((b == F_X || b == F_E) ? 256u : 1u));
         *abortp = (smem_u32(sm) & 1023u) ? 1u : 0u;
         if (*abortp && status) atomicCAS(status, 0u, 0x108u);
         fence_mbar_init();
-        prefetch_tensormap(&mapQ); prefetch_tensormap(&mapK); prefetch_tensormap(&mapV);
+        prefetch_tensormap(&mapQ); prefetch_tensormap(&mapK); prefetch_tensormap(&mapV); prefetch_tensormap(&mapO);
     }
     if (warp == 9) { tmem_alloc(tmem_base_p, kTmemCols); tmem_relinquish(); }
     tc_fence_before();
@@ -281,25 +282,34 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             const float l_all = l * a_me + other.y * a_ot;
             const float inv = 1.f / l_all;
             const float w0 = (h == 0 ? a_me : a_ot) * inv, w1 = (h == 0 ? a_ot : a_me) * inv;   // weights of O_0, O_1
-            __nv_bfloat16 *orow = O + ((size_t)bh * n + row) * D + (D / 2) * h;
+            // O leaves as bf16 through shared memory (the Q tile is no longer read) and a TMA store: a
+            // thread owns a row, so direct stores would be 16 bytes at a 2D-byte stride, one 128-byte line
+            // per lane and instruction.  Rows past n are clipped by the tensor map.
 #pragma unroll
             for (int c = 0; c < D / 2; c += 32) {
                 uint32_t o0[32], o1[32];
                 tmem_ld(lane_addr + kColO + (D / 2) * h + c, o0);
                 tmem_ld(lane_addr + kColO + D + (D / 2) * h + c, o1);
                 tc_wait_ld();
-                if (row < n) {
 #pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        float v[8];
+                for (int i = 0; i < 32; i += 8) {
+                    float v[8];
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) v[u] = __uint_as_float(o0[i + u]) * w0 + __uint_as_float(o1[i + u]) * w1;
-                        uint4 q;
-                        q.x = pack_bf16(v[0], v[1]); q.y = pack_bf16(v[2], v[3]);
-                        q.z = pack_bf16(v[4], v[5]); q.w = pack_bf16(v[6], v[7]);
-                        *reinterpret_cast<uint4 *>(orow + c + i) = q;
-                    }
+                    for (int u = 0; u < 8; ++u) v[u] = __uint_as_float(o0[i + u]) * w0 + __uint_as_float(o1[i + u]) * w1;
+                    uint4 q;
+                    q.x = pack_bf16(v[0], v[1]); q.y = pack_bf16(v[2], v[3]);
+                    q.z = pack_bf16(v[4], v[5]); q.w = pack_bf16(v[6], v[7]);
+                    const int cabs = (D / 2) * h + c + i;                        // first of 8 columns
+                    const int chunk = ((cabs & 63) >> 3) ^ (lane_row & 7);       // 128-byte swizzle, as the map expects
+                    *reinterpret_cast<uint4 *>(sQ + (cabs >> 6) * kBoxBytes + lane_row * 128 + chunk * 16) = q;
                 }
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(bars + F_E);
+            if (tid == 0 && mbar_wait(bars + F_E, 0, abortp, status, ERR_O)) {
+                for (int b = 0; b < kBoxes; ++b) tma_store_3d(&mapO, sQ + b * kBoxBytes, 64 * b, q0, bh);
+                bulk_commit();
+                bulk_wait_read<0>();      // shared memory is read before the CTA may exit
             }
             if (row < n && h == 0) L[(size_t)bh * n + row] = m_all * kLn2 + logf(l_all);
         }
@@ -314,18 +324,19 @@ cudaError_t launch_fwd(const Problem &p, const void *Q, const void *K, const voi
                        cudaStream_t st)
 {
     constexpr int kSmem = 5 * 128 * D * 2 + 8 * (F_COUNT + 2) + 2 * 128 * 8;
-    CUtensorMap mq, mk, mv;
+    CUtensorMap mq, mk, mv, mo;
     const uint64_t heads = (uint64_t)p.BH();
     if (!make_tensor_map_3d(&mq, Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
         !make_tensor_map_3d(&mk, K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mv, V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64))
+        !make_tensor_map_3d(&mv, V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
+        !make_tensor_map_3d(&mo, O, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64))
         return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
     const int nqt = (p.n + BM - 1) / BM;
     LaunchScope scope(MOA_KERNEL_FWD, st);
     tc_fwd_kernel<D><<<(unsigned)(nqt * p.BH()), kThreads, kSmem, st>>>(
-        mq, mk, mv, (__nv_bfloat16 *)O, L, p.n, p.causal, p.scale * kLog2e, nqt, heads_per_group(p, nqt), device_status_ptr());
+        mq, mk, mv, mo, L, p.n, p.causal, p.scale * kLog2e, nqt, heads_per_group(p, nqt), device_status_ptr());
     return cudaGetLastError();
 }
 
