@@ -54,7 +54,7 @@ template <int D>
 __global__ void __launch_bounds__(192, 1)
 mat_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                const __grid_constant__ CUtensorMap mapV, __nv_bfloat16 *__restrict__ O, float *__restrict__ L,
-               __nv_bfloat16 *__restrict__ PT, int n, int n_pad, int causal, float scale_log2, int nqt,
+               __nv_bfloat16 *__restrict__ PT, int n, int n_pad, int causal, float scale_log2, int nqt, int hpg,
                unsigned int *status)
 {
     constexpr int kTile = 128 * D * 2;
@@ -68,8 +68,8 @@ mat_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     volatile uint32_t *abortp = reinterpret_cast<uint32_t *>(bars + 7);
 
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
-    const int bh = blockIdx.x / nqt;
-    const int t = blockIdx.x % nqt;
+    int bh, t;
+    job_from_block((int)blockIdx.x, nqt, (int)gridDim.x / nqt, hpg, bh, t);
     const int qt = causal ? nqt - 1 - t : t;
     const int q0 = qt * 128;
     const int nkt_all = n_pad / 128;
@@ -247,7 +247,7 @@ mat_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
                const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapdO,
                const float *__restrict__ Dp, const __nv_bfloat16 *__restrict__ PT, __nv_bfloat16 *__restrict__ GST,
                __nv_bfloat16 *__restrict__ dK, __nv_bfloat16 *__restrict__ dV,
-               int n, int n_pad, int causal, float scale, int nkt, unsigned int *status)
+               int n, int n_pad, int causal, float scale, int nkt, int hpg, unsigned int *status)
 {
     using SM = MatBwdSmem<D>;
     constexpr int kBoxes = D / 64;
@@ -259,8 +259,8 @@ mat_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     volatile uint32_t *abortp = reinterpret_cast<uint32_t *>(bars + MB_COUNT + 1);
 
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
-    const int bh = blockIdx.x / nkt;
-    const int kt = blockIdx.x % nkt;
+    int bh, kt;
+    job_from_block((int)blockIdx.x, nkt, (int)gridDim.x / nkt, hpg, bh, kt);
     const int k0 = kt * 128;
     const int nqt = n_pad / 128;
     const int i_begin = causal ? kt : 0;
@@ -432,7 +432,7 @@ enum : uint32_t { QERR = 0x600 };
 template <int D>
 __global__ void __launch_bounds__(192, 1)
 mat_dq_kernel(const __grid_constant__ CUtensorMap mapGST, const __grid_constant__ CUtensorMap mapK,
-              __nv_bfloat16 *__restrict__ dQ, int n, int n_pad, int causal, float scale, int nqt, unsigned int *status)
+              __nv_bfloat16 *__restrict__ dQ, int n, int n_pad, int causal, float scale, int nqt, int hpg, unsigned int *status)
 {
     constexpr int kTileK = 128 * D * 2, kTileG = 128 * 128 * 2;
     constexpr int kBoxes = D / 64;
@@ -444,8 +444,8 @@ mat_dq_kernel(const __grid_constant__ CUtensorMap mapGST, const __grid_constant_
     volatile uint32_t *abortp = reinterpret_cast<uint32_t *>(bars + 6);
 
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
-    const int bh = blockIdx.x / nqt;
-    const int t = blockIdx.x % nqt;
+    int bh, t;
+    job_from_block((int)blockIdx.x, nqt, (int)gridDim.x / nqt, hpg, bh, t);
     const int qt = causal ? nqt - 1 - t : t;
     const int q0 = qt * 128;
     const int nkt_all = n_pad / 128;
@@ -543,7 +543,7 @@ cudaError_t run_group(const Problem &p, const void *Q, const void *K, const void
         LaunchScope scope(MOA_KERNEL_FWD, st);
         mat_fwd_kernel<D><<<(unsigned)(nt * p.BH()), 192, kSmem, st>>>(mq, mk, mv, (__nv_bfloat16 *)O, L, (__nv_bfloat16 *)PT,
                                                                       p.n, n_pad, p.causal, p.scale * kLog2e, nt,
-                                                                      device_status_ptr());
+                                                                      heads_per_group(p, nt), device_status_ptr());
         return cudaGetLastError();
     }
     if (!make_tensor_map_3d(&mdo, dO, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
@@ -556,7 +556,7 @@ cudaError_t run_group(const Problem &p, const void *Q, const void *K, const void
         mat_bwd_kernel<D><<<(unsigned)(nt * p.BH()), 320, kSmem, st>>>(mq, mk, mv, mdo, Dp_group, (const __nv_bfloat16 *)PT,
                                                                       (__nv_bfloat16 *)GST, (__nv_bfloat16 *)dK,
                                                                       (__nv_bfloat16 *)dV, p.n, n_pad, p.causal, p.scale, nt,
-                                                                      device_status_ptr());
+                                                                      heads_per_group(p, nt), device_status_ptr());
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     {
@@ -564,7 +564,7 @@ cudaError_t run_group(const Problem &p, const void *Q, const void *K, const void
         if ((e = cudaFuncSetAttribute(mat_dq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem)) != cudaSuccess) return e;
         LaunchScope scope(MOA_KERNEL_BWD_DQ, st);
         mat_dq_kernel<D><<<(unsigned)(nt * p.BH()), 192, kSmem, st>>>(mg, mk, (__nv_bfloat16 *)dQ, p.n, n_pad, p.causal, p.scale,
-                                                                     nt, device_status_ptr());
+                                                                     nt, heads_per_group(p, nt), device_status_ptr());
         return cudaGetLastError();
     }
 }
