@@ -21,9 +21,12 @@
 // TMEM (512 columns): score buffers [0,128) and [128,256), O_0 [256,256+D), O_1 [256+D,256+2D).
 // S, P and the O accumulators never leave the SM: nothing of size n x n reaches HBM.
 //
-// What bounds it (config 4, d = 128): one exp2 per score keeps the MUFU unit as busy as the
-// tensor pipe (both 0.92 ms of a 2.0 ms kernel); the rest is the softmax warps' non-MUFU work
-// and hand-off latency.
+// What bounds it (config 4, d = 128): per 128 x 128 tile the UMMAs need 1024 cycles, the one exp2
+// per score 1024 cycles of the MUFU unit, and shared memory 1250 cycles (an SS UMMA streams both
+// operands at the full 128 B/clk: 64 KB for S, 32 KB of V for PV, 64 KB of TMA writes); the tile
+// takes ~1850 because the two softmax warpgroups run their exp2 phases at the same time and the
+// rest of their work (TMEM load, max, hand-offs, ~600 cycles) is not hidden under them.
+// The O tile leaves through the Q tile's shared memory and a TMA store.
 #include "common.cuh"
 #include "ptx.cuh"
 #include "tensormap.cuh"
