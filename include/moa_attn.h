@@ -89,6 +89,12 @@ typedef struct {
                             writes P and dS to the workspace and reads them back (the paper's
                             "left" ONF, Sec. 1.1); needs an O(n^2) workspace.                  */
     int32_t path;        /* moa_path                                                           */
+    int32_t H_kv;        /* key/value heads.  0 or H: one K/V head per query head.  Otherwise
+                            H_kv must divide H, and query head h reads K/V head h / (H / H_kv):
+                            grouped-query attention (H_kv = 1: multi-query), the head sharing the
+                            paper's decode section treats.  K, V, dK, dV are then [B,H_kv,n,d];
+                            dK, dV sum the contributions of the H / H_kv query heads of a group.
+                            Tensor-core bf16 path only; other paths return MOA_ERR_UNSUPPORTED. */
 } moa_attn_desc;
 
 /* Bytes of caller-provided workspace `op` (a moa_op) needs for `desc`.  Returns 0

@@ -8,6 +8,7 @@ from .attention import (  # noqa: F401
     build,
     num_threads,
     attn_fwd_bwd,
+    attn_fwd_bwd_gqa,
     attn_head_full,
     attn_rows,
     attn_cols,

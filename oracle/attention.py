@@ -107,6 +107,24 @@ def attn_fwd_bwd(Q, K, V, dO, causal: bool, scale: float):
     return dict(O=O, L=L, dQ=dQ, dK=dK, dV=dV)
 
 
+def attn_fwd_bwd_gqa(Q, K, V, dO, causal: bool, scale: float):
+    """Grouped-query attention written out from its definition: Q, dO are [B,H,n,d] and K, V are
+    [B,H_kv,n,d] with H_kv dividing H; query head h attends to K/V head h // (H/H_kv).  Every query
+    head is an ordinary attention head over a copy of its K/V head, and a shared K/V head's gradient
+    is the sum of the gradients of its copies (the head sharing the paper's decode section treats).
+    Returns O, L, dQ as [B,H,...] and dK, dV as [B,H_kv,n,d]."""
+    Q, K, V, dO = map(_f64, (Q, K, V, dO))
+    B, H, n, d = Q.shape
+    Hkv = K.shape[1]
+    if K.shape != (B, Hkv, n, d) or V.shape != K.shape or dO.shape != Q.shape or Hkv < 1 or H % Hkv:
+        raise ValueError("expected Q, dO [B,H,n,d] and K, V [B,H_kv,n,d] with H_kv dividing H")
+    G = H // Hkv
+    r = attn_fwd_bwd(Q, np.repeat(K, G, axis=1), np.repeat(V, G, axis=1), dO, causal, scale)
+    r["dK"] = r["dK"].reshape(B, Hkv, G, n, d).sum(axis=2)
+    r["dV"] = r["dV"].reshape(B, Hkv, G, n, d).sum(axis=2)
+    return r
+
+
 def attn_head_full(Q, K, V, dO, causal: bool, scale: float):
     """One head ([n,d] inputs); additionally returns the n x n arrays P and dS
     and the row vector D, for the invariants the tests check."""

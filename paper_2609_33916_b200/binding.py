@@ -32,7 +32,8 @@ EXPORTS = (
 class moa_attn_desc(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("n", ctypes.c_int32), ("d", ctypes.c_int32),
                 ("causal", ctypes.c_int32), ("scale", ctypes.c_float), ("dtype", ctypes.c_int32),
-                ("dq_mode", ctypes.c_int32), ("materialize", ctypes.c_int32), ("path", ctypes.c_int32)]
+                ("dq_mode", ctypes.c_int32), ("materialize", ctypes.c_int32), ("path", ctypes.c_int32),
+                ("H_kv", ctypes.c_int32)]
 
 
 MOA_KERNEL_KINDS = 6
@@ -86,9 +87,10 @@ def lib() -> ctypes.CDLL:
 
 
 def make_desc(B, H, n, d, causal, scale, dtype=MOA_BF16, dq_mode=MOA_DQ_AUTO, materialize=0,
-              path=MOA_PATH_AUTO) -> moa_attn_desc:
+              path=MOA_PATH_AUTO, H_kv=0) -> moa_attn_desc:
+    """H_kv: key/value heads (0 or H: one per query head; a divisor of H: grouped-query attention)."""
     return moa_attn_desc(int(B), int(H), int(n), int(d), int(bool(causal)), float(scale), int(dtype),
-                         int(dq_mode), int(materialize), int(path))
+                         int(dq_mode), int(materialize), int(path), int(H_kv))
 
 
 def _ptr(x):

@@ -12,7 +12,11 @@ struct Problem {
     int B, H, n, d;
     int causal;
     float scale;
+    int Hkv = 0;                                   // key/value heads; 0: same as H
     int BH() const { return B * H; }
+    int kv_heads() const { return Hkv > 0 ? Hkv : H; }
+    int group() const { return H / kv_heads(); }    // query heads per key/value head
+    int BHkv() const { return B * kv_heads(); }
 };
 
 // Block order of the tile-parallel kernels.  Heads are taken in groups of `hpg`; inside a group

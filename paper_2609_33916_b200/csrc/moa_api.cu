@@ -106,6 +106,12 @@ moa_status check_desc(const moa_attn_desc *d)
         !(d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->d == 128 && d->scale > 0.f))
         return MOA_ERR_UNSUPPORTED;
     if (d->path == MOA_PATH_TC && !(d->scale > 0.f)) return MOA_ERR_UNSUPPORTED;   // non-positive scale: SIMT path only
+    if (d->H_kv < 0 || d->H_kv > d->H) return MOA_ERR_INVALID_ARG;
+    if (d->H_kv > 0 && d->H % d->H_kv != 0) return MOA_ERR_INVALID_ARG;
+    // shared K/V heads: tensor-core kernels only
+    if (d->H_kv > 0 && d->H_kv != d->H &&
+        !(d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->scale > 0.f && !d->materialize))
+        return MOA_ERR_UNSUPPORTED;
     return MOA_OK;
 }
 
@@ -172,7 +178,7 @@ MatWorkspace mat_workspace(const moa_attn_desc *d, int op)
     return w;
 }
 
-Problem to_problem(const moa_attn_desc *d) { return Problem{d->B, d->H, d->n, d->d, d->causal, d->scale}; }
+Problem to_problem(const moa_attn_desc *d) { return Problem{d->B, d->H, d->n, d->d, d->causal, d->scale, d->H_kv}; }
 
 // Materialising variant.  with_bwd = false: forward only (P^T is written and dropped).
 moa_status run_materialized(const moa_attn_desc *d, const void *Q, const void *K, const void *V, const void *dO,
@@ -188,7 +194,7 @@ moa_status run_materialized(const moa_attn_desc *d, const void *Q, const void *K
     const size_t esz = 2, hs = (size_t)d->n * d->d * esz;
     for (int g0 = 0; g0 < heads; g0 += w.group) {
         const int g = heads - g0 < w.group ? heads - g0 : w.group;
-        Problem p{1, g, d->n, d->d, d->causal, d->scale};
+        Problem p{1, g, d->n, d->d, d->causal, d->scale, 0};
         const char *q = (const char *)Q + g0 * hs, *k = (const char *)K + g0 * hs, *v = (const char *)V + g0 * hs;
         char *o = (char *)O + g0 * hs;
         float *l = L + (size_t)g0 * d->n;

@@ -157,8 +157,8 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
               const __grid_constant__ CUtensorMap mapdQ, const __grid_constant__ CUtensorMap mapdK,
               const __grid_constant__ CUtensorMap mapdV, const float *__restrict__ Lp, const float *__restrict__ Dp,
               float *__restrict__ dQacc,
-              int n, int n_pad, int causal, float scale, float scale_log2, int nkt, int hpg, int skip_dq,
-              unsigned int *status)
+              int n, int n_pad, int causal, float scale, float scale_log2, int nkt, int hpg, int group,
+              int skip_dq, unsigned int *status)
 {
     using SM = BwdSmem<D, kBulk>;
     constexpr int kDoSlots = SM::kDoSlots;
@@ -185,7 +185,13 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     const int k0 = kt * 128;
     const int nqt = n_pad / 128;
     const int i_begin = causal ? kt : 0;
-    const int niter_all = nqt - i_begin;
+    // With shared K/V heads (group > 1) `bh` counts K/V heads and the CTA walks the query tiles of
+    // all `group` query heads that read this K/V tile: dK and dV accumulate over the whole group in
+    // TMEM, still written once by one CTA, with no atomics.
+    const int nq_per = nqt - i_begin;
+    const int niter_all = group * nq_per;
+    auto q_head = [&](int it) { return bh * group + it / nq_per; };
+    auto q_tile = [&](int it) { return i_begin + it % nq_per; };
 
     if (tid == 0) {
         for (int b = 0; b < B_COUNT; ++b) {
@@ -227,18 +233,18 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         // issued in the middle of tile i.  dO has one slot: it is read only by dP(i) and dV(i),
         // early in tile i, and is refilled as soon as dV(i) has completed.
         auto load_q = [&](int it) {
-            const int s = it & 1, q0 = (i_begin + it) * 128;
+            const int s = it & 1, q0 = q_tile(it) * 128, qh = q_head(it);
             uint8_t *sQ = sm + SM::offQ + s * SM::kTile;
             mbar_arrive_expect_tx(bars + B_QFULL + s, SM::kTile + 1024);
-            for (int b = 0; b < kBoxes; ++b) tma_load_3d(sQ + b * kBoxBytes, &mapQ, bars + B_QFULL + s, 64 * b, q0, bh);
-            bulk_load_1d(sL + s * 128, Lp + (size_t)bh * n_pad + q0, 512, bars + B_QFULL + s);
-            bulk_load_1d(sD + s * 128, Dp + (size_t)bh * n_pad + q0, 512, bars + B_QFULL + s);
+            for (int b = 0; b < kBoxes; ++b) tma_load_3d(sQ + b * kBoxBytes, &mapQ, bars + B_QFULL + s, 64 * b, q0, qh);
+            bulk_load_1d(sL + s * 128, Lp + (size_t)qh * n_pad + q0, 512, bars + B_QFULL + s);
+            bulk_load_1d(sD + s * 128, Dp + (size_t)qh * n_pad + q0, 512, bars + B_QFULL + s);
         };
         auto load_do = [&](int it) {
-            const int s = it % kDoSlots, q0 = (i_begin + it) * 128;
+            const int s = it % kDoSlots, q0 = q_tile(it) * 128, qh = q_head(it);
             uint8_t *sdO = sm + SM::offdO + s * SM::kTile;
             mbar_arrive_expect_tx(bars + B_DOFULL + s, SM::kTile);
-            for (int b = 0; b < kBoxes; ++b) tma_load_3d(sdO + b * kBoxBytes, &mapdO, bars + B_DOFULL + s, 64 * b, q0, bh);
+            for (int b = 0; b < kBoxes; ++b) tma_load_3d(sdO + b * kBoxBytes, &mapdO, bars + B_DOFULL + s, 64 * b, q0, qh);
         };
         if (lane == 0 && niter > 0) {
             load_q(0);
@@ -360,14 +366,14 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         const int lane_row = 32 * (warp % 4) + lane;
         const uint32_t lane_addr = tbase + ((uint32_t)(32 * (warp % 4)) << 16);
         for (int it = 0; it < (skip_dq ? 0 : niter); ++it) {
-            const int qrow = (i_begin + it) * 128 + lane_row;
+            const int qrow = q_tile(it) * 128 + lane_row, qh = q_head(it);
             if (!mbar_wait(bars + B_DQ, it & 1, abortp, status, ERR_DQ)) break;
             tc_fence_after();
             uint32_t r[D / 32][32];
             if (kTransposeDQ) {
                 // lanes are d (this thread: column lane_row of every dQ row), TMEM columns are queries
-                const int q0 = (i_begin + it) * 128;
-                float *dst = dQacc + ((size_t)bh * n + q0) * D + lane_row;
+                const int q0 = q_tile(it) * 128;
+                float *dst = dQacc + ((size_t)qh * n + q0) * D + lane_row;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) tmem_ld(lane_addr + colDQ + 32 * c, r[c]);
                 tc_wait_ld();
@@ -397,7 +403,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                         }
                         mbar_arrive(bars + B_STGFULL + st);
                         if (leader && stage_ok && mbar_wait(bars + B_STGFULL + st, (g >> 1) & 1, abortp, status, ERR_STAGE)) {
-                            tma_reduce_add_3d(&mapdQ, stage, 0, q0 + 32 * c, bh);
+                            tma_reduce_add_3d(&mapdQ, stage, 0, q0 + 32 * c, qh);
                             bulk_commit();
                         }
                     }
@@ -411,7 +417,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                             if (32 * c + e < valid) red_add_f32(dst + (size_t)(32 * c + e) * D, __uint_as_float(r[c][e]));
                 }
             } else {
-                float *dst = dQacc + ((size_t)bh * n + qrow) * D;
+                float *dst = dQacc + ((size_t)qh * n + qrow) * D;
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) tmem_ld(lane_addr + colDQ + 32 * c, r[c]);
                 tc_wait_ld();
@@ -444,7 +450,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         // its scheduler with these warps.
         auto p_phase = [&](int it) -> bool {
             const int s = it & 1;
-            const bool diag = causal && (i_begin + it == kt);
+            const bool diag = causal && (q_tile(it) == kt);
             if (!mbar_wait(bars + B_S, it & 1, abortp, status, ERR_SDP)) return false;
             tc_fence_after();
             const float *Ls = sL + s * 128;    // -L log2e
@@ -576,13 +582,13 @@ cudaError_t launch_bwd(const Problem &p, const void *Q, const void *K, const voi
                        const float *Lp, const float *Dp, void *dK, void *dV, float *dQacc, cudaStream_t st)
 {
     CUtensorMap mq, mk, mv, mdo, mdq, mdk, mdv;
-    const uint64_t heads = (uint64_t)p.BH();
+    const uint64_t heads = (uint64_t)p.BH(), kv_heads = (uint64_t)p.BHkv();
     if (!make_tensor_map_3d(&mq, Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mk, K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mv, V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
+        !make_tensor_map_3d(&mk, K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, kv_heads, p.n, D, 128, 64) ||
+        !make_tensor_map_3d(&mv, V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, kv_heads, p.n, D, 128, 64) ||
         !make_tensor_map_3d(&mdo, dO, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mdk, dK, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mdv, dV, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64))
+        !make_tensor_map_3d(&mdk, dK, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, kv_heads, p.n, D, 128, 64) ||
+        !make_tensor_map_3d(&mdv, dV, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, kv_heads, p.n, D, 128, 64))
         return cudaErrorInvalidValue;
     // fp32 accumulator as [heads, n, D] with boxes of 32 rows x D floats (no swizzle); also encoded when unused
     if (!make_tensor_map_3d(&mdq, dQacc ? (const void *)dQacc : Q, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, heads, p.n, D, 32, D))
@@ -592,9 +598,13 @@ cudaError_t launch_bwd(const Problem &p, const void *Q, const void *K, const voi
     if (e != cudaSuccess) return e;
     const int nkt = (p.n + 127) / 128;
     LaunchScope scope(MOA_KERNEL_BWD_KV, st);
-    tc_bwd_kernel<D, kBulk><<<(unsigned)(nkt * p.BH()), kThreads, kSmem, st>>>(
+    // one CTA per (K/V head, key tile); the block order groups K/V heads
+    Problem pkv = p;
+    pkv.H = p.kv_heads();
+    pkv.Hkv = 0;
+    tc_bwd_kernel<D, kBulk><<<(unsigned)(nkt * p.BHkv()), kThreads, kSmem, st>>>(
         mq, mk, mv, mdo, mdq, mdk, mdv, Lp, Dp, dQacc, p.n, nkt * 128, p.causal,
-        p.scale, p.scale * kLog2e, nkt, heads_per_group(p, nkt), dQacc == nullptr ? 1 : 0, device_status_ptr());
+        p.scale, p.scale * kLog2e, nkt, heads_per_group(pkv, nkt), p.group(), dQacc == nullptr ? 1 : 0, device_status_ptr());
     return cudaGetLastError();
 }
 

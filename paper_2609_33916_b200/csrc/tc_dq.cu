@@ -44,7 +44,7 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
              const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapdO,
              const float *__restrict__ Lp, const float *__restrict__ Dp, __nv_bfloat16 *__restrict__ dQ,
              int n, int n_pad, int causal, float scale, float scale_log2, int nqt, int hpg,
-             unsigned int *status)
+             int group, unsigned int *status)
 {
     using SM = DqSmem<D>;
     constexpr int kBoxes = D / 64;
@@ -58,6 +58,7 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
     int bh, t;
     job_from_block((int)blockIdx.x, nqt, (int)gridDim.x / nqt, hpg, bh, t);
+    const int kvh = bh / group;                 // the K/V head this query head reads
     const int qt = causal ? nqt - 1 - t : t;   // causal: longest rows first
     const int q0 = qt * 128;
     const int nkt_all = n_pad / 128;
@@ -92,8 +93,8 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
             if (lane == 0) {
                 mbar_arrive_expect_tx(bars + B_KVFULL + s, 2 * SM::kTile);
                 for (int b = 0; b < kBoxes; ++b) {
-                    tma_load_3d(sm + SM::offK + s * SM::kTile + b * kBoxBytes, &mapK, bars + B_KVFULL + s, 64 * b, j * 128, bh);
-                    tma_load_3d(sm + SM::offV + s * SM::kTile + b * kBoxBytes, &mapV, bars + B_KVFULL + s, 64 * b, j * 128, bh);
+                    tma_load_3d(sm + SM::offK + s * SM::kTile + b * kBoxBytes, &mapK, bars + B_KVFULL + s, 64 * b, j * 128, kvh);
+                    tma_load_3d(sm + SM::offV + s * SM::kTile + b * kBoxBytes, &mapV, bars + B_KVFULL + s, 64 * b, j * 128, kvh);
                 }
             }
             __syncwarp();
@@ -209,8 +210,8 @@ cudaError_t launch_dq(const Problem &p, const void *Q, const void *K, const void
     CUtensorMap mq, mk, mv, mdo;
     const uint64_t heads = (uint64_t)p.BH();
     if (!make_tensor_map_3d(&mq, Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mk, K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mv, V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
+        !make_tensor_map_3d(&mk, K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)p.BHkv(), p.n, D, 128, 64) ||
+        !make_tensor_map_3d(&mv, V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)p.BHkv(), p.n, D, 128, 64) ||
         !make_tensor_map_3d(&mdo, dO, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64))
         return cudaErrorInvalidValue;
     constexpr int kSmem = DqSmem<D>::kTotal;
@@ -220,7 +221,7 @@ cudaError_t launch_dq(const Problem &p, const void *Q, const void *K, const void
     LaunchScope scope(MOA_KERNEL_BWD_DQ, st);
     tc_dq_kernel<D><<<(unsigned)(nqt * p.BH()), kThreads, kSmem, st>>>(
         mq, mk, mv, mdo, Lp, Dp, (__nv_bfloat16 *)dQ, p.n, nqt * 128, p.causal, p.scale, p.scale * kLog2e, nqt,
-        heads_per_group(p, nqt), device_status_ptr());
+        heads_per_group(p, nqt), p.group(), device_status_ptr());
     return cudaGetLastError();
 }
 

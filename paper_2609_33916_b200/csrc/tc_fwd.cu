@@ -56,7 +56,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
               const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapO,
               float *__restrict__ L,
-              int n, int causal, float scale_log2, int nqt, int hpg, unsigned int *status)
+              int n, int causal, float scale_log2, int nqt, int hpg, int group, unsigned int *status)
 {
     constexpr int kTileBytes = 128 * D * 2;
     constexpr int kBoxes = D / 64;         // 64-column (128-byte) swizzled boxes per tile
@@ -70,6 +70,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
     int bh, t;
     job_from_block((int)blockIdx.x, nqt, (int)gridDim.x / nqt, hpg, bh, t);
+    const int kvh = bh / group;                 // the K/V head this query head reads (group > 1: shared heads)
     const int qt = causal ? nqt - 1 - t : t;   // causal: longest rows first
     const int q0 = qt * BM;
     const int nkt_all = (n + BN - 1) / BN;
@@ -101,13 +102,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             if (lane == 0) {
                 mbar_arrive_expect_tx(bars + F_KFULL + s, kTileBytes);
                 for (int b = 0; b < kBoxes; ++b)
-                    tma_load_3d(sK + s * kTileBytes + b * kBoxBytes, &mapK, bars + F_KFULL + s, 64 * b, j * BN, bh);
+                    tma_load_3d(sK + s * kTileBytes + b * kBoxBytes, &mapK, bars + F_KFULL + s, 64 * b, j * BN, kvh);
             }
             if (j >= 2 && !mbar_wait(bars + F_VEMPTY + s, ((j >> 1) - 1) & 1, abortp, status, ERR_V)) break;
             if (lane == 0) {
                 mbar_arrive_expect_tx(bars + F_VFULL + s, kTileBytes);
                 for (int b = 0; b < kBoxes; ++b)
-                    tma_load_3d(sV + s * kTileBytes + b * kBoxBytes, &mapV, bars + F_VFULL + s, 64 * b, j * BN, bh);
+                    tma_load_3d(sV + s * kTileBytes + b * kBoxBytes, &mapV, bars + F_VFULL + s, 64 * b, j * BN, kvh);
             }
             __syncwarp();
         }
@@ -330,8 +331,8 @@ cudaError_t launch_fwd(const Problem &p, const void *Q, const void *K, const voi
     CUtensorMap mq, mk, mv, mo;
     const uint64_t heads = (uint64_t)p.BH();
     if (!make_tensor_map_3d(&mq, Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mk, K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mv, V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
+        !make_tensor_map_3d(&mk, K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)p.BHkv(), p.n, D, 128, 64) ||
+        !make_tensor_map_3d(&mv, V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)p.BHkv(), p.n, D, 128, 64) ||
         !make_tensor_map_3d(&mo, O, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64))
         return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
@@ -339,7 +340,7 @@ cudaError_t launch_fwd(const Problem &p, const void *Q, const void *K, const voi
     const int nqt = (p.n + BM - 1) / BM;
     LaunchScope scope(MOA_KERNEL_FWD, st);
     tc_fwd_kernel<D><<<(unsigned)(nqt * p.BH()), kThreads, kSmem, st>>>(
-        mq, mk, mv, mo, L, p.n, p.causal, p.scale * kLog2e, nqt, heads_per_group(p, nqt), device_status_ptr());
+        mq, mk, mv, mo, L, p.n, p.causal, p.scale * kLog2e, nqt, heads_per_group(p, nqt), p.group(), device_status_ptr());
     return cudaGetLastError();
 }
 

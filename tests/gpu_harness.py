@@ -28,12 +28,14 @@ def run_library(inp: dict, dtype: str, causal: bool, scale: float, *, op: str = 
                 poison: bool = True) -> dict:
     """op: 'fused' (one call) or 'split' (moa_attn_fwd then moa_attn_bwd) or 'fwd'."""
     B, H, n, d = inp["Q"].shape
+    Hkv = inp["K"].shape[1]          # fewer K/V heads than query heads: grouped-query attention
     Q, K, V, dO = (to_device(inp[k], dtype) for k in ("Q", "K", "V", "dO"))
     desc = mb.make_desc(B, H, n, d, causal, scale, mb.MOA_BF16 if dtype == "bf16" else mb.MOA_F32,
-                        dq_mode, materialize, path)
+                        dq_mode, materialize, path, H_kv=0 if Hkv == H else Hkv)
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
     fill = float("nan") if poison else 0.0   # unwritten elements must show up
-    O, dQ, dK, dV = (torch.full((B, H, n, d), fill, dtype=tdt, device="cuda") for _ in range(4))
+    O, dQ = (torch.full((B, H, n, d), fill, dtype=tdt, device="cuda") for _ in range(2))
+    dK, dV = (torch.full((B, Hkv, n, d), fill, dtype=tdt, device="cuda") for _ in range(2))
     L = torch.full((B, H, n), fill, dtype=torch.float32, device="cuda")
     ws_bytes = mb.moa_attn_workspace_bytes(desc, mb.MOA_OP_FUSED if op != "fwd" else mb.MOA_OP_FWD)
     if materialize and op == "split":

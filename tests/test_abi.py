@@ -35,7 +35,7 @@ def test_version_and_strings(lib):
 
 
 def test_desc_struct_layout_matches_header():
-    assert ctypes.sizeof(mb.moa_attn_desc) == 40
+    assert ctypes.sizeof(mb.moa_attn_desc) == 44
     assert mb.moa_attn_desc.scale.offset == 20
 
 
@@ -85,3 +85,19 @@ def test_argument_errors_need_no_device(lib):
     assert mb.moa_attn_fused_fwd_bwd(d, a, a, a, a, a, a, a, a, a, a, ws_bytes=need - 1, check=False) == mb.MOA_ERR_WORKSPACE
     with pytest.raises(mb.MoaError):
         mb.moa_attn_fwd(good, 0, a, a, a, a)
+
+
+def test_shared_kv_heads_argument_checks(lib):
+    a = 4096  # fake, aligned, never dereferenced: checks fail first
+    def fwd(**kw):
+        d = mb.make_desc(1, 8, 256, 128, True, 0.1, **kw)
+        return mb.moa_attn_fwd(d, a, a, a, a, a, a, ws_bytes=1 << 40, check=False)
+    assert fwd(H_kv=3) == mb.MOA_ERR_INVALID_ARG           # must divide H
+    assert fwd(H_kv=16) == mb.MOA_ERR_INVALID_ARG
+    assert fwd(H_kv=-1) == mb.MOA_ERR_INVALID_ARG
+    assert fwd(H_kv=2, dtype=mb.MOA_F32) == mb.MOA_ERR_UNSUPPORTED      # tensor-core bf16 path only
+    assert fwd(H_kv=2, path=mb.MOA_PATH_SIMT) == mb.MOA_ERR_UNSUPPORTED
+    assert fwd(H_kv=2, materialize=1) == mb.MOA_ERR_UNSUPPORTED
+    # the workspace does not depend on the number of K/V heads: D, L' and the dQ accumulator are per query head
+    w = lambda hkv: mb.moa_attn_workspace_bytes(mb.make_desc(1, 8, 256, 128, True, 0.1, H_kv=hkv), mb.MOA_OP_FUSED)
+    assert w(0) == w(8) == w(2) == w(1) > 0

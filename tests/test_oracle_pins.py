@@ -182,6 +182,45 @@ def test_against_torch_autograd(causal):
     np.testing.assert_allclose(r["L"], torch.logsumexp(s, -1).numpy(), atol=1e-13)
 
 
+# ------------------------------------- grouped-query attention (shared K/V heads)
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("Hkv", [1, 2, 6])
+def test_gqa_against_torch_autograd(causal, Hkv):
+    """K/V heads shared by groups of query heads: torch's own grouped-query attention on the CPU
+    (an independent implementation) gives the same O and, through autograd, the same gradients
+    -- dK, dV summed over the query heads of a group."""
+    torch = pytest.importorskip("torch")
+    B, H, n, d, scale = 2, 6, 19, 5, 0.37
+    rng = np.random.default_rng(17)
+    Q, dO = (rng.standard_normal((B, H, n, d)) for _ in range(2))
+    K, V = (rng.standard_normal((B, Hkv, n, d)) for _ in range(2))
+    r = oracle.attn_fwd_bwd_gqa(Q, K, V, dO, causal, scale)
+    assert r["dK"].shape == (B, Hkv, n, d) and r["dV"].shape == (B, Hkv, n, d)
+    q, k, v = (torch.tensor(x, dtype=torch.float64, requires_grad=True) for x in (Q, K, V))
+    o = torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=causal, scale=scale, enable_gqa=True)
+    o.backward(torch.tensor(dO))
+    for key, t in (("O", o.detach()), ("dQ", q.grad), ("dK", k.grad), ("dV", v.grad)):
+        np.testing.assert_allclose(r[key], t.numpy(), atol=1e-13, err_msg=key)
+
+
+def test_gqa_head_mapping_by_hand():
+    """Query head h reads K/V head h // (H / H_kv): with H = 4, H_kv = 2 heads 0, 1 use K/V head 0
+    and heads 2, 3 use K/V head 1, checked head by head against the single-head oracle."""
+    B, H, Hkv, n, d, scale = 1, 4, 2, 9, 3, 0.6
+    rng = np.random.default_rng(23)
+    Q, dO = (rng.standard_normal((B, H, n, d)) for _ in range(2))
+    K, V = (rng.standard_normal((B, Hkv, n, d)) for _ in range(2))
+    r = oracle.attn_fwd_bwd_gqa(Q, K, V, dO, True, scale)
+    dK = np.zeros((Hkv, n, d)); dV = np.zeros((Hkv, n, d))
+    for h, kv in ((0, 0), (1, 0), (2, 1), (3, 1)):
+        one = oracle.attn_head_full(Q[0, h], K[0, kv], V[0, kv], dO[0, h], True, scale)
+        np.testing.assert_allclose(r["O"][0, h], one["O"], atol=1e-14)
+        np.testing.assert_allclose(r["dQ"][0, h], one["dQ"], atol=1e-14)
+        dK[kv] += one["dK"]; dV[kv] += one["dV"]
+    np.testing.assert_allclose(r["dK"][0], dK, atol=1e-13)
+    np.testing.assert_allclose(r["dV"][0], dV, atol=1e-13)
+
+
 # --------------------------------------------------------- P6: brute force, tiny
 @pytest.mark.parametrize("causal", [False, True])
 def test_brute_force_no_max_subtraction(causal):

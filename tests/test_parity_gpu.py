@@ -223,6 +223,53 @@ def test_c5_causal_sweep_large_sizes_sampled(H, n):
     _sampled_check(H, w, heads=[(0, 31)] if n > 8192 else [(0, 0), (0, 31)], nrows=12, ncols=12)
 
 
+# ------------------------------------------- shared K/V heads (grouped-query attention)
+def _gqa_inputs(B, Hq, Hkv, n, d, seed):
+    q = mi.make_inputs(B, Hq, n, d, seed, "bf16")
+    kv = mi.make_inputs(B, Hkv, n, d, seed + 1000, "bf16")
+    return {"Q": q["Q"], "dO": q["dO"], "K": kv["K"], "V": kv["V"]}
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(4, 2), (6, 1), (8, 2)])
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("n,d", [(320, 128), (200, 64)])
+@pytest.mark.parametrize("dq_mode", [0, 1, 3])
+def test_gqa_matches_oracle(H, Hq, Hkv, causal, n, d, dq_mode):
+    """K, V, dK, dV are [B,H_kv,n,d]; a K/V head's gradient sums over its group of query heads,
+    accumulated inside one CTA without atomics.  Every element against the fp64 oracle."""
+    inp = _gqa_inputs(2, Hq, Hkv, n, d, seed=40 + Hq + n)
+    got = H.run_library(inp, "bf16", causal, 1.0 / math.sqrt(d), dq_mode=dq_mode)
+    f = H.f64_inputs(inp, "bf16")
+    ref = oracle.attn_fwd_bwd_gqa(f["Q"], f["K"], f["V"], f["dO"], causal, 1.0 / math.sqrt(d))
+    assert got["dK"].shape == ref["dK"].shape == (2, Hkv, n, d)
+    H.assert_close(got, ref, H.TOL_BF16, tag=f"gqa {Hq}/{Hkv} n{n} d{d} causal{causal} dq{dq_mode}")
+    assert mi.rel_err(got["L"], ref["L"]) <= 1e-3
+
+
+def test_gqa_fused_call_equals_fwd_then_bwd(H):
+    inp = _gqa_inputs(1, 8, 2, 384, 128, seed=77)
+    a = H.run_library(inp, "bf16", True, 0.09, op="fused", dq_mode=3)
+    b = H.run_library(inp, "bf16", True, 0.09, op="split", dq_mode=3)
+    for k in ("O", "L", "dQ", "dK", "dV"):
+        np.testing.assert_array_equal(a[k], b[k], err_msg=k)
+
+
+def test_gqa_equals_replicated_kv_heads(H):
+    """The same problem stated with every K/V head copied G times: O, L and dQ are identical bit for
+    bit in the deterministic mode, and the copies' dK, dV add up to the shared heads' (to rounding)."""
+    B, Hq, Hkv, n, d = 1, 8, 2, 512, 128
+    G = Hq // Hkv
+    inp = _gqa_inputs(B, Hq, Hkv, n, d, seed=91)
+    rep = dict(inp, K=np.repeat(inp["K"], G, axis=1), V=np.repeat(inp["V"], G, axis=1))
+    a = H.run_library(inp, "bf16", True, 0.088, dq_mode=3)
+    b = H.run_library(rep, "bf16", True, 0.088, dq_mode=3)
+    for k in ("O", "L", "dQ"):
+        np.testing.assert_array_equal(a[k], b[k], err_msg=k)
+    for k in ("dK", "dV"):
+        summed = b[k].reshape(B, Hkv, G, n, d).sum(2)
+        assert mi.rel_err(a[k], summed) <= 8e-3, k     # the copies were rounded to bf16 one by one
+
+
 def test_causal_block_order_with_a_partial_head_group(H):
     """Causal launches take the heads in groups (tile-major inside a group, so that the longest
     jobs start first).  19 heads at n = 4096, d = 128 make groups of 16 with a last group of 3:
