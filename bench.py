@@ -279,6 +279,8 @@ def main():
     ap.add_argument("--path", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--materialize", type=int, default=0)
+    ap.add_argument("--hkv", type=int, default=0,
+                    help="key/value heads (grouped-query attention); 0: one per query head, as in every named config")
     ap.add_argument("--sweep", action="store_true", help="config-5 strategy sweep (study table, not the contract line)")
     ap.add_argument("--sweep-sizes", default="")
     ap.add_argument("--dist-backend", default="nccl", help="control-plane backend for N > 1 (nccl; gloo for tests)")
@@ -321,13 +323,17 @@ def main():
     peaks, peaks_kind = load_peaks()
 
     B, H, n, d = w.B, w.H, w.n, w.d
-    desc = mb.make_desc(B, H, n, d, w.causal, w.scale, mb.MOA_BF16, args.dq_mode, args.materialize, args.path)
+    desc = mb.make_desc(B, H, n, d, w.causal, w.scale, mb.MOA_BF16, args.dq_mode, args.materialize, args.path,
+                        H_kv=args.hkv)
     shape = (B, H, n, d)
+    kv_shape = (B, args.hkv or H, n, d)       # K, V, dK, dV
+    shapes_in = (shape, kv_shape, kv_shape, shape)            # Q, K, V, dO
+    shapes_out = (shape, shape, kv_shape, kv_shape)           # O, dQ, dK, dV
     base_mem = torch.cuda.memory_allocated()
     gen = torch.Generator(device="cuda").manual_seed(w.seed + 1000 * rank)
-    Q, K, V, dO = (torch.randn(shape, generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
-                   for _ in range(4))
-    O, dQ, dK, dV = (torch.empty(shape, dtype=torch.bfloat16, device="cuda") for _ in range(4))
+    Q, K, V, dO = (torch.randn(sh, generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+                   for sh in shapes_in)
+    O, dQ, dK, dV = (torch.empty(sh, dtype=torch.bfloat16, device="cuda") for sh in shapes_out)
     L = torch.empty((B, H, n), dtype=torch.float32, device="cuda")
     ws_bytes = mb.moa_attn_workspace_bytes(desc, mb.MOA_OP_FUSED)
     ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device="cuda")
@@ -400,14 +406,14 @@ def main():
     # The three legs run on three streams over two buffer sets, so step k+1's upload and step
     # k-1's download overlap step k's kernels (the library call takes the stream it runs on).
     hQ, hK, hV, hdO = (t.cpu().pin_memory() for t in (Q, K, V, dO))
-    hO, hdQ, hdK, hdV = (torch.empty(shape, dtype=torch.bfloat16).pin_memory() for _ in range(4))
+    hO, hdQ, hdK, hdV = (torch.empty(sh, dtype=torch.bfloat16).pin_memory() for sh in shapes_out)
     hL = torch.empty((B, H, n), dtype=torch.float32).pin_memory()
     h2d = sum(t.numel() * t.element_size() for t in (hQ, hK, hV, hdO))
     d2h = sum(t.numel() * t.element_size() for t in (hO, hdQ, hdK, hdV, hL))
     sets = []
     for _ in range(2):
-        ins = [torch.empty(shape, dtype=torch.bfloat16, device="cuda") for _ in range(4)]
-        outs = [torch.empty(shape, dtype=torch.bfloat16, device="cuda") for _ in range(4)]
+        ins = [torch.empty(sh, dtype=torch.bfloat16, device="cuda") for sh in shapes_in]
+        outs = [torch.empty(sh, dtype=torch.bfloat16, device="cuda") for sh in shapes_out]
         sets.append({"in": ins, "out": outs, "L": torch.empty((B, H, n), dtype=torch.float32, device="cuda"),
                      "ws": torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device="cuda"),
                      "up": torch.cuda.Event(), "done": torch.cuda.Event(), "down": torch.cuda.Event()})
@@ -490,7 +496,9 @@ def main():
         "gpu_launches": int(launches),
         "roofline": roofline,
     }
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if args.hkv:
+        line["config"]["H_kv"] = args.hkv
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.hkv:
         v, dt, cores, desc_s = time_oracle_sample(w, 20.0)
         line["cpu_baseline"] = {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
                                 "sample": desc_s, "seconds": dt}

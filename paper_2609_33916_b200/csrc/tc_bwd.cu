@@ -150,7 +150,7 @@ enum {
     B_EPI = 19 /*dK, dV tiles staged in shared memory*/, B_COUNT = 20
 };
 
-template <int D, bool kBulk>
+template <int D, bool kBulk, bool kGrouped>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
               const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapdO,
@@ -188,10 +188,19 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     // With shared K/V heads (group > 1) `bh` counts K/V heads and the CTA walks the query tiles of
     // all `group` query heads that read this K/V tile: dK and dV accumulate over the whole group in
     // TMEM, still written once by one CTA, with no atomics.
-    const int nq_per = nqt - i_begin;
-    const int niter_all = group * nq_per;
-    auto q_head = [&](int it) { return bh * group + it / nq_per; };
-    auto q_tile = [&](int it) { return i_begin + it % nq_per; };
+    const int niter_all = (kGrouped ? group : 1) * (nqt - i_begin);
+    // (query head, query tile) of consecutive iterations, advanced without a division: each role
+    // keeps a walker of its own, in step with the iterations it handles.  kGrouped = false (one K/V
+    // head per query head) compiles to the plain tile counter.
+    struct TileWalk {
+        int qh, qi, first, end;
+        __device__ void next()
+        {
+            ++qi;
+            if (kGrouped && qi == end) { qi = first; ++qh; }
+        }
+    };
+    const TileWalk walk0{kGrouped ? bh * group : bh, i_begin, i_begin, nqt};
 
     if (tid == 0) {
         for (int b = 0; b < B_COUNT; ++b) {
@@ -232,8 +241,10 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         // Q tiles (with L, D) go through a two-slot ring and are fetched two tiles ahead: S(i+1) is
         // issued in the middle of tile i.  dO has one slot: it is read only by dP(i) and dV(i),
         // early in tile i, and is refilled as soon as dV(i) has completed.
+        TileWalk wq = walk0, wdo = walk0;     // load_q and load_do are each called for it = 0, 1, 2, ... in order
         auto load_q = [&](int it) {
-            const int s = it & 1, q0 = q_tile(it) * 128, qh = q_head(it);
+            const int s = it & 1, q0 = wq.qi * 128, qh = wq.qh;
+            wq.next();
             uint8_t *sQ = sm + SM::offQ + s * SM::kTile;
             mbar_arrive_expect_tx(bars + B_QFULL + s, SM::kTile + 1024);
             for (int b = 0; b < kBoxes; ++b) tma_load_3d(sQ + b * kBoxBytes, &mapQ, bars + B_QFULL + s, 64 * b, q0, qh);
@@ -241,7 +252,8 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             bulk_load_1d(sD + s * 128, Dp + (size_t)qh * n_pad + q0, 512, bars + B_QFULL + s);
         };
         auto load_do = [&](int it) {
-            const int s = it % kDoSlots, q0 = q_tile(it) * 128, qh = q_head(it);
+            const int s = it % kDoSlots, q0 = wdo.qi * 128, qh = wdo.qh;
+            wdo.next();
             uint8_t *sdO = sm + SM::offdO + s * SM::kTile;
             mbar_arrive_expect_tx(bars + B_DOFULL + s, SM::kTile);
             for (int b = 0; b < kBoxes; ++b) tma_load_3d(sdO + b * kBoxBytes, &mapdO, bars + B_DOFULL + s, 64 * b, q0, qh);
@@ -365,14 +377,16 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         // ------------------------------------------------- dQ reduce warps: lanes are query rows
         const int lane_row = 32 * (warp % 4) + lane;
         const uint32_t lane_addr = tbase + ((uint32_t)(32 * (warp % 4)) << 16);
+        TileWalk wr = walk0;
         for (int it = 0; it < (skip_dq ? 0 : niter); ++it) {
-            const int qrow = q_tile(it) * 128 + lane_row, qh = q_head(it);
+            const int qtile = wr.qi, qh = wr.qh, qrow = qtile * 128 + lane_row;
+            wr.next();
             if (!mbar_wait(bars + B_DQ, it & 1, abortp, status, ERR_DQ)) break;
             tc_fence_after();
             uint32_t r[D / 32][32];
             if (kTransposeDQ) {
                 // lanes are d (this thread: column lane_row of every dQ row), TMEM columns are queries
-                const int q0 = q_tile(it) * 128;
+                const int q0 = qtile * 128;
                 float *dst = dQacc + ((size_t)qh * n + q0) * D + lane_row;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) tmem_ld(lane_addr + colDQ + 32 * c, r[c]);
@@ -403,7 +417,12 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                         }
                         mbar_arrive(bars + B_STGFULL + st);
                         if (leader && stage_ok && mbar_wait(bars + B_STGFULL + st, (g >> 1) & 1, abortp, status, ERR_STAGE)) {
-                            tma_reduce_add_3d(&mapdQ, stage, 0, q0 + 32 * c, qh);
+                            // (query head, tile) of this iteration: recomputed here, by the one thread that
+                            // needs them, rather than kept live beside the 128 registers of the tile
+                            const int nq_per = nqt - i_begin;
+                            const int hh = kGrouped ? it / nq_per : 0;
+                            tma_reduce_add_3d(&mapdQ, stage, 0, (i_begin + it - hh * nq_per) * 128 + 32 * c,
+                                              (kGrouped ? bh * group : bh) + hh);
                             bulk_commit();
                         }
                     }
@@ -448,9 +467,11 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         // written as bf16 over the first half of this warpgroup's S^T columns.  Arithmetic is
         // on fp32 pairs (f32x2) to halve the instruction count: the UMMA-issuing warp shares
         // its scheduler with these warps.
+        TileWalk wp = walk0;
         auto p_phase = [&](int it) -> bool {
             const int s = it & 1;
-            const bool diag = causal && (q_tile(it) == kt);
+            const bool diag = causal && (wp.qi == kt);     // p_phase runs for it = 0, 1, 2, ... in order
+            wp.next();
             if (!mbar_wait(bars + B_S, it & 1, abortp, status, ERR_SDP)) return false;
             tc_fence_after();
             const float *Ls = sL + s * 128;    // -L log2e
@@ -577,8 +598,8 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     if (warp == kMmaWarp) tmem_dealloc(tbase, kTmemCols);
 }
 
-template <int D, bool kBulk>
-cudaError_t launch_bwd(const Problem &p, const void *Q, const void *K, const void *V, const void *dO,
+template <int D, bool kBulk, bool kGrouped>
+cudaError_t launch_bwd_g(const Problem &p, const void *Q, const void *K, const void *V, const void *dO,
                        const float *Lp, const float *Dp, void *dK, void *dV, float *dQacc, cudaStream_t st)
 {
     CUtensorMap mq, mk, mv, mdo, mdq, mdk, mdv;
@@ -594,7 +615,7 @@ cudaError_t launch_bwd(const Problem &p, const void *Q, const void *K, const voi
     if (!make_tensor_map_3d(&mdq, dQacc ? (const void *)dQacc : Q, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, heads, p.n, D, 32, D))
         return cudaErrorInvalidValue;
     constexpr int kSmem = BwdSmem<D, kBulk>::kTotal;
-    cudaError_t e = cudaFuncSetAttribute(tc_bwd_kernel<D, kBulk>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    cudaError_t e = cudaFuncSetAttribute(tc_bwd_kernel<D, kBulk, kGrouped>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
     const int nkt = (p.n + 127) / 128;
     LaunchScope scope(MOA_KERNEL_BWD_KV, st);
@@ -602,10 +623,18 @@ cudaError_t launch_bwd(const Problem &p, const void *Q, const void *K, const voi
     Problem pkv = p;
     pkv.H = p.kv_heads();
     pkv.Hkv = 0;
-    tc_bwd_kernel<D, kBulk><<<(unsigned)(nkt * p.BHkv()), kThreads, kSmem, st>>>(
+    tc_bwd_kernel<D, kBulk, kGrouped><<<(unsigned)(nkt * p.BHkv()), kThreads, kSmem, st>>>(
         mq, mk, mv, mdo, mdq, mdk, mdv, Lp, Dp, dQacc, p.n, nkt * 128, p.causal,
         p.scale, p.scale * kLog2e, nkt, heads_per_group(pkv, nkt), p.group(), dQacc == nullptr ? 1 : 0, device_status_ptr());
     return cudaGetLastError();
+}
+
+template <int D, bool kBulk>
+cudaError_t launch_bwd(const Problem &p, const void *Q, const void *K, const void *V, const void *dO,
+                       const float *Lp, const float *Dp, void *dK, void *dV, float *dQacc, cudaStream_t st)
+{
+    return p.group() > 1 ? launch_bwd_g<D, kBulk, true>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st)
+                         : launch_bwd_g<D, kBulk, false>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
 }
 
 }  // namespace
