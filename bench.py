@@ -279,6 +279,7 @@ def main():
     ap.add_argument("--path", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--materialize", type=int, default=0)
+    ap.add_argument("--layout", type=int, default=0, help="0: tensors [B,H,n,d] (every named config); 1: [B,n,H,d]")
     ap.add_argument("--hkv", type=int, default=0,
                     help="key/value heads (grouped-query attention); 0: one per query head, as in every named config")
     ap.add_argument("--sweep", action="store_true", help="config-5 strategy sweep (study table, not the contract line)")
@@ -324,9 +325,9 @@ def main():
 
     B, H, n, d = w.B, w.H, w.n, w.d
     desc = mb.make_desc(B, H, n, d, w.causal, w.scale, mb.MOA_BF16, args.dq_mode, args.materialize, args.path,
-                        H_kv=args.hkv)
-    shape = (B, H, n, d)
-    kv_shape = (B, args.hkv or H, n, d)       # K, V, dK, dV
+                        H_kv=args.hkv, layout=args.layout)
+    shape = (B, n, H, d) if args.layout else (B, H, n, d)
+    kv_shape = (B, n, args.hkv or H, d) if args.layout else (B, args.hkv or H, n, d)       # K, V, dK, dV
     shapes_in = (shape, kv_shape, kv_shape, shape)            # Q, K, V, dO
     shapes_out = (shape, shape, kv_shape, kv_shape)           # O, dQ, dK, dV
     base_mem = torch.cuda.memory_allocated()
@@ -498,7 +499,9 @@ def main():
     }
     if args.hkv:
         line["config"]["H_kv"] = args.hkv
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.hkv:
+    if args.layout:
+        line["config"]["layout"] = "[B,n,H,d]"
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.hkv and not args.layout:
         v, dt, cores, desc_s = time_oracle_sample(w, 20.0)
         line["cpu_baseline"] = {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
                                 "sample": desc_s, "seconds": dt}

@@ -79,6 +79,13 @@ typedef enum {
 
 typedef enum { MOA_OP_FWD = 0, MOA_OP_BWD = 1, MOA_OP_FUSED = 2 } moa_op;
 
+/* Memory layout of Q, K, V, dO, O, dQ, dK, dV (all eight; L is always [B,H,n]).
+ * BHND: [B,H,n,d] contiguous (the layout of every named configuration).
+ * BNHD: [B,n,H,d] contiguous (token-major, as projection GEMMs produce it); the tensor
+ * maps take the strides, the arithmetic and the results are the same.  Tensor-core bf16
+ * path only; other paths return MOA_ERR_UNSUPPORTED. */
+typedef enum { MOA_LAYOUT_BHND = 0, MOA_LAYOUT_BNHD = 1 } moa_layout;
+
 typedef struct {
     int32_t B, H, n, d;
     int32_t causal;      /* 0 or 1                                                            */
@@ -95,6 +102,7 @@ typedef struct {
                             paper's decode section treats.  K, V, dK, dV are then [B,H_kv,n,d];
                             dK, dV sum the contributions of the H / H_kv query heads of a group.
                             Tensor-core bf16 path only; other paths return MOA_ERR_UNSUPPORTED. */
+    int32_t layout;      /* moa_layout                                                         */
 } moa_attn_desc;
 
 /* Bytes of caller-provided workspace `op` (a moa_op) needs for `desc`.  Returns 0

@@ -13,6 +13,7 @@ struct Problem {
     int causal;
     float scale;
     int Hkv = 0;                                   // key/value heads; 0: same as H
+    int bnhd = 0;                                  // 1: the caller's tensors are [B,n,H,d] in memory (L stays [B,H,n])
     int BH() const { return B * H; }
     int kv_heads() const { return Hkv > 0 ? Hkv : H; }
     int group() const { return H / kv_heads(); }    // query heads per key/value head
@@ -111,5 +112,7 @@ cudaError_t simt_bwd_dq(const Problem &p, int dtype, const void *Q, const void *
                         const void *dO, const float *L, const float *Dv, void *dQ, cudaStream_t st);
 // dst[i] = (bf16)(mul * src[i])
 cudaError_t convert_f32_to_bf16(const float *src, void *dst, size_t count, float mul, cudaStream_t st);
+// the same into a [B,n,H,d] tensor from the [B*H, n, d] accumulator
+cudaError_t convert_f32_to_bf16_bnhd(const float *src, void *dst, int B, int H, int n, int d, float mul, cudaStream_t st);
 
 }  // namespace moa

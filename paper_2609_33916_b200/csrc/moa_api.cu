@@ -106,6 +106,11 @@ moa_status check_desc(const moa_attn_desc *d)
         !(d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->d == 128 && d->scale > 0.f))
         return MOA_ERR_UNSUPPORTED;
     if (d->path == MOA_PATH_TC && !(d->scale > 0.f)) return MOA_ERR_UNSUPPORTED;   // non-positive scale: SIMT path only
+    if (d->layout != MOA_LAYOUT_BHND && d->layout != MOA_LAYOUT_BNHD) return MOA_ERR_INVALID_ARG;
+    // token-major tensors: tensor-core kernels only
+    if (d->layout == MOA_LAYOUT_BNHD &&
+        !(d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->scale > 0.f && !d->materialize))
+        return MOA_ERR_UNSUPPORTED;
     if (d->H_kv < 0 || d->H_kv > d->H) return MOA_ERR_INVALID_ARG;
     if (d->H_kv > 0 && d->H % d->H_kv != 0) return MOA_ERR_INVALID_ARG;
     // shared K/V heads: tensor-core kernels only
@@ -178,7 +183,10 @@ MatWorkspace mat_workspace(const moa_attn_desc *d, int op)
     return w;
 }
 
-Problem to_problem(const moa_attn_desc *d) { return Problem{d->B, d->H, d->n, d->d, d->causal, d->scale, d->H_kv}; }
+Problem to_problem(const moa_attn_desc *d)
+{
+    return Problem{d->B, d->H, d->n, d->d, d->causal, d->scale, d->H_kv, d->layout == MOA_LAYOUT_BNHD ? 1 : 0};
+}
 
 // Materialising variant.  with_bwd = false: forward only (P^T is written and dropped).
 moa_status run_materialized(const moa_attn_desc *d, const void *Q, const void *K, const void *V, const void *dO,
@@ -237,7 +245,8 @@ moa_status run_bwd(const moa_attn_desc *d, const void *Q, const void *K, const v
         }
         MOA_TRY(cudaMemsetAsync(dQacc, 0, elems * sizeof(float), st));
         MOA_TRY(tc_bwd_kv(p, Q, K, V, dO, Lp, Dv, dK, dV, dQacc, mode == MOA_DQ_BULK_REDUCE, st));
-        MOA_TRY(convert_f32_to_bf16(dQacc, dQ, elems, p.scale, st));
+        if (p.bnhd) MOA_TRY(convert_f32_to_bf16_bnhd(dQacc, dQ, p.B, p.H, p.n, p.d, p.scale, st));
+        else MOA_TRY(convert_f32_to_bf16(dQacc, dQ, elems, p.scale, st));
         return MOA_OK;
     }
     MOA_TRY(row_dot(p, d->dtype, dO, O, Dv, st));

@@ -394,6 +394,30 @@ convert_kernel(const float *__restrict__ src, __nv_bfloat16 *__restrict__ dst, s
         for (size_t i = quads * 4; i < count; ++i) dst[i] = __float2bfloat16_rn(src[i] * mul);
 }
 
+// The same conversion into a [B,n,H,d] tensor: the accumulator is [B*H, n, d], so a row of d
+// elements moves as a unit; one thread converts four consecutive elements of a row.
+__global__ void __launch_bounds__(256)
+convert_bnhd_kernel(const float *__restrict__ src, __nv_bfloat16 *__restrict__ dst, size_t rows, int n, int H, int d,
+                    float mul)
+{
+    const int quads_per_row = d / 4;
+    const size_t total = rows * (size_t)quads_per_row;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t q = (size_t)blockIdx.x * blockDim.x + threadIdx.x; q < total; q += stride) {
+        const size_t row = q / quads_per_row;             // flat (b*H + h)*n + r
+        const int c4 = (int)(q - row * quads_per_row);
+        const size_t bh = row / (size_t)n;
+        const size_t r = row - bh * (size_t)n, bb = bh / (size_t)H, h = bh - bb * (size_t)H;
+        const size_t drow = (bb * (size_t)n + r) * (size_t)H + h;
+        const float4 v = __ldcs(reinterpret_cast<const float4 *>(src + row * d) + c4);
+        __nv_bfloat162 a = __floats2bfloat162_rn(v.x * mul, v.y * mul), b = __floats2bfloat162_rn(v.z * mul, v.w * mul);
+        uint2 u;
+        u.x = *reinterpret_cast<uint32_t *>(&a);
+        u.y = *reinterpret_cast<uint32_t *>(&b);
+        *reinterpret_cast<uint2 *>(dst + drow * d + 4 * c4) = u;
+    }
+}
+
 constexpr size_t fwd_smem(int D) { return (size_t)(3 * BM * (D + 1) + BM * SLD) * sizeof(float); }
 constexpr size_t bwd_smem(int D) { return (size_t)(4 * BM * (D + 1) + 2 * BM * SLD + 2 * BM) * sizeof(float); }
 
@@ -498,6 +522,17 @@ cudaError_t convert_f32_to_bf16(const float *src, void *dst, size_t count, float
     const unsigned grid = (unsigned)blocks;
     LaunchScope scope(MOA_KERNEL_CONVERT, st);
     convert_kernel<<<grid, 256, 0, st>>>(src, (__nv_bfloat16 *)dst, count, mul);
+    return cudaGetLastError();
+}
+
+cudaError_t convert_f32_to_bf16_bnhd(const float *src, void *dst, int B, int H, int n, int d, float mul, cudaStream_t st)
+{
+    const size_t rows = (size_t)B * H * n, quads = rows * (size_t)(d / 4);
+    size_t blocks = (quads + 255) / 256;
+    if (blocks < 1) blocks = 1;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    LaunchScope scope(MOA_KERNEL_CONVERT, st);
+    convert_bnhd_kernel<<<(unsigned)blocks, 256, 0, st>>>(src, (__nv_bfloat16 *)dst, rows, n, H, d, mul);
     return cudaGetLastError();
 }
 

@@ -74,7 +74,7 @@ template <int D>
 __global__ void __launch_bounds__(256)
 bwd_preprocess_kernel(const __nv_bfloat16 *__restrict__ dO, const __nv_bfloat16 *__restrict__ O,
                       const float *__restrict__ L, float *__restrict__ Lp, float *__restrict__ Dp,
-                      int n, int n_pad, size_t padded_rows)
+                      int n, int n_pad, size_t padded_rows, int H, int bnhd)
 {
     constexpr int kLanesPerRow = D / 8;
     constexpr int kRowsPerPass = 32 / kLanesPerRow;
@@ -95,9 +95,14 @@ bwd_preprocess_kernel(const __nv_bfloat16 *__restrict__ dO, const __nv_bfloat16 
         a[p] = b[p] = make_uint4(0u, 0u, 0u, 0u);
         lv[p] = 0.f;
         if (real[p]) {
-            const size_t row = bh * (size_t)n + r;
-            a[p] = __ldcs(reinterpret_cast<const uint4 *>(dO + row * D) + l);
-            b[p] = __ldcs(reinterpret_cast<const uint4 *>(O + row * D) + l);
+            const size_t row = bh * (size_t)n + r;                      // row of L: always [B,H,n]
+            size_t trow = row;                                          // row of dO, O in the caller's layout
+            if (bnhd) {
+                const size_t bb = bh / (size_t)H;
+                trow = (bb * (size_t)n + r) * (size_t)H + (bh - bb * (size_t)H);
+            }
+            a[p] = __ldcs(reinterpret_cast<const uint4 *>(dO + trow * D) + l);
+            b[p] = __ldcs(reinterpret_cast<const uint4 *>(O + trow * D) + l);
             if (l == 0) lv[p] = L[row];
         }
     }
@@ -158,7 +163,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
               const __grid_constant__ CUtensorMap mapdV, const float *__restrict__ Lp, const float *__restrict__ Dp,
               float *__restrict__ dQacc,
               int n, int n_pad, int causal, float scale, float scale_log2, int nkt, int hpg, int group,
-              int skip_dq, unsigned int *status)
+              int Hkv, int skip_dq, unsigned int *status)
 {
     using SM = BwdSmem<D, kBulk>;
     constexpr int kDoSlots = SM::kDoSlots;
@@ -188,6 +193,11 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     // With shared K/V heads (group > 1) `bh` counts K/V heads and the CTA walks the query tiles of
     // all `group` query heads that read this K/V tile: dK and dV accumulate over the whole group in
     // TMEM, still written once by one CTA, with no atomics.
+    // coordinates of the 4-D tensor maps of the caller's tensors: batch, K/V head, and the first
+    // query head of the group; the flat query-head index (walkers below) addresses the internal
+    // [B*H, ...] arrays (L', D, the dQ accumulator)
+    const int bb = bh / Hkv, hk = bh - bb * Hkv;
+    const int hq0 = hk * (kGrouped ? group : 1) - bh * (kGrouped ? group : 1);   // query head in batch = flat index + hq0
     const int niter_all = (kGrouped ? group : 1) * (nqt - i_begin);
     // (query head, query tile) of consecutive iterations, advanced without a division: each role
     // keeps a walker of its own, in step with the iterations it handles.  kGrouped = false (one K/V
@@ -234,8 +244,8 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         if (lane == 0 && niter > 0) {
             mbar_arrive_expect_tx(bars + B_KV, 2 * SM::kTile);
             for (int b = 0; b < kBoxes; ++b) {
-                tma_load_3d(sK + b * kBoxBytes, &mapK, bars + B_KV, 64 * b, k0, bh);
-                tma_load_3d(sV + b * kBoxBytes, &mapV, bars + B_KV, 64 * b, k0, bh);
+                tma_load_4d(sK + b * kBoxBytes, &mapK, bars + B_KV, 64 * b, k0, hk, bb);
+                tma_load_4d(sV + b * kBoxBytes, &mapV, bars + B_KV, 64 * b, k0, hk, bb);
             }
         }
         // Q tiles (with L, D) go through a two-slot ring and are fetched two tiles ahead: S(i+1) is
@@ -247,7 +257,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             wq.next();
             uint8_t *sQ = sm + SM::offQ + s * SM::kTile;
             mbar_arrive_expect_tx(bars + B_QFULL + s, SM::kTile + 1024);
-            for (int b = 0; b < kBoxes; ++b) tma_load_3d(sQ + b * kBoxBytes, &mapQ, bars + B_QFULL + s, 64 * b, q0, qh);
+            for (int b = 0; b < kBoxes; ++b) tma_load_4d(sQ + b * kBoxBytes, &mapQ, bars + B_QFULL + s, 64 * b, q0, qh + hq0, bb);
             bulk_load_1d(sL + s * 128, Lp + (size_t)qh * n_pad + q0, 512, bars + B_QFULL + s);
             bulk_load_1d(sD + s * 128, Dp + (size_t)qh * n_pad + q0, 512, bars + B_QFULL + s);
         };
@@ -256,7 +266,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             wdo.next();
             uint8_t *sdO = sm + SM::offdO + s * SM::kTile;
             mbar_arrive_expect_tx(bars + B_DOFULL + s, SM::kTile);
-            for (int b = 0; b < kBoxes; ++b) tma_load_3d(sdO + b * kBoxBytes, &mapdO, bars + B_DOFULL + s, 64 * b, q0, qh);
+            for (int b = 0; b < kBoxes; ++b) tma_load_4d(sdO + b * kBoxBytes, &mapdO, bars + B_DOFULL + s, 64 * b, q0, qh + hq0, bb);
         };
         if (lane == 0 && niter > 0) {
             load_q(0);
@@ -585,8 +595,8 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             mbar_arrive(bars + B_EPI);
             if (tid == 0 && mbar_wait(bars + B_EPI, 0, abortp, status, ERR_DQ)) {
                 for (int b = 0; b < kBoxes; ++b) {
-                    tma_store_3d(&mapdV, sV + b * kBoxBytes, 64 * b, k0, bh);
-                    tma_store_3d(&mapdK, sK + b * kBoxBytes, 64 * b, k0, bh);
+                    tma_store_4d(&mapdV, sV + b * kBoxBytes, 64 * b, k0, hk, bb);
+                    tma_store_4d(&mapdK, sK + b * kBoxBytes, 64 * b, k0, hk, bb);
                 }
                 bulk_commit();
                 bulk_wait_read<0>();      // shared memory is read before the CTA may exit
@@ -603,13 +613,15 @@ cudaError_t launch_bwd_g(const Problem &p, const void *Q, const void *K, const v
                        const float *Lp, const float *Dp, void *dK, void *dV, float *dQacc, cudaStream_t st)
 {
     CUtensorMap mq, mk, mv, mdo, mdq, mdk, mdv;
-    const uint64_t heads = (uint64_t)p.BH(), kv_heads = (uint64_t)p.BHkv();
-    if (!make_tensor_map_3d(&mq, Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mk, K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, kv_heads, p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mv, V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, kv_heads, p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mdo, dO, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mdk, dK, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, kv_heads, p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mdv, dV, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, kv_heads, p.n, D, 128, 64))
+    const uint64_t heads = (uint64_t)p.BH();
+    const bool bnhd = p.bnhd != 0;
+    const auto bf = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    if (!make_tensor_map_4d(&mq, Q, bf, 2, p.B, p.H, p.n, D, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mk, K, bf, 2, p.B, p.kv_heads(), p.n, D, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mv, V, bf, 2, p.B, p.kv_heads(), p.n, D, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mdo, dO, bf, 2, p.B, p.H, p.n, D, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mdk, dK, bf, 2, p.B, p.kv_heads(), p.n, D, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mdv, dV, bf, 2, p.B, p.kv_heads(), p.n, D, bnhd, 128, 64))
         return cudaErrorInvalidValue;
     // fp32 accumulator as [heads, n, D] with boxes of 32 rows x D floats (no swizzle); also encoded when unused
     if (!make_tensor_map_3d(&mdq, dQacc ? (const void *)dQacc : Q, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, heads, p.n, D, 32, D))
@@ -625,7 +637,7 @@ cudaError_t launch_bwd_g(const Problem &p, const void *Q, const void *K, const v
     pkv.Hkv = 0;
     tc_bwd_kernel<D, kBulk, kGrouped><<<(unsigned)(nkt * p.BHkv()), kThreads, kSmem, st>>>(
         mq, mk, mv, mdo, mdq, mdk, mdv, Lp, Dp, dQacc, p.n, nkt * 128, p.causal,
-        p.scale, p.scale * kLog2e, nkt, heads_per_group(pkv, nkt), p.group(), dQacc == nullptr ? 1 : 0, device_status_ptr());
+        p.scale, p.scale * kLog2e, nkt, heads_per_group(pkv, nkt), p.group(), p.kv_heads(), dQacc == nullptr ? 1 : 0, device_status_ptr());
     return cudaGetLastError();
 }
 
@@ -650,10 +662,10 @@ cudaError_t tc_bwd_preprocess(const Problem &p, const void *dO, const void *O, c
     LaunchScope scope(MOA_KERNEL_PREPROCESS, st);
     if (p.d == 64)
         bwd_preprocess_kernel<64><<<grid, wpb * 32, 0, st>>>((const __nv_bfloat16 *)dO, (const __nv_bfloat16 *)O, L,
-                                                             Lp, Dp, p.n, n_pad, rows);
+                                                             Lp, Dp, p.n, n_pad, rows, p.H, p.bnhd);
     else
         bwd_preprocess_kernel<128><<<grid, wpb * 32, 0, st>>>((const __nv_bfloat16 *)dO, (const __nv_bfloat16 *)O, L,
-                                                              Lp, Dp, p.n, n_pad, rows);
+                                                              Lp, Dp, p.n, n_pad, rows, p.H, p.bnhd);
     return cudaGetLastError();
 }
 

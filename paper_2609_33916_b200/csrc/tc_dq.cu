@@ -44,7 +44,7 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
              const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapdO,
              const float *__restrict__ Lp, const float *__restrict__ Dp, __nv_bfloat16 *__restrict__ dQ,
              int n, int n_pad, int causal, float scale, float scale_log2, int nqt, int hpg,
-             int group, unsigned int *status)
+             int group, int H, int bnhd, unsigned int *status)
 {
     using SM = DqSmem<D>;
     constexpr int kBoxes = D / 64;
@@ -58,7 +58,8 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
     int bh, t;
     job_from_block((int)blockIdx.x, nqt, (int)gridDim.x / nqt, hpg, bh, t);
-    const int kvh = bh / group;                 // the K/V head this query head reads
+    const int bb = bh / H, hq = bh - bb * H;    // batch and query head: coordinates of the 4-D tensor maps
+    const int hk = hq / group;                  // the K/V head this query head reads
     const int qt = causal ? nqt - 1 - t : t;   // causal: longest rows first
     const int q0 = qt * 128;
     const int nkt_all = n_pad / 128;
@@ -83,8 +84,8 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
         if (lane == 0 && nkt > 0) {
             mbar_arrive_expect_tx(bars + B_Q, 2 * SM::kTile);
             for (int b = 0; b < kBoxes; ++b) {
-                tma_load_3d(sm + SM::offQ + b * kBoxBytes, &mapQ, bars + B_Q, 64 * b, q0, bh);
-                tma_load_3d(sm + SM::offdO + b * kBoxBytes, &mapdO, bars + B_Q, 64 * b, q0, bh);
+                tma_load_4d(sm + SM::offQ + b * kBoxBytes, &mapQ, bars + B_Q, 64 * b, q0, hq, bb);
+                tma_load_4d(sm + SM::offdO + b * kBoxBytes, &mapdO, bars + B_Q, 64 * b, q0, hq, bb);
             }
         }
         for (int j = 0; j < nkt; ++j) {
@@ -93,8 +94,8 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
             if (lane == 0) {
                 mbar_arrive_expect_tx(bars + B_KVFULL + s, 2 * SM::kTile);
                 for (int b = 0; b < kBoxes; ++b) {
-                    tma_load_3d(sm + SM::offK + s * SM::kTile + b * kBoxBytes, &mapK, bars + B_KVFULL + s, 64 * b, j * 128, kvh);
-                    tma_load_3d(sm + SM::offV + s * SM::kTile + b * kBoxBytes, &mapV, bars + B_KVFULL + s, 64 * b, j * 128, kvh);
+                    tma_load_4d(sm + SM::offK + s * SM::kTile + b * kBoxBytes, &mapK, bars + B_KVFULL + s, 64 * b, j * 128, hk, bb);
+                    tma_load_4d(sm + SM::offV + s * SM::kTile + b * kBoxBytes, &mapV, bars + B_KVFULL + s, 64 * b, j * 128, hk, bb);
                 }
             }
             __syncwarp();
@@ -178,7 +179,8 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
         if (ok && mbar_wait(bars + B_DONE, 0, abortp, status, ERR_DONE)) {
             tc_fence_after();
             const int qrow = q0 + lane_row;
-            __nv_bfloat16 *outp = dQ + ((size_t)bh * n + qrow) * D + (D / 2) * wg;
+            const size_t qrow_index = bnhd ? ((size_t)bb * n + qrow) * H + hq : (size_t)bh * n + qrow;   // row of dQ in the caller's layout
+            __nv_bfloat16 *outp = dQ + qrow_index * D + (D / 2) * wg;
 #pragma unroll
             for (int c = 0; c < D / 2; c += 32) {
                 uint32_t r[32];
@@ -208,11 +210,12 @@ cudaError_t launch_dq(const Problem &p, const void *Q, const void *K, const void
                       const float *Lp, const float *Dp, void *dQ, cudaStream_t st)
 {
     CUtensorMap mq, mk, mv, mdo;
-    const uint64_t heads = (uint64_t)p.BH();
-    if (!make_tensor_map_3d(&mq, Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mk, K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)p.BHkv(), p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mv, V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)p.BHkv(), p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mdo, dO, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64))
+    const bool bnhd = p.bnhd != 0;
+    const auto bf = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    if (!make_tensor_map_4d(&mq, Q, bf, 2, p.B, p.H, p.n, D, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mk, K, bf, 2, p.B, p.kv_heads(), p.n, D, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mv, V, bf, 2, p.B, p.kv_heads(), p.n, D, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mdo, dO, bf, 2, p.B, p.H, p.n, D, bnhd, 128, 64))
         return cudaErrorInvalidValue;
     constexpr int kSmem = DqSmem<D>::kTotal;
     cudaError_t e = cudaFuncSetAttribute(tc_dq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
@@ -221,7 +224,7 @@ cudaError_t launch_dq(const Problem &p, const void *Q, const void *K, const void
     LaunchScope scope(MOA_KERNEL_BWD_DQ, st);
     tc_dq_kernel<D><<<(unsigned)(nqt * p.BH()), kThreads, kSmem, st>>>(
         mq, mk, mv, mdo, Lp, Dp, (__nv_bfloat16 *)dQ, p.n, nqt * 128, p.causal, p.scale, p.scale * kLog2e, nqt,
-        heads_per_group(p, nqt), p.group(), device_status_ptr());
+        heads_per_group(p, nqt), p.group(), p.H, p.bnhd, device_status_ptr());
     return cudaGetLastError();
 }
 

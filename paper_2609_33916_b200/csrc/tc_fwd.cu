@@ -56,7 +56,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
               const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapO,
               float *__restrict__ L,
-              int n, int causal, float scale_log2, int nqt, int hpg, int group, unsigned int *status)
+              int n, int causal, float scale_log2, int nqt, int hpg, int group, int H, unsigned int *status)
 {
     constexpr int kTileBytes = 128 * D * 2;
     constexpr int kBoxes = D / 64;         // 64-column (128-byte) swizzled boxes per tile
@@ -70,7 +70,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
     int bh, t;
     job_from_block((int)blockIdx.x, nqt, (int)gridDim.x / nqt, hpg, bh, t);
-    const int kvh = bh / group;                 // the K/V head this query head reads (group > 1: shared heads)
+    const int bb = bh / H, hq = bh - bb * H;    // batch and query head: coordinates of the 4-D tensor maps
+    const int hk = hq / group;                  // the K/V head this query head reads (group > 1: shared heads)
     const int qt = causal ? nqt - 1 - t : t;   // causal: longest rows first
     const int q0 = qt * BM;
     const int nkt_all = (n + BN - 1) / BN;
@@ -94,7 +95,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0 && nkt > 0) {
             mbar_arrive_expect_tx(bars + F_Q, kTileBytes);
-            for (int b = 0; b < kBoxes; ++b) tma_load_3d(sQ + b * kBoxBytes, &mapQ, bars + F_Q, 64 * b, q0, bh);
+            for (int b = 0; b < kBoxes; ++b) tma_load_4d(sQ + b * kBoxBytes, &mapQ, bars + F_Q, 64 * b, q0, hq, bb);
         }
         for (int j = 0; j < nkt; ++j) {
             const int s = j & 1;
@@ -102,13 +103,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             if (lane == 0) {
                 mbar_arrive_expect_tx(bars + F_KFULL + s, kTileBytes);
                 for (int b = 0; b < kBoxes; ++b)
-                    tma_load_3d(sK + s * kTileBytes + b * kBoxBytes, &mapK, bars + F_KFULL + s, 64 * b, j * BN, kvh);
+                    tma_load_4d(sK + s * kTileBytes + b * kBoxBytes, &mapK, bars + F_KFULL + s, 64 * b, j * BN, hk, bb);
             }
             if (j >= 2 && !mbar_wait(bars + F_VEMPTY + s, ((j >> 1) - 1) & 1, abortp, status, ERR_V)) break;
             if (lane == 0) {
                 mbar_arrive_expect_tx(bars + F_VFULL + s, kTileBytes);
                 for (int b = 0; b < kBoxes; ++b)
-                    tma_load_3d(sV + s * kTileBytes + b * kBoxBytes, &mapV, bars + F_VFULL + s, 64 * b, j * BN, kvh);
+                    tma_load_4d(sV + s * kTileBytes + b * kBoxBytes, &mapV, bars + F_VFULL + s, 64 * b, j * BN, hk, bb);
             }
             __syncwarp();
         }
@@ -311,7 +312,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             fence_proxy_async_smem();
             mbar_arrive(bars + F_E);
             if (tid == 0 && mbar_wait(bars + F_E, 0, abortp, status, ERR_O)) {
-                for (int b = 0; b < kBoxes; ++b) tma_store_3d(&mapO, sQ + b * kBoxBytes, 64 * b, q0, bh);
+                for (int b = 0; b < kBoxes; ++b) tma_store_4d(&mapO, sQ + b * kBoxBytes, 64 * b, q0, hq, bb);
                 bulk_commit();
                 bulk_wait_read<0>();      // shared memory is read before the CTA may exit
             }
@@ -329,18 +330,19 @@ cudaError_t launch_fwd(const Problem &p, const void *Q, const void *K, const voi
 {
     constexpr int kSmem = 5 * 128 * D * 2 + 8 * (F_COUNT + 2) + 2 * 128 * 8;
     CUtensorMap mq, mk, mv, mo;
-    const uint64_t heads = (uint64_t)p.BH();
-    if (!make_tensor_map_3d(&mq, Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mk, K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)p.BHkv(), p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mv, V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)p.BHkv(), p.n, D, 128, 64) ||
-        !make_tensor_map_3d(&mo, O, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.n, D, 128, 64))
+    const bool bnhd = p.bnhd != 0;
+    const auto bf = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    if (!make_tensor_map_4d(&mq, Q, bf, 2, p.B, p.H, p.n, D, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mk, K, bf, 2, p.B, p.kv_heads(), p.n, D, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mv, V, bf, 2, p.B, p.kv_heads(), p.n, D, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mo, O, bf, 2, p.B, p.H, p.n, D, bnhd, 128, 64))
         return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
     const int nqt = (p.n + BM - 1) / BM;
     LaunchScope scope(MOA_KERNEL_FWD, st);
     tc_fwd_kernel<D><<<(unsigned)(nqt * p.BH()), kThreads, kSmem, st>>>(
-        mq, mk, mv, mo, L, p.n, p.causal, p.scale * kLog2e, nqt, heads_per_group(p, nqt), p.group(), device_status_ptr());
+        mq, mk, mv, mo, L, p.n, p.causal, p.scale * kLog2e, nqt, heads_per_group(p, nqt), p.group(), p.H, device_status_ptr());
     return cudaGetLastError();
 }
 

@@ -13,4 +13,12 @@ namespace moa {
 bool make_tensor_map_3d(CUtensorMap *map, const void *base, CUtensorMapDataType dt, int elem_bytes,
                         uint64_t heads, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_cols);
 
+// Tiled map over one of the caller's [B, heads, rows, cols] tensors in either memory layout
+// (bnhd = false: [B,H,n,d] contiguous; true: [B,n,H,d] contiguous), as a 4-D tensor
+// (cols, rows, heads, B) with boxes of [1, 1, box_rows, box_cols]; 128-byte swizzle when
+// box_cols * elem_bytes == 128.  Rows past `rows` read as zero and are clipped on store.
+bool make_tensor_map_4d(CUtensorMap *map, const void *base, CUtensorMapDataType dt, int elem_bytes,
+                        uint64_t batch, uint64_t heads, uint64_t rows, uint64_t cols, bool bnhd,
+                        uint32_t box_rows, uint32_t box_cols);
+
 }  // namespace moa

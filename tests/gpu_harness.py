@@ -25,17 +25,22 @@ def to_host_f64(t: torch.Tensor) -> np.ndarray:
 
 def run_library(inp: dict, dtype: str, causal: bool, scale: float, *, op: str = "fused",
                 dq_mode: int = mb.MOA_DQ_AUTO, path: int = mb.MOA_PATH_AUTO, materialize: int = 0,
-                poison: bool = True) -> dict:
-    """op: 'fused' (one call) or 'split' (moa_attn_fwd then moa_attn_bwd) or 'fwd'."""
+                poison: bool = True, layout: int = 0) -> dict:
+    """op: 'fused' (one call) or 'split' (moa_attn_fwd then moa_attn_bwd) or 'fwd'.
+    layout = 1: the library sees every tensor as [B,n,H,d] in memory (inputs are permuted on the way
+    in, results permuted back), so the returned arrays are [B,H,n,d] either way."""
     B, H, n, d = inp["Q"].shape
     Hkv = inp["K"].shape[1]          # fewer K/V heads than query heads: grouped-query attention
     Q, K, V, dO = (to_device(inp[k], dtype) for k in ("Q", "K", "V", "dO"))
+    if layout:
+        Q, K, V, dO = (t.permute(0, 2, 1, 3).contiguous() for t in (Q, K, V, dO))
     desc = mb.make_desc(B, H, n, d, causal, scale, mb.MOA_BF16 if dtype == "bf16" else mb.MOA_F32,
-                        dq_mode, materialize, path, H_kv=0 if Hkv == H else Hkv)
+                        dq_mode, materialize, path, H_kv=0 if Hkv == H else Hkv, layout=layout)
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
     fill = float("nan") if poison else 0.0   # unwritten elements must show up
-    O, dQ = (torch.full((B, H, n, d), fill, dtype=tdt, device="cuda") for _ in range(2))
-    dK, dV = (torch.full((B, Hkv, n, d), fill, dtype=tdt, device="cuda") for _ in range(2))
+    q_shape, kv_shape = ((B, n, H, d), (B, n, Hkv, d)) if layout else ((B, H, n, d), (B, Hkv, n, d))
+    O, dQ = (torch.full(q_shape, fill, dtype=tdt, device="cuda") for _ in range(2))
+    dK, dV = (torch.full(kv_shape, fill, dtype=tdt, device="cuda") for _ in range(2))
     L = torch.full((B, H, n), fill, dtype=torch.float32, device="cuda")
     ws_bytes = mb.moa_attn_workspace_bytes(desc, mb.MOA_OP_FUSED if op != "fwd" else mb.MOA_OP_FWD)
     if materialize and op == "split":
@@ -52,6 +57,8 @@ def run_library(inp: dict, dtype: str, causal: bool, scale: float, *, op: str = 
         raise ValueError(op)
     st = mb.moa_last_device_status()
     assert st == mb.MOA_OK, mb.status_string(st)
+    if layout:
+        O, dQ, dK, dV = (t.permute(0, 2, 1, 3) for t in (O, dQ, dK, dV))
     out = dict(O=to_host_f64(O), L=to_host_f64(L))
     if op != "fwd":
         out.update(dQ=to_host_f64(dQ), dK=to_host_f64(dK), dV=to_host_f64(dV))

@@ -35,7 +35,7 @@ def test_version_and_strings(lib):
 
 
 def test_desc_struct_layout_matches_header():
-    assert ctypes.sizeof(mb.moa_attn_desc) == 44
+    assert ctypes.sizeof(mb.moa_attn_desc) == 48
     assert mb.moa_attn_desc.scale.offset == 20
 
 
@@ -98,6 +98,10 @@ def test_shared_kv_heads_argument_checks(lib):
     assert fwd(H_kv=2, dtype=mb.MOA_F32) == mb.MOA_ERR_UNSUPPORTED      # tensor-core bf16 path only
     assert fwd(H_kv=2, path=mb.MOA_PATH_SIMT) == mb.MOA_ERR_UNSUPPORTED
     assert fwd(H_kv=2, materialize=1) == mb.MOA_ERR_UNSUPPORTED
+    assert fwd(layout=2) == mb.MOA_ERR_INVALID_ARG
+    assert fwd(layout=1, dtype=mb.MOA_F32) == mb.MOA_ERR_UNSUPPORTED    # token-major: tensor-core bf16 path only
+    assert fwd(layout=1, path=mb.MOA_PATH_SIMT) == mb.MOA_ERR_UNSUPPORTED
+    assert fwd(layout=1, materialize=1) == mb.MOA_ERR_UNSUPPORTED
     # the workspace does not depend on the number of K/V heads: D, L' and the dQ accumulator are per query head
     w = lambda hkv: mb.moa_attn_workspace_bytes(mb.make_desc(1, 8, 256, 128, True, 0.1, H_kv=hkv), mb.MOA_OP_FUSED)
     assert w(0) == w(8) == w(2) == w(1) > 0

@@ -270,6 +270,34 @@ def test_gqa_equals_replicated_kv_heads(H):
         assert mi.rel_err(a[k], summed) <= 8e-3, k     # the copies were rounded to bf16 one by one
 
 
+# ------------------------------------------------------- token-major tensors [B,n,H,d]
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("B,Hq,Hkv,n,d", [(2, 3, 3, 300, 128), (3, 4, 2, 257, 64), (1, 6, 1, 128, 128)])
+@pytest.mark.parametrize("dq_mode", [0, 1, 3])
+def test_bnhd_layout_matches_oracle(H, causal, B, Hq, Hkv, n, d, dq_mode):
+    """Every tensor handed over as [B,n,H,d] (strided tensor maps, a strided preprocess and a
+    strided dQ conversion): same results as the oracle, element by element, ragged n included,
+    with and without shared K/V heads."""
+    inp = _gqa_inputs(B, Hq, Hkv, n, d, seed=300 + n + Hq)
+    got = H.run_library(inp, "bf16", causal, 1.0 / math.sqrt(d), dq_mode=dq_mode, layout=1)
+    f = H.f64_inputs(inp, "bf16")
+    ref = oracle.attn_fwd_bwd_gqa(f["Q"], f["K"], f["V"], f["dO"], causal, 1.0 / math.sqrt(d))
+    H.assert_close(got, ref, H.TOL_BF16, tag=f"bnhd B{B} H{Hq}/{Hkv} n{n} d{d} causal{causal} dq{dq_mode}")
+    assert mi.rel_err(got["L"], ref["L"]) <= 1e-3
+
+
+def test_bnhd_layout_is_bitwise_the_bhnd_result(H):
+    """The layout changes addresses only: in the deterministic mode both layouts give identical bits."""
+    inp = _gqa_inputs(2, 4, 2, 384, 128, seed=123)
+    a = H.run_library(inp, "bf16", True, 0.09, dq_mode=3, layout=0)
+    b = H.run_library(inp, "bf16", True, 0.09, dq_mode=3, layout=1)
+    for k in ("O", "L", "dQ", "dK", "dV"):
+        np.testing.assert_array_equal(a[k], b[k], err_msg=k)
+    c = H.run_library(inp, "bf16", True, 0.09, op="split", dq_mode=3, layout=1)
+    for k in ("O", "L", "dQ", "dK", "dV"):
+        np.testing.assert_array_equal(b[k], c[k], err_msg=k)
+
+
 def test_causal_block_order_with_a_partial_head_group(H):
     """Causal launches take the heads in groups (tile-major inside a group, so that the longest
     jobs start first).  19 heads at n = 4096, d = 128 make groups of 16 with a last group of 3:
