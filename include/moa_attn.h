@@ -77,7 +77,7 @@ typedef enum {
     MOA_PATH_TC = 2     /* tcgen05/TMEM/TMA kernels (bf16 only)                                */
 } moa_path;
 
-typedef enum { MOA_OP_FWD = 0, MOA_OP_BWD = 1, MOA_OP_FUSED = 2 } moa_op;
+typedef enum { MOA_OP_FWD = 0, MOA_OP_BWD = 1, MOA_OP_FUSED = 2, MOA_OP_ROWPARALLEL = 3 } moa_op;
 
 /* Memory layout of Q, K, V, dO, O, dQ, dK, dV (all eight; L is always [B,H,n]).
  * BHND: [B,H,n,d] contiguous (the layout of every named configuration).
@@ -163,6 +163,21 @@ moa_status moa_attn_fused_fwd_bwd(const moa_attn_desc *desc,
                                   const void *Q, const void *K, const void *V, const void *dO,
                                   void *O, float *L, void *dQ, void *dK, void *dV,
                                   void *ws, size_t ws_bytes, void *stream);
+
+/* The paper's own fused design, kept as a comparison variant (Sec. 4, "fused v1" and "v3"):
+ * ONE kernel, parallel over query rows, does the forward of its rows and then their backward;
+ * dQ stays local and the dK (atomic_sites = 1) or dK and dV (atomic_sites = 2) contributions of
+ * every (query tile, key tile) pair are added into fp32 accumulators with atomics -- the paper's
+ * GK and GV atomic sites, whose count it found to set the device time (2 sites = 2.0000x the
+ * atomic instructions = 1.97x the time).  With atomic_sites = 1, dV comes from an atomic-free
+ * key-parallel kernel of its own, as in the paper's v3.  fp32 CUDA-core arithmetic (bf16 or fp32
+ * tensors, [B,H,n,d], one K/V head per query head); same results as moa_attn_fused_fwd_bwd up
+ * to rounding.  Workspace: moa_attn_workspace_bytes(desc, MOA_OP_ROWPARALLEL) (D plus, for bf16,
+ * two fp32 [B,H,n,d] accumulators).  desc->dq_mode, path and materialize are ignored. */
+moa_status moa_attn_fused_rowparallel(const moa_attn_desc *desc,
+                                      const void *Q, const void *K, const void *V, const void *dO,
+                                      void *O, float *L, void *dQ, void *dK, void *dV,
+                                      int atomic_sites, void *ws, size_t ws_bytes, void *stream);
 
 /* Synchronises `stream` and returns MOA_ERR_TIMEOUT if any kernel launched by this
  * library on the current device gave up a bounded wait since the last call of this

@@ -20,13 +20,13 @@ MOA_BF16, MOA_F32 = 0, 1
 MOA_DQ_AUTO, MOA_DQ_RED, MOA_DQ_BULK_REDUCE, MOA_DQ_SEPARATE_PASS = 0, 1, 2, 3
 MOA_PATH_AUTO, MOA_PATH_SIMT, MOA_PATH_TC = 0, 1, 2
 MOA_LAYOUT_BHND, MOA_LAYOUT_BNHD = 0, 1
-MOA_OP_FWD, MOA_OP_BWD, MOA_OP_FUSED = 0, 1, 2
+MOA_OP_FWD, MOA_OP_BWD, MOA_OP_FUSED, MOA_OP_ROWPARALLEL = 0, 1, 2, 3
 
 #: every symbol include/moa_attn.h declares
 EXPORTS = (
     "moa_attn_workspace_bytes", "moa_attn_fwd", "moa_attn_bwd", "moa_attn_fused_fwd_bwd",
     "moa_last_device_status", "moa_launch_count", "moa_status_string", "moa_version",
-    "moa_profile_enable", "moa_profile_read", "moa_attn_bwd_static_scratch",
+    "moa_profile_enable", "moa_profile_read", "moa_attn_bwd_static_scratch", "moa_attn_fused_rowparallel",
 )
 
 
@@ -73,6 +73,8 @@ def lib() -> ctypes.CDLL:
         L.moa_attn_bwd_static_scratch.argtypes = [dp] + [vp] * 9 + [vp]
         L.moa_attn_fused_fwd_bwd.restype = ctypes.c_int
         L.moa_attn_fused_fwd_bwd.argtypes = [dp] + [vp] * 9 + [vp, sz, vp]
+        L.moa_attn_fused_rowparallel.restype = ctypes.c_int
+        L.moa_attn_fused_rowparallel.argtypes = [dp] + [vp] * 9 + [ctypes.c_int, vp, sz, vp]
         L.moa_last_device_status.restype = ctypes.c_int
         L.moa_last_device_status.argtypes = [vp]
         L.moa_launch_count.restype = ctypes.c_uint64
@@ -171,6 +173,16 @@ def moa_attn_fused_fwd_bwd(desc, Q, K, V, dO, O, L, dQ, dK, dV, ws=None, stream=
                                      _nbytes(ws) if ws_bytes is None else ws_bytes, _stream(stream))
     if check and s != MOA_OK:
         raise MoaError(s, "moa_attn_fused_fwd_bwd")
+    return s
+
+
+def moa_attn_fused_rowparallel(desc, Q, K, V, dO, O, L, dQ, dK, dV, atomic_sites, ws=None, stream=None,
+                               ws_bytes=None, check=True) -> int:
+    s = lib().moa_attn_fused_rowparallel(ctypes.byref(desc), _ptr(Q), _ptr(K), _ptr(V), _ptr(dO), _ptr(O),
+                                         _ptr(L), _ptr(dQ), _ptr(dK), _ptr(dV), int(atomic_sites), _ptr(ws),
+                                         _nbytes(ws) if ws_bytes is None else ws_bytes, _stream(stream))
+    if check and s != MOA_OK:
+        raise MoaError(s, "moa_attn_fused_rowparallel")
     return s
 
 

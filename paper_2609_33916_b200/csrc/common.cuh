@@ -108,6 +108,10 @@ cudaError_t simt_bwd_kv(const Problem &p, int dtype, const void *Q, const void *
                         const void *dO, const float *L, const float *Dv,
                         void *dK, void *dV, float *dQacc, cudaStream_t st);
 // atomic-free query-parallel dQ pass
+// Row-parallel fused forward+backward in one kernel with dK (sites = 1) or dK and dV (sites = 2)
+// accumulated by fp32 atomics into dKacc / dVacc [B*H, n, d]; writes O, L, D, dQ.
+cudaError_t simt_rowpar(const Problem &p, int dtype, const void *Q, const void *K, const void *V, const void *dO,
+                        void *O, float *L, float *Dv, void *dQ, float *dKacc, float *dVacc, int sites, cudaStream_t st);
 cudaError_t simt_bwd_dq(const Problem &p, int dtype, const void *Q, const void *K, const void *V,
                         const void *dO, const float *L, const float *Dv, void *dQ, cudaStream_t st);
 // dst[i] = (bf16)(mul * src[i])

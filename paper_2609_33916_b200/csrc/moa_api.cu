@@ -290,6 +290,15 @@ void *static_scratch_ptr()
 
 using namespace moa;
 
+// Workspace of the row-parallel comparison variant: [ D | dKacc | dVacc ] (accumulators for bf16 only;
+// fp32 tensors accumulate in place)
+static size_t rowpar_workspace(const moa_attn_desc *d)
+{
+    const size_t rows = (size_t)d->B * d->H * d->n;
+    const size_t acc = d->dtype == MOA_BF16 ? align_up(rows * d->d * sizeof(float)) : 0;
+    return align_up(rows * sizeof(float)) + 2 * acc;
+}
+
 extern "C" {
 
 size_t moa_attn_workspace_bytes(const moa_attn_desc *desc, int op)
@@ -298,6 +307,7 @@ size_t moa_attn_workspace_bytes(const moa_attn_desc *desc, int op)
     if (desc->materialize) return (op == MOA_OP_FWD || op == MOA_OP_FUSED) ? mat_workspace(desc, op).total : 0;
     if (op == MOA_OP_FWD) return 0;
     if (op == MOA_OP_BWD || op == MOA_OP_FUSED) return bwd_workspace(desc).total;
+    if (op == MOA_OP_ROWPARALLEL) return rowpar_workspace(desc);
     return 0;
 }
 
@@ -373,6 +383,43 @@ moa_status moa_attn_fused_fwd_bwd(const moa_attn_desc *desc, const void *Q, cons
     if (desc->materialize) return run_materialized(desc, Q, K, V, dO, O, L, dQ, dK, dV, ws, true, (cudaStream_t)stream);
     if ((s = run_fwd(desc, Q, K, V, O, L, (cudaStream_t)stream)) != MOA_OK) return s;
     return run_bwd(desc, Q, K, V, O, L, dO, dQ, dK, dV, ws, (cudaStream_t)stream);
+}
+
+moa_status moa_attn_fused_rowparallel(const moa_attn_desc *desc, const void *Q, const void *K, const void *V,
+                                      const void *dO, void *O, float *L, void *dQ, void *dK, void *dV,
+                                      int atomic_sites, void *ws, size_t ws_bytes, void *stream)
+{
+    moa_status s = check_desc(desc);
+    if (s != MOA_OK) return s;
+    if (atomic_sites != 1 && atomic_sites != 2) return MOA_ERR_INVALID_ARG;
+    if ((desc->H_kv > 0 && desc->H_kv != desc->H) || desc->layout != MOA_LAYOUT_BHND) return MOA_ERR_UNSUPPORTED;
+    if (!Q || !K || !V || !O || !L || !dO || !dQ || !dK || !dV) return MOA_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(L) || !aligned16(dO) ||
+        !aligned16(dQ) || !aligned16(dK) || !aligned16(dV))
+        return MOA_ERR_INVALID_ARG;
+    if (!ws || ws_bytes < rowpar_workspace(desc)) return MOA_ERR_WORKSPACE;
+    if (!aligned16(ws)) return MOA_ERR_INVALID_ARG;
+    if ((s = check_arch()) != MOA_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    Problem p = to_problem(desc);
+    p.Hkv = 0;
+    const size_t rows = (size_t)p.BH() * p.n, elems = rows * p.d;
+    float *Dv = (float *)ws;
+    const bool bf = desc->dtype == MOA_BF16;
+    float *dKacc = bf ? (float *)((char *)ws + align_up(rows * sizeof(float))) : (float *)dK;
+    float *dVacc = bf ? dKacc + align_up(elems * sizeof(float)) / sizeof(float) : (float *)dV;
+#define MOA_TRY(x) do { if ((x) != cudaSuccess) return MOA_ERR_CUDA; } while (0)
+    MOA_TRY(cudaMemsetAsync(dKacc, 0, elems * sizeof(float), st));
+    if (atomic_sites == 2) MOA_TRY(cudaMemsetAsync(dVacc, 0, elems * sizeof(float), st));
+    MOA_TRY(simt_rowpar(p, desc->dtype, Q, K, V, dO, O, L, Dv, dQ, dKacc, dVacc, atomic_sites, st));
+    if (atomic_sites == 1)   // dV by the atomic-free key-parallel kernel (no dK, no dQ from it)
+        MOA_TRY(simt_bwd_kv(p, desc->dtype, Q, K, V, dO, L, Dv, nullptr, dV, nullptr, st));
+    if (bf) {
+        MOA_TRY(convert_f32_to_bf16(dKacc, dK, elems, 1.f, st));
+        if (atomic_sites == 2) MOA_TRY(convert_f32_to_bf16(dVacc, dV, elems, 1.f, st));
+    }
+#undef MOA_TRY
+    return MOA_OK;
 }
 
 moa_status moa_last_device_status(void *stream)

@@ -228,7 +228,8 @@ simt_bwd_kv_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__
     const int bh = blockIdx.x / nkt;
     const int k0 = kt * BN;
     const size_t base = (size_t)bh * n * D;
-    Q += base; K += base; V += base; dO += base; dK += base; dV += base;
+    Q += base; K += base; V += base; dO += base; dV += base;
+    if (dK) dK += base;
     L += (size_t)bh * n; Dv += (size_t)bh * n;
     if (dQacc) dQacc += base;
     const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
@@ -301,7 +302,7 @@ simt_bwd_kv_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__
         if (row >= n) continue;
 #pragma unroll
         for (int c = 0; c < NC; ++c) {
-            dK[(size_t)row * D + tx + 16 * c] = from_float<T>(dk[a][c]);
+            if (dK) dK[(size_t)row * D + tx + 16 * c] = from_float<T>(dk[a][c]);   // nullptr: dV only
             dV[(size_t)row * D + tx + 16 * c] = from_float<T>(dv[a][c]);
         }
     }
@@ -357,6 +358,202 @@ simt_bwd_dq_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__
             for (int a = 0; a < 4; ++a)
 #pragma unroll
                 for (int c = 0; c < NC; ++c) dq[a][c] = fmaf(gv[a], kk[c], dq[a][c]);
+        }
+    }
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+        const int row = q0 + ty * 4 + a;
+        if (row >= n) continue;
+#pragma unroll
+        for (int c = 0; c < NC; ++c) dQ[(size_t)row * D + tx + 16 * c] = from_float<T>(dq[a][c]);
+    }
+}
+
+// ------------------ row-parallel fused forward+backward in one kernel, dK/dV by atomics
+// The paper's own fused design (Sec. 4, its first GPU version): one kernel, parallel over query
+// rows.  A CTA runs the forward of its 64 query rows (online softmax; O, L), takes D = rowsum(dO o O)
+// from the O it holds, and runs the backward of the same rows straight away: every row statistic it
+// needs is its own, so no other CTA is waited for.  dQ stays local; the dV and dK contributions of
+// every (query tile, key tile) pair are added into global fp32 accumulators with atomics -- the
+// paper's GV and GK atomic sites.  kSites = 2: both sites (the paper's v1).  kSites = 1: only dK;
+// dV then comes from an atomic-free key-parallel kernel of its own, as in the paper's v3.
+template <typename T, int D, int kSites>
+__global__ void __launch_bounds__(NTHREADS)
+simt_rowpar_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__restrict__ V,
+                   const T *__restrict__ dO, T *__restrict__ O, float *__restrict__ L, float *__restrict__ Dv,
+                   T *__restrict__ dQ, float *__restrict__ dKacc, float *__restrict__ dVacc,
+                   int n, int causal, float scale, int nqt)
+{
+    constexpr int LD = D + 1;
+    constexpr int NC = D / 16;
+    extern __shared__ float smem[];
+    float *Ks = smem, *Vs = Ks + BN * LD, *Qs = Vs + BN * LD, *dOs = Qs + BM * LD;
+    float *Ps = dOs + BM * LD, *dSs = Ps + BM * SLD, *Ls = dSs + BM * SLD, *Ds = Ls + BM;
+
+    int qt = blockIdx.x % nqt;
+    const int bh = blockIdx.x / nqt;
+    if (causal) qt = nqt - 1 - qt;  // longest rows first
+    const int q0 = qt * BM;
+    const size_t base = (size_t)bh * n * D;
+    Q += base; K += base; V += base; dO += base; O += base; dQ += base; dKacc += base;
+    if (kSites == 2) dVacc += base;
+    L += (size_t)bh * n; Dv += (size_t)bh * n;
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+    load_tile<T, D>(Qs, Q, q0, n);
+    load_tile<T, D>(dOs, dO, q0, n);
+    const int kend = causal ? min(n, q0 + BM) : n;
+
+    // ---- forward of these rows (as simt_fwd_kernel; the P tile goes through Ps)
+    {
+        float m[4], l[4], o[4][NC];
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+            m[a] = -INFINITY; l[a] = 0.f;
+#pragma unroll
+            for (int c = 0; c < NC; ++c) o[a][c] = 0.f;
+        }
+        for (int k0 = 0; k0 < kend; k0 += BN) {
+            __syncthreads();
+            load_tile<T, D>(Ks, K, k0, n);
+            load_tile<T, D>(Vs, V, k0, n);
+            __syncthreads();
+            float s[4][4];
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) s[a][b] = 0.f;
+#pragma unroll 4
+            for (int k = 0; k < D; ++k) {
+                float qv[4], kv[4];
+#pragma unroll
+                for (int a = 0; a < 4; ++a) qv[a] = Qs[(ty * 4 + a) * LD + k];
+#pragma unroll
+                for (int b = 0; b < 4; ++b) kv[b] = Ks[(tx + 16 * b) * LD + k];
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) s[a][b] = fmaf(qv[a], kv[b], s[a][b]);
+            }
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+                const int row = q0 + ty * 4 + a;
+                float mx = -INFINITY;
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    const int col = k0 + tx + 16 * b;
+                    float v = s[a][b] * scale;
+                    if (col >= n || (causal && col > row)) v = -INFINITY;
+                    s[a][b] = v;
+                    mx = fmaxf(mx, v);
+                }
+                mx = group16_max(mx);
+                float mn = fmaxf(m[a], mx);
+                if (mn == -INFINITY) mn = 0.f;  // whole row masked so far (padding rows only)
+                const float alpha = expf(m[a] - mn);
+                float sum = 0.f;
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    const float pv = expf(s[a][b] - mn);
+                    sum += pv;
+                    Ps[(ty * 4 + a) * SLD + tx + 16 * b] = pv;
+                }
+                sum = group16_sum(sum);
+                l[a] = l[a] * alpha + sum;
+                m[a] = mn;
+#pragma unroll
+                for (int c = 0; c < NC; ++c) o[a][c] *= alpha;
+            }
+            __syncthreads();
+#pragma unroll 4
+            for (int j = 0; j < BN; ++j) {
+                float pv[4], vv[NC];
+#pragma unroll
+                for (int a = 0; a < 4; ++a) pv[a] = Ps[(ty * 4 + a) * SLD + j];
+#pragma unroll
+                for (int c = 0; c < NC; ++c) vv[c] = Vs[j * LD + tx + 16 * c];
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+#pragma unroll
+                    for (int c = 0; c < NC; ++c) o[a][c] = fmaf(pv[a], vv[c], o[a][c]);
+            }
+        }
+        // O, L, and D = rowsum(dO o O) from the fp32 O held here (the paper's precompute pass)
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+            const int r = ty * 4 + a, row = q0 + r;
+            const float inv = row < n ? 1.f / l[a] : 0.f;
+            float dsum = 0.f;
+#pragma unroll
+            for (int c = 0; c < NC; ++c) {
+                const float ov = o[a][c] * inv;
+                dsum = fmaf(ov, dOs[r * LD + tx + 16 * c], dsum);
+                if (row < n) O[(size_t)row * D + tx + 16 * c] = from_float<T>(ov);
+            }
+            dsum = group16_sum(dsum);
+            if (tx == 0) {
+                const float lse = row < n ? m[a] + logf(l[a]) : 0.f;
+                Ls[r] = lse;
+                Ds[r] = row < n ? dsum : 0.f;
+                if (row < n) { L[row] = lse; Dv[row] = dsum; }
+            }
+        }
+    }
+
+    // ---- backward of the same rows
+    float dq[4][NC];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int c = 0; c < NC; ++c) dq[a][c] = 0.f;
+    for (int k0 = 0; k0 < kend; k0 += BN) {
+        __syncthreads();
+        load_tile<T, D>(Ks, K, k0, n);
+        load_tile<T, D>(Vs, V, k0, n);
+        __syncthreads();
+        bwd_tile_p_ds<D>(Qs, dOs, Ks, Vs, Ls, Ds, Ps, dSs, q0, k0, n, causal, scale, tx, ty);
+        __syncthreads();
+#pragma unroll 2
+        for (int j = 0; j < BN; ++j) {
+            float gv[4], kk[NC];
+#pragma unroll
+            for (int a = 0; a < 4; ++a) gv[a] = dSs[(ty * 4 + a) * SLD + j];
+#pragma unroll
+            for (int c = 0; c < NC; ++c) kk[c] = Ks[j * LD + tx + 16 * c];
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int c = 0; c < NC; ++c) dq[a][c] = fmaf(gv[a], kk[c], dq[a][c]);
+        }
+        // this tile pair's dK (and dV) contribution: [keys][d], thread (ty,tx) owns keys ty*4+a
+        float dk[4][NC], dv[4][NC];
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int c = 0; c < NC; ++c) { dk[a][c] = 0.f; dv[a][c] = 0.f; }
+#pragma unroll 2
+        for (int q = 0; q < BM; ++q) {
+            float pv[4], gv[4], gq[NC], qq[NC];
+#pragma unroll
+            for (int a = 0; a < 4; ++a) { pv[a] = Ps[q * SLD + ty * 4 + a]; gv[a] = dSs[q * SLD + ty * 4 + a]; }
+#pragma unroll
+            for (int c = 0; c < NC; ++c) { gq[c] = dOs[q * LD + tx + 16 * c]; qq[c] = Qs[q * LD + tx + 16 * c]; }
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int c = 0; c < NC; ++c) {
+                    if (kSites == 2) dv[a][c] = fmaf(pv[a], gq[c], dv[a][c]);
+                    dk[a][c] = fmaf(gv[a], qq[c], dk[a][c]);
+                }
+        }
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+            const int row = k0 + ty * 4 + a;
+            if (row >= n) continue;
+#pragma unroll
+            for (int c = 0; c < NC; ++c) {
+                atomicAdd(&dKacc[(size_t)row * D + tx + 16 * c], dk[a][c]);                     // atomic site GK
+                if (kSites == 2) atomicAdd(&dVacc[(size_t)row * D + tx + 16 * c], dv[a][c]);    // atomic site GV
+            }
         }
     }
 #pragma unroll
@@ -466,6 +663,26 @@ cudaError_t bwd_dq_t(const Problem &p, const void *Q, const void *K, const void 
     return cudaGetLastError();
 }
 
+template <typename T, int D>
+cudaError_t rowpar_t(const Problem &p, const void *Q, const void *K, const void *V, const void *dO, void *O, float *L,
+                     float *Dv, void *dQ, float *dKacc, float *dVacc, int sites, cudaStream_t st)
+{
+    const int nqt = (p.n + BM - 1) / BM;
+    cudaError_t e = set_smem(simt_rowpar_kernel<T, D, 1>, bwd_smem(D));
+    if (e == cudaSuccess) e = set_smem(simt_rowpar_kernel<T, D, 2>, bwd_smem(D));
+    if (e != cudaSuccess) return e;
+    LaunchScope scope(MOA_KERNEL_OTHER, st);
+    if (sites == 2)
+        simt_rowpar_kernel<T, D, 2><<<(unsigned)(nqt * p.BH()), NTHREADS, bwd_smem(D), st>>>(
+            (const T *)Q, (const T *)K, (const T *)V, (const T *)dO, (T *)O, L, Dv, (T *)dQ, dKacc, dVacc,
+            p.n, p.causal, p.scale, nqt);
+    else
+        simt_rowpar_kernel<T, D, 1><<<(unsigned)(nqt * p.BH()), NTHREADS, bwd_smem(D), st>>>(
+            (const T *)Q, (const T *)K, (const T *)V, (const T *)dO, (T *)O, L, Dv, (T *)dQ, dKacc, dVacc,
+            p.n, p.causal, p.scale, nqt);
+    return cudaGetLastError();
+}
+
 #define MOA_DISPATCH(FN, ...)                                                         \
     do {                                                                              \
         if (dtype == MOA_F32) {                                                       \
@@ -491,6 +708,12 @@ cudaError_t simt_bwd_kv(const Problem &p, int dtype, const void *Q, const void *
                         void *dK, void *dV, float *dQacc, cudaStream_t st)
 {
     MOA_DISPATCH(bwd_kv_t, p, Q, K, V, dO, L, Dv, dK, dV, dQacc, st);
+}
+
+cudaError_t simt_rowpar(const Problem &p, int dtype, const void *Q, const void *K, const void *V, const void *dO,
+                        void *O, float *L, float *Dv, void *dQ, float *dKacc, float *dVacc, int sites, cudaStream_t st)
+{
+    MOA_DISPATCH(rowpar_t, p, Q, K, V, dO, O, L, Dv, dQ, dKacc, dVacc, sites, st);
 }
 
 cudaError_t simt_bwd_dq(const Problem &p, int dtype, const void *Q, const void *K, const void *V,

@@ -46,7 +46,11 @@ def run_library(inp: dict, dtype: str, causal: bool, scale: float, *, op: str = 
     if materialize and op == "split":
         raise ValueError("the materialising variant has no separate backward call")
     ws = torch.full((max(ws_bytes, 16),), 0xFF, dtype=torch.uint8, device="cuda")
-    if op == "fused":
+    if op in ("rowpar1", "rowpar2"):      # the row-parallel single-kernel comparison variant, 1 or 2 atomic sites
+        ws_bytes = mb.moa_attn_workspace_bytes(desc, mb.MOA_OP_ROWPARALLEL)
+        ws = torch.full((max(ws_bytes, 16),), 0xFF, dtype=torch.uint8, device="cuda")
+        mb.moa_attn_fused_rowparallel(desc, Q, K, V, dO, O, L, dQ, dK, dV, int(op[-1]), ws)
+    elif op == "fused":
         mb.moa_attn_fused_fwd_bwd(desc, Q, K, V, dO, O, L, dQ, dK, dV, ws)
     elif op == "split":
         mb.moa_attn_fwd(desc, Q, K, V, O, L, ws)

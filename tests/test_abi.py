@@ -105,3 +105,17 @@ def test_shared_kv_heads_argument_checks(lib):
     # the workspace does not depend on the number of K/V heads: D, L' and the dQ accumulator are per query head
     w = lambda hkv: mb.moa_attn_workspace_bytes(mb.make_desc(1, 8, 256, 128, True, 0.1, H_kv=hkv), mb.MOA_OP_FUSED)
     assert w(0) == w(8) == w(2) == w(1) > 0
+
+
+def test_rowparallel_variant_argument_checks(lib):
+    a = 4096
+    d = mb.make_desc(1, 4, 256, 64, True, 0.1)
+    call = lambda desc, sites, wsb=1 << 40: mb.moa_attn_fused_rowparallel(desc, a, a, a, a, a, a, a, a, a, sites, a,
+                                                                          ws_bytes=wsb, check=False)
+    assert call(d, 0) == mb.MOA_ERR_INVALID_ARG and call(d, 3) == mb.MOA_ERR_INVALID_ARG
+    assert call(mb.make_desc(1, 4, 256, 64, True, 0.1, H_kv=2), 2) == mb.MOA_ERR_UNSUPPORTED
+    assert call(d, 2, wsb=16) == mb.MOA_ERR_WORKSPACE
+    need = mb.moa_attn_workspace_bytes(d, mb.MOA_OP_ROWPARALLEL)
+    assert need == 4 * 256 * 4 + 2 * 4 * 256 * 64 * 4          # D + two fp32 accumulators (bf16 tensors)
+    d32 = mb.make_desc(1, 4, 256, 64, True, 0.1, mb.MOA_F32)
+    assert mb.moa_attn_workspace_bytes(d32, mb.MOA_OP_ROWPARALLEL) == 4 * 256 * 4
