@@ -279,6 +279,8 @@ def main():
     ap.add_argument("--path", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--materialize", type=int, default=0)
+    ap.add_argument("--rowparallel", type=int, default=0,
+                    help="1 or 2: time the row-parallel single-kernel comparison variant with that many atomic sites")
     ap.add_argument("--layout", type=int, default=0, help="0: tensors [B,H,n,d] (every named config); 1: [B,n,H,d]")
     ap.add_argument("--hkv", type=int, default=0,
                     help="key/value heads (grouped-query attention); 0: one per query head, as in every named config")
@@ -342,8 +344,15 @@ def main():
     resident_bytes = torch.cuda.memory_allocated() - base_mem
     stream = torch.cuda.current_stream()
 
+    if args.rowparallel:
+        ws_bytes = mb.moa_attn_workspace_bytes(desc, mb.MOA_OP_ROWPARALLEL)
+        ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device="cuda")
+
     def step():
-        mb.moa_attn_fused_fwd_bwd(desc, Q, K, V, dO, O, L, dQ, dK, dV, ws, stream)
+        if args.rowparallel:
+            mb.moa_attn_fused_rowparallel(desc, Q, K, V, dO, O, L, dQ, dK, dV, args.rowparallel, ws, stream)
+        else:
+            mb.moa_attn_fused_fwd_bwd(desc, Q, K, V, dO, O, L, dQ, dK, dV, ws, stream)
 
     def barrier():
         torch.cuda.synchronize()
@@ -430,8 +439,12 @@ def main():
         with torch.cuda.stream(s_run):
             s_run.wait_event(b["up"])
             s_run.wait_event(b["down"])          # its previous results have been read back
-            mb.moa_attn_fused_fwd_bwd(desc, b["in"][0], b["in"][1], b["in"][2], b["in"][3], b["out"][0], b["L"],
-                                      b["out"][1], b["out"][2], b["out"][3], b["ws"], s_run)
+            if args.rowparallel:
+                mb.moa_attn_fused_rowparallel(desc, b["in"][0], b["in"][1], b["in"][2], b["in"][3], b["out"][0], b["L"],
+                                              b["out"][1], b["out"][2], b["out"][3], args.rowparallel, b["ws"], s_run)
+            else:
+                mb.moa_attn_fused_fwd_bwd(desc, b["in"][0], b["in"][1], b["in"][2], b["in"][3], b["out"][0], b["L"],
+                                          b["out"][1], b["out"][2], b["out"][3], b["ws"], s_run)
             b["done"].record(s_run)
         with torch.cuda.stream(s_down):
             s_down.wait_event(b["done"])
@@ -501,7 +514,9 @@ def main():
         line["config"]["H_kv"] = args.hkv
     if args.layout:
         line["config"]["layout"] = "[B,n,H,d]"
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.hkv and not args.layout:
+    if args.rowparallel:
+        line["config"]["variant"] = f"row-parallel single kernel, {args.rowparallel} atomic site(s), fp32 CUDA cores"
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.hkv and not args.layout and not args.rowparallel:
         v, dt, cores, desc_s = time_oracle_sample(w, 20.0)
         line["cpu_baseline"] = {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
                                 "sample": desc_s, "seconds": dt}

@@ -50,6 +50,9 @@ CONFIGS = {
     "c4_long": Workload("c4_long", 1, 16, 16384, 128, False, "bf16", 3),
 }
 # a small non-causal case for profiler captures: larger than L2 in total, short kernels
+# the shape of the paper's own GPU tables (B = 2, no heads, D = 64), for the atomic-site comparison
+CONFIGS["paper_b2_n2048_d64"] = Workload("paper_b2_n2048_d64", 2, 1, 2048, 64, False, "bf16", 6)
+CONFIGS["paper_b2_n8192_d64"] = Workload("paper_b2_n8192_d64", 2, 1, 8192, 64, False, "bf16", 7)
 CONFIGS["prof_h8_n8192"] = Workload("prof_h8_n8192", 1, 8, 8192, 128, False, "bf16", 5)
 C5_SIZES = (512, 1024, 2048, 4096, 8192, 16384, 32768)
 for _n in C5_SIZES:
