@@ -13,3 +13,4 @@ from .attention import (  # noqa: F401
     attn_rows,
     attn_cols,
 )
+from .decode import decode_attn  # noqa: F401,E402

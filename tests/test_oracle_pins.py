@@ -300,3 +300,63 @@ def test_paper_counts_fix_array_shapes():
     a = g["atomic_counts_n2048"]
     assert B * N * N * D == a["backward_gk_only"]
     assert 2 * B * N * N * D == a["fused_gv_and_gk"]
+
+
+# ----------------------------------------------------------------- decode attention
+def test_decode_uniform_and_one_hot_closed_forms():
+    """q = 0: every key weighs 1/n, so o is the mean of V and lse = log n.  One key with a huge
+    score: o is that key's value row."""
+    rng = np.random.default_rng(5)
+    B, H, Hkv, n, d = 2, 4, 2, 37, 6
+    K, V = (rng.standard_normal((B, Hkv, n, d)) for _ in range(2))
+    r = oracle.decode_attn(np.zeros((B, H, d)), K, V, 0.7)
+    for h in range(H):
+        np.testing.assert_allclose(r["o"][:, h], V[:, h // 2].mean(1), atol=1e-14)
+    np.testing.assert_allclose(r["lse"], math.log(n), atol=1e-14)
+    q = rng.standard_normal((B, H, d))
+    K2 = 0.01 * K
+    K2[:, :, 11] = 0.0
+    K2[0, 0, 11] = 50.0 * q[0, 1] / np.dot(q[0, 1], q[0, 1])      # score 50 * scale^-1 ... for query head 1 (K/V head 0)
+    r2 = oracle.decode_attn(q, K2, V, 1.0)
+    np.testing.assert_allclose(r2["o"][0, 1], V[0, 0, 11], atol=1e-12)
+
+
+@pytest.mark.parametrize("Hkv", [1, 3, 6])
+def test_decode_is_the_last_row_of_causal_attention(Hkv):
+    """The token at position n-1 sees the whole cache: decode of that query equals row n-1 of the
+    causal attention the pinned forward oracle computes (and its L there)."""
+    rng = np.random.default_rng(8)
+    B, H, n, d, scale = 2, 6, 23, 5, 0.41
+    Q, dO = (rng.standard_normal((B, H, n, d)) for _ in range(2))
+    K, V = (rng.standard_normal((B, Hkv, n, d)) for _ in range(2))
+    full = oracle.attn_fwd_bwd_gqa(Q, K, V, dO, True, scale)
+    r = oracle.decode_attn(Q[:, :, n - 1], K, V, scale)
+    np.testing.assert_allclose(r["o"], full["O"][:, :, n - 1], atol=1e-13)
+    np.testing.assert_allclose(r["lse"], full["L"][:, :, n - 1], atol=1e-13)
+
+
+def test_decode_against_torch():
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(9)
+    B, H, Hkv, n, d, scale = 3, 8, 2, 41, 16, 0.2
+    q = rng.standard_normal((B, H, d))
+    K, V = (rng.standard_normal((B, Hkv, n, d)) for _ in range(2))
+    r = oracle.decode_attn(q, K, V, scale)
+    o = torch.nn.functional.scaled_dot_product_attention(torch.tensor(q)[:, :, None, :], torch.tensor(K), torch.tensor(V),
+                                                         scale=scale, enable_gqa=True)
+    np.testing.assert_allclose(r["o"], o[:, :, 0].numpy(), atol=1e-13)
+
+
+def test_decode_segments_merge_by_logsumexp():
+    """Splitting the cache and merging the parts with their lse weights gives the whole: the identity
+    a split-cache kernel relies on."""
+    rng = np.random.default_rng(10)
+    B, H, n, d = 1, 2, 50, 4
+    q = rng.standard_normal((B, H, d)); K, V = (rng.standard_normal((B, H, n, d)) for _ in range(2))
+    whole = oracle.decode_attn(q, K, V, 0.5)
+    a = oracle.decode_attn(q, K[:, :, :17], V[:, :, :17], 0.5)
+    b = oracle.decode_attn(q, K[:, :, 17:], V[:, :, 17:], 0.5)
+    lse = np.logaddexp(a["lse"], b["lse"])
+    o = np.exp(a["lse"] - lse)[..., None] * a["o"] + np.exp(b["lse"] - lse)[..., None] * b["o"]
+    np.testing.assert_allclose(o, whole["o"], atol=1e-14)
+    np.testing.assert_allclose(lse, whole["lse"], atol=1e-14)
