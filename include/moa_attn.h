@@ -179,6 +179,23 @@ moa_status moa_attn_fused_rowparallel(const moa_attn_desc *desc,
                                       void *O, float *L, void *dQ, void *dK, void *dV,
                                       int atomic_sites, void *ws, size_t ws_bytes, void *stream);
 
+/* Decode attention (the paper's inference section): one new query per head over a cache of n
+ * keys and values, O(n) work, every cached element read once:
+ *     out[b,h,:] = softmax_j(scale * q[b,h,:] . K[b,kv,j,:]) V[b,kv,:,:],   kv = h / (H / H_kv).
+ * q, out: [B,H,d]; K, V: [B,H_kv,n,d] (H_kv = 0 means H; grouped-query heads share one pass over
+ * their K/V head); lse: [B,H] fp32 natural-log logsumexp of the scaled scores, may be NULL.
+ * dtype: MOA_BF16 or MOA_F32 (fp32 accumulation either way); d in {64, 128}.  All device
+ * pointers, 16-byte aligned; the caller owns every buffer; asynchronous on `stream`.
+ * Workspace: moa_decode_workspace_bytes(desc) (partial results of the cache segments). */
+typedef struct {
+    int32_t B, H, H_kv, n, d;
+    float   scale;
+    int32_t dtype;       /* moa_dtype */
+} moa_decode_desc;
+size_t moa_decode_workspace_bytes(const moa_decode_desc *desc);
+moa_status moa_decode_attn(const moa_decode_desc *desc, const void *q, const void *K, const void *V,
+                           void *out, float *lse, void *ws, size_t ws_bytes, void *stream);
+
 /* Synchronises `stream` and returns MOA_ERR_TIMEOUT if any kernel launched by this
  * library on the current device gave up a bounded wait since the last call of this
  * function (the flag is then cleared), MOA_ERR_CUDA if the stream reports an error,

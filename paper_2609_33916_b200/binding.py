@@ -27,6 +27,7 @@ EXPORTS = (
     "moa_attn_workspace_bytes", "moa_attn_fwd", "moa_attn_bwd", "moa_attn_fused_fwd_bwd",
     "moa_last_device_status", "moa_launch_count", "moa_status_string", "moa_version",
     "moa_profile_enable", "moa_profile_read", "moa_attn_bwd_static_scratch", "moa_attn_fused_rowparallel",
+    "moa_decode_workspace_bytes", "moa_decode_attn",
 )
 
 
@@ -35,6 +36,11 @@ class moa_attn_desc(ctypes.Structure):
                 ("causal", ctypes.c_int32), ("scale", ctypes.c_float), ("dtype", ctypes.c_int32),
                 ("dq_mode", ctypes.c_int32), ("materialize", ctypes.c_int32), ("path", ctypes.c_int32),
                 ("H_kv", ctypes.c_int32), ("layout", ctypes.c_int32)]
+
+
+class moa_decode_desc(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("H_kv", ctypes.c_int32), ("n", ctypes.c_int32),
+                ("d", ctypes.c_int32), ("scale", ctypes.c_float), ("dtype", ctypes.c_int32)]
 
 
 MOA_KERNEL_KINDS = 6
@@ -75,6 +81,10 @@ def lib() -> ctypes.CDLL:
         L.moa_attn_fused_fwd_bwd.argtypes = [dp] + [vp] * 9 + [vp, sz, vp]
         L.moa_attn_fused_rowparallel.restype = ctypes.c_int
         L.moa_attn_fused_rowparallel.argtypes = [dp] + [vp] * 9 + [ctypes.c_int, vp, sz, vp]
+        L.moa_decode_workspace_bytes.restype = sz
+        L.moa_decode_workspace_bytes.argtypes = [ctypes.POINTER(moa_decode_desc)]
+        L.moa_decode_attn.restype = ctypes.c_int
+        L.moa_decode_attn.argtypes = [ctypes.POINTER(moa_decode_desc)] + [vp] * 5 + [vp, sz, vp]
         L.moa_last_device_status.restype = ctypes.c_int
         L.moa_last_device_status.argtypes = [vp]
         L.moa_launch_count.restype = ctypes.c_uint64
@@ -183,6 +193,22 @@ def moa_attn_fused_rowparallel(desc, Q, K, V, dO, O, L, dQ, dK, dV, atomic_sites
                                          _nbytes(ws) if ws_bytes is None else ws_bytes, _stream(stream))
     if check and s != MOA_OK:
         raise MoaError(s, "moa_attn_fused_rowparallel")
+    return s
+
+
+def make_decode_desc(B, H, n, d, scale, dtype=MOA_BF16, H_kv=0) -> moa_decode_desc:
+    return moa_decode_desc(int(B), int(H), int(H_kv), int(n), int(d), float(scale), int(dtype))
+
+
+def moa_decode_workspace_bytes(desc: moa_decode_desc) -> int:
+    return int(lib().moa_decode_workspace_bytes(ctypes.byref(desc)))
+
+
+def moa_decode_attn(desc, q, K, V, out, lse=None, ws=None, stream=None, ws_bytes=None, check=True) -> int:
+    s = lib().moa_decode_attn(ctypes.byref(desc), _ptr(q), _ptr(K), _ptr(V), _ptr(out), _ptr(lse), _ptr(ws),
+                              _nbytes(ws) if ws_bytes is None else ws_bytes, _stream(stream))
+    if check and s != MOA_OK:
+        raise MoaError(s, "moa_decode_attn")
     return s
 
 

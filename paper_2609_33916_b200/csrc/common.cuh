@@ -49,6 +49,17 @@ inline int heads_per_group(const Problem &p, int tiles)
     return (int)g;
 }
 
+// ---- decode attention (decode.cu) ----------------------------------------------------
+struct DecodeProblem {
+    int B, H, Hkv, n, d;     // Hkv resolved (never 0)
+    float scale;
+};
+int decode_splits(const DecodeProblem &p);                  // cache segments per K/V head
+size_t decode_workspace_floats(const DecodeProblem &p);     // partial outputs, maxima and sums of all segments
+// q [B,H,d], K, V [B,Hkv,n,d] -> out [B,H,d] (dtype of the inputs), lse [B,H] fp32 (may be null)
+cudaError_t decode_attn(const DecodeProblem &p, int dtype, const void *q, const void *K, const void *V, void *out,
+                        float *lse, float *ws, cudaStream_t st);
+
 // Host-side launch counter (moa_launch_count).
 void count_launch(int k = 1);
 

@@ -1,0 +1,302 @@
+// Decode attention: one new query per head over a cache of n keys and values (the paper's
+// decode section: O(n) work per token, every cached element read exactly once).
+//
+// HBM-bound: 2 n d elements of cache per K/V head against 4 n d flop per query head, so the
+// kernel is organised around keeping reads in flight, not around the tensor cores (a tile of
+// 1..8 query rows would fill 1-6 % of a 128-row UMMA).  One CTA streams a segment of the cache
+// of one K/V head and serves all query heads that share it (grouped-query attention: the cache
+// is read once per group, not once per query head):
+//   * a row of d elements is fetched by d*sizeof(T)/16 lanes with one 16-byte streaming load
+//     each, so every warp instruction reads whole rows, fully coalesced; a warp keeps kUnroll
+//     row groups of K and of V in flight;
+//   * score = q . k: per-lane partial dot (the lane's 16 bytes of the row against the same
+//     elements of q, kept in registers, pre-multiplied by scale*log2 e), then an xor-shuffle
+//     butterfly over the lanes of the row;
+//   * online softmax per lane group (exp2, running max and sum), out += p * v on the lane's own
+//     elements of the V row: no further exchange inside the loop;
+//   * at the end the lane groups of a warp, the warps of the CTA (through shared memory) and,
+//     in a second tiny kernel, the CTAs of a head are merged by their running maxima.
+#include "common.cuh"
+
+namespace moa {
+namespace {
+
+constexpr int kWarps = 8;
+constexpr int kThreads = kWarps * 32;
+constexpr int kUnroll = 4;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+template <typename T> struct Vec16;
+template <> struct Vec16<__nv_bfloat16> {
+    static constexpr int kElems = 8;
+    __device__ static void unpack(const uint4 &v, float *f)
+    {
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 p = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&w[i]));
+            f[2 * i] = p.x;
+            f[2 * i + 1] = p.y;
+        }
+    }
+};
+template <> struct Vec16<float> {
+    static constexpr int kElems = 4;
+    __device__ static void unpack(const uint4 &v, float *f)
+    {
+        f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y); f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+    }
+};
+
+// Partial results of one cache segment: for every query head the running maximum m (log2 domain),
+// the sum l of 2^(s - m) and the unnormalised output sum_j 2^(s_j - m) v_j.
+//   part_o [splits][B*H][D], part_ml [splits][B*H][2]
+template <typename T, int D, int GC>
+__global__ void __launch_bounds__(kThreads)
+decode_split_kernel(const T *__restrict__ q, const T *__restrict__ K, const T *__restrict__ V,
+                    float *__restrict__ part_o, float *__restrict__ part_ml,
+                    int n, int H, int Hkv, int group, int splits, int keys_per_split, size_t BH, float scale_log2)
+{
+    constexpr int E = Vec16<T>::kElems;      // elements per lane
+    constexpr int LPR = D / E;               // lanes per row
+    constexpr int RPW = 32 / LPR;            // rows per warp-wide load
+    static_assert(LPR >= 1 && LPR <= 32 && 32 % LPR == 0, "row must map onto a warp");
+    const int split = blockIdx.x % splits;
+    const int bkv = blockIdx.x / splits;                 // b * Hkv + kv head
+    const int g0 = blockIdx.y * GC;                      // first query head of the group handled here
+    const int gcount = min(GC, group - g0);
+    const int b = bkv / Hkv, kvh = bkv - b * Hkv;
+    const int hq0 = kvh * group + g0;                    // first query head (within the batch element)
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int sub = lane / LPR, l = lane % LPR;          // row of the group, lane of the row
+    const T *Kh = K + (size_t)bkv * n * D;
+    const T *Vh = V + (size_t)bkv * n * D;
+    const int k_begin = split * keys_per_split, k_end = min(n, k_begin + keys_per_split);
+
+    // this lane's elements of every query of the group, pre-scaled
+    float qv[GC][E];
+#pragma unroll
+    for (int g = 0; g < GC; ++g) {
+        float f[E];
+        if (g < gcount) {
+            const uint4 raw = *reinterpret_cast<const uint4 *>(q + ((size_t)b * H + hq0 + g) * D + l * E);
+            Vec16<T>::unpack(raw, f);
+        } else {
+#pragma unroll
+            for (int e = 0; e < E; ++e) f[e] = 0.f;
+        }
+#pragma unroll
+        for (int e = 0; e < E; ++e) qv[g][e] = f[e] * scale_log2;
+    }
+
+    float m[GC], lsum[GC], acc[GC][E];
+#pragma unroll
+    for (int g = 0; g < GC; ++g) {
+        m[g] = -INFINITY;
+        lsum[g] = 0.f;
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[g][e] = 0.f;
+    }
+
+    constexpr int kRowsPerIter = kUnroll * RPW;          // rows one warp consumes per iteration
+    for (int base = k_begin + warp * kRowsPerIter; base < k_end; base += kWarps * kRowsPerIter) {
+        uint4 kraw[kUnroll], vraw[kUnroll];
+        bool live[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const int row = base + u * RPW + sub;
+            live[u] = row < k_end;
+            const size_t off = (size_t)(live[u] ? row : k_begin) * D + l * E;
+            kraw[u] = __ldcs(reinterpret_cast<const uint4 *>(Kh + off));
+            vraw[u] = __ldcs(reinterpret_cast<const uint4 *>(Vh + off));
+        }
+        float s[kUnroll][GC];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            float kf[E];
+            Vec16<T>::unpack(kraw[u], kf);
+#pragma unroll
+            for (int g = 0; g < GC; ++g) {
+                float d0 = 0.f;
+#pragma unroll
+                for (int e = 0; e < E; ++e) d0 = fmaf(qv[g][e], kf[e], d0);
+#pragma unroll
+                for (int o = LPR / 2; o >= 1; o >>= 1) d0 += __shfl_xor_sync(0xffffffffu, d0, o);
+                s[u][g] = live[u] ? d0 : -INFINITY;
+            }
+        }
+#pragma unroll
+        for (int g = 0; g < GC; ++g) {
+            float mx = m[g];
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) mx = fmaxf(mx, s[u][g]);
+            const float ref = (mx == -INFINITY) ? 0.f : mx;      // nothing visible yet: any finite reference
+            const float alpha = exp2f(m[g] - ref);
+            m[g] = mx;
+            lsum[g] *= alpha;
+#pragma unroll
+            for (int e = 0; e < E; ++e) acc[g][e] *= alpha;
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) s[u][g] = exp2f(s[u][g] - ref);     // now the weight p
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            float vf[E];
+            Vec16<T>::unpack(vraw[u], vf);
+#pragma unroll
+            for (int g = 0; g < GC; ++g) {
+                lsum[g] += s[u][g];
+#pragma unroll
+                for (int e = 0; e < E; ++e) acc[g][e] = fmaf(s[u][g], vf[e], acc[g][e]);
+            }
+        }
+    }
+
+    // ---- merge the RPW lane groups of the warp (same elements, different rows)
+#pragma unroll
+    for (int o = LPR; o < 32; o <<= 1) {
+#pragma unroll
+        for (int g = 0; g < GC; ++g) {
+            const float mo = __shfl_xor_sync(0xffffffffu, m[g], o);
+            const float lo = __shfl_xor_sync(0xffffffffu, lsum[g], o);
+            const float mx = fmaxf(m[g], mo);
+            const float ref = (mx == -INFINITY) ? 0.f : mx;
+            const float a = exp2f(m[g] - ref), bo = exp2f(mo - ref);
+            lsum[g] = lsum[g] * a + lo * bo;
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                const float ao = __shfl_xor_sync(0xffffffffu, acc[g][e], o);
+                acc[g][e] = acc[g][e] * a + ao * bo;
+            }
+            m[g] = mx;
+        }
+    }
+    // ---- merge the warps through shared memory: [warp][g][D + 2]
+    extern __shared__ float sm[];
+    constexpr int kStride = D + 2;
+    if (sub == 0) {
+#pragma unroll
+        for (int g = 0; g < GC; ++g) {
+            float *dst = sm + (warp * GC + g) * kStride;
+#pragma unroll
+            for (int e = 0; e < E; ++e) dst[l * E + e] = acc[g][e];
+            if (l == 0) { dst[D] = m[g]; dst[D + 1] = lsum[g]; }
+        }
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < gcount * D; idx += kThreads) {
+        const int g = idx / D, c = idx - g * D;
+        float mx = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) mx = fmaxf(mx, sm[(w * GC + g) * kStride + D]);
+        const float ref = (mx == -INFINITY) ? 0.f : mx;
+        float o = 0.f, ls = 0.f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+            const float *src = sm + (w * GC + g) * kStride;
+            const float a = exp2f(src[D] - ref);
+            o = fmaf(src[c], a, o);
+            ls = fmaf(src[D + 1], a, ls);
+        }
+        const size_t head = (size_t)b * H + hq0 + g;
+        part_o[((size_t)split * BH + head) * D + c] = o;
+        if (c == 0) {
+            part_ml[((size_t)split * BH + head) * 2] = mx;
+            part_ml[((size_t)split * BH + head) * 2 + 1] = ls;
+        }
+    }
+}
+
+// One block per query head: merge the segments, normalise, write out (and the natural-log lse).
+template <typename T, int D>
+__global__ void decode_merge_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml,
+                                    T *__restrict__ out, float *__restrict__ lse, int splits, size_t BH)
+{
+    const size_t head = blockIdx.x;
+    const int c = threadIdx.x;
+    float mx = -INFINITY;
+    for (int s = 0; s < splits; ++s) mx = fmaxf(mx, part_ml[((size_t)s * BH + head) * 2]);
+    float o = 0.f, ls = 0.f;
+    for (int s = 0; s < splits; ++s) {
+        const float a = exp2f(part_ml[((size_t)s * BH + head) * 2] - mx);
+        o = fmaf(part_o[((size_t)s * BH + head) * D + c], a, o);
+        ls = fmaf(part_ml[((size_t)s * BH + head) * 2 + 1], a, ls);
+    }
+    out[head * D + c] = from_float<T>(o / ls);
+    if (lse && c == 0) lse[head] = (mx + log2f(ls)) * kLn2;
+}
+
+int group_chunk(int group) { return group >= 8 ? 8 : group >= 4 ? 4 : group >= 2 ? 2 : 1; }
+
+template <typename T, int D, int GC>
+cudaError_t launch_split(const DecodeProblem &p, const void *q, const void *K, const void *V, float *part_o,
+                         float *part_ml, int splits, int keys_per_split, cudaStream_t st)
+{
+    const int group = p.H / p.Hkv;
+    const size_t smem = (size_t)kWarps * GC * (D + 2) * sizeof(float);
+    cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<T, D, GC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    dim3 grid((unsigned)(p.B * p.Hkv * splits), (unsigned)((group + GC - 1) / GC));
+    LaunchScope scope(MOA_KERNEL_OTHER, st);
+    decode_split_kernel<T, D, GC><<<grid, kThreads, smem, st>>>((const T *)q, (const T *)K, (const T *)V, part_o, part_ml,
+                                                                p.n, p.H, p.Hkv, group, splits, keys_per_split,
+                                                                (size_t)p.B * p.H, p.scale * kLog2e);
+    return cudaGetLastError();
+}
+
+template <typename T, int D>
+cudaError_t launch_decode(const DecodeProblem &p, const void *q, const void *K, const void *V, void *out, float *lse,
+                          float *ws, cudaStream_t st)
+{
+    const int splits = decode_splits(p);
+    const int keys_per_split = (p.n + splits - 1) / splits;
+    const size_t BH = (size_t)p.B * p.H;
+    float *part_o = ws, *part_ml = ws + (size_t)splits * BH * D;
+    const int gc = group_chunk(p.H / p.Hkv);
+    cudaError_t e = gc == 8 ? launch_split<T, D, 8>(p, q, K, V, part_o, part_ml, splits, keys_per_split, st)
+                  : gc == 4 ? launch_split<T, D, 4>(p, q, K, V, part_o, part_ml, splits, keys_per_split, st)
+                  : gc == 2 ? launch_split<T, D, 2>(p, q, K, V, part_o, part_ml, splits, keys_per_split, st)
+                            : launch_split<T, D, 1>(p, q, K, V, part_o, part_ml, splits, keys_per_split, st);
+    if (e != cudaSuccess) return e;
+    LaunchScope scope(MOA_KERNEL_OTHER, st);
+    decode_merge_kernel<T, D><<<(unsigned)BH, D, 0, st>>>(part_o, part_ml, (T *)out, lse, splits, BH);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+// Segments of the cache per K/V head: enough CTAs to fill the GPU a few times over, each with at
+// least 256 keys.
+int decode_splits(const DecodeProblem &p)
+{
+    const int group = p.H / p.Hkv;
+    const int gc = group >= 8 ? 8 : group >= 4 ? 4 : group >= 2 ? 2 : 1;
+    const long long ctas_per_split = (long long)p.B * p.Hkv * ((group + gc - 1) / gc);
+    long long s = (4LL * 148 + ctas_per_split - 1) / ctas_per_split;
+    const long long cap = (p.n + 255) / 256;
+    if (s > cap) s = cap;
+    if (s < 1) s = 1;
+    if (s > 1024) s = 1024;
+    return (int)s;
+}
+
+size_t decode_workspace_floats(const DecodeProblem &p)
+{
+    return (size_t)decode_splits(p) * p.B * p.H * (p.d + 2);
+}
+
+cudaError_t decode_attn(const DecodeProblem &p, int dtype, const void *q, const void *K, const void *V, void *out,
+                        float *lse, float *ws, cudaStream_t st)
+{
+    if (dtype == MOA_F32) {
+        if (p.d == 64) return launch_decode<float, 64>(p, q, K, V, out, lse, ws, st);
+        if (p.d == 128) return launch_decode<float, 128>(p, q, K, V, out, lse, ws, st);
+    } else {
+        if (p.d == 64) return launch_decode<__nv_bfloat16, 64>(p, q, K, V, out, lse, ws, st);
+        if (p.d == 128) return launch_decode<__nv_bfloat16, 128>(p, q, K, V, out, lse, ws, st);
+    }
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace moa

@@ -422,6 +422,42 @@ moa_status moa_attn_fused_rowparallel(const moa_attn_desc *desc, const void *Q, 
     return MOA_OK;
 }
 
+static moa_status check_decode_desc(const moa_decode_desc *d, DecodeProblem *p)
+{
+    if (!d) return MOA_ERR_INVALID_ARG;
+    if (d->B <= 0 || d->H <= 0 || d->n <= 0 || d->d <= 0 || d->H_kv < 0 || d->H_kv > d->H) return MOA_ERR_INVALID_ARG;
+    const int hkv = d->H_kv > 0 ? d->H_kv : d->H;
+    if (d->H % hkv != 0) return MOA_ERR_INVALID_ARG;
+    if (d->dtype != MOA_BF16 && d->dtype != MOA_F32) return MOA_ERR_INVALID_ARG;
+    if (!(d->scale == d->scale) || d->scale - d->scale != 0.f) return MOA_ERR_INVALID_ARG;
+    if (d->d != 64 && d->d != 128) return MOA_ERR_UNSUPPORTED;
+    if ((long long)d->B * d->H > (1 << 24)) return MOA_ERR_UNSUPPORTED;
+    *p = DecodeProblem{d->B, d->H, hkv, d->n, d->d, d->scale};
+    return MOA_OK;
+}
+
+size_t moa_decode_workspace_bytes(const moa_decode_desc *desc)
+{
+    DecodeProblem p;
+    if (check_decode_desc(desc, &p) != MOA_OK) return 0;
+    return decode_workspace_floats(p) * sizeof(float);
+}
+
+moa_status moa_decode_attn(const moa_decode_desc *desc, const void *q, const void *K, const void *V,
+                           void *out, float *lse, void *ws, size_t ws_bytes, void *stream)
+{
+    DecodeProblem p;
+    moa_status s = check_decode_desc(desc, &p);
+    if (s != MOA_OK) return s;
+    if (!q || !K || !V || !out) return MOA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(K) || !aligned16(V) || !aligned16(out) || (lse && !aligned16(lse))) return MOA_ERR_INVALID_ARG;
+    if (!ws || ws_bytes < decode_workspace_floats(p) * sizeof(float)) return MOA_ERR_WORKSPACE;
+    if (!aligned16(ws)) return MOA_ERR_INVALID_ARG;
+    if ((s = check_arch()) != MOA_OK) return s;
+    return decode_attn(p, desc->dtype, q, K, V, out, lse, (float *)ws, (cudaStream_t)stream) == cudaSuccess ? MOA_OK
+                                                                                                             : MOA_ERR_CUDA;
+}
+
 moa_status moa_last_device_status(void *stream)
 {
     if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return MOA_ERR_CUDA;

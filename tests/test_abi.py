@@ -119,3 +119,16 @@ def test_rowparallel_variant_argument_checks(lib):
     assert need == 4 * 256 * 4 + 2 * 4 * 256 * 64 * 4          # D + two fp32 accumulators (bf16 tensors)
     d32 = mb.make_desc(1, 4, 256, 64, True, 0.1, mb.MOA_F32)
     assert mb.moa_attn_workspace_bytes(d32, mb.MOA_OP_ROWPARALLEL) == 4 * 256 * 4
+
+
+def test_decode_argument_checks(lib):
+    a = 4096
+    call = lambda d, wsb=1 << 40: mb.moa_decode_attn(d, a, a, a, a, a, a, ws_bytes=wsb, check=False)
+    assert ctypes.sizeof(mb.moa_decode_desc) == 28
+    assert call(mb.make_decode_desc(1, 8, 1024, 128, 0.1, H_kv=3)) == mb.MOA_ERR_INVALID_ARG
+    assert call(mb.make_decode_desc(1, 8, 0, 128, 0.1)) == mb.MOA_ERR_INVALID_ARG
+    assert call(mb.make_decode_desc(1, 8, 1024, 96, 0.1)) == mb.MOA_ERR_UNSUPPORTED
+    d = mb.make_decode_desc(2, 8, 100000, 128, 0.1, H_kv=2)
+    need = mb.moa_decode_workspace_bytes(d)
+    assert 0 < need <= 1024 * 2 * 8 * 130 * 4                 # segments x heads x (d + 2) floats: independent of n beyond the cap
+    assert call(d, wsb=need - 1) == mb.MOA_ERR_WORKSPACE
