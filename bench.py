@@ -192,6 +192,117 @@ def workload_config(w, args):
             "parallelism": f"independent (b,h) shards x{args.gpus}"}
 
 
+# ---------------------------------------------------------------------------- decode
+DECODE_WORKLOADS = {
+    # name: (B, H, H_kv, n, d, dtype)
+    "decode_gqa_n32768": (8, 32, 8, 32768, 128, "bf16"),       # 1.07 GB of cache, groups of 4 query heads
+    "decode_mha_n8192": (16, 32, 32, 8192, 128, "bf16"),       # 2.15 GB, one K/V head per query head
+    "decode_paper_n1m": (1, 1, 1, 1048576, 64, "f32"),         # the paper's largest cache, its fp32, one head: 0.54 GB
+}
+
+
+def run_decode(args):
+    """Decode attention (one query per head over a resident K/V cache): a second bench line, not the
+    contract's default.  The path is HBM-bound, so the roofline entry is achieved GB/s of the
+    algorithmic bytes (the cache, read once, plus q and out) against the measured copy bandwidth."""
+    import numpy as np
+    import torch
+    from paper_2609_33916_b200 import binding as mb
+    from paper_2609_33916_b200 import build as mbuild
+    import oracle
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    B, H, Hkv, n, d, dtype = DECODE_WORKLOADS[args.decode]
+    mbuild.build()
+    mb.lib()
+    peaks, peaks_kind = load_peaks()
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    gen = torch.Generator(device="cuda").manual_seed(11)
+    q = torch.randn((B, H, d), generator=gen, device="cuda").to(tdt)
+    K = torch.randn((B, Hkv, n, d), generator=gen, device="cuda").to(tdt)
+    V = torch.randn((B, Hkv, n, d), generator=gen, device="cuda").to(tdt)
+    out = torch.empty((B, H, d), dtype=tdt, device="cuda")
+    lse = torch.empty((B, H), dtype=torch.float32, device="cuda")
+    scale = 1.0 / math.sqrt(d)
+    desc = mb.make_decode_desc(B, H, n, d, scale, mb.MOA_BF16 if dtype == "bf16" else mb.MOA_F32, H_kv=Hkv)
+    ws = torch.empty(max(mb.moa_decode_workspace_bytes(desc), 16), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    esz = 2 if dtype == "bf16" else 4
+    alg_bytes = 2.0 * B * Hkv * n * d * esz + 2.0 * B * H * d * esz + 4.0 * B * H
+
+    def step():
+        mb.moa_decode_attn(desc, q, K, V, out, lse, ws, stream)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(physical_gpu_index(0))
+    sampler.start()
+    l0 = mb.moa_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    sampler.stop()
+    launches = mb.moa_launch_count() - l0
+    ms = e0.elapsed_time(e1) / args.steps
+    gbs = alg_bytes / (ms * 1e-3) / 1e9
+    # end to end: the cache stays on the device (it is the state of a running decode); the new
+    # query comes from pinned host memory and the result goes back, every step
+    hq = q.cpu().pin_memory()
+    hout = torch.empty((B, H, d), dtype=tdt).pin_memory()
+    t0e, t1e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0e.record(stream)
+    for _ in range(args.steps):
+        q.copy_(hq, non_blocking=True)
+        step()
+        hout.copy_(out, non_blocking=True)
+    t1e.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = t0e.elapsed_time(t1e) / args.steps
+    st = mb.moa_last_device_status(stream)
+    if st != mb.MOA_OK:
+        raise SystemExit(f"device status: {mb.status_string(st)}")
+    line = {
+        "metric": "decode attention: GB/s of K/V cache read (one query per head)", "value": gbs, "unit": "GB/s",
+        "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": dtype, "data": "synthetic",
+        "config": {"workload": args.decode, "B": B, "H": H, "H_kv": Hkv, "n": n, "d": d, "scale": "1/sqrt(d)",
+                   "l2": "the cache of one step exceeds the 126 MB L2; no explicit flush"},
+        "tokens_per_s": B / (ms * 1e-3),
+        "clocks": sampler.summary(),
+        "e2e": {"value": alg_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "h2d_bytes_per_step": B * H * d * esz,
+                "d2h_bytes_per_step": B * H * d * esz, "ms_per_step": e2e_ms,
+                "how": "cache resident on the device; the step's query comes from pinned host memory and its output goes back"},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "kernel": "decode_split_kernel", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                     "peak_source": f"{peaks_kind} hbm_gbs (copy bandwidth)",
+                     "algorithmic_bytes_per_step": alg_bytes},
+    }
+    if not args.no_cpu_baseline:
+        heads = min(B * H, 4)
+        hb = min(B, max(1, heads // H)) if H <= heads else 1
+        qs = q[:hb, :heads].float().cpu().numpy().astype(np.float64)
+        ks = K[:hb, :max(1, heads * Hkv // H)].float().cpu().numpy().astype(np.float64)
+        vs = V[:hb, :max(1, heads * Hkv // H)].float().cpu().numpy().astype(np.float64)
+        t0 = time.perf_counter()
+        reps = 0
+        while time.perf_counter() - t0 < 5.0:
+            oracle.decode_attn(qs, ks, vs, scale)
+            reps += 1
+        dt = (time.perf_counter() - t0) / reps
+        sample_bytes = 2.0 * ks.shape[0] * ks.shape[1] * n * d * esz
+        line["cpu_baseline"] = {"value": sample_bytes / dt / 1e9, "unit": "GB/s", "cores": os.cpu_count(), "kind": "oracle",
+                                "sample": f"{qs.shape[0]}x{qs.shape[1]} query heads over {ks.shape[1]} K/V head(s), numpy fp64",
+                                "seconds": dt * reps}
+    print(json.dumps(line))
+    return 0
+
+
 # ----------------------------------------------------------------------------- sweep
 def run_sweep(args):
     """Config-5 style sweep: for each n and each strategy (the three dQ modes of the fused path
@@ -279,6 +390,8 @@ def main():
     ap.add_argument("--path", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--materialize", type=int, default=0)
+    ap.add_argument("--decode", default="", choices=[""] + sorted(DECODE_WORKLOADS),
+                    help="time decode attention on that workload instead of the fused forward+backward")
     ap.add_argument("--rowparallel", type=int, default=0,
                     help="1 or 2: time the row-parallel single-kernel comparison variant with that many atomic sites")
     ap.add_argument("--layout", type=int, default=0, help="0: tensors [B,H,n,d] (every named config); 1: [B,n,H,d]")
@@ -292,6 +405,8 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "moa" else args.warmup
 
+    if args.decode:
+        return run_decode(args)
     from paper_2609_33916_b200 import inputs as mi
     w = mi.CONFIGS[args.workload]
     if args.impl == "reference":

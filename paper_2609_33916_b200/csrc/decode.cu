@@ -17,6 +17,7 @@
 //   * at the end the lane groups of a warp, the warps of the CTA (through shared memory) and,
 //     in a second tiny kernel, the CTAs of a head are merged by their running maxima.
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace moa {
 namespace {
@@ -49,71 +50,43 @@ template <> struct Vec16<float> {
     }
 };
 
-// Partial results of one cache segment: for every query head the running maximum m (log2 domain),
-// the sum l of 2^(s - m) and the unnormalised output sum_j 2^(s_j - m) v_j.
-//   part_o [splits][B*H][D], part_ml [splits][B*H][2]
+// The running state of one lane group (the lanes that share rows): per query head of the group the
+// maximum m (log2 domain), the sum l of 2^(s - m) and this lane's E elements of sum_j 2^(s_j - m) v_j.
 template <typename T, int D, int GC>
-__global__ void __launch_bounds__(kThreads)
-decode_split_kernel(const T *__restrict__ q, const T *__restrict__ K, const T *__restrict__ V,
-                    float *__restrict__ part_o, float *__restrict__ part_ml,
-                    int n, int H, int Hkv, int group, int splits, int keys_per_split, size_t BH, float scale_log2)
-{
-    constexpr int E = Vec16<T>::kElems;      // elements per lane
-    constexpr int LPR = D / E;               // lanes per row
-    constexpr int RPW = 32 / LPR;            // rows per warp-wide load
+struct DecodeState {
+    static constexpr int E = Vec16<T>::kElems;      // elements per lane
+    static constexpr int LPR = D / E;               // lanes per row
+    static constexpr int RPW = 32 / LPR;            // rows per warp-wide access
     static_assert(LPR >= 1 && LPR <= 32 && 32 % LPR == 0, "row must map onto a warp");
-    const int split = blockIdx.x % splits;
-    const int bkv = blockIdx.x / splits;                 // b * Hkv + kv head
-    const int g0 = blockIdx.y * GC;                      // first query head of the group handled here
-    const int gcount = min(GC, group - g0);
-    const int b = bkv / Hkv, kvh = bkv - b * Hkv;
-    const int hq0 = kvh * group + g0;                    // first query head (within the batch element)
-    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-    const int sub = lane / LPR, l = lane % LPR;          // row of the group, lane of the row
-    const T *Kh = K + (size_t)bkv * n * D;
-    const T *Vh = V + (size_t)bkv * n * D;
-    const int k_begin = split * keys_per_split, k_end = min(n, k_begin + keys_per_split);
+    float qv[GC][E], m[GC], lsum[GC], acc[GC][E];
 
-    // this lane's elements of every query of the group, pre-scaled
-    float qv[GC][E];
+    // this lane's elements of every query of the group, pre-multiplied by scale * log2 e
+    __device__ void init(const T *q_first, int gcount, int l, float scale_log2)
+    {
 #pragma unroll
-    for (int g = 0; g < GC; ++g) {
-        float f[E];
-        if (g < gcount) {
-            const uint4 raw = *reinterpret_cast<const uint4 *>(q + ((size_t)b * H + hq0 + g) * D + l * E);
-            Vec16<T>::unpack(raw, f);
-        } else {
+        for (int g = 0; g < GC; ++g) {
+            float f[E];
+            if (g < gcount) {
+                Vec16<T>::unpack(*reinterpret_cast<const uint4 *>(q_first + (size_t)g * D + l * E), f);
+            } else {
 #pragma unroll
-            for (int e = 0; e < E; ++e) f[e] = 0.f;
+                for (int e = 0; e < E; ++e) f[e] = 0.f;
+            }
+#pragma unroll
+            for (int e = 0; e < E; ++e) { qv[g][e] = f[e] * scale_log2; acc[g][e] = 0.f; }
+            m[g] = -INFINITY;
+            lsum[g] = 0.f;
         }
-#pragma unroll
-        for (int e = 0; e < E; ++e) qv[g][e] = f[e] * scale_log2;
     }
 
-    float m[GC], lsum[GC], acc[GC][E];
+    // U rows (one per lane group each): scores by per-lane partial dots and a butterfly over the lanes of
+    // the row, one online-softmax step over the U rows, then out += p * v on the lane's own elements
+    template <int U>
+    __device__ void consume(const uint4 (&kraw)[U], const uint4 (&vraw)[U], const bool (&live)[U])
+    {
+        float s[U][GC];
 #pragma unroll
-    for (int g = 0; g < GC; ++g) {
-        m[g] = -INFINITY;
-        lsum[g] = 0.f;
-#pragma unroll
-        for (int e = 0; e < E; ++e) acc[g][e] = 0.f;
-    }
-
-    constexpr int kRowsPerIter = kUnroll * RPW;          // rows one warp consumes per iteration
-    for (int base = k_begin + warp * kRowsPerIter; base < k_end; base += kWarps * kRowsPerIter) {
-        uint4 kraw[kUnroll], vraw[kUnroll];
-        bool live[kUnroll];
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const int row = base + u * RPW + sub;
-            live[u] = row < k_end;
-            const size_t off = (size_t)(live[u] ? row : k_begin) * D + l * E;
-            kraw[u] = __ldcs(reinterpret_cast<const uint4 *>(Kh + off));
-            vraw[u] = __ldcs(reinterpret_cast<const uint4 *>(Vh + off));
-        }
-        float s[kUnroll][GC];
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
+        for (int u = 0; u < U; ++u) {
             float kf[E];
             Vec16<T>::unpack(kraw[u], kf);
 #pragma unroll
@@ -130,7 +103,7 @@ decode_split_kernel(const T *__restrict__ q, const T *__restrict__ K, const T *_
         for (int g = 0; g < GC; ++g) {
             float mx = m[g];
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) mx = fmaxf(mx, s[u][g]);
+            for (int u = 0; u < U; ++u) mx = fmaxf(mx, s[u][g]);
             const float ref = (mx == -INFINITY) ? 0.f : mx;      // nothing visible yet: any finite reference
             const float alpha = exp2f(m[g] - ref);
             m[g] = mx;
@@ -138,10 +111,10 @@ decode_split_kernel(const T *__restrict__ q, const T *__restrict__ K, const T *_
 #pragma unroll
             for (int e = 0; e < E; ++e) acc[g][e] *= alpha;
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) s[u][g] = exp2f(s[u][g] - ref);     // now the weight p
+            for (int u = 0; u < U; ++u) s[u][g] = exp2f(s[u][g] - ref);     // now the weight p
         }
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
+        for (int u = 0; u < U; ++u) {
             float vf[E];
             Vec16<T>::unpack(vraw[u], vf);
 #pragma unroll
@@ -153,59 +126,201 @@ decode_split_kernel(const T *__restrict__ q, const T *__restrict__ K, const T *_
         }
     }
 
-    // ---- merge the RPW lane groups of the warp (same elements, different rows)
+    // Merge the lane groups of the warp, then the warps of the CTA through `sm` ([warp][g][D + 2]
+    // floats), and write this segment's partial result: part_o [splits][B*H][D], part_ml [splits][B*H][2].
+    __device__ void finish(float *sm, int warp, int lane, int nwarps, int gcount, size_t head0, int split, size_t BH,
+                           float *part_o, float *part_ml, int nthreads)
+    {
+        const int sub = lane / LPR, l = lane % LPR;
 #pragma unroll
-    for (int o = LPR; o < 32; o <<= 1) {
+        for (int o = LPR; o < 32; o <<= 1) {
 #pragma unroll
-        for (int g = 0; g < GC; ++g) {
-            const float mo = __shfl_xor_sync(0xffffffffu, m[g], o);
-            const float lo = __shfl_xor_sync(0xffffffffu, lsum[g], o);
-            const float mx = fmaxf(m[g], mo);
-            const float ref = (mx == -INFINITY) ? 0.f : mx;
-            const float a = exp2f(m[g] - ref), bo = exp2f(mo - ref);
-            lsum[g] = lsum[g] * a + lo * bo;
+            for (int g = 0; g < GC; ++g) {
+                const float mo = __shfl_xor_sync(0xffffffffu, m[g], o);
+                const float lo = __shfl_xor_sync(0xffffffffu, lsum[g], o);
+                const float mx = fmaxf(m[g], mo);
+                const float ref = (mx == -INFINITY) ? 0.f : mx;
+                const float a = exp2f(m[g] - ref), bo = exp2f(mo - ref);
+                lsum[g] = lsum[g] * a + lo * bo;
 #pragma unroll
-            for (int e = 0; e < E; ++e) {
-                const float ao = __shfl_xor_sync(0xffffffffu, acc[g][e], o);
-                acc[g][e] = acc[g][e] * a + ao * bo;
+                for (int e = 0; e < E; ++e) {
+                    const float ao = __shfl_xor_sync(0xffffffffu, acc[g][e], o);
+                    acc[g][e] = acc[g][e] * a + ao * bo;
+                }
+                m[g] = mx;
             }
-            m[g] = mx;
+        }
+        constexpr int kStride = D + 2;
+        if (warp < nwarps && sub == 0) {
+#pragma unroll
+            for (int g = 0; g < GC; ++g) {
+                float *dst = sm + (warp * GC + g) * kStride;
+#pragma unroll
+                for (int e = 0; e < E; ++e) dst[l * E + e] = acc[g][e];
+                if (l == 0) { dst[D] = m[g]; dst[D + 1] = lsum[g]; }
+            }
+        }
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < gcount * D; idx += nthreads) {
+            const int g = idx / D, c = idx - g * D;
+            float mx = -INFINITY;
+            for (int w = 0; w < nwarps; ++w) mx = fmaxf(mx, sm[(w * GC + g) * kStride + D]);
+            const float ref = (mx == -INFINITY) ? 0.f : mx;
+            float o = 0.f, ls = 0.f;
+            for (int w = 0; w < nwarps; ++w) {
+                const float *src = sm + (w * GC + g) * kStride;
+                const float a = exp2f(src[D] - ref);
+                o = fmaf(src[c], a, o);
+                ls = fmaf(src[D + 1], a, ls);
+            }
+            const size_t at = (size_t)split * BH + head0 + g;
+            part_o[at * D + c] = o;
+            if (c == 0) { part_ml[at * 2] = mx; part_ml[at * 2 + 1] = ls; }
         }
     }
-    // ---- merge the warps through shared memory: [warp][g][D + 2]
-    extern __shared__ float sm[];
-    constexpr int kStride = D + 2;
-    if (sub == 0) {
+};
+
+// Where a CTA works: K/V head, the query heads of its group it serves, its segment of the cache.
+struct DecodeJob {
+    int split, bkv, g0, gcount, b, kvh, k_begin, k_end;
+    size_t head0;      // flat index b * H + first query head
+    __device__ DecodeJob(int splits, int GC, int group, int H, int Hkv, int n, int keys_per_split)
+    {
+        split = blockIdx.x % splits;
+        bkv = blockIdx.x / splits;
+        g0 = blockIdx.y * GC;
+        gcount = min(GC, group - g0);
+        b = bkv / Hkv;
+        kvh = bkv - b * Hkv;
+        head0 = (size_t)b * H + kvh * group + g0;
+        k_begin = split * keys_per_split;
+        k_end = min(n, k_begin + keys_per_split);
+    }
+};
+
+// ---- variant 1: rows straight from global memory into registers (16-byte streaming loads, kUnroll row
+// groups of K and of V in flight per warp).  Few registers when the group is small, so several CTAs
+// per SM keep enough bytes in flight: used for one or two query heads per K/V head.
+template <typename T, int D, int GC>
+__global__ void __launch_bounds__(kThreads)
+decode_split_kernel(const T *__restrict__ q, const T *__restrict__ K, const T *__restrict__ V,
+                    float *__restrict__ part_o, float *__restrict__ part_ml,
+                    int n, int H, int Hkv, int group, int splits, int keys_per_split, size_t BH, float scale_log2)
+{
+    using State = DecodeState<T, D, GC>;
+    constexpr int E = State::E, LPR = State::LPR, RPW = State::RPW;
+    const DecodeJob job(splits, GC, group, H, Hkv, n, keys_per_split);
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int sub = lane / LPR, l = lane % LPR;          // row of the group, lane of the row
+    const T *Kh = K + (size_t)job.bkv * n * D;
+    const T *Vh = V + (size_t)job.bkv * n * D;
+    State st;
+    st.init(q + job.head0 * D, job.gcount, l, scale_log2);
+    constexpr int kRowsPerIter = kUnroll * RPW;          // rows one warp consumes per iteration
+    for (int base = job.k_begin + warp * kRowsPerIter; base < job.k_end; base += kWarps * kRowsPerIter) {
+        uint4 kraw[kUnroll], vraw[kUnroll];
+        bool live[kUnroll];
 #pragma unroll
-        for (int g = 0; g < GC; ++g) {
-            float *dst = sm + (warp * GC + g) * kStride;
-#pragma unroll
-            for (int e = 0; e < E; ++e) dst[l * E + e] = acc[g][e];
-            if (l == 0) { dst[D] = m[g]; dst[D + 1] = lsum[g]; }
+        for (int u = 0; u < kUnroll; ++u) {
+            const int row = base + u * RPW + sub;
+            live[u] = row < job.k_end;
+            const size_t off = (size_t)(live[u] ? row : job.k_begin) * D + l * E;
+            kraw[u] = __ldcs(reinterpret_cast<const uint4 *>(Kh + off));
+            vraw[u] = __ldcs(reinterpret_cast<const uint4 *>(Vh + off));
         }
+        st.template consume<kUnroll>(kraw, vraw, live);
+    }
+    extern __shared__ float sm[];
+    st.finish(sm, warp, lane, kWarps, job.gcount, job.head0, job.split, BH, part_o, part_ml, kThreads);
+}
+
+// ---- variant 2: the cache segment streams through a shared-memory ring filled by bulk copies (a tile
+// of 64 rows of one head is contiguous in memory: one copy per tile and tensor), so the bytes in
+// flight are the whole ring whatever the register budget of the consumers: used for groups of four or
+// more query heads, whose state (GC x E accumulators and queries per lane) leaves one or two CTAs per SM.
+// Warp 8 produces; warps 0-7 each consume 8 rows of every tile.  Every wait is bounded.
+constexpr int kRingThreads = kThreads + 32;
+constexpr int kTileRows = 64;
+// K and V tile per stage; about 190 KB of ring, eight stages at most
+template <typename T, int D>
+struct Ring {
+    static constexpr int kFit = (190 * 1024) / (2 * kTileRows * D * (int)sizeof(T));
+    static constexpr int kStages = kFit > 8 ? 8 : kFit;
+};
+
+template <typename T, int D, int GC>
+__global__ void __launch_bounds__(kRingThreads, 1)
+decode_ring_kernel(const T *__restrict__ q, const T *__restrict__ K, const T *__restrict__ V,
+                   float *__restrict__ part_o, float *__restrict__ part_ml,
+                   int n, int H, int Hkv, int group, int splits, int keys_per_split, size_t BH, float scale_log2,
+                   unsigned int *status)
+{
+    using namespace ptx;
+    using State = DecodeState<T, D, GC>;
+    constexpr int E = State::E, LPR = State::LPR, RPW = State::RPW;
+    constexpr int kStages = Ring<T, D>::kStages;
+    constexpr int kRowBytes = D * (int)sizeof(T), kTileBytes = kTileRows * kRowBytes;
+    constexpr int U = (kTileRows / kWarps) / RPW;         // row groups per warp and tile
+    static_assert(U >= 1, "a warp consumes at least one row group per tile");
+    extern __shared__ __align__(128) uint8_t ring[];
+    uint64_t *full = reinterpret_cast<uint64_t *>(ring + (size_t)kStages * 2 * kTileBytes);
+    uint64_t *empty = full + kStages;
+    volatile uint32_t *abortp = reinterpret_cast<uint32_t *>(empty + kStages);
+
+    const DecodeJob job(splits, GC, group, H, Hkv, n, keys_per_split);
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int ntiles = job.k_end > job.k_begin ? (job.k_end - job.k_begin + kTileRows - 1) / kTileRows : 0;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, kWarps); }
+        *abortp = 0;
+        fence_mbar_init();
     }
     __syncthreads();
-    for (int idx = threadIdx.x; idx < gcount * D; idx += kThreads) {
-        const int g = idx / D, c = idx - g * D;
-        float mx = -INFINITY;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) mx = fmaxf(mx, sm[(w * GC + g) * kStride + D]);
-        const float ref = (mx == -INFINITY) ? 0.f : mx;
-        float o = 0.f, ls = 0.f;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) {
-            const float *src = sm + (w * GC + g) * kStride;
-            const float a = exp2f(src[D] - ref);
-            o = fmaf(src[c], a, o);
-            ls = fmaf(src[D + 1], a, ls);
+    State st;
+    if (warp == kWarps) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            const uint8_t *Kh = reinterpret_cast<const uint8_t *>(K) + ((size_t)job.bkv * n + job.k_begin) * kRowBytes;
+            const uint8_t *Vh = reinterpret_cast<const uint8_t *>(V) + ((size_t)job.bkv * n + job.k_begin) * kRowBytes;
+            for (int t = 0; t < ntiles; ++t) {
+                const int s = t % kStages;
+                if (t >= kStages && !mbar_wait(empty + s, (t / kStages - 1) & 1, abortp, status, 0x301u)) break;
+                const int rows = min(kTileRows, job.k_end - job.k_begin - t * kTileRows);
+                const uint32_t bytes = (uint32_t)rows * kRowBytes;
+                mbar_arrive_expect_tx(full + s, 2 * bytes);
+                bulk_load_1d(ring + (size_t)s * 2 * kTileBytes, Kh + (size_t)t * kTileBytes, bytes, full + s);
+                bulk_load_1d(ring + (size_t)s * 2 * kTileBytes + kTileBytes, Vh + (size_t)t * kTileBytes, bytes, full + s);
+            }
         }
-        const size_t head = (size_t)b * H + hq0 + g;
-        part_o[((size_t)split * BH + head) * D + c] = o;
-        if (c == 0) {
-            part_ml[((size_t)split * BH + head) * 2] = mx;
-            part_ml[((size_t)split * BH + head) * 2 + 1] = ls;
+    } else {
+        // ----------------------------------------------------------------- consumers
+        const int sub = lane / LPR, l = lane % LPR;
+        st.init(q + job.head0 * D, job.gcount, l, scale_log2);
+        for (int t = 0; t < ntiles; ++t) {
+            const int s = t % kStages;
+            if (!mbar_wait(full + s, (t / kStages) & 1, abortp, status, 0x302u)) break;
+            const uint8_t *tk = ring + (size_t)s * 2 * kTileBytes, *tv = tk + kTileBytes;
+            const int row0 = job.k_begin + t * kTileRows;
+            uint4 kraw[U], vraw[U];
+            bool live[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int r = warp * (kTileRows / kWarps) + u * RPW + sub;      // row of the tile
+                live[u] = row0 + r < job.k_end;
+                // rows past the segment were not copied: read row 0 of the tile instead (always present)
+                const int rr = live[u] ? r : 0;
+                kraw[u] = *reinterpret_cast<const uint4 *>(tk + rr * kRowBytes + l * 16);
+                vraw[u] = *reinterpret_cast<const uint4 *>(tv + rr * kRowBytes + l * 16);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty + s);      // the tile is in registers: the stage may be refilled
+            st.template consume<U>(kraw, vraw, live);
         }
     }
+    __syncthreads();       // every consumer is done with the ring: reuse its start for the merge
+    if (warp == kWarps) st.init(q + job.head0 * D, 0, 0, 0.f);     // the producer warp holds no state
+    st.finish(reinterpret_cast<float *>(ring), warp, lane, kWarps, job.gcount, job.head0, job.split, BH, part_o,
+              part_ml, kRingThreads);
 }
 
 // One block per query head: merge the segments, normalise, write out (and the natural-log lse).
@@ -234,14 +349,26 @@ cudaError_t launch_split(const DecodeProblem &p, const void *q, const void *K, c
                          float *part_ml, int splits, int keys_per_split, cudaStream_t st)
 {
     const int group = p.H / p.Hkv;
-    const size_t smem = (size_t)kWarps * GC * (D + 2) * sizeof(float);
-    cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<T, D, GC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
     dim3 grid((unsigned)(p.B * p.Hkv * splits), (unsigned)((group + GC - 1) / GC));
+    const size_t merge_smem = (size_t)kWarps * GC * (D + 2) * sizeof(float);
     LaunchScope scope(MOA_KERNEL_OTHER, st);
-    decode_split_kernel<T, D, GC><<<grid, kThreads, smem, st>>>((const T *)q, (const T *)K, (const T *)V, part_o, part_ml,
-                                                                p.n, p.H, p.Hkv, group, splits, keys_per_split,
-                                                                (size_t)p.B * p.H, p.scale * kLog2e);
+    if (GC >= 4) {
+        constexpr int kStages = Ring<T, D>::kStages;
+        const size_t smem = (size_t)kStages * 2 * kTileRows * D * sizeof(T) + 2 * kStages * sizeof(uint64_t) + 16;
+        cudaError_t e = cudaFuncSetAttribute(decode_ring_kernel<T, D, GC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)(smem > merge_smem ? smem : merge_smem));
+        if (e != cudaSuccess) return e;
+        decode_ring_kernel<T, D, GC><<<grid, kRingThreads, smem > merge_smem ? smem : merge_smem, st>>>(
+            (const T *)q, (const T *)K, (const T *)V, part_o, part_ml, p.n, p.H, p.Hkv, group, splits, keys_per_split,
+            (size_t)p.B * p.H, p.scale * kLog2e, device_status_ptr());
+        return cudaGetLastError();
+    }
+    cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<T, D, GC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)merge_smem);
+    if (e != cudaSuccess) return e;
+    decode_split_kernel<T, D, GC><<<grid, kThreads, merge_smem, st>>>((const T *)q, (const T *)K, (const T *)V, part_o,
+                                                                      part_ml, p.n, p.H, p.Hkv, group, splits,
+                                                                      keys_per_split, (size_t)p.B * p.H, p.scale * kLog2e);
     return cudaGetLastError();
 }
 
