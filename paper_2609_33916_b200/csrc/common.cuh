@@ -49,16 +49,21 @@ inline int heads_per_group(const Problem &p, int tiles)
     return (int)g;
 }
 
+// Decode through the tensor-core forward kernel (tc_fwd.cu): the G query heads of a K/V head are
+// the rows of one query tile, the cache is split among CTAs; partial results to be merged.
+cudaError_t tc_fwd_decode(int B, int Hkv, int G, int n, int d, float scale, const void *q, const void *K, const void *V,
+                          void *O_part, float *L_part, int splits, int tiles_per_split, cudaStream_t st);
+
 // ---- decode attention (decode.cu) ----------------------------------------------------
 struct DecodeProblem {
     int B, H, Hkv, n, d;     // Hkv resolved (never 0)
     float scale;
 };
-int decode_splits(const DecodeProblem &p);                  // cache segments per K/V head
-size_t decode_workspace_floats(const DecodeProblem &p);     // partial outputs, maxima and sums of all segments
+int decode_splits(const DecodeProblem &p);                            // cache segments per K/V head (CUDA-core route)
+size_t decode_workspace_bytes(const DecodeProblem &p, int dtype);    // partial results of all segments
 // q [B,H,d], K, V [B,Hkv,n,d] -> out [B,H,d] (dtype of the inputs), lse [B,H] fp32 (may be null)
 cudaError_t decode_attn(const DecodeProblem &p, int dtype, const void *q, const void *K, const void *V, void *out,
-                        float *lse, float *ws, cudaStream_t st);
+                        float *lse, void *ws, cudaStream_t st);
 
 // Host-side launch counter (moa_launch_count).
 void count_launch(int k = 1);

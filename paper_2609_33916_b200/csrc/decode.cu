@@ -324,22 +324,86 @@ decode_ring_kernel(const T *__restrict__ q, const T *__restrict__ K, const T *__
 }
 
 // One block per query head: merge the segments, normalise, write out (and the natural-log lse).
+// 256 threads: thread = (stripe of segments, output column); the stripes are merged in shared memory.
 template <typename T, int D>
-__global__ void decode_merge_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml,
-                                    T *__restrict__ out, float *__restrict__ lse, int splits, size_t BH)
+__global__ void __launch_bounds__(256)
+decode_merge_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml,
+                    T *__restrict__ out, float *__restrict__ lse, int splits, size_t BH)
 {
+    constexpr int kStripes = 256 / D;
+    __shared__ float sh_o[kStripes][D], sh_m[kStripes], sh_l[kStripes];
     const size_t head = blockIdx.x;
-    const int c = threadIdx.x;
-    float mx = -INFINITY;
-    for (int s = 0; s < splits; ++s) mx = fmaxf(mx, part_ml[((size_t)s * BH + head) * 2]);
-    float o = 0.f, ls = 0.f;
-    for (int s = 0; s < splits; ++s) {
-        const float a = exp2f(part_ml[((size_t)s * BH + head) * 2] - mx);
-        o = fmaf(part_o[((size_t)s * BH + head) * D + c], a, o);
-        ls = fmaf(part_ml[((size_t)s * BH + head) * 2 + 1], a, ls);
+    const int c = threadIdx.x % D, stripe = threadIdx.x / D;
+    float mx = -INFINITY, o = 0.f, ls = 0.f;
+    for (int s = stripe; s < splits; s += kStripes) {
+        const size_t at = (size_t)s * BH + head;
+        const float ms = part_ml[at * 2];
+        const float mn = fmaxf(mx, ms);
+        const float ref = (mn == -INFINITY) ? 0.f : mn;
+        const float a = exp2f(mx - ref), b = exp2f(ms - ref);
+        o = o * a + part_o[at * D + c] * b;
+        ls = ls * a + part_ml[at * 2 + 1] * b;
+        mx = mn;
     }
-    out[head * D + c] = from_float<T>(o / ls);
-    if (lse && c == 0) lse[head] = (mx + log2f(ls)) * kLn2;
+    sh_o[stripe][c] = o;
+    if (c == 0) { sh_m[stripe] = mx; sh_l[stripe] = ls; }
+    __syncthreads();
+    if (stripe == 0) {
+        float mt = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < kStripes; ++k) mt = fmaxf(mt, sh_m[k]);
+        float ot = 0.f, lt = 0.f;
+#pragma unroll
+        for (int k = 0; k < kStripes; ++k) {
+            const float a = exp2f(sh_m[k] - mt);
+            ot = fmaf(sh_o[k][c], a, ot);
+            lt = fmaf(sh_l[k], a, lt);
+        }
+        out[head * D + c] = from_float<T>(ot / lt);
+        if (lse && c == 0) lse[head] = (mt + log2f(lt)) * kLn2;
+    }
+}
+
+// Merge for the tensor-core route: O_part [splits*B, Hkv, G, D] bf16 (each normalised over its own
+// segment), L_part [splits, B*Hkv, G] natural-log logsumexp of the segment.  One block per query head.
+template <int D>
+__global__ void __launch_bounds__(256)
+decode_merge_tc_kernel(const __nv_bfloat16 *__restrict__ O_part, const float *__restrict__ L_part,
+                       __nv_bfloat16 *__restrict__ out, float *__restrict__ lse, int splits, int B, int Hkv, int G)
+{
+    constexpr int kStripes = 256 / D;
+    __shared__ float sh_o[kStripes][D], sh_m[kStripes], sh_l[kStripes];
+    const int head = blockIdx.x;                      // b * H + kvh * G + g
+    const int H = Hkv * G;
+    const int b = head / H, hq = head - b * H, kvh = hq / G, g = hq - kvh * G;
+    const int c = threadIdx.x % D, stripe = threadIdx.x / D;
+    float mx = -INFINITY, o = 0.f, ls = 0.f;          // running max of L, sum of weights, weighted output
+    for (int s = stripe; s < splits; s += kStripes) {
+        const float Ls = L_part[((size_t)s * B * Hkv + (size_t)b * Hkv + kvh) * G + g];
+        const float mn = fmaxf(mx, Ls);
+        const float a = __expf(mx - mn), w = __expf(Ls - mn);
+        const float ov = __bfloat162float(O_part[((((size_t)s * B + b) * Hkv + kvh) * G + g) * D + c]);
+        o = o * a + ov * w;
+        ls = ls * a + w;
+        mx = mn;
+    }
+    sh_o[stripe][c] = o;
+    if (c == 0) { sh_m[stripe] = mx; sh_l[stripe] = ls; }
+    __syncthreads();
+    if (stripe == 0) {
+        float mt = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < kStripes; ++k) mt = fmaxf(mt, sh_m[k]);
+        float ot = 0.f, lt = 0.f;
+#pragma unroll
+        for (int k = 0; k < kStripes; ++k) {
+            const float a = __expf(sh_m[k] - mt);
+            ot = fmaf(sh_o[k][c], a, ot);
+            lt = fmaf(sh_l[k], a, lt);
+        }
+        out[(size_t)head * D + c] = __float2bfloat16_rn(ot / lt);
+        if (lse && c == 0) lse[head] = mt + __logf(lt);
+    }
 }
 
 int group_chunk(int group) { return group >= 8 ? 8 : group >= 4 ? 4 : group >= 2 ? 2 : 1; }
@@ -387,11 +451,31 @@ cudaError_t launch_decode(const DecodeProblem &p, const void *q, const void *K, 
                             : launch_split<T, D, 1>(p, q, K, V, part_o, part_ml, splits, keys_per_split, st);
     if (e != cudaSuccess) return e;
     LaunchScope scope(MOA_KERNEL_OTHER, st);
-    decode_merge_kernel<T, D><<<(unsigned)BH, D, 0, st>>>(part_o, part_ml, (T *)out, lse, splits, BH);
+    decode_merge_kernel<T, D><<<(unsigned)BH, 256, 0, st>>>(part_o, part_ml, (T *)out, lse, splits, BH);
     return cudaGetLastError();
 }
 
 }  // namespace
+
+// Groups of 4 to 128 query heads over a bf16 cache go through the tensor-core forward kernel (the
+// group is its query tile); everything else through the CUDA-core streaming kernels above.
+static bool decode_uses_tc(const DecodeProblem &p, int dtype)
+{
+    const int group = p.H / p.Hkv;
+    return dtype == MOA_BF16 && group >= 4 && group <= 128 && p.scale > 0.f;
+}
+
+// Tensor-core route: key tiles of 128 per CTA segment, about six CTAs per SM over the run
+static void decode_tc_splits(const DecodeProblem &p, int *splits, int *tiles_per_split)
+{
+    const int nkt = (p.n + 127) / 128;
+    long long s = (6LL * 148 + (long long)p.B * p.Hkv - 1) / ((long long)p.B * p.Hkv);
+    if (s > nkt) s = nkt;
+    if (s < 1) s = 1;
+    const int tps = (int)((nkt + s - 1) / s);
+    *tiles_per_split = tps;
+    *splits = (nkt + tps - 1) / tps;          // every segment has at least one tile
+}
 
 // Segments of the cache per K/V head: enough CTAs to fill the GPU a few times over, each with at
 // least 256 keys.
@@ -408,20 +492,45 @@ int decode_splits(const DecodeProblem &p)
     return (int)s;
 }
 
-size_t decode_workspace_floats(const DecodeProblem &p)
+size_t decode_workspace_bytes(const DecodeProblem &p, int dtype)
 {
-    return (size_t)decode_splits(p) * p.B * p.H * (p.d + 2);
+    if (decode_uses_tc(p, dtype)) {
+        int splits, tps;
+        decode_tc_splits(p, &splits, &tps);
+        const size_t heads = (size_t)splits * p.B * p.H;
+        return ((heads * p.d * 2 + 255) / 256) * 256 + heads * sizeof(float);
+    }
+    return (size_t)decode_splits(p) * p.B * p.H * (p.d + 2) * sizeof(float);
 }
 
 cudaError_t decode_attn(const DecodeProblem &p, int dtype, const void *q, const void *K, const void *V, void *out,
-                        float *lse, float *ws, cudaStream_t st)
+                        float *lse, void *ws, cudaStream_t st)
 {
+    if (decode_uses_tc(p, dtype)) {
+        int splits, tps;
+        decode_tc_splits(p, &splits, &tps);
+        const int G = p.H / p.Hkv;
+        const size_t heads = (size_t)splits * p.B * p.H;
+        void *O_part = ws;
+        float *L_part = reinterpret_cast<float *>((char *)ws + ((heads * p.d * 2 + 255) / 256) * 256);
+        cudaError_t e = tc_fwd_decode(p.B, p.Hkv, G, p.n, p.d, p.scale, q, K, V, O_part, L_part, splits, tps, st);
+        if (e != cudaSuccess) return e;
+        LaunchScope scope(MOA_KERNEL_OTHER, st);
+        if (p.d == 64)
+            decode_merge_tc_kernel<64><<<(unsigned)(p.B * p.H), 256, 0, st>>>((const __nv_bfloat16 *)O_part, L_part,
+                                                                              (__nv_bfloat16 *)out, lse, splits, p.B, p.Hkv, G);
+        else
+            decode_merge_tc_kernel<128><<<(unsigned)(p.B * p.H), 256, 0, st>>>((const __nv_bfloat16 *)O_part, L_part,
+                                                                               (__nv_bfloat16 *)out, lse, splits, p.B, p.Hkv, G);
+        return cudaGetLastError();
+    }
+    float *wsf = (float *)ws;
     if (dtype == MOA_F32) {
-        if (p.d == 64) return launch_decode<float, 64>(p, q, K, V, out, lse, ws, st);
-        if (p.d == 128) return launch_decode<float, 128>(p, q, K, V, out, lse, ws, st);
+        if (p.d == 64) return launch_decode<float, 64>(p, q, K, V, out, lse, wsf, st);
+        if (p.d == 128) return launch_decode<float, 128>(p, q, K, V, out, lse, wsf, st);
     } else {
-        if (p.d == 64) return launch_decode<__nv_bfloat16, 64>(p, q, K, V, out, lse, ws, st);
-        if (p.d == 128) return launch_decode<__nv_bfloat16, 128>(p, q, K, V, out, lse, ws, st);
+        if (p.d == 64) return launch_decode<__nv_bfloat16, 64>(p, q, K, V, out, lse, wsf, st);
+        if (p.d == 128) return launch_decode<__nv_bfloat16, 128>(p, q, K, V, out, lse, wsf, st);
     }
     return cudaErrorInvalidValue;
 }

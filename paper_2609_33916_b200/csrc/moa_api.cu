@@ -440,7 +440,7 @@ size_t moa_decode_workspace_bytes(const moa_decode_desc *desc)
 {
     DecodeProblem p;
     if (check_decode_desc(desc, &p) != MOA_OK) return 0;
-    return decode_workspace_floats(p) * sizeof(float);
+    return decode_workspace_bytes(p, desc->dtype);
 }
 
 moa_status moa_decode_attn(const moa_decode_desc *desc, const void *q, const void *K, const void *V,
@@ -451,10 +451,10 @@ moa_status moa_decode_attn(const moa_decode_desc *desc, const void *q, const voi
     if (s != MOA_OK) return s;
     if (!q || !K || !V || !out) return MOA_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(K) || !aligned16(V) || !aligned16(out) || (lse && !aligned16(lse))) return MOA_ERR_INVALID_ARG;
-    if (!ws || ws_bytes < decode_workspace_floats(p) * sizeof(float)) return MOA_ERR_WORKSPACE;
+    if (!ws || ws_bytes < decode_workspace_bytes(p, desc->dtype)) return MOA_ERR_WORKSPACE;
     if (!aligned16(ws)) return MOA_ERR_INVALID_ARG;
     if ((s = check_arch()) != MOA_OK) return s;
-    return decode_attn(p, desc->dtype, q, K, V, out, lse, (float *)ws, (cudaStream_t)stream) == cudaSuccess ? MOA_OK
+    return decode_attn(p, desc->dtype, q, K, V, out, lse, ws, (cudaStream_t)stream) == cudaSuccess ? MOA_OK
                                                                                                              : MOA_ERR_CUDA;
 }
 

@@ -51,12 +51,21 @@ enum { F_Q = 0, F_KFULL = 1 /*2*/, F_KEMPTY = 3 /*2*/, F_VFULL = 5 /*2*/, F_VEMP
        F_P = 11 /*[buffer][half]: 4*/, F_O = 15, F_X = 16 /*epilogue exchange*/, F_OB = 17 /*2: score buffer consumed*/,
        F_E = 19 /*O tile staged in shared memory*/, F_COUNT = 20 };
 
+// Split use of the kernel (decode: few query rows, a long cache): the key tiles are divided among
+// `splits` CTAs per (head, query tile); each writes the attention over its tiles alone (normalised O
+// and its logsumexp, batch coordinate split * B + b), to be merged by the caller.  n_q: valid query
+// rows of a head (the main path: n_q = n, splits = 1, tiles_per_split = all tiles).
+struct FwdSplit {
+    int n_q, splits, tiles_per_split;
+};
+
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
               const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapO,
               float *__restrict__ L,
-              int n, int causal, float scale_log2, int nqt, int hpg, int group, int H, unsigned int *status)
+              int n, int causal, float scale_log2, int nqt, int hpg, int group, int H, FwdSplit sp,
+              unsigned int *status)
 {
     constexpr int kTileBytes = 128 * D * 2;
     constexpr int kBoxes = D / 64;         // 64-column (128-byte) swizzled boxes per tile
@@ -69,13 +78,16 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
 
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
     int bh, t;
-    job_from_block((int)blockIdx.x, nqt, (int)gridDim.x / nqt, hpg, bh, t);
+    const int split = sp.splits > 1 ? (int)blockIdx.x % sp.splits : 0;
+    const int heads_all = (int)gridDim.x / sp.splits / nqt;
+    job_from_block(sp.splits > 1 ? (int)blockIdx.x / sp.splits : (int)blockIdx.x, nqt, heads_all, hpg, bh, t);
     const int bb = bh / H, hq = bh - bb * H;    // batch and query head: coordinates of the 4-D tensor maps
     const int hk = hq / group;                  // the K/V head this query head reads (group > 1: shared heads)
     const int qt = causal ? nqt - 1 - t : t;   // causal: longest rows first
     const int q0 = qt * BM;
     const int nkt_all = (n + BN - 1) / BN;
-    const int nkt_want = causal ? min(qt + 1, nkt_all) : nkt_all;
+    const int kt0 = split * sp.tiles_per_split;                       // first key tile of this CTA
+    const int nkt_want = causal ? min(qt + 1, nkt_all) : min(sp.tiles_per_split, nkt_all - kt0);
 
     if (tid == 0) {
         for (int b = 0; b < F_COUNT; ++b) mbar_init(bars + b, (b >= F_P && b < F_P + 4) ? 128u : ((b == F_X || b == F_E) ? 256u : 1u));
@@ -103,13 +115,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             if (lane == 0) {
                 mbar_arrive_expect_tx(bars + F_KFULL + s, kTileBytes);
                 for (int b = 0; b < kBoxes; ++b)
-                    tma_load_4d(sK + s * kTileBytes + b * kBoxBytes, &mapK, bars + F_KFULL + s, 64 * b, j * BN, hk, bb);
+                    tma_load_4d(sK + s * kTileBytes + b * kBoxBytes, &mapK, bars + F_KFULL + s, 64 * b, (kt0 + j) * BN, hk, bb);
             }
             if (j >= 2 && !mbar_wait(bars + F_VEMPTY + s, ((j >> 1) - 1) & 1, abortp, status, ERR_V)) break;
             if (lane == 0) {
                 mbar_arrive_expect_tx(bars + F_VFULL + s, kTileBytes);
                 for (int b = 0; b < kBoxes; ++b)
-                    tma_load_4d(sV + s * kTileBytes + b * kBoxBytes, &mapV, bars + F_VFULL + s, 64 * b, j * BN, hk, bb);
+                    tma_load_4d(sV + s * kTileBytes + b * kBoxBytes, &mapV, bars + F_VFULL + s, 64 * b, (kt0 + j) * BN, hk, bb);
             }
             __syncwarp();
         }
@@ -194,7 +206,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             const uint32_t scol = kColS + 128 * (j & 1) + 64 * h;      // this thread's 64 score columns
             if (!mbar_wait(bars + F_S + (j & 1), (j >> 1) & 1, abortp, status, ERR_S)) { ok = false; break; }
             tc_fence_after();
-            const int k0 = j * BN + 64 * h;
+            const int k0 = (kt0 + j) * BN + 64 * h;
             const bool need_mask = (k0 + 64 > n) || (causal && k0 + 63 > q0);
             uint32_t r[2][32];
 #pragma unroll
@@ -312,11 +324,11 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             fence_proxy_async_smem();
             mbar_arrive(bars + F_E);
             if (tid == 0 && mbar_wait(bars + F_E, 0, abortp, status, ERR_O)) {
-                for (int b = 0; b < kBoxes; ++b) tma_store_4d(&mapO, sQ + b * kBoxBytes, 64 * b, q0, hq, bb);
+                for (int b = 0; b < kBoxes; ++b) tma_store_4d(&mapO, sQ + b * kBoxBytes, 64 * b, q0, hq, split * (heads_all / H) + bb);
                 bulk_commit();
                 bulk_wait_read<0>();      // shared memory is read before the CTA may exit
             }
-            if (row < n && h == 0) L[(size_t)bh * n + row] = m_all * kLn2 + logf(l_all);
+            if (row < sp.n_q && h == 0) L[((size_t)split * heads_all + bh) * sp.n_q + row] = m_all * kLn2 + logf(l_all);
         }
     }
     tc_fence_before();
@@ -342,11 +354,45 @@ cudaError_t launch_fwd(const Problem &p, const void *Q, const void *K, const voi
     const int nqt = (p.n + BM - 1) / BM;
     LaunchScope scope(MOA_KERNEL_FWD, st);
     tc_fwd_kernel<D><<<(unsigned)(nqt * p.BH()), kThreads, kSmem, st>>>(
-        mq, mk, mv, mo, L, p.n, p.causal, p.scale * kLog2e, nqt, heads_per_group(p, nqt), p.group(), p.H, device_status_ptr());
+        mq, mk, mv, mo, L, p.n, p.causal, p.scale * kLog2e, nqt, heads_per_group(p, nqt), p.group(), p.H,
+        FwdSplit{p.n, 1, (p.n + BN - 1) / BN}, device_status_ptr());
+    return cudaGetLastError();
+}
+
+// Decode through the forward kernel: the G query heads that share a K/V head are the query rows of
+// one tile (q [B,H,d] read as [B,Hkv,G,d]; rows G..127 are zero fill and are never written), the
+// cache is divided among `splits` CTAs per K/V head.  O_part [splits*B, Hkv, G, d] bf16, L_part
+// [splits, B*Hkv, G] fp32.
+template <int D>
+cudaError_t launch_fwd_decode(int B, int Hkv, int G, int n, float scale, const void *q, const void *K, const void *V,
+                              void *O_part, float *L_part, int splits, int tiles_per_split, cudaStream_t st)
+{
+    constexpr int kSmem = 5 * 128 * D * 2 + 8 * (F_COUNT + 2) + 2 * 128 * 8;
+    CUtensorMap mq, mk, mv, mo;
+    const auto bf = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    if (!make_tensor_map_4d(&mq, q, bf, 2, B, Hkv, G, D, false, 128, 64) ||
+        !make_tensor_map_4d(&mk, K, bf, 2, B, Hkv, n, D, false, 128, 64) ||
+        !make_tensor_map_4d(&mv, V, bf, 2, B, Hkv, n, D, false, 128, 64) ||
+        !make_tensor_map_4d(&mo, O_part, bf, 2, (uint64_t)splits * B, Hkv, G, D, false, 128, 64))
+        return cudaErrorInvalidValue;
+    cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    if (e != cudaSuccess) return e;
+    LaunchScope scope(MOA_KERNEL_FWD, st);
+    tc_fwd_kernel<D><<<(unsigned)(B * Hkv * splits), kThreads, kSmem, st>>>(
+        mq, mk, mv, mo, L_part, n, 0, scale * kLog2e, 1, 1, 1, Hkv, FwdSplit{G, splits, tiles_per_split},
+        device_status_ptr());
     return cudaGetLastError();
 }
 
 }  // namespace
+
+cudaError_t tc_fwd_decode(int B, int Hkv, int G, int n, int d, float scale, const void *q, const void *K, const void *V,
+                          void *O_part, float *L_part, int splits, int tiles_per_split, cudaStream_t st)
+{
+    if (d == 64) return launch_fwd_decode<64>(B, Hkv, G, n, scale, q, K, V, O_part, L_part, splits, tiles_per_split, st);
+    if (d == 128) return launch_fwd_decode<128>(B, Hkv, G, n, scale, q, K, V, O_part, L_part, splits, tiles_per_split, st);
+    return cudaErrorInvalidValue;
+}
 
 cudaError_t tc_fwd(const Problem &p, const void *Q, const void *K, const void *V, void *O, float *L, cudaStream_t st)
 {
