@@ -334,16 +334,18 @@ decode_merge_kernel(const float *__restrict__ part_o, const float *__restrict__ 
     __shared__ float sh_o[kStripes][D], sh_m[kStripes], sh_l[kStripes];
     const size_t head = blockIdx.x;
     const int c = threadIdx.x % D, stripe = threadIdx.x / D;
+    // two passes, so that the loads of a pass do not wait on the running maximum: first the maximum
+    // of the stripe, then the weighted sums
     float mx = -INFINITY, o = 0.f, ls = 0.f;
+#pragma unroll 8
+    for (int s = stripe; s < splits; s += kStripes) mx = fmaxf(mx, part_ml[((size_t)s * BH + head) * 2]);
+    const float ref = (mx == -INFINITY) ? 0.f : mx;
+#pragma unroll 8
     for (int s = stripe; s < splits; s += kStripes) {
         const size_t at = (size_t)s * BH + head;
-        const float ms = part_ml[at * 2];
-        const float mn = fmaxf(mx, ms);
-        const float ref = (mn == -INFINITY) ? 0.f : mn;
-        const float a = exp2f(mx - ref), b = exp2f(ms - ref);
-        o = o * a + part_o[at * D + c] * b;
-        ls = ls * a + part_ml[at * 2 + 1] * b;
-        mx = mn;
+        const float w = exp2f(part_ml[at * 2] - ref);
+        o = fmaf(part_o[at * D + c], w, o);
+        ls = fmaf(part_ml[at * 2 + 1], w, ls);
     }
     sh_o[stripe][c] = o;
     if (c == 0) { sh_m[stripe] = mx; sh_l[stripe] = ls; }
