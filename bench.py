@@ -599,8 +599,8 @@ def main():
     tc_path = args.path in (0, 2)
     peak = peaks["bf16_tflops_sustained"]
     # DRAM bytes per launch of the backward kernel: ncu capture of a small case (B1 H8 n8192 d128:
-    # 124.9 MB read+written over 65536 tokens), scaled by tokens -- traffic is linear in B*H*n
-    traffic = 124.9e6 / 65536.0 * heads * n if (dominant == "bwd_kv" and d == 128) else None
+    # 123.9 MB read+written over 65536 tokens), scaled by tokens -- traffic is linear in B*H*n
+    traffic = 123.9e6 / 65536.0 * heads * n if (dominant == "bwd_kv" and d == 128) else None
     roofline = {"bound": "tensor", "kernel": dominant, "achieved": achieved, "peak": peak,
                 "unit": "TFLOP/s", "frac": (achieved / peak) if achieved else None, "traffic": traffic,
                 "traffic_source": "ncu dram__bytes_read+write of a smaller case, scaled by tokens" if traffic else None,

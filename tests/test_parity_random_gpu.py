@@ -46,3 +46,40 @@ def test_random_case(case):
     got = H.run_library(inp, "bf16", causal, scale, dq_mode=dq, path=path, materialize=mat)
     H.assert_close(got, ref, H.TOL_BF16, tag=str(case))
     assert mi.rel_err(got["L"], ref["L"]) <= 1e-3
+
+
+def _gqa_cases(count, seed):
+    """Tensor-core path only: random shared-K/V-head groupings and both memory layouts."""
+    rng = np.random.default_rng(seed)
+    edge = [1, 64, 127, 128, 129, 255, 256, 257, 384, 385, 513, 640]
+    out = []
+    for i in range(count):
+        n = int(rng.choice(edge)) if rng.random() < 0.7 else int(rng.integers(1, 700))
+        d = int(rng.choice([64, 128]))
+        causal = bool(rng.integers(0, 2))
+        Hkv = int(rng.integers(1, 4))
+        G = int(rng.choice([1, 2, 3, 5]))
+        B = int(rng.integers(1, 3))
+        dq = int(rng.choice([0, 1, 3] if d == 64 else [0, 1, 2, 3]))
+        layout = int(rng.integers(0, 2))
+        op = "split" if rng.random() < 0.3 else "fused"
+        out.append((i, B, Hkv * G, Hkv, n, d, causal, dq, layout, op))
+    return out
+
+
+@pytest.mark.parametrize("case", _gqa_cases(40, 20261126),
+                         ids=lambda c: f"{c[0]}-H{c[2]}kv{c[3]}-n{c[4]}-d{c[5]}-c{int(c[6])}-dq{c[7]}-l{c[8]}-{c[9]}")
+def test_random_grouped_heads_and_layouts(case):
+    import gpu_harness as H
+    from paper_2609_33916_b200 import build as mbuild
+    mbuild.build()
+    i, B, Hq, Hkv, n, d, causal, dq, layout, op = case
+    scale = float(np.random.default_rng(100 + i).uniform(0.5, 1.5)) / math.sqrt(d)
+    q = mi.make_inputs(B, Hq, n, d, seed=9500 + i, dtype="bf16")
+    kv = mi.make_inputs(B, Hkv, n, d, seed=9700 + i, dtype="bf16")
+    inp = {"Q": q["Q"], "dO": q["dO"], "K": kv["K"], "V": kv["V"]}
+    f = {k: mi.to_f64(v, "bf16") for k, v in inp.items()}
+    ref = oracle.attn_fwd_bwd_gqa(f["Q"], f["K"], f["V"], f["dO"], causal, scale)
+    got = H.run_library(inp, "bf16", causal, scale, dq_mode=dq, layout=layout, op=op)
+    H.assert_close(got, ref, H.TOL_BF16, tag=str(case))
+    assert mi.rel_err(got["L"], ref["L"]) <= 1e-3
