@@ -174,8 +174,8 @@ def _sampled_check(H, w, heads, nrows=24, ncols=24, dq_mode=0, path=0):
         # causal: the first rows see few keys and carry the largest dQ of the head, so they belong in
         # the sample that stands in for the tensor-wide max|ref|
         early = [2, 3, 5, 8, 13] if w.causal else []
-        rows = np.unique(np.concatenate([[0, 1, 127, 128, w.n - 1], early, rng.integers(0, w.n, nrows)])).astype(np.int32)
-        cols = np.unique(np.concatenate([[0, 127, 128, w.n - 129, w.n - 1], rng.integers(0, w.n, ncols)])).astype(np.int32)
+        rows = np.unique(np.clip(np.concatenate([[0, 1, 127, 128, w.n - 1], early, rng.integers(0, w.n, nrows)]), 0, w.n - 1)).astype(np.int32)
+        cols = np.unique(np.clip(np.concatenate([[0, 127, 128, w.n - 129, w.n - 1], rng.integers(0, w.n, ncols)]), 0, w.n - 1)).astype(np.int32)
         rr = oracle.attn_rows(f["Q"], f["K"], f["V"], f["dO"], w.causal, w.scale, rows)
         cc = oracle.attn_cols(f["Q"], f["K"], f["V"], f["dO"], w.causal, w.scale, cols)
         # the denominator is the tensor-wide max|ref|; approximate it from below by the sampled
@@ -312,6 +312,23 @@ def test_bnhd_layout_is_bitwise_the_bhnd_result(H):
     c = H.run_library(inp, "bf16", True, 0.09, op="split", dq_mode=3, layout=1)
     for k in ("O", "L", "dQ", "dK", "dV"):
         np.testing.assert_array_equal(b[k], c[k], err_msg=k)
+
+
+def test_many_heads_short_sequences(H):
+    """2048 heads of 128 tokens: the grid is heads x tiles, so this walks the head index range of every
+    kernel (block order groups, tensor-map batch/head coordinates, workspace rows) far beyond the
+    named configurations.  Oracle on sampled heads, invariants on all."""
+    w = mi.Workload("many_heads", 64, 32, 128, 64, True, "bf16", 21)
+    _sampled_check(H, w, heads=[(0, 0), (17, 5), (63, 31)], nrows=16, ncols=16)
+    w2 = mi.Workload("many_heads_d128", 48, 40, 200, 128, False, "bf16", 22)
+    _sampled_check(H, w2, heads=[(0, 0), (47, 39)], nrows=16, ncols=16, dq_mode=3)
+
+
+def test_sequence_length_between_the_named_sizes(H):
+    """n = 40000 (not a multiple of the tile, longer than any named configuration) with causal masking:
+    sampled rows and columns of one head against the oracle, invariants on both heads."""
+    w = mi.Workload("n40000", 1, 2, 40000, 128, True, "bf16", 23)
+    _sampled_check(H, w, heads=[(0, 1)], nrows=10, ncols=10)
 
 
 def test_causal_block_order_with_a_partial_head_group(H):
