@@ -467,14 +467,27 @@ static bool decode_uses_tc(const DecodeProblem &p, int dtype)
     return dtype == MOA_BF16 && group >= 4 && group <= 128 && p.scale > 0.f;
 }
 
-// Tensor-core route: key tiles of 128 per CTA segment, about six CTAs per SM over the run
+// Tensor-core route: key tiles of 128 per CTA segment, one CTA per SM at a time.  All CTAs are equal,
+// so the run takes ceil(CTAs / 148) rounds of (fixed cost + tiles per segment); the fixed cost of a CTA
+// (pipeline fill, epilogue) was measured at about 3.5 tile times.  Take the segment count that
+// minimises rounds x (3.5 + tiles).
 static void decode_tc_splits(const DecodeProblem &p, int *splits, int *tiles_per_split)
 {
     const int nkt = (p.n + 127) / 128;
-    long long s = (6LL * 148 + (long long)p.B * p.Hkv - 1) / ((long long)p.B * p.Hkv);
-    if (s > nkt) s = nkt;
-    if (s < 1) s = 1;
-    const int tps = (int)((nkt + s - 1) / s);
+    const long long base = (long long)p.B * p.Hkv;
+    long long hi = (32LL * 148 + base - 1) / base;
+    if (hi > nkt) hi = nkt;
+    if (hi < 1) hi = 1;
+    long long best = 1;
+    double best_cost = 1e300;
+    for (long long s = 1; s <= hi; ++s) {
+        const int tps = (int)((nkt + s - 1) / s);
+        const long long real = (nkt + tps - 1) / tps;      // segments that get at least one tile
+        const long long rounds = (base * real + 147) / 148;
+        const double cost = (double)rounds * (3.5 + tps);
+        if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
+    }
+    const int tps = (int)((nkt + best - 1) / best);
     *tiles_per_split = tps;
     *splits = (nkt + tps - 1) / tps;          // every segment has at least one tile
 }
