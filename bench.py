@@ -390,6 +390,8 @@ def main():
     ap.add_argument("--path", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--materialize", type=int, default=0)
+    ap.add_argument("--graph", action="store_true",
+                    help="record the step into a CUDA graph once and time replays (launch-bound small sizes)")
     ap.add_argument("--decode", default="", choices=[""] + sorted(DECODE_WORKLOADS),
                     help="time decode attention on that workload instead of the fused forward+backward")
     ap.add_argument("--rowparallel", type=int, default=0,
@@ -469,6 +471,25 @@ def main():
         else:
             mb.moa_attn_fused_fwd_bwd(desc, Q, K, V, dO, O, L, dQ, dK, dV, ws, stream)
 
+    direct_step = step
+    if args.graph:
+        # the library allocates nothing and synchronises nothing: after one warm-up call (which resolves
+        # the per-device symbols) the step is recorded once and the timed region replays it
+        direct_step()
+        torch.cuda.synchronize()
+        cap = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        user_stream = stream
+        lc0 = mb.moa_launch_count()
+        with torch.cuda.graph(graph, stream=cap):
+            stream = torch.cuda.current_stream()
+            direct_step()
+        launches_per_replay = mb.moa_launch_count() - lc0     # kernels recorded in the graph
+        stream = user_stream
+
+        def step():
+            graph.replay()
+
     def barrier():
         torch.cuda.synchronize()
         if dist is not None:
@@ -505,6 +526,8 @@ def main():
     barrier()
     wall_ms = (time.perf_counter() - wall0) * 1e3 / args.steps
     launches = mb.moa_launch_count() - launches0
+    if args.graph:
+        launches = launches_per_replay * args.steps        # replays launch the recorded kernels without host calls
     sampler.stop()
     ms_total = max_over_ranks(e0.elapsed_time(e1))
     # per-kernel durations: a separate pass after the timed region, so that the event pairs the
@@ -512,7 +535,7 @@ def main():
     mb.moa_profile_read()
     mb.moa_profile_enable(True)
     for _ in range(max(3, min(args.steps, 10))):
-        step()
+        direct_step()
     torch.cuda.synchronize()
     mb.moa_profile_enable(False)
     prof = mb.moa_profile_read()
@@ -629,6 +652,8 @@ def main():
         line["config"]["H_kv"] = args.hkv
     if args.layout:
         line["config"]["layout"] = "[B,n,H,d]"
+    if args.graph:
+        line["config"]["launch"] = "one CUDA graph replay per step"
     if args.rowparallel:
         line["config"]["variant"] = f"row-parallel single kernel, {args.rowparallel} atomic site(s), fp32 CUDA cores"
     if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.hkv and not args.layout and not args.rowparallel:

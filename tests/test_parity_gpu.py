@@ -344,3 +344,37 @@ def test_causal_block_order_with_a_partial_head_group(H):
 def test_c3_other_dq_modes_sampled(H, dq_mode):
     w = mi.CONFIGS["c3_causal_mid"]
     _sampled_check(H, w, heads=[(1, 7)], dq_mode=dq_mode)
+
+
+def test_fused_call_can_be_captured_in_a_cuda_graph_and_replayed(H):
+    """The library allocates nothing, synchronises nothing and takes the caller's stream, so a fused
+    call can be recorded into a CUDA graph once and replayed (the launch-bound small sizes gain
+    from it).  A replay on new input values gives the same bits as a direct call on them."""
+    import torch
+    from paper_2609_33916_b200 import binding as mb
+    B, Hh, n, d = 1, 4, 512, 128
+    desc = mb.make_desc(B, Hh, n, d, True, 1.0 / math.sqrt(d), dq_mode=mb.MOA_DQ_SEPARATE_PASS)
+    gen = torch.Generator(device="cuda").manual_seed(3)
+    mk = lambda: torch.randn((B, Hh, n, d), generator=gen, device="cuda").to(torch.bfloat16)
+    Q, K, V, dO = mk(), mk(), mk(), mk()
+    O, dQ, dK, dV = (torch.empty_like(Q) for _ in range(4))
+    L = torch.empty((B, Hh, n), dtype=torch.float32, device="cuda")
+    ws = torch.empty(max(16, mb.moa_attn_workspace_bytes(desc, mb.MOA_OP_FUSED)), dtype=torch.uint8, device="cuda")
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        mb.moa_attn_fused_fwd_bwd(desc, Q, K, V, dO, O, L, dQ, dK, dV, ws, side)     # warm-up outside the capture
+    side.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        mb.moa_attn_fused_fwd_bwd(desc, Q, K, V, dO, O, L, dQ, dK, dV, ws, torch.cuda.current_stream())
+    # new values in the captured buffers, then replay
+    for t in (Q, K, V, dO):
+        t.copy_(torch.randn(t.shape, generator=gen, device="cuda").to(torch.bfloat16))
+    graph.replay()
+    torch.cuda.synchronize()
+    got = [t.clone() for t in (O, L, dQ, dK, dV)]
+    mb.moa_attn_fused_fwd_bwd(desc, Q, K, V, dO, O, L, dQ, dK, dV, ws)
+    torch.cuda.synchronize()
+    for a, b, name in zip(got, (O, L, dQ, dK, dV), ("O", "L", "dQ", "dK", "dV")):
+        assert torch.equal(a, b), name
+    assert mb.moa_last_device_status() == mb.MOA_OK
