@@ -89,7 +89,9 @@ template <> __device__ __forceinline__ float from_float<float>(float v) { return
 template <> __device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
 // ---- tensor-core path (tc_fwd.cu), bf16 only ---------------------------------------------
-cudaError_t tc_fwd(const Problem &p, const void *Q, const void *K, const void *V, void *O, float *L, cudaStream_t st);
+// zero_acc: nullptr, or the fp32 dQ accumulator [B*H, n, d] of a fused call, which the forward then clears
+cudaError_t tc_fwd(const Problem &p, const void *Q, const void *K, const void *V, void *O, float *L, float *zero_acc,
+                   cudaStream_t st);
 
 // Lp = -L*log2(e) and Dp = -rowsum(dO o O) (negated: fma/add operands), each padded per head to a
 // multiple of 128 rows (-inf / 0 past n)

@@ -65,7 +65,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
               const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapO,
               float *__restrict__ L,
               int n, int causal, float scale_log2, int nqt, int hpg, int group, int H, FwdSplit sp,
-              unsigned int *status)
+              float *__restrict__ zero_acc, unsigned int *status)
 {
     constexpr int kTileBytes = 128 * D * 2;
     constexpr int kBoxes = D / 64;         // 64-column (128-byte) swizzled boxes per tile
@@ -109,7 +109,26 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             mbar_arrive_expect_tx(bars + F_Q, kTileBytes);
             for (int b = 0; b < kBoxes; ++b) tma_load_4d(sQ + b * kBoxBytes, &mapQ, bars + F_Q, 64 * b, q0, hq, bb);
         }
-        for (int j = 0; j < nkt; ++j) {
+        if (zero_acc != nullptr) {
+            // Fused forward+backward: this CTA's 128 rows of the fp32 dQ accumulator ([B*H, n, D]) are
+            // cleared here, by the producer warp while its first loads are in flight (the next slot
+            // frees two tiles from now), so that the step needs no separate clearing pass.
+            // The first two K/V tiles are requested first: they have no slot to wait for.
+            for (int j = 0; j < min(nkt, 2); ++j) {
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(bars + F_KFULL + j, kTileBytes);
+                    for (int b = 0; b < kBoxes; ++b)
+                        tma_load_4d(sK + j * kTileBytes + b * kBoxBytes, &mapK, bars + F_KFULL + j, 64 * b, (kt0 + j) * BN, hk, bb);
+                    mbar_arrive_expect_tx(bars + F_VFULL + j, kTileBytes);
+                    for (int b = 0; b < kBoxes; ++b)
+                        tma_load_4d(sV + j * kTileBytes + b * kBoxBytes, &mapV, bars + F_VFULL + j, 64 * b, (kt0 + j) * BN, hk, bb);
+                }
+            }
+            const int rows = min(BM, n - q0);
+            float4 *dst = reinterpret_cast<float4 *>(zero_acc + ((size_t)bh * n + q0) * D);
+            for (int i = lane; i < rows * (D / 4); i += 32) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        for (int j = (zero_acc != nullptr ? min(nkt, 2) : 0); j < nkt; ++j) {
             const int s = j & 1;
             if (j >= 2 && !mbar_wait(bars + F_KEMPTY + s, ((j >> 1) - 1) & 1, abortp, status, ERR_K)) break;
             if (lane == 0) {
@@ -338,7 +357,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
 
 template <int D>
 cudaError_t launch_fwd(const Problem &p, const void *Q, const void *K, const void *V, void *O, float *L,
-                       cudaStream_t st)
+                       float *zero_acc, cudaStream_t st)
 {
     constexpr int kSmem = 5 * 128 * D * 2 + 8 * (F_COUNT + 2) + 2 * 128 * 8;
     CUtensorMap mq, mk, mv, mo;
@@ -355,7 +374,7 @@ cudaError_t launch_fwd(const Problem &p, const void *Q, const void *K, const voi
     LaunchScope scope(MOA_KERNEL_FWD, st);
     tc_fwd_kernel<D><<<(unsigned)(nqt * p.BH()), kThreads, kSmem, st>>>(
         mq, mk, mv, mo, L, p.n, p.causal, p.scale * kLog2e, nqt, heads_per_group(p, nqt), p.group(), p.H,
-        FwdSplit{p.n, 1, (p.n + BN - 1) / BN}, device_status_ptr());
+        FwdSplit{p.n, 1, (p.n + BN - 1) / BN}, zero_acc, device_status_ptr());
     return cudaGetLastError();
 }
 
@@ -380,7 +399,7 @@ cudaError_t launch_fwd_decode(int B, int Hkv, int G, int n, float scale, const v
     LaunchScope scope(MOA_KERNEL_FWD, st);
     tc_fwd_kernel<D><<<(unsigned)(B * Hkv * splits), kThreads, kSmem, st>>>(
         mq, mk, mv, mo, L_part, n, 0, scale * kLog2e, 1, 1, 1, Hkv, FwdSplit{G, splits, tiles_per_split},
-        device_status_ptr());
+        nullptr, device_status_ptr());
     return cudaGetLastError();
 }
 
@@ -394,10 +413,11 @@ cudaError_t tc_fwd_decode(int B, int Hkv, int G, int n, int d, float scale, cons
     return cudaErrorInvalidValue;
 }
 
-cudaError_t tc_fwd(const Problem &p, const void *Q, const void *K, const void *V, void *O, float *L, cudaStream_t st)
+cudaError_t tc_fwd(const Problem &p, const void *Q, const void *K, const void *V, void *O, float *L, float *zero_acc,
+                   cudaStream_t st)
 {
-    if (p.d == 64) return launch_fwd<64>(p, Q, K, V, O, L, st);
-    if (p.d == 128) return launch_fwd<128>(p, Q, K, V, O, L, st);
+    if (p.d == 64) return launch_fwd<64>(p, Q, K, V, O, L, zero_acc, st);
+    if (p.d == 128) return launch_fwd<128>(p, Q, K, V, O, L, zero_acc, st);
     return cudaErrorInvalidValue;
 }
 
