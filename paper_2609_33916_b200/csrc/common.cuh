@@ -89,9 +89,16 @@ template <> __device__ __forceinline__ float from_float<float>(float v) { return
 template <> __device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
 // ---- tensor-core path (tc_fwd.cu), bf16 only ---------------------------------------------
-// zero_acc: nullptr, or the fp32 dQ accumulator [B*H, n, d] of a fused call, which the forward then clears
-cudaError_t tc_fwd(const Problem &p, const void *Q, const void *K, const void *V, void *O, float *L, float *zero_acc,
-                   cudaStream_t st);
+// What the forward of a fused call does for its backward (all null for a plain forward): it clears the fp32
+// dQ accumulator [B*H, n, d], and writes the backward's per-row inputs -L log2 e and -D = -rowsum(dO o O)
+// (from the fp32 O it holds), padded to n_pad rows per head with -inf / 0.
+struct FwdForBwd {
+    float *zero_acc = nullptr;
+    const void *dO = nullptr;
+    float *Lp = nullptr, *Dp = nullptr;
+};
+cudaError_t tc_fwd(const Problem &p, const void *Q, const void *K, const void *V, void *O, float *L,
+                   const FwdForBwd &fb, cudaStream_t st);
 
 // Lp = -L*log2(e) and Dp = -rowsum(dO o O) (negated: fma/add operands), each padded per head to a
 // multiple of 128 rows (-inf / 0 past n)

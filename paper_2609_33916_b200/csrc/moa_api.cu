@@ -218,19 +218,19 @@ moa_status run_materialized(const moa_attn_desc *d, const void *Q, const void *K
 }
 
 moa_status run_fwd(const moa_attn_desc *d, const void *Q, const void *K, const void *V, void *O, float *L,
-                   float *zero_acc, cudaStream_t st)
+                   const FwdForBwd &fb, cudaStream_t st)
 {
-    // zero_acc: the dQ accumulator of a fused call for the tensor-core forward to clear, or nullptr
-    const cudaError_t e = use_tc_fwd(d) ? tc_fwd(to_problem(d), Q, K, V, O, L, zero_acc, st)
+    // fb: what the tensor-core forward of a fused call prepares for its backward (empty otherwise)
+    const cudaError_t e = use_tc_fwd(d) ? tc_fwd(to_problem(d), Q, K, V, O, L, fb, st)
                              : simt_fwd(to_problem(d), d->dtype, Q, K, V, O, L, st);
     return e == cudaSuccess ? MOA_OK : MOA_ERR_CUDA;
 }
 
 moa_status run_bwd(const moa_attn_desc *d, const void *Q, const void *K, const void *V, const void *O,
-                   const float *L, const void *dO, void *dQ, void *dK, void *dV, void *ws, bool acc_cleared,
+                   const float *L, const void *dO, void *dQ, void *dK, void *dV, void *ws, bool prepared,
                    cudaStream_t st)
 {
-    // acc_cleared: the forward of the same fused call has already cleared the dQ accumulator
+    // prepared: the forward of the same fused call has cleared the dQ accumulator and written -L log2e and -D
     const Problem p = to_problem(d);
     const BwdWorkspace w = bwd_workspace(d);
     float *Dv = (float *)ws;
@@ -240,13 +240,13 @@ moa_status run_bwd(const moa_attn_desc *d, const void *Q, const void *K, const v
     const int mode = resolved_dq_mode(d);
 #define MOA_TRY(x) do { if ((x) != cudaSuccess) return MOA_ERR_CUDA; } while (0)
     if (use_tc_bwd(d)) {
-        MOA_TRY(tc_bwd_preprocess(p, dO, O, L, Lp, Dv, st));
+        if (!prepared) MOA_TRY(tc_bwd_preprocess(p, dO, O, L, Lp, Dv, st));
         if (mode == MOA_DQ_SEPARATE_PASS) {
             MOA_TRY(tc_bwd_kv(p, Q, K, V, dO, Lp, Dv, dK, dV, nullptr, 0, st));
             MOA_TRY(tc_bwd_dq(p, Q, K, V, dO, Lp, Dv, dQ, st));
             return MOA_OK;
         }
-        if (!acc_cleared) MOA_TRY(cudaMemsetAsync(dQacc, 0, elems * sizeof(float), st));
+        if (!prepared) MOA_TRY(cudaMemsetAsync(dQacc, 0, elems * sizeof(float), st));
         MOA_TRY(tc_bwd_kv(p, Q, K, V, dO, Lp, Dv, dK, dV, dQacc, mode == MOA_DQ_BULK_REDUCE, st));
         if (p.bnhd) MOA_TRY(convert_f32_to_bf16_bnhd(dQacc, dQ, p.B, p.H, p.n, p.d, p.scale, st));
         else MOA_TRY(convert_f32_to_bf16(dQacc, dQ, elems, p.scale, st));
@@ -328,7 +328,7 @@ moa_status moa_attn_fwd(const moa_attn_desc *desc, const void *Q, const void *K,
     if ((s = check_arch()) != MOA_OK) return s;
     if (desc->materialize)
         return run_materialized(desc, Q, K, V, nullptr, O, L, nullptr, nullptr, nullptr, ws, false, (cudaStream_t)stream);
-    return run_fwd(desc, Q, K, V, O, L, nullptr, (cudaStream_t)stream);
+    return run_fwd(desc, Q, K, V, O, L, FwdForBwd{}, (cudaStream_t)stream);
 }
 
 moa_status moa_attn_bwd(const moa_attn_desc *desc, const void *Q, const void *K, const void *V,
@@ -385,13 +385,18 @@ moa_status moa_attn_fused_fwd_bwd(const moa_attn_desc *desc, const void *Q, cons
     if ((s = check_arch()) != MOA_OK) return s;
     if (desc->materialize) return run_materialized(desc, Q, K, V, dO, O, L, dQ, dK, dV, ws, true, (cudaStream_t)stream);
     // tensor-core path with an atomic dQ mode: the forward clears the accumulator its backward adds into
-    float *zero_acc = nullptr;
-    if (use_tc_fwd(desc) && use_tc_bwd(desc)) {
+    // and writes the backward's per-row inputs (-L log2e, -D) from the fp32 O it holds
+    FwdForBwd fb;
+    const bool both_tc = use_tc_fwd(desc) && use_tc_bwd(desc);
+    if (both_tc) {
         const BwdWorkspace w = bwd_workspace(desc);
-        if (w.dqacc_bytes) zero_acc = (float *)((char *)ws + w.d_bytes + w.lp_bytes);
+        fb.Dp = (float *)ws;
+        fb.Lp = (float *)((char *)ws + w.d_bytes);
+        fb.dO = dO;
+        if (w.dqacc_bytes) fb.zero_acc = (float *)((char *)ws + w.d_bytes + w.lp_bytes);
     }
-    if ((s = run_fwd(desc, Q, K, V, O, L, zero_acc, (cudaStream_t)stream)) != MOA_OK) return s;
-    return run_bwd(desc, Q, K, V, O, L, dO, dQ, dK, dV, ws, zero_acc != nullptr, (cudaStream_t)stream);
+    if ((s = run_fwd(desc, Q, K, V, O, L, fb, (cudaStream_t)stream)) != MOA_OK) return s;
+    return run_bwd(desc, Q, K, V, O, L, dO, dQ, dK, dV, ws, both_tc, (cudaStream_t)stream);
 }
 
 moa_status moa_attn_fused_rowparallel(const moa_attn_desc *desc, const void *Q, const void *K, const void *V,

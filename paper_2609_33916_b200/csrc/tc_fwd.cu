@@ -59,13 +59,21 @@ struct FwdSplit {
     int n_q, splits, tiles_per_split;
 };
 
+// Fused call only (dO == nullptr otherwise): the backward's per-row inputs, written by the forward
+// epilogue: Lp = -(logsumexp in the log2 domain), Dp = -rowsum(dO o O), [B*H, n_pad] each.
+struct FwdPrep {
+    const __nv_bfloat16 *dO;
+    float *Lp, *Dp;
+    int n_pad, bnhd;
+};
+
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
               const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapO,
               float *__restrict__ L,
               int n, int causal, float scale_log2, int nqt, int hpg, int group, int H, FwdSplit sp,
-              float *__restrict__ zero_acc, unsigned int *status)
+              float *__restrict__ zero_acc, FwdPrep prep, unsigned int *status)
 {
     constexpr int kTileBytes = 128 * D * 2;
     constexpr int kBoxes = D / 64;         // 64-column (128-byte) swizzled boxes per tile
@@ -216,6 +224,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         const uint32_t ocol = kColO + h * D;
         float m_used = 0.f, l = 0.f;
         bool ok = nkt > 0;
+        if (prep.dO != nullptr && row < n) {
+            // fused call: the epilogue reads this thread's 128 bytes (D = 128) of its dO row; ask L2 for
+            // them now so that the read at the end of the job does not wait on HBM
+            const size_t drow = prep.bnhd ? ((size_t)bb * n + row) * H + hq : (size_t)bh * n + row;
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(prep.dO + drow * D + (D / 2) * h));
+        }
         // The exp2 phase of a tile is MUFU-bound and the rest of a tile's work (TMEM load, max,
         // hand-offs) is not: start the second warpgroup a few hundred cycles late, once, so that on
         // each scheduler one warp's exp2 phase overlaps the other's remaining work.  Nothing in the
@@ -307,6 +321,17 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         // ---- epilogue: merge the two key halves.  Each thread publishes (m, l) of its half, then
         // writes D/2 output columns of its row from both accumulators.
         float2 *xch = reinterpret_cast<float2 *>(bars + F_COUNT + 2);   // [2][128] (m, l)
+        float *xd = reinterpret_cast<float *>(xch + 256);               // [2][128] partial rowsum(dO o O)
+        // fused call: this thread's D/2 elements of its dO row, requested before the waits below
+        uint4 dov[D / 16];
+        const bool want_d = prep.dO != nullptr && row < n;
+        if (want_d) {
+            const size_t drow = prep.bnhd ? ((size_t)bb * n + row) * H + hq : (size_t)bh * n + row;
+            const uint4 *src = reinterpret_cast<const uint4 *>(prep.dO + drow * D + (D / 2) * h);
+#pragma unroll
+            for (int k = 0; k < D / 16; ++k) dov[k] = __ldg(src + k);
+        }
+        float dpart = 0.f;
         xch[h * 128 + lane_row] = make_float2(m_used, l);
         mbar_arrive(bars + F_X);
         if (ok && mbar_wait(bars + F_X, 0, abortp, status, ERR_P) &&
@@ -332,6 +357,16 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                     float v[8];
 #pragma unroll
                     for (int u = 0; u < 8; ++u) v[u] = __uint_as_float(o0[i + u]) * w0 + __uint_as_float(o1[i + u]) * w1;
+                    if (want_d) {
+                        const uint4 g = dov[(c + i) / 8];
+                        const uint32_t gw[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const float2 gg = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&gw[u]));
+                            dpart = fmaf(v[2 * u], gg.x, dpart);
+                            dpart = fmaf(v[2 * u + 1], gg.y, dpart);
+                        }
+                    }
                     uint4 q;
                     q.x = pack_bf16(v[0], v[1]); q.y = pack_bf16(v[2], v[3]);
                     q.z = pack_bf16(v[4], v[5]); q.w = pack_bf16(v[6], v[7]);
@@ -340,8 +375,15 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                     *reinterpret_cast<uint4 *>(sQ + (cabs >> 6) * kBoxBytes + lane_row * 128 + chunk * 16) = q;
                 }
             }
+            xd[h * 128 + lane_row] = dpart;
             fence_proxy_async_smem();
             mbar_arrive(bars + F_E);
+            if (prep.dO != nullptr && h == 0 && mbar_wait(bars + F_E, 0, abortp, status, ERR_O)) {
+                // both halves of the row are in: the backward's per-row inputs, in its padded layout
+                const size_t prow = (size_t)bh * prep.n_pad + row;
+                prep.Dp[prow] = row < n ? -(dpart + xd[128 + lane_row]) : 0.f;
+                prep.Lp[prow] = row < n ? -(m_all + log2f(l_all)) : -INFINITY;
+            }
             if (tid == 0 && mbar_wait(bars + F_E, 0, abortp, status, ERR_O)) {
                 for (int b = 0; b < kBoxes; ++b) tma_store_4d(&mapO, sQ + b * kBoxBytes, 64 * b, q0, hq, split * (heads_all / H) + bb);
                 bulk_commit();
@@ -357,9 +399,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
 
 template <int D>
 cudaError_t launch_fwd(const Problem &p, const void *Q, const void *K, const void *V, void *O, float *L,
-                       float *zero_acc, cudaStream_t st)
+                       const FwdForBwd &fb, cudaStream_t st)
 {
-    constexpr int kSmem = 5 * 128 * D * 2 + 8 * (F_COUNT + 2) + 2 * 128 * 8;
+    constexpr int kSmem = 5 * 128 * D * 2 + 8 * (F_COUNT + 2) + 2 * 128 * 8 + 2 * 128 * 4;
     CUtensorMap mq, mk, mv, mo;
     const bool bnhd = p.bnhd != 0;
     const auto bf = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
@@ -374,7 +416,8 @@ cudaError_t launch_fwd(const Problem &p, const void *Q, const void *K, const voi
     LaunchScope scope(MOA_KERNEL_FWD, st);
     tc_fwd_kernel<D><<<(unsigned)(nqt * p.BH()), kThreads, kSmem, st>>>(
         mq, mk, mv, mo, L, p.n, p.causal, p.scale * kLog2e, nqt, heads_per_group(p, nqt), p.group(), p.H,
-        FwdSplit{p.n, 1, (p.n + BN - 1) / BN}, zero_acc, device_status_ptr());
+        FwdSplit{p.n, 1, (p.n + BN - 1) / BN}, fb.zero_acc,
+        FwdPrep{(const __nv_bfloat16 *)fb.dO, fb.Lp, fb.Dp, nqt * BM, p.bnhd}, device_status_ptr());
     return cudaGetLastError();
 }
 
@@ -386,7 +429,7 @@ template <int D>
 cudaError_t launch_fwd_decode(int B, int Hkv, int G, int n, float scale, const void *q, const void *K, const void *V,
                               void *O_part, float *L_part, int splits, int tiles_per_split, cudaStream_t st)
 {
-    constexpr int kSmem = 5 * 128 * D * 2 + 8 * (F_COUNT + 2) + 2 * 128 * 8;
+    constexpr int kSmem = 5 * 128 * D * 2 + 8 * (F_COUNT + 2) + 2 * 128 * 8 + 2 * 128 * 4;
     CUtensorMap mq, mk, mv, mo;
     const auto bf = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     if (!make_tensor_map_4d(&mq, q, bf, 2, B, Hkv, G, D, false, 128, 64) ||
@@ -399,7 +442,7 @@ cudaError_t launch_fwd_decode(int B, int Hkv, int G, int n, float scale, const v
     LaunchScope scope(MOA_KERNEL_FWD, st);
     tc_fwd_kernel<D><<<(unsigned)(B * Hkv * splits), kThreads, kSmem, st>>>(
         mq, mk, mv, mo, L_part, n, 0, scale * kLog2e, 1, 1, 1, Hkv, FwdSplit{G, splits, tiles_per_split},
-        nullptr, device_status_ptr());
+        nullptr, FwdPrep{nullptr, nullptr, nullptr, 0, 0}, device_status_ptr());
     return cudaGetLastError();
 }
 
@@ -413,11 +456,11 @@ cudaError_t tc_fwd_decode(int B, int Hkv, int G, int n, int d, float scale, cons
     return cudaErrorInvalidValue;
 }
 
-cudaError_t tc_fwd(const Problem &p, const void *Q, const void *K, const void *V, void *O, float *L, float *zero_acc,
-                   cudaStream_t st)
+cudaError_t tc_fwd(const Problem &p, const void *Q, const void *K, const void *V, void *O, float *L,
+                   const FwdForBwd &fb, cudaStream_t st)
 {
-    if (p.d == 64) return launch_fwd<64>(p, Q, K, V, O, L, zero_acc, st);
-    if (p.d == 128) return launch_fwd<128>(p, Q, K, V, O, L, zero_acc, st);
+    if (p.d == 64) return launch_fwd<64>(p, Q, K, V, O, L, fb, st);
+    if (p.d == 128) return launch_fwd<128>(p, Q, K, V, O, L, fb, st);
     return cudaErrorInvalidValue;
 }
 

@@ -109,8 +109,21 @@ def test_fused_call_equals_fwd_then_bwd(H, path):
     inp = mi.make_inputs(2, 2, 320, 128, seed=5, dtype="bf16")
     a = H.run_library(inp, "bf16", True, 0.09, op="fused", dq_mode=3, path=path)
     b = H.run_library(inp, "bf16", True, 0.09, op="split", dq_mode=3, path=path)
-    for k in ("O", "L", "dQ", "dK", "dV"):
+    _fused_vs_split(a, b, exact_gradients=(path == 1))
+
+
+def _fused_vs_split(a, b, exact_gradients):
+    """The forward is the same kernel either way: O and L agree bit for bit.  On the tensor-core path the
+    fused call takes the backward's per-row inputs (D = rowsum(dO o O), L in the log2 domain) from the
+    fp32 values its forward holds, the separate backward from the bf16 O and fp32 L it is given, so the
+    gradients agree to a few bf16 roundings, not bitwise; the CUDA-core path is identical either way."""
+    for k in ("O", "L"):
         np.testing.assert_array_equal(a[k], b[k], err_msg=k)
+    for k in ("dQ", "dK", "dV"):
+        if exact_gradients:
+            np.testing.assert_array_equal(a[k], b[k], err_msg=k)
+        else:
+            assert mi.rel_err(a[k], b[k]) <= 8e-3, (k, mi.rel_err(a[k], b[k]))     # one bf16 unit in the last place of the largest element
 
 
 @pytest.mark.parametrize("path", [1, 2])
@@ -266,8 +279,7 @@ def test_gqa_fused_call_equals_fwd_then_bwd(H):
     inp = _gqa_inputs(1, 8, 2, 384, 128, seed=77)
     a = H.run_library(inp, "bf16", True, 0.09, op="fused", dq_mode=3)
     b = H.run_library(inp, "bf16", True, 0.09, op="split", dq_mode=3)
-    for k in ("O", "L", "dQ", "dK", "dV"):
-        np.testing.assert_array_equal(a[k], b[k], err_msg=k)
+    _fused_vs_split(a, b, exact_gradients=False)
 
 
 def test_gqa_equals_replicated_kv_heads(H):
@@ -310,8 +322,10 @@ def test_bnhd_layout_is_bitwise_the_bhnd_result(H):
     for k in ("O", "L", "dQ", "dK", "dV"):
         np.testing.assert_array_equal(a[k], b[k], err_msg=k)
     c = H.run_library(inp, "bf16", True, 0.09, op="split", dq_mode=3, layout=1)
-    for k in ("O", "L", "dQ", "dK", "dV"):
-        np.testing.assert_array_equal(b[k], c[k], err_msg=k)
+    _fused_vs_split(b, c, exact_gradients=False)
+    d = H.run_library(inp, "bf16", True, 0.09, op="split", dq_mode=3, layout=0)
+    for k in ("O", "L", "dQ", "dK", "dV"):       # and the separate calls are bitwise the same in both layouts
+        np.testing.assert_array_equal(c[k], d[k], err_msg=k)
 
 
 def test_many_heads_short_sequences(H):
