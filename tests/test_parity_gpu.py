@@ -216,7 +216,7 @@ def test_c3_causal_mid_sampled(H):
     _sampled_check(H, w, heads=[(0, 0), (1, 15)])
 
 
-@pytest.mark.parametrize("n", [512, 2048])
+@pytest.mark.parametrize("n", [512, 1024, 2048, 4096])
 def test_c5_causal_sweep_small_sizes_sampled(H, n):
     w = mi.CONFIGS[f"c5_causal_n{n}"]
     _sampled_check(H, w, heads=[(0, 0), (0, 31)])
@@ -230,7 +230,7 @@ def test_c4_long_full_size_sampled(H):
     _sampled_check(H, w, heads=[(0, 0), (0, 15)], nrows=16, ncols=16)
 
 
-@pytest.mark.parametrize("n", [8192, 32768])
+@pytest.mark.parametrize("n", [8192, 16384, 32768])
 def test_c5_causal_sweep_large_sizes_sampled(H, n):
     w = mi.CONFIGS[f"c5_causal_n{n}"]
     _sampled_check(H, w, heads=[(0, 31)] if n > 8192 else [(0, 0), (0, 31)], nrows=12, ncols=12)
