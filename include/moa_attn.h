@@ -31,7 +31,10 @@
  *  - Outputs are overwritten, never accumulated into.
  *  - Errors are reported only through the returned moa_status; the library does
  *    not abort or throw.  On any error nothing has been enqueued.
- *  - Supported: d in {64, 128}; any n >= 1 and B, H >= 1 (B*H <= 2^20 and
+ *  - Supported: d in {64, 128} everywhere; on the bf16 tensor-core kernels also every
+ *    other multiple of 8 up to 128 (d = 96, 80, 32, ...: the head runs in the 64- or
+ *    128-column kernel, TMA zero-fills the missing columns on load and drops them on
+ *    store; not with materialize = 1).  Any n >= 1 and B, H >= 1 (B*H <= 2^20 and
  *    ceil(n/64)*B*H < 2^31, else MOA_ERR_UNSUPPORTED); n need not be a multiple
  *    of the tile size.
  *    A device that is not compute capability 10.x gives MOA_ERR_ARCH.
@@ -49,7 +52,7 @@ extern "C" {
 typedef enum {
     MOA_OK = 0,
     MOA_ERR_INVALID_ARG = 1, /* NULL pointer, misaligned pointer, non-positive size, bad enum  */
-    MOA_ERR_UNSUPPORTED = 2, /* well-formed request this build cannot run (e.g. d = 96)       */
+    MOA_ERR_UNSUPPORTED = 2, /* well-formed request this build cannot run (e.g. d = 192)      */
     MOA_ERR_WORKSPACE = 3,   /* ws == NULL or ws_bytes < moa_attn_workspace_bytes(...)         */
     MOA_ERR_ARCH = 4,        /* current device is not sm_100                                   */
     MOA_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed (launch, descriptor encode)  */
@@ -64,9 +67,9 @@ typedef enum { MOA_BF16 = 0, MOA_F32 = 1 } moa_dtype;
  * paper's GK/GV atomic sites and their removal, transposed here onto dQ because
  * the backward kernel is parallel over key tiles). */
 typedef enum {
-    MOA_DQ_AUTO = 0,          /* library's choice: BULK_REDUCE for bf16 d=128, else RED        */
+    MOA_DQ_AUTO = 0,          /* library's choice: BULK_REDUCE for bf16 d > 64, else RED       */
     MOA_DQ_RED = 1,           /* fp32 red.global.add into a [B,H,n,d] fp32 accumulator        */
-    MOA_DQ_BULK_REDUCE = 2,   /* shared-memory tile + cp.reduce.async.bulk add.f32 (bf16 d=128) */
+    MOA_DQ_BULK_REDUCE = 2,   /* shared-memory tile + cp.reduce.async.bulk add.f32 (bf16 d > 64) */
     MOA_DQ_SEPARATE_PASS = 3  /* no atomics: a second, query-parallel kernel recomputes dS     */
 } moa_dq_mode;
 

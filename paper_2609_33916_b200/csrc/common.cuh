@@ -20,6 +20,11 @@ struct Problem {
     int BHkv() const { return B * kv_heads(); }
 };
 
+// Head dimension the tensor-core kernels are compiled for: a head of d columns (a multiple of 8, so
+// that rows stay 16-byte aligned) runs in the 64- or 128-column kernel; the TMA loads fill the
+// columns past d with zeros and the TMA stores drop them, which leaves every result unchanged.
+inline int kernel_d(int d) { return d <= 64 ? 64 : 128; }
+
 // Block order of the tile-parallel kernels.  Heads are taken in groups of `hpg`; inside a group
 // the blocks go tile-major (every head's tile 0, then every head's tile 1, ...).  With causal
 // masking tile t is the t-th longest job, so the hardware's in-order block dispatch becomes
@@ -90,7 +95,7 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(f
 
 // ---- tensor-core path (tc_fwd.cu), bf16 only ---------------------------------------------
 // What the forward of a fused call does for its backward (all null for a plain forward): it clears the fp32
-// dQ accumulator [B*H, n, d], and writes the backward's per-row inputs -L log2 e and -D = -rowsum(dO o O)
+// dQ accumulator [B*H, n, kernel_d(d)], and writes the backward's per-row inputs -L log2 e and -D = -rowsum(dO o O)
 // (from the fp32 O it holds), padded to n_pad rows per head with -inf / 0.
 struct FwdForBwd {
     float *zero_acc = nullptr;
@@ -105,7 +110,7 @@ cudaError_t tc_fwd(const Problem &p, const void *Q, const void *K, const void *V
 cudaError_t tc_bwd_preprocess(const Problem &p, const void *dO, const void *O, const float *L, float *Lp, float *Dp,
                               cudaStream_t st);
 // dK, dV; UNSCALED dQ contributions (dS K, without the factor scale) red-added into dQacc
-// (fp32 [B,H,n,d], pre-zeroed); dQacc == nullptr skips the dQ contraction altogether
+// (fp32 [B,H,n,kernel_d(d)], pre-zeroed); dQacc == nullptr skips the dQ contraction altogether
 cudaError_t tc_bwd_kv(const Problem &p, const void *Q, const void *K, const void *V, const void *dO,
                       const float *Lp, const float *Dp, void *dK, void *dV, float *dQacc, int dq_bulk,
                       cudaStream_t st);   // dq_bulk: TMA bulk add-reduce instead of red.global (d = 128 only)
@@ -141,7 +146,9 @@ cudaError_t simt_bwd_dq(const Problem &p, int dtype, const void *Q, const void *
                         const void *dO, const float *L, const float *Dv, void *dQ, cudaStream_t st);
 // dst[i] = (bf16)(mul * src[i])
 cudaError_t convert_f32_to_bf16(const float *src, void *dst, size_t count, float mul, cudaStream_t st);
-// the same into a [B,n,H,d] tensor from the [B*H, n, d] accumulator
-cudaError_t convert_f32_to_bf16_bnhd(const float *src, void *dst, int B, int H, int n, int d, float mul, cudaStream_t st);
+// the same row by row: the accumulator is [B*H, n, src_ld] (src_ld >= d: the kernels' padded head
+// dimension), the destination [B,H,n,d] or, with bnhd, [B,n,H,d]
+cudaError_t convert_f32_to_bf16_rows(const float *src, int src_ld, void *dst, int B, int H, int n, int d, int bnhd,
+                                     float mul, cudaStream_t st);
 
 }  // namespace moa

@@ -93,7 +93,12 @@ moa_status check_desc(const moa_attn_desc *d)
     if (d->materialize != 0 && d->materialize != 1) return MOA_ERR_INVALID_ARG;
     if (d->path < MOA_PATH_AUTO || d->path > MOA_PATH_TC) return MOA_ERR_INVALID_ARG;
     if (!(d->scale == d->scale) || d->scale - d->scale != 0.f) return MOA_ERR_INVALID_ARG;  // NaN / inf
-    if (d->d != 64 && d->d != 128) return MOA_ERR_UNSUPPORTED;
+    // head dimensions other than 64 and 128: multiples of 8 up to 128, on the tensor-core kernels only
+    // (they run in the 64- or 128-column kernel with the missing columns filled with zeros)
+    if (d->d != 64 && d->d != 128 &&
+        !(d->d % 8 == 0 && d->d <= 128 && d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->scale > 0.f &&
+          !d->materialize))
+        return MOA_ERR_UNSUPPORTED;
     if ((long long)d->B * d->H > (1 << 20)) return MOA_ERR_UNSUPPORTED;
     // one CTA per (tile, head) in grid.x
     const long long tiles = ((long long)d->n + 63) / 64;
@@ -101,9 +106,9 @@ moa_status check_desc(const moa_attn_desc *d)
     if (d->path == MOA_PATH_TC && d->dtype != MOA_BF16) return MOA_ERR_UNSUPPORTED;
     // the materialising comparison variant runs on the tensor-core path only
     if (d->materialize && !(d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->scale > 0.f)) return MOA_ERR_UNSUPPORTED;
-    // the bulk-reduce strategy exists in the tensor-core backward for d = 128 only
+    // the bulk-reduce strategy exists in the 128-column tensor-core backward only
     if (d->dq_mode == MOA_DQ_BULK_REDUCE &&
-        !(d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->d == 128 && d->scale > 0.f))
+        !(d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && kernel_d(d->d) == 128 && d->scale > 0.f))
         return MOA_ERR_UNSUPPORTED;
     if (d->path == MOA_PATH_TC && !(d->scale > 0.f)) return MOA_ERR_UNSUPPORTED;   // non-positive scale: SIMT path only
     if (d->layout != MOA_LAYOUT_BHND && d->layout != MOA_LAYOUT_BNHD) return MOA_ERR_INVALID_ARG;
@@ -120,13 +125,13 @@ moa_status check_desc(const moa_attn_desc *d)
     return MOA_OK;
 }
 
-// AUTO: the TMA bulk add-reduce where it exists (tensor-core path, d = 128: measured slightly
-// ahead of plain reds at every size), plain reds otherwise.
+// AUTO: the TMA bulk add-reduce where it exists (tensor-core path, 128-column kernel: measured
+// slightly ahead of plain reds at every size), plain reds otherwise.
 int resolved_dq_mode(const moa_attn_desc *d)
 {
     if (d->dq_mode != MOA_DQ_AUTO) return d->dq_mode;
     const bool tc = d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->scale > 0.f;
-    return (tc && d->d == 128) ? MOA_DQ_BULK_REDUCE : MOA_DQ_RED;
+    return (tc && kernel_d(d->d) == 128) ? MOA_DQ_BULK_REDUCE : MOA_DQ_RED;
 }
 
 // the tensor-core kernels take the row max before scaling, which needs scale > 0
@@ -154,7 +159,9 @@ BwdWorkspace bwd_workspace(const moa_attn_desc *d)
         w.d_bytes = align_up(rows * sizeof(float));
     }
     const bool need_acc = d->dtype == MOA_BF16 && resolved_dq_mode(d) != MOA_DQ_SEPARATE_PASS;
-    w.dqacc_bytes = need_acc ? align_up(rows * d->d * sizeof(float)) : 0;
+    // the tensor-core backward accumulates rows of its own (64 or 128) columns
+    const size_t acc_cols = use_tc_bwd(d) ? (size_t)kernel_d(d->d) : (size_t)d->d;
+    w.dqacc_bytes = need_acc ? align_up(rows * acc_cols * sizeof(float)) : 0;
     w.total = w.d_bytes + w.lp_bytes + w.dqacc_bytes;
     return w;
 }
@@ -246,9 +253,10 @@ moa_status run_bwd(const moa_attn_desc *d, const void *Q, const void *K, const v
             MOA_TRY(tc_bwd_dq(p, Q, K, V, dO, Lp, Dv, dQ, st));
             return MOA_OK;
         }
-        if (!prepared) MOA_TRY(cudaMemsetAsync(dQacc, 0, elems * sizeof(float), st));
+        const int acc_ld = kernel_d(p.d);
+        if (!prepared) MOA_TRY(cudaMemsetAsync(dQacc, 0, (size_t)p.BH() * p.n * acc_ld * sizeof(float), st));
         MOA_TRY(tc_bwd_kv(p, Q, K, V, dO, Lp, Dv, dK, dV, dQacc, mode == MOA_DQ_BULK_REDUCE, st));
-        if (p.bnhd) MOA_TRY(convert_f32_to_bf16_bnhd(dQacc, dQ, p.B, p.H, p.n, p.d, p.scale, st));
+        if (p.bnhd || acc_ld != p.d) MOA_TRY(convert_f32_to_bf16_rows(dQacc, acc_ld, dQ, p.B, p.H, p.n, p.d, p.bnhd, p.scale, st));
         else MOA_TRY(convert_f32_to_bf16(dQacc, dQ, elems, p.scale, st));
         return MOA_OK;
     }
@@ -407,6 +415,7 @@ moa_status moa_attn_fused_rowparallel(const moa_attn_desc *desc, const void *Q, 
     if (s != MOA_OK) return s;
     if (atomic_sites != 1 && atomic_sites != 2) return MOA_ERR_INVALID_ARG;
     if ((desc->H_kv > 0 && desc->H_kv != desc->H) || desc->layout != MOA_LAYOUT_BHND) return MOA_ERR_UNSUPPORTED;
+    if (desc->d != 64 && desc->d != 128) return MOA_ERR_UNSUPPORTED;          // CUDA-core kernels: d in {64, 128}
     if (!Q || !K || !V || !O || !L || !dO || !dQ || !dK || !dV) return MOA_ERR_INVALID_ARG;
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(L) || !aligned16(dO) ||
         !aligned16(dQ) || !aligned16(dK) || !aligned16(dV))

@@ -67,8 +67,9 @@ template <int D>
 __global__ void __launch_bounds__(256)
 bwd_preprocess_kernel(const __nv_bfloat16 *__restrict__ dO, const __nv_bfloat16 *__restrict__ O,
                       const float *__restrict__ L, float *__restrict__ Lp, float *__restrict__ Dp,
-                      int n, int n_pad, size_t padded_rows, int H, int bnhd)
+                      int n, int n_pad, size_t padded_rows, int H, int bnhd, int d)
 {
+    // d <= D: the head dimension in memory (lanes past it contribute zeros)
     constexpr int kLanesPerRow = D / 8;
     constexpr int kRowsPerPass = 32 / kLanesPerRow;
     constexpr int kPasses = 4;
@@ -94,8 +95,10 @@ bwd_preprocess_kernel(const __nv_bfloat16 *__restrict__ dO, const __nv_bfloat16 
                 const size_t bb = bh / (size_t)H;
                 trow = (bb * (size_t)n + r) * (size_t)H + (bh - bb * (size_t)H);
             }
-            a[p] = __ldcs(reinterpret_cast<const uint4 *>(dO + trow * D) + l);
-            b[p] = __ldcs(reinterpret_cast<const uint4 *>(O + trow * D) + l);
+            if (8 * l < d) {
+                a[p] = __ldcs(reinterpret_cast<const uint4 *>(dO + trow * (size_t)d) + l);
+                b[p] = __ldcs(reinterpret_cast<const uint4 *>(O + trow * (size_t)d) + l);
+            }
             if (l == 0) lv[p] = L[row];
         }
     }
@@ -609,12 +612,13 @@ cudaError_t launch_bwd_g(const Problem &p, const void *Q, const void *K, const v
     const uint64_t heads = (uint64_t)p.BH();
     const bool bnhd = p.bnhd != 0;
     const auto bf = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
-    if (!make_tensor_map_4d(&mq, Q, bf, 2, p.B, p.H, p.n, D, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mk, K, bf, 2, p.B, p.kv_heads(), p.n, D, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mv, V, bf, 2, p.B, p.kv_heads(), p.n, D, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mdo, dO, bf, 2, p.B, p.H, p.n, D, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mdk, dK, bf, 2, p.B, p.kv_heads(), p.n, D, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mdv, dV, bf, 2, p.B, p.kv_heads(), p.n, D, bnhd, 128, 64))
+    // p.d <= D columns exist in memory: loads fill the rest of a box with zeros, stores drop it
+    if (!make_tensor_map_4d(&mq, Q, bf, 2, p.B, p.H, p.n, p.d, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mk, K, bf, 2, p.B, p.kv_heads(), p.n, p.d, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mv, V, bf, 2, p.B, p.kv_heads(), p.n, p.d, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mdo, dO, bf, 2, p.B, p.H, p.n, p.d, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mdk, dK, bf, 2, p.B, p.kv_heads(), p.n, p.d, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mdv, dV, bf, 2, p.B, p.kv_heads(), p.n, p.d, bnhd, 128, 64))
         return cudaErrorInvalidValue;
     // fp32 accumulator as [heads, n, D] with boxes of 32 rows x D floats (no swizzle); also encoded when unused
     if (!make_tensor_map_3d(&mdq, dQacc ? (const void *)dQacc : Q, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, heads, p.n, D, 32, D))
@@ -650,24 +654,27 @@ cudaError_t tc_bwd_preprocess(const Problem &p, const void *dO, const void *O, c
     const int n_pad = (p.n + 127) / 128 * 128;
     const size_t rows = (size_t)p.BH() * n_pad;
     const int wpb = 8;
-    const size_t rows_per_block = (size_t)wpb * (32 / (p.d / 8)) * 4;   // warps x rows per pass x passes
+    const int D = kernel_d(p.d);
+    const size_t rows_per_block = (size_t)wpb * (32 / (D / 8)) * 4;   // warps x rows per pass x passes
     const unsigned grid = (unsigned)((rows + rows_per_block - 1) / rows_per_block);
     LaunchScope scope(MOA_KERNEL_PREPROCESS, st);
-    if (p.d == 64)
+    if (D == 64)
         bwd_preprocess_kernel<64><<<grid, wpb * 32, 0, st>>>((const __nv_bfloat16 *)dO, (const __nv_bfloat16 *)O, L,
-                                                             Lp, Dp, p.n, n_pad, rows, p.H, p.bnhd);
+                                                             Lp, Dp, p.n, n_pad, rows, p.H, p.bnhd, p.d);
     else
         bwd_preprocess_kernel<128><<<grid, wpb * 32, 0, st>>>((const __nv_bfloat16 *)dO, (const __nv_bfloat16 *)O, L,
-                                                              Lp, Dp, p.n, n_pad, rows, p.H, p.bnhd);
+                                                              Lp, Dp, p.n, n_pad, rows, p.H, p.bnhd, p.d);
     return cudaGetLastError();
 }
 
 cudaError_t tc_bwd_kv(const Problem &p, const void *Q, const void *K, const void *V, const void *dO,
                       const float *Lp, const float *Dp, void *dK, void *dV, float *dQacc, int dq_bulk, cudaStream_t st)
 {
-    if (p.d == 64 && !dq_bulk) return launch_bwd<64, false>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
-    if (p.d == 128 && !dq_bulk) return launch_bwd<128, false>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
-    if (p.d == 128 && dq_bulk) return launch_bwd<128, true>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
+    if (p.d < 8 || p.d > 128 || p.d % 8) return cudaErrorInvalidValue;
+    const int D = kernel_d(p.d);     // dQacc rows are D floats wide
+    if (D == 64 && !dq_bulk) return launch_bwd<64, false>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
+    if (D == 128 && !dq_bulk) return launch_bwd<128, false>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
+    if (D == 128 && dq_bulk) return launch_bwd<128, true>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
     return cudaErrorInvalidValue;
 }
 

@@ -44,7 +44,7 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
              const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapdO,
              const float *__restrict__ Lp, const float *__restrict__ Dp, __nv_bfloat16 *__restrict__ dQ,
              int n, int n_pad, int causal, float scale, float scale_log2, int nqt, int hpg,
-             int group, int H, int bnhd, unsigned int *status)
+             int group, int H, int bnhd, int d, unsigned int *status)
 {
     using SM = DqSmem<D>;
     constexpr int kBoxes = D / 64;
@@ -180,7 +180,7 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
             tc_fence_after();
             const int qrow = q0 + lane_row;
             const size_t qrow_index = bnhd ? ((size_t)bb * n + qrow) * H + hq : (size_t)bh * n + qrow;   // row of dQ in the caller's layout
-            __nv_bfloat16 *outp = dQ + qrow_index * D + (D / 2) * wg;
+            __nv_bfloat16 *outp = dQ + qrow_index * (size_t)d + (D / 2) * wg;   // d <= D columns exist in memory
 #pragma unroll
             for (int c = 0; c < D / 2; c += 32) {
                 uint32_t r[32];
@@ -194,7 +194,7 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
                         v.y = pack_bf16(__uint_as_float(r[e + 2]) * scale, __uint_as_float(r[e + 3]) * scale);
                         v.z = pack_bf16(__uint_as_float(r[e + 4]) * scale, __uint_as_float(r[e + 5]) * scale);
                         v.w = pack_bf16(__uint_as_float(r[e + 6]) * scale, __uint_as_float(r[e + 7]) * scale);
-                        *reinterpret_cast<uint4 *>(outp + c + e) = v;
+                        if ((D / 2) * wg + c + e < d) *reinterpret_cast<uint4 *>(outp + c + e) = v;
                     }
                 }
             }
@@ -212,10 +212,10 @@ cudaError_t launch_dq(const Problem &p, const void *Q, const void *K, const void
     CUtensorMap mq, mk, mv, mdo;
     const bool bnhd = p.bnhd != 0;
     const auto bf = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
-    if (!make_tensor_map_4d(&mq, Q, bf, 2, p.B, p.H, p.n, D, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mk, K, bf, 2, p.B, p.kv_heads(), p.n, D, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mv, V, bf, 2, p.B, p.kv_heads(), p.n, D, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mdo, dO, bf, 2, p.B, p.H, p.n, D, bnhd, 128, 64))
+    if (!make_tensor_map_4d(&mq, Q, bf, 2, p.B, p.H, p.n, p.d, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mk, K, bf, 2, p.B, p.kv_heads(), p.n, p.d, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mv, V, bf, 2, p.B, p.kv_heads(), p.n, p.d, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mdo, dO, bf, 2, p.B, p.H, p.n, p.d, bnhd, 128, 64))
         return cudaErrorInvalidValue;
     constexpr int kSmem = DqSmem<D>::kTotal;
     cudaError_t e = cudaFuncSetAttribute(tc_dq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
@@ -224,7 +224,7 @@ cudaError_t launch_dq(const Problem &p, const void *Q, const void *K, const void
     LaunchScope scope(MOA_KERNEL_BWD_DQ, st);
     tc_dq_kernel<D><<<(unsigned)(nqt * p.BH()), kThreads, kSmem, st>>>(
         mq, mk, mv, mdo, Lp, Dp, (__nv_bfloat16 *)dQ, p.n, nqt * 128, p.causal, p.scale, p.scale * kLog2e, nqt,
-        heads_per_group(p, nqt), p.group(), p.H, p.bnhd, device_status_ptr());
+        heads_per_group(p, nqt), p.group(), p.H, p.bnhd, p.d, device_status_ptr());
     return cudaGetLastError();
 }
 
@@ -233,9 +233,8 @@ cudaError_t launch_dq(const Problem &p, const void *Q, const void *K, const void
 cudaError_t tc_bwd_dq(const Problem &p, const void *Q, const void *K, const void *V, const void *dO,
                       const float *Lp, const float *Dp, void *dQ, cudaStream_t st)
 {
-    if (p.d == 64) return launch_dq<64>(p, Q, K, V, dO, Lp, Dp, dQ, st);
-    if (p.d == 128) return launch_dq<128>(p, Q, K, V, dO, Lp, Dp, dQ, st);
-    return cudaErrorInvalidValue;
+    if (p.d < 8 || p.d > 128 || p.d % 8) return cudaErrorInvalidValue;
+    return kernel_d(p.d) == 64 ? launch_dq<64>(p, Q, K, V, dO, Lp, Dp, dQ, st) : launch_dq<128>(p, Q, K, V, dO, Lp, Dp, dQ, st);
 }
 
 }  // namespace moa

@@ -65,6 +65,7 @@ struct FwdPrep {
     const __nv_bfloat16 *dO;
     float *Lp, *Dp;
     int n_pad, bnhd;
+    int d;               // columns of a dO row in memory (<= D)
 };
 
 template <int D>
@@ -228,7 +229,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             // fused call: the epilogue reads this thread's 128 bytes (D = 128) of its dO row; ask L2 for
             // them now so that the read at the end of the job does not wait on HBM
             const size_t drow = prep.bnhd ? ((size_t)bb * n + row) * H + hq : (size_t)bh * n + row;
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(prep.dO + drow * D + (D / 2) * h));
+            if ((D / 2) * h < prep.d) asm volatile("prefetch.global.L2 [%0];" ::"l"(prep.dO + drow * (size_t)prep.d + (D / 2) * h));
         }
         // The exp2 phase of a tile is MUFU-bound and the rest of a tile's work (TMEM load, max,
         // hand-offs) is not: start the second warpgroup a few hundred cycles late, once, so that on
@@ -327,9 +328,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         const bool want_d = prep.dO != nullptr && row < n;
         if (want_d) {
             const size_t drow = prep.bnhd ? ((size_t)bb * n + row) * H + hq : (size_t)bh * n + row;
-            const uint4 *src = reinterpret_cast<const uint4 *>(prep.dO + drow * D + (D / 2) * h);
+            const uint4 *src = reinterpret_cast<const uint4 *>(prep.dO + drow * (size_t)prep.d + (D / 2) * h);
 #pragma unroll
-            for (int k = 0; k < D / 16; ++k) dov[k] = __ldg(src + k);
+            for (int k = 0; k < D / 16; ++k)      // columns past the head dimension count as zeros
+                dov[k] = (D / 2) * h + 8 * k < prep.d ? __ldg(src + k) : make_uint4(0u, 0u, 0u, 0u);
         }
         float dpart = 0.f;
         xch[h * 128 + lane_row] = make_float2(m_used, l);
@@ -405,10 +407,11 @@ cudaError_t launch_fwd(const Problem &p, const void *Q, const void *K, const voi
     CUtensorMap mq, mk, mv, mo;
     const bool bnhd = p.bnhd != 0;
     const auto bf = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
-    if (!make_tensor_map_4d(&mq, Q, bf, 2, p.B, p.H, p.n, D, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mk, K, bf, 2, p.B, p.kv_heads(), p.n, D, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mv, V, bf, 2, p.B, p.kv_heads(), p.n, D, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mo, O, bf, 2, p.B, p.H, p.n, D, bnhd, 128, 64))
+    // p.d <= D columns exist in memory: loads fill the rest of a box with zeros, the store drops it
+    if (!make_tensor_map_4d(&mq, Q, bf, 2, p.B, p.H, p.n, p.d, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mk, K, bf, 2, p.B, p.kv_heads(), p.n, p.d, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mv, V, bf, 2, p.B, p.kv_heads(), p.n, p.d, bnhd, 128, 64) ||
+        !make_tensor_map_4d(&mo, O, bf, 2, p.B, p.H, p.n, p.d, bnhd, 128, 64))
         return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
@@ -417,7 +420,7 @@ cudaError_t launch_fwd(const Problem &p, const void *Q, const void *K, const voi
     tc_fwd_kernel<D><<<(unsigned)(nqt * p.BH()), kThreads, kSmem, st>>>(
         mq, mk, mv, mo, L, p.n, p.causal, p.scale * kLog2e, nqt, heads_per_group(p, nqt), p.group(), p.H,
         FwdSplit{p.n, 1, (p.n + BN - 1) / BN}, fb.zero_acc,
-        FwdPrep{(const __nv_bfloat16 *)fb.dO, fb.Lp, fb.Dp, nqt * BM, p.bnhd}, device_status_ptr());
+        FwdPrep{(const __nv_bfloat16 *)fb.dO, fb.Lp, fb.Dp, nqt * BM, p.bnhd, p.d}, device_status_ptr());
     return cudaGetLastError();
 }
 
@@ -442,7 +445,7 @@ cudaError_t launch_fwd_decode(int B, int Hkv, int G, int n, float scale, const v
     LaunchScope scope(MOA_KERNEL_FWD, st);
     tc_fwd_kernel<D><<<(unsigned)(B * Hkv * splits), kThreads, kSmem, st>>>(
         mq, mk, mv, mo, L_part, n, 0, scale * kLog2e, 1, 1, 1, Hkv, FwdSplit{G, splits, tiles_per_split},
-        nullptr, FwdPrep{nullptr, nullptr, nullptr, 0, 0}, device_status_ptr());
+        nullptr, FwdPrep{nullptr, nullptr, nullptr, 0, 0, D}, device_status_ptr());
     return cudaGetLastError();
 }
 
@@ -459,9 +462,8 @@ cudaError_t tc_fwd_decode(int B, int Hkv, int G, int n, int d, float scale, cons
 cudaError_t tc_fwd(const Problem &p, const void *Q, const void *K, const void *V, void *O, float *L,
                    const FwdForBwd &fb, cudaStream_t st)
 {
-    if (p.d == 64) return launch_fwd<64>(p, Q, K, V, O, L, fb, st);
-    if (p.d == 128) return launch_fwd<128>(p, Q, K, V, O, L, fb, st);
-    return cudaErrorInvalidValue;
+    if (p.d < 8 || p.d > 128 || p.d % 8) return cudaErrorInvalidValue;
+    return kernel_d(p.d) == 64 ? launch_fwd<64>(p, Q, K, V, O, L, fb, st) : launch_fwd<128>(p, Q, K, V, O, L, fb, st);
 }
 
 }  // namespace moa

@@ -87,6 +87,31 @@ def test_argument_errors_need_no_device(lib):
         mb.moa_attn_fwd(good, 0, a, a, a, a)
 
 
+def test_other_head_dimensions_argument_checks(lib):
+    """Multiples of 8 up to 128 run on the bf16 tensor-core kernels only."""
+    a = 4096
+
+    def fwd(d, **kw):
+        return mb.moa_attn_fwd(mb.make_desc(1, 2, 256, d, True, 0.1, **kw), a, a, a, a, a, check=False)
+
+    def ws(d, **kw):
+        return mb.moa_attn_workspace_bytes(mb.make_desc(1, 2, 256, d, True, 0.1, **kw), mb.MOA_OP_FUSED)
+
+    for d in (100, 4, 12, 136, 192, 256):
+        assert fwd(d) == mb.MOA_ERR_UNSUPPORTED, d
+        assert ws(d) == 0
+    assert fwd(96, dtype=mb.MOA_F32) == mb.MOA_ERR_UNSUPPORTED
+    assert fwd(96, path=mb.MOA_PATH_SIMT) == mb.MOA_ERR_UNSUPPORTED
+    assert fwd(96, materialize=1) == mb.MOA_ERR_UNSUPPORTED
+    assert fwd(32, dq_mode=mb.MOA_DQ_BULK_REDUCE) == mb.MOA_ERR_UNSUPPORTED      # 64-column kernel: no bulk reduce
+    # the accumulator rows are as wide as the kernel's head dimension
+    assert ws(96) == ws(128) and ws(40) == ws(64) and ws(72) == ws(128)
+    assert ws(96, dq_mode=mb.MOA_DQ_SEPARATE_PASS) == ws(128, dq_mode=mb.MOA_DQ_SEPARATE_PASS) < ws(96)
+    d96 = mb.make_desc(1, 2, 256, 96, True, 0.1)
+    assert mb.moa_attn_fused_rowparallel(d96, a, a, a, a, a, a, a, a, a, 1, a, ws_bytes=1 << 40,
+                                         check=False) == mb.MOA_ERR_UNSUPPORTED
+
+
 def test_shared_kv_heads_argument_checks(lib):
     a = 4096  # fake, aligned, never dereferenced: checks fail first
     def fwd(**kw):

@@ -298,6 +298,64 @@ def test_gqa_equals_replicated_kv_heads(H):
         assert mi.rel_err(a[k], summed) <= 8e-3, k     # the copies were rounded to bf16 one by one
 
 
+# ------------------------------------- head dimensions other than 64 and 128 (zero-filled columns)
+@pytest.mark.parametrize("d", [8, 32, 40, 72, 80, 96, 104, 120])
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("dq_mode", [0, 1, 2, 3])
+def test_other_head_dimensions_match_oracle(H, d, causal, dq_mode):
+    """d a multiple of 8 up to 128 runs in the 64- or 128-column tensor-core kernel: the TMA loads
+    fill the missing columns with zeros (which changes no result) and the stores drop them; the
+    direct-addressed passes (preprocess, dQ conversion, the separate dQ pass) use the true row
+    length.  Every element against the fp64 oracle, ragged n, fused and separate calls."""
+    if dq_mode == 2 and d <= 64:
+        pytest.skip("TMA bulk-reduce dQ exists in the 128-column kernel only")
+    n = 300 if d % 16 else 129
+    inp = mi.make_inputs(2, 3, n, d, seed=600 + d, dtype="bf16")
+    scale = 1.0 / math.sqrt(d)
+    ref = _oracle(inp, "bf16", causal, scale)
+    for op in ("fused", "split"):
+        got = H.run_library(inp, "bf16", causal, scale, dq_mode=dq_mode, op=op)
+        H.assert_close(got, ref, H.TOL_BF16, tag=f"d{d} n{n} causal{causal} dq{dq_mode} {op}")
+        assert mi.rel_err(got["L"], ref["L"]) <= 1e-3
+
+
+@pytest.mark.parametrize("d,dk", [(96, 128), (40, 64)])
+def test_other_head_dimension_is_bitwise_the_zero_padded_problem(H, d, dk):
+    """The same problem with the columns d..dk-1 written out as zeros in memory: identical bits in
+    the deterministic mode (the padded columns of every result are exactly zero)."""
+    B, Hh, n = 1, 2, 384
+    inp = mi.make_inputs(B, Hh, n, d, seed=640 + d, dtype="bf16")
+    pad = {k: np.concatenate([v, np.zeros((B, Hh, n, dk - d), dtype=v.dtype)], axis=3) for k, v in inp.items()}
+    for op in ("fused", "split"):
+        a = H.run_library(inp, "bf16", True, 0.11, dq_mode=3, op=op)
+        b = H.run_library(pad, "bf16", True, 0.11, dq_mode=3, op=op)
+        _same_as_zero_padded(a, b, d)
+
+
+def _same_as_zero_padded(a, b, d):
+    np.testing.assert_array_equal(a["L"], b["L"])
+    for k in ("O", "dQ", "dK", "dV"):
+        np.testing.assert_array_equal(a[k], b[k][..., :d], err_msg=k)
+        assert not b[k][..., d:].any(), k
+
+
+@pytest.mark.parametrize("layout", [0, 1])
+def test_other_head_dimension_with_shared_kv_heads_and_layouts(H, layout):
+    inp = _gqa_inputs(2, 6, 2, 333, 96, seed=671)
+    scale = 1.0 / math.sqrt(96)
+    f = H.f64_inputs(inp, "bf16")
+    ref = oracle.attn_fwd_bwd_gqa(f["Q"], f["K"], f["V"], f["dO"], True, scale)
+    for dq_mode in (0, 1, 3):
+        got = H.run_library(inp, "bf16", True, scale, dq_mode=dq_mode, layout=layout)
+        H.assert_close(got, ref, H.TOL_BF16, tag=f"d96 gqa layout{layout} dq{dq_mode}")
+
+
+def test_head_dimension_96_long_sequence_sampled(H):
+    """B1 H4 n8192 d96 causal: sampled rows and columns of the first and last head."""
+    w = mi.Workload("d96_n8192", 1, 4, 8192, 96, True, "bf16", 77)
+    _sampled_check(H, w, heads=[(0, 0), (0, 3)], nrows=12, ncols=12)
+
+
 # ------------------------------------------------------- token-major tensors [B,n,H,d]
 @pytest.mark.parametrize("causal", [False, True])
 @pytest.mark.parametrize("B,Hq,Hkv,n,d", [(2, 3, 3, 300, 128), (3, 4, 2, 257, 64), (1, 6, 1, 128, 128)])
