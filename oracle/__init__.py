@@ -14,3 +14,4 @@ from .attention import (  # noqa: F401
     attn_cols,
 )
 from .decode import decode_attn  # noqa: F401,E402
+from .block import rmsnorm_fwd_bwd, gated_mlp_fwd_bwd, gated_mlp_bwd_from_saved  # noqa: F401,E402
