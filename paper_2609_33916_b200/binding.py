@@ -28,6 +28,8 @@ EXPORTS = (
     "moa_last_device_status", "moa_launch_count", "moa_status_string", "moa_version",
     "moa_profile_enable", "moa_profile_read", "moa_attn_bwd_static_scratch", "moa_attn_fused_rowparallel",
     "moa_decode_workspace_bytes", "moa_decode_attn",
+    "moa_rmsnorm_workspace_bytes", "moa_rmsnorm_fwd", "moa_rmsnorm_bwd",
+    "moa_gated_mlp_fwd", "moa_gated_mlp_workspace_bytes", "moa_gated_mlp_bwd",
 )
 
 
@@ -41,6 +43,14 @@ class moa_attn_desc(ctypes.Structure):
 class moa_decode_desc(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("H_kv", ctypes.c_int32), ("n", ctypes.c_int32),
                 ("d", ctypes.c_int32), ("scale", ctypes.c_float), ("dtype", ctypes.c_int32)]
+
+
+class moa_rmsnorm_desc(ctypes.Structure):
+    _fields_ = [("n", ctypes.c_int32), ("d", ctypes.c_int32), ("eps", ctypes.c_float), ("dtype", ctypes.c_int32)]
+
+
+class moa_mlp_desc(ctypes.Structure):
+    _fields_ = [("n", ctypes.c_int32), ("d", ctypes.c_int32), ("d_ff", ctypes.c_int32), ("dtype", ctypes.c_int32)]
 
 
 MOA_KERNEL_KINDS = 6
@@ -85,6 +95,20 @@ def lib() -> ctypes.CDLL:
         L.moa_decode_workspace_bytes.argtypes = [ctypes.POINTER(moa_decode_desc)]
         L.moa_decode_attn.restype = ctypes.c_int
         L.moa_decode_attn.argtypes = [ctypes.POINTER(moa_decode_desc)] + [vp] * 5 + [vp, sz, vp]
+        rp = ctypes.POINTER(moa_rmsnorm_desc)
+        L.moa_rmsnorm_workspace_bytes.restype = sz
+        L.moa_rmsnorm_workspace_bytes.argtypes = [rp]
+        L.moa_rmsnorm_fwd.restype = ctypes.c_int
+        L.moa_rmsnorm_fwd.argtypes = [rp] + [vp] * 4 + [vp]
+        L.moa_rmsnorm_bwd.restype = ctypes.c_int
+        L.moa_rmsnorm_bwd.argtypes = [rp] + [vp] * 6 + [vp, sz, vp]
+        mp = ctypes.POINTER(moa_mlp_desc)
+        L.moa_gated_mlp_workspace_bytes.restype = sz
+        L.moa_gated_mlp_workspace_bytes.argtypes = [mp]
+        L.moa_gated_mlp_fwd.restype = ctypes.c_int
+        L.moa_gated_mlp_fwd.argtypes = [mp] + [vp] * 8 + [vp]
+        L.moa_gated_mlp_bwd.restype = ctypes.c_int
+        L.moa_gated_mlp_bwd.argtypes = [mp] + [vp] * 12 + [vp, sz, vp]
         L.moa_last_device_status.restype = ctypes.c_int
         L.moa_last_device_status.argtypes = [vp]
         L.moa_launch_count.restype = ctypes.c_uint64
@@ -193,6 +217,55 @@ def moa_attn_fused_rowparallel(desc, Q, K, V, dO, O, L, dQ, dK, dV, atomic_sites
                                          _nbytes(ws) if ws_bytes is None else ws_bytes, _stream(stream))
     if check and s != MOA_OK:
         raise MoaError(s, "moa_attn_fused_rowparallel")
+    return s
+
+
+def make_rmsnorm_desc(n, d, eps, dtype=MOA_BF16) -> moa_rmsnorm_desc:
+    return moa_rmsnorm_desc(int(n), int(d), float(eps), int(dtype))
+
+
+def moa_rmsnorm_workspace_bytes(desc) -> int:
+    return int(lib().moa_rmsnorm_workspace_bytes(ctypes.byref(desc)))
+
+
+def moa_rmsnorm_fwd(desc, x, g, y, r=None, stream=None, check=True) -> int:
+    s = lib().moa_rmsnorm_fwd(ctypes.byref(desc), _ptr(x), _ptr(g), _ptr(y), _ptr(r), _stream(stream))
+    if check and s != MOA_OK:
+        raise MoaError(s, "moa_rmsnorm_fwd")
+    return s
+
+
+def moa_rmsnorm_bwd(desc, x, g, r, dy, dx, dg, ws=None, stream=None, ws_bytes=None, check=True) -> int:
+    s = lib().moa_rmsnorm_bwd(ctypes.byref(desc), _ptr(x), _ptr(g), _ptr(r), _ptr(dy), _ptr(dx), _ptr(dg), _ptr(ws),
+                              _nbytes(ws) if ws_bytes is None else ws_bytes, _stream(stream))
+    if check and s != MOA_OK:
+        raise MoaError(s, "moa_rmsnorm_bwd")
+    return s
+
+
+def make_mlp_desc(n, d, d_ff, dtype=MOA_BF16) -> moa_mlp_desc:
+    return moa_mlp_desc(int(n), int(d), int(d_ff), int(dtype))
+
+
+def moa_gated_mlp_workspace_bytes(desc) -> int:
+    return int(lib().moa_gated_mlp_workspace_bytes(ctypes.byref(desc)))
+
+
+def moa_gated_mlp_fwd(desc, x, W1, W3, W2, a, u, h, y, stream=None, check=True) -> int:
+    s = lib().moa_gated_mlp_fwd(ctypes.byref(desc), _ptr(x), _ptr(W1), _ptr(W3), _ptr(W2), _ptr(a), _ptr(u), _ptr(h),
+                                _ptr(y), _stream(stream))
+    if check and s != MOA_OK:
+        raise MoaError(s, "moa_gated_mlp_fwd")
+    return s
+
+
+def moa_gated_mlp_bwd(desc, x, W1, W3, W2, a, u, h, dy, dx, dW1, dW3, dW2, ws=None, stream=None, ws_bytes=None,
+                      check=True) -> int:
+    s = lib().moa_gated_mlp_bwd(ctypes.byref(desc), _ptr(x), _ptr(W1), _ptr(W3), _ptr(W2), _ptr(a), _ptr(u), _ptr(h),
+                                _ptr(dy), _ptr(dx), _ptr(dW1), _ptr(dW3), _ptr(dW2), _ptr(ws),
+                                _nbytes(ws) if ws_bytes is None else ws_bytes, _stream(stream))
+    if check and s != MOA_OK:
+        raise MoaError(s, "moa_gated_mlp_bwd")
     return s
 
 

@@ -85,6 +85,21 @@ struct LaunchScope {
 // Device address of the status word kernels write when a bounded wait expires.
 unsigned int *device_status_ptr();
 
+// MOA_OK when the current device is compute capability 10.x, MOA_ERR_ARCH otherwise (cached per device).
+moa_status check_device_arch();
+
+// ---- block pieces (block_norm.cu, tc_gemm.cu), bf16 ------------------------------------
+size_t rmsnorm_workspace_bytes(int n, int d);          // per-CTA partial sums of dg
+cudaError_t rmsnorm_fwd(int n, int d, float eps, const void *x, const void *g, void *y, float *r, cudaStream_t st);
+cudaError_t rmsnorm_bwd(int n, int d, float eps, const void *x, const void *g, const float *r, const void *dy,
+                        void *dx, void *dg, void *ws, cudaStream_t st);
+// gated MLP (tc_gemm.cu): x, y, dy, dx [n,d]; W1, W3 [d_ff,d]; W2 [d,d_ff]; a, u, h, da, du [n,d_ff]
+cudaError_t gated_mlp_fwd(int n, int d, int dff, const void *x, const void *W1, const void *W3, const void *W2,
+                          void *a, void *u, void *h, void *y, cudaStream_t st);
+cudaError_t gated_mlp_bwd(int n, int d, int dff, const void *x, const void *W1, const void *W3, const void *W2,
+                          const void *a, const void *u, const void *h, const void *dy, void *da, void *du,
+                          void *dx, void *dW1, void *dW3, void *dW2, cudaStream_t st);
+
 template <typename T> __device__ __forceinline__ float to_float(T v);
 template <> __device__ __forceinline__ float to_float<float>(float v) { return v; }
 template <> __device__ __forceinline__ float to_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }

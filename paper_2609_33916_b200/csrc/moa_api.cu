@@ -297,6 +297,9 @@ void *static_scratch_ptr()
 }
 
 }  // namespace
+
+moa_status check_device_arch() { return check_arch(); }
+
 }  // namespace moa
 
 using namespace moa;

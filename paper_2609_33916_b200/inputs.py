@@ -97,6 +97,27 @@ def make_workload_inputs(w: Workload) -> dict:
     return make_inputs(w.B, w.H, w.n, w.d, w.seed, w.dtype)
 
 
+def make_norm_inputs(n: int, d: int, seed: int) -> dict:
+    """RMSNorm inputs as bf16 bit patterns: x, dy [n,d] ~ N(0,1) and a gain g [d] ~ 1 + 0.25 N(0,1)."""
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((n, d), dtype=np.float32)
+    g = (1.0 + 0.25 * rng.standard_normal(d)).astype(np.float32)
+    dy = rng.standard_normal((n, d), dtype=np.float32)
+    return {k: f32_to_bf16_bits(v) for k, v in dict(x=x, g=g, dy=dy).items()}
+
+
+def make_mlp_inputs(n: int, d: int, d_ff: int, seed: int) -> dict:
+    """Gated-MLP inputs as bf16 bit patterns: x, dy [n,d] ~ N(0,1); W1, W3 [d_ff,d] ~ N(0,1/d) and
+    W2 [d,d_ff] ~ N(0,1/d_ff) (so that the pre-activations and y have unit scale)."""
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((n, d), dtype=np.float32)
+    W1 = rng.standard_normal((d_ff, d), dtype=np.float32) / np.float32(np.sqrt(d))
+    W3 = rng.standard_normal((d_ff, d), dtype=np.float32) / np.float32(np.sqrt(d))
+    W2 = rng.standard_normal((d, d_ff), dtype=np.float32) / np.float32(np.sqrt(d_ff))
+    dy = rng.standard_normal((n, d), dtype=np.float32)
+    return {k: f32_to_bf16_bits(v) for k, v in dict(x=x, W1=W1, W3=W3, W2=W2, dy=dy).items()}
+
+
 def rel_err(got: np.ndarray, ref: np.ndarray) -> float:
     """The parity metric: max|got - ref| / max|ref| over a whole tensor."""
     ref = np.asarray(ref, dtype=np.float64)

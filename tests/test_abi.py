@@ -19,7 +19,7 @@ def lib():
 
 
 def test_header_symbols_are_exported(lib):
-    hdr = open(os.path.join(ROOT, "include", "moa_attn.h")).read()
+    hdr = "".join(open(os.path.join(ROOT, "include", h)).read() for h in ("moa_attn.h", "moa_block.h"))
     declared = set(re.findall(r"\b(moa_[a-z_0-9]+)\s*\(", hdr))
     assert declared == set(mb.EXPORTS), declared ^ set(mb.EXPORTS)
     for name in declared:
@@ -157,3 +157,34 @@ def test_decode_argument_checks(lib):
     need = mb.moa_decode_workspace_bytes(d)
     assert 0 < need <= 1024 * 2 * 8 * 130 * 4                 # segments x heads x (d + 2) floats: independent of n beyond the cap
     assert call(d, wsb=need - 1) == mb.MOA_ERR_WORKSPACE
+
+
+def test_block_piece_argument_checks(lib):
+    a = 4096
+    assert ctypes.sizeof(mb.moa_rmsnorm_desc) == 16 and ctypes.sizeof(mb.moa_mlp_desc) == 16
+    good = mb.make_rmsnorm_desc(100, 512, 1e-5)
+    assert mb.moa_rmsnorm_workspace_bytes(good) > 0
+    assert mb.moa_rmsnorm_fwd(good, 0, a, a, None, check=False) == mb.MOA_ERR_INVALID_ARG
+    assert mb.moa_rmsnorm_fwd(good, a + 4, a, a, None, check=False) == mb.MOA_ERR_INVALID_ARG
+    assert mb.moa_rmsnorm_bwd(good, a, a, None, a, a, a, None, check=False) == mb.MOA_ERR_WORKSPACE
+    assert mb.moa_rmsnorm_bwd(good, a, a, None, a, a, a, a, ws_bytes=8, check=False) == mb.MOA_ERR_WORKSPACE
+    for n, d, eps, dt, want in ((0, 512, 1e-5, mb.MOA_BF16, mb.MOA_ERR_INVALID_ARG),
+                                (10, 100, 1e-5, mb.MOA_BF16, mb.MOA_ERR_UNSUPPORTED),
+                                (10, 16384, 1e-5, mb.MOA_BF16, mb.MOA_ERR_UNSUPPORTED),
+                                (10, 512, -1.0, mb.MOA_BF16, mb.MOA_ERR_INVALID_ARG),
+                                (10, 512, float("nan"), mb.MOA_BF16, mb.MOA_ERR_INVALID_ARG),
+                                (10, 512, 1e-5, mb.MOA_F32, mb.MOA_ERR_UNSUPPORTED)):
+        d_ = mb.make_rmsnorm_desc(n, d, eps, dt)
+        assert mb.moa_rmsnorm_fwd(d_, a, a, a, None, check=False) == want, (n, d, eps, dt)
+        assert mb.moa_rmsnorm_workspace_bytes(d_) == 0
+    m = mb.make_mlp_desc(256, 512, 2048)
+    assert mb.moa_gated_mlp_workspace_bytes(m) == 2 * 256 * 2048 * 2
+    assert mb.moa_gated_mlp_fwd(m, a, a, a, a, a, a, a, 0, check=False) == mb.MOA_ERR_INVALID_ARG
+    assert mb.moa_gated_mlp_bwd(m, *([a] * 12), None, check=False) == mb.MOA_ERR_WORKSPACE
+    for n, d, dff, dt, want in ((0, 512, 2048, mb.MOA_BF16, mb.MOA_ERR_INVALID_ARG),
+                                (16, 100, 2048, mb.MOA_BF16, mb.MOA_ERR_UNSUPPORTED),
+                                (16, 512, 2044, mb.MOA_BF16, mb.MOA_ERR_UNSUPPORTED),
+                                (16, 512, 2048, mb.MOA_F32, mb.MOA_ERR_UNSUPPORTED)):
+        m_ = mb.make_mlp_desc(n, d, dff, dt)
+        assert mb.moa_gated_mlp_fwd(m_, *([a] * 8), check=False) == want, (n, d, dff, dt)
+        assert mb.moa_gated_mlp_workspace_bytes(m_) == 0

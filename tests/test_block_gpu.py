@@ -1,0 +1,159 @@
+"""Block pieces (RMSNorm, gated MLP; include/moa_block.h) against the fp64 oracle, through the C ABI.
+Bar: max|err|/max|ref| <= 1e-2 per output (bf16 storage, fp32 arithmetic)."""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+import oracle
+from paper_2609_33916_b200 import inputs as mi
+
+TOL = 1e-2
+
+
+@pytest.fixture(scope="module")
+def rt():
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2609_33916_b200 import binding as mb
+    from paper_2609_33916_b200 import build
+    build.build()
+    mb.lib()
+    return torch, mb
+
+
+def _dev(torch, bits):
+    return torch.from_numpy(np.ascontiguousarray(bits)).view(torch.bfloat16).cuda()
+
+
+def _host(t):
+    return t.float().cpu().numpy().astype(np.float64)
+
+
+def _nan_like(torch, shape, dtype=None):
+    return torch.full(shape, float("nan"), dtype=dtype or torch.bfloat16, device="cuda")
+
+
+# ------------------------------------------------------------------------------ RMSNorm
+def _run_rmsnorm(rt, inp, eps, give_r=True):
+    torch, mb = rt
+    n, d = inp["x"].shape
+    x, g, dy = (_dev(torch, inp[k]) for k in ("x", "g", "dy"))
+    desc = mb.make_rmsnorm_desc(n, d, eps)
+    y, dx = _nan_like(torch, (n, d)), _nan_like(torch, (n, d))
+    dg = _nan_like(torch, (d,))
+    r = _nan_like(torch, (n,), torch.float32)
+    ws = torch.full((max(mb.moa_rmsnorm_workspace_bytes(desc), 16),), 0xFF, dtype=torch.uint8, device="cuda")
+    mb.moa_rmsnorm_fwd(desc, x, g, y, r)
+    mb.moa_rmsnorm_bwd(desc, x, g, r if give_r else None, dy, dx, dg, ws)
+    assert mb.moa_last_device_status() == mb.MOA_OK
+    return dict(y=_host(y), r=_host(r), dx=_host(dx), dg=_host(dg))
+
+
+@pytest.mark.parametrize("n,d", [(1, 8), (5, 64), (33, 128), (257, 768), (100, 1024), (64, 2048), (70, 2056),
+                                 (19, 4096), (9, 5120), (7, 8192), (3000, 512), (4099, 2048)])
+@pytest.mark.parametrize("eps", [1e-5, 0.5])
+def test_rmsnorm_matches_oracle(rt, n, d, eps):
+    inp = mi.make_norm_inputs(n, d, seed=1000 + n + d)
+    f = {k: mi.to_f64(v, "bf16") for k, v in inp.items()}
+    ref = oracle.rmsnorm_fwd_bwd(f["x"], f["g"], f["dy"], eps)
+    for give_r in (True, False):
+        got = _run_rmsnorm(rt, inp, eps, give_r)
+        for k in ("y", "dx", "dg"):
+            assert np.all(np.isfinite(got[k])), k
+            assert mi.rel_err(got[k], ref[k]) <= TOL, (k, n, d, mi.rel_err(got[k], ref[k]))
+        assert mi.rel_err(got["r"], ref["r"]) <= 1e-5
+
+
+def test_rmsnorm_is_bitwise_reproducible(rt):
+    inp = mi.make_norm_inputs(5000, 1024, seed=3)
+    a = _run_rmsnorm(rt, inp, 1e-6)
+    b = _run_rmsnorm(rt, inp, 1e-6)
+    for k in ("y", "dx", "dg", "r"):
+        np.testing.assert_array_equal(a[k], b[k], err_msg=k)
+
+
+def test_rmsnorm_rows_far_from_unit_scale(rt):
+    """Rows scaled by 2^-20 .. 2^20: the normalised output does not change (eps = 0) and nothing overflows."""
+    inp = mi.make_norm_inputs(64, 512, seed=4)
+    x = mi.bf16_bits_to_f32(inp["x"])
+    scales = np.float32(2.0) ** np.arange(-20, 44)[:64].clip(-20, 20).astype(np.float32)
+    inp2 = dict(inp, x=mi.f32_to_bf16_bits(x * scales[:, None]))     # powers of two: exact in bf16
+    a = _run_rmsnorm(rt, inp, 0.0)
+    b = _run_rmsnorm(rt, inp2, 0.0)
+    np.testing.assert_allclose(b["y"], a["y"], rtol=1e-2, atol=1e-2)
+    f = {k: mi.to_f64(v, "bf16") for k, v in inp2.items()}
+    ref = oracle.rmsnorm_fwd_bwd(f["x"], f["g"], f["dy"], 0.0)
+    assert mi.rel_err(b["dg"], ref["dg"]) <= TOL
+    # dx rows scale like 1/row scale: compare row by row
+    for i in range(64):
+        assert mi.rel_err(b["dx"][i], ref["dx"][i]) <= TOL, i
+
+
+# ---------------------------------------------------------------------------- gated MLP
+def _run_mlp(rt, inp):
+    torch, mb = rt
+    n, d = inp["x"].shape
+    dff = inp["W1"].shape[0]
+    x, W1, W3, W2, dy = (_dev(torch, inp[k]) for k in ("x", "W1", "W3", "W2", "dy"))
+    desc = mb.make_mlp_desc(n, d, dff)
+    a, u, h = (_nan_like(torch, (n, dff)) for _ in range(3))
+    y, dx = _nan_like(torch, (n, d)), _nan_like(torch, (n, d))
+    dW1, dW3, dW2 = _nan_like(torch, (dff, d)), _nan_like(torch, (dff, d)), _nan_like(torch, (d, dff))
+    ws = torch.full((max(mb.moa_gated_mlp_workspace_bytes(desc), 16),), 0xFF, dtype=torch.uint8, device="cuda")
+    mb.moa_gated_mlp_fwd(desc, x, W1, W3, W2, a, u, h, y)
+    mb.moa_gated_mlp_bwd(desc, x, W1, W3, W2, a, u, h, dy, dx, dW1, dW3, dW2, ws)
+    assert mb.moa_last_device_status() == mb.MOA_OK
+    return {k: _host(v) for k, v in dict(a=a, u=u, h=h, y=y, dx=dx, dW1=dW1, dW3=dW3, dW2=dW2).items()}
+
+
+MLP_CASES = [
+    (128, 64, 256),          # one tile everywhere; the sizes of the paper's own traffic check (n = 512 there)
+    (512, 64, 256),
+    (1, 8, 8),               # smallest
+    (130, 72, 264),          # ragged in every dimension
+    (300, 512, 1024),
+    (1000, 256, 2048),       # several tiles, K of the weight-gradient GEMMs not a multiple of 64
+    (2048, 1024, 4096),
+]
+
+
+@pytest.mark.parametrize("n,d,dff", MLP_CASES)
+def test_gated_mlp_matches_oracle(rt, n, d, dff):
+    inp = mi.make_mlp_inputs(n, d, dff, seed=2000 + n + d)
+    f = {k: mi.to_f64(v, "bf16") for k, v in inp.items()}
+    ref = oracle.gated_mlp_fwd_bwd(f["x"], f["W1"], f["W3"], f["W2"], f["dy"])
+    got = _run_mlp(rt, inp)
+    for k in ("a", "u", "h", "y", "dx", "dW1", "dW3", "dW2"):
+        assert np.all(np.isfinite(got[k])), k
+        e = mi.rel_err(got[k], ref[k])
+        assert e <= TOL, (k, n, d, dff, e)
+
+
+def test_gated_mlp_backward_from_its_stored_activations(rt):
+    """The backward reads the bf16 a, u, h its forward stored: against the oracle's backward evaluated on
+    exactly those stored values, the gradients agree more closely than against the one-piece definition."""
+    n, d, dff = 384, 256, 768
+    inp = mi.make_mlp_inputs(n, d, dff, seed=77)
+    f = {k: mi.to_f64(v, "bf16") for k, v in inp.items()}
+    got = _run_mlp(rt, inp)
+    ref = oracle.gated_mlp_bwd_from_saved(f["x"], got["a"], got["u"], f["W1"], f["W3"], f["W2"], f["dy"])
+    for k in ("dx", "dW1", "dW3"):
+        assert mi.rel_err(got[k], ref[k]) <= 6e-3, (k, mi.rel_err(got[k], ref[k]))
+    # dW2 = dy^T h with the stored h
+    assert mi.rel_err(got["dW2"], f["dy"].T @ got["h"]) <= 6e-3
+
+
+def test_gated_mlp_large_preactivations(rt):
+    """Weights scaled so that |a| reaches the hundreds: the sigmoid saturates without NaN or inf."""
+    n, d, dff = 256, 128, 512
+    inp = mi.make_mlp_inputs(n, d, dff, seed=88)
+    w1 = mi.bf16_bits_to_f32(inp["W1"]) * np.float32(64.0)
+    inp = dict(inp, W1=mi.f32_to_bf16_bits(w1))
+    f = {k: mi.to_f64(v, "bf16") for k, v in inp.items()}
+    ref = oracle.gated_mlp_fwd_bwd(f["x"], f["W1"], f["W3"], f["W2"], f["dy"])
+    got = _run_mlp(rt, inp)
+    for k in ("h", "y", "dx", "dW1", "dW3", "dW2"):
+        assert np.all(np.isfinite(got[k])), k
+        assert mi.rel_err(got[k], ref[k]) <= TOL, (k, mi.rel_err(got[k], ref[k]))
