@@ -303,6 +303,157 @@ def run_decode(args):
     return 0
 
 
+BLOCK_WORKLOADS = {
+    # name: (piece, n tokens, d, d_ff)
+    "rmsnorm_n65536_d2048": ("rmsnorm", 65536, 2048, 0),           # the paper's longest RMSNorm sweep point, a model-sized row
+    "rmsnorm_n65536_d4096": ("rmsnorm", 65536, 4096, 0),
+    "mlp_n16384_d2048_ff8192": ("mlp", 16384, 2048, 8192),          # config 4's tokens, 16 heads x 128, d_ff = 4 d
+    "mlp_n8192_d4096_ff16384": ("mlp", 8192, 4096, 16384),
+    "mlp_paper_n512_d64_ff256": ("mlp", 512, 64, 256),              # the paper's own traffic-check size (B=2, N=256, D=64, DFF=256)
+}
+
+
+def run_block(args):
+    """Block pieces (RMSNorm, gated MLP): one step = forward + backward of the piece.  Further bench
+    lines, not the contract's default.  RMSNorm is HBM-bound (roofline: algorithmic bytes against
+    the measured copy bandwidth), the gated MLP is a dense contraction (model FLOPs against the
+    measured dense bf16 peak)."""
+    import numpy as np
+    import torch
+    from paper_2609_33916_b200 import binding as mb
+    from paper_2609_33916_b200 import build as mbuild
+    import oracle
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    piece, n, d, dff = BLOCK_WORKLOADS[args.block]
+    mbuild.build()
+    mb.lib()
+    peaks, peaks_kind = load_peaks()
+    bf = torch.bfloat16
+    gen = torch.Generator(device="cuda").manual_seed(17)
+    stream = torch.cuda.current_stream()
+    rnd = lambda *shape, s=1.0: (torch.randn(shape, generator=gen, device="cuda") * s).to(bf)
+    x, dy = rnd(n, d), rnd(n, d)
+    dx = torch.empty_like(x)
+    if piece == "rmsnorm":
+        eps = 1e-5
+        g = (1.0 + 0.25 * torch.randn((d,), generator=gen, device="cuda")).to(bf)
+        y, dg = torch.empty_like(x), torch.empty_like(g)
+        r = torch.empty((n,), dtype=torch.float32, device="cuda")
+        desc = mb.make_rmsnorm_desc(n, d, eps)
+        ws = torch.empty(max(mb.moa_rmsnorm_workspace_bytes(desc), 16), dtype=torch.uint8, device="cuda")
+
+        def step():
+            mb.moa_rmsnorm_fwd(desc, x, g, y, r, stream)
+            mb.moa_rmsnorm_bwd(desc, x, g, r, dy, dx, dg, ws, stream)
+
+        # forward: read x, write y, r; backward: read x, dy, r, write dx (+ g, dg and the dg partials: O(d))
+        alg = 5.0 * n * d * 2 + 8.0 * n
+        unit, kernel = "GB/s", "rmsnorm_bwd_kernel"
+        metric = "RMSNorm forward+backward: GB/s of algorithmic bytes"
+    else:
+        W1, W3 = rnd(dff, d, s=1.0 / math.sqrt(d)), rnd(dff, d, s=1.0 / math.sqrt(d))
+        W2 = rnd(d, dff, s=1.0 / math.sqrt(dff))
+        a, u, h = (torch.empty((n, dff), dtype=bf, device="cuda") for _ in range(3))
+        y = torch.empty_like(x)
+        dW1, dW3, dW2 = torch.empty_like(W1), torch.empty_like(W3), torch.empty_like(W2)
+        desc = mb.make_mlp_desc(n, d, dff)
+        ws = torch.empty(max(mb.moa_gated_mlp_workspace_bytes(desc), 16), dtype=torch.uint8, device="cuda")
+
+        def step():
+            mb.moa_gated_mlp_fwd(desc, x, W1, W3, W2, a, u, h, y, stream)
+            mb.moa_gated_mlp_bwd(desc, x, W1, W3, W2, a, u, h, dy, dx, dW1, dW3, dW2, ws, stream)
+
+        alg = 18.0 * n * d * dff           # 3 GEMMs forward, 6 backward, 2 n d d_ff each
+        unit, kernel = "TFLOP/s", "tc_gemm_kernel"
+        metric = "gated MLP forward+backward: model TFLOP/s (18 n d d_ff per step)"
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(physical_gpu_index(0))
+    sampler.start()
+    l0 = mb.moa_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    sampler.stop()
+    launches = mb.moa_launch_count() - l0
+    ms = e0.elapsed_time(e1) / args.steps
+    value = alg / (ms * 1e-3) / (1e9 if piece == "rmsnorm" else 1e12)
+    # end to end: the step's activations (x, dy) come from pinned host memory, dx goes back; weights stay resident
+    hx, hdy = x.cpu().pin_memory(), dy.cpu().pin_memory()
+    hdx = torch.empty((n, d), dtype=bf).pin_memory()
+    t0e, t1e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    esteps = max(4, min(args.steps, 10))
+    t0e.record(stream)
+    for _ in range(esteps):
+        x.copy_(hx, non_blocking=True)
+        dy.copy_(hdy, non_blocking=True)
+        step()
+        hdx.copy_(dx, non_blocking=True)
+    t1e.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = t0e.elapsed_time(t1e) / esteps
+    st = mb.moa_last_device_status(stream)
+    if st != mb.MOA_OK:
+        raise SystemExit(f"device status: {mb.status_string(st)}")
+    if piece == "rmsnorm":
+        roof = {"bound": "hbm", "kernel": kernel, "achieved": value, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": value / peaks["hbm_gbs"], "traffic": None, "peak_source": f"{peaks_kind} hbm_gbs (copy bandwidth)",
+                "algorithmic_bytes_per_step": alg,
+                "note": "whole step (forward, backward, dg reduction) against the copy bandwidth"}
+    else:
+        roof = {"bound": "tensor", "kernel": kernel, "achieved": value, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": value / peaks["bf16_tflops"], "traffic": None,
+                "peak_source": f"{peaks_kind} bf16_tflops (cuBLAS burst)",
+                "frac_of_sustained": value / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
+                "model_flops_per_step": alg,
+                "note": "whole step (the nine GEMMs of forward and backward) against the dense bf16 peak"}
+    line = {
+        "metric": metric, "value": value, "unit": unit, "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": args.block, "n": n, "d": d, "d_ff": dff,
+                   "l2": "the arrays of one step exceed the 126 MB L2; no explicit flush" if n * d * 10 > 126e6 or n * dff * 2 > 126e6
+                   else "small case: resident in L2 between steps (not a bandwidth figure)"},
+        "tokens_per_s": n / (ms * 1e-3),
+        "clocks": sampler.summary(),
+        "e2e": {"value": alg / (e2e_ms * 1e-3) / (1e9 if piece == "rmsnorm" else 1e12), "unit": unit,
+                "h2d_bytes_per_step": 2 * n * d * 2, "d2h_bytes_per_step": n * d * 2, "ms_per_step": e2e_ms,
+                "how": "x and dy from pinned host memory and dx back every step; gain / weights resident"},
+        "gpu_launches": int(launches),
+        "roofline": roof,
+    }
+    if not args.no_cpu_baseline:
+        rows = 4096 if piece == "rmsnorm" else (64 if d * dff > 1 << 20 else n)
+        f64 = lambda t: t.float().cpu().numpy().astype(np.float64)
+        t0 = time.perf_counter()
+        reps = 0
+        if piece == "rmsnorm":
+            xs, gs, ds = f64(x[:rows]), f64(g), f64(dy[:rows])
+            while time.perf_counter() - t0 < 5.0:
+                oracle.rmsnorm_fwd_bwd(xs, gs, ds, eps)
+                reps += 1
+        else:
+            xs, ds, w1, w3, w2 = f64(x[:rows]), f64(dy[:rows]), f64(W1), f64(W3), f64(W2)
+            t0 = time.perf_counter()
+            while time.perf_counter() - t0 < 10.0:
+                oracle.gated_mlp_fwd_bwd(xs, w1, w3, w2, ds)
+                reps += 1
+        dt = (time.perf_counter() - t0) / reps
+        sample = alg * rows / n
+        line["cpu_baseline"] = {"value": sample / dt / (1e9 if piece == "rmsnorm" else 1e12), "unit": unit,
+                                "cores": os.cpu_count(), "kind": "oracle",
+                                "sample": f"{rows} of {n} tokens (all columns / full weights), numpy fp64", "seconds": dt * reps}
+    print(json.dumps(line))
+    return 0
+
+
 # ----------------------------------------------------------------------------- sweep
 def run_sweep(args):
     """Config-5 style sweep: for each n and each strategy (the three dQ modes of the fused path
@@ -394,6 +545,8 @@ def main():
                     help="record the step into a CUDA graph once and time replays (launch-bound small sizes)")
     ap.add_argument("--decode", default="", choices=[""] + sorted(DECODE_WORKLOADS),
                     help="time decode attention on that workload instead of the fused forward+backward")
+    ap.add_argument("--block", default="", choices=[""] + sorted(BLOCK_WORKLOADS),
+                    help="time a block piece (RMSNorm or gated MLP, forward+backward) instead of the attention step")
     ap.add_argument("--rowparallel", type=int, default=0,
                     help="1 or 2: time the row-parallel single-kernel comparison variant with that many atomic sites")
     ap.add_argument("--layout", type=int, default=0, help="0: tensors [B,H,n,d] (every named config); 1: [B,n,H,d]")
@@ -409,6 +562,8 @@ def main():
 
     if args.decode:
         return run_decode(args)
+    if args.block:
+        return run_block(args)
     from paper_2609_33916_b200 import inputs as mi
     w = mi.CONFIGS[args.workload]
     if args.impl == "reference":

@@ -1,12 +1,12 @@
 // RMSNorm forward and backward (bf16 storage, fp32 arithmetic).  HBM-bound: x is read once and y
 // written once by the forward; the backward reads x and dy once and writes dx once.
 //
-// Thread layout (both kernels): a row is covered by `tpr` threads (a power of two, 1..256, at least
-// d/8), each owning the 16-byte vectors v = c, c + tpr, ... of the row (kV of them at most), so a
-// thread always touches the same columns and keeps the gain -- and, in the backward, its share of
-// the dg sums -- in registers.  The 256 threads of a CTA form 256/tpr row lanes, and a lane takes R
-// rows per iteration (R*kV = 8 vectors of x in flight per thread).  Row sums are reduced by
-// shuffles inside a warp and, for tpr > 32, through shared memory across the warps of the lane.
+// Thread layout (both kernels): a row is covered by `tpr` threads (a power of two, 1..256), each
+// owning the 16-byte vectors v = c, c + tpr, ... of the row (kV of them at most), so a thread always
+// touches the same columns and keeps the gain -- and, in the backward, its share of the dg sums --
+// in registers.  The 256 threads of a CTA form 256/tpr row lanes, and a lane takes R rows per
+// iteration.  Row sums are reduced by shuffles inside a warp and, for tpr > 32, through shared
+// memory across the warps of the lane.  Two iterations are kept in registers (see below).
 #include "common.cuh"
 #include "moa_block.h"
 
@@ -64,6 +64,30 @@ __device__ __forceinline__ void lane_sum(float (&v)[R], int tpr, float *red)
     }
 }
 
+// Rows of one iteration of one row lane, as the raw 16-byte vectors this thread owns.
+template <int kV, int R>
+struct RowRegs {
+    uint4 v[R][kV];
+};
+
+template <int kV, int R>
+__device__ __forceinline__ void load_rows(RowRegs<kV, R> &dst, const __nv_bfloat16 *__restrict__ src, long long row0,
+                                          int n, int d, int c, int tpr)
+{
+    const int nvec = d / 8;
+#pragma unroll
+    for (int i = 0; i < R; ++i)
+#pragma unroll
+        for (int j = 0; j < kV; ++j) {
+            const int v = c + j * tpr;
+            dst.v[i][j] = make_uint4(0u, 0u, 0u, 0u);
+            if (row0 + i < n && v < nvec) dst.v[i][j] = __ldcs(reinterpret_cast<const uint4 *>(src + (size_t)(row0 + i) * d) + v);
+        }
+}
+
+// Both kernels keep two iterations in registers: the loads of iteration it + 1 are issued before
+// iteration it is reduced and written, so a CTA always has requests in flight (a load-reduce-store
+// sequence per iteration, with its two block barriers, left HBM idle about 40 % of the time).
 template <int kV, int R>
 __global__ void __launch_bounds__(kNormThreads)
 rmsnorm_fwd_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ g,
@@ -82,19 +106,13 @@ rmsnorm_fwd_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__r
     }
     const long long rows_per_iter = (long long)gridDim.x * lanes * R;
     const int iters = (int)((n + rows_per_iter - 1) / rows_per_iter);
+    const long long first = ((long long)blockIdx.x * lanes + rl) * R;
     const float inv_d = 1.f / (float)d;
+    RowRegs<kV, R> cur, nxt;
+    load_rows<kV, R>(cur, x, first, n, d, c, tpr);
     for (int it = 0; it < iters; ++it) {
-        const long long row0 = it * rows_per_iter + ((long long)blockIdx.x * lanes + rl) * R;
-        uint4 xv[R][kV];
-#pragma unroll
-        for (int i = 0; i < R; ++i)
-#pragma unroll
-            for (int j = 0; j < kV; ++j) {
-                const int v = c + j * tpr;
-                xv[i][j] = make_uint4(0u, 0u, 0u, 0u);
-                if (row0 + i < n && v < nvec)
-                    xv[i][j] = __ldcs(reinterpret_cast<const uint4 *>(x + (size_t)(row0 + i) * d) + v);
-            }
+        const long long row0 = it * rows_per_iter + first;
+        if (it + 1 < iters) load_rows<kV, R>(nxt, x, row0 + rows_per_iter, n, d, c, tpr);
         float ss[R];
 #pragma unroll
         for (int i = 0; i < R; ++i) {
@@ -102,7 +120,7 @@ rmsnorm_fwd_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__r
 #pragma unroll
             for (int j = 0; j < kV; ++j) {
                 float f[8];
-                unpack8(xv[i][j], f);
+                unpack8(cur.v[i][j], f);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) ss[i] = fmaf(f[e], f[e], ss[i]);
             }
@@ -118,12 +136,13 @@ rmsnorm_fwd_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__r
                 const int v = c + j * tpr;
                 if (v >= nvec) continue;
                 float f[8];
-                unpack8(xv[i][j], f);
+                unpack8(cur.v[i][j], f);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) f[e] = f[e] * r * gf[j][e];
                 __stcs(reinterpret_cast<uint4 *>(y + (size_t)(row0 + i) * d) + v, pack8(f));
             }
         }
+        cur = nxt;
     }
 }
 
@@ -151,21 +170,17 @@ rmsnorm_bwd_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__r
     }
     const long long rows_per_iter = (long long)gridDim.x * lanes * R;
     const int iters = (int)((n + rows_per_iter - 1) / rows_per_iter);
+    const long long first = ((long long)blockIdx.x * lanes + rl) * R;
     const float inv_d = 1.f / (float)d;
+    RowRegs<kV, R> xc, dc, xn, dn;
+    load_rows<kV, R>(xc, x, first, n, d, c, tpr);
+    load_rows<kV, R>(dc, dy, first, n, d, c, tpr);
     for (int it = 0; it < iters; ++it) {
-        const long long row0 = it * rows_per_iter + ((long long)blockIdx.x * lanes + rl) * R;
-        uint4 xv[R][kV], dv[R][kV];
-#pragma unroll
-        for (int i = 0; i < R; ++i)
-#pragma unroll
-            for (int j = 0; j < kV; ++j) {
-                const int v = c + j * tpr;
-                xv[i][j] = dv[i][j] = make_uint4(0u, 0u, 0u, 0u);
-                if (row0 + i < n && v < nvec) {
-                    xv[i][j] = __ldcs(reinterpret_cast<const uint4 *>(x + (size_t)(row0 + i) * d) + v);
-                    dv[i][j] = __ldcs(reinterpret_cast<const uint4 *>(dy + (size_t)(row0 + i) * d) + v);
-                }
-            }
+        const long long row0 = it * rows_per_iter + first;
+        if (it + 1 < iters) {
+            load_rows<kV, R>(xn, x, row0 + rows_per_iter, n, d, c, tpr);
+            load_rows<kV, R>(dn, dy, row0 + rows_per_iter, n, d, c, tpr);
+        }
         // per row: t = sum_k x_k g_k dy_k, and sum_k x_k^2 when r is not given
         float t[R], ss[R];
 #pragma unroll
@@ -174,8 +189,8 @@ rmsnorm_bwd_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__r
 #pragma unroll
             for (int j = 0; j < kV; ++j) {
                 float fx[8], fd[8];
-                unpack8(xv[i][j], fx);
-                unpack8(dv[i][j], fd);
+                unpack8(xc.v[i][j], fx);
+                unpack8(dc.v[i][j], fd);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                     t[i] = fmaf(fx[e] * gf[j][e], fd[e], t[i]);
@@ -195,8 +210,8 @@ rmsnorm_bwd_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__r
                 const int v = c + j * tpr;
                 if (v >= nvec) continue;
                 float fx[8], fd[8], o[8];
-                unpack8(xv[i][j], fx);
-                unpack8(dv[i][j], fd);
+                unpack8(xc.v[i][j], fx);
+                unpack8(dc.v[i][j], fd);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                     o[e] = r * gf[j][e] * fd[e] - fx[e] * coef;
@@ -205,6 +220,8 @@ rmsnorm_bwd_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__r
                 __stcs(reinterpret_cast<uint4 *>(dx + (size_t)(row0 + i) * d) + v, pack8(o));
             }
         }
+        xc = xn;
+        dc = dn;
     }
     // CTA partial of dg: the row lanes' sums added in lane order
     float *mine = part + (size_t)blockIdx.x * d;
@@ -246,18 +263,24 @@ rmsnorm_dg_kernel(const float *__restrict__ part, __nv_bfloat16 *__restrict__ dg
 }
 
 struct NormPlan {
-    int tpr, kV, grid;
+    int tpr, kV, R, grid;
 };
-NormPlan norm_plan(int n, int d)
+// Threads per row: the smallest power of two (at least a warp, at most the CTA) that leaves a thread
+// no more than max_kv vectors of a row.  Measured on B200 (n*d = 2^27): a few vectors per thread and
+// one row per lane and iteration beat wider rows of threads (fewer CTA barriers per byte moved).
+NormPlan norm_plan(int n, int d, bool bwd)
 {
     NormPlan p{};
     const int nvec = d / 8;
+    const int max_kv = bwd ? (d > 4096 ? 4 : 2) : 4;
     p.tpr = 1;
-    while (p.tpr < nvec && p.tpr < kNormThreads) p.tpr *= 2;
+    while (p.tpr < nvec && p.tpr < 32) p.tpr *= 2;
+    while ((nvec + p.tpr - 1) / p.tpr > max_kv && p.tpr < kNormThreads) p.tpr *= 2;
     const int need = (nvec + p.tpr - 1) / p.tpr;           // vectors per thread per row
     p.kV = need <= 1 ? 1 : need <= 2 ? 2 : 4;
-    const int R = 8 / p.kV, lanes = kNormThreads / p.tpr;
-    const long long blocks = ((long long)n + (long long)lanes * R - 1) / ((long long)lanes * R);
+    p.R = p.kV == 1 ? 2 : (bwd && p.kV == 4) ? 2 : 1;
+    const int lanes = kNormThreads / p.tpr;
+    const long long blocks = ((long long)n + (long long)lanes * p.R - 1) / ((long long)lanes * p.R);
     p.grid = (int)(blocks < 148 * 4 ? blocks : 148 * 4);
     if (p.grid < 1) p.grid = 1;
     return p;
@@ -265,25 +288,25 @@ NormPlan norm_plan(int n, int d)
 
 }  // namespace
 
-size_t rmsnorm_workspace_bytes(int n, int d) { return (size_t)norm_plan(n, d).grid * d * sizeof(float); }
+size_t rmsnorm_workspace_bytes(int n, int d) { return (size_t)norm_plan(n, d, true).grid * d * sizeof(float); }
 
 cudaError_t rmsnorm_fwd(int n, int d, float eps, const void *x, const void *g, void *y, float *r, cudaStream_t st)
 {
-    const NormPlan p = norm_plan(n, d);
+    const NormPlan p = norm_plan(n, d, false);
     const auto *xb = (const __nv_bfloat16 *)x;
     const auto *gb = (const __nv_bfloat16 *)g;
     auto *yb = (__nv_bfloat16 *)y;
     LaunchScope scope(MOA_KERNEL_OTHER, st);
-    if (p.kV == 1) rmsnorm_fwd_kernel<1, 8><<<p.grid, kNormThreads, 0, st>>>(xb, gb, yb, r, n, d, eps, p.tpr);
-    else if (p.kV == 2) rmsnorm_fwd_kernel<2, 4><<<p.grid, kNormThreads, 0, st>>>(xb, gb, yb, r, n, d, eps, p.tpr);
-    else rmsnorm_fwd_kernel<4, 2><<<p.grid, kNormThreads, 0, st>>>(xb, gb, yb, r, n, d, eps, p.tpr);
+    if (p.kV == 1) rmsnorm_fwd_kernel<1, 2><<<p.grid, kNormThreads, 0, st>>>(xb, gb, yb, r, n, d, eps, p.tpr);
+    else if (p.kV == 2) rmsnorm_fwd_kernel<2, 1><<<p.grid, kNormThreads, 0, st>>>(xb, gb, yb, r, n, d, eps, p.tpr);
+    else rmsnorm_fwd_kernel<4, 1><<<p.grid, kNormThreads, 0, st>>>(xb, gb, yb, r, n, d, eps, p.tpr);
     return cudaGetLastError();
 }
 
 cudaError_t rmsnorm_bwd(int n, int d, float eps, const void *x, const void *g, const float *r, const void *dy,
                         void *dx, void *dg, void *ws, cudaStream_t st)
 {
-    const NormPlan p = norm_plan(n, d);
+    const NormPlan p = norm_plan(n, d, true);
     const auto *xb = (const __nv_bfloat16 *)x;
     const auto *gb = (const __nv_bfloat16 *)g;
     const auto *db = (const __nv_bfloat16 *)dy;
@@ -291,8 +314,8 @@ cudaError_t rmsnorm_bwd(int n, int d, float eps, const void *x, const void *g, c
     float *part = (float *)ws;
     {
         LaunchScope scope(MOA_KERNEL_OTHER, st);
-        if (p.kV == 1) rmsnorm_bwd_kernel<1, 8><<<p.grid, kNormThreads, 0, st>>>(xb, gb, r, db, ob, part, n, d, eps, p.tpr);
-        else if (p.kV == 2) rmsnorm_bwd_kernel<2, 4><<<p.grid, kNormThreads, 0, st>>>(xb, gb, r, db, ob, part, n, d, eps, p.tpr);
+        if (p.kV == 1) rmsnorm_bwd_kernel<1, 2><<<p.grid, kNormThreads, 0, st>>>(xb, gb, r, db, ob, part, n, d, eps, p.tpr);
+        else if (p.kV == 2) rmsnorm_bwd_kernel<2, 1><<<p.grid, kNormThreads, 0, st>>>(xb, gb, r, db, ob, part, n, d, eps, p.tpr);
         else rmsnorm_bwd_kernel<4, 2><<<p.grid, kNormThreads, 0, st>>>(xb, gb, r, db, ob, part, n, d, eps, p.tpr);
         const cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
