@@ -309,6 +309,7 @@ BLOCK_WORKLOADS = {
     "rmsnorm_n65536_d4096": ("rmsnorm", 65536, 4096, 0),
     "mlp_n16384_d2048_ff8192": ("mlp", 16384, 2048, 8192),          # config 4's tokens, 16 heads x 128, d_ff = 4 d
     "mlp_n8192_d4096_ff16384": ("mlp", 8192, 4096, 16384),
+    "mlp_n4096_d1024_ff4096": ("mlp", 4096, 1024, 4096),              # small case for profiler captures (0.4 GB moved per step)
     "mlp_paper_n512_d64_ff256": ("mlp", 512, 64, 256),              # the paper's own traffic-check size (B=2, N=256, D=64, DFF=256)
 }
 
