@@ -90,7 +90,7 @@ template <bool kAMn, bool kBMn, int kEpi>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapB0,
                const __grid_constant__ CUtensorMap mapA1, const __grid_constant__ CUtensorMap mapB1,
-               GemmEpi epi, int M, int N, int K, int nparts, unsigned int *status)
+               GemmEpi epi, int M, int N, int K, int nparts, int nbatch, unsigned int *status)
 {
     constexpr bool kDualN = kEpi == EPI_SWIGLU_FWD;         // B tile = 128 rows of map B0 + 128 rows of map B1
     constexpr int kTileN = kDualN ? 128 : GN;                // output columns a tile covers
@@ -106,7 +106,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
 
     const int tiles_m = (M + GM - 1) / GM, tiles_n = (N + kTileN - 1) / kTileN;
-    const int tiles = tiles_m * tiles_n;
+    // nbatch = 2: two independent products of one shape in one launch (A1 B1^T -> epi.c1 after A0 B0^T ->
+    // epi.c0), so that their tiles share the waves of the persistent grid
+    const int tiles_one = tiles_m * tiles_n, tiles = tiles_one * nbatch;
     const int nk = (K + GK - 1) / GK, nk_total = nk * nparts;
 
     if (tid == 0) {
@@ -138,14 +140,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
         bool ok = true;
         for (int t = blockIdx.x; ok && t < tiles; t += gridDim.x) {
             int tm, tn;
-            tile_coords(t, tiles_m, tiles_n, tm, tn);
+            const int second = t >= tiles_one ? 1 : 0;
+            tile_coords(t - second * tiles_one, tiles_m, tiles_n, tm, tn);
             const int m0 = tm * GM, n0 = tn * kTileN;
             for (int ks = 0; ks < nk_total; ++ks, ++it) {
                 const int s = it % kStages;
                 if (!mbar_wait(bars + G_EMPTY + s, ((it / kStages) & 1) ^ 1, abortp, status, GERR_EMPTY)) { ok = false; break; }
                 const int part = ks / nk, k0 = (ks - part * nk) * GK;
-                const CUtensorMap *ma = part ? &mapA1 : &mapA0;
-                const CUtensorMap *mb = (part && !kDualN) ? &mapB1 : &mapB0;
+                const CUtensorMap *ma = (part || second) ? &mapA1 : &mapA0;
+                const CUtensorMap *mb = ((part || second) && !kDualN) ? &mapB1 : &mapB0;
                 uint8_t *sa = sm + s * kStageBytes, *sb = sa + kABytes;
                 uint64_t *full = bars + G_FULL + s;
                 mbar_arrive_expect_tx(full, kStageBytes);
@@ -203,7 +206,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
         int ti = 0;
         for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++ti) {
             int tm, tn;
-            tile_coords(t, tiles_m, tiles_n, tm, tn);
+            const int second = t >= tiles_one ? 1 : 0;
+            tile_coords(t - second * tiles_one, tiles_m, tiles_n, tm, tn);
             const int buf = ti & 1;
             const int row = tm * GM + lane_row, n0 = tn * kTileN;
             if (!mbar_wait(bars + G_ACCFULL + buf, (ti >> 1) & 1, abortp, status, GERR_ACCFULL)) break;
@@ -262,7 +266,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
 #pragma unroll
                             for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(r[e + i]);
                             if (kEpi == EPI_STORE) {
-                                store8(epi.c0 + rbase + col, f);
+                                store8((second ? epi.c1 : epi.c0) + rbase + col, f);
                             } else {
                                 float fa[8], fu[8], da[8], du[8];
                                 unpack8(va[e / 8], fa);
@@ -303,7 +307,7 @@ bool operand_map(CUtensorMap *m, const Operand &o, bool mn_major, int box_rows)
 
 template <bool kAMn, bool kBMn, int kEpi>
 cudaError_t launch_gemm(const Operand &A0, const Operand &B0, const Operand *A1, const Operand *B1, const GemmEpi &epi,
-                        int M, int N, int K, cudaStream_t st)
+                        int M, int N, int K, cudaStream_t st, int nbatch = 1)
 {
     constexpr bool kDualN = kEpi == EPI_SWIGLU_FWD;
     CUtensorMap ma0, mb0, ma1, mb1;
@@ -314,11 +318,11 @@ cudaError_t launch_gemm(const Operand &A0, const Operand &B0, const Operand *A1,
     auto kernel = tc_gemm_kernel<kAMn, kBMn, kEpi>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
     if (e != cudaSuccess) return e;
-    const int tiles = ((M + GM - 1) / GM) * ((N + (kDualN ? 128 : GN) - 1) / (kDualN ? 128 : GN));
-    const int nparts = (A1 && !kDualN) ? 2 : 1;
+    const int tiles = ((M + GM - 1) / GM) * ((N + (kDualN ? 128 : GN) - 1) / (kDualN ? 128 : GN)) * nbatch;
+    const int nparts = (A1 && !kDualN && nbatch == 1) ? 2 : 1;
     LaunchScope scope(MOA_KERNEL_OTHER, st);
     kernel<<<tiles < 148 ? tiles : 148, kGemmThreads, kGemmSmem, st>>>(ma0, mb0, ma1, mb1, epi, M, N, K, nparts,
-                                                                      device_status_ptr());
+                                                                      nbatch, device_status_ptr());
     return cudaGetLastError();
 }
 
@@ -349,11 +353,9 @@ cudaError_t gated_mlp_bwd(int n, int d, int dff, const void *x, const void *W1, 
     // dW2 [d,d_ff] = dy^T h: both operands read transposed (K = tokens)
     GemmEpi e4{(__nv_bfloat16 *)dW2, nullptr, nullptr, nullptr, nullptr, dff};
     if ((e = launch_gemm<true, true, EPI_STORE>(DY, Hh, nullptr, nullptr, e4, d, dff, n, st)) != cudaSuccess) return e;
-    // dW1 = da^T x, dW3 = du^T x   [d_ff,d]
-    GemmEpi e5{(__nv_bfloat16 *)dW1, nullptr, nullptr, nullptr, nullptr, d};
-    if ((e = launch_gemm<true, true, EPI_STORE>(DA, X, nullptr, nullptr, e5, dff, d, n, st)) != cudaSuccess) return e;
-    GemmEpi e6{(__nv_bfloat16 *)dW3, nullptr, nullptr, nullptr, nullptr, d};
-    if ((e = launch_gemm<true, true, EPI_STORE>(DU, X, nullptr, nullptr, e6, dff, d, n, st)) != cudaSuccess) return e;
+    // dW1 = da^T x, dW3 = du^T x   [d_ff,d]: one launch, so that the two tile sets fill the waves together
+    GemmEpi e5{(__nv_bfloat16 *)dW1, (__nv_bfloat16 *)dW3, nullptr, nullptr, nullptr, d};
+    if ((e = launch_gemm<true, true, EPI_STORE>(DA, X, &DU, &X, e5, dff, d, n, st, 2)) != cudaSuccess) return e;
     // dx = da W1 + du W3: two operand pairs accumulate into one tile (W1, W3 [d_ff,d] as MN-major B)
     GemmEpi e7{(__nv_bfloat16 *)dx, nullptr, nullptr, nullptr, nullptr, d};
     return launch_gemm<false, true, EPI_STORE>(DA, w1, &DU, &w3, e7, n, d, dff, st);
