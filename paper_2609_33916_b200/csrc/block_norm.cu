@@ -181,6 +181,10 @@ rmsnorm_bwd_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__r
             load_rows<kV, R>(xn, x, row0 + rows_per_iter, n, d, c, tpr);
             load_rows<kV, R>(dn, dy, row0 + rows_per_iter, n, d, c, tpr);
         }
+        // the stored r of this iteration's rows: requested here, ahead of the reductions and their barriers
+        float rr[R];
+#pragma unroll
+        for (int i = 0; i < R; ++i) rr[i] = (r_in != nullptr && row0 + i < n) ? __ldg(r_in + row0 + i) : 0.f;
         // per row: t = sum_k x_k g_k dy_k, and sum_k x_k^2 when r is not given
         float t[R], ss[R];
 #pragma unroll
@@ -203,7 +207,7 @@ rmsnorm_bwd_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__r
 #pragma unroll
         for (int i = 0; i < R; ++i) {
             if (row0 + i >= n) continue;
-            const float r = r_in != nullptr ? r_in[row0 + i] : rsqrtf(ss[i] * inv_d + eps);
+            const float r = r_in != nullptr ? rr[i] : rsqrtf(ss[i] * inv_d + eps);
             const float coef = r * r * r * t[i] * inv_d;
 #pragma unroll
             for (int j = 0; j < kV; ++j) {
@@ -241,23 +245,33 @@ rmsnorm_bwd_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__r
     }
 }
 
-// dg[col] = sum over the CTA partials, in a fixed order: a CTA owns 32 columns, its 8 warps take the
-// partial rows w, w + 8, ... and the 8 sums are added in warp order.
-__global__ void __launch_bounds__(256)
+// dg[col] = sum over the CTA partials, in a fixed order: a CTA owns 32 columns, its 16 warps take the
+// partial rows w, w + 16, ... (four independent running sums each, so that the loads overlap) and the
+// sums are added in a fixed order.
+constexpr int kDgWarps = 16;
+__global__ void __launch_bounds__(32 * kDgWarps)
 rmsnorm_dg_kernel(const float *__restrict__ part, __nv_bfloat16 *__restrict__ dg, int parts, int d)
 {
-    __shared__ float s[8][32];
+    __shared__ float s[kDgWarps][32];
     const int cx = threadIdx.x % 32, cy = threadIdx.x / 32;
     const int col = blockIdx.x * 32 + cx;
-    float a = 0.f;
-    if (col < d)
-        for (int p = cy; p < parts; p += 8) a += part[(size_t)p * d + col];
-    s[cy][cx] = a;
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    if (col < d) {
+        int p = cy;
+        for (; p + 3 * kDgWarps < parts; p += 4 * kDgWarps) {
+            a0 += part[(size_t)p * d + col];
+            a1 += part[(size_t)(p + kDgWarps) * d + col];
+            a2 += part[(size_t)(p + 2 * kDgWarps) * d + col];
+            a3 += part[(size_t)(p + 3 * kDgWarps) * d + col];
+        }
+        for (; p < parts; p += kDgWarps) a0 += part[(size_t)p * d + col];
+    }
+    s[cy][cx] = (a0 + a1) + (a2 + a3);
     __syncthreads();
     if (cy == 0 && col < d) {
         float t = 0.f;
 #pragma unroll
-        for (int w = 0; w < 8; ++w) t += s[w][cx];
+        for (int w = 0; w < kDgWarps; ++w) t += s[w][cx];
         dg[col] = __float2bfloat16_rn(t);
     }
 }
@@ -321,7 +335,7 @@ cudaError_t rmsnorm_bwd(int n, int d, float eps, const void *x, const void *g, c
         if (e != cudaSuccess) return e;
     }
     LaunchScope scope(MOA_KERNEL_OTHER, st);
-    rmsnorm_dg_kernel<<<(d + 31) / 32, 256, 0, st>>>(part, (__nv_bfloat16 *)dg, p.grid, d);
+    rmsnorm_dg_kernel<<<(d + 31) / 32, 32 * kDgWarps, 0, st>>>(part, (__nv_bfloat16 *)dg, p.grid, d);
     return cudaGetLastError();
 }
 
