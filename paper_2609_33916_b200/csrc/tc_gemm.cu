@@ -38,30 +38,17 @@ constexpr int kStages = 4;   // three stages measured 7-16 % slower: the ring ha
 constexpr int kGemmThreads = 320;                      // producer, issuer, eight epilogue warps
 constexpr int kABytes = GM * GK * 2, kBBytes = GN * GK * 2, kStageBytes = kABytes + kBBytes;
 constexpr int kMnBox = 64 * GK * 2;                    // one MN-major box: 64 columns x 64 K-rows
-constexpr int kGemmSmem = kStages * kStageBytes + 1024 /* alignment */ + 256 /* barriers */;
+constexpr int kOutBox = 128 * 64 * 2;                  // one staged output chunk: 128 rows x 64 columns, bf16
+constexpr int kGemmSmem = kStages * kStageBytes + 2 * kOutBox + 1024 /* alignment */ + 256 /* barriers */;
 
 enum { EPI_STORE = 0, EPI_SWIGLU_FWD = 1, EPI_SWIGLU_BWD = 2 };
-enum { G_FULL = 0, G_EMPTY = kStages, G_ACCFULL = 2 * kStages, G_ACCEMPTY = 2 * kStages + 2, G_COUNT = 2 * kStages + 4 };
-enum { GERR_EMPTY = 0x301, GERR_FULL = 0x302, GERR_ACCFULL = 0x303, GERR_ACCEMPTY = 0x304 };
+enum { G_FULL = 0, G_EMPTY = kStages, G_ACCFULL = 2 * kStages, G_ACCEMPTY = 2 * kStages + 2, G_EPI = 2 * kStages + 4,
+       G_IN = 2 * kStages + 5, G_COUNT = 2 * kStages + 6 };
+enum { GERR_EMPTY = 0x301, GERR_FULL = 0x302, GERR_ACCFULL = 0x303, GERR_ACCEMPTY = 0x304, GERR_EPI = 0x305, GERR_IN = 0x306 };
 
-struct GemmEpi {
-    __nv_bfloat16 *c0;          // STORE: C.  FWD: a.  BWD: da
-    __nv_bfloat16 *c1;          // FWD: u.  BWD: du
-    __nv_bfloat16 *c2;          // FWD: h
-    const __nv_bfloat16 *a;     // BWD: stored a
-    const __nv_bfloat16 *u;     // BWD: stored u
-    int ldc;                    // row length of every array above
-};
+// Outputs leave through TMA stores (tensor maps C0..C3: STORE: C (and the second product's C); FWD gate: a, u, h;
+// BWD gate: da, du, and the stored a, u as C2, C3, which its epilogue brings in by TMA loads).
 
-__device__ __forceinline__ void store8(__nv_bfloat16 *p, const float *f)
-{
-    uint4 v;
-    v.x = pack_bf16(f[0], f[1]);
-    v.y = pack_bf16(f[2], f[3]);
-    v.z = pack_bf16(f[4], f[5]);
-    v.w = pack_bf16(f[6], f[7]);
-    *reinterpret_cast<uint4 *>(p) = v;
-}
 __device__ __forceinline__ void unpack8(const uint4 &v, float *f)
 {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
@@ -90,24 +77,24 @@ template <bool kAMn, bool kBMn, int kEpi>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapB0,
                const __grid_constant__ CUtensorMap mapA1, const __grid_constant__ CUtensorMap mapB1,
-               GemmEpi epi, int M, int N, int K, int nparts, int nbatch, unsigned int *status)
+               const __grid_constant__ CUtensorMap mapC0, const __grid_constant__ CUtensorMap mapC1,
+               const __grid_constant__ CUtensorMap mapC2, const __grid_constant__ CUtensorMap mapC3, int M, int N, int K, int nparts, int nbatch, unsigned int *status)
 {
     constexpr bool kDualN = kEpi == EPI_SWIGLU_FWD;         // B tile = 128 rows of map B0 + 128 rows of map B1
     constexpr int kTileN = kDualN ? 128 : GN;                // output columns a tile covers
-    // Epilogue warps: two per 32-lane group (one column half each), except in the forward gate epilogue,
-    // where eight warps of stores and exponentials measured 13 % slower than four
-    constexpr int kEpiWarps = kEpi == EPI_SWIGLU_FWD ? 4 : 8;
-    constexpr int kHalfCols = (kDualN ? 128 : GN) / (kEpiWarps / 4);
+    // Epilogue warps: two per 32-lane group of TMEM; together they fill one 64-column output chunk at a time
+    constexpr int kEpiWarps = 8;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *sm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint64_t *bars = reinterpret_cast<uint64_t *>(sm + kStages * kStageBytes);
+    uint8_t *sout = sm + kStages * kStageBytes;               // two staged output chunks (128-byte swizzle)
+    uint64_t *bars = reinterpret_cast<uint64_t *>(sout + 2 * kOutBox);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + G_COUNT);
     volatile uint32_t *abortp = tmem_slot + 1;
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
 
     const int tiles_m = (M + GM - 1) / GM, tiles_n = (N + kTileN - 1) / kTileN;
-    // nbatch = 2: two independent products of one shape in one launch (A1 B1^T -> epi.c1 after A0 B0^T ->
-    // epi.c0), so that their tiles share the waves of the persistent grid
+    // nbatch = 2: two independent products of one shape in one launch (A1 B1^T -> map C1 after A0 B0^T ->
+    // map C0), so that their tiles share the waves of the persistent grid
     const int tiles_one = tiles_m * tiles_n, tiles = tiles_one * nbatch;
     const int nk = (K + GK - 1) / GK, nk_total = nk * nparts;
 
@@ -120,6 +107,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
         mbar_init(bars + G_ACCFULL + 1, 1);
         mbar_init(bars + G_ACCEMPTY + 0, 32 * kEpiWarps);
         mbar_init(bars + G_ACCEMPTY + 1, 32 * kEpiWarps);
+        mbar_init(bars + G_EPI, 32 * kEpiWarps);
+        mbar_init(bars + G_IN, 1);
         *abortp = 0;
         fence_mbar_init();
     }
@@ -200,93 +189,144 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
         }
     } else if (warp >= 2 && warp < 2 + kEpiWarps) {
         // ---------------------------------------------------------------------- epilogue
+        // A thread owns one row of the tile (its TMEM lane) and 32 of the 64 columns of the current chunk.  Results go
+        // to a shared-memory chunk in the 128-byte-swizzle layout and leave as one TMA store per chunk (whole 128-byte
+        // lines; rows and columns past the array are clipped by the tensor map): row-owner 16-byte stores to global
+        // memory cost one L2 request each, and at 6000 requests per tile they slowed the operand loads of the next tile.
         const int lane_row = 32 * (warp % 4) + lane;               // TMEM lane = row of the tile
         const uint32_t lane_addr = tbase + ((uint32_t)(32 * (warp % 4)) << 16);
-        const int half = (warp - 2) / 4;                           // which half of the tile's columns
+        const int half = (warp - 2) / 4;                           // which 32 columns of a 64-column chunk
+        const bool leader = tid == 64;
+        uint32_t epi_phase = 0, chunk_q = 0, in_q = 0;
+        bool ok = true;
+        // all epilogue threads meet (bounded wait)
+        auto epi_sync = [&]() -> bool {
+            mbar_arrive(bars + G_EPI);
+            const bool r = mbar_wait(bars + G_EPI, epi_phase & 1, abortp, status, GERR_EPI);
+            ++epi_phase;
+            return r;
+        };
+        // the 32 values of this thread (as 16 bf16 pairs) -> staged chunk -> TMA store at (row0, col0)
+        auto stage_store = [&](const CUtensorMap *map, const uint32_t (&v)[16], int col0, int row0) -> bool {
+            uint8_t *buf = sout + (chunk_q & 1) * kOutBox;
+            if (leader) bulk_wait_read<1>();                       // the store issued two chunks ago has left this buffer
+            if (!epi_sync()) return false;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                *reinterpret_cast<uint4 *>(buf + lane_row * 128 + (((half * 4 + j) ^ (lane_row & 7)) << 4)) =
+                    make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            fence_proxy_async_smem();
+            if (!epi_sync()) return false;
+            if (leader) {
+                tma_store_3d(map, buf, col0, row0, 0);
+                bulk_commit();
+            }
+            ++chunk_q;
+            return true;
+        };
         int ti = 0;
-        for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++ti) {
+        for (int t = blockIdx.x; ok && t < tiles; t += gridDim.x, ++ti) {
             int tm, tn;
             const int second = t >= tiles_one ? 1 : 0;
             tile_coords(t - second * tiles_one, tiles_m, tiles_n, tm, tn);
             const int buf = ti & 1;
-            const int row = tm * GM + lane_row, n0 = tn * kTileN;
+            const int m0 = tm * GM, n0 = tn * kTileN;
+            if (kEpi == EPI_SWIGLU_BWD && leader) {       // the tile's stored a, u: into L2 while its main loop runs
+#pragma unroll
+                for (int c0 = 0; c0 < GN; c0 += 64) {
+                    tma_prefetch_3d(&mapC2, n0 + c0, m0, 0);
+                    tma_prefetch_3d(&mapC3, n0 + c0, m0, 0);
+                }
+            }
             if (!mbar_wait(bars + G_ACCFULL + buf, (ti >> 1) & 1, abortp, status, GERR_ACCFULL)) break;
             tc_fence_after();
             const uint32_t acc = lane_addr + (uint32_t)(buf * GN);
-            const size_t rbase = (size_t)row * epi.ldc;
             if (kEpi == EPI_SWIGLU_FWD) {
 #pragma unroll 1
-                for (int c = kHalfCols * half; c < kHalfCols * half + kHalfCols; c += 32) {
+                for (int c0 = 0; ok && c0 < 128; c0 += 64) {
+                    const int c = c0 + 32 * half;
                     uint32_t ra[32], ru[32];
                     tmem_ld(acc + c, ra);
                     tmem_ld(acc + 128 + c, ru);
                     tc_wait_ld();
-                    if (row < M) {
-#pragma unroll
-                        for (int e = 0; e < 32; e += 8) {
-                            const int col = n0 + c + e;
-                            if (col >= N) break;
-                            float fa[8], fu[8], fh[8];
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) {
-                                fa[i] = __uint_as_float(ra[e + i]);
-                                fu[i] = __uint_as_float(ru[e + i]);
-                                fh[i] = fa[i] * sigmoidf_fast(fa[i]) * fu[i];
-                            }
-                            store8(epi.c0 + rbase + col, fa);
-                            store8(epi.c1 + rbase + col, fu);
-                            store8(epi.c2 + rbase + col, fh);
-                        }
+                    if (c0 == 64) {                       // last read of this accumulator: hand it back early
+                        tc_fence_before();
+                        mbar_arrive(bars + G_ACCEMPTY + buf);
                     }
+                    uint32_t pa[16], pu[16], ph[16];
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2) {
+                        const float a0 = __uint_as_float(ra[e]), a1 = __uint_as_float(ra[e + 1]);
+                        const float u0 = __uint_as_float(ru[e]), u1 = __uint_as_float(ru[e + 1]);
+                        pa[e / 2] = pack_bf16(a0, a1);
+                        pu[e / 2] = pack_bf16(u0, u1);
+                        ph[e / 2] = pack_bf16(a0 * sigmoidf_fast(a0) * u0, a1 * sigmoidf_fast(a1) * u1);
+                    }
+                    ok = stage_store(&mapC0, pa, n0 + c0, m0) && stage_store(&mapC1, pu, n0 + c0, m0) &&
+                         stage_store(&mapC2, ph, n0 + c0, m0);
+                }
+            } else if (kEpi == EPI_STORE) {
+#pragma unroll 1
+                for (int c0 = 0; ok && c0 < GN; c0 += 64) {
+                    uint32_t r[32];
+                    tmem_ld(acc + c0 + 32 * half, r);
+                    tc_wait_ld();
+                    if (c0 == GN - 64) {                  // last read of this accumulator: hand it back early
+                        tc_fence_before();
+                        mbar_arrive(bars + G_ACCEMPTY + buf);
+                    }
+                    uint32_t pc[16];
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2) pc[e / 2] = pack_bf16(__uint_as_float(r[e]), __uint_as_float(r[e + 1]));
+                    ok = stage_store(second ? &mapC1 : &mapC0, pc, n0 + c0, m0);
                 }
             } else {
+                // Backward gate: per 64-column chunk the stored a and u come into the two staging buffers by TMA, every
+                // thread turns its 32 + 32 values into da, du in place, and the buffers leave by TMA stores.
 #pragma unroll 1
-                for (int c = kHalfCols * half; c < kHalfCols * half + kHalfCols; c += 32) {
-                    // the stored a, u of this chunk are requested before the accumulator is read
-                    uint4 va[4], vu[4];
-                    if (kEpi == EPI_SWIGLU_BWD && row < M) {
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const int col = n0 + c + 8 * q;
-                            if (col < N) {
-                                va[q] = __ldg(reinterpret_cast<const uint4 *>(epi.a + rbase + col));
-                                vu[q] = __ldg(reinterpret_cast<const uint4 *>(epi.u + rbase + col));
-                            }
-                        }
+                for (int c0 = 0; ok && c0 < GN; c0 += 64, ++in_q) {
+                    if (leader) {
+                        bulk_wait_read<0>();              // the previous chunk's stores have left both buffers
+                        mbar_arrive_expect_tx(bars + G_IN, 2 * kOutBox);
+                        tma_load_3d(sout, &mapC2, bars + G_IN, n0 + c0, m0, 0);
+                        tma_load_3d(sout + kOutBox, &mapC3, bars + G_IN, n0 + c0, m0, 0);
                     }
                     uint32_t r[32];
-                    tmem_ld(acc + c, r);
+                    tmem_ld(acc + c0 + 32 * half, r);
                     tc_wait_ld();
-                    if (row < M) {
+                    if (c0 == GN - 64) {
+                        tc_fence_before();
+                        mbar_arrive(bars + G_ACCEMPTY + buf);
+                    }
+                    if (!mbar_wait(bars + G_IN, in_q & 1, abortp, status, GERR_IN)) { ok = false; break; }
 #pragma unroll
-                        for (int e = 0; e < 32; e += 8) {
-                            const int col = n0 + c + e;
-                            if (col >= N) break;
-                            float f[8];
+                    for (int q = 0; q < 4; ++q) {
+                        const uint32_t off = lane_row * 128 + (((half * 4 + q) ^ (lane_row & 7)) << 4);
+                        uint4 *pa = reinterpret_cast<uint4 *>(sout + off), *pu = reinterpret_cast<uint4 *>(sout + kOutBox + off);
+                        float fa[8], fu[8], da[8], du[8];
+                        unpack8(*pa, fa);
+                        unpack8(*pu, fu);
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(r[e + i]);
-                            if (kEpi == EPI_STORE) {
-                                store8((second ? epi.c1 : epi.c0) + rbase + col, f);
-                            } else {
-                                float fa[8], fu[8], da[8], du[8];
-                                unpack8(va[e / 8], fa);
-                                unpack8(vu[e / 8], fu);
-#pragma unroll
-                                for (int i = 0; i < 8; ++i) {
-                                    const float sg = sigmoidf_fast(fa[i]);
-                                    da[i] = f[i] * fu[i] * sg * (1.f + fa[i] * (1.f - sg));
-                                    du[i] = f[i] * fa[i] * sg;
-                                }
-                                store8(epi.c0 + rbase + col, da);
-                                store8(epi.c1 + rbase + col, du);
-                            }
+                        for (int i = 0; i < 8; ++i) {
+                            const float f = __uint_as_float(r[8 * q + i]);
+                            const float sg = sigmoidf_fast(fa[i]);
+                            da[i] = f * fu[i] * sg * (1.f + fa[i] * (1.f - sg));
+                            du[i] = f * fa[i] * sg;
                         }
+                        *pa = make_uint4(pack_bf16(da[0], da[1]), pack_bf16(da[2], da[3]), pack_bf16(da[4], da[5]), pack_bf16(da[6], da[7]));
+                        *pu = make_uint4(pack_bf16(du[0], du[1]), pack_bf16(du[2], du[3]), pack_bf16(du[4], du[5]), pack_bf16(du[6], du[7]));
+                    }
+                    fence_proxy_async_smem();
+                    if (!epi_sync()) { ok = false; break; }
+                    if (leader) {
+                        tma_store_3d(&mapC0, sout, n0 + c0, m0, 0);
+                        tma_store_3d(&mapC1, sout + kOutBox, n0 + c0, m0, 0);
+                        bulk_commit();
                     }
                 }
             }
-            tc_fence_before();
-            mbar_arrive(bars + G_ACCEMPTY + buf);       // this thread has read its lanes of the accumulator
         }
+        if (leader) bulk_wait<0>();       // every store has completed before the CTA gives up its shared memory
     }
     tc_fence_before();
     __syncthreads();
@@ -306,8 +346,10 @@ bool operand_map(CUtensorMap *m, const Operand &o, bool mn_major, int box_rows)
 }
 
 template <bool kAMn, bool kBMn, int kEpi>
-cudaError_t launch_gemm(const Operand &A0, const Operand &B0, const Operand *A1, const Operand *B1, const GemmEpi &epi,
-                        int M, int N, int K, cudaStream_t st, int nbatch = 1)
+// C0..C2: output arrays (row length ldc); unused ones may repeat C0.
+cudaError_t launch_gemm(const Operand &A0, const Operand &B0, const Operand *A1, const Operand *B1, void *C0, void *C1,
+                        const void *C2, const void *C3, int c_rows, int ldc, int M, int N, int K, cudaStream_t st,
+                        int nbatch = 1)
 {
     constexpr bool kDualN = kEpi == EPI_SWIGLU_FWD;
     CUtensorMap ma0, mb0, ma1, mb1;
@@ -315,13 +357,18 @@ cudaError_t launch_gemm(const Operand &A0, const Operand &B0, const Operand *A1,
     if (!operand_map(&ma0, A0, kAMn, GM) || !operand_map(&mb0, B0, kBMn, b_rows)) return cudaErrorInvalidValue;
     if (!operand_map(&ma1, A1 ? *A1 : A0, kAMn, GM) || !operand_map(&mb1, B1 ? *B1 : B0, kBMn, b_rows))
         return cudaErrorInvalidValue;
+    CUtensorMap mc[4];
+    const void *cs[4] = {C0, C1 ? C1 : C0, C2 ? C2 : C0, C3 ? C3 : C0};
+    for (int i = 0; i < 4; ++i)     // [c_rows, ldc] bf16, boxes of 128 rows x 64 columns, 128-byte swizzle
+        if (!make_tensor_map_3d(&mc[i], cs[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 1, (uint64_t)c_rows, (uint64_t)ldc, 128, 64))
+            return cudaErrorInvalidValue;
     auto kernel = tc_gemm_kernel<kAMn, kBMn, kEpi>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
     if (e != cudaSuccess) return e;
     const int tiles = ((M + GM - 1) / GM) * ((N + (kDualN ? 128 : GN) - 1) / (kDualN ? 128 : GN)) * nbatch;
     const int nparts = (A1 && !kDualN && nbatch == 1) ? 2 : 1;
     LaunchScope scope(MOA_KERNEL_OTHER, st);
-    kernel<<<tiles < 148 ? tiles : 148, kGemmThreads, kGemmSmem, st>>>(ma0, mb0, ma1, mb1, epi, M, N, K, nparts,
+    kernel<<<tiles < 148 ? tiles : 148, kGemmThreads, kGemmSmem, st>>>(ma0, mb0, ma1, mb1, mc[0], mc[1], mc[2], mc[3], M, N, K, nparts,
                                                                       nbatch, device_status_ptr());
     return cudaGetLastError();
 }
@@ -333,11 +380,9 @@ cudaError_t gated_mlp_fwd(int n, int d, int dff, const void *x, const void *W1, 
 {
     // a | u = x [W1; W3]^T with the gate in the epilogue, then y = h W2^T
     const Operand X{x, n, d}, w1{W1, dff, d}, w3{W3, dff, d}, Hh{h, n, dff}, w2{W2, d, dff};
-    GemmEpi e1{(__nv_bfloat16 *)a, (__nv_bfloat16 *)u, (__nv_bfloat16 *)h, nullptr, nullptr, dff};
-    cudaError_t e = launch_gemm<false, false, EPI_SWIGLU_FWD>(X, w1, nullptr, &w3, e1, n, dff, d, st);
+    cudaError_t e = launch_gemm<false, false, EPI_SWIGLU_FWD>(X, w1, nullptr, &w3, a, u, h, nullptr, n, dff, n, dff, d, st);
     if (e != cudaSuccess) return e;
-    GemmEpi e2{(__nv_bfloat16 *)y, nullptr, nullptr, nullptr, nullptr, d};
-    return launch_gemm<false, false, EPI_STORE>(Hh, w2, nullptr, nullptr, e2, n, d, dff, st);
+    return launch_gemm<false, false, EPI_STORE>(Hh, w2, nullptr, nullptr, y, nullptr, nullptr, nullptr, n, d, n, d, dff, st);
 }
 
 cudaError_t gated_mlp_bwd(int n, int d, int dff, const void *x, const void *W1, const void *W3, const void *W2,
@@ -347,18 +392,17 @@ cudaError_t gated_mlp_bwd(int n, int d, int dff, const void *x, const void *W1, 
     const Operand X{x, n, d}, w1{W1, dff, d}, w3{W3, dff, d}, w2{W2, d, dff}, Hh{h, n, dff}, DY{dy, n, d};
     const Operand DA{da, n, dff}, DU{du, n, dff};
     // dh = dy W2 (W2 [d,d_ff] read as the MN-major B operand), gate backward in the epilogue -> da, du
-    GemmEpi e3{(__nv_bfloat16 *)da, (__nv_bfloat16 *)du, nullptr, (const __nv_bfloat16 *)a, (const __nv_bfloat16 *)u, dff};
-    cudaError_t e = launch_gemm<false, true, EPI_SWIGLU_BWD>(DY, w2, nullptr, nullptr, e3, n, dff, d, st);
+    cudaError_t e = launch_gemm<false, true, EPI_SWIGLU_BWD>(DY, w2, nullptr, nullptr, da, du, a, u, n, dff, n, dff, d, st);
     if (e != cudaSuccess) return e;
     // dW2 [d,d_ff] = dy^T h: both operands read transposed (K = tokens)
-    GemmEpi e4{(__nv_bfloat16 *)dW2, nullptr, nullptr, nullptr, nullptr, dff};
-    if ((e = launch_gemm<true, true, EPI_STORE>(DY, Hh, nullptr, nullptr, e4, d, dff, n, st)) != cudaSuccess) return e;
+    if ((e = launch_gemm<true, true, EPI_STORE>(DY, Hh, nullptr, nullptr, dW2, nullptr, nullptr, nullptr, d, dff, d, dff, n, st)) !=
+        cudaSuccess)
+        return e;
     // dW1 = da^T x, dW3 = du^T x   [d_ff,d]: one launch, so that the two tile sets fill the waves together
-    GemmEpi e5{(__nv_bfloat16 *)dW1, (__nv_bfloat16 *)dW3, nullptr, nullptr, nullptr, d};
-    if ((e = launch_gemm<true, true, EPI_STORE>(DA, X, &DU, &X, e5, dff, d, n, st, 2)) != cudaSuccess) return e;
+    if ((e = launch_gemm<true, true, EPI_STORE>(DA, X, &DU, &X, dW1, dW3, nullptr, nullptr, dff, d, dff, d, n, st, 2)) != cudaSuccess)
+        return e;
     // dx = da W1 + du W3: two operand pairs accumulate into one tile (W1, W3 [d_ff,d] as MN-major B)
-    GemmEpi e7{(__nv_bfloat16 *)dx, nullptr, nullptr, nullptr, nullptr, d};
-    return launch_gemm<false, true, EPI_STORE>(DA, w1, &DU, &w3, e7, n, d, dff, st);
+    return launch_gemm<false, true, EPI_STORE>(DA, w1, &DU, &w3, dx, nullptr, nullptr, nullptr, n, d, n, d, dff, st);
 }
 
 }  // namespace moa
