@@ -157,3 +157,45 @@ def test_gated_mlp_large_preactivations(rt):
     for k in ("h", "y", "dx", "dW1", "dW3", "dW2"):
         assert np.all(np.isfinite(got[k])), k
         assert mi.rel_err(got[k], ref[k]) <= TOL, (k, mi.rel_err(got[k], ref[k]))
+
+
+# ------------------------------------------------------------------- random shapes
+def _random_block_cases(count, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(count):
+        n = int(rng.choice([1, 7, 64, 127, 128, 129, 255, 257, 500, 1000, 1111]))
+        d = 8 * int(rng.integers(1, 80))                 # 8 .. 632
+        dff = 8 * int(rng.integers(1, 160))              # 8 .. 1272
+        out.append((i, n, d, dff))
+    return out
+
+
+@pytest.mark.parametrize("case", _random_block_cases(24, 20261127), ids=lambda c: f"{c[0]}-n{c[1]}-d{c[2]}-ff{c[3]}")
+def test_random_block_shapes(rt, case):
+    """Random token counts and widths (multiples of 8, tails in every tile dimension): both pieces against the oracle."""
+    i, n, d, dff = case
+    inp = mi.make_mlp_inputs(n, d, dff, seed=5000 + i)
+    f = {k: mi.to_f64(v, "bf16") for k, v in inp.items()}
+    ref = oracle.gated_mlp_fwd_bwd(f["x"], f["W1"], f["W3"], f["W2"], f["dy"])
+    got = _run_mlp(rt, inp)
+    for k in ("a", "u", "h", "y", "dx", "dW1", "dW3", "dW2"):
+        assert np.all(np.isfinite(got[k])), k
+        e = mi.rel_err(got[k], ref[k])
+        assert e <= TOL, (k, case, e)
+    ninp = mi.make_norm_inputs(n, d, seed=6000 + i)
+    f = {k: mi.to_f64(v, "bf16") for k, v in ninp.items()}
+    eps = float(np.random.default_rng(i).choice([0.0, 1e-6, 1e-2]))
+    nref = oracle.rmsnorm_fwd_bwd(f["x"], f["g"], f["dy"], eps)
+    ngot = _run_rmsnorm(rt, ninp, eps, give_r=bool(i % 2))
+    for k in ("y", "dx", "dg"):
+        assert np.all(np.isfinite(ngot[k])), k
+        assert mi.rel_err(ngot[k], nref[k]) <= TOL, (k, case, mi.rel_err(ngot[k], nref[k]))
+
+
+def test_gated_mlp_is_bitwise_reproducible(rt):
+    inp = mi.make_mlp_inputs(700, 264, 520, seed=99)
+    a = _run_mlp(rt, inp)
+    b = _run_mlp(rt, inp)
+    for k in a:
+        np.testing.assert_array_equal(a[k], b[k], err_msg=k)
