@@ -9,6 +9,7 @@
 // memory across the warps of the lane.  Two iterations are kept in registers (see below).
 #include "common.cuh"
 #include "moa_block.h"
+#include "ptx.cuh"
 
 namespace moa {
 namespace {
@@ -245,6 +246,161 @@ rmsnorm_bwd_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__r
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Ring variant (d <= 2048): the rows come through a shared-memory ring filled by bulk copies, so the
+// bytes in flight no longer depend on what the computing warps hold in registers.  One producer
+// thread keeps kRingStages stages of kRingWarps * m consecutive rows requested (x, and dy in the
+// backward; a stage is one contiguous block of memory per array: one bulk copy each); two groups of
+// eight consumer warps compute alternate stages (all of them follow every stage's barriers), a warp one row at a time (32 lanes x up to 8 vectors of
+// 16 bytes), reduce with shuffles only -- no block barrier in the loop -- and write their results
+// straight to global memory in whole 512-byte runs.  A row is read from shared memory twice (sums,
+// then results) rather than held in registers, and the gain sits in shared memory as floats, which
+// keeps the kernel near 100 registers.  Every wait is bounded.
+constexpr int kRingWarps = 8;                 // consumer warps per group = rows per stage / m
+constexpr int kRingGroups = 2;                // consumer groups; group q takes the CTA's stages q, q + 2, ...
+constexpr int kRingThreads = 32 * (kRingGroups * kRingWarps + 1), kRingStages = 3;
+enum { NERR_EMPTY = 0x401, NERR_FULL = 0x402 };
+
+template <int kV, bool kBwd>
+__global__ void __launch_bounds__(kRingThreads, 1)
+rmsnorm_ring_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ g, const float *__restrict__ r_in,
+                    float *__restrict__ r_out, const __nv_bfloat16 *__restrict__ dy, __nv_bfloat16 *__restrict__ out,
+                    float *__restrict__ part, int n, int d, float eps, int m, unsigned int *status)
+{
+    using namespace ptx;
+    extern __shared__ __align__(128) uint8_t nring[];
+    const int rows_stage = kRingWarps * m;
+    const size_t row_bytes = (size_t)d * 2, arr_bytes = (size_t)rows_stage * row_bytes;
+    const size_t stage_bytes = arr_bytes * (kBwd ? 2 : 1);
+    float *gs = reinterpret_cast<float *>(nring + kRingStages * stage_bytes);          // gain as floats [d]
+    uint64_t *full = reinterpret_cast<uint64_t *>(gs + d);
+    uint64_t *empty = full + kRingStages;
+    volatile uint32_t *abortp = reinterpret_cast<uint32_t *>(empty + kRingStages);
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int nvec = d / 8;
+    const long long total_stages = ((long long)n + rows_stage - 1) / rows_stage;
+    const int my_stages = (int)((total_stages - blockIdx.x + gridDim.x - 1) / gridDim.x);   // stages b, b + grid, ...
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kRingStages; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, kRingGroups * kRingWarps); }
+        *abortp = 0;
+        fence_mbar_init();
+    }
+    for (int i = threadIdx.x; i < d; i += kRingThreads) gs[i] = __bfloat162float(g[i]);
+    __syncthreads();
+    float dgacc[kV][8];          // backward only (dead otherwise)
+#pragma unroll
+    for (int j = 0; j < kV; ++j)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) dgacc[j][e] = 0.f;
+
+    if (warp == kRingGroups * kRingWarps) {
+        if (lane == 0) {
+            for (int i = 0; i < my_stages; ++i) {
+                const int s = i % kRingStages;
+                if (!mbar_wait(empty + s, ((i / kRingStages) & 1) ^ 1, abortp, status, NERR_EMPTY)) break;
+                const long long row0 = ((long long)blockIdx.x + (long long)i * gridDim.x) * rows_stage;
+                const int rows = (int)min((long long)rows_stage, (long long)n - row0);
+                const uint32_t bytes = (uint32_t)(rows * row_bytes);
+                mbar_arrive_expect_tx(full + s, kBwd ? 2 * bytes : bytes);
+                bulk_load_1d(nring + s * stage_bytes, x + row0 * d, bytes, full + s);
+                if (kBwd) bulk_load_1d(nring + s * stage_bytes + arr_bytes, dy + row0 * d, bytes, full + s);
+            }
+        }
+    } else {
+        const float inv_d = 1.f / (float)d;
+        const int grp = warp / kRingWarps, gw = warp % kRingWarps;
+        // Every consumer warp waits for every stage and releases it, in order, although it computes only its
+        // group's: a warp that skipped stages could find a slot's barrier still in the phase of an older stage
+        // of the same parity and take it for the one it is waiting for.
+        for (int i = 0; i < my_stages; ++i) {
+            const int s = i % kRingStages;
+            if (!mbar_wait(full + s, (i / kRingStages) & 1, abortp, status, NERR_FULL)) break;
+            if (i % kRingGroups != grp) {
+                if (lane == 0) mbar_arrive(empty + s);
+                continue;
+            }
+            const long long row0 = ((long long)blockIdx.x + (long long)i * gridDim.x) * rows_stage;
+            const uint8_t *sx = nring + s * stage_bytes, *sd = sx + arr_bytes;
+            for (int q = 0; q < m; ++q) {
+                const int lr = gw * m + q;                    // row of the stage
+                const long long row = row0 + lr;
+                if (row >= n) break;                          // warp-uniform
+                float rr = 0.f;
+                if (kBwd && r_in != nullptr) rr = __ldg(r_in + row);
+                float ss = 0.f, t = 0.f;
+#pragma unroll
+                for (int j = 0; j < kV; ++j) {
+                    const int v = lane + 32 * j;
+                    if (v >= nvec) continue;
+                    float fx[8], fd[8];
+                    unpack8(*reinterpret_cast<const uint4 *>(sx + lr * row_bytes + 16 * v), fx);
+                    if (kBwd) unpack8(*reinterpret_cast<const uint4 *>(sd + lr * row_bytes + 16 * v), fd);
+                    const float4 g0 = *reinterpret_cast<const float4 *>(gs + 8 * v), g1 = *reinterpret_cast<const float4 *>(gs + 8 * v + 4);
+                    const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        ss = fmaf(fx[e], fx[e], ss);
+                        if (kBwd) t = fmaf(fx[e] * gg[e], fd[e], t);
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o >= 1; o >>= 1) {
+                    ss += __shfl_xor_sync(0xffffffffu, ss, o);
+                    if (kBwd) t += __shfl_xor_sync(0xffffffffu, t, o);
+                }
+                const float r = (kBwd && r_in != nullptr) ? rr : rsqrtf(ss * inv_d + eps);
+                if (!kBwd && r_out != nullptr && lane == 0) r_out[row] = r;
+                const float coef = r * r * r * t * inv_d;
+                asm volatile("" ::: "memory");      // second pass reads the row again instead of keeping it in registers
+#pragma unroll
+                for (int j = 0; j < kV; ++j) {
+                    const int v = lane + 32 * j;
+                    if (v >= nvec) continue;
+                    float fx[8], fd[8], o8[8];
+                    unpack8(*reinterpret_cast<const uint4 *>(sx + lr * row_bytes + 16 * v), fx);
+                    if (kBwd) unpack8(*reinterpret_cast<const uint4 *>(sd + lr * row_bytes + 16 * v), fd);
+                    const float4 g0 = *reinterpret_cast<const float4 *>(gs + 8 * v), g1 = *reinterpret_cast<const float4 *>(gs + 8 * v + 4);
+                    const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        if (kBwd) {
+                            o8[e] = r * gg[e] * fd[e] - fx[e] * coef;
+                            dgacc[j][e] = fmaf(fd[e] * fx[e], r, dgacc[j][e]);
+                        } else {
+                            o8[e] = fx[e] * r * gg[e];
+                        }
+                    }
+                    __stcs(reinterpret_cast<uint4 *>(out + (size_t)row * d) + v, pack8(o8));
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty + s);
+        }
+    }
+    if (kBwd) {
+        // CTA partial of dg: the eight warps' sums, added in warp order (the ring is free: every consumer is done)
+        __syncthreads();
+        float *accs = reinterpret_cast<float *>(nring);                     // [consumer warps][d]
+        if (warp < kRingGroups * kRingWarps) {
+#pragma unroll
+            for (int j = 0; j < kV; ++j) {
+                const int v = lane + 32 * j;
+                if (v < nvec)
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) accs[(size_t)warp * d + 8 * v + e] = dgacc[j][e];
+            }
+        }
+        __syncthreads();
+        float *mine = part + (size_t)blockIdx.x * d;
+        for (int col = threadIdx.x; col < d; col += kRingThreads) {
+            float a = 0.f;
+#pragma unroll
+            for (int w = 0; w < kRingGroups * kRingWarps; ++w) a += accs[(size_t)w * d + col];
+            mine[col] = a;
+        }
+    }
+}
+
 // dg[col] = sum over the CTA partials, in a fixed order: a CTA owns 32 columns, its 16 warps take the
 // partial rows w, w + 16, ... (four independent running sums each, so that the loads overlap) and the
 // sums are added in a fixed order.
@@ -300,9 +456,50 @@ NormPlan norm_plan(int n, int d, bool bwd)
     return p;
 }
 
+
+// The ring variant serves rows of 256 .. 2048 elements (a warp per row, at most 8 vectors per lane).
+bool norm_uses_ring(int d) { return d >= 256 && d <= 2048; }
+struct RingPlan {
+    int kV, m, grid;
+    size_t smem;
+};
+RingPlan ring_plan(int n, int d, bool bwd)
+{
+    RingPlan p{};
+    const int nvec = d / 8, need = (nvec + 31) / 32;
+    p.kV = need <= 1 ? 1 : need <= 2 ? 2 : need <= 4 ? 4 : 8;
+    p.m = 2048 / d < 1 ? 1 : 2048 / d;                                  // 32 KB per array and stage
+    const long long rows_stage = (long long)kRingWarps * p.m;
+    const long long stages = ((long long)n + rows_stage - 1) / rows_stage;
+    p.grid = (int)(stages < 148 ? stages : 148);
+    p.smem = (size_t)kRingStages * rows_stage * d * 2 * (bwd ? 2 : 1) + (size_t)d * 4 + 2 * kRingStages * 8 + 16;
+    return p;
+}
+
+template <int kV, bool kBwd>
+cudaError_t launch_ring(const RingPlan &p, const __nv_bfloat16 *x, const __nv_bfloat16 *g, const float *r_in, float *r_out,
+                        const __nv_bfloat16 *dy, __nv_bfloat16 *out, float *part, int n, int d, float eps, cudaStream_t st)
+{
+    cudaError_t e = cudaFuncSetAttribute(rmsnorm_ring_kernel<kV, kBwd>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
+    if (e != cudaSuccess) return e;
+    rmsnorm_ring_kernel<kV, kBwd><<<p.grid, kRingThreads, p.smem, st>>>(x, g, r_in, r_out, dy, out, part, n, d, eps, p.m,
+                                                                        device_status_ptr());
+    return cudaGetLastError();
+}
+template <bool kBwd>
+cudaError_t launch_ring_kv(const RingPlan &p, const __nv_bfloat16 *x, const __nv_bfloat16 *g, const float *r_in, float *r_out,
+                           const __nv_bfloat16 *dy, __nv_bfloat16 *out, float *part, int n, int d, float eps, cudaStream_t st)
+{
+    if (p.kV == 1) return launch_ring<1, kBwd>(p, x, g, r_in, r_out, dy, out, part, n, d, eps, st);
+    if (p.kV == 2) return launch_ring<2, kBwd>(p, x, g, r_in, r_out, dy, out, part, n, d, eps, st);
+    if (p.kV == 4) return launch_ring<4, kBwd>(p, x, g, r_in, r_out, dy, out, part, n, d, eps, st);
+    return launch_ring<8, kBwd>(p, x, g, r_in, r_out, dy, out, part, n, d, eps, st);
+}
+
 }  // namespace
 
-size_t rmsnorm_workspace_bytes(int n, int d) { return (size_t)norm_plan(n, d, true).grid * d * sizeof(float); }
+// per-CTA partial sums of dg: at most 148 * 4 CTAs in either variant
+size_t rmsnorm_workspace_bytes(int n, int d) { (void)n; return (size_t)148 * 4 * d * sizeof(float); }
 
 cudaError_t rmsnorm_fwd(int n, int d, float eps, const void *x, const void *g, void *y, float *r, cudaStream_t st)
 {
@@ -311,6 +508,7 @@ cudaError_t rmsnorm_fwd(int n, int d, float eps, const void *x, const void *g, v
     const auto *gb = (const __nv_bfloat16 *)g;
     auto *yb = (__nv_bfloat16 *)y;
     LaunchScope scope(MOA_KERNEL_OTHER, st);
+    if (norm_uses_ring(d)) return launch_ring_kv<false>(ring_plan(n, d, false), xb, gb, nullptr, r, nullptr, yb, nullptr, n, d, eps, st);
     if (p.kV == 1) rmsnorm_fwd_kernel<1, 2><<<p.grid, kNormThreads, 0, st>>>(xb, gb, yb, r, n, d, eps, p.tpr);
     else if (p.kV == 2) rmsnorm_fwd_kernel<2, 1><<<p.grid, kNormThreads, 0, st>>>(xb, gb, yb, r, n, d, eps, p.tpr);
     else rmsnorm_fwd_kernel<4, 1><<<p.grid, kNormThreads, 0, st>>>(xb, gb, yb, r, n, d, eps, p.tpr);
@@ -326,7 +524,14 @@ cudaError_t rmsnorm_bwd(int n, int d, float eps, const void *x, const void *g, c
     const auto *db = (const __nv_bfloat16 *)dy;
     auto *ob = (__nv_bfloat16 *)dx;
     float *part = (float *)ws;
-    {
+    int parts = p.grid;
+    if (norm_uses_ring(d)) {
+        const RingPlan rp = ring_plan(n, d, true);
+        parts = rp.grid;
+        LaunchScope scope(MOA_KERNEL_OTHER, st);
+        const cudaError_t e = launch_ring_kv<true>(rp, xb, gb, r, nullptr, db, ob, part, n, d, eps, st);
+        if (e != cudaSuccess) return e;
+    } else {
         LaunchScope scope(MOA_KERNEL_OTHER, st);
         if (p.kV == 1) rmsnorm_bwd_kernel<1, 2><<<p.grid, kNormThreads, 0, st>>>(xb, gb, r, db, ob, part, n, d, eps, p.tpr);
         else if (p.kV == 2) rmsnorm_bwd_kernel<2, 1><<<p.grid, kNormThreads, 0, st>>>(xb, gb, r, db, ob, part, n, d, eps, p.tpr);
@@ -335,7 +540,7 @@ cudaError_t rmsnorm_bwd(int n, int d, float eps, const void *x, const void *g, c
         if (e != cudaSuccess) return e;
     }
     LaunchScope scope(MOA_KERNEL_OTHER, st);
-    rmsnorm_dg_kernel<<<(d + 31) / 32, 32 * kDgWarps, 0, st>>>(part, (__nv_bfloat16 *)dg, p.grid, d);
+    rmsnorm_dg_kernel<<<(d + 31) / 32, 32 * kDgWarps, 0, st>>>(part, (__nv_bfloat16 *)dg, parts, d);
     return cudaGetLastError();
 }
 

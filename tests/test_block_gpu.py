@@ -199,3 +199,32 @@ def test_gated_mlp_is_bitwise_reproducible(rt):
     b = _run_mlp(rt, inp)
     for k in a:
         np.testing.assert_array_equal(a[k], b[k], err_msg=k)
+
+
+def test_rmsnorm_long_run_through_the_ring(rt):
+    """n = 32768 rows of 2048 (many trips round the shared-memory ring in every CTA): all of y, dx, dg against
+    the oracle, and 200 repeated forward+backward launches give identical bits (no stage taken for another)."""
+    torch, mb = rt
+    n, d, eps = 32768, 2048, 1e-5
+    inp = mi.make_norm_inputs(n, d, seed=31)
+    f = {k: mi.to_f64(v, "bf16") for k, v in inp.items()}
+    ref = oracle.rmsnorm_fwd_bwd(f["x"], f["g"], f["dy"], eps)
+    first = _run_rmsnorm(rt, inp, eps)
+    for k in ("y", "dx", "dg"):
+        assert mi.rel_err(first[k], ref[k]) <= TOL, (k, mi.rel_err(first[k], ref[k]))
+    x, g, dy = (_dev(torch, inp[k]) for k in ("x", "g", "dy"))
+    desc = mb.make_rmsnorm_desc(n, d, eps)
+    y, dx, dg = torch.empty_like(x), torch.empty_like(x), torch.empty_like(g)
+    r = torch.empty((n,), dtype=torch.float32, device="cuda")
+    ws = torch.empty(mb.moa_rmsnorm_workspace_bytes(desc), dtype=torch.uint8, device="cuda")
+    y0 = dx0 = dg0 = None
+    for it in range(200):
+        mb.moa_rmsnorm_fwd(desc, x, g, y, r)
+        mb.moa_rmsnorm_bwd(desc, x, g, r, dy, dx, dg, ws)
+        if it % 50 == 0:
+            if y0 is None:
+                y0, dx0, dg0 = y.clone(), dx.clone(), dg.clone()
+            else:
+                assert torch.equal(y, y0) and torch.equal(dx, dx0) and torch.equal(dg, dg0), it
+    assert mb.moa_last_device_status() == mb.MOA_OK
+    assert torch.equal(y, y0) and torch.equal(dx, dx0) and torch.equal(dg, dg0)
