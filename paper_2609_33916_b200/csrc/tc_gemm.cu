@@ -78,7 +78,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapB0,
                const __grid_constant__ CUtensorMap mapA1, const __grid_constant__ CUtensorMap mapB1,
                const __grid_constant__ CUtensorMap mapC0, const __grid_constant__ CUtensorMap mapC1,
-               const __grid_constant__ CUtensorMap mapC2, const __grid_constant__ CUtensorMap mapC3, int M, int N, int K, int nparts, int nbatch, unsigned int *status)
+               const __grid_constant__ CUtensorMap mapC2, const __grid_constant__ CUtensorMap mapC3, int M, int N, int K, int nparts, int nbatch, int a_blocked, int b_blocked, unsigned int *status)
 {
     constexpr bool kDualN = kEpi == EPI_SWIGLU_FWD;         // B tile = 128 rows of map B0 + 128 rows of map B1
     constexpr int kTileN = kDualN ? 128 : GN;                // output columns a tile covers
@@ -142,14 +142,22 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                 uint64_t *full = bars + G_FULL + s;
                 mbar_arrive_expect_tx(full, kStageBytes);
                 if (kAMn) {
-                    tma_load_3d(sa, ma, full, m0, k0, 0);
-                    tma_load_3d(sa + kMnBox, ma, full, m0 + 64, k0, 0);
+                    if (a_blocked) {                          // one copy: (64 columns, K rows, column blocks)
+                        tma_load_3d(sa, ma, full, 0, k0, m0 / 64);
+                    } else {
+                        tma_load_3d(sa, ma, full, m0, k0, 0);
+                        tma_load_3d(sa + kMnBox, ma, full, m0 + 64, k0, 0);
+                    }
                 } else {
                     tma_load_3d(sa, ma, full, k0, m0, 0);
                 }
                 if (kBMn) {
+                    if (b_blocked) {
+                        tma_load_3d(sb, mb, full, 0, k0, n0 / 64);
+                    } else {
 #pragma unroll
-                    for (int b = 0; b < 4; ++b) tma_load_3d(sb + b * kMnBox, mb, full, n0 + 64 * b, k0, 0);
+                        for (int b = 0; b < 4; ++b) tma_load_3d(sb + b * kMnBox, mb, full, n0 + 64 * b, k0, 0);
+                    }
                 } else if (kDualN) {
                     tma_load_3d(sb, &mapB0, full, k0, n0, 0);
                     tma_load_3d(sb + kBBytes / 2, &mapB1, full, k0, n0, 0);
@@ -338,9 +346,13 @@ struct Operand {
     int rows, cols;          // the array as stored: [rows, cols] row-major
 };
 
-// K-major: stored [MN, K], box of `box_rows` rows x 64 K-elements.  MN-major: stored [K, MN], box of 64 x 64.
-bool operand_map(CUtensorMap *m, const Operand &o, bool mn_major, int box_rows)
+// K-major: stored [MN, K], box of `box_rows` rows x 64 K-elements.  MN-major: stored [K, MN]: one blocked box of
+// box_rows / 64 column blocks x 64 K-rows when `blocked`, else boxes of 64 x 64.
+bool operand_map(CUtensorMap *m, const Operand &o, bool mn_major, int box_rows, bool blocked = false)
 {
+    if (mn_major && blocked)
+        return make_tensor_map_blocked(m, o.p, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)o.rows, (uint64_t)o.cols, 64,
+                                       (uint32_t)box_rows / 64);
     return make_tensor_map_3d(m, o.p, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 1, (uint64_t)o.rows, (uint64_t)o.cols,
                               mn_major ? 64 : (uint32_t)box_rows, 64);
 }
@@ -354,9 +366,15 @@ cudaError_t launch_gemm(const Operand &A0, const Operand &B0, const Operand *A1,
     constexpr bool kDualN = kEpi == EPI_SWIGLU_FWD;
     CUtensorMap ma0, mb0, ma1, mb1;
     const int b_rows = kDualN ? 128 : GN;
-    if (!operand_map(&ma0, A0, kAMn, GM) || !operand_map(&mb0, B0, kBMn, b_rows)) return cudaErrorInvalidValue;
-    if (!operand_map(&ma1, A1 ? *A1 : A0, kAMn, GM) || !operand_map(&mb1, B1 ? *B1 : B0, kBMn, b_rows))
-        return cudaErrorInvalidValue;
+    // MN-major operands whose width is a multiple of 64 come in by one blocked copy per stage (try the encode; if the
+    // driver refuses the map, or a width has a tail, use one copy per 64-column block)
+    const Operand &a1 = A1 ? *A1 : A0, &b1 = B1 ? *B1 : B0;
+    bool a_blocked = kAMn && A0.cols % 64 == 0 && a1.cols % 64 == 0;
+    bool b_blocked = kBMn && B0.cols % 64 == 0 && b1.cols % 64 == 0;
+    if (a_blocked && !(operand_map(&ma0, A0, true, GM, true) && operand_map(&ma1, a1, true, GM, true))) a_blocked = false;
+    if (b_blocked && !(operand_map(&mb0, B0, true, b_rows, true) && operand_map(&mb1, b1, true, b_rows, true))) b_blocked = false;
+    if (!a_blocked && (!operand_map(&ma0, A0, kAMn, GM) || !operand_map(&ma1, a1, kAMn, GM))) return cudaErrorInvalidValue;
+    if (!b_blocked && (!operand_map(&mb0, B0, kBMn, b_rows) || !operand_map(&mb1, b1, kBMn, b_rows))) return cudaErrorInvalidValue;
     CUtensorMap mc[4];
     const void *cs[4] = {C0, C1 ? C1 : C0, C2 ? C2 : C0, C3 ? C3 : C0};
     for (int i = 0; i < 4; ++i)     // [c_rows, ldc] bf16, boxes of 128 rows x 64 columns, 128-byte swizzle
@@ -369,7 +387,8 @@ cudaError_t launch_gemm(const Operand &A0, const Operand &B0, const Operand *A1,
     const int nparts = (A1 && !kDualN && nbatch == 1) ? 2 : 1;
     LaunchScope scope(MOA_KERNEL_OTHER, st);
     kernel<<<tiles < 148 ? tiles : 148, kGemmThreads, kGemmSmem, st>>>(ma0, mb0, ma1, mb1, mc[0], mc[1], mc[2], mc[3], M, N, K, nparts,
-                                                                      nbatch, device_status_ptr());
+                                                                      nbatch, a_blocked ? 1 : 0, b_blocked ? 1 : 0,
+                                                                      device_status_ptr());
     return cudaGetLastError();
 }
 

@@ -59,4 +59,18 @@ bool make_tensor_map_4d(CUtensorMap *map, const void *base, CUtensorMapDataType 
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+bool make_tensor_map_blocked(CUtensorMap *map, const void *base, CUtensorMapDataType dt, int elem_bytes,
+                             uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t nblk)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn || cols % 64 != 0 || elem_bytes != 2) return false;
+    const uint64_t eb = (uint64_t)elem_bytes;
+    cuuint64_t gdim[3] = {64, rows, cols / 64};
+    cuuint64_t gstride[2] = {cols * eb, 64 * eb};          // row stride, then the 128-byte step between column blocks
+    cuuint32_t box[3] = {64, box_rows, nblk};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, dt, 3, const_cast<void *>(base), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace moa
