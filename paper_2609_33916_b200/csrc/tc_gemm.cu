@@ -59,7 +59,16 @@ __device__ __forceinline__ void unpack8(const uint4 &v, float *f)
         f[2 * i + 1] = t.y;
     }
 }
-__device__ __forceinline__ float sigmoidf_fast(float a) { return __frcp_rn(1.f + __expf(-a)); }
+// 1 / (1 + exp(-a)) on the two fast special-function instructions (ex2.approx, rcp.approx).  (__frcp_rn, the
+// correctly rounded reciprocal, is a multi-instruction sequence: with it the backward gate epilogue took 17,000
+// cycles per tile instead of 6,800 and held its GEMM 25 % below the others.)
+__device__ __forceinline__ float sigmoidf_fast(float a)
+{
+    float e, r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(-1.4426950408889634f * a));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.f + e));
+    return r;
+}
 
 // Tile order: groups of 8 tile rows, column-major inside a group, so that the CTAs running at the
 // same time share a few A row blocks and a few B column blocks.
