@@ -14,4 +14,6 @@ from .attention import (  # noqa: F401
     attn_cols,
 )
 from .decode import decode_attn  # noqa: F401,E402
-from .block import rmsnorm_fwd_bwd, gated_mlp_fwd_bwd, gated_mlp_bwd_from_saved  # noqa: F401,E402
+from .block import (  # noqa: F401,E402
+    rmsnorm_fwd_bwd, gated_mlp_fwd_bwd, gated_mlp_bwd_from_saved, gemm, transformer_block_fwd_bwd,
+)

@@ -193,3 +193,48 @@ def test_gated_mlp_invariants():
     b = ob.gated_mlp_bwd_from_saved(x, r["a"], r["u"], W1, W3, W2, dy)
     for k in ("dx", "dW1", "dW3", "dW2", "h"):
         np.testing.assert_allclose(b[k], r[k], rtol=1e-13, atol=1e-14, err_msg=k)
+
+
+# ------------------------------------------------------------- GEMM layouts, the whole block
+def test_gemm_layouts_by_hand():
+    A = np.array([[1.0, 2.0, 3.0], [4.0, 5.0, 6.0]])            # [M=2, K=3]
+    Bm = np.array([[1.0, 0.0, -1.0], [2.0, 1.0, 0.0]])           # [N=2, K=3]
+    want = np.array([[-2.0, 4.0], [-2.0, 13.0]])                 # rows of A dotted with rows of B
+    np.testing.assert_array_equal(ob.gemm(A, Bm), want)
+    np.testing.assert_array_equal(ob.gemm(A.T.copy(), Bm, a_layout=1), want)
+    np.testing.assert_array_equal(ob.gemm(A, Bm.T.copy(), b_layout=1), want)
+    np.testing.assert_array_equal(ob.gemm(A.T.copy(), Bm.T.copy(), a_layout=1, b_layout=1), want)
+    np.testing.assert_array_equal(ob.gemm(A, Bm, R=np.ones((2, 2))), want + 1.0)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_transformer_block_matches_library_autograd(causal):
+    """The composed block against the library's own routines under autograd (fp64): rms_norm, linear,
+    scaled_dot_product_attention, silu."""
+    rng = _rng(21)
+    B, n, H, d, dff, eps = 2, 5, 3, 4, 7, 1e-3
+    T, dm = B * n, H * d
+    x, dy = rng.standard_normal((T, dm)), rng.standard_normal((T, dm))
+    w = dict(g1=1 + 0.3 * rng.standard_normal(dm), g2=1 + 0.3 * rng.standard_normal(dm),
+             Wq=rng.standard_normal((dm, dm)) / 3, Wk=rng.standard_normal((dm, dm)) / 3, Wv=rng.standard_normal((dm, dm)) / 3,
+             Wo=rng.standard_normal((dm, dm)) / 3, W1=rng.standard_normal((dff, dm)) / 3, W3=rng.standard_normal((dff, dm)) / 3,
+             W2=rng.standard_normal((dm, dff)) / 3)
+    ref = ob.transformer_block_fwd_bwd(x, w, dy, B, n, H, causal, eps)
+    F = torch.nn.functional
+    tx = torch.tensor(x, requires_grad=True)
+    tw = {k: torch.tensor(v, requires_grad=True) for k, v in w.items()}
+
+    def heads(t):
+        return t.reshape(B, n, H, d).permute(0, 2, 1, 3)
+
+    h1 = F.rms_norm(tx, (dm,), weight=tw["g1"], eps=eps)
+    q, k, v = (heads(F.linear(h1, tw[m])) for m in ("Wq", "Wk", "Wv"))
+    o = F.scaled_dot_product_attention(q, k, v, is_causal=causal).permute(0, 2, 1, 3).reshape(T, dm)
+    x2 = tx + F.linear(o, tw["Wo"])
+    h2 = F.rms_norm(x2, (dm,), weight=tw["g2"], eps=eps)
+    y = x2 + F.linear(F.silu(F.linear(h2, tw["W1"])) * F.linear(h2, tw["W3"]), tw["W2"])
+    y.backward(torch.tensor(dy))
+    np.testing.assert_allclose(ref["y"], y.detach().numpy(), rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(ref["dx"], tx.grad.numpy(), rtol=1e-10, atol=1e-11)
+    for name in w:
+        np.testing.assert_allclose(ref["d" + name], tw[name].grad.numpy(), rtol=1e-10, atol=1e-11, err_msg=name)
