@@ -1,6 +1,6 @@
 /*
  * moa_block.h -- C ABI of the token-wise pieces of the transformer block for NVIDIA B200
- * (sm_100a): RMSNorm and the gated MLP, each forward and backward.
+ * (sm_100a): RMSNorm and the gated MLP, each forward and backward, and the GEMM of the projections.
  *
  * These are the pieces the paper's block section puts around attention ("RMSNorm, gated MLP",
  * hidden width d_ff, with the gated-MLP backward the dominant kernel of its block profile).
@@ -44,9 +44,11 @@ moa_status moa_rmsnorm_fwd(const moa_rmsnorm_desc *desc, const void *x, const vo
                            void *y, float *r, void *stream);
 
 /* Reads x, g, dy and r (as written by the forward for the same x; NULL: recomputed from x);
- * writes dx and dg. */
+ * writes dx and dg.  dx_add (NULL or [n,d]) is added to dx: the gradient that reaches x past the
+ * norm, along a residual connection. */
 moa_status moa_rmsnorm_bwd(const moa_rmsnorm_desc *desc, const void *x, const void *g, const float *r,
-                           const void *dy, void *dx, void *dg, void *ws, size_t ws_bytes, void *stream);
+                           const void *dy, const void *dx_add, void *dx, void *dg,
+                           void *ws, size_t ws_bytes, void *stream);
 
 /* ----------------------------------------------------------------------- gated MLP
  * SiLU-gated MLP without biases, weights stored [out, in]:
@@ -64,9 +66,10 @@ typedef struct {
     int32_t dtype;
 } moa_mlp_desc;
 
-/* Forward.  Reads x, W1, W3, W2; writes a, u, h (kept for the backward, bf16) and y. */
+/* Forward.  Reads x, W1, W3, W2; writes a, u, h (kept for the backward, bf16) and y.  res (NULL or
+ * [n,d]) is added to y in the epilogue of the last GEMM: the block's residual connection. */
 moa_status moa_gated_mlp_fwd(const moa_mlp_desc *desc, const void *x, const void *W1, const void *W3,
-                             const void *W2, void *a, void *u, void *h, void *y, void *stream);
+                             const void *W2, const void *res, void *a, void *u, void *h, void *y, void *stream);
 
 /* Workspace of the backward: da and du, [n,d_ff] each in the storage type.  0 for an invalid desc. */
 size_t moa_gated_mlp_workspace_bytes(const moa_mlp_desc *desc);
@@ -77,6 +80,22 @@ moa_status moa_gated_mlp_bwd(const moa_mlp_desc *desc, const void *x, const void
                              const void *W2, const void *a, const void *u, const void *h, const void *dy,
                              void *dx, void *dW1, void *dW3, void *dW2,
                              void *ws, size_t ws_bytes, void *stream);
+
+/* ------------------------------------------------------------------------------ GEMM
+ * The product the block's projections and their backward passes need, on the same tensor-core
+ * kernel as the gated MLP:   C[M,N] = A B^T (+ R)
+ * A is given as [M,K] row-major (a_layout = 0) or as [K,M] row-major (a_layout = 1); B as [N,K]
+ * row-major (b_layout = 0) or as [K,N] row-major (b_layout = 1); C and the optional R are [M,N].
+ * With weights stored [out,in]:  y = x W^T is (0,0);  dx = dy W is (0,1);  dW = dy^T x is (1,1) with
+ * M = out, N = in, K = tokens.  R (NULL or [M,N]) is added in the epilogue: a residual connection, or
+ * the running sum of a chain of products.  M, N, K >= 1; the row length of every array a multiple of
+ * 8 (rows stay 16-byte aligned); dtype MOA_BF16; fp32 accumulation. */
+typedef struct {
+    int32_t M, N, K;
+    int32_t a_layout, b_layout;
+    int32_t dtype;
+} moa_gemm_desc;
+moa_status moa_gemm(const moa_gemm_desc *desc, const void *A, const void *B, const void *R, void *C, void *stream);
 
 #ifdef __cplusplus
 }

@@ -29,7 +29,7 @@ EXPORTS = (
     "moa_profile_enable", "moa_profile_read", "moa_attn_bwd_static_scratch", "moa_attn_fused_rowparallel",
     "moa_decode_workspace_bytes", "moa_decode_attn",
     "moa_rmsnorm_workspace_bytes", "moa_rmsnorm_fwd", "moa_rmsnorm_bwd",
-    "moa_gated_mlp_fwd", "moa_gated_mlp_workspace_bytes", "moa_gated_mlp_bwd",
+    "moa_gated_mlp_fwd", "moa_gated_mlp_workspace_bytes", "moa_gated_mlp_bwd", "moa_gemm",
 )
 
 
@@ -47,6 +47,11 @@ class moa_decode_desc(ctypes.Structure):
 
 class moa_rmsnorm_desc(ctypes.Structure):
     _fields_ = [("n", ctypes.c_int32), ("d", ctypes.c_int32), ("eps", ctypes.c_float), ("dtype", ctypes.c_int32)]
+
+
+class moa_gemm_desc(ctypes.Structure):
+    _fields_ = [("M", ctypes.c_int32), ("N", ctypes.c_int32), ("K", ctypes.c_int32), ("a_layout", ctypes.c_int32),
+                ("b_layout", ctypes.c_int32), ("dtype", ctypes.c_int32)]
 
 
 class moa_mlp_desc(ctypes.Structure):
@@ -101,12 +106,14 @@ def lib() -> ctypes.CDLL:
         L.moa_rmsnorm_fwd.restype = ctypes.c_int
         L.moa_rmsnorm_fwd.argtypes = [rp] + [vp] * 4 + [vp]
         L.moa_rmsnorm_bwd.restype = ctypes.c_int
-        L.moa_rmsnorm_bwd.argtypes = [rp] + [vp] * 6 + [vp, sz, vp]
+        L.moa_rmsnorm_bwd.argtypes = [rp] + [vp] * 7 + [vp, sz, vp]
         mp = ctypes.POINTER(moa_mlp_desc)
         L.moa_gated_mlp_workspace_bytes.restype = sz
         L.moa_gated_mlp_workspace_bytes.argtypes = [mp]
         L.moa_gated_mlp_fwd.restype = ctypes.c_int
-        L.moa_gated_mlp_fwd.argtypes = [mp] + [vp] * 8 + [vp]
+        L.moa_gated_mlp_fwd.argtypes = [mp] + [vp] * 9 + [vp]
+        L.moa_gemm.restype = ctypes.c_int
+        L.moa_gemm.argtypes = [ctypes.POINTER(moa_gemm_desc)] + [vp] * 4 + [vp]
         L.moa_gated_mlp_bwd.restype = ctypes.c_int
         L.moa_gated_mlp_bwd.argtypes = [mp] + [vp] * 12 + [vp, sz, vp]
         L.moa_last_device_status.restype = ctypes.c_int
@@ -235,11 +242,24 @@ def moa_rmsnorm_fwd(desc, x, g, y, r=None, stream=None, check=True) -> int:
     return s
 
 
-def moa_rmsnorm_bwd(desc, x, g, r, dy, dx, dg, ws=None, stream=None, ws_bytes=None, check=True) -> int:
-    s = lib().moa_rmsnorm_bwd(ctypes.byref(desc), _ptr(x), _ptr(g), _ptr(r), _ptr(dy), _ptr(dx), _ptr(dg), _ptr(ws),
+def moa_rmsnorm_bwd(desc, x, g, r, dy, dx, dg, ws=None, stream=None, ws_bytes=None, check=True, dx_add=None) -> int:
+    """dx_add (optional, [n,d]): added to dx (the gradient arriving along a residual connection)."""
+    s = lib().moa_rmsnorm_bwd(ctypes.byref(desc), _ptr(x), _ptr(g), _ptr(r), _ptr(dy), _ptr(dx_add), _ptr(dx), _ptr(dg), _ptr(ws),
                               _nbytes(ws) if ws_bytes is None else ws_bytes, _stream(stream))
     if check and s != MOA_OK:
         raise MoaError(s, "moa_rmsnorm_bwd")
+    return s
+
+
+def make_gemm_desc(M, N, K, a_layout=0, b_layout=0, dtype=MOA_BF16) -> moa_gemm_desc:
+    """C[M,N] = A B^T (+ R); a_layout 0: A is [M,K], 1: A is [K,M]; b_layout 0: B is [N,K], 1: B is [K,N]."""
+    return moa_gemm_desc(int(M), int(N), int(K), int(a_layout), int(b_layout), int(dtype))
+
+
+def moa_gemm(desc, A, B, C, R=None, stream=None, check=True) -> int:
+    s = lib().moa_gemm(ctypes.byref(desc), _ptr(A), _ptr(B), _ptr(R), _ptr(C), _stream(stream))
+    if check and s != MOA_OK:
+        raise MoaError(s, "moa_gemm")
     return s
 
 
@@ -251,8 +271,9 @@ def moa_gated_mlp_workspace_bytes(desc) -> int:
     return int(lib().moa_gated_mlp_workspace_bytes(ctypes.byref(desc)))
 
 
-def moa_gated_mlp_fwd(desc, x, W1, W3, W2, a, u, h, y, stream=None, check=True) -> int:
-    s = lib().moa_gated_mlp_fwd(ctypes.byref(desc), _ptr(x), _ptr(W1), _ptr(W3), _ptr(W2), _ptr(a), _ptr(u), _ptr(h),
+def moa_gated_mlp_fwd(desc, x, W1, W3, W2, a, u, h, y, stream=None, check=True, res=None) -> int:
+    """res (optional, [n,d]): added to y (the block's residual connection)."""
+    s = lib().moa_gated_mlp_fwd(ctypes.byref(desc), _ptr(x), _ptr(W1), _ptr(W3), _ptr(W2), _ptr(res), _ptr(a), _ptr(u), _ptr(h),
                                 _ptr(y), _stream(stream))
     if check and s != MOA_OK:
         raise MoaError(s, "moa_gated_mlp_fwd")

@@ -55,17 +55,18 @@ moa_status moa_rmsnorm_fwd(const moa_rmsnorm_desc *desc, const void *x, const vo
 }
 
 moa_status moa_rmsnorm_bwd(const moa_rmsnorm_desc *desc, const void *x, const void *g, const float *r,
-                           const void *dy, void *dx, void *dg, void *ws, size_t ws_bytes, void *stream)
+                           const void *dy, const void *dx_add, void *dx, void *dg, void *ws, size_t ws_bytes, void *stream)
 {
     moa_status s = check_rmsnorm(desc);
     if (s != MOA_OK) return s;
     if (!x || !g || !dy || !dx || !dg) return MOA_ERR_INVALID_ARG;
-    if (!aligned16(x) || !aligned16(g) || !aligned16(dy) || !aligned16(dx) || !aligned16(dg) || (r && !aligned16(r)))
+    if (!aligned16(x) || !aligned16(g) || !aligned16(dy) || !aligned16(dx) || !aligned16(dg) || (r && !aligned16(r)) ||
+        (dx_add && !aligned16(dx_add)))
         return MOA_ERR_INVALID_ARG;
     if (!ws || ws_bytes < rmsnorm_workspace_bytes(desc->n, desc->d)) return MOA_ERR_WORKSPACE;
     if (!aligned16(ws)) return MOA_ERR_INVALID_ARG;
     if ((s = check_device_arch()) != MOA_OK) return s;
-    return rmsnorm_bwd(desc->n, desc->d, desc->eps, x, g, r, dy, dx, dg, ws, (cudaStream_t)stream) == cudaSuccess
+    return rmsnorm_bwd(desc->n, desc->d, desc->eps, x, g, r, dy, dx_add, dx, dg, ws, (cudaStream_t)stream) == cudaSuccess
                ? MOA_OK : MOA_ERR_CUDA;
 }
 
@@ -76,16 +77,16 @@ size_t moa_gated_mlp_workspace_bytes(const moa_mlp_desc *desc)
 }
 
 moa_status moa_gated_mlp_fwd(const moa_mlp_desc *desc, const void *x, const void *W1, const void *W3, const void *W2,
-                             void *a, void *u, void *h, void *y, void *stream)
+                             const void *res, void *a, void *u, void *h, void *y, void *stream)
 {
     moa_status s = check_mlp(desc);
     if (s != MOA_OK) return s;
     if (!x || !W1 || !W3 || !W2 || !a || !u || !h || !y) return MOA_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(W1) || !aligned16(W3) || !aligned16(W2) || !aligned16(a) || !aligned16(u) ||
-        !aligned16(h) || !aligned16(y))
+        !aligned16(h) || !aligned16(y) || (res && !aligned16(res)))
         return MOA_ERR_INVALID_ARG;
     if ((s = check_device_arch()) != MOA_OK) return s;
-    return gated_mlp_fwd(desc->n, desc->d, desc->d_ff, x, W1, W3, W2, a, u, h, y, (cudaStream_t)stream) == cudaSuccess
+    return gated_mlp_fwd(desc->n, desc->d, desc->d_ff, x, W1, W3, W2, res, a, u, h, y, (cudaStream_t)stream) == cudaSuccess
                ? MOA_OK : MOA_ERR_CUDA;
 }
 
@@ -105,6 +106,24 @@ moa_status moa_gated_mlp_bwd(const moa_mlp_desc *desc, const void *x, const void
     void *da = ws, *du = (char *)ws + mlp_half_ws(desc);
     return gated_mlp_bwd(desc->n, desc->d, desc->d_ff, x, W1, W3, W2, a, u, h, dy, da, du, dx, dW1, dW3, dW2,
                          (cudaStream_t)stream) == cudaSuccess ? MOA_OK : MOA_ERR_CUDA;
+}
+
+moa_status moa_gemm(const moa_gemm_desc *desc, const void *A, const void *B, const void *R, void *C, void *stream)
+{
+    if (!desc) return MOA_ERR_INVALID_ARG;
+    if (desc->M <= 0 || desc->N <= 0 || desc->K <= 0) return MOA_ERR_INVALID_ARG;
+    if ((desc->a_layout != 0 && desc->a_layout != 1) || (desc->b_layout != 0 && desc->b_layout != 1)) return MOA_ERR_INVALID_ARG;
+    if (desc->dtype != MOA_BF16 && desc->dtype != MOA_F32) return MOA_ERR_INVALID_ARG;
+    if (desc->dtype != MOA_BF16) return MOA_ERR_UNSUPPORTED;
+    // row lengths: A [M,K] or [K,M]; B [N,K] or [K,N]; C, R [M,N]
+    const int a_cols = desc->a_layout ? desc->M : desc->K, b_cols = desc->b_layout ? desc->N : desc->K;
+    if (a_cols % 8 != 0 || b_cols % 8 != 0 || desc->N % 8 != 0) return MOA_ERR_UNSUPPORTED;
+    if (!A || !B || !C) return MOA_ERR_INVALID_ARG;
+    if (!aligned16(A) || !aligned16(B) || !aligned16(C) || (R && !aligned16(R))) return MOA_ERR_INVALID_ARG;
+    moa_status s = check_device_arch();
+    if (s != MOA_OK) return s;
+    return gemm_bf16(desc->a_layout, desc->b_layout, desc->M, desc->N, desc->K, A, B, R, C, (cudaStream_t)stream) == cudaSuccess
+               ? MOA_OK : MOA_ERR_CUDA;
 }
 
 }  // extern "C"

@@ -153,7 +153,8 @@ template <int kV, int R>
 __global__ void __launch_bounds__(kNormThreads)
 rmsnorm_bwd_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ g,
                    const float *__restrict__ r_in, const __nv_bfloat16 *__restrict__ dy,
-                   __nv_bfloat16 *__restrict__ dx, float *__restrict__ part, int n, int d, float eps, int tpr)
+                   const __nv_bfloat16 *__restrict__ dx_add, __nv_bfloat16 *__restrict__ dx, float *__restrict__ part, int n,
+                   int d, float eps, int tpr)
 {
     __shared__ float red[8 * R];
     __shared__ float acc[kNormThreads * 8];              // [row lane][tpr*8] for one j at a time
@@ -214,12 +215,13 @@ rmsnorm_bwd_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__r
             for (int j = 0; j < kV; ++j) {
                 const int v = c + j * tpr;
                 if (v >= nvec) continue;
-                float fx[8], fd[8], o[8];
+                float fx[8], fd[8], o[8], fa[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
                 unpack8(xc.v[i][j], fx);
                 unpack8(dc.v[i][j], fd);
+                if (dx_add != nullptr) unpack8(__ldcs(reinterpret_cast<const uint4 *>(dx_add + (size_t)(row0 + i) * d) + v), fa);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    o[e] = r * gf[j][e] * fd[e] - fx[e] * coef;
+                    o[e] = r * gf[j][e] * fd[e] - fx[e] * coef + fa[e];
                     dgacc[j][e] = fmaf(fd[e] * fx[e], r, dgacc[j][e]);
                 }
                 __stcs(reinterpret_cast<uint4 *>(dx + (size_t)(row0 + i) * d) + v, pack8(o));
@@ -264,8 +266,9 @@ enum { NERR_EMPTY = 0x401, NERR_FULL = 0x402 };
 template <int kV, bool kBwd>
 __global__ void __launch_bounds__(kRingThreads, 1)
 rmsnorm_ring_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ g, const float *__restrict__ r_in,
-                    float *__restrict__ r_out, const __nv_bfloat16 *__restrict__ dy, __nv_bfloat16 *__restrict__ out,
-                    float *__restrict__ part, int n, int d, float eps, int m, unsigned int *status)
+                    float *__restrict__ r_out, const __nv_bfloat16 *__restrict__ dy, const __nv_bfloat16 *__restrict__ dx_add,
+                    __nv_bfloat16 *__restrict__ out, float *__restrict__ part, int n, int d, float eps, int m,
+                    unsigned int *status)
 {
     using namespace ptx;
     extern __shared__ __align__(128) uint8_t nring[];
@@ -356,15 +359,16 @@ rmsnorm_ring_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__
                 for (int j = 0; j < kV; ++j) {
                     const int v = lane + 32 * j;
                     if (v >= nvec) continue;
-                    float fx[8], fd[8], o8[8];
+                    float fx[8], fd[8], o8[8], fa[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
                     unpack8(*reinterpret_cast<const uint4 *>(sx + lr * row_bytes + 16 * v), fx);
                     if (kBwd) unpack8(*reinterpret_cast<const uint4 *>(sd + lr * row_bytes + 16 * v), fd);
+                    if (kBwd && dx_add != nullptr) unpack8(__ldcs(reinterpret_cast<const uint4 *>(dx_add + (size_t)row * d) + v), fa);
                     const float4 g0 = *reinterpret_cast<const float4 *>(gs + 8 * v), g1 = *reinterpret_cast<const float4 *>(gs + 8 * v + 4);
                     const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
                         if (kBwd) {
-                            o8[e] = r * gg[e] * fd[e] - fx[e] * coef;
+                            o8[e] = r * gg[e] * fd[e] - fx[e] * coef + fa[e];
                             dgacc[j][e] = fmaf(fd[e] * fx[e], r, dgacc[j][e]);
                         } else {
                             o8[e] = fx[e] * r * gg[e];
@@ -478,22 +482,24 @@ RingPlan ring_plan(int n, int d, bool bwd)
 
 template <int kV, bool kBwd>
 cudaError_t launch_ring(const RingPlan &p, const __nv_bfloat16 *x, const __nv_bfloat16 *g, const float *r_in, float *r_out,
-                        const __nv_bfloat16 *dy, __nv_bfloat16 *out, float *part, int n, int d, float eps, cudaStream_t st)
+                        const __nv_bfloat16 *dy, const __nv_bfloat16 *dx_add, __nv_bfloat16 *out, float *part, int n, int d,
+                        float eps, cudaStream_t st)
 {
     cudaError_t e = cudaFuncSetAttribute(rmsnorm_ring_kernel<kV, kBwd>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
     if (e != cudaSuccess) return e;
-    rmsnorm_ring_kernel<kV, kBwd><<<p.grid, kRingThreads, p.smem, st>>>(x, g, r_in, r_out, dy, out, part, n, d, eps, p.m,
-                                                                        device_status_ptr());
+    rmsnorm_ring_kernel<kV, kBwd><<<p.grid, kRingThreads, p.smem, st>>>(x, g, r_in, r_out, dy, dx_add, out, part, n, d, eps,
+                                                                        p.m, device_status_ptr());
     return cudaGetLastError();
 }
 template <bool kBwd>
 cudaError_t launch_ring_kv(const RingPlan &p, const __nv_bfloat16 *x, const __nv_bfloat16 *g, const float *r_in, float *r_out,
-                           const __nv_bfloat16 *dy, __nv_bfloat16 *out, float *part, int n, int d, float eps, cudaStream_t st)
+                           const __nv_bfloat16 *dy, const __nv_bfloat16 *dx_add, __nv_bfloat16 *out, float *part, int n, int d,
+                           float eps, cudaStream_t st)
 {
-    if (p.kV == 1) return launch_ring<1, kBwd>(p, x, g, r_in, r_out, dy, out, part, n, d, eps, st);
-    if (p.kV == 2) return launch_ring<2, kBwd>(p, x, g, r_in, r_out, dy, out, part, n, d, eps, st);
-    if (p.kV == 4) return launch_ring<4, kBwd>(p, x, g, r_in, r_out, dy, out, part, n, d, eps, st);
-    return launch_ring<8, kBwd>(p, x, g, r_in, r_out, dy, out, part, n, d, eps, st);
+    if (p.kV == 1) return launch_ring<1, kBwd>(p, x, g, r_in, r_out, dy, dx_add, out, part, n, d, eps, st);
+    if (p.kV == 2) return launch_ring<2, kBwd>(p, x, g, r_in, r_out, dy, dx_add, out, part, n, d, eps, st);
+    if (p.kV == 4) return launch_ring<4, kBwd>(p, x, g, r_in, r_out, dy, dx_add, out, part, n, d, eps, st);
+    return launch_ring<8, kBwd>(p, x, g, r_in, r_out, dy, dx_add, out, part, n, d, eps, st);
 }
 
 }  // namespace
@@ -508,7 +514,7 @@ cudaError_t rmsnorm_fwd(int n, int d, float eps, const void *x, const void *g, v
     const auto *gb = (const __nv_bfloat16 *)g;
     auto *yb = (__nv_bfloat16 *)y;
     LaunchScope scope(MOA_KERNEL_OTHER, st);
-    if (norm_uses_ring(d)) return launch_ring_kv<false>(ring_plan(n, d, false), xb, gb, nullptr, r, nullptr, yb, nullptr, n, d, eps, st);
+    if (norm_uses_ring(d)) return launch_ring_kv<false>(ring_plan(n, d, false), xb, gb, nullptr, r, nullptr, nullptr, yb, nullptr, n, d, eps, st);
     if (p.kV == 1) rmsnorm_fwd_kernel<1, 2><<<p.grid, kNormThreads, 0, st>>>(xb, gb, yb, r, n, d, eps, p.tpr);
     else if (p.kV == 2) rmsnorm_fwd_kernel<2, 1><<<p.grid, kNormThreads, 0, st>>>(xb, gb, yb, r, n, d, eps, p.tpr);
     else rmsnorm_fwd_kernel<4, 1><<<p.grid, kNormThreads, 0, st>>>(xb, gb, yb, r, n, d, eps, p.tpr);
@@ -516,8 +522,9 @@ cudaError_t rmsnorm_fwd(int n, int d, float eps, const void *x, const void *g, v
 }
 
 cudaError_t rmsnorm_bwd(int n, int d, float eps, const void *x, const void *g, const float *r, const void *dy,
-                        void *dx, void *dg, void *ws, cudaStream_t st)
+                        const void *dx_add, void *dx, void *dg, void *ws, cudaStream_t st)
 {
+    const auto *ab = (const __nv_bfloat16 *)dx_add;
     const NormPlan p = norm_plan(n, d, true);
     const auto *xb = (const __nv_bfloat16 *)x;
     const auto *gb = (const __nv_bfloat16 *)g;
@@ -529,13 +536,13 @@ cudaError_t rmsnorm_bwd(int n, int d, float eps, const void *x, const void *g, c
         const RingPlan rp = ring_plan(n, d, true);
         parts = rp.grid;
         LaunchScope scope(MOA_KERNEL_OTHER, st);
-        const cudaError_t e = launch_ring_kv<true>(rp, xb, gb, r, nullptr, db, ob, part, n, d, eps, st);
+        const cudaError_t e = launch_ring_kv<true>(rp, xb, gb, r, nullptr, db, ab, ob, part, n, d, eps, st);
         if (e != cudaSuccess) return e;
     } else {
         LaunchScope scope(MOA_KERNEL_OTHER, st);
-        if (p.kV == 1) rmsnorm_bwd_kernel<1, 2><<<p.grid, kNormThreads, 0, st>>>(xb, gb, r, db, ob, part, n, d, eps, p.tpr);
-        else if (p.kV == 2) rmsnorm_bwd_kernel<2, 1><<<p.grid, kNormThreads, 0, st>>>(xb, gb, r, db, ob, part, n, d, eps, p.tpr);
-        else rmsnorm_bwd_kernel<4, 2><<<p.grid, kNormThreads, 0, st>>>(xb, gb, r, db, ob, part, n, d, eps, p.tpr);
+        if (p.kV == 1) rmsnorm_bwd_kernel<1, 2><<<p.grid, kNormThreads, 0, st>>>(xb, gb, r, db, ab, ob, part, n, d, eps, p.tpr);
+        else if (p.kV == 2) rmsnorm_bwd_kernel<2, 1><<<p.grid, kNormThreads, 0, st>>>(xb, gb, r, db, ab, ob, part, n, d, eps, p.tpr);
+        else rmsnorm_bwd_kernel<4, 2><<<p.grid, kNormThreads, 0, st>>>(xb, gb, r, db, ab, ob, part, n, d, eps, p.tpr);
         const cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }

@@ -91,11 +91,16 @@ moa_status check_device_arch();
 // ---- block pieces (block_norm.cu, tc_gemm.cu), bf16 ------------------------------------
 size_t rmsnorm_workspace_bytes(int n, int d);          // per-CTA partial sums of dg
 cudaError_t rmsnorm_fwd(int n, int d, float eps, const void *x, const void *g, void *y, float *r, cudaStream_t st);
+// dx_add (may be null): dx = (RMSNorm backward) + dx_add
 cudaError_t rmsnorm_bwd(int n, int d, float eps, const void *x, const void *g, const float *r, const void *dy,
-                        void *dx, void *dg, void *ws, cudaStream_t st);
+                        const void *dx_add, void *dx, void *dg, void *ws, cudaStream_t st);
 // gated MLP (tc_gemm.cu): x, y, dy, dx [n,d]; W1, W3 [d_ff,d]; W2 [d,d_ff]; a, u, h, da, du [n,d_ff]
+// res (may be null): y = h W2^T + res
 cudaError_t gated_mlp_fwd(int n, int d, int dff, const void *x, const void *W1, const void *W3, const void *W2,
-                          void *a, void *u, void *h, void *y, cudaStream_t st);
+                          const void *res, void *a, void *u, void *h, void *y, cudaStream_t st);
+// C[M,N] = A B^T (+ R): A given as [M,K] (a_mn = 0) or [K,M] (a_mn = 1), B as [N,K] (b_mn = 0) or [K,N] (b_mn = 1); bf16
+cudaError_t gemm_bf16(int a_mn, int b_mn, int M, int N, int K, const void *A, const void *B, const void *R, void *C,
+                      cudaStream_t st);
 cudaError_t gated_mlp_bwd(int n, int d, int dff, const void *x, const void *W1, const void *W3, const void *W2,
                           const void *a, const void *u, const void *h, const void *dy, void *da, void *du,
                           void *dx, void *dW1, void *dW3, void *dW2, cudaStream_t st);

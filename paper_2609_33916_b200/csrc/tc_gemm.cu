@@ -17,7 +17,7 @@
 // Tails in M, N and K are handled by the TMA zero fill on loads and by guards on stores.
 //
 // Epilogues:
-//   EPI_STORE       C -> bf16
+//   EPI_STORE       C -> bf16; with a residual R (map C2) C + R -> bf16 (residual connections, sums of products)
 //   EPI_SWIGLU_FWD  the tile's B rows are 128 rows of W1 and the same 128 rows of W3 (two maps), so
 //                   its accumulator holds a | u for 128 hidden units; writes a, u and
 //                   h = silu(a) * u (all from the fp32 values).
@@ -43,8 +43,8 @@ constexpr int kGemmSmem = kStages * kStageBytes + 2 * kOutBox + 1024 /* alignmen
 
 enum { EPI_STORE = 0, EPI_SWIGLU_FWD = 1, EPI_SWIGLU_BWD = 2 };
 enum { G_FULL = 0, G_EMPTY = kStages, G_ACCFULL = 2 * kStages, G_ACCEMPTY = 2 * kStages + 2, G_EPI = 2 * kStages + 4,
-       G_IN = 2 * kStages + 5, G_COUNT = 2 * kStages + 6 };
-enum { GERR_EMPTY = 0x301, GERR_FULL = 0x302, GERR_ACCFULL = 0x303, GERR_ACCEMPTY = 0x304, GERR_EPI = 0x305, GERR_IN = 0x306 };
+       G_IN = 2 * kStages + 5, G_RES = 2 * kStages + 6 /* two */, G_COUNT = 2 * kStages + 8 };
+enum { GERR_EMPTY = 0x301, GERR_FULL = 0x302, GERR_ACCFULL = 0x303, GERR_ACCEMPTY = 0x304, GERR_EPI = 0x305, GERR_IN = 0x306, GERR_RES = 0x307 };
 
 // Outputs leave through TMA stores (tensor maps C0..C3: STORE: C (and the second product's C); FWD gate: a, u, h;
 // BWD gate: da, du, and the stored a, u as C2, C3, which its epilogue brings in by TMA loads).
@@ -87,7 +87,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapB0,
                const __grid_constant__ CUtensorMap mapA1, const __grid_constant__ CUtensorMap mapB1,
                const __grid_constant__ CUtensorMap mapC0, const __grid_constant__ CUtensorMap mapC1,
-               const __grid_constant__ CUtensorMap mapC2, const __grid_constant__ CUtensorMap mapC3, int M, int N, int K, int nparts, int nbatch, int a_blocked, int b_blocked, unsigned int *status)
+               const __grid_constant__ CUtensorMap mapC2, const __grid_constant__ CUtensorMap mapC3, int M, int N, int K, int nparts, int nbatch, int a_blocked, int b_blocked, int has_res, unsigned int *status)
 {
     constexpr bool kDualN = kEpi == EPI_SWIGLU_FWD;         // B tile = 128 rows of map B0 + 128 rows of map B1
     constexpr int kTileN = kDualN ? 128 : GN;                // output columns a tile covers
@@ -118,6 +118,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
         mbar_init(bars + G_ACCEMPTY + 1, 32 * kEpiWarps);
         mbar_init(bars + G_EPI, 32 * kEpiWarps);
         mbar_init(bars + G_IN, 1);
+        mbar_init(bars + G_RES + 0, 1);
+        mbar_init(bars + G_RES + 1, 1);
         *abortp = 0;
         fence_mbar_init();
     }
@@ -241,6 +243,35 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
             ++chunk_q;
             return true;
         };
+        // the same with a residual: the chunk of R comes into the staging buffer by TMA, every thread adds its 32
+        // values in place, and the buffer leaves by a TMA store
+        auto stage_store_res = [&](const CUtensorMap *map, const uint32_t (&racc)[32], int col0, int row0) -> bool {
+            const uint32_t b = chunk_q & 1;
+            uint8_t *buf = sout + b * kOutBox;
+            if (leader) {
+                bulk_wait_read<1>();                                   // the store issued two chunks ago has left this buffer
+                mbar_arrive_expect_tx(bars + G_RES + b, kOutBox);
+                tma_load_3d(buf, &mapC2, bars + G_RES + b, col0, row0, 0);
+            }
+            if (!mbar_wait(bars + G_RES + b, (chunk_q >> 1) & 1, abortp, status, GERR_RES)) return false;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                uint4 *pr = reinterpret_cast<uint4 *>(buf + lane_row * 128 + (((half * 4 + j) ^ (lane_row & 7)) << 4));
+                float r8[8];
+                unpack8(*pr, r8);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) r8[i] += __uint_as_float(racc[8 * j + i]);
+                *pr = make_uint4(pack_bf16(r8[0], r8[1]), pack_bf16(r8[2], r8[3]), pack_bf16(r8[4], r8[5]), pack_bf16(r8[6], r8[7]));
+            }
+            fence_proxy_async_smem();
+            if (!epi_sync()) return false;
+            if (leader) {
+                tma_store_3d(map, buf, col0, row0, 0);
+                bulk_commit();
+            }
+            ++chunk_q;
+            return true;
+        };
         int ti = 0;
         for (int t = blockIdx.x; ok && t < tiles; t += gridDim.x, ++ti) {
             int tm, tn;
@@ -248,6 +279,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
             tile_coords(t - second * tiles_one, tiles_m, tiles_n, tm, tn);
             const int buf = ti & 1;
             const int m0 = tm * GM, n0 = tn * kTileN;
+            if (kEpi == EPI_STORE && has_res && leader) {     // the tile's residual: into L2 while its main loop runs
+#pragma unroll
+                for (int c0 = 0; c0 < GN; c0 += 64) tma_prefetch_3d(&mapC2, n0 + c0, m0, 0);
+            }
             if (kEpi == EPI_SWIGLU_BWD && leader) {       // the tile's stored a, u: into L2 while its main loop runs
 #pragma unroll
                 for (int c0 = 0; c0 < GN; c0 += 64) {
@@ -292,10 +327,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                         tc_fence_before();
                         mbar_arrive(bars + G_ACCEMPTY + buf);
                     }
-                    uint32_t pc[16];
+                    if (has_res) {
+                        ok = stage_store_res(&mapC0, r, n0 + c0, m0);
+                    } else {
+                        uint32_t pc[16];
 #pragma unroll
-                    for (int e = 0; e < 32; e += 2) pc[e / 2] = pack_bf16(__uint_as_float(r[e]), __uint_as_float(r[e + 1]));
-                    ok = stage_store(second ? &mapC1 : &mapC0, pc, n0 + c0, m0);
+                        for (int e = 0; e < 32; e += 2) pc[e / 2] = pack_bf16(__uint_as_float(r[e]), __uint_as_float(r[e + 1]));
+                        ok = stage_store(second ? &mapC1 : &mapC0, pc, n0 + c0, m0);
+                    }
                 }
             } else {
                 // Backward gate: per 64-column chunk the stored a and u come into the two staging buffers by TMA, every
@@ -370,7 +409,7 @@ template <bool kAMn, bool kBMn, int kEpi>
 // C0..C2: output arrays (row length ldc); unused ones may repeat C0.
 cudaError_t launch_gemm(const Operand &A0, const Operand &B0, const Operand *A1, const Operand *B1, void *C0, void *C1,
                         const void *C2, const void *C3, int c_rows, int ldc, int M, int N, int K, cudaStream_t st,
-                        int nbatch = 1)
+                        int nbatch = 1, bool has_res = false)
 {
     constexpr bool kDualN = kEpi == EPI_SWIGLU_FWD;
     CUtensorMap ma0, mb0, ma1, mb1;
@@ -397,20 +436,32 @@ cudaError_t launch_gemm(const Operand &A0, const Operand &B0, const Operand *A1,
     LaunchScope scope(MOA_KERNEL_OTHER, st);
     kernel<<<tiles < 148 ? tiles : 148, kGemmThreads, kGemmSmem, st>>>(ma0, mb0, ma1, mb1, mc[0], mc[1], mc[2], mc[3], M, N, K, nparts,
                                                                       nbatch, a_blocked ? 1 : 0, b_blocked ? 1 : 0,
-                                                                      device_status_ptr());
+                                                                      has_res ? 1 : 0, device_status_ptr());
     return cudaGetLastError();
 }
 
 }  // namespace
 
+// C[M,N] = A B^T (+ R): A given as [M,K] (a_mn = 0) or [K,M] (a_mn = 1), B as [N,K] (b_mn = 0) or [K,N] (b_mn = 1)
+cudaError_t gemm_bf16(int a_mn, int b_mn, int M, int N, int K, const void *A, const void *B, const void *R, void *C,
+                      cudaStream_t st)
+{
+    const Operand a{A, a_mn ? K : M, a_mn ? M : K}, b{B, b_mn ? K : N, b_mn ? N : K};
+    const bool res = R != nullptr;
+    if (!a_mn && !b_mn) return launch_gemm<false, false, EPI_STORE>(a, b, nullptr, nullptr, C, nullptr, R, nullptr, M, N, M, N, K, st, 1, res);
+    if (!a_mn && b_mn) return launch_gemm<false, true, EPI_STORE>(a, b, nullptr, nullptr, C, nullptr, R, nullptr, M, N, M, N, K, st, 1, res);
+    if (a_mn && b_mn) return launch_gemm<true, true, EPI_STORE>(a, b, nullptr, nullptr, C, nullptr, R, nullptr, M, N, M, N, K, st, 1, res);
+    return launch_gemm<true, false, EPI_STORE>(a, b, nullptr, nullptr, C, nullptr, R, nullptr, M, N, M, N, K, st, 1, res);
+}
+
 cudaError_t gated_mlp_fwd(int n, int d, int dff, const void *x, const void *W1, const void *W3, const void *W2,
-                          void *a, void *u, void *h, void *y, cudaStream_t st)
+                          const void *res, void *a, void *u, void *h, void *y, cudaStream_t st)
 {
     // a | u = x [W1; W3]^T with the gate in the epilogue, then y = h W2^T
     const Operand X{x, n, d}, w1{W1, dff, d}, w3{W3, dff, d}, Hh{h, n, dff}, w2{W2, d, dff};
     cudaError_t e = launch_gemm<false, false, EPI_SWIGLU_FWD>(X, w1, nullptr, &w3, a, u, h, nullptr, n, dff, n, dff, d, st);
     if (e != cudaSuccess) return e;
-    return launch_gemm<false, false, EPI_STORE>(Hh, w2, nullptr, nullptr, y, nullptr, nullptr, nullptr, n, d, n, d, dff, st);
+    return launch_gemm<false, false, EPI_STORE>(Hh, w2, nullptr, nullptr, y, nullptr, res, nullptr, n, d, n, d, dff, st, 1, res != nullptr);
 }
 
 cudaError_t gated_mlp_bwd(int n, int d, int dff, const void *x, const void *W1, const void *W3, const void *W2,

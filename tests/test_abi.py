@@ -180,6 +180,15 @@ def test_block_piece_argument_checks(lib):
     m = mb.make_mlp_desc(256, 512, 2048)
     assert mb.moa_gated_mlp_workspace_bytes(m) == 2 * 256 * 2048 * 2
     assert mb.moa_gated_mlp_fwd(m, a, a, a, a, a, a, a, 0, check=False) == mb.MOA_ERR_INVALID_ARG
+    assert mb.moa_gated_mlp_fwd(m, a, a, a, a, a, a, a, a, res=a + 8, check=False) == mb.MOA_ERR_INVALID_ARG
+    assert ctypes.sizeof(mb.moa_gemm_desc) == 24
+    gd = mb.make_gemm_desc(256, 512, 1024)
+    assert mb.moa_gemm(gd, a, a, 0, check=False) == mb.MOA_ERR_INVALID_ARG
+    assert mb.moa_gemm(gd, a, a, a, R=a + 2, check=False) == mb.MOA_ERR_INVALID_ARG
+    for M, N, K, al, bl, dt, want in ((0, 8, 8, 0, 0, mb.MOA_BF16, mb.MOA_ERR_INVALID_ARG), (8, 8, 8, 2, 0, mb.MOA_BF16, mb.MOA_ERR_INVALID_ARG),
+                                      (8, 8, 12, 0, 0, mb.MOA_BF16, mb.MOA_ERR_UNSUPPORTED), (8, 12, 8, 0, 0, mb.MOA_BF16, mb.MOA_ERR_UNSUPPORTED),
+                                      (12, 8, 8, 1, 1, mb.MOA_BF16, mb.MOA_ERR_UNSUPPORTED), (8, 8, 8, 0, 0, mb.MOA_F32, mb.MOA_ERR_UNSUPPORTED)):
+        assert mb.moa_gemm(mb.make_gemm_desc(M, N, K, al, bl, dt), a, a, a, check=False) == want, (M, N, K, al, bl, dt)
     assert mb.moa_gated_mlp_bwd(m, *([a] * 12), None, check=False) == mb.MOA_ERR_WORKSPACE
     for n, d, dff, dt, want in ((0, 512, 2048, mb.MOA_BF16, mb.MOA_ERR_INVALID_ARG),
                                 (16, 100, 2048, mb.MOA_BF16, mb.MOA_ERR_UNSUPPORTED),

@@ -228,3 +228,143 @@ def test_rmsnorm_long_run_through_the_ring(rt):
                 assert torch.equal(y, y0) and torch.equal(dx, dx0) and torch.equal(dg, dg0), it
     assert mb.moa_last_device_status() == mb.MOA_OK
     assert torch.equal(y, y0) and torch.equal(dx, dx0) and torch.equal(dg, dg0)
+
+
+# ------------------------------------------------------------------------------- GEMM
+def _bits(rng, shape, scale=1.0):
+    return mi.f32_to_bf16_bits((scale * rng.standard_normal(shape)).astype(np.float32))
+
+
+@pytest.mark.parametrize("a_layout,b_layout", [(0, 0), (0, 1), (1, 1), (1, 0)])
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (8, 8, 8), (130, 264, 72), (1000, 512, 2048), (384, 1032, 520)])
+@pytest.mark.parametrize("with_r", [False, True])
+def test_gemm_layouts_match_oracle(rt, a_layout, b_layout, M, N, K, with_r):
+    torch, mb = rt
+    if a_layout and M % 8:
+        pytest.skip("rows of A = [K,M] must be 16-byte multiples")
+    rng = np.random.default_rng(M + N + K + 7 * a_layout + 3 * b_layout)
+    A = _bits(rng, (K, M) if a_layout else (M, K))
+    Bm = _bits(rng, (K, N) if b_layout else (N, K), 1.0 / np.sqrt(K))
+    R = _bits(rng, (M, N)) if with_r else None
+    ref = oracle.gemm(mi.to_f64(A, "bf16"), mi.to_f64(Bm, "bf16"), None if R is None else mi.to_f64(R, "bf16"), a_layout, b_layout)
+    C = _nan_like(torch, (M, N))
+    mb.moa_gemm(mb.make_gemm_desc(M, N, K, a_layout, b_layout), _dev(torch, A), _dev(torch, Bm), C,
+                R=None if R is None else _dev(torch, R))
+    assert mb.moa_last_device_status() == mb.MOA_OK
+    got = _host(C)
+    assert np.all(np.isfinite(got))
+    assert mi.rel_err(got, ref) <= TOL, mi.rel_err(got, ref)
+
+
+def test_residual_arguments(rt):
+    """dx_add of the RMSNorm backward and res of the gated-MLP forward: the same as adding afterwards (in fp64)."""
+    torch, mb = rt
+    n, d, dff = 300, 512, 1024
+    rng = np.random.default_rng(5)
+    ninp = mi.make_norm_inputs(n, d, seed=8)
+    add = _bits(rng, (n, d))
+    f = {k: mi.to_f64(v, "bf16") for k, v in ninp.items()}
+    ref = oracle.rmsnorm_fwd_bwd(f["x"], f["g"], f["dy"], 1e-5)
+    x, g, dy = (_dev(torch, ninp[k]) for k in ("x", "g", "dy"))
+    desc = mb.make_rmsnorm_desc(n, d, 1e-5)
+    dx, dg = _nan_like(torch, (n, d)), _nan_like(torch, (d,))
+    ws = torch.empty(mb.moa_rmsnorm_workspace_bytes(desc), dtype=torch.uint8, device="cuda")
+    mb.moa_rmsnorm_bwd(desc, x, g, None, dy, dx, dg, ws, dx_add=_dev(torch, add))
+    assert mi.rel_err(_host(dx), ref["dx"] + mi.to_f64(add, "bf16")) <= TOL
+    assert mi.rel_err(_host(dg), ref["dg"]) <= TOL
+    minp = mi.make_mlp_inputs(n, d, dff, seed=9)
+    f = {k: mi.to_f64(v, "bf16") for k, v in minp.items()}
+    mref = oracle.gated_mlp_fwd_bwd(f["x"], f["W1"], f["W3"], f["W2"], f["dy"])
+    x, W1, W3, W2 = (_dev(torch, minp[k]) for k in ("x", "W1", "W3", "W2"))
+    a, u, h = (_nan_like(torch, (n, dff)) for _ in range(3))
+    y = _nan_like(torch, (n, d))
+    mb.moa_gated_mlp_fwd(mb.make_mlp_desc(n, d, dff), x, W1, W3, W2, a, u, h, y, res=_dev(torch, add))
+    assert mb.moa_last_device_status() == mb.MOA_OK
+    assert mi.rel_err(_host(y), mref["y"] + mi.to_f64(add, "bf16")) <= TOL
+
+
+# ------------------------------------------------------- the block, composed from the pieces
+def run_block(torch, mb, inp, B, n, H, causal, eps):
+    """One pre-norm transformer block forward+backward as a sequence of library calls (every step a kernel of the
+    library; this function only passes pointers): RMSNorm, three projections, attention on token-major tensors,
+    output projection + residual, RMSNorm, gated MLP + residual; then the backward of each, in reverse."""
+    bf = torch.bfloat16
+    dev = {k: _dev(torch, v) for k, v in inp.items()}
+    T, dm = inp["x"].shape
+    d, dff = dm // H, inp["W1"].shape[0]
+    E = lambda *s: torch.full(s, float("nan"), dtype=bf, device="cuda")
+    nd = mb.make_rmsnorm_desc(T, dm, eps)
+    nws = torch.empty(mb.moa_rmsnorm_workspace_bytes(nd), dtype=torch.uint8, device="cuda")
+    ad = mb.make_desc(B, H, n, d, causal, 1.0 / np.sqrt(d), layout=mb.MOA_LAYOUT_BNHD)
+    aws = torch.empty(max(16, mb.moa_attn_workspace_bytes(ad, mb.MOA_OP_BWD)), dtype=torch.uint8, device="cuda")
+    md = mb.make_mlp_desc(T, dm, dff)
+    mws = torch.empty(mb.moa_gated_mlp_workspace_bytes(md), dtype=torch.uint8, device="cuda")
+    proj = mb.make_gemm_desc(T, dm, dm)                  # y = x W^T
+    back = mb.make_gemm_desc(T, dm, dm, 0, 1)            # dx = dy W
+    wgrad = mb.make_gemm_desc(dm, dm, T, 1, 1)           # dW = dy^T x
+    # ---- forward
+    h1, r1 = E(T, dm), torch.empty((T,), dtype=torch.float32, device="cuda")
+    mb.moa_rmsnorm_fwd(nd, dev["x"], dev["g1"], h1, r1)
+    q, k, v = E(T, dm), E(T, dm), E(T, dm)
+    for W, out in (("Wq", q), ("Wk", k), ("Wv", v)):
+        mb.moa_gemm(proj, h1, dev[W], out)
+    o, L = E(T, dm), torch.empty((B, H, n), dtype=torch.float32, device="cuda")
+    mb.moa_attn_fwd(ad, q, k, v, o, L, aws)
+    x2 = E(T, dm)
+    mb.moa_gemm(proj, o, dev["Wo"], x2, R=dev["x"])
+    h2, r2 = E(T, dm), torch.empty((T,), dtype=torch.float32, device="cuda")
+    mb.moa_rmsnorm_fwd(nd, x2, dev["g2"], h2, r2)
+    a, u, h, y = E(T, dff), E(T, dff), E(T, dff), E(T, dm)
+    mb.moa_gated_mlp_fwd(md, h2, dev["W1"], dev["W3"], dev["W2"], a, u, h, y, res=x2)
+    # ---- backward
+    g = {}
+    dh2 = E(T, dm)
+    g["dW1"], g["dW3"], g["dW2"] = E(dff, dm), E(dff, dm), E(dm, dff)
+    mb.moa_gated_mlp_bwd(md, h2, dev["W1"], dev["W3"], dev["W2"], a, u, h, dev["dy"], dh2, g["dW1"], g["dW3"], g["dW2"], mws)
+    dx2, g["dg2"] = E(T, dm), E(dm)
+    mb.moa_rmsnorm_bwd(nd, x2, dev["g2"], r2, dh2, dx2, g["dg2"], nws, dx_add=dev["dy"])
+    g["dWo"], do = E(dm, dm), E(T, dm)
+    mb.moa_gemm(wgrad, dx2, o, g["dWo"])
+    mb.moa_gemm(back, dx2, dev["Wo"], do)
+    dq, dk, dv = E(T, dm), E(T, dm), E(T, dm)
+    mb.moa_attn_bwd(ad, q, k, v, o, L, do, dq, dk, dv, aws)
+    dh1 = E(T, dm)
+    mb.moa_gemm(back, dq, dev["Wq"], dh1)
+    mb.moa_gemm(back, dk, dev["Wk"], dh1, R=dh1)
+    mb.moa_gemm(back, dv, dev["Wv"], dh1, R=dh1)
+    for W, dt in (("dWq", dq), ("dWk", dk), ("dWv", dv)):
+        g[W] = E(dm, dm)
+        mb.moa_gemm(wgrad, dt, h1, g[W])
+    g["dx"], g["dg1"] = E(T, dm), E(dm)
+    mb.moa_rmsnorm_bwd(nd, dev["x"], dev["g1"], r1, dh1, g["dx"], g["dg1"], nws, dx_add=dx2)
+    assert mb.moa_last_device_status() == mb.MOA_OK
+    g["y"] = y
+    return {k_: _host(v_) for k_, v_ in g.items()}
+
+
+def make_block_inputs(B, n, H, d, dff, seed):
+    rng = np.random.default_rng(seed)
+    T, dm = B * n, H * d
+    f = lambda shape, s=1.0: mi.f32_to_bf16_bits((s * rng.standard_normal(shape)).astype(np.float32))
+    return dict(x=f((T, dm)), dy=f((T, dm)), g1=mi.f32_to_bf16_bits((1 + 0.25 * rng.standard_normal(dm)).astype(np.float32)),
+                g2=mi.f32_to_bf16_bits((1 + 0.25 * rng.standard_normal(dm)).astype(np.float32)),
+                Wq=f((dm, dm), dm ** -0.5), Wk=f((dm, dm), dm ** -0.5), Wv=f((dm, dm), dm ** -0.5), Wo=f((dm, dm), dm ** -0.5),
+                W1=f((dff, dm), dm ** -0.5), W3=f((dff, dm), dm ** -0.5), W2=f((dm, dff), dff ** -0.5))
+
+
+@pytest.mark.parametrize("B,n,H,d,dff,causal", [(1, 128, 2, 64, 256, False), (2, 256, 4, 64, 512, True), (1, 300, 2, 128, 520, True),
+                                                (2, 512, 8, 128, 2048, False)])
+def test_transformer_block_composed_from_the_pieces(rt, B, n, H, d, dff, causal):
+    """The complete block (two norms, QKV projection, attention, output projection, gated MLP, two residual
+    connections) forward+backward as 24 library calls against the fp64 block oracle.  Errors of the bf16 stages
+    compound along the block, so the bar here is 2e-2 of each tensor's max (each piece alone is held to 1e-2)."""
+    torch, mb = rt
+    inp = make_block_inputs(B, n, H, d, dff, seed=70 + n)
+    f = {k: mi.to_f64(v, "bf16") for k, v in inp.items()}
+    w = {k: f[k] for k in ("g1", "g2", "Wq", "Wk", "Wv", "Wo", "W1", "W3", "W2")}
+    ref = oracle.transformer_block_fwd_bwd(f["x"], w, f["dy"], B, n, H, causal, 1e-5)
+    got = run_block(torch, mb, inp, B, n, H, causal, 1e-5)
+    for k in ref:
+        assert np.all(np.isfinite(got[k])), k
+        e = mi.rel_err(got[k], ref[k])
+        assert e <= 2e-2, (k, e)
