@@ -311,6 +311,12 @@ BLOCK_WORKLOADS = {
     "mlp_n8192_d4096_ff16384": ("mlp", 8192, 4096, 16384),
     "mlp_n4096_d1024_ff4096": ("mlp", 4096, 1024, 4096),              # small case for profiler captures (0.4 GB moved per step)
     "mlp_paper_n512_d64_ff256": ("mlp", 512, 64, 256),              # the paper's own traffic-check size (B=2, N=256, D=64, DFF=256)
+    # the whole pre-norm block (two norms, QKV projection, attention, output projection, gated MLP, residuals),
+    # composed from library calls: (piece, B, n, H, d, d_ff, causal)
+    "block_c4_b1_n16384_h16_d128_ff8192": ("block", 1, 16384, 16, 128, 8192, False),   # config 4's attention inside a block
+    "block_c3_b2_n4096_h16_d128_ff8192": ("block", 2, 4096, 16, 128, 8192, True),      # config 3's
+    "block_small_b2_n1024_h8_d128_ff4096": ("block", 2, 1024, 8, 128, 4096, True),     # small case for profiler captures
+    "block_paper_b2_n256_h1_d64_ff256": ("block", 2, 256, 1, 64, 256, False),          # the paper's traffic-check size
 }
 
 
@@ -327,6 +333,8 @@ def run_block(args):
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    if BLOCK_WORKLOADS[args.block][0] == "block":
+        return run_whole_block(args)
     piece, n, d, dff = BLOCK_WORKLOADS[args.block]
     mbuild.build()
     mb.lib()
@@ -451,6 +459,117 @@ def run_block(args):
         line["cpu_baseline"] = {"value": sample / dt / (1e9 if piece == "rmsnorm" else 1e12), "unit": unit,
                                 "cores": os.cpu_count(), "kind": "oracle",
                                 "sample": f"{rows} of {n} tokens (all columns / full weights), numpy fp64", "seconds": dt * reps}
+    print(json.dumps(line))
+    return 0
+
+
+def run_whole_block(args):
+    """The complete pre-norm transformer block, forward+backward, as the fixed sequence of library calls of
+    paper_2609_33916_b200/block.py (20 calls, 28 launches).  Metric: model TFLOP/s of the block."""
+    import numpy as np
+    import torch
+    from paper_2609_33916_b200 import binding as mb
+    from paper_2609_33916_b200 import build as mbuild
+    from paper_2609_33916_b200.block import TransformerBlock, WEIGHTS
+    import oracle
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    _, B, n, H, d, dff, causal = BLOCK_WORKLOADS[args.block]
+    mbuild.build()
+    mb.lib()
+    peaks, peaks_kind = load_peaks()
+    T, dm = B * n, H * d
+    bf = torch.bfloat16
+    gen = torch.Generator(device="cuda").manual_seed(19)
+    rnd = lambda *shape, s=1.0: (torch.randn(shape, generator=gen, device="cuda") * s).to(bf)
+    x, dy = rnd(T, dm), rnd(T, dm)
+    w = dict(g1=(1.0 + 0.25 * torch.randn((dm,), generator=gen, device="cuda")).to(bf),
+             g2=(1.0 + 0.25 * torch.randn((dm,), generator=gen, device="cuda")).to(bf),
+             Wq=rnd(dm, dm, s=dm ** -0.5), Wk=rnd(dm, dm, s=dm ** -0.5), Wv=rnd(dm, dm, s=dm ** -0.5), Wo=rnd(dm, dm, s=dm ** -0.5),
+             W1=rnd(dff, dm, s=dm ** -0.5), W3=rnd(dff, dm, s=dm ** -0.5), W2=rnd(dm, dff, s=dff ** -0.5))
+    blk = TransformerBlock(torch, B, n, H, d, dff, causal)
+    stream = torch.cuda.current_stream()
+    flops = blk.model_flops()
+
+    def step():
+        blk.forward(x, w, stream)
+        blk.backward(x, w, dy, stream)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(physical_gpu_index(0))
+    sampler.start()
+    l0 = mb.moa_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    sampler.stop()
+    launches = mb.moa_launch_count() - l0
+    ms = e0.elapsed_time(e1) / args.steps
+    value = flops / (ms * 1e-3) / 1e12
+    # per-kind kernel time of one more step (outside the timed region)
+    mb.moa_profile_read()
+    mb.moa_profile_enable(True)
+    step()
+    torch.cuda.synchronize()
+    mb.moa_profile_enable(False)
+    prof = {k: [round(v[0], 4), v[1]] for k, v in mb.moa_profile_read().items() if v[1]}
+    # end to end: x and dy from pinned host memory, dx back, every step; weights resident
+    hx, hdy = x.cpu().pin_memory(), dy.cpu().pin_memory()
+    hdx = torch.empty((T, dm), dtype=bf).pin_memory()
+    esteps = max(4, min(args.steps, 10))
+    t0e, t1e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0e.record(stream)
+    for _ in range(esteps):
+        x.copy_(hx, non_blocking=True)
+        dy.copy_(hdy, non_blocking=True)
+        step()
+        hdx.copy_(blk.dx, non_blocking=True)
+    t1e.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = t0e.elapsed_time(t1e) / esteps
+    st = mb.moa_last_device_status(stream)
+    if st != mb.MOA_OK:
+        raise SystemExit(f"device status: {mb.status_string(st)}")
+    att = 14.0 * B * H * float(n) ** 2 * d * (0.5 if causal else 1.0)
+    line = {
+        "metric": "transformer block forward+backward: model TFLOP/s", "value": value, "unit": "TFLOP/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.block, "B": B, "n": n, "H": H, "d": d, "d_model": dm, "d_ff": dff, "causal": causal,
+                   "l2": "the activations of one step exceed the 126 MB L2; no explicit flush" if T * dff * 2 > 126e6
+                   else "small case: mostly resident in L2 between steps"},
+        "model_flops": {"total": flops, "attention": att, "projections": 24.0 * T * dm * dm, "gated_mlp": 18.0 * T * dm * dff},
+        "tokens_per_s": T / (ms * 1e-3),
+        "clocks": sampler.summary(),
+        "e2e": {"value": flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": 2 * T * dm * 2,
+                "d2h_bytes_per_step": T * dm * 2, "ms_per_step": e2e_ms,
+                "how": "x and dy from pinned host memory and dx back every step; weights resident"},
+        "gpu_launches": int(launches),
+        "per_kind_ms": prof,
+        "roofline": {"bound": "tensor", "kernel": "whole step (attention, GEMMs)", "achieved": value, "peak": peaks["bf16_tflops"],
+                     "unit": "TFLOP/s", "frac": value / peaks["bf16_tflops"], "traffic": None,
+                     "peak_source": f"{peaks_kind} bf16_tflops (cuBLAS burst)",
+                     "frac_of_sustained": value / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])},
+    }
+    if not args.no_cpu_baseline:
+        # the oracle block on a shorter sequence of the same widths (attention is O(n^2): the rate differs by piece)
+        ns = min(n, 256)
+        f64 = lambda t: t.float().cpu().numpy().astype(np.float64)
+        ws = {k: f64(v) for k, v in w.items()}
+        xs, ds = f64(x[:ns]), f64(dy[:ns])
+        t0 = time.perf_counter()
+        oracle.transformer_block_fwd_bwd(xs, ws, ds, 1, ns, H, causal, 1e-5)
+        dt = time.perf_counter() - t0
+        sf = 24.0 * ns * dm * dm + 14.0 * H * float(ns) ** 2 * d * (0.5 if causal else 1.0) + 18.0 * ns * dm * dff
+        line["cpu_baseline"] = {"value": sf / dt / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count(), "kind": "oracle",
+                                "sample": f"one sequence of {ns} tokens, same widths and weights, numpy fp64 + the C attention oracle",
+                                "seconds": dt}
     print(json.dumps(line))
     return 0
 

@@ -70,11 +70,12 @@ __device__ __forceinline__ float sigmoidf_fast(float a)
     return r;
 }
 
-// Tile order: groups of 8 tile rows, column-major inside a group, so that the CTAs running at the
-// same time share a few A row blocks and a few B column blocks.
-__device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int &tm, int &tn)
+// Tile order: groups of `kGroup` tile rows, column-major inside a group, so that the CTAs running at the same time
+// share a few A row blocks and a few B column blocks.  B is swept once per group: the launcher picks taller groups
+// when B is too large to survive in L2 between sweeps (with groups of 8 a [8192 x 2048] x [16384 x 2048]^T product
+// read its 67 MB of B eight times from DRAM: the outputs streaming through L2 evict it in between).
+__device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int kGroup, int &tm, int &tn)
 {
-    constexpr int kGroup = 8;
     const int per_group = kGroup * tiles_n;
     const int g = t / per_group, r = t - g * per_group;
     const int rows = min(kGroup, tiles_m - g * kGroup);
@@ -87,7 +88,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapB0,
                const __grid_constant__ CUtensorMap mapA1, const __grid_constant__ CUtensorMap mapB1,
                const __grid_constant__ CUtensorMap mapC0, const __grid_constant__ CUtensorMap mapC1,
-               const __grid_constant__ CUtensorMap mapC2, const __grid_constant__ CUtensorMap mapC3, int M, int N, int K, int nparts, int nbatch, int a_blocked, int b_blocked, int has_res, unsigned int *status)
+               const __grid_constant__ CUtensorMap mapC2, const __grid_constant__ CUtensorMap mapC3, int M, int N, int K, int nparts, int nbatch, int a_blocked, int b_blocked, int has_res, int group_rows, unsigned int *status)
 {
     constexpr bool kDualN = kEpi == EPI_SWIGLU_FWD;         // B tile = 128 rows of map B0 + 128 rows of map B1
     constexpr int kTileN = kDualN ? 128 : GN;                // output columns a tile covers
@@ -141,7 +142,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
         for (int t = blockIdx.x; ok && t < tiles; t += gridDim.x) {
             int tm, tn;
             const int second = t >= tiles_one ? 1 : 0;
-            tile_coords(t - second * tiles_one, tiles_m, tiles_n, tm, tn);
+            tile_coords(t - second * tiles_one, tiles_m, tiles_n, group_rows, tm, tn);
             const int m0 = tm * GM, n0 = tn * kTileN;
             for (int ks = 0; ks < nk_total; ++ks, ++it) {
                 const int s = it % kStages;
@@ -276,7 +277,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
         for (int t = blockIdx.x; ok && t < tiles; t += gridDim.x, ++ti) {
             int tm, tn;
             const int second = t >= tiles_one ? 1 : 0;
-            tile_coords(t - second * tiles_one, tiles_m, tiles_n, tm, tn);
+            tile_coords(t - second * tiles_one, tiles_m, tiles_n, group_rows, tm, tn);
             const int buf = ti & 1;
             const int m0 = tm * GM, n0 = tn * kTileN;
             if (kEpi == EPI_STORE && has_res && leader) {     // the tile's residual: into L2 while its main loop runs
@@ -433,10 +434,19 @@ cudaError_t launch_gemm(const Operand &A0, const Operand &B0, const Operand *A1,
     if (e != cudaSuccess) return e;
     const int tiles = ((M + GM - 1) / GM) * ((N + (kDualN ? 128 : GN) - 1) / (kDualN ? 128 : GN)) * nbatch;
     const int nparts = (A1 && !kDualN && nbatch == 1) ? 2 : 1;
+    // Groups of 8 tile rows, unless B is too large to stay in L2 between groups (above 48 MB): then groups as tall as
+    // keeps their A rows within 32 MB, so that B is swept fewer times (measured: taller groups cost the products with
+    // a small B 2-5 %, and save the forward gate GEMM, whose B is W1 and W3 together, 3 % and 70 % of its DRAM reads)
+    const long long b_bytes = (long long)B0.rows * B0.cols * 2 * ((kDualN || nparts == 2) ? 2 : 1);
+    long long group_rows = 8;
+    if (b_bytes > (48LL << 20)) {
+        group_rows = (32LL << 20) / ((long long)GM * K * nparts * 2);
+        group_rows = group_rows < 8 ? 8 : group_rows > 64 ? 64 : group_rows;
+    }
     LaunchScope scope(MOA_KERNEL_OTHER, st);
     kernel<<<tiles < 148 ? tiles : 148, kGemmThreads, kGemmSmem, st>>>(ma0, mb0, ma1, mb1, mc[0], mc[1], mc[2], mc[3], M, N, K, nparts,
                                                                       nbatch, a_blocked ? 1 : 0, b_blocked ? 1 : 0,
-                                                                      has_res ? 1 : 0, device_status_ptr());
+                                                                      has_res ? 1 : 0, (int)group_rows, device_status_ptr());
     return cudaGetLastError();
 }
 

@@ -356,7 +356,7 @@ def make_block_inputs(B, n, H, d, dff, seed):
                                                 (2, 512, 8, 128, 2048, False)])
 def test_transformer_block_composed_from_the_pieces(rt, B, n, H, d, dff, causal):
     """The complete block (two norms, QKV projection, attention, output projection, gated MLP, two residual
-    connections) forward+backward as 24 library calls against the fp64 block oracle.  Errors of the bf16 stages
+    connections) forward+backward as 20 library calls against the fp64 block oracle.  Errors of the bf16 stages
     compound along the block, so the bar here is 2e-2 of each tensor's max (each piece alone is held to 1e-2)."""
     torch, mb = rt
     inp = make_block_inputs(B, n, H, d, dff, seed=70 + n)
