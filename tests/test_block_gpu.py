@@ -368,3 +368,45 @@ def test_transformer_block_composed_from_the_pieces(rt, B, n, H, d, dff, causal)
         assert np.all(np.isfinite(got[k])), k
         e = mi.rel_err(got[k], ref[k])
         assert e <= 2e-2, (k, e)
+
+
+def test_gated_mlp_full_bench_size_sampled(rt):
+    """The benchmark's size (n 16384, d 2048, d_ff 8192), in the launch configuration the benchmark times: sampled
+    token rows (a, u, h, y, dx are row-local) and sampled hidden units (columns of a, u, h, da, du give dW2[:,k],
+    dW1[k,:], dW3[k,:]) against fp64 evaluations of the definition."""
+    torch, mb = rt
+    n, d, dff = 16384, 2048, 8192
+    gen = torch.Generator(device="cuda").manual_seed(23)
+    bf = torch.bfloat16
+    rnd = lambda *shape, s=1.0: (torch.randn(shape, generator=gen, device="cuda") * s).to(bf)
+    x, dy = rnd(n, d), rnd(n, d)
+    W1, W3, W2 = rnd(dff, d, s=d ** -0.5), rnd(dff, d, s=d ** -0.5), rnd(d, dff, s=dff ** -0.5)
+    a, u, h = (_nan_like(torch, (n, dff)) for _ in range(3))
+    y, dx = _nan_like(torch, (n, d)), _nan_like(torch, (n, d))
+    dW1, dW3, dW2 = _nan_like(torch, (dff, d)), _nan_like(torch, (dff, d)), _nan_like(torch, (d, dff))
+    desc = mb.make_mlp_desc(n, d, dff)
+    ws = torch.empty(mb.moa_gated_mlp_workspace_bytes(desc), dtype=torch.uint8, device="cuda")
+    mb.moa_gated_mlp_fwd(desc, x, W1, W3, W2, a, u, h, y)
+    mb.moa_gated_mlp_bwd(desc, x, W1, W3, W2, a, u, h, dy, dx, dW1, dW3, dW2, ws)
+    assert mb.moa_last_device_status() == mb.MOA_OK
+    f64 = lambda t: t.float().cpu().numpy().astype(np.float64)
+    xf, dyf, w1, w3, w2 = f64(x), f64(dy), f64(W1), f64(W3), f64(W2)
+    rng = np.random.default_rng(3)
+    rows = np.unique(np.concatenate([[0, 127, 128, n - 1], rng.integers(0, n, 28)]))
+    ref = oracle.gated_mlp_fwd_bwd(xf[rows], w1, w3, w2, dyf[rows])          # row-local outputs of the sampled rows
+    for k, t in (("a", a), ("u", u), ("h", h), ("y", y), ("dx", dx)):
+        e = mi.rel_err(f64(t[torch.from_numpy(rows).cuda()]), ref[k])
+        assert e <= TOL, (k, e)
+    units = np.unique(np.concatenate([[0, 127, 128, dff - 1], rng.integers(0, dff, 12)]))
+    sig = lambda v: 1.0 / (1.0 + np.exp(-v))
+    ak, uk = xf @ w1[units].T, xf @ w3[units].T                                # [n, units]
+    hk = ak * sig(ak) * uk
+    dhk = dyf @ w2[:, units]
+    dak = dhk * uk * sig(ak) * (1.0 + ak * (1.0 - sig(ak)))
+    duk = dhk * ak * sig(ak)
+    ut = torch.from_numpy(units).cuda()
+    assert mi.rel_err(f64(dW2[:, ut]), dyf.T @ hk) <= TOL
+    assert mi.rel_err(f64(dW1[ut]), dak.T @ xf) <= TOL
+    assert mi.rel_err(f64(dW3[ut]), duk.T @ xf) <= TOL
+    for t in (y, dx, dW1, dW3, dW2, a, u, h):
+        assert bool(torch.isfinite(t.float()).all())
