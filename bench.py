@@ -680,10 +680,11 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "moa" else args.warmup
 
-    if args.decode:
-        return run_decode(args)
-    if args.block:
-        return run_block(args)
+    if args.decode or args.block:
+        # single-GPU legs: under a multi-rank launch rank 0 alone runs them
+        if int(os.environ.get("RANK", "0")) != 0:
+            return 0
+        return run_decode(args) if args.decode else run_block(args)
     from paper_2609_33916_b200 import inputs as mi
     w = mi.CONFIGS[args.workload]
     if args.impl == "reference":
