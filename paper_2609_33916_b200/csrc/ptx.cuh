@@ -91,6 +91,37 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     return true;
 }
 
+// After a wait has expired the CTA winds down; copies this thread asked for may still be on their way into the
+// CTA's shared memory.  ArmCounts remembers how often the thread armed each barrier, and mbar_drain gives the last
+// phase armed on each of them a bounded time (about 0.1 s of SM clock) to complete before the thread leaves.
+constexpr long long kDrainCycles = 200000000LL;
+template <int N>
+struct ArmCounts {
+    uint32_t n[N];
+    __device__ __forceinline__ ArmCounts()
+    {
+#pragma unroll
+        for (int i = 0; i < N; ++i) n[i] = 0;
+    }
+};
+template <int N>
+__device__ __forceinline__ void mbar_arm(uint64_t *bars, int idx, uint32_t bytes, ArmCounts<N> &c)
+{
+    mbar_arrive_expect_tx(bars + idx, bytes);
+    ++c.n[idx];
+}
+template <int N>
+__device__ __noinline__ void mbar_drain(uint64_t *bars, const ArmCounts<N> &c)
+{
+    for (int i = 0; i < N; ++i) {
+        if (c.n[i] == 0) continue;
+        const uint32_t parity = (c.n[i] - 1) & 1;
+        const long long t0 = clock64();
+        while (!mbar_try_wait(bars + i, parity))
+            if (clock64() - t0 > kDrainCycles) break;
+    }
+}
+
 // -------------------------------------------------------------------- fences / proxies
 __device__ __forceinline__ void fence_proxy_async_smem()
 {

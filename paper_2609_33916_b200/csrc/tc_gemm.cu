@@ -132,6 +132,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tbase = *tmem_slot;
+    ArmCounts<G_COUNT> armed;        // barriers this thread armed for copies into shared memory (producer, epilogue leader)
 
     if (warp == 0 && lane == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -152,7 +153,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                 const CUtensorMap *mb = ((part || second) && !kDualN) ? &mapB1 : &mapB0;
                 uint8_t *sa = sm + s * kStageBytes, *sb = sa + kABytes;
                 uint64_t *full = bars + G_FULL + s;
-                mbar_arrive_expect_tx(full, kStageBytes);
+                mbar_arm(bars, G_FULL + s, kStageBytes, armed);
                 if (kAMn) {
                     if (a_blocked) {                          // one copy: (64 columns, K rows, column blocks)
                         tma_load_3d(sa, ma, full, 0, k0, m0 / 64);
@@ -251,7 +252,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
             uint8_t *buf = sout + b * kOutBox;
             if (leader) {
                 bulk_wait_read<1>();                                   // the store issued two chunks ago has left this buffer
-                mbar_arrive_expect_tx(bars + G_RES + b, kOutBox);
+                mbar_arm(bars, G_RES + (int)b, kOutBox, armed);
                 tma_load_3d(buf, &mapC2, bars + G_RES + b, col0, row0, 0);
             }
             if (!mbar_wait(bars + G_RES + b, (chunk_q >> 1) & 1, abortp, status, GERR_RES)) return false;
@@ -344,7 +345,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                 for (int c0 = 0; ok && c0 < GN; c0 += 64, ++in_q) {
                     if (leader) {
                         bulk_wait_read<0>();              // the previous chunk's stores have left both buffers
-                        mbar_arrive_expect_tx(bars + G_IN, 2 * kOutBox);
+                        mbar_arm(bars, G_IN, 2 * kOutBox, armed);
                         tma_load_3d(sout, &mapC2, bars + G_IN, n0 + c0, m0, 0);
                         tma_load_3d(sout + kOutBox, &mapC3, bars + G_IN, n0 + c0, m0, 0);
                     }
@@ -388,6 +389,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tbase, 512);
+    if (*abortp) mbar_drain(bars, armed);      // a wait expired: let copies still on their way land (bounded)
 }
 
 struct Operand {
