@@ -298,16 +298,18 @@ rmsnorm_ring_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__
 
     if (warp == kRingGroups * kRingWarps) {
         if (lane == 0) {
+            ArmCounts<kRingStages> armed;     // stages armed for copies into the ring
             for (int i = 0; i < my_stages; ++i) {
                 const int s = i % kRingStages;
                 if (!mbar_wait(empty + s, ((i / kRingStages) & 1) ^ 1, abortp, status, NERR_EMPTY)) break;
                 const long long row0 = ((long long)blockIdx.x + (long long)i * gridDim.x) * rows_stage;
                 const int rows = (int)min((long long)rows_stage, (long long)n - row0);
                 const uint32_t bytes = (uint32_t)(rows * row_bytes);
-                mbar_arrive_expect_tx(full + s, kBwd ? 2 * bytes : bytes);
+                mbar_arm(full, s, kBwd ? 2 * bytes : bytes, armed);
                 bulk_load_1d(nring + s * stage_bytes, x + row0 * d, bytes, full + s);
                 if (kBwd) bulk_load_1d(nring + s * stage_bytes + arr_bytes, dy + row0 * d, bytes, full + s);
             }
+            mbar_drain(full, armed);      // copies still on their way land before the CTA leaves (bounded)
         }
     } else {
         const float inv_d = 1.f / (float)d;

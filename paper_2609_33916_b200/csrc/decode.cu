@@ -282,15 +282,17 @@ decode_ring_kernel(const T *__restrict__ q, const T *__restrict__ K, const T *__
         if (lane == 0) {
             const uint8_t *Kh = reinterpret_cast<const uint8_t *>(K) + ((size_t)job.bkv * n + job.k_begin) * kRowBytes;
             const uint8_t *Vh = reinterpret_cast<const uint8_t *>(V) + ((size_t)job.bkv * n + job.k_begin) * kRowBytes;
+            ArmCounts<kStages> armed;     // stages armed for copies into the ring
             for (int t = 0; t < ntiles; ++t) {
                 const int s = t % kStages;
                 if (t >= kStages && !mbar_wait(empty + s, (t / kStages - 1) & 1, abortp, status, 0x301u)) break;
                 const int rows = min(kTileRows, job.k_end - job.k_begin - t * kTileRows);
                 const uint32_t bytes = (uint32_t)rows * kRowBytes;
-                mbar_arrive_expect_tx(full + s, 2 * bytes);
+                mbar_arm(full, s, 2 * bytes, armed);
                 bulk_load_1d(ring + (size_t)s * 2 * kTileBytes, Kh + (size_t)t * kTileBytes, bytes, full + s);
                 bulk_load_1d(ring + (size_t)s * 2 * kTileBytes + kTileBytes, Vh + (size_t)t * kTileBytes, bytes, full + s);
             }
+            mbar_drain(full, armed);      // copies still on their way land before the CTA leaves (bounded)
         }
     } else {
         // ----------------------------------------------------------------- consumers

@@ -104,11 +104,25 @@ struct ArmCounts {
         for (int i = 0; i < N; ++i) n[i] = 0;
     }
 };
+// The same for one barrier that was armed `uses` times (kernels whose producer counts its loads in registers).
+__device__ __forceinline__ void mbar_drain_one(uint64_t *bar, int uses)
+{
+    if (uses <= 0) return;
+    const uint32_t parity = (uint32_t)(uses - 1) & 1u;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity))
+        if (clock64() - t0 > kDrainCycles) break;
+}
 template <int N>
 __device__ __forceinline__ void mbar_arm(uint64_t *bars, int idx, uint32_t bytes, ArmCounts<N> &c)
 {
     mbar_arrive_expect_tx(bars + idx, bytes);
     ++c.n[idx];
+}
+template <int N>
+__device__ __forceinline__ void mbar_arm(uint64_t *bars, uint64_t *bar, uint32_t bytes, ArmCounts<N> &c)
+{
+    mbar_arm(bars, (int)(bar - bars), bytes, c);
 }
 template <int N>
 __device__ __noinline__ void mbar_drain(uint64_t *bars, const ArmCounts<N> &c)

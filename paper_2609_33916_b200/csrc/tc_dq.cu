@@ -81,8 +81,9 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
 
     if (warp == 8) {
         // ------------------------------------------------------------------ TMA producer
+        ArmCounts<B_COUNT> armed;     // barriers armed for copies into shared memory
         if (lane == 0 && nkt > 0) {
-            mbar_arrive_expect_tx(bars + B_Q, 2 * SM::kTile);
+            mbar_arm(bars, bars + B_Q, 2 * SM::kTile, armed);
             for (int b = 0; b < kBoxes; ++b) {
                 tma_load_4d(sm + SM::offQ + b * kBoxBytes, &mapQ, bars + B_Q, 64 * b, q0, hq, bb);
                 tma_load_4d(sm + SM::offdO + b * kBoxBytes, &mapdO, bars + B_Q, 64 * b, q0, hq, bb);
@@ -92,7 +93,7 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
             const int s = j & 1;
             if (j >= 2 && !mbar_wait(bars + B_KVEMPTY + s, ((j >> 1) - 1) & 1, abortp, status, ERR_EMPTY)) break;
             if (lane == 0) {
-                mbar_arrive_expect_tx(bars + B_KVFULL + s, 2 * SM::kTile);
+                mbar_arm(bars, bars + B_KVFULL + s, 2 * SM::kTile, armed);
                 for (int b = 0; b < kBoxes; ++b) {
                     tma_load_4d(sm + SM::offK + s * SM::kTile + b * kBoxBytes, &mapK, bars + B_KVFULL + s, 64 * b, j * 128, hk, bb);
                     tma_load_4d(sm + SM::offV + s * SM::kTile + b * kBoxBytes, &mapV, bars + B_KVFULL + s, 64 * b, j * 128, hk, bb);
@@ -100,6 +101,7 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
             }
             __syncwarp();
         }
+        if (lane == 0) mbar_drain(bars, armed);     // copies of this CTA still on their way land before it leaves (bounded)
     } else if (warp == 9 && lane == 0) {
         // ------------------------------------------------------- UMMA issuer (one thread)
         constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0);

@@ -114,6 +114,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
 
     if (warp == 8) {
         // ------------------------------------------------------------------ TMA producer
+        int nk = 0, nv = 0;     // K and V tiles requested so far (slot = count & 1)
         if (lane == 0 && nkt > 0) {
             mbar_arrive_expect_tx(bars + F_Q, kTileBytes);
             for (int b = 0; b < kBoxes; ++b) tma_load_4d(sQ + b * kBoxBytes, &mapQ, bars + F_Q, 64 * b, q0, hq, bb);
@@ -126,9 +127,11 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             for (int j = 0; j < min(nkt, 2); ++j) {
                 if (lane == 0) {
                     mbar_arrive_expect_tx(bars + F_KFULL + j, kTileBytes);
+                    ++nk;
                     for (int b = 0; b < kBoxes; ++b)
                         tma_load_4d(sK + j * kTileBytes + b * kBoxBytes, &mapK, bars + F_KFULL + j, 64 * b, (kt0 + j) * BN, hk, bb);
                     mbar_arrive_expect_tx(bars + F_VFULL + j, kTileBytes);
+                    ++nv;
                     for (int b = 0; b < kBoxes; ++b)
                         tma_load_4d(sV + j * kTileBytes + b * kBoxBytes, &mapV, bars + F_VFULL + j, 64 * b, (kt0 + j) * BN, hk, bb);
                 }
@@ -142,16 +145,26 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             if (j >= 2 && !mbar_wait(bars + F_KEMPTY + s, ((j >> 1) - 1) & 1, abortp, status, ERR_K)) break;
             if (lane == 0) {
                 mbar_arrive_expect_tx(bars + F_KFULL + s, kTileBytes);
+                ++nk;
                 for (int b = 0; b < kBoxes; ++b)
                     tma_load_4d(sK + s * kTileBytes + b * kBoxBytes, &mapK, bars + F_KFULL + s, 64 * b, (kt0 + j) * BN, hk, bb);
             }
             if (j >= 2 && !mbar_wait(bars + F_VEMPTY + s, ((j >> 1) - 1) & 1, abortp, status, ERR_V)) break;
             if (lane == 0) {
                 mbar_arrive_expect_tx(bars + F_VFULL + s, kTileBytes);
+                ++nv;
                 for (int b = 0; b < kBoxes; ++b)
                     tma_load_4d(sV + s * kTileBytes + b * kBoxBytes, &mapV, bars + F_VFULL + s, 64 * b, (kt0 + j) * BN, hk, bb);
             }
             __syncwarp();
+        }
+        if (lane == 0 && *abortp) {
+            // a wait expired somewhere in the CTA: copies still on their way land before it leaves (bounded)
+            mbar_drain_one(bars + F_Q, nkt > 0 ? 1 : 0);
+            for (int s = 0; s < 2; ++s) {
+                mbar_drain_one(bars + F_KFULL + s, nk > s ? (nk - s + 1) / 2 : 0);
+                mbar_drain_one(bars + F_VFULL + s, nv > s ? (nv - s + 1) / 2 : 0);
+            }
         }
     } else if (warp == 9 && lane == 0) {
         // ------------------------------------------- UMMA issuer for the score GEMMs (one thread)

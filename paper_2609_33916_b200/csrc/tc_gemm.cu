@@ -132,12 +132,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tbase = *tmem_slot;
-    ArmCounts<G_COUNT> armed;        // barriers this thread armed for copies into shared memory (producer, epilogue leader)
 
     if (warp == 0 && lane == 0) {
         // ------------------------------------------------------------------ TMA producer
         prefetch_tensormap(&mapA0);
         prefetch_tensormap(&mapB0);
+        ArmCounts<G_COUNT> armed;     // barriers armed for copies into shared memory
         int it = 0;
         bool ok = true;
         for (int t = blockIdx.x; ok && t < tiles; t += gridDim.x) {
@@ -179,6 +179,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                 }
             }
         }
+        mbar_drain(bars, armed);      // copies of this CTA still on their way land before it leaves (bounded)
     } else if (warp == 1 && lane == 0) {
         // ------------------------------------------------------------------- UMMA issuer
         constexpr uint32_t idesc = idesc_bf16_f32(GM, GN, kAMn ? 1 : 0, kBMn ? 1 : 0);
@@ -219,6 +220,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
         const int half = (warp - 2) / 4;                           // which 32 columns of a 64-column chunk
         const bool leader = tid == 64;
         uint32_t epi_phase = 0, chunk_q = 0, in_q = 0;
+        ArmCounts<G_COUNT> armed;     // barriers the leader armed for copies into the staging buffers
         bool ok = true;
         // all epilogue threads meet (bounded wait)
         auto epi_sync = [&]() -> bool {
@@ -384,12 +386,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                 }
             }
         }
-        if (leader) bulk_wait<0>();       // every store has completed before the CTA gives up its shared memory
+        if (leader) {
+            bulk_wait<0>();               // every store has completed before the CTA gives up its shared memory
+            mbar_drain(bars, armed);      // and so has every copy into the staging buffers (bounded)
+        }
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tbase, 512);
-    if (*abortp) mbar_drain(bars, armed);      // a wait expired: let copies still on their way land (bounded)
 }
 
 struct Operand {

@@ -91,26 +91,28 @@ mat_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     const int total = 2 * nkt;   // pass 1: statistics; pass 2: P out, O += P V
 
     if (warp == 4) {
+        ArmCounts<6> armed;     // barriers armed for copies into shared memory
         if (lane == 0 && nkt > 0) {
-            mbar_arrive_expect_tx(bar_q, kTile);
+            mbar_arm(bars, bar_q, kTile, armed);
             for (int b = 0; b < kBoxes; ++b) tma_load_3d(sQ + b * kBoxBytes, &mapQ, bar_q, 64 * b, q0, bh);
         }
         for (int jj = 0; jj < total; ++jj) {
             const int pass2 = jj >= nkt, j = jj - pass2 * nkt;
             if (jj > 0 && !mbar_wait(bar_s, (jj - 1) & 1, abortp, status, FERR + 1)) break;   // K buffer free
             if (lane == 0) {
-                mbar_arrive_expect_tx(bar_k, kTile);
+                mbar_arm(bars, bar_k, kTile, armed);
                 for (int b = 0; b < kBoxes; ++b) tma_load_3d(sK + b * kBoxBytes, &mapK, bar_k, 64 * b, j * 128, bh);
             }
             if (pass2) {
                 if (j > 0 && !mbar_wait(bar_o, (j - 1) & 1, abortp, status, FERR + 2)) break;  // V buffer free
                 if (lane == 0) {
-                    mbar_arrive_expect_tx(bar_v, kTile);
+                    mbar_arm(bars, bar_v, kTile, armed);
                     for (int b = 0; b < kBoxes; ++b) tma_load_3d(sV + b * kBoxBytes, &mapV, bar_v, 64 * b, j * 128, bh);
                 }
             }
             __syncwarp();
         }
+        if (lane == 0) mbar_drain(bars, armed);     // copies still on their way land before the CTA leaves (bounded)
     } else if (warp == 5 && lane == 0) {
         constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0);
         constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, 0, 1);
@@ -279,8 +281,9 @@ mat_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     const int niter = (*abortp == 0) ? (nqt - i_begin) : 0;
 
     if (warp == 8) {
+        ArmCounts<MB_COUNT> armed;     // barriers armed for copies into shared memory
         if (lane == 0 && niter > 0) {
-            mbar_arrive_expect_tx(bars + MB_KV, 2 * SM::kTile);
+            mbar_arm(bars, bars + MB_KV, 2 * SM::kTile, armed);
             for (int b = 0; b < kBoxes; ++b) {
                 tma_load_3d(sm + SM::offK + b * kBoxBytes, &mapK, bars + MB_KV, 64 * b, k0, bh);
                 tma_load_3d(sm + SM::offV + b * kBoxBytes, &mapV, bars + MB_KV, 64 * b, k0, bh);
@@ -290,19 +293,20 @@ mat_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
             const int s = it & 1, q0 = (i_begin + it) * 128;
             if (it >= 2 && !mbar_wait(bars + MB_DOEMPTY + s, ((it >> 1) - 1) & 1, abortp, status, BERR + 1)) break;
             if (lane == 0) {
-                mbar_arrive_expect_tx(bars + MB_DOFULL + s, SM::kTile);
+                mbar_arm(bars, bars + MB_DOFULL + s, SM::kTile, armed);
                 for (int b = 0; b < kBoxes; ++b)
                     tma_load_3d(sm + SM::offdO + s * SM::kTile + b * kBoxBytes, &mapdO, bars + MB_DOFULL + s, 64 * b, q0, bh);
             }
             if (it >= 2 && !mbar_wait(bars + MB_QEMPTY + s, ((it >> 1) - 1) & 1, abortp, status, BERR + 2)) break;
             if (lane == 0) {
-                mbar_arrive_expect_tx(bars + MB_QFULL + s, SM::kTile + 512);
+                mbar_arm(bars, bars + MB_QFULL + s, SM::kTile + 512, armed);
                 for (int b = 0; b < kBoxes; ++b)
                     tma_load_3d(sm + SM::offQ + s * SM::kTile + b * kBoxBytes, &mapQ, bars + MB_QFULL + s, 64 * b, q0, bh);
                 bulk_load_1d(sD + s * 128, Dp + (size_t)bh * n_pad + q0, 512, bars + MB_QFULL + s);
             }
             __syncwarp();
         }
+        if (lane == 0) mbar_drain(bars, armed);     // copies still on their way land before the CTA leaves (bounded)
     } else if (warp == 9 && lane == 0) {
         constexpr uint32_t idesc_st = idesc_bf16_f32(128, 128, 0, 0);
         constexpr uint32_t idesc_acc = idesc_bf16_f32(128, D, 0, 1);
@@ -465,11 +469,12 @@ mat_dq_kernel(const __grid_constant__ CUtensorMap mapGST, const __grid_constant_
     const int nkt = (*abortp == 0) ? nkt_want : 0;
 
     if (warp == 4) {
+        ArmCounts<5> armed;     // barriers armed for copies into shared memory
         for (int j = 0; j < nkt; ++j) {
             const int s = j & 1;
             if (j >= 2 && !mbar_wait(bar_empty + s, ((j >> 1) - 1) & 1, abortp, status, QERR + 1)) break;
             if (lane == 0) {
-                mbar_arrive_expect_tx(bar_full + s, kTileG + kTileK);
+                mbar_arm(bars, bar_full + s, kTileG + kTileK, armed);
                 // dS^T tile: rows = keys j*128.., columns = queries q0.. (two 64-column boxes)
                 for (int b = 0; b < 2; ++b)
                     tma_load_3d(sG + s * kTileG + b * kBoxBytes, &mapGST, bar_full + s, q0 + 64 * b, j * 128, bh);
@@ -478,6 +483,7 @@ mat_dq_kernel(const __grid_constant__ CUtensorMap mapGST, const __grid_constant_
             }
             __syncwarp();
         }
+        if (lane == 0) mbar_drain(bars, armed);     // copies still on their way land before the CTA leaves (bounded)
     } else if (warp == 5 && lane == 0) {
         constexpr uint32_t idesc = idesc_bf16_f32(128, D, 1, 1);   // A = dS^T tile (MN-major), B = K (MN-major)
         const DescParts dp = desc_parts();
