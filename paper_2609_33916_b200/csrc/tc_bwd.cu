@@ -602,6 +602,13 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     if (warp == kMmaWarp) tmem_dealloc(tbase, kTmemCols);
+    if (*abortp && tid == kLoadWarp * 32) {
+        // A wait expired: copies this thread asked for may still be on their way into the CTA's shared memory.  It
+        // stays for a fixed 400,000 cycles (hundreds of times a copy's latency) before the CTA can leave.  (The other
+        // kernels wait on the barriers they armed; here that bookkeeping cost 1.5-3 % under the role's register cap.)
+        const long long t0 = clock64();
+        while (clock64() - t0 < 400000LL) { }
+    }
 }
 
 template <int D, bool kBulk, bool kGrouped>
