@@ -205,6 +205,14 @@ moa_status moa_decode_attn(const moa_decode_desc *desc, const void *q, const voi
  * else MOA_OK.  Outputs of a timed-out kernel are undefined. */
 moa_status moa_last_device_status(void *stream);
 
+/* Self-test of that mechanism: enqueues one warp that waits on a barrier nothing will ever
+ * complete, with a limit of `limit_cycles` SM cycles (clamped to 1,000 .. 2,000,000,000; a
+ * million is about half a millisecond) instead of the kernels' two seconds.  The wait expires,
+ * the warp records the expiry and returns; the next moa_last_device_status on the stream then
+ * reports MOA_ERR_TIMEOUT (once) and the device stays usable.  Nothing faults and nothing hangs:
+ * this is the path a real kernel takes when a copy or a partner never arrives. */
+moa_status moa_selftest_expired_wait(long long limit_cycles, void *stream);
+
 /* Per-kernel device timing, for benchmarks.  The paper's lesson that device time and
  * wall time differ (Sec. 3, device-timer vs wall clock) is why this exists: while
  * enabled, the library records a CUDA event pair on the caller's stream around each

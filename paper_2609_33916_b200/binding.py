@@ -30,6 +30,7 @@ EXPORTS = (
     "moa_decode_workspace_bytes", "moa_decode_attn",
     "moa_rmsnorm_workspace_bytes", "moa_rmsnorm_fwd", "moa_rmsnorm_bwd",
     "moa_gated_mlp_fwd", "moa_gated_mlp_workspace_bytes", "moa_gated_mlp_bwd", "moa_gemm",
+    "moa_selftest_expired_wait",
 )
 
 
@@ -118,6 +119,8 @@ def lib() -> ctypes.CDLL:
         L.moa_gated_mlp_bwd.argtypes = [mp] + [vp] * 12 + [vp, sz, vp]
         L.moa_last_device_status.restype = ctypes.c_int
         L.moa_last_device_status.argtypes = [vp]
+        L.moa_selftest_expired_wait.restype = ctypes.c_int
+        L.moa_selftest_expired_wait.argtypes = [ctypes.c_longlong, vp]
         L.moa_launch_count.restype = ctypes.c_uint64
         L.moa_status_string.restype = ctypes.c_char_p
         L.moa_status_string.argtypes = [ctypes.c_int]
@@ -249,6 +252,12 @@ def moa_rmsnorm_bwd(desc, x, g, r, dy, dx, dg, ws=None, stream=None, ws_bytes=No
     if check and s != MOA_OK:
         raise MoaError(s, "moa_rmsnorm_bwd")
     return s
+
+
+def moa_selftest_expired_wait(limit_cycles=1000000, stream=None) -> int:
+    """Enqueues one warp whose bounded wait expires after `limit_cycles`; moa_last_device_status then reports
+    MOA_ERR_TIMEOUT once."""
+    return int(lib().moa_selftest_expired_wait(int(limit_cycles), _stream(stream)))
 
 
 def make_gemm_desc(M, N, K, a_layout=0, b_layout=0, dtype=MOA_BF16) -> moa_gemm_desc:

@@ -1,6 +1,7 @@
 // C-ABI entry points (include/moa_attn.h): argument checks, workspace carving and
 // the sequence of kernel launches of each operation.  No arithmetic here.
 #include "common.cuh"
+#include "ptx.cuh"
 #include <atomic>
 #include <mutex>
 #include <vector>
@@ -496,6 +497,33 @@ moa_status moa_last_device_status(void *stream)
         return MOA_ERR_TIMEOUT;
     }
     return MOA_OK;
+}
+
+// One warp waits on a barrier that nothing completes; the bounded wait expires and records it.
+__global__ void selftest_expired_wait_kernel(unsigned int *status, long long limit)
+{
+    __shared__ uint64_t bar;
+    __shared__ uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        moa::ptx::mbar_init(&bar, 1);
+        abort_flag = 0;
+        moa::ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    moa::ptx::mbar_wait(&bar, 0, &abort_flag, status, 0x7F1u, limit);
+}
+
+moa_status moa_selftest_expired_wait(long long limit_cycles, void *stream)
+{
+    moa_status s = check_device_arch();
+    if (s != MOA_OK) return s;
+    if (limit_cycles < 1000) limit_cycles = 1000;
+    if (limit_cycles > 2000000000LL) limit_cycles = 2000000000LL;
+    unsigned int *p = device_status_ptr();
+    if (!p) return MOA_ERR_CUDA;
+    count_launch();
+    selftest_expired_wait_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(p, limit_cycles);
+    return cudaGetLastError() == cudaSuccess ? MOA_OK : MOA_ERR_CUDA;
 }
 
 moa_status moa_profile_enable(int on)

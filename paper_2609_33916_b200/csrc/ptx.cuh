@@ -72,7 +72,7 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity)
 }
 
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
-                                          unsigned int *status, uint32_t code)
+                                          unsigned int *status, uint32_t code, long long limit = kWaitCycles)
 {
     if (mbar_test_wait(bar, parity)) return true;
     if (mbar_try_wait(bar, parity)) return true;
@@ -81,7 +81,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 7u) == 0) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitCycles) {
+            if (clock64() - t0 > limit) {
                 *abort_flag = 1;
                 if (status) atomicCAS(status, 0u, code);
                 return false;
