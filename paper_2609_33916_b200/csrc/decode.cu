@@ -198,13 +198,83 @@ struct DecodeJob {
     }
 };
 
+// Merge of one query head's segments (thread = (stripe of segments, output column), the stripes merged through
+// `sh`: kStripes * (D + 2) floats), normalise, write out (and the natural-log lse).  Called by every thread of a CTA
+// of at least 256 threads; threads past 256 only take part in the barriers.  The partial results are read with
+// ld.global.cg: other CTAs wrote them.
+template <typename T, int D>
+__device__ __forceinline__ void merge_head(const float *__restrict__ part_o, const float *__restrict__ part_ml,
+                                           T *__restrict__ out, float *__restrict__ lse, int splits, size_t BH, size_t head,
+                                           float *sh)
+{
+    constexpr int kStripes = 256 / D;
+    float *sh_o = sh, *sh_m = sh + kStripes * D, *sh_l = sh_m + kStripes;
+    const bool active = threadIdx.x < 256;
+    const int c = threadIdx.x % D, stripe = (threadIdx.x / D) % kStripes;
+    // two passes, so that the loads of a pass do not wait on the running maximum: first the maximum
+    // of the stripe, then the weighted sums
+    float mx = -INFINITY, o = 0.f, ls = 0.f;
+    if (active) {
+#pragma unroll 8
+        for (int s = stripe; s < splits; s += kStripes) mx = fmaxf(mx, __ldcg(part_ml + ((size_t)s * BH + head) * 2));
+        const float ref = (mx == -INFINITY) ? 0.f : mx;
+#pragma unroll 8
+        for (int s = stripe; s < splits; s += kStripes) {
+            const size_t at = (size_t)s * BH + head;
+            const float w = exp2f(__ldcg(part_ml + at * 2) - ref);
+            o = fmaf(__ldcg(part_o + at * D + c), w, o);
+            ls = fmaf(__ldcg(part_ml + at * 2 + 1), w, ls);
+        }
+        sh_o[stripe * D + c] = o;
+        if (c == 0) { sh_m[stripe] = mx; sh_l[stripe] = ls; }
+    }
+    __syncthreads();
+    if (active && stripe == 0) {
+        float mt = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < kStripes; ++k) mt = fmaxf(mt, sh_m[k]);
+        float ot = 0.f, lt = 0.f;
+#pragma unroll
+        for (int k = 0; k < kStripes; ++k) {
+            const float a = exp2f(sh_m[k] - mt);
+            ot = fmaf(sh_o[k * D + c], a, ot);
+            lt = fmaf(sh_l[k], a, lt);
+        }
+        out[head * D + c] = from_float<T>(ot / lt);
+        if (lse && c == 0) lse[head] = (mt + log2f(lt)) * kLn2;
+    }
+    __syncthreads();
+}
+
+// The CTA that finishes last among the `splits` CTAs of a group of query heads merges their partial results, so
+// the merge needs no launch of its own and runs while other heads are still streaming.  No CTA waits for another:
+// each one publishes its partials (fence), then adds one to the group's counter (zeroed by the host before the
+// launch); whoever reads splits - 1 is the last.
+template <typename T, int D>
+__device__ __forceinline__ void merge_if_last(unsigned int *counters, const DecodeJob &job, int splits, size_t BH,
+                                              const float *part_o, const float *part_ml, T *out, float *lse, float *sh)
+{
+    __shared__ int s_last;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned int old = atomicAdd(counters + (size_t)job.bkv * gridDim.y + blockIdx.y, 1u);
+        s_last = old == (unsigned int)(splits - 1);
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    for (int g = 0; g < job.gcount; ++g) merge_head<T, D>(part_o, part_ml, out, lse, splits, BH, job.head0 + g, sh);
+}
+
 // ---- variant 1: rows straight from global memory into registers (16-byte streaming loads, kUnroll row
 // groups of K and of V in flight per warp).  Few registers when the group is small, so several CTAs
 // per SM keep enough bytes in flight: used for one or two query heads per K/V head.
 template <typename T, int D, int GC>
 __global__ void __launch_bounds__(kThreads)
 decode_split_kernel(const T *__restrict__ q, const T *__restrict__ K, const T *__restrict__ V,
-                    float *__restrict__ part_o, float *__restrict__ part_ml,
+                    float *__restrict__ part_o, float *__restrict__ part_ml, T *__restrict__ out, float *__restrict__ lse,
+                    unsigned int *__restrict__ counters,
                     int n, int H, int Hkv, int group, int splits, int keys_per_split, size_t BH, float scale_log2)
 {
     using State = DecodeState<T, D, GC>;
@@ -232,6 +302,7 @@ decode_split_kernel(const T *__restrict__ q, const T *__restrict__ K, const T *_
     }
     extern __shared__ float sm[];
     st.finish(sm, warp, lane, kWarps, job.gcount, job.head0, job.split, BH, part_o, part_ml, kThreads);
+    merge_if_last<T, D>(counters, job, splits, BH, part_o, part_ml, out, lse, sm);
 }
 
 // ---- variant 2: the cache segment streams through a shared-memory ring filled by bulk copies (a tile
@@ -251,7 +322,8 @@ struct Ring {
 template <typename T, int D, int GC>
 __global__ void __launch_bounds__(kRingThreads, 1)
 decode_ring_kernel(const T *__restrict__ q, const T *__restrict__ K, const T *__restrict__ V,
-                   float *__restrict__ part_o, float *__restrict__ part_ml,
+                   float *__restrict__ part_o, float *__restrict__ part_ml, T *__restrict__ out, float *__restrict__ lse,
+                   unsigned int *__restrict__ counters,
                    int n, int H, int Hkv, int group, int splits, int keys_per_split, size_t BH, float scale_log2,
                    unsigned int *status)
 {
@@ -323,49 +395,7 @@ decode_ring_kernel(const T *__restrict__ q, const T *__restrict__ K, const T *__
     if (warp == kWarps) st.init(q + job.head0 * D, 0, 0, 0.f);     // the producer warp holds no state
     st.finish(reinterpret_cast<float *>(ring), warp, lane, kWarps, job.gcount, job.head0, job.split, BH, part_o,
               part_ml, kRingThreads);
-}
-
-// One block per query head: merge the segments, normalise, write out (and the natural-log lse).
-// 256 threads: thread = (stripe of segments, output column); the stripes are merged in shared memory.
-template <typename T, int D>
-__global__ void __launch_bounds__(256)
-decode_merge_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml,
-                    T *__restrict__ out, float *__restrict__ lse, int splits, size_t BH)
-{
-    constexpr int kStripes = 256 / D;
-    __shared__ float sh_o[kStripes][D], sh_m[kStripes], sh_l[kStripes];
-    const size_t head = blockIdx.x;
-    const int c = threadIdx.x % D, stripe = threadIdx.x / D;
-    // two passes, so that the loads of a pass do not wait on the running maximum: first the maximum
-    // of the stripe, then the weighted sums
-    float mx = -INFINITY, o = 0.f, ls = 0.f;
-#pragma unroll 8
-    for (int s = stripe; s < splits; s += kStripes) mx = fmaxf(mx, part_ml[((size_t)s * BH + head) * 2]);
-    const float ref = (mx == -INFINITY) ? 0.f : mx;
-#pragma unroll 8
-    for (int s = stripe; s < splits; s += kStripes) {
-        const size_t at = (size_t)s * BH + head;
-        const float w = exp2f(part_ml[at * 2] - ref);
-        o = fmaf(part_o[at * D + c], w, o);
-        ls = fmaf(part_ml[at * 2 + 1], w, ls);
-    }
-    sh_o[stripe][c] = o;
-    if (c == 0) { sh_m[stripe] = mx; sh_l[stripe] = ls; }
-    __syncthreads();
-    if (stripe == 0) {
-        float mt = -INFINITY;
-#pragma unroll
-        for (int k = 0; k < kStripes; ++k) mt = fmaxf(mt, sh_m[k]);
-        float ot = 0.f, lt = 0.f;
-#pragma unroll
-        for (int k = 0; k < kStripes; ++k) {
-            const float a = exp2f(sh_m[k] - mt);
-            ot = fmaf(sh_o[k][c], a, ot);
-            lt = fmaf(sh_l[k], a, lt);
-        }
-        out[head * D + c] = from_float<T>(ot / lt);
-        if (lse && c == 0) lse[head] = (mt + log2f(lt)) * kLn2;
-    }
+    merge_if_last<T, D>(counters, job, splits, BH, part_o, part_ml, out, lse, reinterpret_cast<float *>(ring));
 }
 
 // Merge for the tensor-core route: O_part [splits*B, Hkv, G, D] bf16 (each normalised over its own
@@ -414,11 +444,16 @@ int group_chunk(int group) { return group >= 8 ? 8 : group >= 4 ? 4 : group >= 2
 
 template <typename T, int D, int GC>
 cudaError_t launch_split(const DecodeProblem &p, const void *q, const void *K, const void *V, float *part_o,
-                         float *part_ml, int splits, int keys_per_split, cudaStream_t st)
+                         float *part_ml, void *out, float *lse, unsigned int *counters, int splits, int keys_per_split,
+                         cudaStream_t st)
 {
     const int group = p.H / p.Hkv;
     dim3 grid((unsigned)(p.B * p.Hkv * splits), (unsigned)((group + GC - 1) / GC));
-    const size_t merge_smem = (size_t)kWarps * GC * (D + 2) * sizeof(float);
+    size_t merge_smem = (size_t)kWarps * GC * (D + 2) * sizeof(float);       // warps' states; then the stripes of merge_head
+    if (merge_smem < (size_t)(256 / D) * (D + 2) * sizeof(float)) merge_smem = (size_t)(256 / D) * (D + 2) * sizeof(float);
+    // one counter per (K/V head, chunk of query heads): the last of its CTAs to finish merges
+    cudaError_t ce = cudaMemsetAsync(counters, 0, (size_t)p.B * p.Hkv * grid.y * sizeof(unsigned int), st);
+    if (ce != cudaSuccess) return ce;
     LaunchScope scope(MOA_KERNEL_OTHER, st);
     if (GC >= 4) {
         constexpr int kStages = Ring<T, D>::kStages;
@@ -427,16 +462,17 @@ cudaError_t launch_split(const DecodeProblem &p, const void *q, const void *K, c
                                              (int)(smem > merge_smem ? smem : merge_smem));
         if (e != cudaSuccess) return e;
         decode_ring_kernel<T, D, GC><<<grid, kRingThreads, smem > merge_smem ? smem : merge_smem, st>>>(
-            (const T *)q, (const T *)K, (const T *)V, part_o, part_ml, p.n, p.H, p.Hkv, group, splits, keys_per_split,
-            (size_t)p.B * p.H, p.scale * kLog2e, device_status_ptr());
+            (const T *)q, (const T *)K, (const T *)V, part_o, part_ml, (T *)out, lse, counters, p.n, p.H, p.Hkv, group, splits,
+            keys_per_split, (size_t)p.B * p.H, p.scale * kLog2e, device_status_ptr());
         return cudaGetLastError();
     }
     cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<T, D, GC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)merge_smem);
     if (e != cudaSuccess) return e;
     decode_split_kernel<T, D, GC><<<grid, kThreads, merge_smem, st>>>((const T *)q, (const T *)K, (const T *)V, part_o,
-                                                                      part_ml, p.n, p.H, p.Hkv, group, splits,
-                                                                      keys_per_split, (size_t)p.B * p.H, p.scale * kLog2e);
+                                                                      part_ml, (T *)out, lse, counters, p.n, p.H, p.Hkv,
+                                                                      group, splits, keys_per_split, (size_t)p.B * p.H,
+                                                                      p.scale * kLog2e);
     return cudaGetLastError();
 }
 
@@ -448,15 +484,13 @@ cudaError_t launch_decode(const DecodeProblem &p, const void *q, const void *K, 
     const int keys_per_split = (p.n + splits - 1) / splits;
     const size_t BH = (size_t)p.B * p.H;
     float *part_o = ws, *part_ml = ws + (size_t)splits * BH * D;
+    unsigned int *counters = reinterpret_cast<unsigned int *>(part_ml + (size_t)splits * BH * 2);
     const int gc = group_chunk(p.H / p.Hkv);
-    cudaError_t e = gc == 8 ? launch_split<T, D, 8>(p, q, K, V, part_o, part_ml, splits, keys_per_split, st)
-                  : gc == 4 ? launch_split<T, D, 4>(p, q, K, V, part_o, part_ml, splits, keys_per_split, st)
-                  : gc == 2 ? launch_split<T, D, 2>(p, q, K, V, part_o, part_ml, splits, keys_per_split, st)
-                            : launch_split<T, D, 1>(p, q, K, V, part_o, part_ml, splits, keys_per_split, st);
-    if (e != cudaSuccess) return e;
-    LaunchScope scope(MOA_KERNEL_OTHER, st);
-    decode_merge_kernel<T, D><<<(unsigned)BH, 256, 0, st>>>(part_o, part_ml, (T *)out, lse, splits, BH);
-    return cudaGetLastError();
+    // the merge of a head's segments is done by the last of its CTAs to finish (no merge launch)
+    return gc == 8 ? launch_split<T, D, 8>(p, q, K, V, part_o, part_ml, out, lse, counters, splits, keys_per_split, st)
+         : gc == 4 ? launch_split<T, D, 4>(p, q, K, V, part_o, part_ml, out, lse, counters, splits, keys_per_split, st)
+         : gc == 2 ? launch_split<T, D, 2>(p, q, K, V, part_o, part_ml, out, lse, counters, splits, keys_per_split, st)
+                   : launch_split<T, D, 1>(p, q, K, V, part_o, part_ml, out, lse, counters, splits, keys_per_split, st);
 }
 
 }  // namespace
@@ -517,7 +551,8 @@ size_t decode_workspace_bytes(const DecodeProblem &p, int dtype)
         const size_t heads = (size_t)splits * p.B * p.H;
         return ((heads * p.d * 2 + 255) / 256) * 256 + heads * sizeof(float);
     }
-    return (size_t)decode_splits(p) * p.B * p.H * (p.d + 2) * sizeof(float);
+    // partial results of the segments, then one counter per (K/V head, chunk of query heads)
+    return (size_t)decode_splits(p) * p.B * p.H * (p.d + 2) * sizeof(float) + (size_t)p.B * p.H * sizeof(unsigned int);
 }
 
 cudaError_t decode_attn(const DecodeProblem &p, int dtype, const void *q, const void *K, const void *V, void *out,
