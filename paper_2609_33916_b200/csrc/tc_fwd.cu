@@ -49,7 +49,7 @@ enum : uint32_t { ERR_Q = 0x101, ERR_K = 0x102, ERR_V = 0x103, ERR_S = 0x104, ER
 
 enum { F_Q = 0, F_KFULL = 1 /*2*/, F_KEMPTY = 3 /*2*/, F_VFULL = 5 /*2*/, F_VEMPTY = 7 /*2*/, F_S = 9 /*2*/,
        F_P = 11 /*[buffer][half]: 4*/, F_O = 15, F_X = 16 /*epilogue exchange*/, F_OB = 17 /*2: score buffer consumed*/,
-       F_E = 19 /*O tile staged in shared memory*/, F_COUNT = 20 };
+       F_E = 19 /*O tile staged in shared memory*/, F_DONE = 20 /*last P V of the job has completed*/, F_COUNT = 21 };
 
 // Split use of the kernel (decode: few query rows, a long cache): the key tiles are divided among
 // `splits` CTAs per (head, query tile); each writes the attention over its tiles alone (normalised O
@@ -225,6 +225,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             umma_commit(bars + F_OB + b);
             umma_commit(bars + F_VEMPTY + b);
             umma_commit(bars + F_O);
+            if (j == nkt - 1) umma_commit(bars + F_DONE);
         }
     } else if (warp < 8) {
         // ---------------------------------------------------------------- softmax warps
@@ -350,7 +351,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         xch[h * 128 + lane_row] = make_float2(m_used, l);
         mbar_arrive(bars + F_X);
         if (ok && mbar_wait(bars + F_X, 0, abortp, status, ERR_P) &&
-            mbar_wait(bars + F_O, (nkt - 1) & 1, abortp, status, ERR_O)) {
+            mbar_wait(bars + F_DONE, 0, abortp, status, ERR_O)) {
+            // (F_DONE, not the per-tile F_O with the last tile's parity: the softmax threads can finish the last
+            // tile while the P V products of the last TWO tiles are still pending -- the S and P V issuers are
+            // different threads -- and a wait on F_O's parity would then be satisfied by the tile before those,
+            // which has the same parity.  Seen in decode through this kernel, where tiles arrive at HBM pace:
+            // about one CTA in a hundred wrote an O that missed its last tiles.)
             tc_fence_after();
             const float2 other = xch[(h ^ 1) * 128 + lane_row];
             const float m_all = fmaxf(m_used, other.x);
