@@ -4,11 +4,22 @@
 //   C[M,N] = sum over operand pairs p of  A_p[M,K] * B_p[N,K]^T
 //
 // One persistent CTA per SM walks output tiles of 128 x 256.  Warp 0 is the TMA producer (a ring of
-// kStages stages of 64 K-elements: 16 KB of A, 32 KB of B), warp 1 allocates TMEM and issues the
+// stages of 64 K-elements: 16 KB of A, 32 KB of B), warp 1 allocates TMEM and issues the
 // UMMAs (M = 128, N = 256, K = 16 each, four per stage), warps 2-9 are the epilogue (two warps per
 // 32-lane group of TMEM, one column half each).  The two
 // 256-column halves of TMEM alternate between tiles, so the epilogue of a tile runs under the main
 // loop of the next one.  Every wait is bounded (ptx::mbar_wait).
+//
+// kPair: the same roles in each of the two CTAs of a cluster, on tiles of 256 x 256: the CTA of rank 0
+// issues UMMAs of M = 256 (tcgen05.mma.cta_group::2) that read 128 rows of A and HALF of the B rows
+// from each CTA's shared memory and write 128 x 256 accumulators in each CTA's TMEM.  Per SM and
+// unit of work the B traffic (L2 -> shared memory, shared memory -> tensor core) halves, and a stage
+// is 32 KB, so the ring has six.  Both producers' copies complete on the full barrier of rank 0; its
+// commits arrive on the empty and accumulator-full barriers of both CTAs; both epilogues hand the
+// accumulator back on the barrier of rank 0; a cluster-wide barrier at both ends keeps either CTA
+// from touching the other before it is set up or after it has left.  Measured: K-major products
+// 1340 -> 1430-1440 TFLOP/s; products with an MN-major A gain nothing (they ran at 1440 already) and
+// stay on single CTAs, as do launches with fewer 256-row tiles than SM pairs.
 //
 // Operand storage is a template choice per operand, because the backward's GEMMs read the same
 // arrays transposed:
@@ -34,12 +45,20 @@ namespace {
 using namespace ptx;
 
 constexpr int GM = 128, GN = 256, GK = 64;
-constexpr int kStages = 4;   // three stages measured 7-16 % slower: the ring has to cover the L2 latency
 constexpr int kGemmThreads = 320;                      // producer, issuer, eight epilogue warps
-constexpr int kABytes = GM * GK * 2, kBBytes = GN * GK * 2, kStageBytes = kABytes + kBBytes;
+constexpr int kABytes = GM * GK * 2, kBBytes = GN * GK * 2;
+// A CTA on its own stages 16 KB of A and 32 KB of B per 64 K-elements, four stages (three measured 7-16 % slower: the
+// ring has to cover the L2 latency).  A CTA of a pair stages 16 KB of A and its half of B, 16 KB: six stages.
+constexpr int kMaxStages = 6;
+__host__ __device__ constexpr int gemm_stages(bool pair) { return pair ? 6 : 4; }
+__host__ __device__ constexpr int gemm_stage_bytes(bool pair) { return kABytes + (pair ? kBBytes / 2 : kBBytes); }
 constexpr int kMnBox = 64 * GK * 2;                    // one MN-major box: 64 columns x 64 K-rows
 constexpr int kOutBox = 128 * 64 * 2;                  // one staged output chunk: 128 rows x 64 columns, bf16
-constexpr int kGemmSmem = kStages * kStageBytes + 2 * kOutBox + 1024 /* alignment */ + 256 /* barriers */;
+__host__ __device__ constexpr int gemm_smem(bool pair)
+{
+    return gemm_stages(pair) * gemm_stage_bytes(pair) + 2 * kOutBox + 1024 /* alignment */ + 256 /* barriers */;
+}
+constexpr int kStages = kMaxStages;                    // barrier slots (the ring uses gemm_stages(pair) of them)
 
 enum { EPI_STORE = 0, EPI_SWIGLU_FWD = 1, EPI_SWIGLU_BWD = 2 };
 enum { G_FULL = 0, G_EMPTY = kStages, G_ACCFULL = 2 * kStages, G_ACCEMPTY = 2 * kStages + 2, G_EPI = 2 * kStages + 4,
@@ -83,7 +102,7 @@ __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int
     tm = g * kGroup + (r - tn * rows);
 }
 
-template <bool kAMn, bool kBMn, int kEpi>
+template <bool kAMn, bool kBMn, int kEpi, bool kPair>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapB0,
                const __grid_constant__ CUtensorMap mapA1, const __grid_constant__ CUtensorMap mapB1,
@@ -94,15 +113,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
     constexpr int kTileN = kDualN ? 128 : GN;                // output columns a tile covers
     // Epilogue warps: two per 32-lane group of TMEM; together they fill one 64-column output chunk at a time
     constexpr int kEpiWarps = 8;
+    // kPair: the two CTAs of a cluster share tiles of 256 rows: UMMAs of M = 256 issued by the CTA of rank 0 read the
+    // A rows and the B half staged in each CTA (this CTA: rows rank*128.. of the tile, B rows rank*128.. of its 256)
+    // and write each CTA's accumulator; every CTA runs its own producer and epilogue.
+    constexpr int kSt = gemm_stages(kPair), kStageBytes = gemm_stage_bytes(kPair), kTileM = kPair ? 2 * GM : GM;
+    const uint32_t rank = kPair ? cluster_ctarank() : 0u;
+    const int cta = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x, ncta = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *sm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t *sout = sm + kStages * kStageBytes;               // two staged output chunks (128-byte swizzle)
+    uint8_t *sout = sm + kSt * kStageBytes;               // two staged output chunks (128-byte swizzle)
     uint64_t *bars = reinterpret_cast<uint64_t *>(sout + 2 * kOutBox);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + G_COUNT);
     volatile uint32_t *abortp = tmem_slot + 1;
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
 
-    const int tiles_m = (M + GM - 1) / GM, tiles_n = (N + kTileN - 1) / kTileN;
+    const int tiles_m = (M + kTileM - 1) / kTileM, tiles_n = (N + kTileN - 1) / kTileN;
     // nbatch = 2: two independent products of one shape in one launch (A1 B1^T -> map C1 after A0 B0^T ->
     // map C0), so that their tiles share the waves of the persistent grid
     const int tiles_one = tiles_m * tiles_n, tiles = tiles_one * nbatch;
@@ -115,8 +140,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
         }
         mbar_init(bars + G_ACCFULL + 0, 1);
         mbar_init(bars + G_ACCFULL + 1, 1);
-        mbar_init(bars + G_ACCEMPTY + 0, 32 * kEpiWarps);
-        mbar_init(bars + G_ACCEMPTY + 1, 32 * kEpiWarps);
+        mbar_init(bars + G_ACCEMPTY + 0, (kPair ? 2 : 1) * 32 * kEpiWarps);   // a pair: the epilogue threads of both CTAs
+        mbar_init(bars + G_ACCEMPTY + 1, (kPair ? 2 : 1) * 32 * kEpiWarps);
         mbar_init(bars + G_EPI, 32 * kEpiWarps);
         mbar_init(bars + G_IN, 1);
         mbar_init(bars + G_RES + 0, 1);
@@ -125,11 +150,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
         fence_mbar_init();
     }
     if (warp == 1) {
-        tmem_alloc(tmem_slot, 512);
-        tmem_relinquish();
+        if (kPair) {
+            tmem_alloc_pair(tmem_slot, 512);
+            tmem_relinquish_pair();
+        } else {
+            tmem_alloc(tmem_slot, 512);
+            tmem_relinquish();
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (kPair) cluster_sync_all();       // the other CTA's barriers are initialised before anything arrives on them
     tc_fence_after();
     const uint32_t tbase = *tmem_slot;
 
@@ -140,74 +171,97 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
         ArmCounts<G_COUNT> armed;     // barriers armed for copies into shared memory
         int it = 0;
         bool ok = true;
-        for (int t = blockIdx.x; ok && t < tiles; t += gridDim.x) {
+        for (int t = cta; ok && t < tiles; t += ncta) {
             int tm, tn;
             const int second = t >= tiles_one ? 1 : 0;
             tile_coords(t - second * tiles_one, tiles_m, tiles_n, group_rows, tm, tn);
-            const int m0 = tm * GM, n0 = tn * kTileN;
+            const int m0 = tm * kTileM + (int)rank * GM, n0 = tn * kTileN;
+            const int nb0 = n0 + ((kPair && !kDualN) ? (int)rank * (GN / 2) : 0);    // first B row this CTA stages
             for (int ks = 0; ks < nk_total; ++ks, ++it) {
-                const int s = it % kStages;
-                if (!mbar_wait(bars + G_EMPTY + s, ((it / kStages) & 1) ^ 1, abortp, status, GERR_EMPTY)) { ok = false; break; }
+                const int s = it % kSt;
+                if (!mbar_wait(bars + G_EMPTY + s, ((it / kSt) & 1) ^ 1, abortp, status, GERR_EMPTY)) { ok = false; break; }
                 const int part = ks / nk, k0 = (ks - part * nk) * GK;
                 const CUtensorMap *ma = (part || second) ? &mapA1 : &mapA0;
                 const CUtensorMap *mb = ((part || second) && !kDualN) ? &mapB1 : &mapB0;
                 uint8_t *sa = sm + s * kStageBytes, *sb = sa + kABytes;
                 uint64_t *full = bars + G_FULL + s;
-                mbar_arm(bars, G_FULL + s, kStageBytes, armed);
+                // a pair: the copies of both CTAs complete on the barrier of rank 0, which its producer arms for both
+                const uint32_t full_pair = kPair ? mapa_u32(smem_u32(full), 0) : 0u;
+                if (!kPair || rank == 0) mbar_arm(bars, G_FULL + s, (kPair ? 2 : 1) * kStageBytes, armed);
+                auto load = [&](void *dst, const CUtensorMap *m, int x, int y, int z) {
+                    if (kPair) tma_load_3d_pair(dst, m, full_pair, x, y, z);
+                    else tma_load_3d(dst, m, full, x, y, z);
+                };
                 if (kAMn) {
                     if (a_blocked) {                          // one copy: (64 columns, K rows, column blocks)
-                        tma_load_3d(sa, ma, full, 0, k0, m0 / 64);
+                        load(sa, ma, 0, k0, m0 / 64);
                     } else {
-                        tma_load_3d(sa, ma, full, m0, k0, 0);
-                        tma_load_3d(sa + kMnBox, ma, full, m0 + 64, k0, 0);
+                        load(sa, ma, m0, k0, 0);
+                        load(sa + kMnBox, ma, m0 + 64, k0, 0);
                     }
                 } else {
-                    tma_load_3d(sa, ma, full, k0, m0, 0);
+                    load(sa, ma, k0, m0, 0);
                 }
                 if (kBMn) {
                     if (b_blocked) {
-                        tma_load_3d(sb, mb, full, 0, k0, n0 / 64);
+                        load(sb, mb, 0, k0, nb0 / 64);
                     } else {
 #pragma unroll
-                        for (int b = 0; b < 4; ++b) tma_load_3d(sb + b * kMnBox, mb, full, n0 + 64 * b, k0, 0);
+                        for (int b = 0; b < (kPair ? 2 : 4); ++b) load(sb + b * kMnBox, mb, nb0 + 64 * b, k0, 0);
                     }
                 } else if (kDualN) {
-                    tma_load_3d(sb, &mapB0, full, k0, n0, 0);
-                    tma_load_3d(sb + kBBytes / 2, &mapB1, full, k0, n0, 0);
+                    if (kPair) {                              // rank 0 stages the W1 rows, rank 1 the W3 rows
+                        load(sb, rank ? &mapB1 : &mapB0, k0, n0, 0);
+                    } else {
+                        load(sb, &mapB0, k0, n0, 0);
+                        load(sb + kBBytes / 2, &mapB1, k0, n0, 0);
+                    }
                 } else {
-                    tma_load_3d(sb, mb, full, k0, n0, 0);
+                    load(sb, mb, k0, nb0, 0);
                 }
             }
         }
         mbar_drain(bars, armed);      // copies of this CTA still on their way land before it leaves (bounded)
-    } else if (warp == 1 && lane == 0) {
+    } else if (warp == 1 && lane == 0 && rank == 0) {
         // ------------------------------------------------------------------- UMMA issuer
-        constexpr uint32_t idesc = idesc_bf16_f32(GM, GN, kAMn ? 1 : 0, kBMn ? 1 : 0);
+        constexpr uint32_t idesc = idesc_bf16_f32(kTileM, GN, kAMn ? 1 : 0, kBMn ? 1 : 0);
         const uint64_t km_proto = smem_desc_sw128(0, 16, 1024), mn_proto = smem_desc_sw128(0, kMnBox, 1024);
         const uint32_t a_hi = (uint32_t)((kAMn ? mn_proto : km_proto) >> 32), b_hi = (uint32_t)((kBMn ? mn_proto : km_proto) >> 32);
         const uint32_t a_lo0 = (uint32_t)(kAMn ? mn_proto : km_proto), b_lo0 = (uint32_t)(kBMn ? mn_proto : km_proto);
         constexpr uint32_t a_step = (kAMn ? 2048 : 32) >> 4, b_step = (kBMn ? 2048 : 32) >> 4;   // per 16 K-elements
         int it = 0, ti = 0;
         bool ok = true;
-        for (int t = blockIdx.x; ok && t < tiles; t += gridDim.x, ++ti) {
+        for (int t = cta; ok && t < tiles; t += ncta, ++ti) {
             const int buf = ti & 1;
             if (!mbar_wait(bars + G_ACCEMPTY + buf, ((ti >> 1) & 1) ^ 1, abortp, status, GERR_ACCEMPTY)) break;
             tc_fence_after();
             const uint32_t acc = tbase + (uint32_t)(buf * GN);
             for (int ks = 0; ks < nk_total; ++ks, ++it) {
-                const int s = it % kStages;
-                if (!mbar_wait(bars + G_FULL + s, (it / kStages) & 1, abortp, status, GERR_FULL)) { ok = false; break; }
+                const int s = it % kSt;
+                if (!mbar_wait(bars + G_FULL + s, (it / kSt) & 1, abortp, status, GERR_FULL)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t a_lo = a_lo0 + ((smem_u32(sm + s * kStageBytes) >> 4) & 0x3FFFu);
                 const uint32_t b_lo = b_lo0 + ((smem_u32(sm + s * kStageBytes + kABytes) >> 4) & 0x3FFFu);
-                if (ks == 0) umma_ss2<false>(acc, a_lo, a_hi, b_lo, b_hi, idesc);
-                else         umma_ss2<true>(acc, a_lo, a_hi, b_lo, b_hi, idesc);
+                if (kPair) {
+                    if (ks == 0) umma_ss2_pair<false>(acc, a_lo, a_hi, b_lo, b_hi, idesc);
+                    else         umma_ss2_pair<true>(acc, a_lo, a_hi, b_lo, b_hi, idesc);
 #pragma unroll
-                for (int q = 1; q < GK / 16; ++q)
-                    umma_ss2<true>(acc, a_lo + q * a_step, a_hi, b_lo + q * b_step, b_hi, idesc);
-                umma_commit(bars + G_EMPTY + s);          // the stage is free once these UMMAs have read it
+                    for (int q = 1; q < GK / 16; ++q)
+                        umma_ss2_pair<true>(acc, a_lo + q * a_step, a_hi, b_lo + q * b_step, b_hi, idesc);
+                    umma_commit_pair(bars + G_EMPTY + s);     // frees the stage in both CTAs
+                } else {
+                    if (ks == 0) umma_ss2<false>(acc, a_lo, a_hi, b_lo, b_hi, idesc);
+                    else         umma_ss2<true>(acc, a_lo, a_hi, b_lo, b_hi, idesc);
+#pragma unroll
+                    for (int q = 1; q < GK / 16; ++q)
+                        umma_ss2<true>(acc, a_lo + q * a_step, a_hi, b_lo + q * b_step, b_hi, idesc);
+                    umma_commit(bars + G_EMPTY + s);          // the stage is free once these UMMAs have read it
+                }
             }
-            if (ok) umma_commit(bars + G_ACCFULL + buf);
+            if (ok) {
+                if (kPair) umma_commit_pair(bars + G_ACCFULL + buf);
+                else umma_commit(bars + G_ACCFULL + buf);
+            }
         }
     } else if (warp >= 2 && warp < 2 + kEpiWarps) {
         // ---------------------------------------------------------------------- epilogue
@@ -222,6 +276,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
         uint32_t epi_phase = 0, chunk_q = 0, in_q = 0;
         ArmCounts<G_COUNT> armed;     // barriers the leader armed for copies into the staging buffers
         bool ok = true;
+        // hands an accumulator back to the issuer (a pair: to the issuer in the CTA of rank 0)
+        const uint32_t accempty_pair = kPair ? mapa_u32(smem_u32(bars + G_ACCEMPTY), 0) : 0u;
+        auto acc_release = [&](int b) {
+            tc_fence_before();
+            if (kPair) mbar_arrive_cluster(accempty_pair + 8u * (uint32_t)b);
+            else mbar_arrive(bars + G_ACCEMPTY + b);
+        };
         // all epilogue threads meet (bounded wait)
         auto epi_sync = [&]() -> bool {
             mbar_arrive(bars + G_EPI);
@@ -241,7 +302,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
             fence_proxy_async_smem();
             if (!epi_sync()) return false;
             if (leader) {
-                tma_store_3d(map, buf, col0, row0, 0);
+                if (row0 < M) tma_store_3d(map, buf, col0, row0, 0);   // (a pair's second half can lie past the last row)
                 bulk_commit();
             }
             ++chunk_q;
@@ -270,19 +331,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
             fence_proxy_async_smem();
             if (!epi_sync()) return false;
             if (leader) {
-                tma_store_3d(map, buf, col0, row0, 0);
+                if (row0 < M) tma_store_3d(map, buf, col0, row0, 0);   // (a pair's second half can lie past the last row)
                 bulk_commit();
             }
             ++chunk_q;
             return true;
         };
         int ti = 0;
-        for (int t = blockIdx.x; ok && t < tiles; t += gridDim.x, ++ti) {
+        for (int t = cta; ok && t < tiles; t += ncta, ++ti) {
             int tm, tn;
             const int second = t >= tiles_one ? 1 : 0;
             tile_coords(t - second * tiles_one, tiles_m, tiles_n, group_rows, tm, tn);
             const int buf = ti & 1;
-            const int m0 = tm * GM, n0 = tn * kTileN;
+            const int m0 = tm * kTileM + (int)rank * GM, n0 = tn * kTileN;
             if (kEpi == EPI_STORE && has_res && leader) {     // the tile's residual: into L2 while its main loop runs
 #pragma unroll
                 for (int c0 = 0; c0 < GN; c0 += 64) tma_prefetch_3d(&mapC2, n0 + c0, m0, 0);
@@ -306,8 +367,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                     tmem_ld(acc + 128 + c, ru);
                     tc_wait_ld();
                     if (c0 == 64) {                       // last read of this accumulator: hand it back early
-                        tc_fence_before();
-                        mbar_arrive(bars + G_ACCEMPTY + buf);
+                        acc_release(buf);
                     }
                     uint32_t pa[16], pu[16], ph[16];
 #pragma unroll
@@ -328,8 +388,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                     tmem_ld(acc + c0 + 32 * half, r);
                     tc_wait_ld();
                     if (c0 == GN - 64) {                  // last read of this accumulator: hand it back early
-                        tc_fence_before();
-                        mbar_arrive(bars + G_ACCEMPTY + buf);
+                        acc_release(buf);
                     }
                     if (has_res) {
                         ok = stage_store_res(&mapC0, r, n0 + c0, m0);
@@ -355,8 +414,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                     tmem_ld(acc + c0 + 32 * half, r);
                     tc_wait_ld();
                     if (c0 == GN - 64) {
-                        tc_fence_before();
-                        mbar_arrive(bars + G_ACCEMPTY + buf);
+                        acc_release(buf);
                     }
                     if (!mbar_wait(bars + G_IN, in_q & 1, abortp, status, GERR_IN)) { ok = false; break; }
 #pragma unroll
@@ -379,8 +437,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                     fence_proxy_async_smem();
                     if (!epi_sync()) { ok = false; break; }
                     if (leader) {
-                        tma_store_3d(&mapC0, sout, n0 + c0, m0, 0);
-                        tma_store_3d(&mapC1, sout + kOutBox, n0 + c0, m0, 0);
+                        if (m0 < M) {
+                            tma_store_3d(&mapC0, sout, n0 + c0, m0, 0);
+                            tma_store_3d(&mapC1, sout + kOutBox, n0 + c0, m0, 0);
+                        }
                         bulk_commit();
                     }
                 }
@@ -393,7 +453,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tbase, 512);
+    if (kPair) {
+        // neither CTA leaves, or frees its TMEM, while the other may still read its shared memory, write its
+        // accumulator or arrive on its barriers
+        __syncwarp();
+        cluster_sync_all();
+        if (warp == 1) tmem_dealloc_pair(tbase, 512);
+    } else if (warp == 1) {
+        tmem_dealloc(tbase, 512);
+    }
 }
 
 struct Operand {
@@ -412,15 +480,15 @@ bool operand_map(CUtensorMap *m, const Operand &o, bool mn_major, int box_rows, 
                               mn_major ? 64 : (uint32_t)box_rows, 64);
 }
 
-template <bool kAMn, bool kBMn, int kEpi>
+template <bool kAMn, bool kBMn, int kEpi, bool kPair>
 // C0..C2: output arrays (row length ldc); unused ones may repeat C0.
-cudaError_t launch_gemm(const Operand &A0, const Operand &B0, const Operand *A1, const Operand *B1, void *C0, void *C1,
+cudaError_t launch_gemm_as(const Operand &A0, const Operand &B0, const Operand *A1, const Operand *B1, void *C0, void *C1,
                         const void *C2, const void *C3, int c_rows, int ldc, int M, int N, int K, cudaStream_t st,
                         int nbatch = 1, bool has_res = false)
 {
     constexpr bool kDualN = kEpi == EPI_SWIGLU_FWD;
     CUtensorMap ma0, mb0, ma1, mb1;
-    const int b_rows = kDualN ? 128 : GN;
+    const int b_rows = (kDualN || kPair) ? 128 : GN;     // B rows one CTA stages per copy
     // MN-major operands whose width is a multiple of 64 come in by one blocked copy per stage (try the encode; if the
     // driver refuses the map, or a width has a tail, use one copy per 64-column block)
     const Operand &a1 = A1 ? *A1 : A0, &b1 = B1 ? *B1 : B0;
@@ -435,10 +503,11 @@ cudaError_t launch_gemm(const Operand &A0, const Operand &B0, const Operand *A1,
     for (int i = 0; i < 4; ++i)     // [c_rows, ldc] bf16, boxes of 128 rows x 64 columns, 128-byte swizzle
         if (!make_tensor_map_3d(&mc[i], cs[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 1, (uint64_t)c_rows, (uint64_t)ldc, 128, 64))
             return cudaErrorInvalidValue;
-    auto kernel = tc_gemm_kernel<kAMn, kBMn, kEpi>;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
+    auto kernel = tc_gemm_kernel<kAMn, kBMn, kEpi, kPair>;
+    constexpr int kSmem = gemm_smem(kPair), kTileM = kPair ? 2 * GM : GM;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
-    const int tiles = ((M + GM - 1) / GM) * ((N + (kDualN ? 128 : GN) - 1) / (kDualN ? 128 : GN)) * nbatch;
+    const int tiles = ((M + kTileM - 1) / kTileM) * ((N + (kDualN ? 128 : GN) - 1) / (kDualN ? 128 : GN)) * nbatch;
     const int nparts = (A1 && !kDualN && nbatch == 1) ? 2 : 1;
     // Groups of 8 tile rows, unless B is too large to stay in L2 between groups (above 48 MB): then groups as tall as
     // keeps their A rows within 32 MB, so that B is swept fewer times (measured: taller groups cost the products with
@@ -449,11 +518,48 @@ cudaError_t launch_gemm(const Operand &A0, const Operand &B0, const Operand *A1,
         group_rows = (32LL << 20) / ((long long)GM * K * nparts * 2);
         group_rows = group_rows < 8 ? 8 : group_rows > 64 ? 64 : group_rows;
     }
+    if (kPair) group_rows = group_rows / 2 < 2 ? 2 : group_rows / 2;     // tile rows of 256
     LaunchScope scope(MOA_KERNEL_OTHER, st);
-    kernel<<<tiles < 148 ? tiles : 148, kGemmThreads, kGemmSmem, st>>>(ma0, mb0, ma1, mb1, mc[0], mc[1], mc[2], mc[3], M, N, K, nparts,
-                                                                      nbatch, a_blocked ? 1 : 0, b_blocked ? 1 : 0,
-                                                                      has_res ? 1 : 0, (int)group_rows, device_status_ptr());
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    const int ctas = kPair ? 2 * (tiles < 74 ? tiles : 74) : (tiles < 148 ? tiles : 148);
+    cfg.gridDim = dim3((unsigned)ctas);
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = kSmem;
+    cfg.stream = st;
+    if (kPair) {
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+    return cudaLaunchKernelEx(&cfg, kernel, ma0, mb0, ma1, mb1, mc[0], mc[1], mc[2], mc[3], M, N, K, nparts, nbatch,
+                              a_blocked ? 1 : 0, b_blocked ? 1 : 0, has_res ? 1 : 0, (int)group_rows, device_status_ptr());
+}
+
+// Pairs of CTAs (tiles of 256 rows, half the B traffic per SM) when there are at least as many 256-row tiles as
+// pairs; single CTAs otherwise.
+int gemm_pair_mode()
+{
+    static int mode = -1;
+    if (mode < 0) {
+        const char *e = getenv("MOA_GEMM_PAIR");
+        mode = e ? atoi(e) : 1;
+    }
+    return mode;
+}
+template <bool kAMn, bool kBMn, int kEpi>
+cudaError_t launch_gemm(const Operand &A0, const Operand &B0, const Operand *A1, const Operand *B1, void *C0, void *C1,
+                        const void *C2, const void *C3, int c_rows, int ldc, int M, int N, int K, cudaStream_t st,
+                        int nbatch = 1, bool has_res = false)
+{
+    const int tn = kEpi == EPI_SWIGLU_FWD ? 128 : GN;
+    const long long pair_tiles = (long long)((M + 2 * GM - 1) / (2 * GM)) * ((N + tn - 1) / tn) * nbatch;
+    if (gemm_pair_mode() == 2 || (gemm_pair_mode() && pair_tiles >= 74 && !kAMn && (kEpi == EPI_STORE || K >= 2048)))
+        return launch_gemm_as<kAMn, kBMn, kEpi, true>(A0, B0, A1, B1, C0, C1, C2, C3, c_rows, ldc, M, N, K, st, nbatch, has_res);
+    return launch_gemm_as<kAMn, kBMn, kEpi, false>(A0, B0, A1, B1, C0, C1, C2, C3, c_rows, ldc, M, N, K, st, nbatch, has_res);
 }
 
 }  // namespace
