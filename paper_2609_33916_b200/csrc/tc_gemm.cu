@@ -520,9 +520,15 @@ cudaError_t launch_gemm_as(const Operand &A0, const Operand &B0, const Operand *
     }
     if (kPair) group_rows = group_rows / 2 < 2 ? 2 : group_rows / 2;     // tile rows of 256
     LaunchScope scope(MOA_KERNEL_OTHER, st);
+    const int ctas = kPair ? 2 * (tiles < 74 ? tiles : 74) : (tiles < 148 ? tiles : 148);
+    if (!kPair) {
+        kernel<<<ctas, kGemmThreads, kSmem, st>>>(ma0, mb0, ma1, mb1, mc[0], mc[1], mc[2], mc[3], M, N, K, nparts, nbatch,
+                                                  a_blocked ? 1 : 0, b_blocked ? 1 : 0, has_res ? 1 : 0, (int)group_rows,
+                                                  device_status_ptr());
+        return cudaGetLastError();
+    }
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
-    const int ctas = kPair ? 2 * (tiles < 74 ? tiles : 74) : (tiles < 148 ? tiles : 148);
     cfg.gridDim = dim3((unsigned)ctas);
     cfg.blockDim = dim3(kGemmThreads);
     cfg.dynamicSmemBytes = kSmem;
