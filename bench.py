@@ -311,6 +311,10 @@ BLOCK_WORKLOADS = {
     "mlp_n8192_d4096_ff16384": ("mlp", 8192, 4096, 16384),
     "mlp_n4096_d1024_ff4096": ("mlp", 4096, 1024, 4096),              # small case for profiler captures (0.4 GB moved per step)
     "mlp_paper_n512_d64_ff256": ("mlp", 512, 64, 256),              # the paper's own traffic-check size (B=2, N=256, D=64, DFF=256)
+    # one product C[M,N] = A[M,K] B[N,K]^T through moa_gemm: (piece, M, K, N)
+    "gemm_m8192_n8192_k8192": ("gemm", 8192, 8192, 8192),
+    "gemm_m16384_n2048_k2048": ("gemm", 16384, 2048, 2048),            # one projection of the block at config 4's tokens
+    "gemm_m8192_n2048_k2048": ("gemm", 8192, 2048, 2048),              # small case for profiler captures
     # the whole pre-norm block (two norms, QKV projection, attention, output projection, gated MLP, residuals),
     # composed from library calls: (piece, B, n, H, d, d_ff, causal)
     "block_c4_b1_n16384_h16_d128_ff8192": ("block", 1, 16384, 16, 128, 8192, False),   # config 4's attention inside a block
@@ -345,7 +349,20 @@ def run_block(args):
     rnd = lambda *shape, s=1.0: (torch.randn(shape, generator=gen, device="cuda") * s).to(bf)
     x, dy = rnd(n, d), rnd(n, d)
     dx = torch.empty_like(x)
-    if piece == "rmsnorm":
+    uploads, result = [x, dy], dx          # what the end-to-end step moves
+    if piece == "gemm":
+        Wb = rnd(dff, d, s=1.0 / math.sqrt(d))
+        C = torch.empty((n, dff), dtype=bf, device="cuda")
+        desc = mb.make_gemm_desc(n, dff, d, 0, 0)
+        uploads, result = [x], C
+
+        def step():
+            mb.moa_gemm(desc, x, Wb, C, None, stream)
+
+        alg = 2.0 * n * d * dff
+        unit, kernel = "TFLOP/s", "tc_gemm_kernel"
+        metric = "bf16 GEMM C = A B^T: TFLOP/s"
+    elif piece == "rmsnorm":
         eps = 1e-5
         g = (1.0 + 0.25 * torch.randn((d,), generator=gen, device="cuda")).to(bf)
         y, dg = torch.empty_like(x), torch.empty_like(g)
@@ -395,16 +412,16 @@ def run_block(args):
     ms = e0.elapsed_time(e1) / args.steps
     value = alg / (ms * 1e-3) / (1e9 if piece == "rmsnorm" else 1e12)
     # end to end: the step's activations (x, dy) come from pinned host memory, dx goes back; weights stay resident
-    hx, hdy = x.cpu().pin_memory(), dy.cpu().pin_memory()
-    hdx = torch.empty((n, d), dtype=bf).pin_memory()
+    hup = [t.cpu().pin_memory() for t in uploads]
+    hres = torch.empty(tuple(result.shape), dtype=bf).pin_memory()
     t0e, t1e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     esteps = max(4, min(args.steps, 10))
     t0e.record(stream)
     for _ in range(esteps):
-        x.copy_(hx, non_blocking=True)
-        dy.copy_(hdy, non_blocking=True)
+        for t, ht in zip(uploads, hup):
+            t.copy_(ht, non_blocking=True)
         step()
-        hdx.copy_(dx, non_blocking=True)
+        hres.copy_(result, non_blocking=True)
     t1e.record(stream)
     torch.cuda.synchronize()
     e2e_ms = t0e.elapsed_time(t1e) / esteps
@@ -422,28 +439,37 @@ def run_block(args):
                 "peak_source": f"{peaks_kind} bf16_tflops (cuBLAS burst)",
                 "frac_of_sustained": value / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
                 "model_flops_per_step": alg,
-                "note": "whole step (the nine GEMMs of forward and backward) against the dense bf16 peak"}
+                "note": ("one product against the dense bf16 peak" if piece == "gemm" else
+                         "whole step (the nine GEMMs of forward and backward) against the dense bf16 peak")}
     line = {
         "metric": metric, "value": value, "unit": unit, "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": args.block, "n": n, "d": d, "d_ff": dff,
+        "config": {"workload": args.block, **({"M": n, "K": d, "N": dff} if piece == "gemm" else {"n": n, "d": d, "d_ff": dff}),
                    "l2": "the arrays of one step exceed the 126 MB L2; no explicit flush" if n * d * 10 > 126e6 or n * dff * 2 > 126e6
                    else "small case: resident in L2 between steps (not a bandwidth figure)"},
         "tokens_per_s": n / (ms * 1e-3),
         "clocks": sampler.summary(),
         "e2e": {"value": alg / (e2e_ms * 1e-3) / (1e9 if piece == "rmsnorm" else 1e12), "unit": unit,
-                "h2d_bytes_per_step": 2 * n * d * 2, "d2h_bytes_per_step": n * d * 2, "ms_per_step": e2e_ms,
-                "how": "x and dy from pinned host memory and dx back every step; gain / weights resident"},
+                "h2d_bytes_per_step": sum(t.numel() for t in uploads) * 2, "d2h_bytes_per_step": result.numel() * 2,
+                "ms_per_step": e2e_ms,
+                "how": ("A from pinned host memory and C back every step; B resident" if piece == "gemm" else
+                        "x and dy from pinned host memory and dx back every step; gain / weights resident")},
         "gpu_launches": int(launches),
         "roofline": roof,
     }
     if not args.no_cpu_baseline:
-        rows = 4096 if piece == "rmsnorm" else (64 if d * dff > 1 << 20 else n)
+        rows = 4096 if piece == "rmsnorm" else (256 if piece == "gemm" else (64 if d * dff > 1 << 20 else n))
         f64 = lambda t: t.float().cpu().numpy().astype(np.float64)
         t0 = time.perf_counter()
         reps = 0
-        if piece == "rmsnorm":
+        if piece == "gemm":
+            xs, wb = f64(x[:rows]), f64(Wb)
+            t0 = time.perf_counter()
+            while time.perf_counter() - t0 < 5.0:
+                oracle.gemm(xs, wb)
+                reps += 1
+        elif piece == "rmsnorm":
             xs, gs, ds = f64(x[:rows]), f64(g), f64(dy[:rows])
             while time.perf_counter() - t0 < 5.0:
                 oracle.rmsnorm_fwd_bwd(xs, gs, ds, eps)
