@@ -52,7 +52,7 @@ def _run_rmsnorm(rt, inp, eps, give_r=True):
 
 
 @pytest.mark.parametrize("n,d", [(1, 8), (5, 64), (33, 128), (257, 768), (100, 1024), (64, 2048), (70, 2056),
-                                 (19, 4096), (9, 5120), (7, 8192), (3000, 512), (4099, 2048)])
+                                 (19, 4096), (9, 5120), (7, 8192), (3000, 512), (4099, 2048), (2500, 4096), (1031, 3000), (600, 2560)])
 @pytest.mark.parametrize("eps", [1e-5, 0.5])
 def test_rmsnorm_matches_oracle(rt, n, d, eps):
     inp = mi.make_norm_inputs(n, d, seed=1000 + n + d)
