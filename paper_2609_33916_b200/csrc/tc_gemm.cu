@@ -49,9 +49,14 @@ constexpr int kGemmThreads = 320;                      // producer, issuer, eigh
 constexpr int kABytes = GM * GK * 2, kBBytes = GN * GK * 2;
 // A CTA on its own stages 16 KB of A and 32 KB of B per 64 K-elements, four stages (three measured 7-16 % slower: the
 // ring has to cover the L2 latency).  A CTA of a pair stages 16 KB of A and its half of B, 16 KB: six stages.
+// In a pair a stage holds two such blocks (128 K-elements, 64 KB) and the ring has three: one wait and one commit of
+// the issuing thread per eight UMMAs instead of per four (that thread's time per stage is on the critical path: a
+// second commit per stage cost 3-4 %).
 constexpr int kMaxStages = 6;
-__host__ __device__ constexpr int gemm_stages(bool pair) { return pair ? 6 : 4; }
-__host__ __device__ constexpr int gemm_stage_bytes(bool pair) { return kABytes + (pair ? kBBytes / 2 : kBBytes); }
+__host__ __device__ constexpr int gemm_sub(bool pair) { return pair ? 2 : 1; }                 // 64-element K blocks per stage
+__host__ __device__ constexpr int gemm_stages(bool pair) { return pair ? 3 : 4; }
+__host__ __device__ constexpr int gemm_sub_bytes(bool pair) { return kABytes + (pair ? kBBytes / 2 : kBBytes); }
+__host__ __device__ constexpr int gemm_stage_bytes(bool pair) { return gemm_sub(pair) * gemm_sub_bytes(pair); }
 constexpr int kMnBox = 64 * GK * 2;                    // one MN-major box: 64 columns x 64 K-rows
 constexpr int kOutBox = 128 * 64 * 2;                  // one staged output chunk: 128 rows x 64 columns, bf16
 __host__ __device__ constexpr int gemm_smem(bool pair)
@@ -117,6 +122,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
     // A rows and the B half staged in each CTA (this CTA: rows rank*128.. of the tile, B rows rank*128.. of its 256)
     // and write each CTA's accumulator; every CTA runs its own producer and epilogue.
     constexpr int kSt = gemm_stages(kPair), kStageBytes = gemm_stage_bytes(kPair), kTileM = kPair ? 2 * GM : GM;
+    constexpr int kSub = gemm_sub(kPair), kSubBytes = gemm_sub_bytes(kPair);
     const uint32_t rank = kPair ? cluster_ctarank() : 0u;
     const int cta = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x, ncta = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     extern __shared__ uint8_t smem_raw[];
@@ -131,7 +137,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
     // nbatch = 2: two independent products of one shape in one launch (A1 B1^T -> map C1 after A0 B0^T ->
     // map C0), so that their tiles share the waves of the persistent grid
     const int tiles_one = tiles_m * tiles_n, tiles = tiles_one * nbatch;
-    const int nk = (K + GK - 1) / GK, nk_total = nk * nparts;
+    const int nk = (K + GK * kSub - 1) / (GK * kSub), nk_total = nk * nparts;     // stages per operand pair
 
     if (tid == 0) {
         for (int i = 0; i < kStages; ++i) {
@@ -180,10 +186,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
             for (int ks = 0; ks < nk_total; ++ks, ++it) {
                 const int s = it % kSt;
                 if (!mbar_wait(bars + G_EMPTY + s, ((it / kSt) & 1) ^ 1, abortp, status, GERR_EMPTY)) { ok = false; break; }
-                const int part = ks / nk, k0 = (ks - part * nk) * GK;
+                const int part = ks / nk;
                 const CUtensorMap *ma = (part || second) ? &mapA1 : &mapA0;
                 const CUtensorMap *mb = ((part || second) && !kDualN) ? &mapB1 : &mapB0;
-                uint8_t *sa = sm + s * kStageBytes, *sb = sa + kABytes;
                 uint64_t *full = bars + G_FULL + s;
                 // a pair: the copies of both CTAs complete on the barrier of rank 0, which its producer arms for both
                 const uint32_t full_pair = kPair ? mapa_u32(smem_u32(full), 0) : 0u;
@@ -192,6 +197,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                     if (kPair) tma_load_3d_pair(dst, m, full_pair, x, y, z);
                     else tma_load_3d(dst, m, full, x, y, z);
                 };
+#pragma unroll
+              for (int sub = 0; sub < kSub; ++sub) {          // (a block past K is filled with zeros by the copy)
+                const int k0 = ((ks - part * nk) * kSub + sub) * GK;
+                uint8_t *sa = sm + s * kStageBytes + sub * kSubBytes, *sb = sa + kABytes;
                 if (kAMn) {
                     if (a_blocked) {                          // one copy: (64 columns, K rows, column blocks)
                         load(sa, ma, 0, k0, m0 / 64);
@@ -219,6 +228,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                 } else {
                     load(sb, mb, k0, nb0, 0);
                 }
+              }
             }
         }
         mbar_drain(bars, armed);      // copies of this CTA still on their way land before it leaves (bounded)
@@ -243,11 +253,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                 const uint32_t a_lo = a_lo0 + ((smem_u32(sm + s * kStageBytes) >> 4) & 0x3FFFu);
                 const uint32_t b_lo = b_lo0 + ((smem_u32(sm + s * kStageBytes + kABytes) >> 4) & 0x3FFFu);
                 if (kPair) {
-                    if (ks == 0) umma_ss2_pair<false>(acc, a_lo, a_hi, b_lo, b_hi, idesc);
-                    else         umma_ss2_pair<true>(acc, a_lo, a_hi, b_lo, b_hi, idesc);
 #pragma unroll
-                    for (int q = 1; q < GK / 16; ++q)
-                        umma_ss2_pair<true>(acc, a_lo + q * a_step, a_hi, b_lo + q * b_step, b_hi, idesc);
+                    for (int sub = 0; sub < kSub; ++sub) {
+                        const uint32_t a_s = a_lo + (uint32_t)(sub * (kSubBytes >> 4)), b_s = b_lo + (uint32_t)(sub * (kSubBytes >> 4));
+                        if (ks == 0 && sub == 0) umma_ss2_pair<false>(acc, a_s, a_hi, b_s, b_hi, idesc);
+                        else                     umma_ss2_pair<true>(acc, a_s, a_hi, b_s, b_hi, idesc);
+#pragma unroll
+                        for (int q = 1; q < GK / 16; ++q)
+                            umma_ss2_pair<true>(acc, a_s + q * a_step, a_hi, b_s + q * b_step, b_hi, idesc);
+                    }
                     umma_commit_pair(bars + G_EMPTY + s);     // frees the stage in both CTAs
                 } else {
                     if (ks == 0) umma_ss2<false>(acc, a_lo, a_hi, b_lo, b_hi, idesc);
