@@ -13,12 +13,12 @@
 // kPair: the same roles in each of the two CTAs of a cluster, on tiles of 256 x 256: the CTA of rank 0
 // issues UMMAs of M = 256 (tcgen05.mma.cta_group::2) that read 128 rows of A and HALF of the B rows
 // from each CTA's shared memory and write 128 x 256 accumulators in each CTA's TMEM.  Per SM and
-// unit of work the B traffic (L2 -> shared memory, shared memory -> tensor core) halves, and a stage
-// is 32 KB, so the ring has six.  Both producers' copies complete on the full barrier of rank 0; its
+// unit of work the B traffic (L2 -> shared memory, shared memory -> tensor core) halves; a stage holds
+// two 64-element K blocks (64 KB) and the ring has three.  Both producers' copies complete on the full barrier of rank 0; its
 // commits arrive on the empty and accumulator-full barriers of both CTAs; both epilogues hand the
 // accumulator back on the barrier of rank 0; a cluster-wide barrier at both ends keeps either CTA
 // from touching the other before it is set up or after it has left.  Measured: K-major products
-// 1340 -> 1430-1440 TFLOP/s; products with an MN-major A gain nothing (they ran at 1440 already) and
+// 1340 -> 1380-1480 TFLOP/s; products with an MN-major A gain nothing (they ran at 1440 already) and
 // stay on single CTAs, as do launches with fewer 256-row tiles than SM pairs.
 //
 // Operand storage is a template choice per operand, because the backward's GEMMs read the same
