@@ -90,9 +90,8 @@ moa_status moa_gated_mlp_bwd(const moa_mlp_desc *desc, const void *x, const void
  * M = out, N = in, K = tokens.  R (NULL or [M,N]) is added in the epilogue: a residual connection, or
  * the running sum of a chain of products.  M, N, K >= 1; the row length of every array a multiple of
  * 8 (rows stay 16-byte aligned); dtype MOA_BF16; fp32 accumulation.
- * Tiling: 128 x 256 output tiles on single CTAs, or 256 x 256 tiles on pairs of CTAs (one cluster of two, UMMAs of
- * M = 256 reading half of B from each CTA's shared memory) where A is stored [M,K] and the launch has at least one
- * such tile per pair of SMs.  The environment variable MOA_GEMM_PAIR, read once per process, overrides the choice for
+ * Tiling: 256 x 256 tiles on pairs of CTAs (one cluster of two, UMMAs of M = 256 reading half of B from each CTA's
+ * shared memory), or 128 x 256 output tiles on single CTAs where M is so small that pairs would need more waves.  The environment variable MOA_GEMM_PAIR, read once per process, overrides the choice for
  * tests and measurements: 0 = never pairs, 2 = always pairs; the results do not depend on it beyond rounding order
  * (they are the same bits: every output element is one fp32 accumulation over K in the same order). */
 typedef struct {

@@ -17,9 +17,9 @@
 // two 64-element K blocks (64 KB) and the ring has three.  Both producers' copies complete on the full barrier of rank 0; its
 // commits arrive on the empty and accumulator-full barriers of both CTAs; both epilogues hand the
 // accumulator back on the barrier of rank 0; a cluster-wide barrier at both ends keeps either CTA
-// from touching the other before it is set up or after it has left.  Measured: K-major products
-// 1340 -> 1380-1480 TFLOP/s; products with an MN-major A gain nothing (they ran at 1440 already) and
-// stay on single CTAs, as do launches with fewer 256-row tiles than SM pairs.
+// from touching the other before it is set up or after it has left.  Measured: products of every
+// operand layout 1240-1340 -> 1350-1530 TFLOP/s; launches of a few tiles, and shapes whose M is so
+// small that pairs would need more waves, stay on single CTAs.
 //
 // Operand storage is a template choice per operand, because the backward's GEMMs read the same
 // arrays transposed:
@@ -559,8 +559,8 @@ cudaError_t launch_gemm_as(const Operand &A0, const Operand &B0, const Operand *
                               a_blocked ? 1 : 0, b_blocked ? 1 : 0, has_res ? 1 : 0, (int)group_rows, device_status_ptr());
 }
 
-// Pairs of CTAs (tiles of 256 rows, half the B traffic per SM) when there are at least as many 256-row tiles as
-// pairs; single CTAs otherwise.
+// Pairs of CTAs (tiles of 256 rows, half the B traffic per SM) by default; single CTAs where pairs would need more
+// waves.  MOA_GEMM_PAIR (read once): 0 never pairs, 2 always.
 int gemm_pair_mode()
 {
     static int mode = -1;
@@ -576,8 +576,13 @@ cudaError_t launch_gemm(const Operand &A0, const Operand &B0, const Operand *A1,
                         int nbatch = 1, bool has_res = false)
 {
     const int tn = kEpi == EPI_SWIGLU_FWD ? 128 : GN;
-    const long long pair_tiles = (long long)((M + 2 * GM - 1) / (2 * GM)) * ((N + tn - 1) / tn) * nbatch;
-    if (gemm_pair_mode() == 2 || (gemm_pair_mode() && pair_tiles >= 74 && !kAMn && (kEpi == EPI_STORE || K >= 2048)))
+    const long long cols = (N + tn - 1) / tn;
+    const long long pair_tiles = (long long)((M + 2 * GM - 1) / (2 * GM)) * cols * nbatch;
+    const long long single_tiles = (long long)((M + GM - 1) / GM) * cols * nbatch;
+    // pairs unless they would need more waves than single CTAs (tiny M); the two gate GEMMs only when the main loop
+    // outlasts their epilogue
+    const bool fits = pair_tiles >= 8 && (pair_tiles + 73) / 74 <= (single_tiles + 147) / 148;   // (a few tiles: launch-bound)
+    if (gemm_pair_mode() == 2 || (gemm_pair_mode() && fits && (kEpi == EPI_STORE || K >= 2048)))
         return launch_gemm_as<kAMn, kBMn, kEpi, true>(A0, B0, A1, B1, C0, C1, C2, C3, c_rows, ldc, M, N, K, st, nbatch, has_res);
     return launch_gemm_as<kAMn, kBMn, kEpi, false>(A0, B0, A1, B1, C0, C1, C2, C3, c_rows, ldc, M, N, K, st, nbatch, has_res);
 }
