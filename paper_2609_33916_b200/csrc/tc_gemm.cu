@@ -582,7 +582,7 @@ cudaError_t launch_gemm(const Operand &A0, const Operand &B0, const Operand *A1,
     // pairs unless they would need more waves than single CTAs (tiny M); the two gate GEMMs only when the main loop
     // outlasts their epilogue
     const bool fits = pair_tiles >= 8 && (pair_tiles + 73) / 74 <= (single_tiles + 147) / 148;   // (a few tiles: launch-bound)
-    if (gemm_pair_mode() == 2 || (gemm_pair_mode() && fits && (kEpi == EPI_STORE || K >= 2048)))
+    if (gemm_pair_mode() == 2 || (gemm_pair_mode() && fits && (kEpi == EPI_STORE || K >= 1024)))
         return launch_gemm_as<kAMn, kBMn, kEpi, true>(A0, B0, A1, B1, C0, C1, C2, C3, c_rows, ldc, M, N, K, st, nbatch, has_res);
     return launch_gemm_as<kAMn, kBMn, kEpi, false>(A0, B0, A1, B1, C0, C1, C2, C3, c_rows, ldc, M, N, K, st, nbatch, has_res);
 }
