@@ -25,12 +25,17 @@
  *    d fastest, 16-byte aligned; element type bfloat16 (MOA_BF16) or float
  *    (MOA_F32) per desc->dtype.  L is a DEVICE pointer to float [B,H,n].
  *  - The caller owns every buffer, workspace included.  The library never
- *    allocates or frees device memory and keeps no per-call state.
+ *    allocates or frees device memory.  What it keeps between calls is small and
+ *    per process: a device status word (moa_last_device_status), the event records
+ *    of moa_profile_*, a launch counter and per-device attribute caches.
  *  - Calls enqueue kernels on `stream` (a cudaStream_t passed as void*; NULL is
  *    the legacy default stream) and return without synchronising the host.
  *  - Outputs are overwritten, never accumulated into.
  *  - Errors are reported only through the returned moa_status; the library does
- *    not abort or throw.  On any error nothing has been enqueued.
+ *    not abort or throw.  Argument, workspace, scratch-limit and architecture errors
+ *    are found before anything is enqueued.  MOA_ERR_CUDA can come from a later
+ *    launch, clear or descriptor encode of a call that consists of several: kernels
+ *    enqueued before it still run, and the outputs and the workspace are undefined.
  *  - Supported: d in {64, 128} everywhere; on the bf16 tensor-core kernels also every
  *    other multiple of 8 up to 128 (d = 96, 80, 32, ...: the head runs in the 64- or
  *    128-column kernel, TMA zero-fills the missing columns on load and drops them on
@@ -152,12 +157,24 @@ moa_status moa_attn_bwd(const moa_attn_desc *desc,
  *  - All calls on a device share the one array, and it keeps whatever the previous
  *    call left in it; the parts that must start from zero are cleared on the stream at
  *    the start of every call.  Two calls that can overlap on the GPU (different
- *    streams, or different host threads) therefore race on it: serialise them. */
+ *    streams, or different host threads) therefore race on it: serialise them.
+ *  - Device ordinals 0..63 are supported (the per-device address cache); beyond that the
+ *    call returns MOA_ERR_CUDA. */
 #define MOA_STATIC_SCRATCH_BYTES (16u << 20)
 moa_status moa_attn_bwd_static_scratch(const moa_attn_desc *desc,
                                        const void *Q, const void *K, const void *V,
                                        const void *O, const float *L, const void *dO,
                                        void *dQ, void *dK, void *dV, void *stream);
+
+/* Which form of the bf16 tensor-core backward runs for head dimensions 72..128: mode 0 (the default) one CTA
+ * per key tile; mode 1 pairs of CTAs (two adjacent key tiles per cluster, tcgen05 cta_group::2, the dS tile
+ * halves exchanged through the cluster's shared memory); mode < 0 only queries.  Returns the mode in force
+ * before the call.  Process-wide; the environment variable MOA_BWD_PAIR=1 sets the initial mode to 1.
+ * Both forms compute the same dK and dV bit for bit (one writer per element, the paper's Sec. 4 fix, same
+ * summation order); dQ differs by the order of its fp32 additions.  The paired form halves the operand
+ * traffic per SM but measured slower (its hand-offs cross SMs); it is kept for that comparison.  No passage
+ * of the paper corresponds to the switch. */
+int moa_bwd_pair_mode(int mode);
 
 /* Fused forward+backward (the paper's Algorithm 2 as one library call): several
  * launches on one stream, no n x n array in memory.  Reads Q,K,V,dO; writes O, L,

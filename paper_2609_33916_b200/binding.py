@@ -30,7 +30,7 @@ EXPORTS = (
     "moa_decode_workspace_bytes", "moa_decode_attn",
     "moa_rmsnorm_workspace_bytes", "moa_rmsnorm_fwd", "moa_rmsnorm_bwd",
     "moa_gated_mlp_fwd", "moa_gated_mlp_workspace_bytes", "moa_gated_mlp_bwd", "moa_gemm",
-    "moa_selftest_expired_wait",
+    "moa_selftest_expired_wait", "moa_bwd_pair_mode",
 )
 
 
@@ -121,6 +121,8 @@ def lib() -> ctypes.CDLL:
         L.moa_last_device_status.argtypes = [vp]
         L.moa_selftest_expired_wait.restype = ctypes.c_int
         L.moa_selftest_expired_wait.argtypes = [ctypes.c_longlong, vp]
+        L.moa_bwd_pair_mode.restype = ctypes.c_int
+        L.moa_bwd_pair_mode.argtypes = [ctypes.c_int]
         L.moa_launch_count.restype = ctypes.c_uint64
         L.moa_status_string.restype = ctypes.c_char_p
         L.moa_status_string.argtypes = [ctypes.c_int]
@@ -252,6 +254,12 @@ def moa_rmsnorm_bwd(desc, x, g, r, dy, dx, dg, ws=None, stream=None, ws_bytes=No
     if check and s != MOA_OK:
         raise MoaError(s, "moa_rmsnorm_bwd")
     return s
+
+
+def moa_bwd_pair_mode(mode: int = -1) -> int:
+    """Sets (mode 0 or 1) or queries (mode < 0) whether the tensor-core backward runs on CTA pairs; returns the
+    mode in force before the call."""
+    return int(lib().moa_bwd_pair_mode(int(mode)))
 
 
 def moa_selftest_expired_wait(limit_cycles=1000000, stream=None) -> int:

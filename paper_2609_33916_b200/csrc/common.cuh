@@ -135,6 +135,14 @@ cudaError_t tc_bwd_kv(const Problem &p, const void *Q, const void *K, const void
                       const float *Lp, const float *Dp, void *dK, void *dV, float *dQacc, int dq_bulk,
                       cudaStream_t st);   // dq_bulk: TMA bulk add-reduce instead of red.global (d = 128 only)
 
+// The same on pairs of CTAs (tc_bwd_pair.cu; the 128-column kernel only), and whether tc_bwd_kv hands such
+// problems to it (moa_bwd_pair_mode; environment variable MOA_BWD_PAIR=1 for the initial mode; default: no)
+cudaError_t tc_bwd_kv_pair(const Problem &p, const void *Q, const void *K, const void *V, const void *dO,
+                           const float *Lp, const float *Dp, void *dK, void *dV, float *dQacc, int dq_bulk,
+                           cudaStream_t st);
+bool bwd_pair_enabled();
+int bwd_pair_mode(int set);      // set < 0: query; returns the mode in force before the call
+
 // atomic-free query-parallel dQ pass on the tensor cores (tc_dq.cu); writes dQ (bf16) directly
 cudaError_t tc_bwd_dq(const Problem &p, const void *Q, const void *K, const void *V, const void *dO,
                       const float *Lp, const float *Dp, void *dQ, cudaStream_t st);

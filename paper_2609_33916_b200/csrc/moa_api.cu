@@ -551,6 +551,8 @@ moa_status moa_profile_read(moa_profile *out)
     return rc;
 }
 
+int moa_bwd_pair_mode(int mode) { return bwd_pair_mode(mode); }
+
 uint64_t moa_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char *moa_status_string(moa_status s)

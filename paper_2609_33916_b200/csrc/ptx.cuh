@@ -1,6 +1,8 @@
 // Thin inline-PTX wrappers for the sm_100a features the tensor-core kernels use:
-// mbarrier, TMA (cp.async.bulk.tensor, no multicast anywhere), tcgen05 (TMEM
-// allocation, UMMA, commit, ld/st) and the shared-memory / instruction descriptors.
+// mbarrier, TMA (cp.async.bulk.tensor; no load is multicast: every CTA fetches its own tiles),
+// tcgen05 (TMEM allocation, UMMA, commit, ld/st) and the shared-memory / instruction
+// descriptors.  The one multicast form in here is the tcgen05.commit of a CTA pair, which is an
+// mbarrier arrival in both CTAs of one cluster on one GPU, not a copy.
 #pragma once
 #include <cuda_runtime.h>
 #include <cuda.h>
@@ -327,6 +329,91 @@ __device__ __forceinline__ void umma_ss2_pair(uint32_t d_tmem, uint32_t a_lo, ui
         ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(kAccumulate ? 1 : 0)
         : "memory");
 }
+template <bool kAccumulate>
+__device__ __forceinline__ void umma_ts2_pair(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(kAccumulate ? 1 : 0)
+        : "memory");
+}
+// 4-D tiled load of a CTA of a pair: the bytes complete on the barrier named by its shared::cluster address
+// (a barrier of either CTA of the pair); no multicast, each CTA fetches what it stages itself
+__device__ __forceinline__ void tma_load_4d_pair(void *dst, const CUtensorMap *m, uint32_t bar_cluster_addr, int x, int y,
+                                                 int z, int w)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster_addr), "r"(x), "r"(y), "r"(z), "r"(w)
+        : "memory");
+}
+// Arrival on a barrier of any CTA of the cluster that publishes this thread's earlier writes (also those to the other
+// CTA's shared memory) to whoever waits on it with cluster scope
+__device__ __forceinline__ void mbar_arrive_release_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(MOA_SUSPEND_HINT_NS)
+        : "memory");
+    return ok != 0;
+}
+// mbar_wait for a barrier of this CTA on which threads of the other CTA of the pair arrive (cluster-scope acquire)
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                                  unsigned int *status, uint32_t code, long long limit = kWaitCycles)
+{
+    if (mbar_test_wait(bar, parity) && mbar_try_wait_cluster(bar, parity)) return true;
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t spins = 0;
+    while (!mbar_try_wait_cluster(bar, parity)) {
+        if ((++spins & 7u) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > limit) {
+                *abort_flag = 1;
+                if (status) atomicCAS(status, 0u, code);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+// Arrival on a barrier of the other CTA of the cluster with no ordering of this thread's other memory accesses (a
+// cluster-scope release costs about a thousand cycles; what such an arrival announces here -- TMEM contents after
+// tcgen05.wait, shared memory after a proxy fence -- is complete before the instruction is issued)
+__device__ __forceinline__ void mbar_arrive_relaxed_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Bulk copy of `bytes` contiguous bytes from this CTA's shared memory into the shared memory of another CTA of the
+// cluster; the bytes are counted on an mbarrier of the receiving CTA when they have landed (both destination addresses
+// from mapa_u32; 16-byte aligned addresses and size).  The whole transfer runs in the asynchronous proxy, like a TMA load.
+__device__ __forceinline__ void bulk_copy_to_cluster(uint32_t dst_cluster_addr, const void *src, uint32_t bytes,
+                                                     uint32_t bar_cluster_addr)
+{
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_cluster_addr), "r"(smem_u32(src)), "r"(bytes), "r"(bar_cluster_addr)
+                 : "memory");
+}
+// 16-byte store into the shared memory of a CTA of the cluster (address from mapa_u32)
+__device__ __forceinline__ void st_cluster_v4(uint32_t cluster_addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "r"(a), "r"(b), "r"(c), "r"(d)
+                 : "memory");
+}
+// generic-proxy writes (also those to another CTA's shared memory) ordered before later async-proxy reads
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
 // Arrive, on the barrier at this offset in BOTH CTAs of the pair, when all previously issued UMMAs have completed.
 __device__ __forceinline__ void umma_commit_pair(uint64_t *bar)
 {

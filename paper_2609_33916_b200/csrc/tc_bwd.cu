@@ -679,6 +679,7 @@ cudaError_t tc_bwd_kv(const Problem &p, const void *Q, const void *K, const void
 {
     if (p.d < 8 || p.d > 128 || p.d % 8) return cudaErrorInvalidValue;
     const int D = kernel_d(p.d);     // dQacc rows are D floats wide
+    if (D == 128 && bwd_pair_enabled()) return tc_bwd_kv_pair(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, dq_bulk, st);
     if (D == 64 && !dq_bulk) return launch_bwd<64, false>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
     if (D == 128 && !dq_bulk) return launch_bwd<128, false>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
     if (D == 128 && dq_bulk) return launch_bwd<128, true>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
