@@ -333,6 +333,10 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 umma_commit(bars + B_DP);
             }
             if (!mbar_wait(bars + B_P, it & 1, abortp, status, ERR_PDS)) break;
+            // (the probe for S(i+1)'s operand sits here, not between dV and S: a thread that reads shared memory between
+            // two UMMAs first waits for the ones it issued to complete, and the pipe then idles until the next one
+            // arrives -- 150-185 cycles per such point in a replay of this loop's issue pattern)
+            if (it + 1 < niter && !mbar_wait(bars + B_QFULL + ((it + 1) & 1), ((it + 1) >> 1) & 1, abortp, status, ERR_FULL)) break;
             tc_fence_after();
             if (lane == 0) {
                 // 16 queries per step; the very first UMMA of the CTA overwrites the accumulator
@@ -345,12 +349,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 }
                 umma_commit(bars + B_DOEMPTY + sdo);
             }
-            if (it + 1 < niter) {
-                const int s1 = (it + 1) & 1;
-                if (!mbar_wait(bars + B_QFULL + s1, ((it + 1) >> 1) & 1, abortp, status, ERR_FULL)) break;
-                tc_fence_after();
-                if (lane == 0) issue_S(q_km0 + s1 * kSlot);
-                }
+            if (it + 1 < niter) issue_S(q_km0 + ((it + 1) & 1) * kSlot);
             if (!mbar_wait(bars + B_DS, it & 1, abortp, status, ERR_PDS)) break;
             if (!kAliasDQ && !skip_dq && it > 0 && !mbar_wait(bars + B_DQR, (it - 1) & 1, abortp, status, ERR_DQR)) break;
             tc_fence_after();
