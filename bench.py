@@ -7,10 +7,13 @@
 A step is one moa_attn_fused_fwd_bwd call (forward, preprocess, backward, dQ
 conversion) over one batch of synthetic bf16 inputs.  The metric is model
 TFLOP/s: 4 n^2 d forward + 10 n^2 d backward per head, halved when causal.
-With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank
-runs the whole workload on its own GPU -- (batch, head) pairs are independent,
-so there is no collective on the data path -- and the value is the sum over
-ranks divided by the slowest rank's time (weak scaling).
+With N > 1 (launched by torch.distributed.run, one rank per GPU) there are two modes, neither with a
+collective on the data path, because (batch, head) pairs are independent:
+  --shard replicas (default)  every rank runs the whole workload on its own GPU; the value is the sum
+                              over ranks divided by the slowest rank's time ("scaling": "weak")
+  --shard heads               the workload's B*H heads are partitioned into contiguous blocks, one per
+                              rank (config 4: 16 heads -> 2 per GPU on 8); total work is fixed
+                              ("scaling": "strong")
 
 Prints ONE JSON line on rank 0.
 """
@@ -42,6 +45,16 @@ def load_peaks():
         return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
     except Exception:
         return dict(FALLBACK_PEAKS), "fallback"
+
+
+def load_traffic_record(kernel: str):
+    """The committed record of the last ncu DRAM-traffic capture of `kernel` (profiles/traffic.json, written by
+    `python -m paper_2609_33916_b200.profile_summary`), or None."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
+            return json.load(f).get(kernel)
+    except Exception:
+        return None
 
 
 # ------------------------------------------------------------------- clock sampling
@@ -155,6 +168,21 @@ def time_oracle_sample(w, budget_s: float):
                                              f"8nd flop per row credited")
 
 
+def time_oracle_one_thread(w, budget_s: float):
+    """The same sample with OMP_NUM_THREADS=1, in a child process (the thread count is read when the oracle's library
+    is loaded).  The paper found that over-threading small n costs its CPU kernels up to 14.5x (Sec. 3, CPU scaling),
+    so for the small configurations both counts are timed and the better one is named."""
+    import subprocess
+    code = ("import json, sys; sys.path.insert(0, %r); import bench; from paper_2609_33916_b200 import inputs as mi; "
+            "v, dt, c, d = bench.time_oracle_sample(mi.CONFIGS[%r], %f); print(json.dumps(dict(value=v, seconds=dt, cores=c, sample=d)))"
+            % (ROOT, w.name, budget_s))
+    r = subprocess.run([sys.executable, "-c", code], env=dict(os.environ, OMP_NUM_THREADS="1"), capture_output=True,
+                       text=True, timeout=600)
+    if r.returncode != 0:
+        return None
+    return json.loads(r.stdout.strip().splitlines()[-1])
+
+
 def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -189,7 +217,81 @@ def workload_config(w, args):
     return {"workload": w.name, "B": w.B, "H": w.H, "n": w.n, "d": w.d, "causal": w.causal,
             "scale": "1/sqrt(d)", "dq_mode": args.dq_mode, "path": args.path, "materialize": getattr(args, "materialize", 0),
             "l2": "inputs+outputs per step exceed the 126 MB L2; no explicit flush",
-            "parallelism": f"independent (b,h) shards x{args.gpus}"}
+            "parallelism": (f"{w.B * w.H} heads partitioned over {args.gpus} ranks" if getattr(args, "shard", "replicas") == "heads" and args.gpus > 1
+                            else f"independent replicas x{args.gpus}")}
+
+
+def rank_plan(w, world: int, rank: int, shard: str, hkv: int = 0) -> dict:
+    """What one rank computes.  replicas: the whole workload.  heads: a contiguous block of the flattened (batch, head)
+    pairs -- heads are independent, so the block is handed to the library as B = 1, H = count (with shared K/V heads
+    the unit is a K/V head with its group of query heads)."""
+    from paper_2609_33916_b200 import sharding
+    per_head = w.model_flops / (w.B * w.H)
+    if shard == "replicas" or world == 1:
+        return {"B": w.B, "H": w.H, "H_kv": hkv, "first_head": 0, "heads": w.B * w.H, "flops": w.model_flops}
+    if shard != "heads":
+        raise ValueError(f"unknown shard mode {shard}")
+    group = (w.H // hkv) if hkv else 1
+    units = w.B * w.H // group                   # K/V heads (or plain heads) to hand out
+    first, count = sharding.head_shard(units, world, rank)
+    return {"B": 1, "H": count * group, "H_kv": count if hkv else 0, "first_head": first * group, "heads": count * group,
+            "flops": per_head * count * group}
+
+
+def job_value(flops_per_rank: list, ms_slowest: float) -> float:
+    """Whole-job TFLOP/s: the flops all ranks processed per step over the slowest rank's time per step."""
+    from paper_2609_33916_b200 import sharding
+    return sharding.aggregate_rate(flops_per_rank, [ms_slowest * 1e-3] * len(flops_per_rank)) / 1e12
+
+
+def run_stub(args, w):
+    """Testing aid (--stub-ms-per-tflop): the rank and shard bookkeeping of a multi-rank run -- process group, shard
+    plan, barriers, max-over-ranks timing, whole-job value, the JSON line -- with the library call replaced by a
+    sleep proportional to the rank's flops.  Needs no GPU; run with --dist-backend gloo."""
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    dist = None
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+        dist.init_process_group(args.dist_backend)
+    plan = rank_plan(w, world, rank, args.shard, args.hkv)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+
+    def gather(x: float) -> list:
+        if dist is None:
+            return [x]
+        import torch
+        t = [torch.zeros(1, dtype=torch.float64) for _ in range(world)]
+        dist.all_gather(t, torch.tensor([x], dtype=torch.float64))
+        return [float(v.item()) for v in t]
+
+    def step():
+        time.sleep(plan["flops"] / 1e12 * args.stub_ms_per_tflop * 1e-3)
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    ms_mine = (time.perf_counter() - t0) * 1e3 / args.steps
+    barrier()
+    ms_all, flops_all = gather(ms_mine), gather(plan["flops"])
+    line = {"metric": METRIC, "value": job_value(flops_all, max(ms_all)), "unit": "TFLOP/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": max(ms_all), "higher_is_better": True,
+            "scaling": "strong" if (args.shard == "heads" and world > 1) else "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic", "config": workload_config(w, args), "stub": True,
+            "shards": {"heads_per_rank": [int(round(f / (w.model_flops / (w.B * w.H)))) for f in flops_all],
+                       "first_head_rank": plan["first_head"]}}
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
 
 
 # ---------------------------------------------------------------------------- decode
@@ -720,6 +822,10 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="config-5 strategy sweep (study table, not the contract line)")
     ap.add_argument("--sweep-sizes", default="")
     ap.add_argument("--dist-backend", default="nccl", help="control-plane backend for N > 1 (nccl; gloo for tests)")
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "heads"],
+                    help="N > 1: every rank runs the whole workload (weak), or the heads are partitioned over the ranks (strong)")
+    ap.add_argument("--stub-ms-per-tflop", type=float, default=0.0,
+                    help="testing aid: replace the library call by a sleep of this many ms per TFLOP (no GPU needed)")
     ap.add_argument("--all-ranks-on-device0", action="store_true",
                     help="testing aid: every rank uses cuda:0 (ranks never wait on one another's kernels)")
     args = ap.parse_args()
@@ -736,6 +842,8 @@ def main():
         return run_reference(args, w)
     if args.sweep:
         return run_sweep(args)
+    if args.stub_ms_per_tflop > 0:
+        return run_stub(args, w)
 
     import torch
     from paper_2609_33916_b200 import binding as mb
@@ -763,11 +871,15 @@ def main():
     mb.lib()
     peaks, peaks_kind = load_peaks()
 
-    B, H, n, d = w.B, w.H, w.n, w.d
+    plan = rank_plan(w, world, rank, args.shard, args.hkv)      # this rank's share: everything, or a block of heads
+    if plan["heads"] == 0:
+        raise SystemExit(f"rank {rank}: more ranks than heads to hand out ({w.B * w.H} heads, {world} ranks)")
+    B, H, n, d = plan["B"], plan["H"], w.n, w.d
+    hkv = plan["H_kv"]
     desc = mb.make_desc(B, H, n, d, w.causal, w.scale, mb.MOA_BF16, args.dq_mode, args.materialize, args.path,
-                        H_kv=args.hkv, layout=args.layout)
+                        H_kv=hkv, layout=args.layout)
     shape = (B, n, H, d) if args.layout else (B, H, n, d)
-    kv_shape = (B, n, args.hkv or H, d) if args.layout else (B, args.hkv or H, n, d)       # K, V, dK, dV
+    kv_shape = (B, n, hkv or H, d) if args.layout else (B, hkv or H, n, d)       # K, V, dK, dV
     shapes_in = (shape, kv_shape, kv_shape, shape)            # Q, K, V, dO
     shapes_out = (shape, shape, kv_shape, kv_shape)           # O, dQ, dK, dV
     base_mem = torch.cuda.memory_allocated()
@@ -824,6 +936,13 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
 
+    def sum_over_ranks(x: float) -> float:
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda" if args.dist_backend == "nccl" else "cpu")
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        return float(t.item())
+
     for _ in range(args.warmup):
         step()
     st = mb.moa_last_device_status(stream)
@@ -866,8 +985,9 @@ def main():
     # hiding in wall-clock timings (Sec. 3), so both are reported
     timing = {"ms_min": per_step[0], "ms_median": statistics.median(per_step), "ms_mean": ms_per_step,
               "wall_ms_per_step_incl_final_sync": wall_ms}
-    flops_step = w.model_flops
-    value = world * flops_step / (ms_per_step * 1e-3) / 1e12
+    flops_step = plan["flops"]                       # this rank's model flops per step
+    flops_job = sum_over_ranks(flops_step)           # all ranks'
+    value = flops_job / (ms_per_step * 1e-3) / 1e12
     peak_bytes = torch.cuda.max_memory_allocated() - base_mem
 
     # ---- end to end: pinned host inputs -> device, call, results -> pinned host ----
@@ -924,7 +1044,7 @@ def main():
     t1e.record(s_down)
     barrier()
     e2e_ms = max_over_ranks(t0e.elapsed_time(t1e)) / e2e_steps
-    e2e_value = world * flops_step / (e2e_ms * 1e-3) / 1e12
+    e2e_value = flops_job / (e2e_ms * 1e-3) / 1e12
     st = mb.moa_last_device_status(stream)
     if st != mb.MOA_OK:
         raise SystemExit(f"device status: {mb.status_string(st)}")
@@ -937,31 +1057,59 @@ def main():
     if prof["bwd_dq"][1] > 0:   # separate pass: dQ's 2 n^2 d moves to that kernel (its recompute is not credited)
         alg_flops["bwd_kv"] = 8.0 * heads * n * n * d * causal_f
         alg_flops["bwd_dq"] = 2.0 * heads * n * n * d * causal_f
+    # algorithmic HBM bytes per launch (bf16 tensors read and written once, fp32 row vectors, the fp32 dQ accumulator
+    # added into and read back by the conversion): what the method must move, for comparison with measured traffic
+    kvh = (hkv or H) * B
+    alg_bytes = {"fwd": 2.0 * n * d * (2 * heads + 2 * kvh) + 4.0 * heads * n,
+                 "bwd_kv": 2.0 * n * d * (2 * heads + 4 * kvh) + 8.0 * heads * n + 4.0 * heads * n * d,
+                 "bwd_dq": 2.0 * n * d * (3 * heads + 2 * kvh) + 8.0 * heads * n}
     dominant = max(("fwd", "bwd_kv", "bwd_dq"), key=lambda k: prof[k][0])
     dom_ms = prof[dominant][0] / max(1, prof[dominant][1])
     achieved = alg_flops[dominant] / (dom_ms * 1e-3) / 1e12 if dom_ms > 0 else None
-    tc_path = args.path in (0, 2)
-    peak = peaks["bf16_tflops_sustained"]
-    # DRAM bytes per launch of the backward kernel: ncu capture of a small case (B1 H8 n8192 d128:
-    # 123.9 MB read+written over 65536 tokens), scaled by tokens -- traffic is linear in B*H*n
-    traffic = 123.9e6 / 65536.0 * heads * n if (dominant == "bwd_kv" and d == 128) else None
+    # Denominator: MEASURED_PEAKS holds a burst figure (a kernel timed alone or in a sub-second run, clocks near
+    # their maximum) and a sustained one (a seconds-long loop under the power cap).  The one that applies follows
+    # from the timed region's own length; both fractions are carried.
+    long_run = ms_total >= 1000.0
+    peak_name = "bf16_tflops_sustained" if long_run else "bf16_tflops"
+    peak = peaks[peak_name]
+    # DRAM traffic of the dominant kernel: from the committed record of an ncu capture (profiles/traffic.json), for
+    # the kernel family that was captured only, scaled by tokens (traffic is linear in B*H*n); null otherwise
+    traffic, traffic_source = None, None
+    rec = load_traffic_record(dominant)
+    fam = rec and rec.get("family", {})
+    if rec and dominant == "bwd_kv" and d == fam.get("d") and bool(w.causal) == bool(fam.get("causal")) and \
+            not hkv and not args.layout and not args.materialize and args.path in (0, 2) and \
+            (args.dq_mode or 2) == fam.get("dq_mode") and not mb.moa_bwd_pair_mode(-1):
+        traffic = rec["dram_bytes_per_launch"] / rec["tokens"] * heads * n
+        traffic_source = (f"extrapolated from an ncu capture of {rec['case']} ({rec['dram_bytes_per_launch'] / 1e6:.1f} MB "
+                          f"read+written per launch), scaled by tokens")
     roofline = {"bound": "tensor", "kernel": dominant, "achieved": achieved, "peak": peak,
-                "unit": "TFLOP/s", "frac": (achieved / peak) if achieved else None, "traffic": traffic,
-                "traffic_source": "ncu dram__bytes_read+write of a smaller case, scaled by tokens" if traffic else None,
-                "peak_source": f"{peaks_kind} bf16_tflops_sustained (kernel timed inside a long step)",
+                "unit": "TFLOP/s", "frac": (achieved / peak) if achieved else None,
+                "frac_of_burst": (achieved / peaks["bf16_tflops"]) if achieved else None,
+                "frac_of_sustained": (achieved / peaks["bf16_tflops_sustained"]) if achieved else None,
+                "traffic": traffic, "traffic_source": traffic_source,
+                "algorithmic_hbm_bytes": alg_bytes.get(dominant),
+                "peak_source": f"{peaks_kind} {peak_name}: the timed region ran {ms_total / 1e3:.2f} s "
+                               f"({'a second or more: sustained' if long_run else 'under a second: burst'})",
                 "kernel_ms": dom_ms,
                 "per_kernel_ms": {k: (v[0] / max(1, v[1]), v[1]) for k, v in prof.items() if v[1]}}
+    # clock-normalised figure: ms x median SM MHz under load (runs at different power-capped clocks compare on it)
+    clk = sampler.summary()
+    if clk.get("sm_mhz"):
+        timing["ms_times_sm_mhz"] = ms_per_step * clk["sm_mhz"]
+        timing["value_at_max_clock"] = value * clk["sm_max_mhz"] / clk["sm_mhz"] if clk.get("sm_max_mhz") else None
 
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "strong" if (args.shard == "heads" and world > 1) else "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(w, args),
         "pct_of_peak": {"of_measured_burst": 100 * value / world / peaks["bf16_tflops"],
                         "of_measured_sustained": 100 * value / world / peaks["bf16_tflops_sustained"],
                         "of_nominal_2250": 100 * value / world / NOMINAL_BF16_TFLOPS, "peaks": peaks_kind},
         "hbm_bytes": {"resident_inputs_outputs_workspace": resident_bytes, "peak_allocated": peak_bytes,
                       "workspace": ws_bytes, "one_nxn_fp32_array_all_heads_not_allocated": 4 * heads * n * n},
-        "clocks": sampler.summary(),
+        "clocks": clk,
         "timing": timing,
         "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms, "how": "pinned host buffers; upload, kernels and download on three streams, "
@@ -981,6 +1129,13 @@ def main():
         v, dt, cores, desc_s = time_oracle_sample(w, 20.0)
         line["cpu_baseline"] = {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
                                 "sample": desc_s, "seconds": dt}
+        if w.n <= 1024 and cores > 1:       # small n: one thread may beat all cores (the paper's over-threading finding)
+            one = time_oracle_one_thread(w, 10.0)
+            if one:
+                line["cpu_baseline"]["one_thread"] = one
+                if one["value"] > v:
+                    line["cpu_baseline"].update(value=one["value"], cores=1, sample=one["sample"], seconds=one["seconds"],
+                                                all_cores={"value": v, "cores": cores, "seconds": dt})
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:
