@@ -91,8 +91,14 @@ typedef enum { MOA_OP_FWD = 0, MOA_OP_BWD = 1, MOA_OP_FUSED = 2, MOA_OP_ROWPARAL
  * BHND: [B,H,n,d] contiguous (the layout of every named configuration).
  * BNHD: [B,n,H,d] contiguous (token-major, as projection GEMMs produce it); the tensor
  * maps take the strides, the arithmetic and the results are the same.  Tensor-core bf16
- * path only; other paths return MOA_ERR_UNSUPPORTED. */
-typedef enum { MOA_LAYOUT_BHND = 0, MOA_LAYOUT_BNHD = 1 } moa_layout;
+ * path only; other paths return MOA_ERR_UNSUPPORTED.
+ * STRIDED: every tensor is addressed through explicit strides (desc->q_stride, kv_stride, o_stride: elements
+ * between consecutive rows, heads and batches; the d elements of a row stay contiguous), e.g. the three
+ * thirds of a packed [B,n,3,H,d] projection output handed over as Q, K, V with row stride 3*H*d, so that one
+ * projection GEMM can feed the attention without a copy (the block composition the paper's full-block
+ * section times).  Every stride must be a multiple of 8 elements and at least d.  Same restriction
+ * to the tensor-core bf16 path. */
+typedef enum { MOA_LAYOUT_BHND = 0, MOA_LAYOUT_BNHD = 1, MOA_LAYOUT_STRIDED = 2 } moa_layout;
 
 typedef struct {
     int32_t B, H, n, d;
@@ -111,6 +117,12 @@ typedef struct {
                             dK, dV sum the contributions of the H / H_kv query heads of a group.
                             Tensor-core bf16 path only; other paths return MOA_ERR_UNSUPPORTED. */
     int32_t layout;      /* moa_layout                                                         */
+    int32_t reserved;    /* 0 (keeps the 64-bit fields below aligned)                          */
+    /* MOA_LAYOUT_STRIDED only (ignored otherwise): {row, head, batch} strides in elements of
+     * Q and dQ | K, V, dK and dV | O and dO.  L stays [B,H,n]. */
+    int64_t q_stride[3];
+    int64_t kv_stride[3];
+    int64_t o_stride[3];
 } moa_attn_desc;
 
 /* Bytes of caller-provided workspace `op` (a moa_op) needs for `desc`.  Returns 0

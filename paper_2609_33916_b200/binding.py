@@ -19,7 +19,7 @@ MOA_STATIC_SCRATCH_BYTES = 16 << 20
 MOA_BF16, MOA_F32 = 0, 1
 MOA_DQ_AUTO, MOA_DQ_RED, MOA_DQ_BULK_REDUCE, MOA_DQ_SEPARATE_PASS = 0, 1, 2, 3
 MOA_PATH_AUTO, MOA_PATH_SIMT, MOA_PATH_TC = 0, 1, 2
-MOA_LAYOUT_BHND, MOA_LAYOUT_BNHD = 0, 1
+MOA_LAYOUT_BHND, MOA_LAYOUT_BNHD, MOA_LAYOUT_STRIDED = 0, 1, 2
 MOA_OP_FWD, MOA_OP_BWD, MOA_OP_FUSED, MOA_OP_ROWPARALLEL = 0, 1, 2, 3
 
 #: every symbol include/moa_attn.h declares
@@ -38,7 +38,8 @@ class moa_attn_desc(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("n", ctypes.c_int32), ("d", ctypes.c_int32),
                 ("causal", ctypes.c_int32), ("scale", ctypes.c_float), ("dtype", ctypes.c_int32),
                 ("dq_mode", ctypes.c_int32), ("materialize", ctypes.c_int32), ("path", ctypes.c_int32),
-                ("H_kv", ctypes.c_int32), ("layout", ctypes.c_int32)]
+                ("H_kv", ctypes.c_int32), ("layout", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("q_stride", ctypes.c_int64 * 3), ("kv_stride", ctypes.c_int64 * 3), ("o_stride", ctypes.c_int64 * 3)]
 
 
 class moa_decode_desc(ctypes.Structure):
@@ -136,11 +137,23 @@ def lib() -> ctypes.CDLL:
 
 
 def make_desc(B, H, n, d, causal, scale, dtype=MOA_BF16, dq_mode=MOA_DQ_AUTO, materialize=0,
-              path=MOA_PATH_AUTO, H_kv=0, layout=0) -> moa_attn_desc:
+              path=MOA_PATH_AUTO, H_kv=0, layout=0, strides=None) -> moa_attn_desc:
     """H_kv: key/value heads (0 or H: one per query head; a divisor of H: grouped-query attention).
-    layout: MOA_LAYOUT_BHND (0) or MOA_LAYOUT_BNHD (1: tensors are [B,n,H,d] in memory)."""
-    return moa_attn_desc(int(B), int(H), int(n), int(d), int(bool(causal)), float(scale), int(dtype),
-                         int(dq_mode), int(materialize), int(path), int(H_kv), int(layout))
+    layout: MOA_LAYOUT_BHND (0), MOA_LAYOUT_BNHD (1: tensors are [B,n,H,d] in memory) or MOA_LAYOUT_STRIDED (2) with
+    strides = (q, kv, o), each a (row, head, batch) triple in elements."""
+    desc = moa_attn_desc(int(B), int(H), int(n), int(d), int(bool(causal)), float(scale), int(dtype),
+                         int(dq_mode), int(materialize), int(path), int(H_kv), int(layout), 0)
+    if strides is not None:
+        for name, tri in zip(("q_stride", "kv_stride", "o_stride"), strides):
+            setattr(desc, name, (ctypes.c_int64 * 3)(*[int(x) for x in tri]))
+    return desc
+
+
+def strides_of(t):
+    """(row, head, batch) element strides of a torch tensor viewed as [B, H, n, d] (any permutation or slice of a
+    larger buffer whose last dimension is contiguous)."""
+    assert t.dim() == 4 and t.stride(3) == 1
+    return (t.stride(2), t.stride(1), t.stride(0))
 
 
 def _ptr(x):

@@ -8,12 +8,39 @@
 
 namespace moa {
 
+// Where element (b, h, row, 0) of one of the caller's tensors lives: b * batch + h * head + row * row elements past
+// its base pointer (the d elements of a row are contiguous).
+struct Strides {
+    long long row, head, batch;
+    __host__ __device__ size_t at(long long b, long long h, long long r) const { return (size_t)(b * batch + h * head + r * row); }
+};
+
 struct Problem {
     int B, H, n, d;
     int causal;
     float scale;
     int Hkv = 0;                                   // key/value heads; 0: same as H
     int bnhd = 0;                                  // 1: the caller's tensors are [B,n,H,d] in memory (L stays [B,H,n])
+    // strides of the three tensor classes: Q, dQ | K, V, dK, dV | O, dO.  Filled by with_layout() from the fixed
+    // layouts, or taken from the descriptor (MOA_LAYOUT_STRIDED).
+    Strides sq{0, 0, 0}, skv{0, 0, 0}, so{0, 0, 0};
+    Problem &with_layout()
+    {
+        const long long hk = kv_heads();
+        if (bnhd) {
+            sq = so = Strides{(long long)H * d, d, (long long)n * H * d};
+            skv = Strides{hk * d, d, (long long)n * hk * d};
+        } else {
+            sq = so = Strides{d, (long long)n * d, (long long)H * n * d};
+            skv = Strides{d, (long long)n * d, hk * n * d};
+        }
+        return *this;
+    }
+    bool contiguous_bhnd() const     // every tensor is a plain [B,heads,n,d] array
+    {
+        return sq.row == d && sq.head == (long long)n * d && sq.batch == (long long)H * n * d && so.row == sq.row &&
+               so.head == sq.head && so.batch == sq.batch;
+    }
     int BH() const { return B * H; }
     int kv_heads() const { return Hkv > 0 ? Hkv : H; }
     int group() const { return H / kv_heads(); }    // query heads per key/value head
@@ -175,8 +202,8 @@ cudaError_t simt_bwd_dq(const Problem &p, int dtype, const void *Q, const void *
 // dst[i] = (bf16)(mul * src[i])
 cudaError_t convert_f32_to_bf16(const float *src, void *dst, size_t count, float mul, cudaStream_t st);
 // the same row by row: the accumulator is [B*H, n, src_ld] (src_ld >= d: the kernels' padded head
-// dimension), the destination [B,H,n,d] or, with bnhd, [B,n,H,d]
-cudaError_t convert_f32_to_bf16_rows(const float *src, int src_ld, void *dst, int B, int H, int n, int d, int bnhd,
+// dimension), the destination addressed through the strides `ds` of the caller's dQ
+cudaError_t convert_f32_to_bf16_rows(const float *src, int src_ld, void *dst, int B, int H, int n, int d, Strides ds,
                                      float mul, cudaStream_t st);
 
 }  // namespace moa

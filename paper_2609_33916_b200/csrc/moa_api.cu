@@ -6,6 +6,12 @@
 #include <mutex>
 #include <vector>
 
+#include <cstddef>
+
+// the layout the Python binding mirrors
+static_assert(sizeof(moa_attn_desc) == 128 && offsetof(moa_attn_desc, scale) == 20 && offsetof(moa_attn_desc, layout) == 44 &&
+              offsetof(moa_attn_desc, q_stride) == 56 && offsetof(moa_attn_desc, o_stride) == 104, "moa_attn_desc layout");
+
 namespace moa {
 
 static std::atomic<uint64_t> g_launches{0};
@@ -112,9 +118,17 @@ moa_status check_desc(const moa_attn_desc *d)
         !(d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && kernel_d(d->d) == 128 && d->scale > 0.f))
         return MOA_ERR_UNSUPPORTED;
     if (d->path == MOA_PATH_TC && !(d->scale > 0.f)) return MOA_ERR_UNSUPPORTED;   // non-positive scale: SIMT path only
-    if (d->layout != MOA_LAYOUT_BHND && d->layout != MOA_LAYOUT_BNHD) return MOA_ERR_INVALID_ARG;
-    // token-major tensors: tensor-core kernels only
-    if (d->layout == MOA_LAYOUT_BNHD &&
+    if (d->layout != MOA_LAYOUT_BHND && d->layout != MOA_LAYOUT_BNHD && d->layout != MOA_LAYOUT_STRIDED) return MOA_ERR_INVALID_ARG;
+    if (d->layout == MOA_LAYOUT_STRIDED) {
+        // rows of d contiguous elements; every stride positive, a multiple of 8 elements (16 bytes: what the
+        // tensor maps and the 16-byte row accesses need) and at least one row long
+        const int64_t *cls[3] = {d->q_stride, d->kv_stride, d->o_stride};
+        for (int c = 0; c < 3; ++c)
+            for (int k = 0; k < 3; ++k)
+                if (cls[c][k] < d->d || cls[c][k] % 8 != 0) return MOA_ERR_INVALID_ARG;
+    }
+    // token-major and strided tensors: tensor-core kernels only
+    if (d->layout != MOA_LAYOUT_BHND &&
         !(d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->scale > 0.f && !d->materialize))
         return MOA_ERR_UNSUPPORTED;
     if (d->H_kv < 0 || d->H_kv > d->H) return MOA_ERR_INVALID_ARG;
@@ -193,7 +207,14 @@ MatWorkspace mat_workspace(const moa_attn_desc *d, int op)
 
 Problem to_problem(const moa_attn_desc *d)
 {
-    return Problem{d->B, d->H, d->n, d->d, d->causal, d->scale, d->H_kv, d->layout == MOA_LAYOUT_BNHD ? 1 : 0};
+    Problem p{d->B, d->H, d->n, d->d, d->causal, d->scale, d->H_kv, d->layout == MOA_LAYOUT_BNHD ? 1 : 0};
+    p.with_layout();
+    if (d->layout == MOA_LAYOUT_STRIDED) {
+        p.sq = Strides{d->q_stride[0], d->q_stride[1], d->q_stride[2]};
+        p.skv = Strides{d->kv_stride[0], d->kv_stride[1], d->kv_stride[2]};
+        p.so = Strides{d->o_stride[0], d->o_stride[1], d->o_stride[2]};
+    }
+    return p;
 }
 
 // Materialising variant.  with_bwd = false: forward only (P^T is written and dropped).
@@ -211,6 +232,7 @@ moa_status run_materialized(const moa_attn_desc *d, const void *Q, const void *K
     for (int g0 = 0; g0 < heads; g0 += w.group) {
         const int g = heads - g0 < w.group ? heads - g0 : w.group;
         Problem p{1, g, d->n, d->d, d->causal, d->scale, 0};
+        p.with_layout();
         const char *q = (const char *)Q + g0 * hs, *k = (const char *)K + g0 * hs, *v = (const char *)V + g0 * hs;
         char *o = (char *)O + g0 * hs;
         float *l = L + (size_t)g0 * d->n;
@@ -257,7 +279,7 @@ moa_status run_bwd(const moa_attn_desc *d, const void *Q, const void *K, const v
         const int acc_ld = kernel_d(p.d);
         if (!prepared) MOA_TRY(cudaMemsetAsync(dQacc, 0, (size_t)p.BH() * p.n * acc_ld * sizeof(float), st));
         MOA_TRY(tc_bwd_kv(p, Q, K, V, dO, Lp, Dv, dK, dV, dQacc, mode == MOA_DQ_BULK_REDUCE, st));
-        if (p.bnhd || acc_ld != p.d) MOA_TRY(convert_f32_to_bf16_rows(dQacc, acc_ld, dQ, p.B, p.H, p.n, p.d, p.bnhd, p.scale, st));
+        if (!p.contiguous_bhnd() || acc_ld != p.d) MOA_TRY(convert_f32_to_bf16_rows(dQacc, acc_ld, dQ, p.B, p.H, p.n, p.d, p.sq, p.scale, st));
         else MOA_TRY(convert_f32_to_bf16(dQacc, dQ, elems, p.scale, st));
         return MOA_OK;
     }

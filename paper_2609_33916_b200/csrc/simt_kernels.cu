@@ -595,7 +595,7 @@ convert_kernel(const float *__restrict__ src, __nv_bfloat16 *__restrict__ dst, s
 // and / or a [B,n,H,d] destination; one thread converts four consecutive elements of a row.
 __global__ void __launch_bounds__(256)
 convert_rows_kernel(const float *__restrict__ src, int src_ld, __nv_bfloat16 *__restrict__ dst, size_t rows, int n, int H,
-                    int d, int bnhd, float mul)
+                    int d, Strides ds, float mul)
 {
     const int quads_per_row = d / 4;
     const size_t total = rows * (size_t)quads_per_row;
@@ -605,13 +605,13 @@ convert_rows_kernel(const float *__restrict__ src, int src_ld, __nv_bfloat16 *__
         const int c4 = (int)(q - row * quads_per_row);
         const size_t bh = row / (size_t)n;
         const size_t r = row - bh * (size_t)n, bb = bh / (size_t)H, h = bh - bb * (size_t)H;
-        const size_t drow = bnhd ? (bb * (size_t)n + r) * (size_t)H + h : row;
+        const size_t doff = ds.at((long long)bb, (long long)h, (long long)r);
         const float4 v = __ldcs(reinterpret_cast<const float4 *>(src + row * (size_t)src_ld) + c4);
         __nv_bfloat162 a = __floats2bfloat162_rn(v.x * mul, v.y * mul), b = __floats2bfloat162_rn(v.z * mul, v.w * mul);
         uint2 u;
         u.x = *reinterpret_cast<uint32_t *>(&a);
         u.y = *reinterpret_cast<uint32_t *>(&b);
-        *reinterpret_cast<uint2 *>(dst + drow * d + 4 * c4) = u;
+        *reinterpret_cast<uint2 *>(dst + doff + 4 * c4) = u;
     }
 }
 
@@ -748,7 +748,7 @@ cudaError_t convert_f32_to_bf16(const float *src, void *dst, size_t count, float
     return cudaGetLastError();
 }
 
-cudaError_t convert_f32_to_bf16_rows(const float *src, int src_ld, void *dst, int B, int H, int n, int d, int bnhd,
+cudaError_t convert_f32_to_bf16_rows(const float *src, int src_ld, void *dst, int B, int H, int n, int d, Strides ds,
                                      float mul, cudaStream_t st)
 {
     const size_t rows = (size_t)B * H * n, quads = rows * (size_t)(d / 4);
@@ -756,7 +756,7 @@ cudaError_t convert_f32_to_bf16_rows(const float *src, int src_ld, void *dst, in
     if (blocks < 1) blocks = 1;
     if (blocks > 148 * 16) blocks = 148 * 16;
     LaunchScope scope(MOA_KERNEL_CONVERT, st);
-    convert_rows_kernel<<<(unsigned)blocks, 256, 0, st>>>(src, src_ld, (__nv_bfloat16 *)dst, rows, n, H, d, bnhd, mul);
+    convert_rows_kernel<<<(unsigned)blocks, 256, 0, st>>>(src, src_ld, (__nv_bfloat16 *)dst, rows, n, H, d, ds, mul);
     return cudaGetLastError();
 }
 

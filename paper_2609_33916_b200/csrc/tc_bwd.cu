@@ -67,7 +67,7 @@ template <int D>
 __global__ void __launch_bounds__(256)
 bwd_preprocess_kernel(const __nv_bfloat16 *__restrict__ dO, const __nv_bfloat16 *__restrict__ O,
                       const float *__restrict__ L, float *__restrict__ Lp, float *__restrict__ Dp,
-                      int n, int n_pad, size_t padded_rows, int H, int bnhd, int d)
+                      int n, int n_pad, size_t padded_rows, int H, Strides so, int d)
 {
     // d <= D: the head dimension in memory (lanes past it contribute zeros)
     constexpr int kLanesPerRow = D / 8;
@@ -90,14 +90,11 @@ bwd_preprocess_kernel(const __nv_bfloat16 *__restrict__ dO, const __nv_bfloat16 
         lv[p] = 0.f;
         if (real[p]) {
             const size_t row = bh * (size_t)n + r;                      // row of L: always [B,H,n]
-            size_t trow = row;                                          // row of dO, O in the caller's layout
-            if (bnhd) {
-                const size_t bb = bh / (size_t)H;
-                trow = (bb * (size_t)n + r) * (size_t)H + (bh - bb * (size_t)H);
-            }
+            const size_t bb = bh / (size_t)H;
+            const size_t toff = so.at((long long)bb, (long long)(bh - bb * (size_t)H), r);      // first element of the row of dO, O
             if (8 * l < d) {
-                a[p] = __ldcs(reinterpret_cast<const uint4 *>(dO + trow * (size_t)d) + l);
-                b[p] = __ldcs(reinterpret_cast<const uint4 *>(O + trow * (size_t)d) + l);
+                a[p] = __ldcs(reinterpret_cast<const uint4 *>(dO + toff) + l);
+                b[p] = __ldcs(reinterpret_cast<const uint4 *>(O + toff) + l);
             }
             if (l == 0) lv[p] = L[row];
         }
@@ -616,15 +613,14 @@ cudaError_t launch_bwd_g(const Problem &p, const void *Q, const void *K, const v
 {
     CUtensorMap mq, mk, mv, mdo, mdq, mdk, mdv;
     const uint64_t heads = (uint64_t)p.BH();
-    const bool bnhd = p.bnhd != 0;
     const auto bf = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     // p.d <= D columns exist in memory: loads fill the rest of a box with zeros, stores drop it
-    if (!make_tensor_map_4d(&mq, Q, bf, 2, p.B, p.H, p.n, p.d, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mk, K, bf, 2, p.B, p.kv_heads(), p.n, p.d, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mv, V, bf, 2, p.B, p.kv_heads(), p.n, p.d, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mdo, dO, bf, 2, p.B, p.H, p.n, p.d, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mdk, dK, bf, 2, p.B, p.kv_heads(), p.n, p.d, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mdv, dV, bf, 2, p.B, p.kv_heads(), p.n, p.d, bnhd, 128, 64))
+    if (!make_tensor_map_4d_strided(&mq, Q, bf, 2, p.B, p.H, p.n, p.d, p.sq.row, p.sq.head, p.sq.batch, 128, 64) ||
+        !make_tensor_map_4d_strided(&mk, K, bf, 2, p.B, p.kv_heads(), p.n, p.d, p.skv.row, p.skv.head, p.skv.batch, 128, 64) ||
+        !make_tensor_map_4d_strided(&mv, V, bf, 2, p.B, p.kv_heads(), p.n, p.d, p.skv.row, p.skv.head, p.skv.batch, 128, 64) ||
+        !make_tensor_map_4d_strided(&mdo, dO, bf, 2, p.B, p.H, p.n, p.d, p.so.row, p.so.head, p.so.batch, 128, 64) ||
+        !make_tensor_map_4d_strided(&mdk, dK, bf, 2, p.B, p.kv_heads(), p.n, p.d, p.skv.row, p.skv.head, p.skv.batch, 128, 64) ||
+        !make_tensor_map_4d_strided(&mdv, dV, bf, 2, p.B, p.kv_heads(), p.n, p.d, p.skv.row, p.skv.head, p.skv.batch, 128, 64))
         return cudaErrorInvalidValue;
     // fp32 accumulator as [heads, n, D] with boxes of 32 rows x D floats (no swizzle); also encoded when unused
     if (!make_tensor_map_3d(&mdq, dQacc ? (const void *)dQacc : Q, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, heads, p.n, D, 32, D))
@@ -666,10 +662,10 @@ cudaError_t tc_bwd_preprocess(const Problem &p, const void *dO, const void *O, c
     LaunchScope scope(MOA_KERNEL_PREPROCESS, st);
     if (D == 64)
         bwd_preprocess_kernel<64><<<grid, wpb * 32, 0, st>>>((const __nv_bfloat16 *)dO, (const __nv_bfloat16 *)O, L,
-                                                             Lp, Dp, p.n, n_pad, rows, p.H, p.bnhd, p.d);
+                                                             Lp, Dp, p.n, n_pad, rows, p.H, p.so, p.d);
     else
         bwd_preprocess_kernel<128><<<grid, wpb * 32, 0, st>>>((const __nv_bfloat16 *)dO, (const __nv_bfloat16 *)O, L,
-                                                              Lp, Dp, p.n, n_pad, rows, p.H, p.bnhd, p.d);
+                                                              Lp, Dp, p.n, n_pad, rows, p.H, p.so, p.d);
     return cudaGetLastError();
 }
 

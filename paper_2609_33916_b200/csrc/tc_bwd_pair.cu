@@ -650,19 +650,18 @@ cudaError_t launch_pair(const Problem &p, const void *Q, const void *K, const vo
 {
     CUtensorMap mqr, mqc, mdor, mdoc, mk, mv, mkd, mdq, mdk, mdv;
     const uint64_t heads = (uint64_t)p.BH();
-    const bool bnhd = p.bnhd != 0;
     const auto bf = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     const int hkv = p.kv_heads();
     // p.d <= 128 columns exist in memory: loads fill the rest of a box with zeros, stores drop it
-    if (!make_tensor_map_4d(&mqr, Q, bf, 2, p.B, p.H, p.n, p.d, bnhd, 64, 64) ||
-        !make_tensor_map_4d(&mqc, Q, bf, 2, p.B, p.H, p.n, p.d, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mdor, dO, bf, 2, p.B, p.H, p.n, p.d, bnhd, 64, 64) ||
-        !make_tensor_map_4d(&mdoc, dO, bf, 2, p.B, p.H, p.n, p.d, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mk, K, bf, 2, p.B, hkv, p.n, p.d, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mv, V, bf, 2, p.B, hkv, p.n, p.d, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mkd, K, bf, 2, p.B, hkv, p.n, p.d, bnhd, 256, 64) ||
-        !make_tensor_map_4d(&mdk, dK, bf, 2, p.B, hkv, p.n, p.d, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mdv, dV, bf, 2, p.B, hkv, p.n, p.d, bnhd, 128, 64))
+    if (!make_tensor_map_4d_strided(&mqr, Q, bf, 2, p.B, p.H, p.n, p.d, p.sq.row, p.sq.head, p.sq.batch, 64, 64) ||
+        !make_tensor_map_4d_strided(&mqc, Q, bf, 2, p.B, p.H, p.n, p.d, p.sq.row, p.sq.head, p.sq.batch, 128, 64) ||
+        !make_tensor_map_4d_strided(&mdor, dO, bf, 2, p.B, p.H, p.n, p.d, p.so.row, p.so.head, p.so.batch, 64, 64) ||
+        !make_tensor_map_4d_strided(&mdoc, dO, bf, 2, p.B, p.H, p.n, p.d, p.so.row, p.so.head, p.so.batch, 128, 64) ||
+        !make_tensor_map_4d_strided(&mk, K, bf, 2, p.B, hkv, p.n, p.d, p.skv.row, p.skv.head, p.skv.batch, 128, 64) ||
+        !make_tensor_map_4d_strided(&mv, V, bf, 2, p.B, hkv, p.n, p.d, p.skv.row, p.skv.head, p.skv.batch, 128, 64) ||
+        !make_tensor_map_4d_strided(&mkd, K, bf, 2, p.B, hkv, p.n, p.d, p.skv.row, p.skv.head, p.skv.batch, 256, 64) ||
+        !make_tensor_map_4d_strided(&mdk, dK, bf, 2, p.B, hkv, p.n, p.d, p.skv.row, p.skv.head, p.skv.batch, 128, 64) ||
+        !make_tensor_map_4d_strided(&mdv, dV, bf, 2, p.B, hkv, p.n, p.d, p.skv.row, p.skv.head, p.skv.batch, 128, 64))
         return cudaErrorInvalidValue;
     // fp32 accumulator as [heads, n, 128] with boxes of 32 rows x 64 floats (no swizzle); also encoded when unused
     if (!make_tensor_map_3d(&mdq, dQacc ? (const void *)dQacc : Q, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, heads, p.n, D, 32, 64))

@@ -44,7 +44,7 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
              const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapdO,
              const float *__restrict__ Lp, const float *__restrict__ Dp, __nv_bfloat16 *__restrict__ dQ,
              int n, int n_pad, int causal, float scale, float scale_log2, int nqt, int hpg,
-             int group, int H, int bnhd, int d, unsigned int *status)
+             int group, int H, Strides sq, int d, unsigned int *status)
 {
     using SM = DqSmem<D>;
     constexpr int kBoxes = D / 64;
@@ -181,8 +181,7 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
         if (ok && mbar_wait(bars + B_DONE, 0, abortp, status, ERR_DONE)) {
             tc_fence_after();
             const int qrow = q0 + lane_row;
-            const size_t qrow_index = bnhd ? ((size_t)bb * n + qrow) * H + hq : (size_t)bh * n + qrow;   // row of dQ in the caller's layout
-            __nv_bfloat16 *outp = dQ + qrow_index * (size_t)d + (D / 2) * wg;   // d <= D columns exist in memory
+            __nv_bfloat16 *outp = dQ + sq.at(bb, hq, qrow) + (D / 2) * wg;   // row of dQ in the caller's layout; d <= D columns exist in memory
 #pragma unroll
             for (int c = 0; c < D / 2; c += 32) {
                 uint32_t r[32];
@@ -212,12 +211,11 @@ cudaError_t launch_dq(const Problem &p, const void *Q, const void *K, const void
                       const float *Lp, const float *Dp, void *dQ, cudaStream_t st)
 {
     CUtensorMap mq, mk, mv, mdo;
-    const bool bnhd = p.bnhd != 0;
     const auto bf = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
-    if (!make_tensor_map_4d(&mq, Q, bf, 2, p.B, p.H, p.n, p.d, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mk, K, bf, 2, p.B, p.kv_heads(), p.n, p.d, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mv, V, bf, 2, p.B, p.kv_heads(), p.n, p.d, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mdo, dO, bf, 2, p.B, p.H, p.n, p.d, bnhd, 128, 64))
+    if (!make_tensor_map_4d_strided(&mq, Q, bf, 2, p.B, p.H, p.n, p.d, p.sq.row, p.sq.head, p.sq.batch, 128, 64) ||
+        !make_tensor_map_4d_strided(&mk, K, bf, 2, p.B, p.kv_heads(), p.n, p.d, p.skv.row, p.skv.head, p.skv.batch, 128, 64) ||
+        !make_tensor_map_4d_strided(&mv, V, bf, 2, p.B, p.kv_heads(), p.n, p.d, p.skv.row, p.skv.head, p.skv.batch, 128, 64) ||
+        !make_tensor_map_4d_strided(&mdo, dO, bf, 2, p.B, p.H, p.n, p.d, p.so.row, p.so.head, p.so.batch, 128, 64))
         return cudaErrorInvalidValue;
     constexpr int kSmem = DqSmem<D>::kTotal;
     cudaError_t e = cudaFuncSetAttribute(tc_dq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
@@ -226,7 +224,7 @@ cudaError_t launch_dq(const Problem &p, const void *Q, const void *K, const void
     LaunchScope scope(MOA_KERNEL_BWD_DQ, st);
     tc_dq_kernel<D><<<(unsigned)(nqt * p.BH()), kThreads, kSmem, st>>>(
         mq, mk, mv, mdo, Lp, Dp, (__nv_bfloat16 *)dQ, p.n, nqt * 128, p.causal, p.scale, p.scale * kLog2e, nqt,
-        heads_per_group(p, nqt), p.group(), p.H, p.bnhd, p.d, device_status_ptr());
+        heads_per_group(p, nqt), p.group(), p.H, p.sq, p.d, device_status_ptr());
     return cudaGetLastError();
 }
 

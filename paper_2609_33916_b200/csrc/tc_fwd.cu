@@ -64,7 +64,8 @@ struct FwdSplit {
 struct FwdPrep {
     const __nv_bfloat16 *dO;
     float *Lp, *Dp;
-    int n_pad, bnhd;
+    int n_pad;
+    Strides so;          // where the rows of dO live
     int d;               // columns of a dO row in memory (<= D)
 };
 
@@ -242,8 +243,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         if (prep.dO != nullptr && row < n) {
             // fused call: the epilogue reads this thread's 128 bytes (D = 128) of its dO row; ask L2 for
             // them now so that the read at the end of the job does not wait on HBM
-            const size_t drow = prep.bnhd ? ((size_t)bb * n + row) * H + hq : (size_t)bh * n + row;
-            if ((D / 2) * h < prep.d) asm volatile("prefetch.global.L2 [%0];" ::"l"(prep.dO + drow * (size_t)prep.d + (D / 2) * h));
+            const size_t doff = prep.so.at(bb, hq, row);
+            if ((D / 2) * h < prep.d) asm volatile("prefetch.global.L2 [%0];" ::"l"(prep.dO + doff + (D / 2) * h));
         }
         // The exp2 phase of a tile is MUFU-bound and the rest of a tile's work (TMEM load, max,
         // hand-offs) is not: start the second warpgroup a few hundred cycles late, once, so that on
@@ -341,8 +342,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         uint4 dov[D / 16];
         const bool want_d = prep.dO != nullptr && row < n;
         if (want_d) {
-            const size_t drow = prep.bnhd ? ((size_t)bb * n + row) * H + hq : (size_t)bh * n + row;
-            const uint4 *src = reinterpret_cast<const uint4 *>(prep.dO + drow * (size_t)prep.d + (D / 2) * h);
+            const uint4 *src = reinterpret_cast<const uint4 *>(prep.dO + prep.so.at(bb, hq, row) + (D / 2) * h);
 #pragma unroll
             for (int k = 0; k < D / 16; ++k)      // columns past the head dimension count as zeros
                 dov[k] = (D / 2) * h + 8 * k < prep.d ? __ldg(src + k) : make_uint4(0u, 0u, 0u, 0u);
@@ -424,13 +424,12 @@ cudaError_t launch_fwd(const Problem &p, const void *Q, const void *K, const voi
 {
     constexpr int kSmem = 5 * 128 * D * 2 + 8 * (F_COUNT + 2) + 2 * 128 * 8 + 2 * 128 * 4;
     CUtensorMap mq, mk, mv, mo;
-    const bool bnhd = p.bnhd != 0;
     const auto bf = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     // p.d <= D columns exist in memory: loads fill the rest of a box with zeros, the store drops it
-    if (!make_tensor_map_4d(&mq, Q, bf, 2, p.B, p.H, p.n, p.d, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mk, K, bf, 2, p.B, p.kv_heads(), p.n, p.d, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mv, V, bf, 2, p.B, p.kv_heads(), p.n, p.d, bnhd, 128, 64) ||
-        !make_tensor_map_4d(&mo, O, bf, 2, p.B, p.H, p.n, p.d, bnhd, 128, 64))
+    if (!make_tensor_map_4d_strided(&mq, Q, bf, 2, p.B, p.H, p.n, p.d, p.sq.row, p.sq.head, p.sq.batch, 128, 64) ||
+        !make_tensor_map_4d_strided(&mk, K, bf, 2, p.B, p.kv_heads(), p.n, p.d, p.skv.row, p.skv.head, p.skv.batch, 128, 64) ||
+        !make_tensor_map_4d_strided(&mv, V, bf, 2, p.B, p.kv_heads(), p.n, p.d, p.skv.row, p.skv.head, p.skv.batch, 128, 64) ||
+        !make_tensor_map_4d_strided(&mo, O, bf, 2, p.B, p.H, p.n, p.d, p.so.row, p.so.head, p.so.batch, 128, 64))
         return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
@@ -439,7 +438,7 @@ cudaError_t launch_fwd(const Problem &p, const void *Q, const void *K, const voi
     tc_fwd_kernel<D><<<(unsigned)(nqt * p.BH()), kThreads, kSmem, st>>>(
         mq, mk, mv, mo, L, p.n, p.causal, p.scale * kLog2e, nqt, heads_per_group(p, nqt), p.group(), p.H,
         FwdSplit{p.n, 1, (p.n + BN - 1) / BN}, fb.zero_acc,
-        FwdPrep{(const __nv_bfloat16 *)fb.dO, fb.Lp, fb.Dp, nqt * BM, p.bnhd, p.d}, device_status_ptr());
+        FwdPrep{(const __nv_bfloat16 *)fb.dO, fb.Lp, fb.Dp, nqt * BM, p.so, p.d}, device_status_ptr());
     return cudaGetLastError();
 }
 

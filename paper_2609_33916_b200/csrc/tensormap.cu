@@ -59,6 +59,23 @@ bool make_tensor_map_4d(CUtensorMap *map, const void *base, CUtensorMapDataType 
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+bool make_tensor_map_4d_strided(CUtensorMap *map, const void *base, CUtensorMapDataType dt, int elem_bytes,
+                                uint64_t batch, uint64_t heads, uint64_t rows, uint64_t cols, long long row_stride,
+                                long long head_stride, long long batch_stride, uint32_t box_rows, uint32_t box_cols)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn || row_stride <= 0 || head_stride <= 0 || batch_stride <= 0) return false;
+    const uint64_t eb = (uint64_t)elem_bytes;
+    cuuint64_t gdim[4] = {cols, rows, heads, batch};
+    cuuint64_t gstride[3] = {(uint64_t)row_stride * eb, (uint64_t)head_stride * eb, (uint64_t)batch_stride * eb};
+    cuuint32_t box[4] = {box_cols, box_rows, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUtensorMapSwizzle sw =
+        (box_cols * (uint32_t)elem_bytes == 128) ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE;
+    return fn(map, dt, 4, const_cast<void *>(base), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool make_tensor_map_blocked(CUtensorMap *map, const void *base, CUtensorMapDataType dt, int elem_bytes,
                              uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t nblk)
 {

@@ -21,6 +21,13 @@ bool make_tensor_map_4d(CUtensorMap *map, const void *base, CUtensorMapDataType 
                         uint64_t batch, uint64_t heads, uint64_t rows, uint64_t cols, bool bnhd,
                         uint32_t box_rows, uint32_t box_cols);
 
+// The same with explicit strides in ELEMENTS between rows, heads and batches (each a multiple of 16 bytes; the cols
+// elements of a row are contiguous): any memory layout a caller's projection produces, e.g. the Q third of a packed
+// [B, n, 3, H, d] array.
+bool make_tensor_map_4d_strided(CUtensorMap *map, const void *base, CUtensorMapDataType dt, int elem_bytes,
+                                uint64_t batch, uint64_t heads, uint64_t rows, uint64_t cols, long long row_stride,
+                                long long head_stride, long long batch_stride, uint32_t box_rows, uint32_t box_cols);
+
 // Map over a [rows, cols] array (cols fastest, cols a multiple of 64) seen as (64 columns, rows, cols/64 column
 // blocks): one box of [nblk, box_rows, 64] lands in shared memory block by block -- nblk consecutive tiles of
 // box_rows rows x 128 bytes, 128-byte swizzle -- which is the layout an MN-major UMMA operand wants, fetched by one

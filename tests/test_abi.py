@@ -35,8 +35,10 @@ def test_version_and_strings(lib):
 
 
 def test_desc_struct_layout_matches_header():
-    assert ctypes.sizeof(mb.moa_attn_desc) == 48
+    assert ctypes.sizeof(mb.moa_attn_desc) == 128        # the same figures are static_asserts in the library
     assert mb.moa_attn_desc.scale.offset == 20
+    assert mb.moa_attn_desc.layout.offset == 44
+    assert mb.moa_attn_desc.q_stride.offset == 56 and mb.moa_attn_desc.o_stride.offset == 104
 
 
 def test_workspace_is_linear_in_n(lib):
@@ -197,3 +199,20 @@ def test_block_piece_argument_checks(lib):
         m_ = mb.make_mlp_desc(n, d, dff, dt)
         assert mb.moa_gated_mlp_fwd(m_, *([a] * 8), check=False) == want, (n, d, dff, dt)
         assert mb.moa_gated_mlp_workspace_bytes(m_) == 0
+
+
+def test_strided_layout_descriptor_checks(lib):
+    """MOA_LAYOUT_STRIDED: strides are checked before anything touches a device."""
+    good = ((384, 128, 384 * 300), (256, 128, 256 * 300), (384, 128, 384 * 300))
+    d = mb.make_desc(1, 3, 300, 128, True, 0.1, layout=mb.MOA_LAYOUT_STRIDED, strides=good)
+    assert mb.moa_attn_workspace_bytes(d, mb.MOA_OP_FUSED) > 0
+    a = 4096
+    for bad in (((100, 128, 115200),) * 3,            # row stride shorter than a row
+                ((132, 128, 115200),) * 3,            # not a multiple of 8 elements (16 bytes)
+                ((384, 0, 115200),) * 3):             # zero head stride
+        d = mb.make_desc(1, 3, 300, 128, True, 0.1, layout=mb.MOA_LAYOUT_STRIDED, strides=bad)
+        assert mb.moa_attn_workspace_bytes(d, mb.MOA_OP_FUSED) == 0
+        assert mb.moa_attn_fwd(d, a, a, a, a, a, check=False) == mb.MOA_ERR_INVALID_ARG
+    # the CUDA-core path has no strided form
+    d = mb.make_desc(1, 3, 300, 128, True, 0.1, mb.MOA_F32, layout=mb.MOA_LAYOUT_STRIDED, strides=good)
+    assert mb.moa_attn_fwd(d, a, a, a, a, a, check=False) == mb.MOA_ERR_UNSUPPORTED
