@@ -457,7 +457,8 @@ NormPlan norm_plan(int n, int d, bool bwd)
     p.R = p.kV == 1 ? 2 : (bwd && p.kV == 4) ? 2 : 1;
     const int lanes = kNormThreads / p.tpr;
     const long long blocks = ((long long)n + (long long)lanes * p.R - 1) / ((long long)lanes * p.R);
-    p.grid = (int)(blocks < 148 * 4 ? blocks : 148 * 4);
+    const long long cap = 4LL * device_info().sms;
+    p.grid = (int)(blocks < cap ? blocks : cap);
     if (p.grid < 1) p.grid = 1;
     return p;
 }
@@ -477,7 +478,8 @@ RingPlan ring_plan(int n, int d, bool bwd)
     p.m = 2048 / d < 1 ? 1 : 2048 / d;                                  // 32 KB per array and stage
     const long long rows_stage = (long long)kRingWarps * p.m;
     const long long stages = ((long long)n + rows_stage - 1) / rows_stage;
-    p.grid = (int)(stages < 148 ? stages : 148);
+    const long long sms = device_info().sms;
+    p.grid = (int)(stages < sms ? stages : sms);
     p.smem = (size_t)kRingStages * rows_stage * d * 2 * (bwd ? 2 : 1) + (size_t)d * 4 + 2 * kRingStages * 8 + 16;
     return p;
 }
@@ -506,8 +508,8 @@ cudaError_t launch_ring_kv(const RingPlan &p, const __nv_bfloat16 *x, const __nv
 
 }  // namespace
 
-// per-CTA partial sums of dg: at most 148 * 4 CTAs in either variant
-size_t rmsnorm_workspace_bytes(int n, int d) { (void)n; return (size_t)148 * 4 * d * sizeof(float); }
+// per-CTA partial sums of dg: at most four CTAs per SM in either variant
+size_t rmsnorm_workspace_bytes(int n, int d) { (void)n; return (size_t)device_info().sms * 4 * d * sizeof(float); }
 
 cudaError_t rmsnorm_fwd(int n, int d, float eps, const void *x, const void *g, void *y, float *r, cudaStream_t st)
 {

@@ -67,17 +67,28 @@ __device__ __forceinline__ void job_from_block(int block, int tiles, int heads, 
     bh = group * hpg + (r - t * cur);
 }
 
+// What the launch arithmetic needs to know about the current device, read once per device
+// (cudaDevAttrMultiProcessorCount, cudaDevAttrL2CacheSize); a B200 gives 148 SMs and 126 MB.
+struct DeviceInfo {
+    int sms;             // streaming multiprocessors
+    long long l2_bytes;  // L2 cache
+};
+const DeviceInfo &device_info();
+
 // Heads per group: enough jobs per group that its longest job (tiles iterations) is shorter than
-// the group's share of 148 SMs, and as many heads as keep Q, K, V, dO of a group within half of L2.
+// the group's share of the SMs, and as many heads as keep Q, K, V, dO of a group within half of L2.
 inline int heads_per_group(const Problem &p, int tiles)
 {
     if (!p.causal) return 1;
+    const DeviceInfo &dev = device_info();
     const long long per_head = 4LL * p.n * p.d * 2;
-    const long long fit = (64LL << 20) / (per_head > 0 ? per_head : 1);
-    long long g = (2 * 148 + tiles) / (tiles + 1);
+    const long long fit = (dev.l2_bytes / 2 + per_head / 2) / (per_head > 0 ? per_head : 1);     // to the nearest head
+    long long g = (2 * dev.sms + tiles) / (tiles + 1);
     if (fit > g) g = fit;
     if (g < 1) g = 1;
     if (g > p.BH()) g = p.BH();
+    const long long groups = (p.BH() + g - 1) / g;      // groups of equal size (to within one head)
+    g = (p.BH() + groups - 1) / groups;
     return (int)g;
 }
 

@@ -504,14 +504,14 @@ static bool decode_uses_tc(const DecodeProblem &p, int dtype)
 }
 
 // Tensor-core route: key tiles of 128 per CTA segment, one CTA per SM at a time.  All CTAs are equal,
-// so the run takes ceil(CTAs / 148) rounds of (fixed cost + tiles per segment); the fixed cost of a CTA
+// so the run takes ceil(CTAs / SMs) rounds of (fixed cost + tiles per segment); the fixed cost of a CTA
 // (pipeline fill, epilogue) was measured at about 3.5 tile times.  Take the segment count that
 // minimises rounds x (3.5 + tiles).
 static void decode_tc_splits(const DecodeProblem &p, int *splits, int *tiles_per_split)
 {
     const int nkt = (p.n + 127) / 128;
-    const long long base = (long long)p.B * p.Hkv;
-    long long hi = (32LL * 148 + base - 1) / base;
+    const long long base = (long long)p.B * p.Hkv, sms = device_info().sms;
+    long long hi = (32LL * sms + base - 1) / base;
     if (hi > nkt) hi = nkt;
     if (hi < 1) hi = 1;
     long long best = 1;
@@ -519,7 +519,7 @@ static void decode_tc_splits(const DecodeProblem &p, int *splits, int *tiles_per
     for (long long s = 1; s <= hi; ++s) {
         const int tps = (int)((nkt + s - 1) / s);
         const long long real = (nkt + tps - 1) / tps;      // segments that get at least one tile
-        const long long rounds = (base * real + 147) / 148;
+        const long long rounds = (base * real + sms - 1) / sms;
         const double cost = (double)rounds * (3.5 + tps);
         if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
     }
@@ -535,7 +535,7 @@ int decode_splits(const DecodeProblem &p)
     const int group = p.H / p.Hkv;
     const int gc = group >= 8 ? 8 : group >= 4 ? 4 : group >= 2 ? 2 : 1;
     const long long ctas_per_split = (long long)p.B * p.Hkv * ((group + gc - 1) / gc);
-    long long s = (4LL * 148 + ctas_per_split - 1) / ctas_per_split;
+    long long s = (4LL * device_info().sms + ctas_per_split - 1) / ctas_per_split;
     const long long cap = (p.n + 255) / 256;
     if (s > cap) s = cap;
     if (s < 1) s = 1;

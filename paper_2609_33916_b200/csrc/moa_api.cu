@@ -67,6 +67,24 @@ unsigned int *device_status_ptr()
     return cache[dev];
 }
 
+const DeviceInfo &device_info()
+{
+    constexpr int kMaxDev = 64;
+    static DeviceInfo cache[kMaxDev];
+    static std::atomic<int> known[kMaxDev];
+    static const DeviceInfo fallback{148, 126LL << 20};      // B200, if the attributes cannot be read
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return fallback;
+    if (!known[dev].load(std::memory_order_acquire)) {
+        int sms = 0, l2 = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return fallback;
+        if (cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) != cudaSuccess || l2 <= 0) return fallback;
+        cache[dev] = DeviceInfo{sms, (long long)l2};
+        known[dev].store(1, std::memory_order_release);
+    }
+    return cache[dev];
+}
+
 namespace {
 
 constexpr size_t kAlign = 256;

@@ -741,7 +741,7 @@ cudaError_t convert_f32_to_bf16(const float *src, void *dst, size_t count, float
     const size_t quads = (count + 3) / 4;
     size_t blocks = (quads + 4 * 256 - 1) / (4 * 256);
     if (blocks < 1) blocks = 1;
-    if (blocks > 148 * 16) blocks = 148 * 16;     // grid-stride beyond 16 blocks per SM
+    if (blocks > 16LL * device_info().sms) blocks = 16LL * device_info().sms;     // grid-stride beyond 16 blocks per SM
     const unsigned grid = (unsigned)blocks;
     LaunchScope scope(MOA_KERNEL_CONVERT, st);
     convert_kernel<<<grid, 256, 0, st>>>(src, (__nv_bfloat16 *)dst, count, mul);
@@ -754,7 +754,7 @@ cudaError_t convert_f32_to_bf16_rows(const float *src, int src_ld, void *dst, in
     const size_t rows = (size_t)B * H * n, quads = rows * (size_t)(d / 4);
     size_t blocks = (quads + 255) / 256;
     if (blocks < 1) blocks = 1;
-    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks > 16LL * device_info().sms) blocks = 16LL * device_info().sms;
     LaunchScope scope(MOA_KERNEL_CONVERT, st);
     convert_rows_kernel<<<(unsigned)blocks, 256, 0, st>>>(src, src_ld, (__nv_bfloat16 *)dst, rows, n, H, d, ds, mul);
     return cudaGetLastError();

@@ -12,16 +12,23 @@
 //     dV  += P^T dO_i                (TS-UMMA: P^T bf16 in TMEM, dO_i MN-major in smem)
 //     dK  += dS^T Q_i                (TS-UMMA: dS^T bf16 in TMEM, Q_i MN-major in smem)
 //     dQ_i = dS K                    (SS-UMMA: dS^T tile in smem as MN-major A, K MN-major)
-// dQ_i is one key tile's contribution; it is added into an fp32 [B,H,n,d] accumulator
-// with vector red.global.add (the contended step the dq_mode knob is about).
+// dQ_i is one key tile's contribution; it is added into an fp32 [B,H,n,d] accumulator (the contended step the
+// dq_mode knob is about): for D = 128 the tile is produced transposed (dQ_i^T = K^T dS^T, lanes = d) and leaves
+// either as warp-wide red.global.add.f32 (one full 128-byte line per instruction) or, by default, staged 32 rows
+// at a time in shared memory and handed to the TMA engine as cp.reduce.async.bulk.tensor add.f32; D = 64 uses
+// red.global.add.v4.f32 on the untransposed tile.
 //
-// Roles (512 threads; registers are re-split per warpgroup with setmaxnreg: 152 / 152 / 56): warps 0-7 elementwise work (thread = TMEM lane = key, the two
-// warpgroups split the query columns), warps 8-11 read each finished dQ tile out of TMEM
-// and issue the reds, warp 12 TMA producer (K,V once; Q_i with L_i, D_i and dO_i in
-// two-slot rings with separate release points), warp 13 UMMA issuer and TMEM owner.
+// Roles (512 threads; registers are re-split per warpgroup with setmaxnreg: 144 / 144 / 144 / 80): warps 0-7
+// elementwise work (thread = TMEM lane = key, the two warpgroups split the query columns), warps 8-11 read each
+// finished dQ tile out of TMEM and send it to the accumulator, warp 12 TMA producer (K,V once; Q_i with L_i, D_i
+// two tiles ahead in a two-slot ring; dO_i in two slots, or one when the staging buffers of the bulk reduce take
+// the other), warp 13 (one thread) UMMA issuer and TMEM owner.
 // UMMA issue order per query tile: dP(i), dV(i), S(i+1), dK(i), dQ(i), so that the
 // exp2 work of tile i+1 overlaps the dK/dQ UMMAs of tile i and the dS work of tile i
-// overlaps dV(i) and S(i+1).
+// overlaps dV(i) and S(i+1).  One thread issues everything: two splits of the issue over two threads
+// ({S, dV} | {dP, dK, dQ} and {S, dP, dV} | {dK, dQ}) were correct and 18-22 % slower, because the second thread's
+// products then share the in-order pipe with the products at the head of the dependency chain
+// dS(i) -> dK(i), dQ(i) -> read-out -> dP(i+1) -> dS(i+1), which is what paces the loop.
 //
 // TMEM columns (512): S^T [0,128), dP^T [128,256), dV [256,256+D), dK [256+D,256+2D);
 // P^T / dS^T (bf16) overwrite the front of their fp32 source columns; for D = 128 the dQ

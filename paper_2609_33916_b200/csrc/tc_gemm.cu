@@ -494,6 +494,36 @@ bool operand_map(CUtensorMap *m, const Operand &o, bool mn_major, int box_rows, 
                               mn_major ? 64 : (uint32_t)box_rows, 64);
 }
 
+// Clusters of two CTAs of `kernel` that can be resident at once (cudaOccupancyMaxActiveClusters; cached per kernel
+// and device); half the SM count if the query fails.
+template <typename K>
+int max_active_pairs(K kernel, int smem)
+{
+    constexpr int kMaxDev = 64;
+    static int cache[kMaxDev] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return device_info().sms / 2;
+    if (cache[dev] > 0) return cache[dev];
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    cfg.gridDim = dim3((unsigned)device_info().sms / 2 * 2);
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = smem;
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n <= 0) {
+        (void)cudaGetLastError();
+        n = device_info().sms / 2;
+    }
+    if (n > device_info().sms / 2) n = device_info().sms / 2;
+    return cache[dev] = n;
+}
+
 template <bool kAMn, bool kBMn, int kEpi, bool kPair>
 // C0..C2: output arrays (row length ldc); unused ones may repeat C0.
 cudaError_t launch_gemm_as(const Operand &A0, const Operand &B0, const Operand *A1, const Operand *B1, void *C0, void *C1,
@@ -534,7 +564,9 @@ cudaError_t launch_gemm_as(const Operand &A0, const Operand &B0, const Operand *
     }
     if (kPair) group_rows = group_rows / 2 < 2 ? 2 : group_rows / 2;     // tile rows of 256
     LaunchScope scope(MOA_KERNEL_OTHER, st);
-    const int ctas = kPair ? 2 * (tiles < 74 ? tiles : 74) : (tiles < 148 ? tiles : 148);
+    // persistent grid: one CTA per SM, or as many clusters of two as the device can hold at once
+    const int sms = device_info().sms, pairs = kPair ? max_active_pairs(kernel, kSmem) : 0;
+    const int ctas = kPair ? 2 * (tiles < pairs ? tiles : pairs) : (tiles < sms ? tiles : sms);
     if (!kPair) {
         kernel<<<ctas, kGemmThreads, kSmem, st>>>(ma0, mb0, ma1, mb1, mc[0], mc[1], mc[2], mc[3], M, N, K, nparts, nbatch,
                                                   a_blocked ? 1 : 0, b_blocked ? 1 : 0, has_res ? 1 : 0, (int)group_rows,
@@ -581,7 +613,8 @@ cudaError_t launch_gemm(const Operand &A0, const Operand &B0, const Operand *A1,
     const long long single_tiles = (long long)((M + GM - 1) / GM) * cols * nbatch;
     // pairs unless they would need more waves than single CTAs (tiny M); the two gate GEMMs only when the main loop
     // outlasts their epilogue
-    const bool fits = pair_tiles >= 8 && (pair_tiles + 73) / 74 <= (single_tiles + 147) / 148;   // (a few tiles: launch-bound)
+    const long long sms = device_info().sms, pairs = sms / 2;
+    const bool fits = pair_tiles >= 8 && (pair_tiles + pairs - 1) / pairs <= (single_tiles + sms - 1) / sms;   // (a few tiles: launch-bound)
     if (gemm_pair_mode() == 2 || (gemm_pair_mode() && fits && (kEpi == EPI_STORE || K >= 1024)))
         return launch_gemm_as<kAMn, kBMn, kEpi, true>(A0, B0, A1, B1, C0, C1, C2, C3, c_rows, ldc, M, N, K, st, nbatch, has_res);
     return launch_gemm_as<kAMn, kBMn, kEpi, false>(A0, B0, A1, B1, C0, C1, C2, C3, c_rows, ldc, M, N, K, st, nbatch, has_res);
