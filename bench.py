@@ -876,7 +876,8 @@ def main():
         raise SystemExit(f"rank {rank}: more ranks than heads to hand out ({w.B * w.H} heads, {world} ranks)")
     B, H, n, d = plan["B"], plan["H"], w.n, w.d
     hkv = plan["H_kv"]
-    desc = mb.make_desc(B, H, n, d, w.causal, w.scale, mb.MOA_BF16, args.dq_mode, args.materialize, args.path,
+    tdt = torch.float32 if w.dtype == "f32" else torch.bfloat16      # config 1 is the fp32 path
+    desc = mb.make_desc(B, H, n, d, w.causal, w.scale, mb.MOA_F32 if w.dtype == "f32" else mb.MOA_BF16, args.dq_mode, args.materialize, args.path,
                         H_kv=hkv, layout=args.layout)
     shape = (B, n, H, d) if args.layout else (B, H, n, d)
     kv_shape = (B, n, hkv or H, d) if args.layout else (B, hkv or H, n, d)       # K, V, dK, dV
@@ -884,9 +885,9 @@ def main():
     shapes_out = (shape, shape, kv_shape, kv_shape)           # O, dQ, dK, dV
     base_mem = torch.cuda.memory_allocated()
     gen = torch.Generator(device="cuda").manual_seed(w.seed + 1000 * rank)
-    Q, K, V, dO = (torch.randn(sh, generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    Q, K, V, dO = (torch.randn(sh, generator=gen, device="cuda", dtype=torch.float32).to(tdt)
                    for sh in shapes_in)
-    O, dQ, dK, dV = (torch.empty(sh, dtype=torch.bfloat16, device="cuda") for sh in shapes_out)
+    O, dQ, dK, dV = (torch.empty(sh, dtype=tdt, device="cuda") for sh in shapes_out)
     L = torch.empty((B, H, n), dtype=torch.float32, device="cuda")
     ws_bytes = mb.moa_attn_workspace_bytes(desc, mb.MOA_OP_FUSED)
     ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device="cuda")
@@ -995,14 +996,14 @@ def main():
     # The three legs run on three streams over two buffer sets, so step k+1's upload and step
     # k-1's download overlap step k's kernels (the library call takes the stream it runs on).
     hQ, hK, hV, hdO = (t.cpu().pin_memory() for t in (Q, K, V, dO))
-    hO, hdQ, hdK, hdV = (torch.empty(sh, dtype=torch.bfloat16).pin_memory() for sh in shapes_out)
+    hO, hdQ, hdK, hdV = (torch.empty(sh, dtype=tdt).pin_memory() for sh in shapes_out)
     hL = torch.empty((B, H, n), dtype=torch.float32).pin_memory()
     h2d = sum(t.numel() * t.element_size() for t in (hQ, hK, hV, hdO))
     d2h = sum(t.numel() * t.element_size() for t in (hO, hdQ, hdK, hdV, hL))
     sets = []
     for _ in range(2):
-        ins = [torch.empty(sh, dtype=torch.bfloat16, device="cuda") for sh in shapes_in]
-        outs = [torch.empty(sh, dtype=torch.bfloat16, device="cuda") for sh in shapes_out]
+        ins = [torch.empty(sh, dtype=tdt, device="cuda") for sh in shapes_in]
+        outs = [torch.empty(sh, dtype=tdt, device="cuda") for sh in shapes_out]
         sets.append({"in": ins, "out": outs, "L": torch.empty((B, H, n), dtype=torch.float32, device="cuda"),
                      "ws": torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device="cuda"),
                      "up": torch.cuda.Event(), "done": torch.cuda.Event(), "down": torch.cuda.Event()})
@@ -1103,7 +1104,7 @@ def main():
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "strong" if (args.shard == "heads" and world > 1) else "weak",
-        "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(w, args),
+        "vs_baseline": None, "dtype": w.dtype, "data": "synthetic", "config": workload_config(w, args),
         "pct_of_peak": {"of_measured_burst": 100 * value / world / peaks["bf16_tflops"],
                         "of_measured_sustained": 100 * value / world / peaks["bf16_tflops_sustained"],
                         "of_nominal_2250": 100 * value / world / NOMINAL_BF16_TFLOPS, "peaks": peaks_kind},
