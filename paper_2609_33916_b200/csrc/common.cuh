@@ -48,9 +48,10 @@ struct Problem {
 };
 
 // Head dimension the tensor-core kernels are compiled for: a head of d columns (a multiple of 8, so
-// that rows stay 16-byte aligned) runs in the 64- or 128-column kernel; the TMA loads fill the
+// that rows stay 16-byte aligned) runs in the 64-, 128- or 256-column kernels; the TMA loads fill the
 // columns past d with zeros and the TMA stores drop them, which leaves every result unchanged.
-inline int kernel_d(int d) { return d <= 64 ? 64 : 128; }
+// 256: the two-pass kernels for head dimensions 136..256 (tc_fwd.cu with KC = 2, tc_bwd_wide.cu).
+inline int kernel_d(int d) { return d <= 64 ? 64 : d <= 128 ? 128 : 256; }
 
 // Block order of the tile-parallel kernels.  Heads are taken in groups of `hpg`; inside a group
 // the blocks go tile-major (every head's tile 0, then every head's tile 1, ...).  With causal
@@ -180,6 +181,11 @@ cudaError_t tc_bwd_kv_pair(const Problem &p, const void *Q, const void *K, const
                            cudaStream_t st);
 bool bwd_pair_enabled();
 int bwd_pair_mode(int set);      // set < 0: query; returns the mode in force before the call
+
+// Head dimensions 136..256 (tc_bwd_wide.cu): tiles of 128 keys x 64 queries, two passes over the halves of d; dQ by
+// red.global into dQacc (fp32 [B,H,n,256], pre-zeroed)
+cudaError_t tc_bwd_kv_wide(const Problem &p, const void *Q, const void *K, const void *V, const void *dO,
+                           const float *Lp, const float *Dp, void *dK, void *dV, float *dQacc, cudaStream_t st);
 
 // atomic-free query-parallel dQ pass on the tensor cores (tc_dq.cu); writes dQ (bf16) directly
 cudaError_t tc_bwd_dq(const Problem &p, const void *Q, const void *K, const void *V, const void *dO,

@@ -118,12 +118,14 @@ moa_status check_desc(const moa_attn_desc *d)
     if (d->materialize != 0 && d->materialize != 1) return MOA_ERR_INVALID_ARG;
     if (d->path < MOA_PATH_AUTO || d->path > MOA_PATH_TC) return MOA_ERR_INVALID_ARG;
     if (!(d->scale == d->scale) || d->scale - d->scale != 0.f) return MOA_ERR_INVALID_ARG;  // NaN / inf
-    // head dimensions other than 64 and 128: multiples of 8 up to 128, on the tensor-core kernels only
-    // (they run in the 64- or 128-column kernel with the missing columns filled with zeros)
+    // head dimensions other than 64 and 128: multiples of 8 up to 256, on the tensor-core kernels only
+    // (they run in the 64-, 128- or 256-column kernels with the missing columns filled with zeros)
     if (d->d != 64 && d->d != 128 &&
-        !(d->d % 8 == 0 && d->d <= 128 && d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->scale > 0.f &&
+        !(d->d % 8 == 0 && d->d <= 256 && d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->scale > 0.f &&
           !d->materialize))
         return MOA_ERR_UNSUPPORTED;
+    // above 128 the backward exists with plain reds only (no bulk reduce, no separate dQ pass)
+    if (d->d > 128 && (d->dq_mode == MOA_DQ_BULK_REDUCE || d->dq_mode == MOA_DQ_SEPARATE_PASS)) return MOA_ERR_UNSUPPORTED;
     if ((long long)d->B * d->H > (1 << 20)) return MOA_ERR_UNSUPPORTED;
     // one CTA per (tile, head) in grid.x
     const long long tiles = ((long long)d->n + 63) / 64;
@@ -439,7 +441,8 @@ moa_status moa_attn_fused_fwd_bwd(const moa_attn_desc *desc, const void *Q, cons
     // tensor-core path with an atomic dQ mode: the forward clears the accumulator its backward adds into
     // and writes the backward's per-row inputs (-L log2e, -D) from the fp32 O it holds
     FwdForBwd fb;
-    const bool both_tc = use_tc_fwd(desc) && use_tc_bwd(desc);
+    // (head dimensions above 128: a forward CTA holds half of an O row, so the backward prepares its own inputs)
+    const bool both_tc = use_tc_fwd(desc) && use_tc_bwd(desc) && kernel_d(desc->d) <= 128;
     if (both_tc) {
         const BwdWorkspace w = bwd_workspace(desc);
         fb.Dp = (float *)ws;

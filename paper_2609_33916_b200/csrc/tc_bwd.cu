@@ -667,7 +667,10 @@ cudaError_t tc_bwd_preprocess(const Problem &p, const void *dO, const void *O, c
     const size_t rows_per_block = (size_t)wpb * (32 / (D / 8)) * 4;   // warps x rows per pass x passes
     const unsigned grid = (unsigned)((rows + rows_per_block - 1) / rows_per_block);
     LaunchScope scope(MOA_KERNEL_PREPROCESS, st);
-    if (D == 64)
+    if (D == 256)
+        bwd_preprocess_kernel<256><<<grid, wpb * 32, 0, st>>>((const __nv_bfloat16 *)dO, (const __nv_bfloat16 *)O, L,
+                                                              Lp, Dp, p.n, n_pad, rows, p.H, p.so, p.d);
+    else if (D == 64)
         bwd_preprocess_kernel<64><<<grid, wpb * 32, 0, st>>>((const __nv_bfloat16 *)dO, (const __nv_bfloat16 *)O, L,
                                                              Lp, Dp, p.n, n_pad, rows, p.H, p.so, p.d);
     else
@@ -679,8 +682,9 @@ cudaError_t tc_bwd_preprocess(const Problem &p, const void *dO, const void *O, c
 cudaError_t tc_bwd_kv(const Problem &p, const void *Q, const void *K, const void *V, const void *dO,
                       const float *Lp, const float *Dp, void *dK, void *dV, float *dQacc, int dq_bulk, cudaStream_t st)
 {
-    if (p.d < 8 || p.d > 128 || p.d % 8) return cudaErrorInvalidValue;
+    if (p.d < 8 || p.d > 256 || p.d % 8) return cudaErrorInvalidValue;
     const int D = kernel_d(p.d);     // dQacc rows are D floats wide
+    if (D == 256) return dq_bulk ? cudaErrorInvalidValue : tc_bwd_kv_wide(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
     if (D == 128 && bwd_pair_enabled()) return tc_bwd_kv_pair(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, dq_bulk, st);
     if (D == 64 && !dq_bulk) return launch_bwd<64, false>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
     if (D == 128 && !dq_bulk) return launch_bwd<128, false>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);

@@ -27,6 +27,12 @@
 // takes ~1850 because the two softmax warpgroups run their exp2 phases at the same time and the
 // rest of their work (TMEM load, max, hand-offs, ~600 cycles) is not hidden under them.
 // The O tile leaves through the Q tile's shared memory and a TMA store.
+//
+// Head dimensions 136..256 (KC = 2): the scores need the whole head dimension, the output does not.  S = Q K^T is
+// accumulated over KC chunks of 128 columns -- Q holds all of them, the K ring carries one chunk per slot, so a key
+// tile passes through it KC times -- and the grid has KC CTAs per (head, query tile), each with the V columns and the
+// O columns of one 128-column half (the scores and the softmax are computed KC times; O(n d) memory as before).
+// The backward's per-row inputs are then not prepared here (a CTA holds half of an O row).
 #include "common.cuh"
 #include "ptx.cuh"
 #include "tensormap.cuh"
@@ -69,7 +75,7 @@ struct FwdPrep {
     int d;               // columns of a dO row in memory (<= D)
 };
 
-template <int D>
+template <int D, int KC>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
               const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapO,
@@ -81,16 +87,19 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     constexpr int kBoxes = D / 64;         // 64-column (128-byte) swizzled boxes per tile
     constexpr int kBoxBytes = 128 * 128;   // 128 rows x 128 bytes
     extern __shared__ __align__(1024) uint8_t sm[];
-    uint8_t *sQ = sm, *sK = sm + kTileBytes /*2 slots*/, *sV = sm + 3 * kTileBytes /*2 slots*/;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(sm + 5 * kTileBytes);
+    uint8_t *sQ = sm /*KC chunks*/, *sK = sm + KC * kTileBytes /*2 slots of one chunk*/, *sV = sm + (KC + 2) * kTileBytes /*2 slots*/;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(sm + (KC + 4) * kTileBytes);
     uint32_t *tmem_base_p = reinterpret_cast<uint32_t *>(bars + F_COUNT);
     volatile uint32_t *abortp = reinterpret_cast<uint32_t *>(bars + F_COUNT + 1);
 
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
     int bh, t;
-    const int split = sp.splits > 1 ? (int)blockIdx.x % sp.splits : 0;
-    const int heads_all = (int)gridDim.x / sp.splits / nqt;
-    job_from_block(sp.splits > 1 ? (int)blockIdx.x / sp.splits : (int)blockIdx.x, nqt, heads_all, hpg, bh, t);
+    // KC > 1: KC consecutive CTAs share a job, CTA `pass` computes output columns [D pass, D pass + D)
+    const int pass = KC > 1 ? (int)blockIdx.x % KC : 0;
+    const int blk = KC > 1 ? (int)blockIdx.x / KC : (int)blockIdx.x;
+    const int split = sp.splits > 1 ? blk % sp.splits : 0;
+    const int heads_all = (int)gridDim.x / KC / sp.splits / nqt;
+    job_from_block(sp.splits > 1 ? blk / sp.splits : blk, nqt, heads_all, hpg, bh, t);
     const int bb = bh / H, hq = bh - bb * H;    // batch and query head: coordinates of the 4-D tensor maps
     const int hk = hq / group;                  // the K/V head this query head reads (group > 1: shared heads)
     const int qt = causal ? nqt - 1 - t : t;   // causal: longest rows first
@@ -117,46 +126,49 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         // ------------------------------------------------------------------ TMA producer
         int nk = 0, nv = 0;     // K and V tiles requested so far (slot = count & 1)
         if (lane == 0 && nkt > 0) {
-            mbar_arrive_expect_tx(bars + F_Q, kTileBytes);
-            for (int b = 0; b < kBoxes; ++b) tma_load_4d(sQ + b * kBoxBytes, &mapQ, bars + F_Q, 64 * b, q0, hq, bb);
+            mbar_arrive_expect_tx(bars + F_Q, KC * kTileBytes);
+            for (int b = 0; b < KC * kBoxes; ++b) tma_load_4d(sQ + b * kBoxBytes, &mapQ, bars + F_Q, 64 * b, q0, hq, bb);
         }
+        // chunk g of the K stream: 128 columns [D c, D c + D) of key tile j, g = j KC + c, ring slot g & 1
+        auto load_k = [&](int g) {
+            const int s = g & 1, j = g / KC, c = g % KC;
+            mbar_arrive_expect_tx(bars + F_KFULL + s, kTileBytes);
+            ++nk;
+            for (int b = 0; b < kBoxes; ++b)
+                tma_load_4d(sK + s * kTileBytes + b * kBoxBytes, &mapK, bars + F_KFULL + s, D * c + 64 * b, (kt0 + j) * BN, hk, bb);
+        };
+        auto load_v = [&](int j) {            // this CTA's column half of V tile j
+            const int s = j & 1;
+            mbar_arrive_expect_tx(bars + F_VFULL + s, kTileBytes);
+            ++nv;
+            for (int b = 0; b < kBoxes; ++b)
+                tma_load_4d(sV + s * kTileBytes + b * kBoxBytes, &mapV, bars + F_VFULL + s, D * pass + 64 * b, (kt0 + j) * BN, hk, bb);
+        };
         if (zero_acc != nullptr) {
-            // Fused forward+backward: this CTA's 128 rows of the fp32 dQ accumulator ([B*H, n, D]) are
+            // Fused forward+backward (KC = 1): this CTA's 128 rows of the fp32 dQ accumulator ([B*H, n, D]) are
             // cleared here, by the producer warp while its first loads are in flight (the next slot
             // frees two tiles from now), so that the step needs no separate clearing pass.
             // The first two K/V tiles are requested first: they have no slot to wait for.
             for (int j = 0; j < min(nkt, 2); ++j) {
                 if (lane == 0) {
-                    mbar_arrive_expect_tx(bars + F_KFULL + j, kTileBytes);
-                    ++nk;
-                    for (int b = 0; b < kBoxes; ++b)
-                        tma_load_4d(sK + j * kTileBytes + b * kBoxBytes, &mapK, bars + F_KFULL + j, 64 * b, (kt0 + j) * BN, hk, bb);
-                    mbar_arrive_expect_tx(bars + F_VFULL + j, kTileBytes);
-                    ++nv;
-                    for (int b = 0; b < kBoxes; ++b)
-                        tma_load_4d(sV + j * kTileBytes + b * kBoxBytes, &mapV, bars + F_VFULL + j, 64 * b, (kt0 + j) * BN, hk, bb);
+                    load_k(j);
+                    load_v(j);
                 }
             }
             const int rows = min(BM, n - q0);
             float4 *dst = reinterpret_cast<float4 *>(zero_acc + ((size_t)bh * n + q0) * D);
             for (int i = lane; i < rows * (D / 4); i += 32) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        for (int j = (zero_acc != nullptr ? min(nkt, 2) : 0); j < nkt; ++j) {
-            const int s = j & 1;
-            if (j >= 2 && !mbar_wait(bars + F_KEMPTY + s, ((j >> 1) - 1) & 1, abortp, status, ERR_K)) break;
-            if (lane == 0) {
-                mbar_arrive_expect_tx(bars + F_KFULL + s, kTileBytes);
-                ++nk;
-                for (int b = 0; b < kBoxes; ++b)
-                    tma_load_4d(sK + s * kTileBytes + b * kBoxBytes, &mapK, bars + F_KFULL + s, 64 * b, (kt0 + j) * BN, hk, bb);
+        bool live = true;
+        for (int j = (zero_acc != nullptr ? min(nkt, 2) : 0); live && j < nkt; ++j) {
+            for (int c = 0; c < KC; ++c) {
+                const int g = j * KC + c;
+                if (g >= 2 && !mbar_wait(bars + F_KEMPTY + (g & 1), ((g >> 1) - 1) & 1, abortp, status, ERR_K)) { live = false; break; }
+                if (lane == 0) load_k(g);
             }
-            if (j >= 2 && !mbar_wait(bars + F_VEMPTY + s, ((j >> 1) - 1) & 1, abortp, status, ERR_V)) break;
-            if (lane == 0) {
-                mbar_arrive_expect_tx(bars + F_VFULL + s, kTileBytes);
-                ++nv;
-                for (int b = 0; b < kBoxes; ++b)
-                    tma_load_4d(sV + s * kTileBytes + b * kBoxBytes, &mapV, bars + F_VFULL + s, 64 * b, (kt0 + j) * BN, hk, bb);
-            }
+            if (!live) break;
+            if (j >= 2 && !mbar_wait(bars + F_VEMPTY + (j & 1), ((j >> 1) - 1) & 1, abortp, status, ERR_V)) break;
+            if (lane == 0) load_v(j);
             __syncwarp();
         }
         if (lane == 0 && *abortp) {
@@ -184,18 +196,25 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         bool ok = nkt > 0 && mbar_wait(bars + F_Q, 0, abortp, status, ERR_Q);
         for (int j = 0; ok && j < nkt; ++j) {
             const int b = j & 1;
-            const uint32_t k_lo = k_lo0 + b * kSlot, dcol = tbase + kColS + 128 * b;
-            if (!mbar_wait(bars + F_KFULL + b, (j >> 1) & 1, abortp, status, ERR_K)) break;
-            if (j >= 2 && !mbar_wait(bars + F_OB + b, ((j >> 1) - 1) & 1, abortp, status, ERR_O)) break;
-            tc_fence_after();
-            umma_ss2<false>(dcol, q_lo, km_hi, k_lo, km_hi, idesc_s);
+            const uint32_t dcol = tbase + kColS + 128 * b;
 #pragma unroll
-            for (int ks = 1; ks < D / 16; ++ks) {
-                const uint32_t off = (uint32_t)(((ks / 4) * kBoxBytes + (ks % 4) * 32) >> 4);
-                umma_ss2<true>(dcol, q_lo + off, km_hi, k_lo + off, km_hi, idesc_s);
+            for (int c = 0; c < KC; ++c) {          // the contraction over the head dimension, 128 columns per K chunk
+                const int g = j * KC + c, sl = g & 1;
+                const uint32_t k_lo = k_lo0 + sl * kSlot, q_c = q_lo + c * kSlot;
+                if (!mbar_wait(bars + F_KFULL + sl, (g >> 1) & 1, abortp, status, ERR_K)) { ok = false; break; }
+                if (c == 0 && j >= 2 && !mbar_wait(bars + F_OB + b, ((j >> 1) - 1) & 1, abortp, status, ERR_O)) { ok = false; break; }
+                tc_fence_after();
+                if (c == 0) umma_ss2<false>(dcol, q_c, km_hi, k_lo, km_hi, idesc_s);
+                else        umma_ss2<true>(dcol, q_c, km_hi, k_lo, km_hi, idesc_s);
+#pragma unroll
+                for (int ks = 1; ks < D / 16; ++ks) {
+                    const uint32_t off = (uint32_t)(((ks / 4) * kBoxBytes + (ks % 4) * 32) >> 4);
+                    umma_ss2<true>(dcol, q_c + off, km_hi, k_lo + off, km_hi, idesc_s);
+                }
+                umma_commit(bars + F_KEMPTY + sl);
             }
+            if (!ok) break;
             umma_commit(bars + F_S + b);
-            umma_commit(bars + F_KEMPTY + b);
         }
     } else if (warp == 10 && lane == 0) {
         // ------------------------------------------------ UMMA issuer for O += P V (one thread)
@@ -406,11 +425,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 prep.Lp[prow] = row < n ? -(m_all + log2f(l_all)) : -INFINITY;
             }
             if (tid == 0 && mbar_wait(bars + F_E, 0, abortp, status, ERR_O)) {
-                for (int b = 0; b < kBoxes; ++b) tma_store_4d(&mapO, sQ + b * kBoxBytes, 64 * b, q0, hq, split * (heads_all / H) + bb);
+                for (int b = 0; b < kBoxes; ++b)
+                    if (D * pass + 64 * b < prep.d)       // (a box wholly past the head dimension has nothing to store)
+                        tma_store_4d(&mapO, sQ + b * kBoxBytes, D * pass + 64 * b, q0, hq, split * (heads_all / H) + bb);
                 bulk_commit();
                 bulk_wait_read<0>();      // shared memory is read before the CTA may exit
             }
-            if (row < sp.n_q && h == 0) L[((size_t)split * heads_all + bh) * sp.n_q + row] = m_all * kLn2 + logf(l_all);
+            if (row < sp.n_q && h == 0 && pass == 0) L[((size_t)split * heads_all + bh) * sp.n_q + row] = m_all * kLn2 + logf(l_all);
         }
     }
     tc_fence_before();
@@ -418,11 +439,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     if (warp == 9) tmem_dealloc(tbase, kTmemCols);
 }
 
-template <int D>
+template <int D, int KC>
 cudaError_t launch_fwd(const Problem &p, const void *Q, const void *K, const void *V, void *O, float *L,
                        const FwdForBwd &fb, cudaStream_t st)
 {
-    constexpr int kSmem = 5 * 128 * D * 2 + 8 * (F_COUNT + 2) + 2 * 128 * 8 + 2 * 128 * 4;
+    constexpr int kSmem = (KC + 4) * 128 * D * 2 + 8 * (F_COUNT + 2) + 2 * 128 * 8 + 2 * 128 * 4;
+    if (KC > 1 && (fb.dO != nullptr || fb.zero_acc != nullptr)) return cudaErrorInvalidValue;   // no fused preparation with KC > 1
     CUtensorMap mq, mk, mv, mo;
     const auto bf = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     // p.d <= D columns exist in memory: loads fill the rest of a box with zeros, the store drops it
@@ -431,11 +453,11 @@ cudaError_t launch_fwd(const Problem &p, const void *Q, const void *K, const voi
         !make_tensor_map_4d_strided(&mv, V, bf, 2, p.B, p.kv_heads(), p.n, p.d, p.skv.row, p.skv.head, p.skv.batch, 128, 64) ||
         !make_tensor_map_4d_strided(&mo, O, bf, 2, p.B, p.H, p.n, p.d, p.so.row, p.so.head, p.so.batch, 128, 64))
         return cudaErrorInvalidValue;
-    cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel<D, KC>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
     const int nqt = (p.n + BM - 1) / BM;
     LaunchScope scope(MOA_KERNEL_FWD, st);
-    tc_fwd_kernel<D><<<(unsigned)(nqt * p.BH()), kThreads, kSmem, st>>>(
+    tc_fwd_kernel<D, KC><<<(unsigned)(nqt * p.BH() * KC), kThreads, kSmem, st>>>(
         mq, mk, mv, mo, L, p.n, p.causal, p.scale * kLog2e, nqt, heads_per_group(p, nqt), p.group(), p.H,
         FwdSplit{p.n, 1, (p.n + BN - 1) / BN}, fb.zero_acc,
         FwdPrep{(const __nv_bfloat16 *)fb.dO, fb.Lp, fb.Dp, nqt * BM, p.so, p.d}, device_status_ptr());
@@ -458,12 +480,12 @@ cudaError_t launch_fwd_decode(int B, int Hkv, int G, int n, float scale, const v
         !make_tensor_map_4d(&mv, V, bf, 2, B, Hkv, n, D, false, 128, 64) ||
         !make_tensor_map_4d(&mo, O_part, bf, 2, (uint64_t)splits * B, Hkv, G, D, false, 128, 64))
         return cudaErrorInvalidValue;
-    cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel<D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
     LaunchScope scope(MOA_KERNEL_FWD, st);
-    tc_fwd_kernel<D><<<(unsigned)(B * Hkv * splits), kThreads, kSmem, st>>>(
+    tc_fwd_kernel<D, 1><<<(unsigned)(B * Hkv * splits), kThreads, kSmem, st>>>(
         mq, mk, mv, mo, L_part, n, 0, scale * kLog2e, 1, 1, 1, Hkv, FwdSplit{G, splits, tiles_per_split},
-        nullptr, FwdPrep{nullptr, nullptr, nullptr, 0, 0, D}, device_status_ptr());
+        nullptr, FwdPrep{nullptr, nullptr, nullptr, 0, Strides{0, 0, 0}, D}, device_status_ptr());
     return cudaGetLastError();
 }
 
@@ -480,8 +502,9 @@ cudaError_t tc_fwd_decode(int B, int Hkv, int G, int n, int d, float scale, cons
 cudaError_t tc_fwd(const Problem &p, const void *Q, const void *K, const void *V, void *O, float *L,
                    const FwdForBwd &fb, cudaStream_t st)
 {
-    if (p.d < 8 || p.d > 128 || p.d % 8) return cudaErrorInvalidValue;
-    return kernel_d(p.d) == 64 ? launch_fwd<64>(p, Q, K, V, O, L, fb, st) : launch_fwd<128>(p, Q, K, V, O, L, fb, st);
+    if (p.d < 8 || p.d > 256 || p.d % 8) return cudaErrorInvalidValue;
+    if (p.d > 128) return launch_fwd<128, 2>(p, Q, K, V, O, L, fb, st);      // two 128-column passes, scores over both chunks
+    return kernel_d(p.d) == 64 ? launch_fwd<64, 1>(p, Q, K, V, O, L, fb, st) : launch_fwd<128, 1>(p, Q, K, V, O, L, fb, st);
 }
 
 }  // namespace moa

@@ -90,7 +90,7 @@ def test_argument_errors_need_no_device(lib):
 
 
 def test_other_head_dimensions_argument_checks(lib):
-    """Multiples of 8 up to 128 run on the bf16 tensor-core kernels only."""
+    """Multiples of 8 up to 256 run on the bf16 tensor-core kernels only; above 128 with the plain-red dQ strategy."""
     a = 4096
 
     def fwd(d, **kw):
@@ -99,9 +99,16 @@ def test_other_head_dimensions_argument_checks(lib):
     def ws(d, **kw):
         return mb.moa_attn_workspace_bytes(mb.make_desc(1, 2, 256, d, True, 0.1, **kw), mb.MOA_OP_FUSED)
 
-    for d in (100, 4, 12, 136, 192, 256):
+    for d in (100, 4, 12, 260, 264, 512):
         assert fwd(d) == mb.MOA_ERR_UNSUPPORTED, d
         assert ws(d) == 0
+    for d in (136, 192, 256):
+        assert fwd(d, dtype=mb.MOA_F32) == mb.MOA_ERR_UNSUPPORTED
+        assert fwd(d, dq_mode=mb.MOA_DQ_BULK_REDUCE) == mb.MOA_ERR_UNSUPPORTED
+        assert fwd(d, dq_mode=mb.MOA_DQ_SEPARATE_PASS) == mb.MOA_ERR_UNSUPPORTED
+        assert fwd(d, materialize=1) == mb.MOA_ERR_UNSUPPORTED
+        # accumulator rows of 256 floats
+        assert ws(d) == 2 * (2 * 256 * 4) + 2 * 256 * 256 * 4
     assert fwd(96, dtype=mb.MOA_F32) == mb.MOA_ERR_UNSUPPORTED
     assert fwd(96, path=mb.MOA_PATH_SIMT) == mb.MOA_ERR_UNSUPPORTED
     assert fwd(96, materialize=1) == mb.MOA_ERR_UNSUPPORTED
