@@ -37,9 +37,12 @@
  *    launch, clear or descriptor encode of a call that consists of several: kernels
  *    enqueued before it still run, and the outputs and the workspace are undefined.
  *  - Supported: d in {64, 128} everywhere; on the bf16 tensor-core kernels also every
- *    other multiple of 8 up to 128 (d = 96, 80, 32, ...: the head runs in the 64- or
- *    128-column kernel, TMA zero-fills the missing columns on load and drops them on
- *    store; not with materialize = 1).  Any n >= 1 and B, H >= 1 (B*H <= 2^20 and
+ *    other multiple of 8 up to 256 (d = 96, 80, 32, 192, ...: the head runs in the 64-,
+ *    128- or 256-column kernel, TMA zero-fills the missing columns on load and drops
+ *    them on store; not with materialize = 1).  Above 128 the forward accumulates the
+ *    scores over two 128-column chunks and the backward works on 128 x 64 tiles in two
+ *    passes over the halves of d; there dq_mode is MOA_DQ_AUTO or MOA_DQ_RED
+ *    (BULK_REDUCE and SEPARATE_PASS give MOA_ERR_UNSUPPORTED).  Any n >= 1 and B, H >= 1 (B*H <= 2^20 and
  *    ceil(n/64)*B*H < 2^31, else MOA_ERR_UNSUPPORTED); n need not be a multiple
  *    of the tile size.
  *    A device that is not compute capability 10.x gives MOA_ERR_ARCH.
@@ -57,7 +60,7 @@ extern "C" {
 typedef enum {
     MOA_OK = 0,
     MOA_ERR_INVALID_ARG = 1, /* NULL pointer, misaligned pointer, non-positive size, bad enum  */
-    MOA_ERR_UNSUPPORTED = 2, /* well-formed request this build cannot run (e.g. d = 192)      */
+    MOA_ERR_UNSUPPORTED = 2, /* well-formed request this build cannot run (e.g. d = 320)      */
     MOA_ERR_WORKSPACE = 3,   /* ws == NULL or ws_bytes < moa_attn_workspace_bytes(...)         */
     MOA_ERR_ARCH = 4,        /* current device is not sm_100                                   */
     MOA_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed (launch, descriptor encode)  */
