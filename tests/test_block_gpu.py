@@ -412,8 +412,40 @@ def test_gated_mlp_full_bench_size_sampled(rt):
         assert bool(torch.isfinite(t.float()).all())
 
 
+@pytest.mark.parametrize("B,n,H,d,dff,causal", [(2, 256, 4, 64, 512, True), (1, 333, 2, 128, 384, False), (2, 200, 3, 96, 320, True)])
+def test_block_class_packed_projection_matches_oracle_and_the_three_gemm_form(rt, B, n, H, d, dff, causal):
+    """block.TransformerBlock with one projection GEMM for Q, K and V (a packed [B,n,3,H,d] array read and written by
+    the attention through explicit strides) against the fp64 block oracle, and against the same class with three
+    projection GEMMs: the forward agrees bit for bit (same products, same attention), gradients to rounding."""
+    torch, mb = rt
+    from paper_2609_33916_b200.block import TransformerBlock
+    inp = make_block_inputs(B, n, H, d, dff, seed=170 + n)
+    dev = {k: _dev(torch, v) for k, v in inp.items()}
+    w = {k: dev[k] for k in ("g1", "g2", "Wq", "Wk", "Wv", "Wo", "W1", "W3", "W2")}
+    out = {}
+    for packed in (True, False):
+        blk = TransformerBlock(torch, B, n, H, d, dff, causal, packed_qkv=packed)
+        wp = blk.prepare_weights(w)
+        assert ("Wqkv" in wp) == packed
+        blk.forward(dev["x"], wp)
+        blk.backward(dev["x"], wp, dev["dy"])
+        torch.cuda.synchronize()
+        assert mb.moa_last_device_status() == mb.MOA_OK
+        got = {"y": _host(blk.y), "dx": _host(blk.dx)}
+        for k_, v_ in blk.grads.items():
+            got["d" + k_] = _host(v_)
+        out[packed] = got
+    f = {k: mi.to_f64(v, "bf16") for k, v in inp.items()}
+    wf = {k: f[k] for k in ("g1", "g2", "Wq", "Wk", "Wv", "Wo", "W1", "W3", "W2")}
+    ref = oracle.transformer_block_fwd_bwd(f["x"], wf, f["dy"], B, n, H, causal, 1e-5)
+    np.testing.assert_array_equal(out[True]["y"], out[False]["y"])
+    for k_ in out[True]:
+        assert mi.rel_err(out[True][k_], ref[k_]) <= 2e-2, (k_, mi.rel_err(out[True][k_], ref[k_]))
+        assert mi.rel_err(out[True][k_], out[False][k_]) <= 8e-3, k_
+
+
 def test_block_can_be_captured_in_a_cuda_graph_and_replayed(rt):
-    """The 20 calls of a block step allocate nothing and synchronise nothing: recorded once in a CUDA graph, a replay
+    """The calls of a block step allocate nothing and synchronise nothing: recorded once in a CUDA graph, a replay
     gives the bits of a direct run for everything the forward writes, and gradients within rounding of it (the
     attention backward's dQ accumulation order is not fixed in its default mode)."""
     torch, mb = rt
@@ -422,7 +454,7 @@ def test_block_can_be_captured_in_a_cuda_graph_and_replayed(rt):
     inp = make_block_inputs(B, n, H, d, dff, seed=5)
     dev = {k: _dev(torch, v) for k, v in inp.items()}
     blk = TransformerBlock(torch, B, n, H, d, dff, True)
-    w = {k: dev[k] for k in ("g1", "g2", "Wq", "Wk", "Wv", "Wo", "W1", "W3", "W2")}
+    w = blk.prepare_weights({k: dev[k] for k in ("g1", "g2", "Wq", "Wk", "Wv", "Wo", "W1", "W3", "W2")})
     blk.forward(dev["x"], w)
     blk.backward(dev["x"], w, dev["dy"])
     torch.cuda.synchronize()
