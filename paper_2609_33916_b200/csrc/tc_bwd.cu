@@ -10,7 +10,8 @@
 //     dS^T = P^T o (dP^T - D_i)                        (D = rowsum(dO o O); the factor
 //                                                       `scale` of dK and dQ is applied at the end)
 //     dV  += P^T dO_i                (TS-UMMA: P^T bf16 in TMEM, dO_i MN-major in smem)
-//     dK  += dS^T Q_i                (TS-UMMA: dS^T bf16 in TMEM, Q_i MN-major in smem)
+//     dK  += dS^T Q_i                (D = 128: SS-UMMA, the dS^T tile in smem as K-major A, Q_i MN-major;
+//                                     D = 64: TS-UMMA, dS^T bf16 in TMEM)
 //     dQ_i = dS K                    (SS-UMMA: dS^T tile in smem as MN-major A, K MN-major)
 // dQ_i is one key tile's contribution; it is added into an fp32 [B,H,n,d] accumulator (the contended step the
 // dq_mode knob is about): for D = 128 the tile is produced transposed (dQ_i^T = K^T dS^T, lanes = d) and leaves
@@ -23,16 +24,16 @@
 // finished dQ tile out of TMEM and send it to the accumulator, warp 12 TMA producer (K,V once; Q_i with L_i, D_i
 // two tiles ahead in a two-slot ring; dO_i in two slots, or one when the staging buffers of the bulk reduce take
 // the other), warp 13 (one thread) UMMA issuer and TMEM owner.
-// UMMA issue order per query tile: dP(i), dV(i), S(i+1), dK(i), dQ(i), so that the
-// exp2 work of tile i+1 overlaps the dK/dQ UMMAs of tile i and the dS work of tile i
-// overlaps dV(i) and S(i+1).  One thread issues everything: two splits of the issue over two threads
+// UMMA issue order per query tile: dP(i), dV(i), S(i+1), then dQ(i), dK(i) (D = 128; dK(i), dQ(i) for D = 64), so that
+// the exp2 work of tile i+1 overlaps the dK/dQ UMMAs of tile i, the dS work of tile i overlaps dV(i) and S(i+1), and
+// the read-out of dQ(i), which dP(i+1) waits for because the tile sits on the dP^T columns, runs under dK(i).  One thread issues everything: two splits of the issue over two threads
 // ({S, dV} | {dP, dK, dQ} and {S, dP, dV} | {dK, dQ}) were correct and 18-22 % slower, because the second thread's
 // products then share the in-order pipe with the products at the head of the dependency chain
 // dS(i) -> dK(i), dQ(i) -> read-out -> dP(i+1) -> dS(i+1), which is what paces the loop.
 //
 // TMEM columns (512): S^T [0,128), dP^T [128,256), dV [256,256+D), dK [256+D,256+2D);
-// P^T / dS^T (bf16) overwrite the front of their fp32 source columns; for D = 128 the dQ
-// tile reuses the dP^T columns (the UMMAs that read dS^T there are issued before it).
+// P^T (bf16) overwrites the front of its fp32 source columns (for D = 64 so does dS^T); for D = 128 the dQ
+// tile reuses the dP^T columns, which are free once the elementwise threads have read dP^T.
 //
 // Rows past n need no masking: TMA zero-fills K, V, Q, dO there, the preprocess kernel
 // pads L with +inf (so P = 0) and D with 0, and stores are row-guarded.
@@ -175,6 +176,10 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     // 32 consecutive floats of one dQ row: a full 128-byte line per request instead of 32
     // half-used sectors.  (UMMA needs M = 128, so D = 64 keeps lanes = queries.)
     constexpr bool kTransposeDQ = (D == 128);
+    // D = 128: dK(i) reads dS^T from the shared-memory tile (as dQ(i) does) instead of a bf16 copy in TMEM, so that
+    // dQ(i), which lands on the dP^T columns, can be issued FIRST and its read-out runs under dK(i) instead of between
+    // dQ(i) and dP(i+1), on the chain dS(i) -> dQ(i) -> read-out -> dP(i+1) -> dS(i+1) that paces the loop.
+    constexpr bool kDKfromSmem = (D == 128);
     constexpr uint32_t colS = 0, colDP = 128, colDV = 256, colDK = 256 + D, colDQ = kAliasDQ ? 128 : 384;
     extern __shared__ __align__(1024) uint8_t sm[];
     uint8_t *sK = sm + SM::offK, *sV = sm + SM::offV, *sdS = sm + SM::offdS;
@@ -288,7 +293,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
       } else if (warp == kMmaWarp && lane == 0) {
         // the whole role runs in one thread: no warp re-convergence between waits and issues
         // ------------------------------------------------------------------- UMMA issuer
-        // Issue order per query tile i:  dP(i), dV(i), S(i+1), dK(i), dQ(i).
+        // Issue order per query tile i:  dP(i), dV(i), S(i+1), dQ(i), dK(i)  (D = 64: dK(i), dQ(i)).
         constexpr uint32_t idesc_st = idesc_bf16_f32(128, 128, 0, 0);   // S^T, dP^T
         constexpr uint32_t idesc_acc = idesc_bf16_f32(128, D, 0, 1);    // dV, dK: A in TMEM, B MN-major
         constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, 1, 1);     // dQ: A and B MN-major
@@ -304,6 +309,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         auto field = [](const void *ptr) { return (smem_u32(ptr) >> 4) & 0x3FFFu; };
         const uint32_t k_km = km_lo + field(sK), v_km = km_lo + field(sV);            // A of S^T, dP^T
         const uint32_t k_mn = mn_lo + field(sK), ds_mn = mn_lo + field(sdS);          // dQ operands
+        const uint32_t ds_km = km_lo + field(sdS);                                    // dS^T as the K-major A of dK
         const uint32_t q_km0 = km_lo + field(sm + SM::offQ), q_mn0 = mn_lo + field(sm + SM::offQ);
         const uint32_t do_km0 = km_lo + field(sm + SM::offdO), do_mn0 = mn_lo + field(sm + SM::offdO);
         constexpr uint32_t kSlot = (uint32_t)(SM::kTile >> 4);   // address-field step between the two slots
@@ -357,7 +363,23 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             if (!mbar_wait(bars + B_DS, it & 1, abortp, status, ERR_PDS)) break;
             if (!kAliasDQ && !skip_dq && it > 0 && !mbar_wait(bars + B_DQR, (it - 1) & 1, abortp, status, ERR_DQR)) break;
             tc_fence_after();
-            if (lane == 0) {
+            if (lane == 0 && kDKfromSmem) {
+                // dQ^T first (16 keys per step), then dK += dS^T Q_i with dS^T from shared memory (16 queries per step)
+                if (!skip_dq) {
+                    umma_ss2<false>(tbase + colDQ, k_mn, mn_hi, ds_mn, mn_hi, idesc_dqt);
+#pragma unroll
+                    for (int ks = 1; ks < 8; ++ks)
+                        umma_ss2<true>(tbase + colDQ, k_mn + moff(ks), mn_hi, ds_mn + moff(ks), mn_hi, idesc_dqt);
+                }
+                umma_commit(bars + B_DQ);
+                if (it > 0) umma_ss2<true>(tbase + colDK, ds_km, km_hi, q_mn, mn_hi, idesc_acc);
+                else        umma_ss2<false>(tbase + colDK, ds_km, km_hi, q_mn, mn_hi, idesc_acc);
+#pragma unroll
+                for (int ks = 1; ks < 8; ++ks)
+                    umma_ss2<true>(tbase + colDK, ds_km + koff(ks), km_hi, q_mn + moff(ks), mn_hi, idesc_acc);
+                umma_commit(bars + B_QEMPTY + s);   // Q slot (and, on the last tile, everything issued) is done
+            }
+            if (lane == 0 && !kDKfromSmem) {
                 if (it > 0) umma_ts2<true>(tbase + colDK, tbase + colDP, q_mn, mn_hi, idesc_acc);
                 else        umma_ts2<false>(tbase + colDK, tbase + colDP, q_mn, mn_hi, idesc_acc);
 #pragma unroll
@@ -544,7 +566,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                     gk[e / 2] = pack_bf16(g0, g1);
                     gk[e / 2 + 1] = pack_bf16(g2, g3);
                 }
-                tmem_st(lane_addr + colDP + 64 * wg + 16 * c, gk);
+                if (!kDKfromSmem) tmem_st(lane_addr + colDP + 64 * wg + 16 * c, gk);
                 // dS^T row (this key) into the MN-major smem tile: box wg, 128-byte row, swizzled 16-byte chunks
                 uint8_t *rowp = sdS + wg * kBoxBytes + lane_row * 128;
 #pragma unroll
@@ -554,13 +576,14 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                         make_uint4(gk[4 * jj], gk[4 * jj + 1], gk[4 * jj + 2], gk[4 * jj + 3]);
                 }
             }
-            tc_wait_st();
+            if (!kDKfromSmem) tc_wait_st();
             tc_fence_before();
             fence_proxy_async_smem();
             mbar_arrive(bars + B_DS);
             if (it + 1 < niter) ok = p_phase(it + 1);
         }
-        if (ok && mbar_wait(bars + B_DQ, (niter - 1) & 1, abortp, status, ERR_DQ)) {
+        if (ok && mbar_wait(bars + B_DQ, (niter - 1) & 1, abortp, status, ERR_DQ) &&
+            (!kDKfromSmem || mbar_wait(bars + B_QEMPTY + ((niter - 1) & 1), ((niter - 1) >> 1) & 1, abortp, status, ERR_DQ))) {
             // All UMMAs have completed.  dV and scale*dK go out as bf16 through shared memory (the K and V
             // tiles are no longer read) and TMA stores: a thread owns a row, so direct stores would be 16
             // bytes at a 2D-byte stride, one 128-byte line per lane and instruction -- 4096 line requests
