@@ -8,7 +8,8 @@
 //              accumulator, so the two halves are independent online-softmax streams that are
 //              merged only in the epilogue.  Per tile: 64 fp32 scores from TMEM into registers,
 //              max (3-input, independent chains), exp2 + row sum on packed fp32 pairs, bf16 P back
-//              into TMEM over the front of the same score columns; O_h in TMEM is rescaled only
+//              into TMEM over the front of the same score columns (handed to the P V issuer 32 keys at a
+//              time, so that its first UMMAs run under the second half of the exponentials); O_h in TMEM is rescaled only
 //              when the max has grown by more than 8 (log2 domain).
 //   warp 8     TMA producer: Q once, K and V tiles in two-slot rings.
 //   warp 9     UMMA issuer (one thread) for S = Q K^T (SS, both operands K-major), into two
@@ -55,7 +56,8 @@ enum : uint32_t { ERR_Q = 0x101, ERR_K = 0x102, ERR_V = 0x103, ERR_S = 0x104, ER
 
 enum { F_Q = 0, F_KFULL = 1 /*2*/, F_KEMPTY = 3 /*2*/, F_VFULL = 5 /*2*/, F_VEMPTY = 7 /*2*/, F_S = 9 /*2*/,
        F_P = 11 /*[buffer][half]: 4*/, F_O = 15, F_X = 16 /*epilogue exchange*/, F_OB = 17 /*2: score buffer consumed*/,
-       F_E = 19 /*O tile staged in shared memory*/, F_DONE = 20 /*last P V of the job has completed*/, F_COUNT = 21 };
+       F_E = 19 /*O tile staged in shared memory*/, F_DONE = 20 /*last P V of the job has completed*/,
+       F_P2 = 21 /*[buffer][half]: 4, the second 32 keys of a half*/, F_COUNT = 25 };
 
 // Split use of the kernel (decode: few query rows, a long cache): the key tiles are divided among
 // `splits` CTAs per (head, query tile); each writes the attention over its tiles alone (normalised O
@@ -109,7 +111,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     const int nkt_want = causal ? min(qt + 1, nkt_all) : min(sp.tiles_per_split, nkt_all - kt0);
 
     if (tid == 0) {
-        for (int b = 0; b < F_COUNT; ++b) mbar_init(bars + b, (b >= F_P && b < F_P + 4) ? 128u : ((b == F_X || b == F_E) ? 256u : 1u));
+        for (int b = 0; b < F_COUNT; ++b) mbar_init(bars + b, ((b >= F_P && b < F_P + 4) || (b >= F_P2 && b < F_P2 + 4)) ? 128u : ((b == F_X || b == F_E) ? 256u : 1u));
         *abortp = (smem_u32(sm) & 1023u) ? 1u : 0u;
         if (*abortp && status) atomicCAS(status, 0u, 0x108u);
         fence_mbar_init();
@@ -235,10 +237,14 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 if (!mbar_wait(bars + F_P + 2 * b + h, (j >> 1) & 1, abortp, status, ERR_P)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t ocol = tbase + kColO + h * D, acol = pcol + 64 * h, vh = v_lo + (uint32_t)((h * 4 * 2048) >> 4);
+                // the first 32 keys of the half as soon as they are written, the other 32 when they are
                 if (j > 0) umma_ts2<true>(ocol, acol, vh, mn_hi, idesc_pv);
                 else       umma_ts2<false>(ocol, acol, vh, mn_hi, idesc_pv);
+                umma_ts2<true>(ocol, acol + 8, vh + (uint32_t)(2048 >> 4), mn_hi, idesc_pv);
+                if (!mbar_wait(bars + F_P2 + 2 * b + h, (j >> 1) & 1, abortp, status, ERR_P)) { ok = false; break; }
+                tc_fence_after();
 #pragma unroll
-                for (int ks = 1; ks < 4; ++ks)
+                for (int ks = 2; ks < 4; ++ks)
                     umma_ts2<true>(ocol, acol + ks * 8, vh + (uint32_t)((ks * 2048) >> 4), mn_hi, idesc_pv);
             }
             if (!ok) break;
@@ -342,6 +348,11 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                     pk[i / 2] = pack_bf16(p0, p1);
                 }
                 tmem_st(lane_addr + scol + 16 * c, pk);
+                if (c == 0) {       // the first 32 keys can enter the P V product while the others are exponentiated
+                    tc_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(bars + F_P + 2 * (j & 1) + h);
+                }
             }
             {
                 float s0, s1, s2, s3;
@@ -351,7 +362,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             }
             tc_wait_st();
             tc_fence_before();
-            mbar_arrive(bars + F_P + 2 * (j & 1) + h);
+            mbar_arrive(bars + F_P2 + 2 * (j & 1) + h);
         }
         // ---- epilogue: merge the two key halves.  Each thread publishes (m, l) of its half, then
         // writes D/2 output columns of its row from both accumulators.
