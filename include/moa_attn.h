@@ -31,6 +31,11 @@
  *  - Calls enqueue kernels on `stream` (a cudaStream_t passed as void*; NULL is
  *    the legacy default stream) and return without synchronising the host.
  *  - Outputs are overwritten, never accumulated into.
+ *  - A call is one to four kernels in stream order.  The tensor-core backward kernel and the dQ conversion are
+ *    launched as programmatic dependents of the kernel in front of them (they set themselves up while it drains and
+ *    wait for its completion before reading or adding to anything it wrote); the first kernel of every call is an
+ *    ordinary launch, so a call never starts before work the caller enqueued earlier has finished.  MOA_PDL=0 in the
+ *    environment (read once per process) launches everything in plain stream order.
  *  - Errors are reported only through the returned moa_status; the library does
  *    not abort or throw.  Argument, workspace, scratch-limit and architecture errors
  *    are found before anything is enqueued.  MOA_ERR_CUDA can come from a later

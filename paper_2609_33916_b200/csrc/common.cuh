@@ -121,6 +121,26 @@ struct LaunchScope {
     cudaStream_t st;
 };
 
+// Launch `kernel` so that it may start before the kernel in front of it in the stream has finished (programmatic
+// dependent launch): the kernel itself calls ptx::grid_dependency_wait() before it touches anything that kernel
+// wrote.  MOA_PDL=0 in the environment turns the attribute off (plain stream order).
+bool pdl_enabled();
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = pdl_enabled() ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // Device address of the status word kernels write when a bounded wait expires.
 unsigned int *device_status_ptr();
 

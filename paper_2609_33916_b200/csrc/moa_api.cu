@@ -67,6 +67,12 @@ unsigned int *device_status_ptr()
     return cache[dev];
 }
 
+bool pdl_enabled()
+{
+    static const bool on = [] { const char *e = getenv("MOA_PDL"); return !(e && e[0] == '0'); }();
+    return on;
+}
+
 const DeviceInfo &device_info()
 {
     constexpr int kMaxDev = 64;
@@ -595,6 +601,7 @@ moa_status moa_profile_read(moa_profile *out)
 }
 
 int moa_bwd_pair_mode(int mode) { return bwd_pair_mode(mode); }
+
 
 uint64_t moa_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

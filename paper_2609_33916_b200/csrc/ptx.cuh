@@ -34,6 +34,14 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t by
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
+// Programmatic dependent launch.  A kernel launched with the programmatic-stream-serialization attribute may start while
+// the kernel before it in the stream is still running; grid_dependency_wait() then blocks until that kernel has completed and
+// its memory operations are visible (without the attribute it returns at once).  grid_launch_dependents() tells the
+// scheduler that, as far as this CTA is concerned, the next kernel's CTAs may be started (they are, once every CTA of this grid
+// has said so or exited, on whatever SM resources are free).
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ void mbar_arrive(uint64_t *bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");

@@ -570,6 +570,7 @@ simt_rowpar_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__
 __global__ void __launch_bounds__(256)
 convert_kernel(const float *__restrict__ src, __nv_bfloat16 *__restrict__ dst, size_t count, float mul)
 {
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // launched as a programmatic dependent of the kernel that fills src
     const size_t quads = count / 4;
     const size_t stride = (size_t)gridDim.x * blockDim.x;
     size_t q = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -597,6 +598,7 @@ __global__ void __launch_bounds__(256)
 convert_rows_kernel(const float *__restrict__ src, int src_ld, __nv_bfloat16 *__restrict__ dst, size_t rows, int n, int H,
                     int d, Strides ds, float mul)
 {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int quads_per_row = d / 4;
     const size_t total = rows * (size_t)quads_per_row;
     const size_t stride = (size_t)gridDim.x * blockDim.x;
@@ -744,8 +746,7 @@ cudaError_t convert_f32_to_bf16(const float *src, void *dst, size_t count, float
     if (blocks > 16LL * device_info().sms) blocks = 16LL * device_info().sms;     // grid-stride beyond 16 blocks per SM
     const unsigned grid = (unsigned)blocks;
     LaunchScope scope(MOA_KERNEL_CONVERT, st);
-    convert_kernel<<<grid, 256, 0, st>>>(src, (__nv_bfloat16 *)dst, count, mul);
-    return cudaGetLastError();
+    return launch_dependent(convert_kernel, dim3(grid), dim3(256), (size_t)0, st, src, (__nv_bfloat16 *)dst, count, mul);
 }
 
 cudaError_t convert_f32_to_bf16_rows(const float *src, int src_ld, void *dst, int B, int H, int n, int d, Strides ds,
@@ -756,8 +757,8 @@ cudaError_t convert_f32_to_bf16_rows(const float *src, int src_ld, void *dst, in
     if (blocks < 1) blocks = 1;
     if (blocks > 16LL * device_info().sms) blocks = 16LL * device_info().sms;
     LaunchScope scope(MOA_KERNEL_CONVERT, st);
-    convert_rows_kernel<<<(unsigned)blocks, 256, 0, st>>>(src, src_ld, (__nv_bfloat16 *)dst, rows, n, H, d, ds, mul);
-    return cudaGetLastError();
+    return launch_dependent(convert_rows_kernel, dim3((unsigned)blocks), dim3(256), (size_t)0, st, src, src_ld, (__nv_bfloat16 *)dst, rows, n, H, d,
+                            ds, mul);
 }
 
 }  // namespace moa

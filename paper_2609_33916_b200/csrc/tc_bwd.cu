@@ -78,6 +78,7 @@ bwd_preprocess_kernel(const __nv_bfloat16 *__restrict__ dO, const __nv_bfloat16 
                       int n, int n_pad, size_t padded_rows, int H, Strides so, int d)
 {
     // d <= D: the head dimension in memory (lanes past it contribute zeros)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // the backward kernel behind this one may set itself up
     constexpr int kLanesPerRow = D / 8;
     constexpr int kRowsPerPass = 32 / kLanesPerRow;
     constexpr int kPasses = 4;
@@ -234,6 +235,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    grid_launch_dependents();      // the dQ conversion that follows may be set up while this grid drains
     const uint32_t tbase = *tmem_base_s;
     // a misaligned shared-memory base (swizzled tiles would be misplaced) turns every role into a no-op
     const int niter = (*abortp == 0) ? niter_all : 0;
@@ -256,13 +258,17 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         // Q tiles (with L, D) go through a two-slot ring and are fetched two tiles ahead: S(i+1) is
         // issued in the middle of tile i.  dO has one slot: it is read only by dP(i) and dV(i),
         // early in tile i, and is refilled as soon as dV(i) has completed.
+        // K, V, Q and dO are the caller's tensors; L', D and the cleared dQ accumulator were written by the kernel in front of
+        // this one in the stream (the forward or the preprocess kernel), which may still be running: the first tiles are
+        // requested, then this warp waits for that kernel before it asks for L' and D.
         TileWalk wq = walk0, wdo = walk0;     // load_q and load_do are each called for it = 0, 1, 2, ... in order
-        auto load_q = [&](int it) {
+        auto load_q = [&](int it, bool wait_first) {
             const int s = it & 1, q0 = wq.qi * 128, qh = wq.qh;
             wq.next();
             uint8_t *sQ = sm + SM::offQ + s * SM::kTile;
             mbar_arrive_expect_tx(bars + B_QFULL + s, SM::kTile + 1024);
             for (int b = 0; b < kBoxes; ++b) tma_load_4d(sQ + b * kBoxBytes, &mapQ, bars + B_QFULL + s, 64 * b, q0, qh + hq0, bb);
+            if (wait_first) grid_dependency_wait();
             bulk_load_1d(sL + s * 128, Lp + (size_t)qh * n_pad + q0, 512, bars + B_QFULL + s);
             bulk_load_1d(sD + s * 128, Dp + (size_t)qh * n_pad + q0, 512, bars + B_QFULL + s);
         };
@@ -274,11 +280,12 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             for (int b = 0; b < kBoxes; ++b) tma_load_4d(sdO + b * kBoxBytes, &mapdO, bars + B_DOFULL + s, 64 * b, q0, qh + hq0, bb);
         };
         if (lane == 0 && niter > 0) {
-            load_q(0);
             load_do(0);
-            if (niter > 1) load_q(1);
             if (kDoSlots == 2 && niter > 1) load_do(1);
+            load_q(0, true);
+            if (niter > 1) load_q(1, false);
         }
+        grid_dependency_wait();     // (the lanes that issued nothing, and a CTA without tiles)
         for (int it = 0; it < niter; ++it) {
             if (it + kDoSlots < niter) {     // dV(it) done: its dO slot takes tile it + kDoSlots
                 if (!mbar_wait(bars + B_DOEMPTY + it % kDoSlots, (it / kDoSlots) & 1, abortp, status, ERR_EMPTY)) break;
@@ -286,7 +293,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             }
             if (it + 2 < niter) {     // dK(it) done: its Q slot takes tile it+2
                 if (!mbar_wait(bars + B_QEMPTY + (it & 1), (it >> 1) & 1, abortp, status, ERR_EMPTY)) break;
-                if (lane == 0) load_q(it + 2);
+                if (lane == 0) load_q(it + 2, false);
             }
             __syncwarp();
         }
@@ -406,6 +413,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     } else if (warp >= kReduceWarp0) {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 144;");
         // ------------------------------------------------- dQ reduce warps: lanes are query rows
+        grid_dependency_wait();      // the accumulator these warps add into was cleared by the kernel in front
         const int lane_row = 32 * (warp % 4) + lane;
         const uint32_t lane_addr = tbase + ((uint32_t)(32 * (warp % 4)) << 16);
         TileWalk wr = walk0;
@@ -668,10 +676,9 @@ cudaError_t launch_bwd_g(const Problem &p, const void *Q, const void *K, const v
     Problem pkv = p;
     pkv.H = p.kv_heads();
     pkv.Hkv = 0;
-    tc_bwd_kernel<D, kBulk, kGrouped><<<(unsigned)(nkt * p.BHkv()), kThreads, kSmem, st>>>(
-        mq, mk, mv, mdo, mdq, mdk, mdv, Lp, Dp, dQacc, p.n, nkt * 128, p.causal,
-        p.scale, p.scale * kLog2e, nkt, heads_per_group(pkv, nkt), p.group(), p.kv_heads(), dQacc == nullptr ? 1 : 0, device_status_ptr());
-    return cudaGetLastError();
+    return launch_dependent(tc_bwd_kernel<D, kBulk, kGrouped>, dim3((unsigned)(nkt * p.BHkv())), dim3(kThreads), (size_t)kSmem, st,
+                            mq, mk, mv, mdo, mdq, mdk, mdv, Lp, Dp, dQacc, p.n, nkt * 128, p.causal, p.scale, p.scale * kLog2e, nkt,
+                            heads_per_group(pkv, nkt), p.group(), p.kv_heads(), dQacc == nullptr ? 1 : 0, device_status_ptr());
 }
 
 template <int D, bool kBulk>

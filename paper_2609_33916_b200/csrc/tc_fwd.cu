@@ -121,6 +121,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    grid_launch_dependents();      // the backward that follows may set itself up on SMs this grid no longer needs
     const uint32_t tbase = *tmem_base_p;
     const int nkt = (*abortp == 0) ? nkt_want : 0;   // misaligned shared memory: every role is a no-op
 

@@ -2,6 +2,7 @@
 oracle on the same seeded inputs.  Bar: max|err|/max|ref| <= 1e-2 per output for
 bf16 storage (fp32 accumulation), <= 1e-5 for the fp32 path."""
 import math
+import os
 
 import numpy as np
 import pytest
@@ -450,3 +451,22 @@ def test_fused_call_can_be_captured_in_a_cuda_graph_and_replayed(H):
     for a, b, name in zip(got, (O, L, dQ, dK, dV), ("O", "L", "dQ", "dK", "dV")):
         assert torch.equal(a, b), name
     assert mb.moa_last_device_status() == mb.MOA_OK
+
+
+def test_parity_tests_pass_without_programmatic_dependent_launch():
+    """The backward and the dQ conversion are launched as programmatic dependents of the kernel in front of them (they set
+    themselves up while it drains and wait for it before touching what it wrote); MOA_PDL=0 launches them in plain stream
+    order.  A selection of the tests above, in a child process with the switch off."""
+    import subprocess
+    import sys
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, MOA_PDL="0")
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.abspath(__file__), "-x", "-q", "-m", "gpu",
+                        "-k", "bf16_shapes or gqa_matches or c3_causal", "-p", "no:cacheprovider"],
+                       cwd=root, env=env, capture_output=True, text=True, timeout=1200)
+    tail = (r.stdout or "")[-1500:] + (r.stderr or "")[-500:]
+    assert r.returncode == 0, tail
+    assert " passed" in r.stdout and " failed" not in r.stdout, tail
