@@ -2,31 +2,35 @@
 // fp32 accumulate.
 //
 // One CTA (one per SM) owns 128 query rows of one (batch, head) and walks the key/value
-// tiles of 128 keys.  Roles (352 threads):
-//   warps 0-7  softmax: thread = query row = TMEM lane; warpgroup h = warp / 4 owns key
-//              columns [64h, 64h+64) of every tile with its own running max, row sum and O
-//              accumulator, so the two halves are independent online-softmax streams that are
-//              merged only in the epilogue.  Per tile: 64 fp32 scores from TMEM into registers,
-//              max (3-input, independent chains), exp2 + row sum on packed fp32 pairs, bf16 P back
-//              into TMEM over the front of the same score columns (handed to the P V issuer 32 keys at a
-//              time, so that its first UMMAs run under the second half of the exponentials); O_h in TMEM is rescaled only
-//              when the max has grown by more than 8 (log2 domain).
-//   warp 8     TMA producer: Q once, K and V tiles in two-slot rings.
-//   warp 9     UMMA issuer (one thread) for S = Q K^T (SS, both operands K-major), into two
-//              alternating score buffers: S(j+1) is computed while the softmax works on S(j).
-//   warp 10    UMMA issuer (one thread) for O_h += P_h V (TS: P from TMEM, V MN-major in smem).
-// Two issuing threads because a barrier probe or a commit costs an issuer ~100 cycles in which
-// it feeds nothing and the tensor pipe queues only a few UMMAs; UMMAs of different threads are
-// unordered, so the one hazard between the streams (S(j) overwriting the buffer that held
-// P(j-2)) goes through an mbarrier.
-// TMEM (512 columns): score buffers [0,128) and [128,256), O_0 [256,256+D), O_1 [256+D,256+2D).
-// S, P and the O accumulators never leave the SM: nothing of size n x n reaches HBM.
+// tiles of 128 keys.  Roles (384 threads; registers re-split with setmaxnreg: 208 for the softmax
+// warpgroups, 88 for the rest):
+//   warps 0-7  softmax: thread = query row = TMEM lane.  Warpgroup h = warp / 4 takes the key tiles
+//              j = h, h + 2, ... whole -- 128 fp32 scores from TMEM into registers, max (3-input,
+//              independent chains), exp2 + row sum on packed fp32 pairs, bf16 P into the stream's own
+//              64 TMEM columns -- with its own running max, row sum and O accumulator: two independent
+//              online-softmax streams, merged only in the epilogue; O_h in TMEM is rescaled only when
+//              the max has grown by more than 8 (log2 domain).
+//   warp 8     TMA producer of Q (once) and of the K ring; warp 11 of the V ring (a thread each: the K
+//              ring follows the score products, the V ring the P V products, and a single producer made
+//              the next K tile wait for a V slot, i.e. for a P V product).
+//   warp 9     UMMA issuer (one thread) for S = Q K^T (SS, both operands K-major) into the ONE score
+//              buffer: S(j+1) is issued as soon as the warpgroup of tile j holds that tile's scores in
+//              registers, and runs under tile j's exponentials.
+//   warp 10    UMMA issuer (one thread) for O_h += P V (TS: P from TMEM, V MN-major in smem).  It lets
+//              S(j+2) through the pipe before it issues P V(j): the warpgroup that waits for those scores
+//              has nothing else to do, and UMMAs of two threads issued together interleave, so that both
+//              products take twice as long.
+// The two warpgroups take turns on the score buffer, so one is in its exp2 loop while the other waits,
+// loads and takes its maxima; with both working on halves of the same tile (the earlier form of this
+// kernel) the two exp2 loops ran together, the MUFU unit was saturated during them and idle otherwise.
+// UMMAs of different threads are unordered; every hazard between them goes through an mbarrier.
+// TMEM (512 columns): scores [0,128), P of stream 0 / 1 [128,192) / [192,256), O_0 [256,256+D),
+// O_1 [256+D,256+2D).  S, P and the O accumulators never leave the SM: nothing of size n x n reaches HBM.
 //
-// What bounds it (config 4, d = 128): per 128 x 128 tile the UMMAs need 1024 cycles, the one exp2
-// per score 1024 cycles of the MUFU unit, and shared memory 1250 cycles (an SS UMMA streams both
-// operands at the full 128 B/clk: 64 KB for S, 32 KB of V for PV, 64 KB of TMA writes); the tile
-// takes ~1850 because the two softmax warpgroups run their exp2 phases at the same time and the
-// rest of their work (TMEM load, max, hand-offs, ~600 cycles) is not hidden under them.
+// What bounds it (config 4, d = 128): per 128 x 128 tile the UMMAs need 1024 cycles and the one exp2 per
+// score 1024 cycles of the MUFU unit; a warpgroup is busy about 2650 cycles per tile of its own (load 220,
+// maxima 620, exp2 loop 1750 when the other warpgroup's loop overlaps it, hand-off 65), i.e. 1330 per tile
+// with two of them, and the tile takes about 1550.
 // The O tile leaves through the Q tile's shared memory and a TMA store.
 //
 // Head dimensions 136..256 (KC = 2): the scores need the whole head dimension, the output does not.  S = Q K^T is
@@ -45,19 +49,23 @@ using namespace ptx;
 
 constexpr int BM = 128;            // query rows per CTA
 constexpr int BN = 128;            // keys per tile
-constexpr int kThreads = 352;      // warps 0-7 softmax, 8 TMA, 9 UMMA issuer for S, 10 UMMA issuer for PV
-constexpr int kTmemCols = 512;     // two score buffers: columns [0,128), [128,256); two O accumulators from 256
-constexpr uint32_t kColS = 0, kColO = 256;
+constexpr int kThreads = 384;      // warps 0-7 softmax, 8 TMA, 9 UMMA issuer for S, 10 UMMA issuer for PV, 11 idle
+constexpr int kTmemCols = 512;     // scores [0,128); bf16 P of the two streams [128,192), [192,256); two O accumulators from 256
+constexpr uint32_t kColS = 0, kColP = 128, kColO = 256;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.f;
 
 enum : uint32_t { ERR_Q = 0x101, ERR_K = 0x102, ERR_V = 0x103, ERR_S = 0x104, ERR_P = 0x105, ERR_O = 0x106 };
 
-enum { F_Q = 0, F_KFULL = 1 /*2*/, F_KEMPTY = 3 /*2*/, F_VFULL = 5 /*2*/, F_VEMPTY = 7 /*2*/, F_S = 9 /*2*/,
-       F_P = 11 /*[buffer][half]: 4*/, F_O = 15, F_X = 16 /*epilogue exchange*/, F_OB = 17 /*2: score buffer consumed*/,
-       F_E = 19 /*O tile staged in shared memory*/, F_DONE = 20 /*last P V of the job has completed*/,
-       F_P2 = 21 /*[buffer][half]: 4, the second 32 keys of a half*/, F_COUNT = 25 };
+enum { F_Q = 0, F_KFULL = 1 /*2*/, F_KEMPTY = 3 /*2*/, F_VFULL = 5 /*2*/, F_VEMPTY = 7 /*2*/, F_S_UNUSED = 9 /*2*/,
+       F_P = 11 /*2: per stream*/, F_SFREE = 13 /*2: per stream, the tile's scores are in registers*/, F_O = 15 /*unused*/,
+       F_X = 16 /*epilogue exchange*/, F_OB = 17 /*2: per stream, P V of the stream's tile has completed*/,
+       F_E = 19 /*O tile staged in shared memory*/, F_DONE = 20 /*last P V of the job has completed*/, 
+       F_S = 21 /*[stream][tile count of the stream & 1]: 4.  Two barriers per stream, taken in turn: the P V issuer, which
+                  lets S(j+2) pass before it issues P V(j), may be stalled on the V ring while the scores run two tiles of
+                  the stream ahead of it, and a parity wait must never fall two phases of one barrier behind*/,
+       F_COUNT = 25 };
 
 // Split use of the kernel (decode: few query rows, a long cache): the key tiles are divided among
 // `splits` CTAs per (head, query tile); each writes the attention over its tiles alone (normalised O
@@ -111,7 +119,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     const int nkt_want = causal ? min(qt + 1, nkt_all) : min(sp.tiles_per_split, nkt_all - kt0);
 
     if (tid == 0) {
-        for (int b = 0; b < F_COUNT; ++b) mbar_init(bars + b, ((b >= F_P && b < F_P + 4) || (b >= F_P2 && b < F_P2 + 4)) ? 128u : ((b == F_X || b == F_E) ? 256u : 1u));
+        for (int b = 0; b < F_COUNT; ++b)
+            mbar_init(bars + b, ((b >= F_P && b < F_P + 2) || (b >= F_SFREE && b < F_SFREE + 2)) ? 128u : ((b == F_X || b == F_E) ? 256u : 1u));
         *abortp = (smem_u32(sm) & 1023u) ? 1u : 0u;
         if (*abortp && status) atomicCAS(status, 0u, 0x108u);
         fence_mbar_init();
@@ -121,13 +130,18 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    grid_launch_dependents();      // the backward that follows may set itself up on SMs this grid no longer needs
     const uint32_t tbase = *tmem_base_p;
     const int nkt = (*abortp == 0) ? nkt_want : 0;   // misaligned shared memory: every role is a no-op
 
-    if (warp == 8) {
+    // 384 threads start with 168 registers each; the last warpgroup (TMA, the two issuers, an idle warp) gives most of its
+    // share to the softmax warpgroups, whose threads hold the 128 scores of a row.  The two counts must add up to what the
+    // CTA was launched with (128 x 88 + 256 x 208 = 384 x 168): an increase that asks for more than the decrease frees
+    // waits for registers forever.
+    if (warp >= 8) {
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
+      if (warp == 8) {
         // ------------------------------------------------------------------ TMA producer
-        int nk = 0, nv = 0;     // K and V tiles requested so far (slot = count & 1)
+        int nk = 0;             // K chunks requested so far (slot = count & 1)
         if (lane == 0 && nkt > 0) {
             mbar_arrive_expect_tx(bars + F_Q, KC * kTileBytes);
             for (int b = 0; b < KC * kBoxes; ++b) tma_load_4d(sQ + b * kBoxBytes, &mapQ, bars + F_Q, 64 * b, q0, hq, bb);
@@ -140,24 +154,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             for (int b = 0; b < kBoxes; ++b)
                 tma_load_4d(sK + s * kTileBytes + b * kBoxBytes, &mapK, bars + F_KFULL + s, D * c + 64 * b, (kt0 + j) * BN, hk, bb);
         };
-        auto load_v = [&](int j) {            // this CTA's column half of V tile j
-            const int s = j & 1;
-            mbar_arrive_expect_tx(bars + F_VFULL + s, kTileBytes);
-            ++nv;
-            for (int b = 0; b < kBoxes; ++b)
-                tma_load_4d(sV + s * kTileBytes + b * kBoxBytes, &mapV, bars + F_VFULL + s, D * pass + 64 * b, (kt0 + j) * BN, hk, bb);
-        };
         if (zero_acc != nullptr) {
             // Fused forward+backward (KC = 1): this CTA's 128 rows of the fp32 dQ accumulator ([B*H, n, D]) are
             // cleared here, by the producer warp while its first loads are in flight (the next slot
             // frees two tiles from now), so that the step needs no separate clearing pass.
             // The first two K/V tiles are requested first: they have no slot to wait for.
-            for (int j = 0; j < min(nkt, 2); ++j) {
-                if (lane == 0) {
-                    load_k(j);
-                    load_v(j);
-                }
-            }
+            for (int j = 0; j < min(nkt, 2); ++j)
+                if (lane == 0) load_k(j);
             const int rows = min(BM, n - q0);
             float4 *dst = reinterpret_cast<float4 *>(zero_acc + ((size_t)bh * n + q0) * D);
             for (int i = lane; i < rows * (D / 4); i += 32) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -170,19 +173,32 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 if (lane == 0) load_k(g);
             }
             if (!live) break;
-            if (j >= 2 && !mbar_wait(bars + F_VEMPTY + (j & 1), ((j >> 1) - 1) & 1, abortp, status, ERR_V)) break;
-            if (lane == 0) load_v(j);
             __syncwarp();
         }
         if (lane == 0 && *abortp) {
             // a wait expired somewhere in the CTA: copies still on their way land before it leaves (bounded)
             mbar_drain_one(bars + F_Q, nkt > 0 ? 1 : 0);
-            for (int s = 0; s < 2; ++s) {
-                mbar_drain_one(bars + F_KFULL + s, nk > s ? (nk - s + 1) / 2 : 0);
-                mbar_drain_one(bars + F_VFULL + s, nv > s ? (nv - s + 1) / 2 : 0);
-            }
+            for (int s = 0; s < 2; ++s) mbar_drain_one(bars + F_KFULL + s, nk > s ? (nk - s + 1) / 2 : 0);
         }
-    } else if (warp == 9 && lane == 0) {
+      } else if (warp == 11) {
+        // ------------------------------------------------------------------ TMA producer of the V stream
+        // (a thread of its own: the V ring follows the P V products, the K ring the score products, and neither waits
+        // for the other's slots)
+        int nv = 0;
+        for (int j = 0; j < nkt; ++j) {
+            if (j >= 2 && !mbar_wait(bars + F_VEMPTY + (j & 1), ((j >> 1) - 1) & 1, abortp, status, ERR_V)) break;
+            if (lane == 0) {
+                const int s = j & 1;
+                mbar_arrive_expect_tx(bars + F_VFULL + s, kTileBytes);
+                ++nv;
+                for (int b = 0; b < kBoxes; ++b)
+                    tma_load_4d(sV + s * kTileBytes + b * kBoxBytes, &mapV, bars + F_VFULL + s, D * pass + 64 * b, (kt0 + j) * BN, hk, bb);
+            }
+            __syncwarp();
+        }
+        if (lane == 0 && *abortp)
+            for (int s = 0; s < 2; ++s) mbar_drain_one(bars + F_VFULL + s, nv > s ? (nv - s + 1) / 2 : 0);
+      } else if (warp == 9 && lane == 0) {
         // ------------------------------------------- UMMA issuer for the score GEMMs (one thread)
         // Two issuing threads (this one for S = Q K^T, warp 10 for O += P V): a successful barrier
         // probe or a commit costs an issuing thread ~100 cycles during which it feeds nothing, and
@@ -198,14 +214,14 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         constexpr uint32_t kSlot = (uint32_t)(kTileBytes >> 4);
         bool ok = nkt > 0 && mbar_wait(bars + F_Q, 0, abortp, status, ERR_Q);
         for (int j = 0; ok && j < nkt; ++j) {
-            const int b = j & 1;
-            const uint32_t dcol = tbase + kColS + 128 * b;
+            const uint32_t dcol = tbase + kColS;
 #pragma unroll
             for (int c = 0; c < KC; ++c) {          // the contraction over the head dimension, 128 columns per K chunk
                 const int g = j * KC + c, sl = g & 1;
                 const uint32_t k_lo = k_lo0 + sl * kSlot, q_c = q_lo + c * kSlot;
                 if (!mbar_wait(bars + F_KFULL + sl, (g >> 1) & 1, abortp, status, ERR_K)) { ok = false; break; }
-                if (c == 0 && j >= 2 && !mbar_wait(bars + F_OB + b, ((j >> 1) - 1) & 1, abortp, status, ERR_O)) { ok = false; break; }
+                // the one score buffer is free once the warpgroup of tile j-1 holds that tile's scores in registers
+                if (c == 0 && j >= 1 && !mbar_wait(bars + F_SFREE + ((j - 1) & 1), ((j - 1) >> 1) & 1, abortp, status, ERR_O)) { ok = false; break; }
                 tc_fence_after();
                 if (c == 0) umma_ss2<false>(dcol, q_c, km_hi, k_lo, km_hi, idesc_s);
                 else        umma_ss2<true>(dcol, q_c, km_hi, k_lo, km_hi, idesc_s);
@@ -217,9 +233,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 umma_commit(bars + F_KEMPTY + sl);
             }
             if (!ok) break;
-            umma_commit(bars + F_S + b);
+            umma_commit(bars + F_S + 2 * (j & 1) + ((j >> 1) & 1));
         }
-    } else if (warp == 10 && lane == 0) {
+      } else if (warp == 10 && lane == 0) {
         // ------------------------------------------------ UMMA issuer for O += P V (one thread)
         constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, 0, 1);
         const uint64_t mn_proto = smem_desc_sw128(0, kBoxBytes, 1024);
@@ -227,44 +243,40 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         const uint32_t v_lo0 = (uint32_t)mn_proto + ((smem_u32(sV) >> 4) & 0x3FFFu);
         constexpr uint32_t kSlot = (uint32_t)(kTileBytes >> 4);
         for (int j = 0; j < nkt; ++j) {
-            const int b = j & 1;
-            const uint32_t v_lo = v_lo0 + b * kSlot, pcol = tbase + kColS + 128 * b;
+            const int b = j & 1;        // V ring slot and stream of tile j
+            const uint32_t v_lo = v_lo0 + b * kSlot, acol = tbase + kColP + 64 * b, ocol = tbase + kColO + b * D;
             if (!mbar_wait(bars + F_VFULL + b, (j >> 1) & 1, abortp, status, ERR_V)) break;
-            bool ok = true;
-            // key half h of the tile: P_h (64 keys = 32 TMEM columns at the front of that half of the
-            // score buffer) times V rows 64h.., into its own accumulator O_h
+            if (!mbar_wait(bars + F_P + b, (j >> 1) & 1, abortp, status, ERR_P)) break;
+            // The scores come first: this product waits until S(j+2), which is issued the moment tile j+1's scores are in
+            // registers, is through the pipe (two issuing threads' UMMAs interleave and both products take twice as long).
+            if (j + 2 < nkt && !mbar_wait(bars + F_S + 2 * (j & 1) + (((j + 2) >> 1) & 1), ((j + 2) >> 2) & 1, abortp, status, ERR_S)) break;
+            tc_fence_after();
+            // O_b (+)= P(j) V(j): 128 keys = eight k-steps; P (bf16) is 64 TMEM columns, V rows 16 ks .. 16 ks + 15
+            if (j > 1) umma_ts2<true>(ocol, acol, v_lo, mn_hi, idesc_pv);
+            else       umma_ts2<false>(ocol, acol, v_lo, mn_hi, idesc_pv);      // the stream's first tile
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                if (!mbar_wait(bars + F_P + 2 * b + h, (j >> 1) & 1, abortp, status, ERR_P)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t ocol = tbase + kColO + h * D, acol = pcol + 64 * h, vh = v_lo + (uint32_t)((h * 4 * 2048) >> 4);
-                // the first 32 keys of the half as soon as they are written, the other 32 when they are
-                if (j > 0) umma_ts2<true>(ocol, acol, vh, mn_hi, idesc_pv);
-                else       umma_ts2<false>(ocol, acol, vh, mn_hi, idesc_pv);
-                umma_ts2<true>(ocol, acol + 8, vh + (uint32_t)(2048 >> 4), mn_hi, idesc_pv);
-                if (!mbar_wait(bars + F_P2 + 2 * b + h, (j >> 1) & 1, abortp, status, ERR_P)) { ok = false; break; }
-                tc_fence_after();
-#pragma unroll
-                for (int ks = 2; ks < 4; ++ks)
-                    umma_ts2<true>(ocol, acol + ks * 8, vh + (uint32_t)((ks * 2048) >> 4), mn_hi, idesc_pv);
-            }
-            if (!ok) break;
+            for (int ks = 1; ks < 8; ++ks)
+                umma_ts2<true>(ocol, acol + ks * 8, v_lo + (uint32_t)((ks * 2048) >> 4), mn_hi, idesc_pv);
             umma_commit(bars + F_OB + b);
             umma_commit(bars + F_VEMPTY + b);
-            umma_commit(bars + F_O);
             if (j == nkt - 1) umma_commit(bars + F_DONE);
         }
-    } else if (warp < 8) {
+      }
+    } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
         // ---------------------------------------------------------------- softmax warps
-        // Thread = query row (TMEM lane); warpgroup h = warp / 4 owns key columns [64h, 64h+64) of
-        // every tile, with its own running max, row sum and O accumulator: the two halves never
-        // talk to each other until the epilogue, which merges them like two online-softmax streams.
+        // Thread = query row (TMEM lane).  Warpgroup h = warp / 4 takes the key tiles j = h, h + 2, ... whole (128 scores
+        // per thread), with its own running max, row sum, P buffer and O accumulator: two independent online-softmax
+        // streams, merged only in the epilogue.  The two warpgroups take turns on the one score buffer -- S(j+1) is issued
+        // as soon as the warpgroup of tile j holds its scores in registers -- so one of them is in its exp2 loop while the
+        // other waits, loads and takes its maxima: the MUFU unit, which two warps per scheduler saturate when they run
+        // their exp2 loops together, is busy through both.
         const int h = warp / 4;
         const int lane_row = 32 * (warp % 4) + lane;
         const int row = q0 + lane_row;
         const uint32_t lane_addr = tbase + ((uint32_t)(32 * (warp % 4)) << 16);
-        const uint32_t ocol = kColO + h * D;
-        float m_used = 0.f, l = 0.f;
+        const uint32_t ocol = kColO + h * D, pcol = kColP + 64 * h;
+        float m_used = -1e30f, l = 0.f;      // (a stream without tiles contributes nothing to the merge)
         bool ok = nkt > 0;
         if (prep.dO != nullptr && row < n) {
             // fused call: the epilogue reads this thread's 128 bytes (D = 128) of its dO row; ask L2 for
@@ -272,49 +284,48 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             const size_t doff = prep.so.at(bb, hq, row);
             if ((D / 2) * h < prep.d) asm volatile("prefetch.global.L2 [%0];" ::"l"(prep.dO + doff + (D / 2) * h));
         }
-        // The exp2 phase of a tile is MUFU-bound and the rest of a tile's work (TMEM load, max,
-        // hand-offs) is not: start the second warpgroup a few hundred cycles late, once, so that on
-        // each scheduler one warp's exp2 phase overlaps the other's remaining work.  Nothing in the
-        // loop re-synchronises the two halves.
-        if (h == 1) __nanosleep(300);
-        for (int j = 0; ok && j < nkt; ++j) {
-            const uint32_t scol = kColS + 128 * (j & 1) + 64 * h;      // this thread's 64 score columns
-            if (!mbar_wait(bars + F_S + (j & 1), (j >> 1) & 1, abortp, status, ERR_S)) { ok = false; break; }
+        for (int j = h; ok && j < nkt; j += 2) {
+            const int t = j >> 1;                                      // this stream's tile count
+            if (!mbar_wait(bars + F_S + 2 * h + (t & 1), (t >> 1) & 1, abortp, status, ERR_S)) { ok = false; break; }
             tc_fence_after();
-            const int k0 = (kt0 + j) * BN + 64 * h;
-            const bool need_mask = (k0 + 64 > n) || (causal && k0 + 63 > q0);
-            uint32_t r[2][32];
+            const int k0 = (kt0 + j) * BN;
+            const bool need_mask = (k0 + BN > n) || (causal && k0 + BN - 1 > q0);
+            uint32_t r[4][32];
 #pragma unroll
-            for (int c = 0; c < 2; ++c) tmem_ld(lane_addr + scol + 32 * c, r[c]);
+            for (int c = 0; c < 4; ++c) tmem_ld(lane_addr + kColS + 32 * c, r[c]);
             tc_wait_ld();
+            tc_fence_before();
+            mbar_arrive(bars + F_SFREE + h);      // the score columns are free: S(j+1) runs under this tile's exponentials
             if (need_mask) {
 #pragma unroll
-                for (int c = 0; c < 2; ++c)
+                for (int c = 0; c < 4; ++c)
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
                         const int col = k0 + 32 * c + i;
                         if (col >= n || (causal && col > row)) r[c][i] = 0xff800000u;   // -inf
                     }
             }
-            // max of the raw scores (scale_log2 > 0, so scaling commutes with max): 3-input max, eight
+            // max of the raw scores (scale_log2 > 0, so scaling commutes with max): 3-input max, sixteen
             // independent chains so that the dependent-issue latency does not add up
-            float mx8[8];
+            float mx16[16];
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
+            for (int q = 0; q < 16; ++q) {
                 const int c = q >> 2, i0 = 8 * (q & 3);
                 float a = fmax3(__uint_as_float(r[c][i0]), __uint_as_float(r[c][i0 + 1]), __uint_as_float(r[c][i0 + 2]));
                 a = fmax3(a, __uint_as_float(r[c][i0 + 3]), __uint_as_float(r[c][i0 + 4]));
                 a = fmax3(a, __uint_as_float(r[c][i0 + 5]), __uint_as_float(r[c][i0 + 6]));
-                mx8[q] = fmaxf(a, __uint_as_float(r[c][i0 + 7]));
+                mx16[q] = fmaxf(a, __uint_as_float(r[c][i0 + 7]));
             }
-            const float mx = fmax3(fmax3(mx8[0], mx8[1], mx8[2]), fmax3(mx8[3], mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])) * scale_log2;
-            if (j == 0) {
-                m_used = (mx == -INFINITY) ? -1e30f : mx;     // a half with no visible key yet: any finite reference
+#pragma unroll
+            for (int q = 0; q < 8; ++q) mx16[q] = fmaxf(mx16[q], mx16[q + 8]);
+            const float mx = fmax3(fmax3(mx16[0], mx16[1], mx16[2]), fmax3(mx16[3], mx16[4], mx16[5]), fmaxf(mx16[6], mx16[7])) * scale_log2;
+            if (t == 0) {
+                m_used = (mx == -INFINITY) ? -1e30f : mx;     // a stream with no visible key yet: any finite reference
             } else {
                 const bool grow = mx > m_used + kRescaleThreshold;
                 if (__any_sync(0xffffffffu, grow)) {
-                    // O_h must be stable: PV(j-1) complete (PV(j) is not issued before this thread arrives)
-                    if (!mbar_wait(bars + F_O, (j - 1) & 1, abortp, status, ERR_O)) { ok = false; break; }
+                    // O_h must be stable for a rescale: P V(j-2) has completed
+                    if (!mbar_wait(bars + F_OB + h, (t - 1) & 1, abortp, status, ERR_O)) { ok = false; break; }
                     tc_fence_after();
                     const float alpha = grow ? ex2(m_used - mx) : 1.f;
                     if (grow) m_used = mx;
@@ -330,30 +341,28 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                     }
                 }
             }
-            // P = 2^(s scale_log2 - m_used), row sum, bf16 P into TMEM over the first 32 of this half's
-            // score columns.  Arithmetic runs on fp32 pairs (f32x2) to halve the instruction count.
+            // P = 2^(s scale_log2 - m_used), row sum, bf16 P into the stream's own 64 TMEM columns.
+            // Arithmetic runs on fp32 pairs (f32x2) to halve the instruction count.
             const uint64_t sl2 = pack_f32x2(scale_log2, scale_log2);
             const uint64_t negm2 = pack_f32x2(-m_used, -m_used);
             uint64_t ls2[2] = {0ull, 0ull};
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
+            for (int c = 0; c < 4; ++c) {
                 uint32_t pk[16];
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
-                    const uint64_t t = fma_f32x2(pack_f32x2(__uint_as_float(r[c][i]), __uint_as_float(r[c][i + 1])), sl2, negm2);
+                    const uint64_t tt = fma_f32x2(pack_f32x2(__uint_as_float(r[c][i]), __uint_as_float(r[c][i + 1])), sl2, negm2);
                     float p0, p1;
-                    unpack_f32x2(t, p0, p1);
+                    unpack_f32x2(tt, p0, p1);
                     p0 = ex2(p0);
                     p1 = ex2(p1);
                     ls2[(i >> 1) & 1] = add_f32x2(ls2[(i >> 1) & 1], pack_f32x2(p0, p1));
                     pk[i / 2] = pack_bf16(p0, p1);
                 }
-                tmem_st(lane_addr + scol + 16 * c, pk);
-                if (c == 0) {       // the first 32 keys can enter the P V product while the others are exponentiated
-                    tc_wait_st();
-                    tc_fence_before();
-                    mbar_arrive(bars + F_P + 2 * (j & 1) + h);
-                }
+                // P(j) goes where P(j-2) was: P V(j-2), which gave way to S(j) in the pipe, has read it by now (the first
+                // 32 exponentials of the tile ran under the rest of that product)
+                if (c == 0 && t > 0 && !mbar_wait(bars + F_OB + h, (t - 1) & 1, abortp, status, ERR_O)) { ok = false; break; }
+                tmem_st(lane_addr + pcol + 16 * c, pk);
             }
             {
                 float s0, s1, s2, s3;
@@ -363,9 +372,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             }
             tc_wait_st();
             tc_fence_before();
-            mbar_arrive(bars + F_P2 + 2 * (j & 1) + h);
+            mbar_arrive(bars + F_P + h);
         }
-        // ---- epilogue: merge the two key halves.  Each thread publishes (m, l) of its half, then
+        // ---- epilogue: merge the two streams.  Each thread publishes (m, l) of its stream, then
         // writes D/2 output columns of its row from both accumulators.
         float2 *xch = reinterpret_cast<float2 *>(bars + F_COUNT + 2);   // [2][128] (m, l)
         float *xd = reinterpret_cast<float *>(xch + 256);               // [2][128] partial rowsum(dO o O)
@@ -395,6 +404,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             const float l_all = l * a_me + other.y * a_ot;
             const float inv = 1.f / l_all;
             const float w0 = (h == 0 ? a_me : a_ot) * inv, w1 = (h == 0 ? a_ot : a_me) * inv;   // weights of O_0, O_1
+            const bool has1 = nkt > 1;      // (one key tile: the second stream's accumulator was never written)
             // O leaves as bf16 through shared memory (the Q tile is no longer read) and a TMA store: a
             // thread owns a row, so direct stores would be 16 bytes at a 2D-byte stride, one 128-byte line
             // per lane and instruction.  Rows past n are clipped by the tensor map.
@@ -402,13 +412,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             for (int c = 0; c < D / 2; c += 32) {
                 uint32_t o0[32], o1[32];
                 tmem_ld(lane_addr + kColO + (D / 2) * h + c, o0);
-                tmem_ld(lane_addr + kColO + D + (D / 2) * h + c, o1);
+                if (has1) tmem_ld(lane_addr + kColO + D + (D / 2) * h + c, o1);
                 tc_wait_ld();
 #pragma unroll
                 for (int i = 0; i < 32; i += 8) {
                     float v[8];
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) v[u] = __uint_as_float(o0[i + u]) * w0 + __uint_as_float(o1[i + u]) * w1;
+                    for (int u = 0; u < 8; ++u) v[u] = __uint_as_float(o0[i + u]) * w0 + (has1 ? __uint_as_float(o1[i + u]) * w1 : 0.f);
                     if (want_d) {
                         const uint4 g = dov[(c + i) / 8];
                         const uint32_t gw[4] = {g.x, g.y, g.z, g.w};
