@@ -3,7 +3,7 @@ roofline entries of bench.py rest on, one block per captured launch; with --reco
 measured DRAM traffic of a kernel into profiles/traffic.json, the record bench.py scales by tokens for
 `roofline.traffic` (so that the bench line never carries a number typed in by hand).
 
-    python -m paper_2609_33916_b200.profile_summary gpurun_out/prof_bwd.ncu-rep \\
+    python -m paper_2609_33916_b200.profile_summary prof_bwd.ncu-rep \\
         --record bwd_kv --case "B1 H8 n8192 d128 non-causal, TMA bulk reduce" --tokens 65536 --d 128 --dq-mode 2
 
 No GPU is needed to read a report.  Nothing here is on the product path.
