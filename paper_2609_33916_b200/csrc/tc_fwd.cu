@@ -297,13 +297,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             tc_fence_before();
             mbar_arrive(bars + F_SFREE + h);      // the score columns are free: S(j+1) runs under this tile's exponentials
             if (need_mask) {
+                // columns of this tile the row may see: keys below n and, causal, not past the row itself
+                const int lim = min(n, causal ? row + 1 : n) - k0;
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const int col = k0 + 32 * c + i;
-                        if (col >= n || (causal && col > row)) r[c][i] = 0xff800000u;   // -inf
-                    }
+                    for (int i = 0; i < 32; ++i)
+                        if (32 * c + i >= lim) r[c][i] = 0xff800000u;   // -inf
             }
             // max of the raw scores (scale_log2 > 0, so scaling commutes with max): 3-input max, sixteen
             // independent chains so that the dependent-issue latency does not add up
