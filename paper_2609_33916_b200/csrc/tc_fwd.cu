@@ -118,13 +118,46 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     const int kt0 = split * sp.tiles_per_split;                       // first key tile of this CTA
     const int nkt_want = causal ? min(qt + 1, nkt_all) : min(sp.tiles_per_split, nkt_all - kt0);
 
-    if (tid == 0) {
-        for (int b = 0; b < F_COUNT; ++b)
-            mbar_init(bars + b, ((b >= F_P && b < F_P + 2) || (b >= F_SFREE && b < F_SFREE + 2)) ? 128u : ((b == F_X || b == F_E) ? 256u : 1u));
-        *abortp = (smem_u32(sm) & 1023u) ? 1u : 0u;
-        if (*abortp && status) atomicCAS(status, 0u, 0x108u);
+    // The two producer threads initialise the barriers of their own loads and send the job's first loads off at once:
+    // Q, the first two K chunks and the first two V tiles are on their way while the rest of the set-up (the other
+    // barriers, the TMEM allocation, the CTA-wide barrier) still runs, instead of starting behind it.
+    const bool aligned = (smem_u32(sm) & 1023u) == 0;      // (swizzled tiles need the 1024-byte alignment)
+    const int early_k = aligned ? min(nkt_want * KC, 2) : 0, early_v = aligned ? min(nkt_want, 2) : 0;
+    if (warp == 8 && lane == 0) {
+        mbar_init(bars + F_Q, 1u);
+        mbar_init(bars + F_KFULL, 1u);
+        mbar_init(bars + F_KFULL + 1, 1u);
         fence_mbar_init();
-        prefetch_tensormap(&mapQ); prefetch_tensormap(&mapK); prefetch_tensormap(&mapV); prefetch_tensormap(&mapO);
+        if (early_k > 0) {
+            mbar_arrive_expect_tx(bars + F_Q, KC * kTileBytes);
+            for (int b = 0; b < KC * kBoxes; ++b) tma_load_4d(sQ + b * kBoxBytes, &mapQ, bars + F_Q, 64 * b, q0, hq, bb);
+            for (int g = 0; g < early_k; ++g) {       // chunk g: columns [D c, D c + D) of key tile j, g = j KC + c
+                const int j = g / KC, c = g % KC;
+                mbar_arrive_expect_tx(bars + F_KFULL + g, kTileBytes);
+                for (int b = 0; b < kBoxes; ++b)
+                    tma_load_4d(sK + g * kTileBytes + b * kBoxBytes, &mapK, bars + F_KFULL + g, D * c + 64 * b, (kt0 + j) * BN, hk, bb);
+            }
+        }
+    }
+    if (warp == 11 && lane == 0) {
+        mbar_init(bars + F_VFULL, 1u);
+        mbar_init(bars + F_VFULL + 1, 1u);
+        fence_mbar_init();
+        for (int j = 0; j < early_v; ++j) {
+            mbar_arrive_expect_tx(bars + F_VFULL + j, kTileBytes);
+            for (int b = 0; b < kBoxes; ++b)
+                tma_load_4d(sV + j * kTileBytes + b * kBoxBytes, &mapV, bars + F_VFULL + j, D * pass + 64 * b, (kt0 + j) * BN, hk, bb);
+        }
+    }
+    if (tid == 0) {
+        for (int b = 0; b < F_COUNT; ++b) {
+            if (b == F_Q || b == F_KFULL || b == F_KFULL + 1 || b == F_VFULL || b == F_VFULL + 1) continue;   // (the producers' own)
+            mbar_init(bars + b, ((b >= F_P && b < F_P + 2) || (b >= F_SFREE && b < F_SFREE + 2)) ? 128u : ((b == F_X || b == F_E) ? 256u : 1u));
+        }
+        *abortp = aligned ? 0u : 1u;
+        if (!aligned && status) atomicCAS(status, 0u, 0x108u);
+        fence_mbar_init();
+        prefetch_tensormap(&mapO);
     }
     if (warp == 9) { tmem_alloc(tmem_base_p, kTmemCols); tmem_relinquish(); }
     tc_fence_before();
@@ -141,11 +174,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
       asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
       if (warp == 8) {
         // ------------------------------------------------------------------ TMA producer
-        int nk = 0;             // K chunks requested so far (slot = count & 1)
-        if (lane == 0 && nkt > 0) {
-            mbar_arrive_expect_tx(bars + F_Q, KC * kTileBytes);
-            for (int b = 0; b < KC * kBoxes; ++b) tma_load_4d(sQ + b * kBoxBytes, &mapQ, bars + F_Q, 64 * b, q0, hq, bb);
-        }
+        int nk = early_k;       // K chunks requested so far (slot = count & 1): Q and the first two went out before the set-up
         // chunk g of the K stream: 128 columns [D c, D c + D) of key tile j, g = j KC + c, ring slot g & 1
         auto load_k = [&](int g) {
             const int s = g & 1, j = g / KC, c = g % KC;
@@ -158,16 +187,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             // Fused forward+backward (KC = 1): this CTA's 128 rows of the fp32 dQ accumulator ([B*H, n, D]) are
             // cleared here, by the producer warp while its first loads are in flight (the next slot
             // frees two tiles from now), so that the step needs no separate clearing pass.
-            // The first two K/V tiles are requested first: they have no slot to wait for.
-            for (int j = 0; j < min(nkt, 2); ++j)
-                if (lane == 0) load_k(j);
             const int rows = min(BM, n - q0);
             float4 *dst = reinterpret_cast<float4 *>(zero_acc + ((size_t)bh * n + q0) * D);
             for (int i = lane; i < rows * (D / 4); i += 32) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         bool live = true;
-        for (int j = (zero_acc != nullptr ? min(nkt, 2) : 0); live && j < nkt; ++j) {
-            for (int c = 0; c < KC; ++c) {
+        for (int j = early_k / KC; live && j < nkt; ++j) {
+            for (int c = (j == early_k / KC ? early_k % KC : 0); c < KC; ++c) {
                 const int g = j * KC + c;
                 if (g >= 2 && !mbar_wait(bars + F_KEMPTY + (g & 1), ((g >> 1) - 1) & 1, abortp, status, ERR_K)) { live = false; break; }
                 if (lane == 0) load_k(g);
@@ -184,8 +210,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         // ------------------------------------------------------------------ TMA producer of the V stream
         // (a thread of its own: the V ring follows the P V products, the K ring the score products, and neither waits
         // for the other's slots)
-        int nv = 0;
-        for (int j = 0; j < nkt; ++j) {
+        int nv = early_v;       // (the first two tiles went out before the set-up)
+        for (int j = early_v; j < nkt; ++j) {
             if (j >= 2 && !mbar_wait(bars + F_VEMPTY + (j & 1), ((j >> 1) - 1) & 1, abortp, status, ERR_V)) break;
             if (lane == 0) {
                 const int s = j & 1;
