@@ -80,9 +80,9 @@ typedef enum { MOA_BF16 = 0, MOA_F32 = 1 } moa_dtype;
  * paper's GK/GV atomic sites and their removal, transposed here onto dQ because
  * the backward kernel is parallel over key tiles). */
 typedef enum {
-    MOA_DQ_AUTO = 0,          /* library's choice: BULK_REDUCE for bf16 d > 64, else RED       */
+    MOA_DQ_AUTO = 0,          /* library's choice: BULK_REDUCE for bf16 d <= 128, else RED     */
     MOA_DQ_RED = 1,           /* fp32 red.global.add into a [B,H,n,d] fp32 accumulator        */
-    MOA_DQ_BULK_REDUCE = 2,   /* shared-memory tile + cp.reduce.async.bulk add.f32 (bf16 d > 64) */
+    MOA_DQ_BULK_REDUCE = 2,   /* shared-memory tile + cp.reduce.async.bulk add.f32 (bf16 d <= 128) */
     MOA_DQ_SEPARATE_PASS = 3  /* no atomics: a second, query-parallel kernel recomputes dS     */
 } moa_dq_mode;
 

@@ -139,9 +139,9 @@ moa_status check_desc(const moa_attn_desc *d)
     if (d->path == MOA_PATH_TC && d->dtype != MOA_BF16) return MOA_ERR_UNSUPPORTED;
     // the materialising comparison variant runs on the tensor-core path only
     if (d->materialize && !(d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->scale > 0.f)) return MOA_ERR_UNSUPPORTED;
-    // the bulk-reduce strategy exists in the 128-column tensor-core backward only
+    // the bulk-reduce strategy exists in the 64- and 128-column tensor-core backward only
     if (d->dq_mode == MOA_DQ_BULK_REDUCE &&
-        !(d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && kernel_d(d->d) == 128 && d->scale > 0.f))
+        !(d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && kernel_d(d->d) <= 128 && d->scale > 0.f))
         return MOA_ERR_UNSUPPORTED;
     if (d->path == MOA_PATH_TC && !(d->scale > 0.f)) return MOA_ERR_UNSUPPORTED;   // non-positive scale: SIMT path only
     if (d->layout != MOA_LAYOUT_BHND && d->layout != MOA_LAYOUT_BNHD && d->layout != MOA_LAYOUT_STRIDED) return MOA_ERR_INVALID_ARG;
@@ -166,13 +166,13 @@ moa_status check_desc(const moa_attn_desc *d)
     return MOA_OK;
 }
 
-// AUTO: the TMA bulk add-reduce where it exists (tensor-core path, 128-column kernel: measured
-// slightly ahead of plain reds at every size), plain reds otherwise.
+// AUTO: the TMA bulk add-reduce where it exists (tensor-core path, 64- and 128-column kernels: measured slightly ahead of
+// plain reds at every size at 128 columns, 15-25 % ahead at 64, where the reds fill half a sector each), plain reds otherwise.
 int resolved_dq_mode(const moa_attn_desc *d)
 {
     if (d->dq_mode != MOA_DQ_AUTO) return d->dq_mode;
     const bool tc = d->dtype == MOA_BF16 && d->path != MOA_PATH_SIMT && d->scale > 0.f;
-    return (tc && kernel_d(d->d) == 128) ? MOA_DQ_BULK_REDUCE : MOA_DQ_RED;
+    return (tc && kernel_d(d->d) <= 128) ? MOA_DQ_BULK_REDUCE : MOA_DQ_RED;
 }
 
 // the tensor-core kernels take the row max before scaling, which needs scale > 0

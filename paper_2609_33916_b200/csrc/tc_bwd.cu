@@ -16,8 +16,9 @@
 // dQ_i is one key tile's contribution; it is added into an fp32 [B,H,n,d] accumulator (the contended step the
 // dq_mode knob is about): for D = 128 the tile is produced transposed (dQ_i^T = K^T dS^T, lanes = d) and leaves
 // either as warp-wide red.global.add.f32 (one full 128-byte line per instruction) or, by default, staged 32 rows
-// at a time in shared memory and handed to the TMA engine as cp.reduce.async.bulk.tensor add.f32; D = 64 uses
-// red.global.add.v4.f32 on the untransposed tile.
+// at a time in shared memory and handed to the TMA engine as cp.reduce.async.bulk.tensor add.f32; D = 64 keeps the
+// untransposed tile (UMMA needs M = 128, so lanes stay queries): each reduce warp stages its own 32 rows as two swizzled boxes
+// and sends them by the same instruction (default), or the rows leave as red.global.add.v4.f32 (half a sector per lane).
 //
 // Roles (512 threads; registers are re-split per warpgroup with setmaxnreg: 144 / 144 / 144 / 80): warps 0-7
 // elementwise work (thread = TMEM lane = key, the two warpgroups split the query columns), warps 8-11 read each
@@ -129,7 +130,7 @@ bwd_preprocess_kernel(const __nv_bfloat16 *__restrict__ dO, const __nv_bfloat16 
     }
 }
 
-// kBulk: the dQ tile goes out through the TMA add-reduce; that needs 32 KB of staging, which is
+// kBulk: the dQ tile goes out through the TMA add-reduce; at D = 128 that needs 32 KB of staging, which is
 // taken from the second dO slot (dO_i is only read early in tile i, by dP and dV, so one slot
 // works, at the price of a later refill).  Without it dO has two slots like Q.
 template <int D, bool kBulk>
@@ -139,11 +140,12 @@ struct BwdSmem {
     static constexpr int offK = 0;
     static constexpr int offV = offK + kTile;
     static constexpr int offQ = offV + kTile;        // 2 slots
-    static constexpr int kDoSlots = kBulk ? 1 : 2;
+    static constexpr int kDoSlots = (kBulk && D == 128) ? 1 : 2;      // (D = 64 has the room for both)
     static constexpr int offdO = offQ + 2 * kTile;
     static constexpr int offStage = offdO + kDoSlots * kTile;   // 2 x [32 rows][D] fp32 staging (kBulk only)
     static constexpr int kStage = kBulk ? 32 * D * 4 : 0;
-    static constexpr int offdS = offStage + 2 * kStage;
+    // D = 128: two stages of 32 rows, filled by all four reduce warps in turn; D = 64: a stage per reduce warp (its own 32 rows)
+    static constexpr int offdS = offStage + (D == 128 ? 2 : 4) * kStage;
     static constexpr int offL = offdS + kdS;         // 2 x 128 floats, travels with the Q slot
     static constexpr int offD = offL + 2 * 512;      // 2 x 128 floats, travels with the Q slot
     static constexpr int offBar = offD + 2 * 512;    // mbarriers + tmem base + abort flag
@@ -481,7 +483,33 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 tc_wait_ld();
                 tc_fence_before();
                 mbar_arrive(bars + B_DQR);
-                if (qrow < n) {
+                if (dq_bulk) {
+                    // D = 64, bulk reduce: a thread holds the 64 floats of its query row, a warp 32 consecutive rows -- one
+                    // box pair of the accumulator's tensor map (32 rows x 32 floats each, 128-byte swizzle), staged and sent
+                    // by the warp alone: no hand-off between the warps.  `red.global.add.v4` from here fills half a sector
+                    // per lane and instruction; the staged rows leave as whole lines.
+                    uint8_t *wstage = sm + SM::offStage + (warp % 4) * SM::kStage;
+                    if (it > 0) {       // the reduces of the tile before have read the boxes
+                        if (lane == 0) bulk_wait_read<0>();
+                        __syncwarp();
+                    }
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c)
+#pragma unroll
+                        for (int jj = 0; jj < 8; ++jj) {
+                            const int chunk = jj ^ (lane & 7);
+                            *reinterpret_cast<uint4 *>(wstage + c * 4096 + lane * 128 + chunk * 16) =
+                                make_uint4(r[c][4 * jj], r[c][4 * jj + 1], r[c][4 * jj + 2], r[c][4 * jj + 3]);
+                        }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    const int row0 = qtile * 128 + 32 * (warp % 4);
+                    if (lane == 0 && row0 < n) {        // (rows past n inside the box are clipped by the map)
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) tma_reduce_add_3d(&mapdQ, wstage + c * 4096, 32 * c, row0, qh);
+                        bulk_commit();
+                    }
+                } else if (qrow < n) {
 #pragma unroll
                     for (int c = 0; c < D / 32; ++c)
 #pragma unroll
@@ -492,6 +520,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             }
         }
         if (kTransposeDQ && dq_bulk && tid == kReduceWarp0 * 32) bulk_wait<0>();   // all reduces done before exit
+        if (!kTransposeDQ && dq_bulk && lane == 0) bulk_wait<0>();                 // (D = 64: every reduce warp sent its own)
     } else {
         // ----------------------------------------------------------- elementwise warps 0-7
         asm volatile("setmaxnreg.inc.sync.aligned.u32 144;");
@@ -665,7 +694,8 @@ cudaError_t launch_bwd_g(const Problem &p, const void *Q, const void *K, const v
         !make_tensor_map_4d_strided(&mdv, dV, bf, 2, p.B, p.kv_heads(), p.n, p.d, p.skv.row, p.skv.head, p.skv.batch, 128, 64))
         return cudaErrorInvalidValue;
     // fp32 accumulator as [heads, n, D] with boxes of 32 rows x D floats (no swizzle); also encoded when unused
-    if (!make_tensor_map_3d(&mdq, dQacc ? (const void *)dQacc : Q, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, heads, p.n, D, 32, D))
+    // (D = 64: boxes of 32 rows x 32 floats with the 128-byte swizzle, two per warp and tile)
+    if (!make_tensor_map_3d(&mdq, dQacc ? (const void *)dQacc : Q, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, heads, p.n, D, 32, D == 64 ? 32 : D))
         return cudaErrorInvalidValue;
     constexpr int kSmem = BwdSmem<D, kBulk>::kTotal;
     cudaError_t e = cudaFuncSetAttribute(tc_bwd_kernel<D, kBulk, kGrouped>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
@@ -721,6 +751,7 @@ cudaError_t tc_bwd_kv(const Problem &p, const void *Q, const void *K, const void
     if (D == 256) return dq_bulk ? cudaErrorInvalidValue : tc_bwd_kv_wide(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
     if (D == 128 && bwd_pair_enabled()) return tc_bwd_kv_pair(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, dq_bulk, st);
     if (D == 64 && !dq_bulk) return launch_bwd<64, false>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
+    if (D == 64 && dq_bulk) return launch_bwd<64, true>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
     if (D == 128 && !dq_bulk) return launch_bwd<128, false>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
     if (D == 128 && dq_bulk) return launch_bwd<128, true>(p, Q, K, V, dO, Lp, Dp, dK, dV, dQacc, st);
     return cudaErrorInvalidValue;

@@ -112,7 +112,8 @@ def test_other_head_dimensions_argument_checks(lib):
     assert fwd(96, dtype=mb.MOA_F32) == mb.MOA_ERR_UNSUPPORTED
     assert fwd(96, path=mb.MOA_PATH_SIMT) == mb.MOA_ERR_UNSUPPORTED
     assert fwd(96, materialize=1) == mb.MOA_ERR_UNSUPPORTED
-    assert fwd(32, dq_mode=mb.MOA_DQ_BULK_REDUCE) == mb.MOA_ERR_UNSUPPORTED      # 64-column kernel: no bulk reduce
+    assert fwd(32, dq_mode=mb.MOA_DQ_BULK_REDUCE) != mb.MOA_ERR_UNSUPPORTED      # the 64-column kernel has the bulk reduce too
+    assert fwd(32, dq_mode=mb.MOA_DQ_BULK_REDUCE, path=mb.MOA_PATH_SIMT) == mb.MOA_ERR_UNSUPPORTED
     # the accumulator rows are as wide as the kernel's head dimension
     assert ws(96) == ws(128) and ws(40) == ws(64) and ws(72) == ws(128)
     assert ws(96, dq_mode=mb.MOA_DQ_SEPARATE_PASS) == ws(128, dq_mode=mb.MOA_DQ_SEPARATE_PASS) < ws(96)

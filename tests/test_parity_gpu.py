@@ -72,8 +72,8 @@ BF16_CASES = [
 @pytest.mark.parametrize("B,Hh,n,d,causal", BF16_CASES)
 @pytest.mark.parametrize("path,dq_mode", [(1, 1), (1, 3), (2, 1), (2, 3), (2, 2)])
 def test_bf16_shapes(H, B, Hh, n, d, causal, dq_mode, path):
-    if dq_mode == 2 and d != 128:
-        pytest.skip("TMA bulk-reduce dQ exists for d = 128 only")
+    if dq_mode == 2 and d not in (64, 128):
+        pytest.skip("TMA bulk-reduce dQ exists in the 64- and 128-column kernels")
     inp = mi.make_inputs(B, Hh, n, d, seed=200 + n, dtype="bf16")
     scale = 1.0 / math.sqrt(d)
     ref = _oracle(inp, "bf16", causal, scale)
@@ -308,8 +308,6 @@ def test_other_head_dimensions_match_oracle(H, d, causal, dq_mode):
     fill the missing columns with zeros (which changes no result) and the stores drop them; the
     direct-addressed passes (preprocess, dQ conversion, the separate dQ pass) use the true row
     length.  Every element against the fp64 oracle, ragged n, fused and separate calls."""
-    if dq_mode == 2 and d <= 64:
-        pytest.skip("TMA bulk-reduce dQ exists in the 128-column kernel only")
     n = 300 if d % 16 else 129
     inp = mi.make_inputs(2, 3, n, d, seed=600 + d, dtype="bf16")
     scale = 1.0 / math.sqrt(d)

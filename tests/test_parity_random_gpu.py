@@ -24,7 +24,7 @@ def _cases(count, seed):
         kind = rng.integers(0, 10)
         if kind < 6:        # tensor-core path, one of the dQ strategies
             path, mat = 2, 0
-            dq = int(rng.choice([1, 3] if d == 64 else [1, 2, 3]))
+            dq = int(rng.choice([1, 2, 3]))
         elif kind < 8:      # SIMT path
             path, mat, dq = 1, 0, int(rng.choice([1, 3]))
         else:               # materialising variant
@@ -60,7 +60,7 @@ def _gqa_cases(count, seed):
         Hkv = int(rng.integers(1, 4))
         G = int(rng.choice([1, 2, 3, 5]))
         B = int(rng.integers(1, 3))
-        dq = int(rng.choice([0, 1, 3] if d <= 64 else [0, 1, 2, 3]))
+        dq = int(rng.choice([0, 1, 2, 3]))
         layout = int(rng.integers(0, 2))
         op = "split" if rng.random() < 0.3 else "fused"
         out.append((i, B, Hkv * G, Hkv, n, d, causal, dq, layout, op))
