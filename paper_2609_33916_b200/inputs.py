@@ -54,6 +54,7 @@ CONFIGS = {
 CONFIGS["paper_b2_n2048_d64"] = Workload("paper_b2_n2048_d64", 2, 1, 2048, 64, False, "bf16", 6)
 CONFIGS["paper_b2_n8192_d64"] = Workload("paper_b2_n8192_d64", 2, 1, 8192, 64, False, "bf16", 7)
 CONFIGS["prof_h8_n8192"] = Workload("prof_h8_n8192", 1, 8, 8192, 128, False, "bf16", 5)
+CONFIGS["prof_d64_h32_n8192"] = Workload("prof_d64_h32_n8192", 1, 32, 8192, 64, False, "bf16", 11)     # the same at 64 columns
 # head dimensions above 128 (the two-pass kernels): the profiler case's shape at d = 256 and 192, and a causal one
 CONFIGS["d256_h8_n8192"] = Workload("d256_h8_n8192", 1, 8, 8192, 256, False, "bf16", 8)
 CONFIGS["d192_h8_n8192"] = Workload("d192_h8_n8192", 1, 8, 8192, 192, False, "bf16", 9)
